@@ -1,0 +1,327 @@
+"""CPU oracle for attention over a page-aligned, position-free chunk KV cache.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain, fp64 statement of
+what the MEPIC hot path computes.  The CUDA library never imports, links or
+calls it, and it never imports the library; only the tests, the smoke check
+and the CPU-baseline leg of the benchmark may use it.
+
+What it states, and where the paper fixes it:
+
+* Scheduling path (Section 3.2, Algorithm 1): chunk segments are padded at the
+  front and prompt segments at the back so that every chunk starts on a KV
+  block boundary; the last prompt segment is left unpadded (Section 3.2.1).
+  A chunk's identity is its padded token sequence (Section 3.2.3, "KV Block
+  Allocation"); its first KV block is private to each request and the
+  remaining blocks are shared by every request that uses the chunk
+  (Section 3.2.3, Section 3.3.1).  A request is rejected when the pool cannot
+  supply its blocks (Algorithm 1, admission check).
+* Computation path (Section 3.3): recomputed K/V rows are written straight
+  into their assigned pages (Section 3.3.2); pages hold keys WITHOUT rotary
+  position embedding, and the rotation is applied to K when the attention
+  operator reads it (Section 3.3.3).  The result is therefore ordinary softmax
+  attention with RoPE applied at each token's assigned position: that
+  definition is what `decode_attention` and `prefill_attention` write out.
+
+Readings taken where the paper is silent (each also listed in the design
+notes): split-half ("rotate_half") RoPE pairing with inverse frequencies
+theta**(-2i/D) and no frequency scaling; V is never rotated; a token's
+position is its index in the padded logical sequence, i.e. block-table entry
+e starts at position e*P; pad slots are ordinary attended tokens; causality
+is by logical slot while rotation is by position; free pages are handed out
+first-in-first-out starting from 0..num_pages-1, and released pages rejoin the
+queue in ascending order.
+
+Parity unpinned by the paper: the RoPE pairing convention and the physical
+page-id assignment order (the paper gives neither); they are pinned only by
+the specification above, which the oracle and the library implement
+independently.
+"""
+from __future__ import annotations
+
+from collections import deque
+from dataclasses import dataclass
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+KIND_CHUNK = 0
+KIND_PROMPT = 1
+
+
+class Reject(Exception):
+    """Algorithm 1's Reject: the pool cannot supply the blocks a call needs."""
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    b = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (b.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+
+
+# ----------------------------------------------------------------------------
+# Scheduling path (Section 3.2, Algorithm 1): integer work, exact.
+# ----------------------------------------------------------------------------
+
+@dataclass
+class OracleTable:
+    page_ids: List[int]
+    pos_base: List[int]
+    kv_len: int
+    recompute_slots: List[int]
+
+
+class OracleStore:
+    """Page pool + chunk index, keyed by chunk CONTENT (no hash function)."""
+
+    def __init__(self, page_size: int, num_pages: int, pad_token_id: int = 0):
+        self.P = int(page_size)
+        self.num_pages = int(num_pages)
+        self.pad = int(pad_token_id)
+        self.free = deque(range(self.num_pages))
+        self.chunks: Dict[Tuple[int, ...], dict] = {}
+        self.requests: Dict[int, dict] = {}
+        self.dedup_hits = 0
+
+    # Section 3.2.1: leading pad so that the chunk fills whole blocks.
+    def canonical_chunk(self, tokens: Sequence[int]) -> Tuple[int, ...]:
+        n = len(tokens)
+        lead = (-n) % self.P
+        return tuple([self.pad] * lead + [int(t) for t in tokens])
+
+    # Section 3.2.2 / 3.2.3: residency lookup, then allocation of the shareable blocks.
+    def register_chunk(self, tokens: Sequence[int]):
+        if len(tokens) == 0:
+            raise ValueError("empty chunk")
+        key = self.canonical_chunk(tokens)
+        if key in self.chunks:
+            self.dedup_hits += 1
+            return key, True, list(self.chunks[key]["shared"])
+        n_pages = len(key) // self.P
+        n_shared = n_pages - 1          # first block is private per request
+        if n_shared > len(self.free):
+            raise Reject("no space for shared pages")
+        shared = [self.free.popleft() for _ in range(n_shared)]
+        self.chunks[key] = {"shared": shared, "refs": 0, "n_pages": n_pages}
+        return key, False, list(shared)
+
+    # Algorithm 1, last stage: walk the segments in order and assign blocks.
+    def build_block_table(self, request_id: int, segments: Sequence[Tuple[int, object]]) -> OracleTable:
+        if request_id in self.requests:
+            raise ValueError("request already has a table")
+        segs = [(k, v) for (k, v) in segments if not (k == KIND_PROMPT and int(v) == 0)]
+        if not segs:
+            raise ValueError("no tokens")
+        need = 0
+        for i, (kind, val) in enumerate(segs):
+            if kind == KIND_CHUNK:
+                if val not in self.chunks:
+                    raise KeyError("chunk not registered")
+                need += 1
+            else:
+                need += -(-int(val) // self.P)
+        if need > len(self.free):
+            raise Reject("no space for private pages")     # nothing was allocated yet
+        pages: List[int] = []
+        private: List[int] = []
+        recompute: List[int] = []
+        used: List[Tuple[int, ...]] = []
+        kv_len = 0
+        for i, (kind, val) in enumerate(segs):
+            start = len(pages) * self.P
+            if kind == KIND_CHUNK:
+                c = self.chunks[val]
+                first = self.free.popleft()
+                private.append(first)
+                pages.append(first)
+                pages.extend(c["shared"])
+                recompute.extend(range(start, start + self.P))
+                c["refs"] += 1
+                used.append(val)
+                kv_len = len(pages) * self.P
+            else:
+                n = int(val)
+                n_pages = -(-n // self.P)
+                for _ in range(n_pages):
+                    pg = self.free.popleft()
+                    private.append(pg)
+                    pages.append(pg)
+                last = (i == len(segs) - 1)
+                seg_len = n if last else n_pages * self.P      # trailing pad unless final
+                recompute.extend(range(start, start + seg_len))
+                kv_len = start + seg_len
+        pos_base = [e * self.P for e in range(len(pages))]
+        self.requests[request_id] = {"private": private, "chunks": used, "entries": len(pages)}
+        return OracleTable(pages, pos_base, kv_len, recompute)
+
+    def release(self, request_id: int) -> None:
+        r = self.requests.pop(request_id)
+        for key in r["chunks"]:
+            self.chunks[key]["refs"] -= 1
+        for pg in sorted(r["private"]):
+            self.free.append(pg)
+
+    def stats(self) -> dict:
+        shared = sum(len(c["shared"]) for c in self.chunks.values())
+        private = sum(len(r["private"]) for r in self.requests.values())
+        return {
+            "pages_total": self.num_pages,
+            "pages_free": len(self.free),
+            "pages_shared_held": shared,
+            "pages_private_held": private,
+            "chunks_resident": len(self.chunks),
+            "chunk_refs": sum(c["refs"] for c in self.chunks.values()),
+            "dedup_hits": self.dedup_hits,
+            "unshared_equivalent_pages": sum(r["entries"] for r in self.requests.values()),
+            "live_requests": len(self.requests),
+        }
+
+
+# ----------------------------------------------------------------------------
+# Computation path (Section 3.3): fp64.
+# ----------------------------------------------------------------------------
+
+def rope_angles(pos: np.ndarray, head_dim: int, theta: float) -> np.ndarray:
+    """phi[..., i] = pos * theta**(-2 i / D), i < D/2."""
+    half = head_dim // 2
+    inv_freq = np.float64(theta) ** (-2.0 * np.arange(half, dtype=np.float64) / head_dim)
+    return np.asarray(pos, dtype=np.float64)[..., None] * inv_freq
+
+
+def rope_rotate(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
+    """Rotary embedding, split-half pairing (i, i + D/2), on the last axis.
+
+    ``pos`` broadcasts against ``x.shape[:-1]``.
+    """
+    x = np.asarray(x, dtype=np.float64)
+    d = x.shape[-1]
+    half = d // 2
+    phi = rope_angles(np.broadcast_to(np.asarray(pos), x.shape[:-1]), d, theta)
+    c, s = np.cos(phi), np.sin(phi)
+    lo, hi = x[..., :half], x[..., half:]
+    return np.concatenate([lo * c - hi * s, lo * s + hi * c], axis=-1)
+
+
+def gather_pages(pool: np.ndarray, page_ids: Sequence[int], kv_len: int) -> np.ndarray:
+    """pool ``[num_pages, Hkv, P, D]`` -> logical ``[kv_len, Hkv, D]`` (same dtype)."""
+    P = pool.shape[2]
+    n_entries = -(-kv_len // P)
+    g = pool[np.asarray(page_ids[:n_entries], dtype=np.int64)]        # [E, Hkv, P, D]
+    g = np.transpose(g, (0, 2, 1, 3)).reshape(n_entries * P, pool.shape[1], pool.shape[3])
+    return g[:kv_len]
+
+
+def slot_positions(pos_base: Sequence[int], kv_len: int, P: int) -> np.ndarray:
+    t = np.arange(kv_len, dtype=np.int64)
+    return np.asarray(pos_base, dtype=np.int64)[t // P] + t % P
+
+
+def _softmax_rows(s: np.ndarray) -> np.ndarray:
+    m = s.max(axis=-1, keepdims=True)
+    e = np.exp(s - m)
+    return e / e.sum(axis=-1, keepdims=True)
+
+
+def decode_attention_one(q_bits: np.ndarray, k_pool: np.ndarray, v_pool: np.ndarray,
+                         page_ids: Sequence[int], pos_base: Sequence[int], kv_len: int,
+                         q_pos: int, sm_scale: float, theta: float,
+                         rotate: bool = True) -> np.ndarray:
+    """One request, one query token: ``q_bits`` uint16 ``[Hq, D]`` -> fp64 ``[Hq, D]``.
+
+    Section 3.3.3 as a definition: gather the request's pages, rotate every K
+    row at its assigned position and q at ``q_pos``, then dense softmax
+    attention; q head h reads KV head h // (Hq / Hkv).
+    """
+    P = k_pool.shape[2]
+    K = bf16_bits_to_f64(gather_pages(k_pool, page_ids, kv_len))        # [L, Hkv, D]
+    V = bf16_bits_to_f64(gather_pages(v_pool, page_ids, kv_len))
+    q = bf16_bits_to_f64(q_bits)                                        # [Hq, D]
+    if rotate:
+        pos = slot_positions(pos_base, kv_len, P)
+        K = rope_rotate(K, pos[:, None], theta)
+        q = rope_rotate(q, np.int64(q_pos), theta)
+    Hq, Hkv = q.shape[0], K.shape[1]
+    G = Hq // Hkv
+    out = np.empty_like(q)
+    for h in range(Hq):
+        kh = h // G
+        s = sm_scale * (K[:, kh, :] @ q[h])                             # [L]
+        p = _softmax_rows(s[None, :])[0]
+        out[h] = p @ V[:, kh, :]
+    return out
+
+
+def decode_attention(q_bits: np.ndarray, k_pool: np.ndarray, v_pool: np.ndarray,
+                     tables: Sequence[OracleTable], q_pos: Sequence[int],
+                     sm_scale: float, theta: float) -> np.ndarray:
+    """Batch of decode requests: ``q_bits`` uint16 ``[B, Hq, D]`` -> fp64 ``[B, Hq, D]``."""
+    return np.stack([
+        decode_attention_one(q_bits[b], k_pool, v_pool, t.page_ids, t.pos_base, t.kv_len,
+                             q_pos[b], sm_scale, theta)
+        for b, t in enumerate(tables)])
+
+
+def commit_rows(k_pool: np.ndarray, v_pool: np.ndarray, page_ids: Sequence[int],
+                q_slot: Sequence[int], k_new: np.ndarray, v_new: np.ndarray) -> None:
+    """Section 3.3.2: write the new rows' bits, un-rotated, at (page, slot). In place."""
+    P = k_pool.shape[2]
+    for i, slot in enumerate(q_slot):
+        pg = page_ids[slot // P]
+        k_pool[pg, :, slot % P, :] = k_new[i]
+        v_pool[pg, :, slot % P, :] = v_new[i]
+
+
+def prefill_attention_one(q_new: np.ndarray, k_new: np.ndarray, v_new: np.ndarray,
+                          q_slot: Sequence[int], k_pool: np.ndarray, v_pool: np.ndarray,
+                          page_ids: Sequence[int], pos_base: Sequence[int], kv_len: int,
+                          sm_scale: float, theta: float,
+                          rows: Optional[Sequence[int]] = None) -> np.ndarray:
+    """Selective-recompute prefill for one request (Sections 3.3.1-3.3.3).
+
+    Commits ``k_new/v_new`` (uint16 ``[R, Hkv, D]``) into the pools IN PLACE,
+    then lets every new row i attend, causally by logical slot, over slots
+    ``0..q_slot[i]`` of the paged context with K rotated at its position and
+    the row's q rotated at the position of its own slot.  Returns fp64
+    ``[R, Hq, D]`` (or only the listed ``rows``).
+    """
+    P = k_pool.shape[2]
+    commit_rows(k_pool, v_pool, page_ids, q_slot, k_new, v_new)
+    K = bf16_bits_to_f64(gather_pages(k_pool, page_ids, kv_len))
+    V = bf16_bits_to_f64(gather_pages(v_pool, page_ids, kv_len))
+    pos = slot_positions(pos_base, kv_len, P)
+    K = rope_rotate(K, pos[:, None], theta)
+    sel = list(range(len(q_slot))) if rows is None else list(rows)
+    Hq, Hkv = q_new.shape[1], K.shape[1]
+    G = Hq // Hkv
+    out = np.empty((len(sel), Hq, q_new.shape[2]), dtype=np.float64)
+    for j, i in enumerate(sel):
+        slot = int(q_slot[i])
+        q = rope_rotate(bf16_bits_to_f64(q_new[i]), np.int64(pos[slot]), theta)   # [Hq, D]
+        for h in range(Hq):
+            kh = h // G
+            s = sm_scale * (K[:slot + 1, kh, :] @ q[h])
+            p = _softmax_rows(s[None, :])[0]
+            out[j, h] = p @ V[:slot + 1, kh, :]
+    return out
+
+
+def merge_partials(m: np.ndarray, l: np.ndarray, o: np.ndarray) -> np.ndarray:
+    """Combine split-KV partial results.
+
+    Split s covers a subset of the keys and carries its running maximum
+    ``m[s]``, its sum of ``exp(score - m[s])`` as ``l[s]`` and the matching
+    un-normalised weighted sum of V as ``o[s]``.  The combination
+    ``m* = max m``, ``l* = sum l e^{m-m*}``, ``o* = sum o e^{m-m*} / l*`` equals
+    attention over the union of the subsets (standard log-sum-exp algebra; the
+    paper has no counterpart, the split is this implementation's).
+    """
+    m = np.asarray(m, dtype=np.float64)
+    w = np.exp(m - m.max(axis=0, keepdims=True))
+    l_star = (np.asarray(l, dtype=np.float64) * w).sum(axis=0)
+    return (np.asarray(o, dtype=np.float64) * w[..., None]).sum(axis=0) / l_star[..., None]
+
+
+def partial_attention(q: np.ndarray, K: np.ndarray, V: np.ndarray, sm_scale: float):
+    """(m, l, o) of one key subset, for ``merge_partials``: q ``[D]``, K/V ``[n, D]``."""
+    s = sm_scale * (K @ q)
+    m = s.max()
+    e = np.exp(s - m)
+    return m, e.sum(), e @ V
