@@ -1,0 +1,263 @@
+/*
+ * mepic.h - C ABI of the B200 (sm_100a) hot path of MEPIC: attention over a
+ * page-aligned, position-free chunk KV cache.
+ *
+ * Shared chunk pages hold UN-ROTATED keys (the paper's NoPE KV format,
+ * Section 3.3.3); rotary position embedding is applied to K inside the
+ * attention kernels, from the logical position base that every block-table
+ * entry carries.  The host side implements the scheduling path of Section 3.2
+ * / Algorithm 1 (canonical padding, chunk identity by hash of the padded
+ * tokens, first KV block private per request, remaining blocks shared); the
+ * device side implements the computation path of Section 3.3 (commit of
+ * recomputed K/V into the assigned pages, fused-RoPE attention).
+ *
+ * Conventions
+ *  - Every function returns an int32_t status: MEPIC_OK (0) or a negative
+ *    MEPIC_E_* code.  Nothing throws or aborts across this boundary;
+ *    mepic_last_error() returns thread-local text for the last failure.
+ *  - "host" / "device" is stated for every pointer.  The CALLER owns every
+ *    device buffer and the CUDA stream; the library owns only the host
+ *    metadata inside mepic_store_t.  The library never allocates or frees
+ *    device memory and never synchronises the stream: kernels are enqueued
+ *    and the call returns.
+ *  - Device-side problems (a page id outside the pool, a bounded wait that ran
+ *    out) never fault or hang the GPU: the kernel records a code in the device
+ *    status word the caller passes and carries on with safe values.  Read the
+ *    word after synchronising; 0 means clean.
+ *  - bf16 tensors are passed as plain pointers to 16-bit words.
+ *  - Layouts (row-major, last index fastest):
+ *        K pool, V pool : [num_pages][n_kv_heads][page_size][head_dim]  bf16
+ *        q (decode)     : [batch][n_q_heads][head_dim]                   bf16
+ *        block table    : page_ids[batch][table_stride], pos_base[batch][table_stride]  int32
+ *        rope table     : [max_position + 1][head_dim / 2][2] fp32 = (cos, sin)
+ *    q head h reads KV head h / (n_q_heads / n_kv_heads).
+ *  - RoPE convention (the paper does not state one): split-half pairing
+ *    (i, i + head_dim/2), angle = position * rope_theta^(-2 i / head_dim), no
+ *    frequency scaling.  V is never rotated.
+ *  - Logical slot t of a request lives in block-table entry e = t / page_size,
+ *    at in-page slot t % page_size, and has position pos_base[e] + t % page_size.
+ *    Causality is by logical slot; rotation is by position.
+ */
+#ifndef MEPIC_H_
+#define MEPIC_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define MEPIC_OK                 0
+#define MEPIC_E_INVAL           -1  /* bad argument, unsupported shape, misaligned pointer */
+#define MEPIC_E_NOSPACE         -2  /* Algorithm 1's Reject: the page pool cannot supply the blocks */
+#define MEPIC_E_NOTFOUND        -3  /* unknown chunk id or request id */
+#define MEPIC_E_CAPACITY        -4  /* caller's output array too small; required count written back */
+#define MEPIC_E_CUDA            -5  /* a CUDA runtime call failed; see mepic_last_error() */
+#define MEPIC_E_EXISTS          -6  /* request id already has a live block table */
+
+/* Codes a kernel may OR into the device status word. */
+#define MEPIC_DEV_BAD_PAGE      0x1 /* a block-table entry named a page outside [0, num_pages) */
+#define MEPIC_DEV_WAIT_EXPIRED  0x2 /* a bounded wait on an on-chip barrier ran out */
+#define MEPIC_DEV_BAD_POSITION  0x4 /* a position fell outside the rope table */
+#define MEPIC_DEV_BAD_SLOT      0x8 /* a new row's logical slot fell outside its request */
+
+#define MEPIC_SEG_CHUNK  0
+#define MEPIC_SEG_PROMPT 1
+
+typedef struct mepic_store mepic_store_t;
+
+typedef struct {
+  int32_t page_size;     /* tokens per KV block ("page"); power of two, >= 16 */
+  int32_t n_q_heads;
+  int32_t n_kv_heads;    /* divides n_q_heads; group size n_q_heads/n_kv_heads in {1,2,4,5,8} */
+  int32_t head_dim;      /* 64 or 128 */
+  int32_t num_pages;     /* pages in the pool */
+  int32_t pad_token_id;  /* token used for canonical padding; part of the hashed sequence */
+  int32_t max_position;  /* largest position the rope table covers (inclusive) */
+  float   rope_theta;
+} mepic_config_t;
+
+typedef struct {
+  int64_t pages_total;
+  int64_t pages_free;
+  int64_t pages_shared_held;          /* pages owned by resident chunks (all but their first block) */
+  int64_t pages_private_held;         /* pages owned by live requests */
+  int64_t chunks_resident;
+  int64_t chunk_refs;                 /* sum over chunks of live requests aliasing them */
+  int64_t dedup_hits;                 /* mepic_chunk_register calls that found the chunk resident */
+  int64_t unshared_equivalent_pages;  /* sum of block-table entries of live requests = pages a
+                                         per-request copy of every chunk would hold */
+  int64_t live_requests;
+} mepic_stats_t;
+
+typedef struct {
+  int32_t  kind;       /* MEPIC_SEG_CHUNK or MEPIC_SEG_PROMPT */
+  int32_t  n_tokens;   /* prompt segments: token count (0 = skipped); ignored for chunks */
+  uint64_t chunk_id;   /* chunk segments: id returned by mepic_chunk_register */
+} mepic_segment_t;
+
+const char* mepic_last_error(void);
+
+/* Number of kernels this library has launched in this process (all threads). */
+int64_t mepic_launch_count(void);
+
+/* ---------------------------------------------------------------- scheduling path (host only)
+ *
+ * mepic_store_create: make an empty store over a pool of cfg->num_pages pages.  Free pages are
+ * handed out first-in-first-out starting from 0,1,2,...; released pages rejoin the queue in
+ * ascending order (the paper leaves the order open; this one makes tables reproducible).
+ * cfg: host.  out: host, receives the handle.  Errors: E_INVAL.
+ */
+int32_t mepic_store_create(const mepic_config_t* cfg, mepic_store_t** out);
+void    mepic_store_destroy(mepic_store_t* store);
+
+/*
+ * mepic_chunk_register - Section 3.2.1 (canonical leading pad), Section 3.2.2 (residency lookup),
+ * Section 3.2.3 "KV Block Allocation" (identity = hash of the PADDED token sequence; the first
+ * block is recomputed per request, the remaining blocks are the shareable chunk KV).
+ *
+ * tokens (host, n_tokens > 0 int32): the UNPADDED chunk.  The store pads it at the front with
+ * pad_token_id to a multiple of page_size, hashes the padded sequence (64-bit FNV-1a, confirmed by
+ * a full token compare, so identity is by content) and looks it up.  On a miss it takes
+ * ceil(n/page_size) - 1 pages from the pool for the shareable blocks; on a hit it allocates
+ * nothing.  out_chunk_id, out_was_resident (0/1), out_lead_pad (pad tokens added), out_n_shared:
+ * host, each may be NULL.  out_shared_pages (host, cap entries, may be NULL when cap == 0)
+ * receives the shared page ids in block order.
+ * Errors: E_INVAL; E_NOSPACE (nothing allocated, chunk not registered); E_CAPACITY (cap too small:
+ * *out_n_shared holds the count needed; the registration itself HAS taken place).
+ */
+int32_t mepic_chunk_register(mepic_store_t* store, const int32_t* tokens, int32_t n_tokens,
+                             uint64_t* out_chunk_id, int32_t* out_was_resident, int32_t* out_lead_pad,
+                             int32_t* out_shared_pages, int32_t cap, int32_t* out_n_shared);
+
+/*
+ * mepic_build_block_table - Algorithm 1 (segment -> pad -> admission check -> block assignment)
+ * for one request whose chunks are already registered.
+ *
+ * segs (host, n_segs): the request's segments in order.  A chunk segment contributes one freshly
+ * allocated PRIVATE first page followed by the chunk's shared pages; a prompt segment contributes
+ * ceil(n_tokens/page_size) private pages and is padded at the back to a block boundary unless it
+ * is the request's last segment.  Entry e gets pos_base[e] = e * page_size (a token's position is
+ * its index in the padded sequence).  Outputs (host): out_page_ids / out_pos_base (cap_entries
+ * each), *out_n_entries, *out_kv_len (padded length; pads are ordinary tokens), and
+ * out_recompute_slots (cap_slots): the logical slots whose K/V the caller must compute and hand
+ * to mepic_attn_prefill = every slot below kv_len that lives on a private page, ascending.
+ * The admission check runs before any allocation: on E_NOSPACE nothing is held.
+ * Errors: E_INVAL (no tokens, bad kind), E_NOTFOUND (chunk id), E_EXISTS (request id live),
+ * E_NOSPACE, E_CAPACITY (required counts written to *out_n_entries / *out_n_slots; nothing held).
+ */
+int32_t mepic_build_block_table(mepic_store_t* store, int64_t request_id,
+                                const mepic_segment_t* segs, int32_t n_segs,
+                                int32_t* out_page_ids, int32_t* out_pos_base, int32_t cap_entries,
+                                int32_t* out_n_entries, int32_t* out_kv_len,
+                                int32_t* out_recompute_slots, int32_t cap_slots, int32_t* out_n_slots);
+
+/* Request end (Section 3.2.3 "Eviction Policy"): private pages go back to the pool in ascending
+ * order, the reference count of every chunk the request aliased drops by one; chunks stay
+ * resident.  Errors: E_NOTFOUND. */
+int32_t mepic_request_release(mepic_store_t* store, int64_t request_id);
+
+/* Snapshot of the pool ("HBM usage" of Section 4 in units of pages).  out: host. */
+int32_t mepic_store_stats(const mepic_store_t* store, mepic_stats_t* out);
+
+/* ---------------------------------------------------------------- rope table (host, set-up)
+ *
+ * Section 3.3.3 applies "the appropriate rotary offsets" without giving the formula; the table
+ * holds (cos, sin)(p * rope_theta^(-2i/head_dim)) for p in [0, max_position], i < head_dim/2,
+ * computed in double precision and rounded to fp32.  The caller uploads it once and passes the
+ * device copy to the attention calls.  mepic_rope_table_floats returns the float count
+ * (max_position+1) * head_dim, or 0 for a bad config; mepic_rope_table_fill writes that many
+ * floats to out (host).  Errors: E_INVAL.
+ */
+size_t  mepic_rope_table_floats(const mepic_config_t* cfg);
+int32_t mepic_rope_table_fill(const mepic_config_t* cfg, float* out);
+
+/* ---------------------------------------------------------------- decode (device)
+ *
+ * mepic_attn_decode - Section 3.3.3 for one new token per request: for every request b and query
+ * head h,
+ *     out[b,h,:] = sum_t softmax_t( sm_scale * < R(q_pos[b]) q[b,h,:] , R(pos_t) K_t > ) V_t ,
+ * t over the kv_len[b] logical slots of the request, K_t / V_t read through the block table from
+ * the un-rotated pools, R the rotary embedding.  The work is split over the KV axis across the
+ * whole GPU; partial (max, sum, weighted V) triples go to the workspace and a second kernel
+ * combines them (log-sum-exp merge) and writes bf16.
+ *
+ * All pointers in the struct are DEVICE pointers.  kv_len[b] >= 1; entries beyond
+ * ceil(kv_len[b]/page_size) are not read; slots at or beyond kv_len[b] in the last page are
+ * ignored whatever bits they hold.  workspace: at least mepic_attn_decode_workspace() bytes,
+ * 16-byte aligned; contents need not be initialised and are overwritten.  status: one int32 the
+ * caller zeroed; MEPIC_DEV_* bits are ORed in.  Two calls that overlap on the GPU must not share
+ * a workspace.  Errors: E_INVAL (null/misaligned pointer, unsupported shape, workspace too small),
+ * E_CUDA.
+ */
+typedef struct {
+  const void*    q;            /* bf16 [batch][n_q_heads][head_dim], un-rotated */
+  const void*    k_pool;       /* bf16 pool, K un-rotated; 16-byte aligned */
+  const void*    v_pool;       /* bf16 pool; 16-byte aligned */
+  const int32_t* page_ids;     /* [batch][table_stride] */
+  const int32_t* pos_base;     /* [batch][table_stride] */
+  const int32_t* kv_len;       /* [batch] */
+  const int32_t* q_pos;        /* [batch] position of the query token */
+  const float*   rope_table;   /* see above */
+  void*          out;          /* bf16 [batch][n_q_heads][head_dim] */
+  void*          workspace;
+  size_t         workspace_bytes;
+  int32_t*       status;
+  int32_t        table_stride;
+  int32_t        batch;
+  float          sm_scale;
+} mepic_decode_args_t;
+
+/* Bytes of workspace mepic_attn_decode needs for this config and batch on the CURRENT device
+ * (depends on its SM count); 0 on error. */
+size_t  mepic_attn_decode_workspace(const mepic_config_t* cfg, int32_t batch);
+int32_t mepic_attn_decode(const mepic_config_t* cfg, const mepic_decode_args_t* args, void* cuda_stream);
+
+/* ---------------------------------------------------------------- prefill (device)
+ *
+ * mepic_attn_prefill - Sections 3.3.1-3.3.3 for the rows a request recomputes (the first block of
+ * every chunk plus its prompt segments).  Step 1 (commit, Section 3.3.2): row i's k_new / v_new
+ * bits are written, un-rotated, to page page_ids[b][q_slot[i]/P], slot q_slot[i]%P of the pools.
+ * Step 2: every new row attends causally, by logical slot, over slots 0..q_slot[i] of its
+ * request's paged context (which now contains the committed rows), K rotated at each slot's
+ * position and the row's q at the position of its own slot:
+ *     out[i,h,:] = sum_{t <= q_slot[i]} softmax_t( sm_scale * < R(pos_{q_slot[i]}) q_new[i,h,:], R(pos_t) K_t > ) V_t .
+ * bf16 tensor-core products, fp32 accumulation.
+ *
+ * Rows are grouped by request: rows row_offsets[b] .. row_offsets[b+1]-1 belong to request b and
+ * their q_slot values are strictly ascending.  The caller guarantees that the slots named lie on
+ * the request's PRIVATE pages (shared pages are never written by a correct caller; the library
+ * cannot tell).  All struct pointers are DEVICE pointers except row_offsets_host (host copy of
+ * row_offsets, batch+1 entries, read during the call for launch sizing).
+ * workspace: mepic_attn_prefill_workspace() bytes, 16-byte aligned.  Errors as for decode.
+ */
+typedef struct {
+  const void*    q_new;        /* bf16 [rows][n_q_heads][head_dim], un-rotated */
+  const void*    k_new;        /* bf16 [rows][n_kv_heads][head_dim], un-rotated */
+  const void*    v_new;        /* bf16 [rows][n_kv_heads][head_dim] */
+  const int32_t* row_offsets;  /* [batch+1] */
+  const int32_t* q_slot;       /* [rows] logical slot of each new row */
+  void*          k_pool;       /* read and written (commit) */
+  void*          v_pool;
+  const int32_t* page_ids;     /* [batch][table_stride] */
+  const int32_t* pos_base;     /* [batch][table_stride] */
+  const int32_t* kv_len;       /* [batch] */
+  const float*   rope_table;
+  void*          out;          /* bf16 [rows][n_q_heads][head_dim] */
+  void*          workspace;
+  size_t         workspace_bytes;
+  int32_t*       status;
+  const int32_t* row_offsets_host;
+  int32_t        table_stride;
+  int32_t        batch;
+  float          sm_scale;
+} mepic_prefill_args_t;
+
+size_t  mepic_attn_prefill_workspace(const mepic_config_t* cfg, int32_t batch, const int32_t* row_offsets_host);
+int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_prefill_args_t* args, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MEPIC_H_ */

@@ -1,0 +1,11 @@
+// Internal declarations shared by the translation units of libmepic (not part of the ABI).
+#ifndef MEPIC_INTERNAL_H_
+#define MEPIC_INTERNAL_H_
+
+#include "mepic.h"
+
+void mepic_set_error(const char* fmt, ...);
+bool mepic_config_ok(const mepic_config_t* cfg);
+void mepic_count_launches(int n);
+
+#endif

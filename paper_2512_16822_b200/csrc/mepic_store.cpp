@@ -1,0 +1,288 @@
+// Host side of the MEPIC hot path: the scheduling path of Section 3.2 / Algorithm 1.
+//
+// A store owns the metadata of one page pool: a FIFO free list, the index of
+// resident chunks (identity = hash of the canonically padded token sequence,
+// Section 3.2.3) and the private pages of every live request.  No device
+// memory is touched here; the K/V bytes live in buffers the caller owns.
+#include "mepic.h"
+#include "mepic_internal.h"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <deque>
+#include <mutex>
+#include <new>
+#include <unordered_map>
+#include <vector>
+
+namespace {
+thread_local char g_err[512] = "";
+}
+
+void mepic_set_error(const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+}
+
+bool mepic_config_ok(const mepic_config_t* c) {
+  if (!c) { mepic_set_error("config is NULL"); return false; }
+  if (c->page_size < 16 || (c->page_size & (c->page_size - 1)) != 0) {
+    mepic_set_error("page_size %d must be a power of two >= 16", c->page_size); return false;
+  }
+  if (c->head_dim != 64 && c->head_dim != 128) { mepic_set_error("head_dim %d must be 64 or 128", c->head_dim); return false; }
+  if (c->n_kv_heads < 1 || c->n_q_heads < 1 || c->n_q_heads % c->n_kv_heads != 0) {
+    mepic_set_error("n_q_heads %d must be a positive multiple of n_kv_heads %d", c->n_q_heads, c->n_kv_heads); return false;
+  }
+  const int g = c->n_q_heads / c->n_kv_heads;
+  if (!(g == 1 || g == 2 || g == 4 || g == 5 || g == 8)) { mepic_set_error("group size %d not in {1,2,4,5,8}", g); return false; }
+  if (c->num_pages < 1) { mepic_set_error("num_pages %d < 1", c->num_pages); return false; }
+  if (c->max_position < c->page_size - 1) { mepic_set_error("max_position %d < page_size-1", c->max_position); return false; }
+  if (!(c->rope_theta > 1.0f)) { mepic_set_error("rope_theta must exceed 1"); return false; }
+  return true;
+}
+
+struct Chunk {
+  std::vector<int32_t> padded;   // canonical form: leading pads + tokens
+  std::vector<int32_t> shared;   // page ids of blocks 1..n-1
+  int64_t refs = 0;
+};
+
+struct LiveRequest {
+  std::vector<int32_t> private_pages;
+  std::vector<uint64_t> chunks;  // one entry per chunk segment
+  int64_t entries = 0;
+};
+
+struct mepic_store {
+  mepic_config_t cfg;
+  std::deque<int32_t> free_pages;
+  std::unordered_map<uint64_t, Chunk> chunks;          // id -> chunk; id = hash, bumped on collision
+  std::unordered_map<int64_t, LiveRequest> requests;
+  int64_t dedup_hits = 0;
+  int64_t shared_held = 0;
+  int64_t private_held = 0;
+  mutable std::mutex mu;
+};
+
+static uint64_t fnv1a64(const std::vector<int32_t>& v) {
+  uint64_t h = 0xcbf29ce484222325ULL;
+  for (int32_t t : v) {
+    uint32_t u = static_cast<uint32_t>(t);
+    for (int b = 0; b < 4; ++b) {               // little-endian bytes of the int32
+      h ^= static_cast<uint64_t>((u >> (8 * b)) & 0xffu);
+      h *= 0x100000001b3ULL;
+    }
+  }
+  return h;
+}
+
+extern "C" const char* mepic_last_error(void) { return g_err; }
+
+extern "C" int32_t mepic_store_create(const mepic_config_t* cfg, mepic_store_t** out) {
+  if (!out) { mepic_set_error("out is NULL"); return MEPIC_E_INVAL; }
+  *out = nullptr;
+  if (!mepic_config_ok(cfg)) return MEPIC_E_INVAL;
+  mepic_store* s = new (std::nothrow) mepic_store();
+  if (!s) { mepic_set_error("out of host memory"); return MEPIC_E_INVAL; }
+  s->cfg = *cfg;
+  for (int32_t p = 0; p < cfg->num_pages; ++p) s->free_pages.push_back(p);
+  *out = s;
+  return MEPIC_OK;
+}
+
+extern "C" void mepic_store_destroy(mepic_store_t* store) { delete store; }
+
+extern "C" int32_t mepic_chunk_register(mepic_store_t* s, const int32_t* tokens, int32_t n_tokens,
+                                        uint64_t* out_chunk_id, int32_t* out_was_resident, int32_t* out_lead_pad,
+                                        int32_t* out_shared_pages, int32_t cap, int32_t* out_n_shared) {
+  if (!s || !tokens || n_tokens <= 0 || cap < 0 || (cap > 0 && !out_shared_pages)) {
+    mepic_set_error("chunk_register: bad argument"); return MEPIC_E_INVAL;
+  }
+  std::lock_guard<std::mutex> lock(s->mu);
+  const int32_t P = s->cfg.page_size;
+  const int32_t lead = (P - n_tokens % P) % P;                 // Section 3.2.1: chunks are padded at the FRONT
+  std::vector<int32_t> padded(static_cast<size_t>(lead) + n_tokens, s->cfg.pad_token_id);
+  std::copy(tokens, tokens + n_tokens, padded.begin() + lead);
+  uint64_t id = fnv1a64(padded);
+  const Chunk* hit = nullptr;
+  for (;; ++id) {                                               // identity is by content: confirm, else probe on
+    auto it = s->chunks.find(id);
+    if (it == s->chunks.end()) break;
+    if (it->second.padded == padded) { hit = &it->second; break; }
+  }
+  int32_t resident = 0;
+  const std::vector<int32_t>* shared = nullptr;
+  if (hit) {
+    resident = 1;
+    s->dedup_hits += 1;
+    shared = &hit->shared;
+  } else {
+    const size_t n_shared = padded.size() / P - 1;              // first block is private to each request
+    if (n_shared > s->free_pages.size()) {
+      mepic_set_error("chunk_register: %zu shared pages needed, %zu free", n_shared, s->free_pages.size());
+      return MEPIC_E_NOSPACE;
+    }
+    Chunk c;
+    c.shared.reserve(n_shared);
+    for (size_t i = 0; i < n_shared; ++i) { c.shared.push_back(s->free_pages.front()); s->free_pages.pop_front(); }
+    c.padded = std::move(padded);
+    s->shared_held += static_cast<int64_t>(n_shared);
+    shared = &s->chunks.emplace(id, std::move(c)).first->second.shared;
+  }
+  if (out_chunk_id) *out_chunk_id = id;
+  if (out_was_resident) *out_was_resident = resident;
+  if (out_lead_pad) *out_lead_pad = lead;
+  if (out_n_shared) *out_n_shared = static_cast<int32_t>(shared->size());
+  if (static_cast<size_t>(cap) < shared->size()) {
+    if (out_shared_pages || cap > 0) { mepic_set_error("chunk_register: cap %d < %zu shared pages", cap, shared->size()); return MEPIC_E_CAPACITY; }
+    return MEPIC_OK;   // caller did not ask for the page list
+  }
+  if (out_shared_pages) std::copy(shared->begin(), shared->end(), out_shared_pages);
+  return MEPIC_OK;
+}
+
+extern "C" int32_t mepic_build_block_table(mepic_store_t* s, int64_t request_id,
+                                           const mepic_segment_t* segs, int32_t n_segs,
+                                           int32_t* out_page_ids, int32_t* out_pos_base, int32_t cap_entries,
+                                           int32_t* out_n_entries, int32_t* out_kv_len,
+                                           int32_t* out_recompute_slots, int32_t cap_slots, int32_t* out_n_slots) {
+  if (!s || !segs || n_segs <= 0 || cap_entries < 0 || cap_slots < 0 ||
+      (cap_entries > 0 && (!out_page_ids || !out_pos_base)) || (cap_slots > 0 && !out_recompute_slots)) {
+    mepic_set_error("build_block_table: bad argument"); return MEPIC_E_INVAL;
+  }
+  std::lock_guard<std::mutex> lock(s->mu);
+  if (s->requests.count(request_id)) { mepic_set_error("request %lld already live", (long long)request_id); return MEPIC_E_EXISTS; }
+  const int64_t P = s->cfg.page_size;
+  // Pass 1 (Algorithm 1, canonicalisation + admission check): sizes only, nothing allocated.
+  int last = -1;
+  for (int i = 0; i < n_segs; ++i) {
+    if (segs[i].kind == MEPIC_SEG_CHUNK) {
+      if (!s->chunks.count(segs[i].chunk_id)) { mepic_set_error("segment %d: unknown chunk id", i); return MEPIC_E_NOTFOUND; }
+      last = i;
+    } else if (segs[i].kind == MEPIC_SEG_PROMPT) {
+      if (segs[i].n_tokens < 0) { mepic_set_error("segment %d: negative length", i); return MEPIC_E_INVAL; }
+      if (segs[i].n_tokens > 0) last = i;                      // empty prompt segments are skipped
+    } else { mepic_set_error("segment %d: bad kind %d", i, segs[i].kind); return MEPIC_E_INVAL; }
+  }
+  if (last < 0) { mepic_set_error("request has no tokens"); return MEPIC_E_INVAL; }
+  int64_t entries = 0, need_private = 0, slots = 0, kv_len = 0;
+  for (int i = 0; i <= last; ++i) {
+    if (segs[i].kind == MEPIC_SEG_CHUNK) {
+      const Chunk& c = s->chunks.at(segs[i].chunk_id);
+      entries += 1 + static_cast<int64_t>(c.shared.size());
+      need_private += 1;
+      slots += P;
+      kv_len = entries * P;
+    } else if (segs[i].n_tokens > 0) {
+      const int64_t n = segs[i].n_tokens, pages = (n + P - 1) / P;
+      const int64_t seg_len = (i == last) ? n : pages * P;     // trailing pad unless final segment
+      kv_len = entries * P + seg_len;
+      slots += seg_len;
+      entries += pages;
+      need_private += pages;
+    }
+  }
+  if (kv_len > INT32_MAX || entries > INT32_MAX) { mepic_set_error("request too long"); return MEPIC_E_INVAL; }
+  if (out_n_entries) *out_n_entries = static_cast<int32_t>(entries);
+  if (out_n_slots) *out_n_slots = static_cast<int32_t>(slots);
+  if (out_kv_len) *out_kv_len = static_cast<int32_t>(kv_len);
+  if (entries > cap_entries || slots > cap_slots) {
+    mepic_set_error("build_block_table: need %lld entries, %lld slots", (long long)entries, (long long)slots);
+    return MEPIC_E_CAPACITY;
+  }
+  if (need_private > static_cast<int64_t>(s->free_pages.size())) {
+    mepic_set_error("build_block_table: %lld private pages needed, %zu free", (long long)need_private, s->free_pages.size());
+    return MEPIC_E_NOSPACE;                                     // Reject; nothing is held
+  }
+  // Pass 2 (block assignment).
+  LiveRequest live;
+  int64_t e = 0, w = 0;
+  auto take = [&]() { int32_t p = s->free_pages.front(); s->free_pages.pop_front(); live.private_pages.push_back(p); return p; };
+  for (int i = 0; i <= last; ++i) {
+    const int64_t start = e * P;
+    if (segs[i].kind == MEPIC_SEG_CHUNK) {
+      Chunk& c = s->chunks.at(segs[i].chunk_id);
+      out_page_ids[e++] = take();                               // first block: private, recomputed
+      for (int32_t p : c.shared) out_page_ids[e++] = p;         // remaining blocks: shared chunk KV
+      for (int64_t t = 0; t < P; ++t) out_recompute_slots[w++] = static_cast<int32_t>(start + t);
+      c.refs += 1;
+      live.chunks.push_back(segs[i].chunk_id);
+    } else if (segs[i].n_tokens > 0) {
+      const int64_t n = segs[i].n_tokens, pages = (n + P - 1) / P;
+      for (int64_t k = 0; k < pages; ++k) out_page_ids[e++] = take();
+      const int64_t seg_len = (i == last) ? n : pages * P;
+      for (int64_t t = 0; t < seg_len; ++t) out_recompute_slots[w++] = static_cast<int32_t>(start + t);
+    }
+  }
+  for (int64_t k = 0; k < entries; ++k) out_pos_base[k] = static_cast<int32_t>(k * P);
+  live.entries = entries;
+  s->private_held += static_cast<int64_t>(live.private_pages.size());
+  s->requests.emplace(request_id, std::move(live));
+  return MEPIC_OK;
+}
+
+extern "C" int32_t mepic_request_release(mepic_store_t* s, int64_t request_id) {
+  if (!s) { mepic_set_error("store is NULL"); return MEPIC_E_INVAL; }
+  std::lock_guard<std::mutex> lock(s->mu);
+  auto it = s->requests.find(request_id);
+  if (it == s->requests.end()) { mepic_set_error("request %lld not live", (long long)request_id); return MEPIC_E_NOTFOUND; }
+  LiveRequest& r = it->second;
+  for (uint64_t id : r.chunks) s->chunks.at(id).refs -= 1;
+  std::sort(r.private_pages.begin(), r.private_pages.end());
+  for (int32_t p : r.private_pages) s->free_pages.push_back(p);
+  s->private_held -= static_cast<int64_t>(r.private_pages.size());
+  s->requests.erase(it);
+  return MEPIC_OK;
+}
+
+extern "C" int32_t mepic_store_stats(const mepic_store_t* s, mepic_stats_t* out) {
+  if (!s || !out) { mepic_set_error("stats: NULL argument"); return MEPIC_E_INVAL; }
+  std::lock_guard<std::mutex> lock(s->mu);
+  out->pages_total = s->cfg.num_pages;
+  out->pages_free = static_cast<int64_t>(s->free_pages.size());
+  out->pages_shared_held = s->shared_held;
+  out->pages_private_held = s->private_held;
+  out->chunks_resident = static_cast<int64_t>(s->chunks.size());
+  int64_t refs = 0;
+  for (const auto& kv : s->chunks) refs += kv.second.refs;
+  out->chunk_refs = refs;
+  out->dedup_hits = s->dedup_hits;
+  int64_t ent = 0;
+  for (const auto& kv : s->requests) ent += kv.second.entries;
+  out->unshared_equivalent_pages = ent;
+  out->live_requests = static_cast<int64_t>(s->requests.size());
+  return MEPIC_OK;
+}
+
+// ---------------------------------------------------------------- rope table (set-up, host)
+extern "C" size_t mepic_rope_table_floats(const mepic_config_t* cfg) {
+  if (!mepic_config_ok(cfg)) return 0;
+  return (static_cast<size_t>(cfg->max_position) + 1) * static_cast<size_t>(cfg->head_dim);
+}
+
+extern "C" int32_t mepic_rope_table_fill(const mepic_config_t* cfg, float* out) {
+  if (!mepic_config_ok(cfg) || !out) { if (cfg && !out) mepic_set_error("rope_table_fill: out is NULL"); return MEPIC_E_INVAL; }
+  const int half = cfg->head_dim / 2;
+  std::vector<double> inv_freq(half);
+  for (int i = 0; i < half; ++i) inv_freq[i] = std::pow(static_cast<double>(cfg->rope_theta), -2.0 * i / cfg->head_dim);
+  for (int64_t p = 0; p <= cfg->max_position; ++p) {
+    float* row = out + p * cfg->head_dim;
+    for (int i = 0; i < half; ++i) {
+      const double a = static_cast<double>(p) * inv_freq[i];
+      row[2 * i] = static_cast<float>(std::cos(a));
+      row[2 * i + 1] = static_cast<float>(std::sin(a));
+    }
+  }
+  return MEPIC_OK;
+}
+
+// ---------------------------------------------------------------- launch counter
+#include <atomic>
+static std::atomic<int64_t> g_launches{0};
+void mepic_count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+extern "C" int64_t mepic_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

@@ -1,0 +1,159 @@
+"""Device-side plumbing around the C ABI: torch tensors, streams, uploads.
+
+Nothing here computes any part of the method; it allocates the buffers the ABI
+asks the caller to own, moves host tables to the device and issues the calls.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass
+from typing import List, Optional, Sequence, Tuple
+
+import numpy as np
+import torch
+
+from . import (Config, Segment, Store, MEPIC_SEG_CHUNK, MEPIC_SEG_PROMPT, mepic_attn_decode,
+               mepic_attn_decode_workspace, mepic_attn_prefill, mepic_attn_prefill_workspace,
+               mepic_rope_table_fill)
+
+
+@dataclass
+class Table:
+    request_id: int
+    page_ids: np.ndarray
+    pos_base: np.ndarray
+    kv_len: int
+    recompute_slots: np.ndarray
+
+
+def build_tables(store: Store, chunks: Sequence[np.ndarray], requests) -> List[Table]:
+    """Register each request's chunks, then build its block table, in request order.
+
+    ``requests`` are objects with ``request_id`` and ``segments`` = [(kind, value)] where a chunk
+    segment's value indexes ``chunks``.
+    """
+    out = []
+    for r in requests:
+        segs = []
+        for kind, val in r.segments:
+            if kind == MEPIC_SEG_CHUNK:
+                cid, _, _, _ = store.chunk_register(chunks[val])
+                segs.append(Segment(MEPIC_SEG_CHUNK, cid))
+            else:
+                segs.append(Segment(MEPIC_SEG_PROMPT, int(val)))
+        pages, base, kv_len, slots = store.build_block_table(r.request_id, segs)
+        out.append(Table(r.request_id, pages, base, kv_len, slots))
+    return out
+
+
+def pack_tables(tables: Sequence[Table], page_size: int) -> Tuple[np.ndarray, np.ndarray, np.ndarray, np.ndarray]:
+    """Host arrays page_ids[B, stride], pos_base[B, stride], kv_len[B], q_pos[B].
+
+    q_pos is the position of the request's last slot: the decode query is the newest token, whose
+    K/V is already in the cache.
+    """
+    stride = max(len(t.page_ids) for t in tables)
+    B = len(tables)
+    page_ids = np.zeros((B, stride), dtype=np.int32)
+    pos_base = np.zeros((B, stride), dtype=np.int32)
+    kv_len = np.zeros(B, dtype=np.int32)
+    for i, t in enumerate(tables):
+        page_ids[i, :len(t.page_ids)] = t.page_ids
+        pos_base[i, :len(t.pos_base)] = t.pos_base
+        kv_len[i] = t.kv_len
+    last = kv_len - 1
+    q_pos = pos_base[np.arange(B), last // page_size] + last % page_size
+    return page_ids, pos_base, kv_len, q_pos.astype(np.int32)
+
+
+def bf16_tensor(bits: np.ndarray, device) -> torch.Tensor:
+    """uint16 bit patterns -> torch.bfloat16 tensor on ``device`` (no value conversion)."""
+    t = torch.from_numpy(np.ascontiguousarray(bits).view(np.int16))
+    return t.to(device).view(torch.bfloat16)
+
+
+def bf16_bits(t: torch.Tensor) -> np.ndarray:
+    return t.detach().contiguous().view(torch.int16).cpu().numpy().view(np.uint16)
+
+
+class Device:
+    """The buffers one pool needs on a GPU: K/V pools, rope table, status word."""
+
+    def __init__(self, cfg: Config, k_bits: Optional[np.ndarray] = None, v_bits: Optional[np.ndarray] = None,
+                 device: str = "cuda:0"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("the MEPIC kernels need a CUDA device; there is no CPU path")
+        self.cfg = cfg
+        self.device = torch.device(device)
+        shape = (cfg.num_pages, cfg.n_kv_heads, cfg.page_size, cfg.head_dim)
+        if k_bits is not None:
+            assert k_bits.shape == shape and v_bits.shape == shape
+            self.k_pool = bf16_tensor(k_bits, self.device)
+            self.v_pool = bf16_tensor(v_bits, self.device)
+        else:
+            self.k_pool = torch.empty(shape, dtype=torch.bfloat16, device=self.device)
+            self.v_pool = torch.empty(shape, dtype=torch.bfloat16, device=self.device)
+        self.rope = torch.from_numpy(mepic_rope_table_fill(cfg)).to(self.device)
+        self.status = torch.zeros(1, dtype=torch.int32, device=self.device)
+
+    def read_status(self) -> int:
+        return int(self.status.item())
+
+
+class DecodeBatch:
+    """Device copies of one decode batch's tables plus output and workspace."""
+
+    def __init__(self, dev: Device, page_ids: np.ndarray, pos_base: np.ndarray, kv_len: np.ndarray,
+                 q_pos: np.ndarray, q_bits: Optional[np.ndarray] = None):
+        cfg = dev.cfg
+        self.dev = dev
+        self.batch, self.stride = page_ids.shape
+        d = dev.device
+        self.page_ids = torch.from_numpy(np.ascontiguousarray(page_ids, dtype=np.int32)).to(d)
+        self.pos_base = torch.from_numpy(np.ascontiguousarray(pos_base, dtype=np.int32)).to(d)
+        self.kv_len = torch.from_numpy(np.ascontiguousarray(kv_len, dtype=np.int32)).to(d)
+        self.q_pos = torch.from_numpy(np.ascontiguousarray(q_pos, dtype=np.int32)).to(d)
+        qshape = (self.batch, cfg.n_q_heads, cfg.head_dim)
+        self.q = bf16_tensor(q_bits, d) if q_bits is not None else torch.empty(qshape, dtype=torch.bfloat16, device=d)
+        self.out = torch.empty(qshape, dtype=torch.bfloat16, device=d)
+        self.ws_bytes = mepic_attn_decode_workspace(cfg, self.batch)
+        self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=d)
+
+    def run(self, sm_scale: float, stream=None) -> torch.Tensor:
+        s = stream if stream is not None else torch.cuda.current_stream(self.dev.device)
+        mepic_attn_decode(self.dev.cfg, q=self.q, k_pool=self.dev.k_pool, v_pool=self.dev.v_pool,
+                          page_ids=self.page_ids, pos_base=self.pos_base, kv_len=self.kv_len, q_pos=self.q_pos,
+                          rope_table=self.dev.rope, out=self.out, workspace=self.workspace,
+                          workspace_bytes=self.ws_bytes, status=self.dev.status, table_stride=self.stride,
+                          batch=self.batch, sm_scale=sm_scale, stream=s)
+        return self.out
+
+
+class PrefillBatch:
+    """Device copies of one prefill batch: new rows, their slots, tables, output, workspace."""
+
+    def __init__(self, dev: Device, page_ids: np.ndarray, pos_base: np.ndarray, kv_len: np.ndarray,
+                 row_offsets: np.ndarray, q_slot: np.ndarray, q_bits: np.ndarray, k_bits: np.ndarray,
+                 v_bits: np.ndarray):
+        cfg = dev.cfg
+        self.dev = dev
+        self.batch, self.stride = page_ids.shape
+        d = dev.device
+        i32 = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).to(d)
+        self.page_ids, self.pos_base, self.kv_len = i32(page_ids), i32(pos_base), i32(kv_len)
+        self.row_offsets_host = np.ascontiguousarray(row_offsets, dtype=np.int32)
+        self.row_offsets, self.q_slot = i32(row_offsets), i32(q_slot)
+        self.q_new, self.k_new, self.v_new = bf16_tensor(q_bits, d), bf16_tensor(k_bits, d), bf16_tensor(v_bits, d)
+        self.out = torch.empty(self.q_new.shape, dtype=torch.bfloat16, device=d)
+        self.ws_bytes = mepic_attn_prefill_workspace(cfg, self.batch, self.row_offsets_host)
+        self.workspace = torch.empty(max(self.ws_bytes, 16), dtype=torch.uint8, device=d)
+
+    def run(self, sm_scale: float, stream=None) -> torch.Tensor:
+        s = stream if stream is not None else torch.cuda.current_stream(self.dev.device)
+        mepic_attn_prefill(self.dev.cfg, q_new=self.q_new, k_new=self.k_new, v_new=self.v_new,
+                           row_offsets=self.row_offsets, q_slot=self.q_slot, k_pool=self.dev.k_pool,
+                           v_pool=self.dev.v_pool, page_ids=self.page_ids, pos_base=self.pos_base,
+                           kv_len=self.kv_len, rope_table=self.dev.rope, out=self.out, workspace=self.workspace,
+                           workspace_bytes=self.ws_bytes, status=self.dev.status,
+                           row_offsets_host=self.row_offsets_host, table_stride=self.stride, batch=self.batch,
+                           sm_scale=sm_scale, stream=s)
+        return self.out
