@@ -1,15 +1,497 @@
-// Prefill (selective recompute) entry points: placeholder translation unit until the kernel lands.
+// Prefill (selective recompute, Sections 3.3.1-3.3.3): commit the recomputed K/V rows
+// un-rotated into their private pages, then let every new row attend causally over its
+// request's paged context with RoPE applied to K on the way from the page pool to the
+// tensor cores.
+//
+// Attention kernel.  One CTA per (request, kv head, tile of query positions).  A tile packs
+// QT = 128 / G query positions x the G query heads of the kv head into the 128 rows of one
+// tcgen05 MMA (M = 128), so that one staged K/V tile serves all G heads.  Per 128-key tile:
+//   1. the CTA reads the K rows through the block table, rotates each row at its position
+//      in fp32 registers (cos/sin from the table row of that position), rounds to bf16 and
+//      stores it into shared memory in the 128-byte-swizzled K-major layout the MMA reads;
+//      V rows are copied into the same physical layout (read by the MMA as MN-major);
+//   2. S = Q' K'^T : 8 x tcgen05.mma (128x128x16, bf16 -> fp32) into tensor memory;
+//   3. thread r owns row r: tcgen05.ld its 128 scores, causal mask by logical slot, online
+//      softmax in the log2 domain, P -> bf16 -> shared memory (K-major, swizzled); the O
+//      accumulator in tensor memory is rescaled when a row's maximum moved;
+//   4. O += P V : 8 x tcgen05.mma (128 x D x 16).
+// Q' carries the rotation at the row's own position and sm_scale * log2(e).
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
 #include "mepic.h"
 #include "mepic_internal.h"
 
-extern "C" size_t mepic_attn_prefill_workspace(const mepic_config_t* cfg, int32_t batch, const int32_t* row_offsets_host) {
-  (void)cfg; (void)batch; (void)row_offsets_host;
-  mepic_set_error("prefill: not built yet");
-  return 0;
+namespace {
+
+constexpr int kThreads = 128;
+constexpr int kTileN = 128;            // keys per staged tile
+constexpr int kBlockBytes = 128 * 128; // one [128 rows x 64 bf16] swizzled block
+constexpr int kTmemCols = 256;         // S: columns 0..127, O: columns 128..128+D-1
+constexpr int kSpinLimit = 1 << 22;
+
+struct Item { int32_t b, h, row0, nq; };   // rows row0 .. row0+nq-1 (global row indices) of request b
+
+struct PrefillParams {
+  const uint16_t* q_new;
+  const uint16_t* k_new;
+  const uint16_t* v_new;
+  const int32_t* row_offsets;
+  const int32_t* q_slot;
+  uint16_t* k_pool;
+  uint16_t* v_pool;
+  const int32_t* page_ids;
+  const int32_t* pos_base;
+  const int32_t* kv_len;
+  const float* rope;
+  uint16_t* out;
+  const Item* items;
+  int32_t* status;
+  int table_stride, batch, n_kv_heads, page_size, num_pages, max_position, total_rows;
+  float scale_log2;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ float ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
+__device__ __forceinline__ float2 bf16x2_to_float2(uint32_t w) {
+  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+}
+// (lo, hi) -> packed bf16x2, round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+// byte offset of 16-byte chunk `chunk` of row `row` inside a [rows x 128 B] block with the 128-byte swizzle
+__device__ __forceinline__ uint32_t sw128(int row, int chunk) { return static_cast<uint32_t>(row * 128 + ((chunk ^ (row & 7)) << 4)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{ .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p; }"
+               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (int i = 0; i < kSpinLimit; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
 }
 
-extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_prefill_args_t* args, void* cuda_stream) {
-  (void)cfg; (void)args; (void)cuda_stream;
-  mepic_set_error("prefill: not built yet");
+// ---- tcgen05 wrappers
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], bf16 inputs, fp32 accumulate; one thread issues
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{ .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }"
+               ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return static_cast<uint64_t>((addr & 0x3ffffu) >> 4) | (static_cast<uint64_t>(lbo_bytes >> 4) << 16) |
+         (static_cast<uint64_t>(sbo_bytes >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// instruction descriptor: fp32 accumulator, bf16 A and B, M x N, majors (0 = K-major, 1 = MN-major)
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn_major, int b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a_mn_major) << 15) |
+         (static_cast<uint32_t>(b_mn_major) << 16) | (static_cast<uint32_t>(N >> 3) << 17) |
+         (static_cast<uint32_t>(M >> 4) << 24);
+}
+
+#define TMEM_LD32(taddr, r, o)                                                                                        \
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "                                                            \
+               "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26," \
+               "%27,%28,%29,%30,%31}, [%32];"                                                                       \
+               : "=r"(r[o + 0]), "=r"(r[o + 1]), "=r"(r[o + 2]), "=r"(r[o + 3]), "=r"(r[o + 4]), "=r"(r[o + 5]),     \
+                 "=r"(r[o + 6]), "=r"(r[o + 7]), "=r"(r[o + 8]), "=r"(r[o + 9]), "=r"(r[o + 10]), "=r"(r[o + 11]),   \
+                 "=r"(r[o + 12]), "=r"(r[o + 13]), "=r"(r[o + 14]), "=r"(r[o + 15]), "=r"(r[o + 16]),                \
+                 "=r"(r[o + 17]), "=r"(r[o + 18]), "=r"(r[o + 19]), "=r"(r[o + 20]), "=r"(r[o + 21]),                \
+                 "=r"(r[o + 22]), "=r"(r[o + 23]), "=r"(r[o + 24]), "=r"(r[o + 25]), "=r"(r[o + 26]),                \
+                 "=r"(r[o + 27]), "=r"(r[o + 28]), "=r"(r[o + 29]), "=r"(r[o + 30]), "=r"(r[o + 31])                 \
+               : "r"(taddr) : "memory")
+
+#define TMEM_ST32(taddr, r, o)                                                                                        \
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "                                                      \
+               "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27," \
+               "%28,%29,%30,%31,%32};"                                                                              \
+               ::"r"(taddr), "r"(r[o + 0]), "r"(r[o + 1]), "r"(r[o + 2]), "r"(r[o + 3]), "r"(r[o + 4]), "r"(r[o + 5]), \
+                 "r"(r[o + 6]), "r"(r[o + 7]), "r"(r[o + 8]), "r"(r[o + 9]), "r"(r[o + 10]), "r"(r[o + 11]),         \
+                 "r"(r[o + 12]), "r"(r[o + 13]), "r"(r[o + 14]), "r"(r[o + 15]), "r"(r[o + 16]), "r"(r[o + 17]),     \
+                 "r"(r[o + 18]), "r"(r[o + 19]), "r"(r[o + 20]), "r"(r[o + 21]), "r"(r[o + 22]), "r"(r[o + 23]),     \
+                 "r"(r[o + 24]), "r"(r[o + 25]), "r"(r[o + 26]), "r"(r[o + 27]), "r"(r[o + 28]), "r"(r[o + 29]),     \
+                 "r"(r[o + 30]), "r"(r[o + 31]) : "memory")
+
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// ---------------------------------------------------------------- commit (Section 3.3.2)
+// One CTA per new row: its K and V bits go, un-rotated, to (page, slot) of the pools.
+__global__ void mepic_prefill_commit(const PrefillParams p, int chunks_per_row) {
+  const int row = blockIdx.x;
+  __shared__ int sh_b;
+  if (threadIdx.x == 0) {
+    int b = 0;
+    while (b + 1 < p.batch && row >= p.row_offsets[b + 1]) ++b;
+    sh_b = b;
+  }
+  __syncthreads();
+  const int b = sh_b;
+  const int slot = p.q_slot[row];
+  if (slot < 0 || slot >= p.kv_len[b]) { if (threadIdx.x == 0) atomicOr(p.status, MEPIC_DEV_BAD_SLOT); return; }
+  const int page = p.page_ids[static_cast<size_t>(b) * p.table_stride + slot / p.page_size];
+  if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { if (threadIdx.x == 0) atomicOr(p.status, MEPIC_DEV_BAD_PAGE); return; }
+  const int D8 = chunks_per_row / p.n_kv_heads;        // 16-byte chunks per head row
+  for (int c = threadIdx.x; c < chunks_per_row; c += blockDim.x) {
+    const int h = c / D8, cc = c % D8;
+    const size_t dst = (((static_cast<size_t>(page) * p.n_kv_heads + h) * p.page_size + slot % p.page_size) * D8 + cc);
+    const size_t src = static_cast<size_t>(row) * chunks_per_row + c;
+    reinterpret_cast<uint4*>(p.k_pool)[dst] = reinterpret_cast<const uint4*>(p.k_new)[src];
+    reinterpret_cast<uint4*>(p.v_pool)[dst] = reinterpret_cast<const uint4*>(p.v_new)[src];
+  }
+}
+
+// ---------------------------------------------------------------- attention
+template <int D, int G>
+__global__ void __launch_bounds__(kThreads, 1) mepic_prefill_attn(const PrefillParams p) {
+  constexpr int NB = D / 64;              // 64-dim blocks per row
+  constexpr int QT = 128 / G;             // query positions per tile
+  constexpr int CH = D / 16;              // (lo, hi) chunk pairs per row: chunk c pairs dims [8c,8c+8) with [D/2+8c, ...)
+  constexpr uint32_t kIdescQK = instr_desc(128, kTileN, 0, 0);
+  constexpr uint32_t kIdescPV = instr_desc(128, D, 0, 1);
+
+  extern __shared__ unsigned char smem_dyn[];
+  // 1024-byte alignment: the swizzle pattern is a function of the address bits
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+  unsigned char* Qs = smem;
+  unsigned char* Ks = Qs + NB * kBlockBytes;
+  unsigned char* Vs = Ks + NB * kBlockBytes;
+  unsigned char* Ps = Vs + NB * kBlockBytes;
+  uint64_t* bar = reinterpret_cast<uint64_t*>(Ps + 2 * kBlockBytes);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar + 1);
+
+  const int tid = threadIdx.x, warp = tid >> 5;
+  const Item item = p.items[blockIdx.x];
+  const int b = item.b, h = item.h;
+  const int kvl = p.kv_len[b];
+  const int32_t* ids = p.page_ids + static_cast<size_t>(b) * p.table_stride;
+  const int32_t* bases = p.pos_base + static_cast<size_t>(b) * p.table_stride;
+  const int n_q_heads = p.n_kv_heads * G;
+
+  if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+  if (tid == 0) {
+    mbar_init(smem_u32(bar), 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    fence_async_smem();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const uint32_t t_row = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);   // this warp's 32 lanes
+  const uint32_t t_S = t_row, t_O = t_row + 128;
+
+  // ---- this thread's row: query position qi, head g, causal limit
+  const int r = tid;
+  const int qi = r / G, g = r % G;
+  const bool row_live = (r < QT * G) && (qi < item.nq);
+  const int last_row = item.row0 + item.nq - 1;
+  int limit = p.q_slot[row_live ? item.row0 + qi : last_row];
+  if (limit < 0 || limit >= kvl) { atomicOr(p.status, MEPIC_DEV_BAD_SLOT); limit = limit < 0 ? 0 : kvl - 1; }
+  int max_limit = p.q_slot[last_row];
+  max_limit = max_limit < 0 ? 0 : (max_limit >= kvl ? kvl - 1 : max_limit);
+  const int n_tiles = max_limit / kTileN + 1;
+
+  // ---- stage Q: rotate each row at its own position, fold in sm_scale*log2e, round to bf16
+  for (int task = tid; task < 128 * CH; task += kThreads) {
+    const int rr = task / CH, c = task % CH;
+    const int qq = rr / G, gg = rr % G;
+    uint32_t lo_w[4] = {0, 0, 0, 0}, hi_w[4] = {0, 0, 0, 0};
+    if (rr < QT * G && qq < item.nq) {
+      const int row = item.row0 + qq;
+      int slot = p.q_slot[row];
+      slot = slot < 0 ? 0 : (slot >= kvl ? kvl - 1 : slot);
+      int pos = bases[slot / p.page_size] + slot % p.page_size;
+      if (pos < 0 || pos > p.max_position) { atomicOr(p.status, MEPIC_DEV_BAD_POSITION); pos = pos < 0 ? 0 : p.max_position; }
+      const uint16_t* src = p.q_new + (static_cast<size_t>(row) * n_q_heads + static_cast<size_t>(h) * G + gg) * D;
+      const uint4 lo = *reinterpret_cast<const uint4*>(src + 8 * c);
+      const uint4 hi = *reinterpret_cast<const uint4*>(src + D / 2 + 8 * c);
+      const float4* cs = reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(pos) * D + 16 * c);
+      const uint32_t lw[4] = {lo.x, lo.y, lo.z, lo.w}, hw[4] = {hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float4 t = __ldg(cs + j);       // (cos, sin) of pairs 8c+2j and 8c+2j+1
+        const float2 a = bf16x2_to_float2(lw[j]), bq = bf16x2_to_float2(hw[j]);
+        const float l0 = (a.x * t.x - bq.x * t.y) * p.scale_log2, h0 = (a.x * t.y + bq.x * t.x) * p.scale_log2;
+        const float l1 = (a.y * t.z - bq.y * t.w) * p.scale_log2, h1 = (a.y * t.w + bq.y * t.z) * p.scale_log2;
+        lo_w[j] = pack_bf16x2(l0, l1);
+        hi_w[j] = pack_bf16x2(h0, h1);
+      }
+    }
+    // chunk index within the row: lo chunk = c, hi chunk = CH + c ; 8 chunks per 64-dim block
+    const int lc = c, hc = CH + c;
+    *reinterpret_cast<uint4*>(Qs + (lc / 8) * kBlockBytes + sw128(rr, lc % 8)) = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
+    *reinterpret_cast<uint4*>(Qs + (hc / 8) * kBlockBytes + sw128(rr, hc % 8)) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
+  }
+
+  float m_run = -INFINITY, l_run = 0.f;
+  uint32_t parity = 0;
+  bool ok = true;
+
+  for (int tile = 0; tile < n_tiles; ++tile) {
+    const int key0 = tile * kTileN;
+    // ---- stage K (rotated) and V for keys key0 .. key0+127
+    for (int task = tid; task < kTileN * CH; task += kThreads) {
+      const int kk = task / CH, c = task % CH;
+      const int kj = key0 + kk;
+      uint32_t lo_w[4] = {0, 0, 0, 0}, hi_w[4] = {0, 0, 0, 0};
+      uint4 v_lo = make_uint4(0, 0, 0, 0), v_hi = make_uint4(0, 0, 0, 0);
+      if (kj < kvl) {
+        const int e = kj / p.page_size, sl = kj % p.page_size;
+        int page = __ldg(ids + e);
+        if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
+        int pos = __ldg(bases + e) + sl;
+        if (pos < 0 || pos > p.max_position) { atomicOr(p.status, MEPIC_DEV_BAD_POSITION); pos = pos < 0 ? 0 : p.max_position; }
+        const size_t off = ((static_cast<size_t>(page) * p.n_kv_heads + h) * p.page_size + sl) * D;
+        const uint4 lo = *reinterpret_cast<const uint4*>(p.k_pool + off + 8 * c);
+        const uint4 hi = *reinterpret_cast<const uint4*>(p.k_pool + off + D / 2 + 8 * c);
+        v_lo = *reinterpret_cast<const uint4*>(p.v_pool + off + 8 * c);
+        v_hi = *reinterpret_cast<const uint4*>(p.v_pool + off + D / 2 + 8 * c);
+        const float4* cs = reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(pos) * D + 16 * c);
+        const uint32_t lw[4] = {lo.x, lo.y, lo.z, lo.w}, hw[4] = {hi.x, hi.y, hi.z, hi.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float4 t = __ldg(cs + j);
+          const float2 a = bf16x2_to_float2(lw[j]), bq = bf16x2_to_float2(hw[j]);
+          lo_w[j] = pack_bf16x2(a.x * t.x - bq.x * t.y, a.y * t.z - bq.y * t.w);
+          hi_w[j] = pack_bf16x2(a.x * t.y + bq.x * t.x, a.y * t.w + bq.y * t.z);
+        }
+      }
+      const int lc = c, hc = CH + c;
+      const uint32_t o_lo = (lc / 8) * kBlockBytes + sw128(kk, lc % 8), o_hi = (hc / 8) * kBlockBytes + sw128(kk, hc % 8);
+      *reinterpret_cast<uint4*>(Ks + o_lo) = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
+      *reinterpret_cast<uint4*>(Ks + o_hi) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
+      *reinterpret_cast<uint4*>(Vs + o_lo) = v_lo;
+      *reinterpret_cast<uint4*>(Vs + o_hi) = v_hi;
+    }
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- S = Q' K'^T
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < D / 16; ++ks) {
+        const uint32_t off = (ks / 4) * kBlockBytes + (ks % 4) * 32;
+        tc_mma(tmem_base, smem_desc(smem_u32(Qs) + off, 16, 1024), smem_desc(smem_u32(Ks) + off, 16, 1024), kIdescQK, ks > 0);
+      }
+      tc_commit(smem_u32(bar));
+    }
+    {
+      const bool landed = mbar_wait_bounded(smem_u32(bar), parity);
+      if (!landed) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
+      ok = __syncthreads_and(landed) != 0;      // leave the loop together or not at all
+    }
+    parity ^= 1u;
+    tc_fence_after();
+    if (!ok) break;
+
+    // ---- softmax of this thread's row
+    uint32_t s[128];
+    TMEM_LD32(t_S + 0, s, 0);
+    TMEM_LD32(t_S + 32, s, 32);
+    TMEM_LD32(t_S + 64, s, 64);
+    TMEM_LD32(t_S + 96, s, 96);
+    tmem_wait_ld();
+    const int n_vis = limit - key0 + 1;          // columns [0, n_vis) are visible to this row
+    float mx = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < 128; ++c) mx = fmaxf(mx, c < n_vis ? __uint_as_float(s[c]) : -INFINITY);
+    const float m_new = fmaxf(m_run, mx);
+    const float alpha = ex2(m_run - m_new);      // first tile: m_run = -inf -> 0; key 0 is visible to every row
+    float sum = 0.f;
+#pragma unroll
+    for (int cc = 0; cc < 16; ++cc) {
+      uint32_t w[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int c0 = 8 * cc + 2 * j;
+        const float p0 = c0 < n_vis ? ex2(__uint_as_float(s[c0]) - m_new) : 0.f;
+        const float p1 = c0 + 1 < n_vis ? ex2(__uint_as_float(s[c0 + 1]) - m_new) : 0.f;
+        sum += p0 + p1;
+        w[j] = pack_bf16x2(p0, p1);
+      }
+      *reinterpret_cast<uint4*>(Ps + (cc / 8) * kBlockBytes + sw128(r, cc % 8)) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    l_run = l_run * alpha + sum;
+    m_run = m_new;
+    // ---- rescale O where a row's maximum moved (warp-uniform decision; nothing to rescale on the first tile)
+    if (tile > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+      for (int cb = 0; cb < D; cb += 32) {
+        uint32_t o[32];
+        TMEM_LD32(t_O + cb, o, 0);
+        tmem_wait_ld();
+#pragma unroll
+        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+        TMEM_ST32(t_O + cb, o, 0);
+      }
+      tmem_wait_st();
+    }
+    fence_async_smem();
+    tc_fence_before();
+    __syncthreads();
+
+    // ---- O += P V
+    if (tid == 0) {
+      tc_fence_after();
+#pragma unroll
+      for (int ks = 0; ks < kTileN / 16; ++ks) {
+        const uint64_t a = smem_desc(smem_u32(Ps) + (ks / 4) * kBlockBytes + (ks % 4) * 32, 16, 1024);
+        const uint64_t bdesc = smem_desc(smem_u32(Vs) + ks * 2048, kBlockBytes, 1024);
+        tc_mma(tmem_base + 128, a, bdesc, kIdescPV, (tile > 0 || ks > 0) ? 1u : 0u);
+      }
+      tc_commit(smem_u32(bar));
+    }
+    {
+      const bool landed = mbar_wait_bounded(smem_u32(bar), parity);
+      if (!landed) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
+      ok = __syncthreads_and(landed) != 0;      // leave the loop together or not at all
+    }
+    parity ^= 1u;
+    tc_fence_after();
+    if (!ok) break;
+  }
+
+  // ---- epilogue: out = O / l
+  if (ok) {
+    const float inv = 1.f / l_run;
+    uint16_t* dst = p.out + (static_cast<size_t>(item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g) * D;
+#pragma unroll
+    for (int cb = 0; cb < D; cb += 32) {
+      uint32_t o[32];
+      TMEM_LD32(t_O + cb, o, 0);
+      tmem_wait_ld();
+      if (row_live) {
+#pragma unroll
+        for (int c = 0; c < 32; c += 8) {
+          uint4 w;
+          w.x = pack_bf16x2(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
+          w.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+          w.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+          w.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+          *reinterpret_cast<uint4*>(dst + cb + c) = w;
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
+}
+
+template <int D>
+constexpr size_t prefill_smem_bytes() { return static_cast<size_t>(3 * (D / 64) + 2) * kBlockBytes + 64 + 1024; }
+
+template <int D, int G>
+int32_t launch_prefill(const PrefillParams& p, int n_items, cudaStream_t stream) {
+  constexpr size_t smem = prefill_smem_bytes<D>();
+  cudaError_t e = cudaFuncSetAttribute(mepic_prefill_attn<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  if (e != cudaSuccess) { mepic_set_error("prefill: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
+  const int chunks_per_row = p.n_kv_heads * D / 8;
+  mepic_prefill_commit<<<p.total_rows, 128, 0, stream>>>(p, chunks_per_row);
+  mepic_prefill_attn<D, G><<<n_items, kThreads, smem, stream>>>(p);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) { mepic_set_error("prefill: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
+  mepic_count_launches(2);
+  return MEPIC_OK;
+}
+
+// Work items, heaviest first: later tiles of a request see more keys.
+bool build_items(const mepic_config_t* cfg, int batch, const int32_t* row_offsets_host, std::vector<Item>* items) {
+  const int G = cfg->n_q_heads / cfg->n_kv_heads, QT = 128 / G;
+  int max_tiles = 0;
+  for (int b = 0; b < batch; ++b) {
+    const int n = row_offsets_host[b + 1] - row_offsets_host[b];
+    if (n < 0) return false;
+    max_tiles = std::max(max_tiles, (n + QT - 1) / QT);
+  }
+  for (int t = max_tiles - 1; t >= 0; --t)
+    for (int b = 0; b < batch; ++b) {
+      const int n = row_offsets_host[b + 1] - row_offsets_host[b];
+      if (t * QT >= n) continue;
+      for (int h = 0; h < cfg->n_kv_heads; ++h)
+        items->push_back(Item{b, h, row_offsets_host[b] + t * QT, std::min(QT, n - t * QT)});
+    }
+  return true;
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" size_t mepic_attn_prefill_workspace(const mepic_config_t* cfg, int32_t batch, const int32_t* row_offsets_host) {
+  if (!mepic_config_ok(cfg) || batch < 1 || !row_offsets_host) { if (cfg) mepic_set_error("prefill_workspace: bad argument"); return 0; }
+  std::vector<Item> items;
+  if (!build_items(cfg, batch, row_offsets_host, &items)) { mepic_set_error("prefill_workspace: row_offsets must be non-decreasing"); return 0; }
+  return std::max<size_t>(items.size(), 1) * sizeof(Item);
+}
+
+extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_prefill_args_t* a, void* cuda_stream) {
+  if (!mepic_config_ok(cfg)) return MEPIC_E_INVAL;
+  if (!a || !a->q_new || !a->k_new || !a->v_new || !a->row_offsets || !a->q_slot || !a->k_pool || !a->v_pool ||
+      !a->page_ids || !a->pos_base || !a->kv_len || !a->rope_table || !a->out || !a->workspace || !a->status ||
+      !a->row_offsets_host) { mepic_set_error("prefill: NULL pointer argument"); return MEPIC_E_INVAL; }
+  if (a->batch < 1 || a->table_stride < 1) { mepic_set_error("prefill: batch and table_stride must be positive"); return MEPIC_E_INVAL; }
+  if (!aligned16(a->q_new) || !aligned16(a->k_new) || !aligned16(a->v_new) || !aligned16(a->k_pool) || !aligned16(a->v_pool) ||
+      !aligned16(a->rope_table) || !aligned16(a->out) || !aligned16(a->workspace)) {
+    mepic_set_error("prefill: pointers must be 16-byte aligned"); return MEPIC_E_INVAL;
+  }
+  if (a->row_offsets_host[0] != 0) { mepic_set_error("prefill: row_offsets[0] must be 0"); return MEPIC_E_INVAL; }
+  std::vector<Item> items;
+  if (!build_items(cfg, a->batch, a->row_offsets_host, &items)) { mepic_set_error("prefill: row_offsets must be non-decreasing"); return MEPIC_E_INVAL; }
+  const int total_rows = a->row_offsets_host[a->batch];
+  if (items.empty() || total_rows == 0) return MEPIC_OK;      // nothing to recompute
+  if (a->workspace_bytes < items.size() * sizeof(Item)) { mepic_set_error("prefill: workspace too small"); return MEPIC_E_INVAL; }
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  cudaError_t e = cudaMemcpyAsync(a->workspace, items.data(), items.size() * sizeof(Item), cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) { mepic_set_error("prefill: work list upload: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
+
+  PrefillParams p;
+  p.q_new = static_cast<const uint16_t*>(a->q_new);
+  p.k_new = static_cast<const uint16_t*>(a->k_new);
+  p.v_new = static_cast<const uint16_t*>(a->v_new);
+  p.row_offsets = a->row_offsets; p.q_slot = a->q_slot;
+  p.k_pool = static_cast<uint16_t*>(a->k_pool); p.v_pool = static_cast<uint16_t*>(a->v_pool);
+  p.page_ids = a->page_ids; p.pos_base = a->pos_base; p.kv_len = a->kv_len;
+  p.rope = a->rope_table;
+  p.out = static_cast<uint16_t*>(a->out);
+  p.items = static_cast<const Item*>(a->workspace);
+  p.status = a->status;
+  p.table_stride = a->table_stride; p.batch = a->batch; p.n_kv_heads = cfg->n_kv_heads; p.page_size = cfg->page_size;
+  p.num_pages = cfg->num_pages; p.max_position = cfg->max_position; p.total_rows = total_rows;
+  p.scale_log2 = a->sm_scale * 1.4426950408889634f;
+  const int D = cfg->head_dim, G = cfg->n_q_heads / cfg->n_kv_heads;
+  const int n_items = static_cast<int>(items.size());
+#define MEPIC_PREFILL_CASE(DD, GG) if (D == DD && G == GG) return launch_prefill<DD, GG>(p, n_items, st);
+  MEPIC_PREFILL_CASE(128, 1) MEPIC_PREFILL_CASE(128, 2) MEPIC_PREFILL_CASE(128, 4) MEPIC_PREFILL_CASE(128, 5) MEPIC_PREFILL_CASE(128, 8)
+  MEPIC_PREFILL_CASE(64, 1) MEPIC_PREFILL_CASE(64, 2) MEPIC_PREFILL_CASE(64, 4) MEPIC_PREFILL_CASE(64, 5) MEPIC_PREFILL_CASE(64, 8)
+#undef MEPIC_PREFILL_CASE
+  mepic_set_error("prefill: unsupported head_dim %d / group size %d", D, G);
   return MEPIC_E_INVAL;
 }

@@ -1,0 +1,178 @@
+"""Prefill (commit + selective-recompute attention, tcgen05) against the fp64 oracle.
+
+Outputs: max-abs <= 2e-2 and mean-abs <= 2e-3 (the stated tolerance for bf16 inputs), plus a
+tighter internal bar on the relative L2 error.  The pool after the call must equal the oracle's
+expected pool BIT FOR BIT (the commit writes un-rotated K/V bits and nothing else).
+"""
+import numpy as np
+import pytest
+import torch
+
+import paper_2512_16822_b200 as M
+from paper_2512_16822_b200 import runtime as RT
+from paper_2512_16822_b200.build import build_library
+from mepic_inputs import make_workload, f32_to_bf16_bits, bf16_bits_to_f64
+from oracle import mepic_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS, REL_L2 = 2e-2, 2e-3, 2e-2
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    build_library()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+
+
+def _check(got_bits, want, what=""):
+    got = bf16_bits_to_f64(got_bits)
+    assert np.isfinite(got).all(), what
+    d = np.abs(got - want)
+    rel = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30)
+    assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (what, d.max(), d.mean())
+    assert rel <= REL_L2, (what, rel)
+
+
+def _run_prefill(cfg, kp, vp, page_ids, pos_base, kv_len, q_slots, rows, sm_scale, theta, sample_rows=None):
+    """q_slots: list (per request) of int arrays; rows: list of PrefillRows-like (q_new, k_new, v_new)."""
+    B = len(q_slots)
+    row_offsets = np.zeros(B + 1, dtype=np.int32)
+    for b in range(B):
+        row_offsets[b + 1] = row_offsets[b] + len(q_slots[b])
+    q_slot = np.concatenate(q_slots).astype(np.int32)
+    qn = np.concatenate([r.q_new for r in rows]); kn = np.concatenate([r.k_new for r in rows])
+    vn = np.concatenate([r.v_new for r in rows])
+    dev = RT.Device(cfg, kp, vp)
+    batch = RT.PrefillBatch(dev, page_ids, pos_base, kv_len, row_offsets, q_slot, qn, kn, vn)
+    out = batch.run(sm_scale)
+    torch.cuda.synchronize()
+    assert dev.read_status() == 0
+    got = RT.bf16_bits(out)
+    got_k, got_v = RT.bf16_bits(dev.k_pool), RT.bf16_bits(dev.v_pool)
+    # oracle: commits into its own copy of the pools, request by request
+    ok, ov = kp.copy(), vp.copy()
+    P = cfg.page_size
+    for b in range(B):
+        n = -(-int(kv_len[b]) // P)
+        sel = None
+        if sample_rows is not None:
+            R = len(q_slots[b])
+            sel = sorted(set(int(x) for x in sample_rows(R) if 0 <= x < R))
+        want = O.prefill_attention_one(rows[b].q_new, rows[b].k_new, rows[b].v_new, list(q_slots[b]), ok, ov,
+                                       list(page_ids[b, :n]), list(pos_base[b, :n]), int(kv_len[b]), sm_scale, theta,
+                                       rows=sel)
+        g = got[row_offsets[b]:row_offsets[b + 1]]
+        _check(g if sel is None else g[sel], want, f"request {b}")
+    assert np.array_equal(got_k, ok) and np.array_equal(got_v, ov), "pool after commit differs from the oracle's"
+    return dev, batch
+
+
+class _Rows:
+    def __init__(self, q, k, v): self.q_new, self.k_new, self.v_new = q, k, v
+
+
+def _manual(seed, *, Hq, Hkv, D, P, specs, theta=1e4, q_std=1.0, jitter=False):
+    """specs: per request (kv_len, list_of_new_slots).  Random pages, optional jittered position bases."""
+    rng = np.random.default_rng(seed)
+    B = len(specs)
+    ents = [-(-L // P) for L, _ in specs]
+    num_pages = sum(ents) + 2
+    perm = rng.permutation(num_pages)
+    stride = max(ents) + 1
+    page_ids = np.full((B, stride), -3, dtype=np.int32); pos_base = np.zeros((B, stride), dtype=np.int32)
+    at = 0
+    for b in range(B):
+        page_ids[b, :ents[b]] = perm[at:at + ents[b]]; at += ents[b]
+        base = np.arange(ents[b]) * P
+        if jitter:
+            base = base + np.cumsum(rng.integers(0, 30, size=ents[b]))
+        pos_base[b, :ents[b]] = base
+    kv_len = np.array([L for L, _ in specs], dtype=np.int32)
+    cfg = M.Config(P, Hq, Hkv, D, num_pages, int(pos_base.max() + P), theta)
+    bits = lambda shape, std=1.0: f32_to_bf16_bits((rng.standard_normal(shape) * std).astype(np.float32))
+    kp, vp = bits((num_pages, Hkv, P, D)), bits((num_pages, Hkv, P, D))
+    q_slots = [np.asarray(s, dtype=np.int32) for _, s in specs]
+    rows = [_Rows(bits((len(s), Hq, D), q_std), bits((len(s), Hkv, D)), bits((len(s), Hkv, D))) for s in q_slots]
+    return cfg, kp, vp, page_ids, pos_base, kv_len, q_slots, rows
+
+
+def test_single_tile_and_multi_tile_small():
+    # first block + question, contexts of 1 tile and of several 128-key tiles with a ragged end
+    specs = [(100, list(range(0, 16)) + list(range(90, 100))),
+             (700, list(range(0, 16)) + list(range(256, 272)) + list(range(640, 700)))]
+    cfg, kp, vp, ids, base, kvl, slots, rows = _manual(1, Hq=8, Hkv=2, D=128, P=16, specs=specs)
+    _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 1.0 / np.sqrt(128), 1e4)
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,P", [(8, 2, 64, 16), (5, 1, 128, 16), (2, 2, 128, 64), (4, 2, 64, 32),
+                                        (8, 1, 128, 16), (10, 2, 64, 16), (4, 1, 128, 16)])
+def test_group_sizes_head_dims_page_sizes(Hq, Hkv, D, P):
+    G = Hq // Hkv
+    QT = 128 // G
+    L = 5 * 128 + 37
+    # more rows than one query tile, not a multiple of it; includes slot 0 and the last slot
+    new = sorted(set(list(range(0, P)) + list(range(2 * P * 3, 2 * P * 3 + P)) + list(range(L - QT - 7, L))))
+    specs = [(L, new), (P + 3, list(range(0, P + 3))), (300, [299])]
+    cfg, kp, vp, ids, base, kvl, slots, rows = _manual(10 + Hq + D + P, Hq=Hq, Hkv=Hkv, D=D, P=P, specs=specs, jitter=True)
+    _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 1.0 / np.sqrt(D), 1e4)
+
+
+def test_last_row_equals_decode_of_the_same_token():
+    # after the commit, the decode kernel on the request's last token must agree with the prefill row
+    specs = [(555, list(range(0, 16)) + list(range(512, 555)))]
+    cfg, kp, vp, ids, base, kvl, slots, rows = _manual(3, Hq=8, Hkv=2, D=128, P=16, specs=specs, theta=5e5)
+    dev, pb = _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 0.09, 5e5)
+    q_last = rows[0].q_new[-1:]
+    q_pos = np.array([base[0, 554 // 16] + 554 % 16], dtype=np.int32)
+    db = RT.DecodeBatch(dev, ids, base, kvl, q_pos, q_last)
+    out = db.run(0.09)
+    torch.cuda.synchronize()
+    a = bf16_bits_to_f64(RT.bf16_bits(out))[0]
+    b = bf16_bits_to_f64(RT.bf16_bits(pb.out))[-1]
+    assert np.abs(a - b).max() <= 4e-3
+
+
+def _config_run(cfg_index, scale, sample_rows):
+    wl = make_workload(cfg_index, scale=scale)
+    cfg = M.Config(wl.page_size, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.num_pages, wl.max_position,
+                   wl.rope_theta, wl.pad_token_id)
+    kp, vp = wl.kv_pool()
+    with M.Store(cfg) as st:
+        if wl.decode_requests:
+            RT.build_tables(st, wl.chunks, wl.decode_requests)        # the decode batch shares the pool
+        tables = RT.build_tables(st, wl.chunks, wl.prefill_requests)
+    page_ids, pos_base, kv_len, _ = RT.pack_tables(tables, wl.page_size)
+    q_slots = [t.recompute_slots for t in tables]
+    rows = [wl.prefill_rows(i, len(t.recompute_slots)) for i, t in enumerate(tables)]
+    _run_prefill(cfg, kp, vp, page_ids, pos_base, kv_len, q_slots, rows, wl.sm_scale, wl.rope_theta, sample_rows)
+
+
+def test_config3_scaled_all_rows():
+    _config_run(3, 0.125, None)
+
+
+def test_config3_full_sampled_rows():
+    # 8 requests x 768 rows over 16 640 cached tokens; the oracle checks sampled rows of every request
+    _config_run(3, 1.0, lambda R: [0, 1, 15, 16, 255, 256, R // 2, R - 257, R - 256, R - 2, R - 1])
+
+
+def test_config5_prefill_part_sampled_rows():
+    _config_run(5, 1.0, lambda R: [0, 15, 16, 100, R // 2, R - 1793, R - 1792, R - 1])
+
+
+def test_bad_slot_and_bad_page_are_reported_not_faulted():
+    specs = [(100, list(range(0, 16)))]
+    cfg, kp, vp, ids, base, kvl, slots, rows = _manual(5, Hq=8, Hkv=2, D=64, P=16, specs=specs)
+    bad = ids.copy(); bad[0, 3] = cfg.num_pages + 9
+    dev = RT.Device(cfg, kp, vp)
+    ro = np.array([0, 16], dtype=np.int32)
+    RT.PrefillBatch(dev, bad, base, kvl, ro, np.arange(40, 56, dtype=np.int32), rows[0].q_new, rows[0].k_new,
+                    rows[0].v_new).run(0.1)
+    torch.cuda.synchronize()
+    assert dev.read_status() & M.MEPIC_DEV_BAD_PAGE
+    dev2 = RT.Device(cfg, kp, vp)
+    RT.PrefillBatch(dev2, ids, base, kvl, ro, np.arange(90, 106, dtype=np.int32), rows[0].q_new, rows[0].k_new,
+                    rows[0].v_new).run(0.1)
+    torch.cuda.synchronize()
+    assert dev2.read_status() & M.MEPIC_DEV_BAD_SLOT
