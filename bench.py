@@ -80,9 +80,19 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def wait_first_sample(self, timeout_s: float = 5.0):
+        t0 = time.time()
+        while self.proc is not None and not self.rows and time.time() - t0 < timeout_s:
+            time.sleep(0.05)
+
+    def mark(self):
+        """Start of the region whose samples count."""
+        self.t_begin = time.time()
 
     def stop(self) -> dict:
+        t_end = time.time()
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -92,7 +102,9 @@ class ClockSampler:
             self.proc.kill()
         sm, smax, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for ts, r in self.rows:
+            if ts < getattr(self, "t_begin", 0.0) or ts > t_end + 0.2:
+                continue
             try:
                 sm.append(float(r[0])); smax.append(float(r[1]))
                 for name, val in zip(names, r[4:8]):
@@ -178,6 +190,52 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def measure_prefill(args, device_index: int):
+    """Config 3 (first-block recompute prefill): one step = one mepic_attn_prefill call (commit + attention)."""
+    import torch
+    import paper_2512_16822_b200 as M
+    from paper_2512_16822_b200 import runtime as RT
+    wl = make_workload(3)
+    cfg = M.Config(wl.page_size, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.num_pages, wl.max_position,
+                   wl.rope_theta, wl.pad_token_id)
+    kp, vp = wl.kv_pool()
+    with M.Store(cfg) as st:
+        tables = RT.build_tables(st, wl.chunks, wl.prefill_requests)
+    page_ids, pos_base, kv_len, _ = RT.pack_tables(tables, wl.page_size)
+    q_slots = [t.recompute_slots for t in tables]
+    rows = [wl.prefill_rows(i, len(t.recompute_slots)) for i, t in enumerate(tables)]
+    row_offsets = np.concatenate([[0], np.cumsum([len(s) for s in q_slots])]).astype(np.int32)
+    dev = RT.Device(cfg, kp, vp, device=f"cuda:{device_index}")
+    pb = RT.PrefillBatch(dev, page_ids, pos_base, kv_len, row_offsets, np.concatenate(q_slots).astype(np.int32),
+                         np.concatenate([r.q_new for r in rows]), np.concatenate([r.k_new for r in rows]),
+                         np.concatenate([r.v_new for r in rows]))
+    stream = torch.cuda.current_stream()
+    # unmasked (row, key) pairs only: QK^T and PV, 2 flops per multiply-add
+    pairs = sum(int((s.astype(np.int64) + 1).sum()) for s in q_slots)
+    flops = 4 * wl.head_dim * wl.n_q_heads * pairs
+    for _ in range(3):
+        pb.run(wl.sm_scale, stream)
+    torch.cuda.synchronize()
+    assert dev.read_status() == 0, "device status word is not clean"
+    steps = max(5, min(args.steps, 20))
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        a.record(stream); pb.run(wl.sm_scale, stream); b.record(stream)
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(b) for a, b in evs]
+    mean_ms = sum(ms) / len(ms)
+    _, _, peaks = measured_peaks()
+    peak = float(peaks.get("bf16_tflops", 1590.0))
+    achieved = flops / (mean_ms * 1e-3) / 1e12
+    return {"workload": f"config3:{wl.name}", "metric": "first_block_recompute_prefill_tflops", "value": achieved,
+            "unit": "TFLOP/s", "ms_per_step": mean_ms, "ms_min": min(ms), "steps": steps, "flops_per_step": flops,
+            "rows": int(row_offsets[-1]), "kv_len": int(kv_len[0]), "dtype": "bf16 MMA, fp32 accumulate",
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                         "frac": achieved / peak, "traffic": None,
+                         "peak_source": "measured burst bf16 (MEASURED_PEAKS.json bf16_tflops)" if peaks else "fallback 1590",
+                         "kernel": "mepic_prefill_attn (+ commit kernel: the C-ABI call is timed as a whole)"}}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -235,6 +293,8 @@ def run_ours(args):
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
+        sampler.wait_first_sample()
+        sampler.mark()
     launches0 = M.mepic_launch_count()
     barrier()
     ms = timed(args.steps, step, flush=True)
@@ -271,6 +331,9 @@ def run_ours(args):
         return float(t.item())
 
     tot, tot_warm, tot_e2e = agg(ms), agg(ms_warm), agg(ms_e2e)
+    prefill = None
+    if rank == 0 and world == 1 and not args.no_prefill:
+        prefill = measure_prefill(args, local_rank)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -302,6 +365,7 @@ def run_ours(args):
                   "shared": stats["pages_shared_held"], "private": stats["pages_private_held"],
                   "unshared_equivalent": stats["unshared_equivalent_pages"], "dedup_hits": stats["dedup_hits"]},
         "table_build_ms": table_build_ms,
+        "prefill": prefill,
     }
     if not args.no_cpu_baseline and world == 1:
         s = oracle_decode_sample(wl, args.cpu_budget)
@@ -319,12 +383,13 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 4, 5])
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill", action="store_true", help="skip the config-3 prefill measurement")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
