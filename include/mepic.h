@@ -214,6 +214,35 @@ typedef struct {
 size_t  mepic_attn_decode_workspace(const mepic_config_t* cfg, int32_t batch);
 int32_t mepic_attn_decode(const mepic_config_t* cfg, const mepic_decode_args_t* args, void* cuda_stream);
 
+/*
+ * mepic_attn_decode_static - the same decode, for callers that cannot allocate device memory.
+ * (The paper has no counterpart; this entry point exists for deployment reasons only.)
+ *
+ * Who needs it: code that runs where asking the device allocator for memory is not allowed or
+ * cannot succeed - inside an allocator or memory-pool callback, in a serving plug-in whose host
+ * process forbids device allocation after start-up, or when the page pool has already been given
+ * all the free device memory - and therefore cannot produce the workspace mepic_attn_decode asks
+ * for.  Here the split-KV partials go to an array built into the library instead:
+ * MEPIC_DECODE_STATIC_SCRATCH_BYTES bytes of device memory that every GPU which loads the library
+ * holds from load until the process exits.
+ *
+ * Arguments are those of mepic_attn_decode; args->workspace and args->workspace_bytes are ignored.
+ * The call allocates nothing and frees nothing, on the host's device allocator or through any
+ * library.  The first call on each device looks up the array's device address (a cheap runtime
+ * query, done once per device with that device current); make that first call outside any stream
+ * capture.  Limit: the config and batch must need no more than the array holds, i.e.
+ * mepic_attn_decode_workspace(cfg, batch) <= MEPIC_DECODE_STATIC_SCRATCH_BYTES; otherwise the call
+ * fails with MEPIC_E_INVAL and a message that states both numbers, and nothing is launched.
+ * All calls on a device share the one array, and it keeps whatever the last call left in it.  No
+ * part of it has to start at zero (every partial that is read has been written by the same call),
+ * so nothing is cleared.  Two calls whose kernels overlap on the GPU (different streams, or
+ * different threads of the process) race on the array and corrupt each other's results: serialise
+ * them, or give one of them mepic_attn_decode with its own workspace.
+ * Errors: as mepic_attn_decode, plus MEPIC_E_CUDA if the address query fails.
+ */
+#define MEPIC_DECODE_STATIC_SCRATCH_BYTES (8u << 20)
+int32_t mepic_attn_decode_static(const mepic_config_t* cfg, const mepic_decode_args_t* args, void* cuda_stream);
+
 /* ---------------------------------------------------------------- prefill (device)
  *
  * mepic_attn_prefill - Sections 3.3.1-3.3.3 for the rows a request recomputes (the first block of

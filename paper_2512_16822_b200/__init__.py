@@ -23,7 +23,8 @@ __all__ = [
     "MepicError", "Config", "Segment", "Store", "lib",
     "mepic_store_create", "mepic_store_destroy", "mepic_chunk_register", "mepic_build_block_table",
     "mepic_request_release", "mepic_store_stats", "mepic_rope_table_floats", "mepic_rope_table_fill",
-    "mepic_attn_decode_workspace", "mepic_attn_decode", "mepic_attn_prefill_workspace",
+    "mepic_attn_decode_workspace", "mepic_attn_decode", "mepic_attn_decode_static",
+    "MEPIC_DECODE_STATIC_SCRATCH_BYTES", "mepic_attn_prefill_workspace",
     "mepic_attn_prefill", "mepic_last_error", "mepic_launch_count",
     "MEPIC_OK", "MEPIC_E_INVAL", "MEPIC_E_NOSPACE", "MEPIC_E_NOTFOUND", "MEPIC_E_CAPACITY",
     "MEPIC_E_CUDA", "MEPIC_E_EXISTS", "MEPIC_SEG_CHUNK", "MEPIC_SEG_PROMPT",
@@ -38,6 +39,7 @@ MEPIC_E_CUDA = -5
 MEPIC_E_EXISTS = -6
 MEPIC_SEG_CHUNK = 0
 MEPIC_SEG_PROMPT = 1
+MEPIC_DECODE_STATIC_SCRATCH_BYTES = 8 << 20
 MEPIC_DEV_BAD_PAGE = 0x1
 MEPIC_DEV_WAIT_EXPIRED = 0x2
 MEPIC_DEV_BAD_POSITION = 0x4
@@ -125,6 +127,7 @@ _PROTOTYPES = {
     "mepic_rope_table_fill": (C.c_int32, [C.POINTER(_ConfigC), C.c_void_p]),
     "mepic_attn_decode_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32]),
     "mepic_attn_decode": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeArgsC), C.c_void_p]),
+    "mepic_attn_decode_static": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeArgsC), C.c_void_p]),
     "mepic_attn_prefill_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32, C.c_void_p]),
     "mepic_attn_prefill": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_PrefillArgsC), C.c_void_p]),
 }
@@ -309,6 +312,20 @@ def mepic_attn_decode(cfg: Config, *, q, k_pool, v_pool, page_ids, pos_base, kv_
                      table_stride, batch, sm_scale)
     c = cfg.c()
     _check(lib().mepic_attn_decode(C.byref(c), C.byref(a), _stream_ptr(stream)))
+
+
+def mepic_attn_decode_static(cfg: Config, *, q, k_pool, v_pool, page_ids, pos_base, kv_len, q_pos, rope_table, out,
+                             status, table_stride: int, batch: int, sm_scale: float, stream=None) -> None:
+    """Decode for callers that cannot allocate device memory: no workspace argument.
+
+    The split-KV partials go to a fixed array inside the library (MEPIC_DECODE_STATIC_SCRATCH_BYTES
+    per GPU) that all calls on a device share, so calls that overlap on the GPU race; sizes beyond
+    the array are refused with MEPIC_E_INVAL.  Nothing is allocated by this call.
+    """
+    a = _DecodeArgsC(_ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(page_ids), _ptr(pos_base), _ptr(kv_len),
+                     _ptr(q_pos), _ptr(rope_table), _ptr(out), None, 0, _ptr(status), table_stride, batch, sm_scale)
+    c = cfg.c()
+    _check(lib().mepic_attn_decode_static(C.byref(c), C.byref(a), _stream_ptr(stream)))
 
 
 def mepic_attn_prefill_workspace(cfg: Config, batch: int, row_offsets_host: np.ndarray) -> int:

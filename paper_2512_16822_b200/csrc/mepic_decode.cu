@@ -22,6 +22,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "mepic.h"
 #include "mepic_internal.h"
 
@@ -622,4 +624,63 @@ extern "C" int32_t mepic_attn_decode(const mepic_config_t* cfg, const mepic_deco
 #undef MEPIC_DECODE_CASE
   mepic_set_error("decode: unsupported head_dim %d / group size %d", D, G);
   return MEPIC_E_INVAL;
+}
+
+// ---------------------------------------------------------------- decode without any allocation by anyone
+//
+// Some callers cannot obtain device memory at the moment they need to decode: code running
+// inside a memory-pool or allocator callback, an inference plug-in whose host forbids calls
+// into the device allocator after start-up, a process whose device memory is fully handed to
+// the page pool.  For them the split-KV partials live in the fixed array below instead of a
+// caller-provided workspace.  Every GPU that loads this library holds the array until the
+// process exits.
+namespace {
+
+__device__ __align__(256) unsigned char g_decode_static_scratch[MEPIC_DECODE_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void* g_static_ptr[kMaxDevices] = {};   // device address of the array, per device ordinal; filled on first use
+
+// In host code the array's name is only a host-side handle, not a device address: the address a
+// kernel can use has to be asked from the runtime, once per device, with that device current.
+int32_t static_scratch_of_current_device(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) { mepic_set_error("decode_static: cudaGetDevice: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
+  if (dev < 0 || dev >= kMaxDevices) { mepic_set_error("decode_static: device ordinal %d not supported", dev); return MEPIC_E_INVAL; }
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  if (!g_static_ptr[dev]) {
+    void* ptr = nullptr;
+    e = cudaGetSymbolAddress(&ptr, g_decode_static_scratch);
+    if (e != cudaSuccess || !ptr) {
+      mepic_set_error("decode_static: cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+      return MEPIC_E_CUDA;
+    }
+    g_static_ptr[dev] = ptr;
+  }
+  *out = g_static_ptr[dev];
+  return MEPIC_OK;
+}
+
+}  // namespace
+
+extern "C" int32_t mepic_attn_decode_static(const mepic_config_t* cfg, const mepic_decode_args_t* a, void* cuda_stream) {
+  if (!mepic_config_ok(cfg)) return MEPIC_E_INVAL;
+  if (!a) { mepic_set_error("decode_static: args is NULL"); return MEPIC_E_INVAL; }
+  if (a->batch < 1) { mepic_set_error("decode_static: batch must be positive"); return MEPIC_E_INVAL; }
+  const size_t need = mepic_attn_decode_workspace(cfg, a->batch);
+  if (need == 0) return MEPIC_E_CUDA;
+  if (need > static_cast<size_t>(MEPIC_DECODE_STATIC_SCRATCH_BYTES)) {
+    mepic_set_error("decode_static: this batch and config need %zu bytes of scratch; the built-in array holds %zu "
+                    "(use mepic_attn_decode with a caller workspace)", need, static_cast<size_t>(MEPIC_DECODE_STATIC_SCRATCH_BYTES));
+    return MEPIC_E_INVAL;
+  }
+  void* scratch = nullptr;
+  const int32_t rc = static_scratch_of_current_device(&scratch);
+  if (rc != MEPIC_OK) return rc;
+  mepic_decode_args_t with_scratch = *a;
+  with_scratch.workspace = scratch;
+  with_scratch.workspace_bytes = MEPIC_DECODE_STATIC_SCRATCH_BYTES;
+  return mepic_attn_decode(cfg, &with_scratch, cuda_stream);
 }
