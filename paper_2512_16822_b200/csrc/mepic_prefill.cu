@@ -5,20 +5,30 @@
 //
 // Attention kernel.  One CTA per (request, kv head, tile of query positions).  A tile packs
 // QT = 128 / G query positions x the G query heads of the kv head into the 128 rows of one
-// tcgen05 MMA (M = 128), so that one staged K/V tile serves all G heads.  Per 128-key tile:
-//   1. the CTA reads the K rows through the block table, rotates each row at its position
-//      in fp32 registers (cos/sin from the table row of that position), rounds to bf16 and
-//      stores it into shared memory in the 128-byte-swizzled K-major layout the MMA reads;
-//      V rows are copied into the same physical layout (read by the MMA as MN-major);
-//   2. S = Q' K'^T : 8 x tcgen05.mma (128x128x16, bf16 -> fp32) into tensor memory;
-//   3. thread r owns row r: tcgen05.ld its 128 scores, causal mask by logical slot, online
-//      softmax in the log2 domain, P -> bf16 -> shared memory (K-major, swizzled); the O
-//      accumulator in tensor memory is rescaled when a row's maximum moved;
-//   4. O += P V : 8 x tcgen05.mma (128 x D x 16).
+// tcgen05 MMA (M = 128), so that one staged K/V tile serves all G heads.  The CTA is warp
+// specialised and pipelines 128-key tiles through two shared-memory stages:
+//   loader warp   : TMA (cp.async.bulk.tensor, 128-byte swizzle) brings the un-rotated K
+//                   rows and the V rows of the tile's pages straight into the layout the
+//                   MMA reads; one 16-row box per 16-token group and 64-dim half.
+//   rotator warps : rotate the K tile IN PLACE in shared memory (fp32 math, bf16 storage).
+//                   A thread walks CH consecutive keys of one 8-pair chunk and advances
+//                   (cos, sin) by one position per key with a complex multiply, starting
+//                   from the table row of its first key: 8 KB of table per tile, not 64.
+//   MMA warp      : one thread issues S = Q' K'^T (8 x tcgen05.mma 128x128x16 into one of
+//                   two S buffers in tensor memory) and O += P V (8 x 128 x D x 16), with
+//                   the next tile's QK^T issued before it waits for this tile's P.
+//   softmax warps : thread r owns row r: tcgen05.ld the scores, causal mask by logical
+//                   slot, online softmax in the log2 domain with a lazily moved reference
+//                   maximum, P -> bf16 -> shared memory; rescales O in tensor memory when
+//                   the reference moved; the epilogue writes O / l as bf16.
 // Q' carries the rotation at the row's own position and sm_scale * log2(e).
+// Every wait is bounded; a wait that runs out raises an abort flag every role checks.
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <algorithm>
+#include <mutex>
 #include <vector>
 
 #include "mepic.h"
@@ -26,11 +36,14 @@
 
 namespace {
 
-constexpr int kThreads = 128;
 constexpr int kTileN = 128;            // keys per staged tile
 constexpr int kBlockBytes = 128 * 128; // one [128 rows x 64 bf16] swizzled block
-constexpr int kTmemCols = 256;         // S: columns 0..127, O: columns 128..128+D-1
+constexpr int kTmemCols = 512;         // S0: 0..127, S1: 128..255, O: 256..256+D-1
+constexpr int kSoftmaxWarps = 4, kRotatorWarps = 4;
+constexpr int kLoaderWarp = 8, kMmaWarp = 9;
+constexpr int kThreads = 320;
 constexpr int kSpinLimit = 1 << 22;
+constexpr float kRescaleThreshold = 8.f;   // move the reference maximum only when it lags by 2^8
 
 struct Item { int32_t b, h, row0, nq; };   // rows row0 .. row0+nq-1 (global row indices) of request b
 
@@ -70,16 +83,36 @@ __device__ __forceinline__ uint32_t sw128(int row, int chunk) { return static_ca
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile("{ .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p; }"
                : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (int i = 0; i < kSpinLimit; ++i)
+// Bounded wait that also gives up when another role has raised the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  for (int i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 1023) == 1023 && *abort_flag) return false;
+  }
+  *abort_flag = 1;
+  atomicOr(status, MEPIC_DEV_WAIT_EXPIRED);
   return false;
+}
+// Same, with one verdict for the whole warp (the callers run warp-collective instructions afterwards).
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  const bool w = mbar_wait(bar, parity, abort_flag, status);
+  return __all_sync(0xffffffffu, w) != 0;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
 }
 
 // ---- tcgen05 wrappers
@@ -166,25 +199,44 @@ __global__ void mepic_prefill_commit(const PrefillParams p, int chunks_per_row) 
 }
 
 // ---------------------------------------------------------------- attention
+template <int D>
+struct PrefillSmem {
+  static constexpr int NB = D / 64;
+  static constexpr int kQ = 0;
+  static constexpr int kK = kQ + NB * kBlockBytes;          // 2 stages
+  static constexpr int kV = kK + 2 * NB * kBlockBytes;      // 2 stages
+  static constexpr int kP = kV + 2 * NB * kBlockBytes;      // 2 buffers of [128 x 128] bf16
+  static constexpr int kBars = kP + 2 * 2 * kBlockBytes;    // mbarriers and small state
+  static constexpr int kBytes = kBars + 256;
+};
+
 template <int D, int G>
-__global__ void __launch_bounds__(kThreads, 1) mepic_prefill_attn(const PrefillParams p) {
+__global__ void __launch_bounds__(kThreads, 1)
+mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
+  using L = PrefillSmem<D>;
   constexpr int NB = D / 64;              // 64-dim blocks per row
   constexpr int QT = 128 / G;             // query positions per tile
   constexpr int CH = D / 16;              // (lo, hi) chunk pairs per row: chunk c pairs dims [8c,8c+8) with [D/2+8c, ...)
   constexpr uint32_t kIdescQK = instr_desc(128, kTileN, 0, 0);
   constexpr uint32_t kIdescPV = instr_desc(128, D, 0, 1);
+  constexpr uint32_t kGroupBytes = 2u * 16u * D * 2u;   // K and V rows of one 16-token group
 
   extern __shared__ unsigned char smem_dyn[];
   // 1024-byte alignment: the swizzle pattern is a function of the address bits
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
-  unsigned char* Qs = smem;
-  unsigned char* Ks = Qs + NB * kBlockBytes;
-  unsigned char* Vs = Ks + NB * kBlockBytes;
-  unsigned char* Ps = Vs + NB * kBlockBytes;
-  uint64_t* bar = reinterpret_cast<uint64_t*>(Ps + 2 * kBlockBytes);
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar + 1);
+  unsigned char* Qs = smem + L::kQ;
+  unsigned char* Ks = smem + L::kK;
+  unsigned char* Vs = smem + L::kV;
+  unsigned char* Ps = smem + L::kP;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBars);
+  // barrier map (index): kv_landed 0,1 | k_ready 2,3 | s_full 4,5 | p_full 6,7 | pv_done 8,9
+  const uint32_t bar0 = smem_u32(bars);
+  auto BAR = [&](int which, int slot) { return bar0 + static_cast<uint32_t>((which * 2 + slot) * 8); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 11);
+  volatile int* gbase = reinterpret_cast<volatile int*>(bars + 12);     // [2][8] position of each 16-key group's first key
 
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const Item item = p.items[blockIdx.x];
   const int b = item.b, h = item.h;
   const int kvl = p.kv_len[b];
@@ -193,30 +245,25 @@ __global__ void __launch_bounds__(kThreads, 1) mepic_prefill_attn(const PrefillP
   const int n_q_heads = p.n_kv_heads * G;
 
   if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-  if (tid == 0) {
-    mbar_init(smem_u32(bar), 1);
+  if (tid == 32) {
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(BAR(0, s), 1);                       // kv_landed: loader's expect_tx + TMA bytes
+      mbar_init(BAR(1, s), kRotatorWarps * 32);      // k_ready
+      mbar_init(BAR(2, s), 1);                       // s_full: tcgen05.commit
+      mbar_init(BAR(3, s), kSoftmaxWarps * 32);      // p_full
+      mbar_init(BAR(4, s), 1);                       // pv_done: tcgen05.commit
+    }
+    *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
-  const uint32_t t_row = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);   // this warp's 32 lanes
-  const uint32_t t_S = t_row, t_O = t_row + 128;
 
-  // ---- this thread's row: query position qi, head g, causal limit
-  const int r = tid;
-  const int qi = r / G, g = r % G;
-  const bool row_live = (r < QT * G) && (qi < item.nq);
   const int last_row = item.row0 + item.nq - 1;
-  int limit = p.q_slot[row_live ? item.row0 + qi : last_row];
-  if (limit < 0 || limit >= kvl) { atomicOr(p.status, MEPIC_DEV_BAD_SLOT); limit = limit < 0 ? 0 : kvl - 1; }
   int max_limit = p.q_slot[last_row];
   max_limit = max_limit < 0 ? 0 : (max_limit >= kvl ? kvl - 1 : max_limit);
   const int n_tiles = max_limit / kTileN + 1;
 
-  // ---- stage Q: rotate each row at its own position, fold in sm_scale*log2e, round to bf16
+  // ---- stage Q (all threads): rotate each row at its own position, fold in sm_scale*log2e, round to bf16
   for (int task = tid; task < 128 * CH; task += kThreads) {
     const int rr = task / CH, c = task % CH;
     const int qq = rr / G, gg = rr % G;
@@ -247,175 +294,267 @@ __global__ void __launch_bounds__(kThreads, 1) mepic_prefill_attn(const PrefillP
     *reinterpret_cast<uint4*>(Qs + (lc / 8) * kBlockBytes + sw128(rr, lc % 8)) = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
     *reinterpret_cast<uint4*>(Qs + (hc / 8) * kBlockBytes + sw128(rr, hc % 8)) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
   }
+  fence_async_smem();          // Q is read by the tensor core (async proxy)
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
 
-  float m_run = -INFINITY, l_run = 0.f;
-  uint32_t parity = 0;
-  bool ok = true;
-
-  for (int tile = 0; tile < n_tiles; ++tile) {
-    const int key0 = tile * kTileN;
-    // ---- stage K (rotated) and V for keys key0 .. key0+127
-    for (int task = tid; task < kTileN * CH; task += kThreads) {
-      const int kk = task / CH, c = task % CH;
-      const int kj = key0 + kk;
-      uint32_t lo_w[4] = {0, 0, 0, 0}, hi_w[4] = {0, 0, 0, 0};
-      uint4 v_lo = make_uint4(0, 0, 0, 0), v_hi = make_uint4(0, 0, 0, 0);
-      if (kj < kvl) {
-        const int e = kj / p.page_size, sl = kj % p.page_size;
-        int page = __ldg(ids + e);
-        if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
-        int pos = __ldg(bases + e) + sl;
-        if (pos < 0 || pos > p.max_position) { atomicOr(p.status, MEPIC_DEV_BAD_POSITION); pos = pos < 0 ? 0 : p.max_position; }
-        const size_t off = ((static_cast<size_t>(page) * p.n_kv_heads + h) * p.page_size + sl) * D;
-        const uint4 lo = *reinterpret_cast<const uint4*>(p.k_pool + off + 8 * c);
-        const uint4 hi = *reinterpret_cast<const uint4*>(p.k_pool + off + D / 2 + 8 * c);
-        v_lo = *reinterpret_cast<const uint4*>(p.v_pool + off + 8 * c);
-        v_hi = *reinterpret_cast<const uint4*>(p.v_pool + off + D / 2 + 8 * c);
-        const float4* cs = reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(pos) * D + 16 * c);
-        const uint32_t lw[4] = {lo.x, lo.y, lo.z, lo.w}, hw[4] = {hi.x, hi.y, hi.z, hi.w};
+  if (warp < kSoftmaxWarps) {
+    // =============================================================== softmax warps: thread r = row r
+    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
+    const uint32_t t_O = t_row + 256;
+    const int r = tid;
+    const int qi = r / G, g = r % G;
+    const bool row_live = (r < QT * G) && (qi < item.nq);
+    int limit = p.q_slot[row_live ? item.row0 + qi : last_row];
+    if (limit < 0 || limit >= kvl) { atomicOr(p.status, MEPIC_DEV_BAD_SLOT); limit = limit < 0 ? 0 : kvl - 1; }
+    float m_ref = -INFINITY, l_run = 0.f;
+    bool ok = true;
+    for (int tile = 0; tile < n_tiles; ++tile) {
+      const int sb = tile & 1;
+      const uint32_t ph = static_cast<uint32_t>(tile >> 1) & 1u;
+      if (!mbar_wait_warp(BAR(2, sb), ph, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      uint32_t s[128];
+      const uint32_t t_S = t_row + static_cast<uint32_t>(sb * 128);
+      TMEM_LD32(t_S + 0, s, 0);
+      TMEM_LD32(t_S + 32, s, 32);
+      TMEM_LD32(t_S + 64, s, 64);
+      TMEM_LD32(t_S + 96, s, 96);
+      tmem_wait_ld();
+      const int n_vis = limit - tile * kTileN + 1;          // columns [0, n_vis) are visible to this row
+      float mx = -INFINITY;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float4 t = __ldg(cs + j);
-          const float2 a = bf16x2_to_float2(lw[j]), bq = bf16x2_to_float2(hw[j]);
-          lo_w[j] = pack_bf16x2(a.x * t.x - bq.x * t.y, a.y * t.z - bq.y * t.w);
-          hi_w[j] = pack_bf16x2(a.x * t.y + bq.x * t.x, a.y * t.w + bq.y * t.z);
+      for (int c = 0; c < 128; ++c) mx = fmaxf(mx, c < n_vis ? __uint_as_float(s[c]) : -INFINITY);
+      // move the reference only when it lags by more than the threshold (exponents stay below 2^8 otherwise)
+      float alpha = 1.f;
+      if (mx > m_ref + kRescaleThreshold) {       // always true on the first tile (m_ref = -inf; key 0 is visible)
+        alpha = ex2(m_ref - mx);
+        m_ref = mx;
+      }
+      float sum = 0.f;
+      uint32_t pw[64];
+#pragma unroll
+      for (int c = 0; c < 128; c += 2) {
+        const float p0 = c < n_vis ? ex2(__uint_as_float(s[c]) - m_ref) : 0.f;
+        const float p1 = c + 1 < n_vis ? ex2(__uint_as_float(s[c + 1]) - m_ref) : 0.f;
+        sum += p0 + p1;
+        pw[c / 2] = pack_bf16x2(p0, p1);
+      }
+      l_run = l_run * alpha + sum;
+      // O is stable and P buffer `sb` is free once the previous tile's PV has completed
+      if (tile > 0) {
+        const int pt = tile - 1;
+        if (!mbar_wait_warp(BAR(4, pt & 1), static_cast<uint32_t>(pt >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll
+          for (int cb = 0; cb < D; cb += 32) {
+            uint32_t o[32];
+            TMEM_LD32(t_O + cb, o, 0);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+            TMEM_ST32(t_O + cb, o, 0);
+          }
+          tmem_wait_st();
         }
       }
-      const int lc = c, hc = CH + c;
-      const uint32_t o_lo = (lc / 8) * kBlockBytes + sw128(kk, lc % 8), o_hi = (hc / 8) * kBlockBytes + sw128(kk, hc % 8);
-      *reinterpret_cast<uint4*>(Ks + o_lo) = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
-      *reinterpret_cast<uint4*>(Ks + o_hi) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
-      *reinterpret_cast<uint4*>(Vs + o_lo) = v_lo;
-      *reinterpret_cast<uint4*>(Vs + o_hi) = v_hi;
+      unsigned char* Pb = Ps + sb * 2 * kBlockBytes;
+#pragma unroll
+      for (int cc = 0; cc < 16; ++cc)
+        *reinterpret_cast<uint4*>(Pb + (cc / 8) * kBlockBytes + sw128(r, cc % 8)) =
+            make_uint4(pw[4 * cc], pw[4 * cc + 1], pw[4 * cc + 2], pw[4 * cc + 3]);
+      fence_async_smem();
+      tc_fence_before();
+      mbar_arrive(BAR(3, sb));
     }
-    fence_async_smem();
-    tc_fence_before();
-    __syncthreads();
-
-    // ---- S = Q' K'^T
-    if (tid == 0) {
+    // ---- epilogue: out = O / l once the last PV has completed
+    if (ok) {
+      const int lt = n_tiles - 1;
+      ok = mbar_wait_warp(BAR(4, lt & 1), static_cast<uint32_t>(lt >> 1) & 1u, abort_flag, p.status);
+    }
+    if (ok) {
       tc_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < D / 16; ++ks) {
-        const uint32_t off = (ks / 4) * kBlockBytes + (ks % 4) * 32;
-        tc_mma(tmem_base, smem_desc(smem_u32(Qs) + off, 16, 1024), smem_desc(smem_u32(Ks) + off, 16, 1024), kIdescQK, ks > 0);
-      }
-      tc_commit(smem_u32(bar));
-    }
-    {
-      const bool landed = mbar_wait_bounded(smem_u32(bar), parity);
-      if (!landed) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
-      ok = __syncthreads_and(landed) != 0;      // leave the loop together or not at all
-    }
-    parity ^= 1u;
-    tc_fence_after();
-    if (!ok) break;
-
-    // ---- softmax of this thread's row
-    uint32_t s[128];
-    TMEM_LD32(t_S + 0, s, 0);
-    TMEM_LD32(t_S + 32, s, 32);
-    TMEM_LD32(t_S + 64, s, 64);
-    TMEM_LD32(t_S + 96, s, 96);
-    tmem_wait_ld();
-    const int n_vis = limit - key0 + 1;          // columns [0, n_vis) are visible to this row
-    float mx = -INFINITY;
-#pragma unroll
-    for (int c = 0; c < 128; ++c) mx = fmaxf(mx, c < n_vis ? __uint_as_float(s[c]) : -INFINITY);
-    const float m_new = fmaxf(m_run, mx);
-    const float alpha = ex2(m_run - m_new);      // first tile: m_run = -inf -> 0; key 0 is visible to every row
-    float sum = 0.f;
-#pragma unroll
-    for (int cc = 0; cc < 16; ++cc) {
-      uint32_t w[4];
-#pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int c0 = 8 * cc + 2 * j;
-        const float p0 = c0 < n_vis ? ex2(__uint_as_float(s[c0]) - m_new) : 0.f;
-        const float p1 = c0 + 1 < n_vis ? ex2(__uint_as_float(s[c0 + 1]) - m_new) : 0.f;
-        sum += p0 + p1;
-        w[j] = pack_bf16x2(p0, p1);
-      }
-      *reinterpret_cast<uint4*>(Ps + (cc / 8) * kBlockBytes + sw128(r, cc % 8)) = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-    l_run = l_run * alpha + sum;
-    m_run = m_new;
-    // ---- rescale O where a row's maximum moved (warp-uniform decision; nothing to rescale on the first tile)
-    if (tile > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+      const float inv = 1.f / l_run;
+      uint16_t* dst = p.out + (static_cast<size_t>(item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g) * D;
 #pragma unroll
       for (int cb = 0; cb < D; cb += 32) {
         uint32_t o[32];
         TMEM_LD32(t_O + cb, o, 0);
         tmem_wait_ld();
+        if (row_live) {
 #pragma unroll
-        for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-        TMEM_ST32(t_O + cb, o, 0);
-      }
-      tmem_wait_st();
-    }
-    fence_async_smem();
-    tc_fence_before();
-    __syncthreads();
-
-    // ---- O += P V
-    if (tid == 0) {
-      tc_fence_after();
-#pragma unroll
-      for (int ks = 0; ks < kTileN / 16; ++ks) {
-        const uint64_t a = smem_desc(smem_u32(Ps) + (ks / 4) * kBlockBytes + (ks % 4) * 32, 16, 1024);
-        const uint64_t bdesc = smem_desc(smem_u32(Vs) + ks * 2048, kBlockBytes, 1024);
-        tc_mma(tmem_base + 128, a, bdesc, kIdescPV, (tile > 0 || ks > 0) ? 1u : 0u);
-      }
-      tc_commit(smem_u32(bar));
-    }
-    {
-      const bool landed = mbar_wait_bounded(smem_u32(bar), parity);
-      if (!landed) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
-      ok = __syncthreads_and(landed) != 0;      // leave the loop together or not at all
-    }
-    parity ^= 1u;
-    tc_fence_after();
-    if (!ok) break;
-  }
-
-  // ---- epilogue: out = O / l
-  if (ok) {
-    const float inv = 1.f / l_run;
-    uint16_t* dst = p.out + (static_cast<size_t>(item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g) * D;
-#pragma unroll
-    for (int cb = 0; cb < D; cb += 32) {
-      uint32_t o[32];
-      TMEM_LD32(t_O + cb, o, 0);
-      tmem_wait_ld();
-      if (row_live) {
-#pragma unroll
-        for (int c = 0; c < 32; c += 8) {
-          uint4 w;
-          w.x = pack_bf16x2(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
-          w.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
-          w.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
-          w.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
-          *reinterpret_cast<uint4*>(dst + cb + c) = w;
+          for (int c = 0; c < 32; c += 8) {
+            uint4 w;
+            w.x = pack_bf16x2(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
+            w.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+            w.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+            w.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+            *reinterpret_cast<uint4*>(dst + cb + c) = w;
+          }
         }
       }
     }
+  } else if (warp < kSoftmaxWarps + kRotatorWarps) {
+    // =============================================================== rotator warps: K tile, in place
+    const int rt = tid - kSoftmaxWarps * 32;     // 0..127
+    const int c = rt % CH;                       // chunk pair: dims [8c, 8c+8) and [D/2+8c, ...)
+    const int k0 = (rt / CH) * CH;               // first of this thread's CH consecutive keys
+    // one-position step of this chunk's 8 pairs: table row 1
+    float c1[8], s1[8];
+    {
+      const float4* row1 = reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(1) * D + 16 * c);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float4 t = __ldg(row1 + j);
+        c1[2 * j] = t.x; s1[2 * j] = t.y; c1[2 * j + 1] = t.z; s1[2 * j + 1] = t.w;
+      }
+    }
+    const int lc = c, hc = CH + c;
+    for (int tile = 0; tile < n_tiles; ++tile) {
+      const int st = tile & 1;
+      const uint32_t ph = static_cast<uint32_t>(tile >> 1) & 1u;
+      if (!mbar_wait(BAR(0, st), ph, abort_flag, p.status)) break;
+      unsigned char* Kb = Ks + st * NB * kBlockBytes;
+      unsigned char* Vb = Vs + st * NB * kBlockBytes;
+      const int key0 = tile * kTileN;
+      int pos = gbase[st * 8 + k0 / 16] + (k0 & 15);
+      if (pos < 0 || pos > p.max_position) {
+        if (key0 + k0 < kvl) atomicOr(p.status, MEPIC_DEV_BAD_POSITION);
+        pos = 0;
+      }
+      float cc[8], ss[8];
+      {
+        const float4* row = reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(pos) * D + 16 * c);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float4 t = __ldg(row + j);
+          cc[2 * j] = t.x; ss[2 * j] = t.y; cc[2 * j + 1] = t.z; ss[2 * j + 1] = t.w;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < CH; ++i) {
+        const int kk = k0 + i;
+        uint4* plo = reinterpret_cast<uint4*>(Kb + (lc / 8) * kBlockBytes + sw128(kk, lc % 8));
+        uint4* phi = reinterpret_cast<uint4*>(Kb + (hc / 8) * kBlockBytes + sw128(kk, hc % 8));
+        const uint4 lo = *plo, hi = *phi;
+        const uint32_t lw[4] = {lo.x, lo.y, lo.z, lo.w}, hw[4] = {hi.x, hi.y, hi.z, hi.w};
+        uint32_t lo_w[4], hi_w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const float2 a = bf16x2_to_float2(lw[j]), bq = bf16x2_to_float2(hw[j]);
+          lo_w[j] = pack_bf16x2(a.x * cc[2 * j] - bq.x * ss[2 * j], a.y * cc[2 * j + 1] - bq.y * ss[2 * j + 1]);
+          hi_w[j] = pack_bf16x2(a.x * ss[2 * j] + bq.x * cc[2 * j], a.y * ss[2 * j + 1] + bq.y * cc[2 * j + 1]);
+        }
+        *plo = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
+        *phi = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
+        if (i + 1 < CH) {
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {          // (cos, sin)(pos+1) = (cos, sin)(pos) x (cos, sin)(1)
+            const float cn = cc[j] * c1[j] - ss[j] * s1[j];
+            ss[j] = ss[j] * c1[j] + cc[j] * s1[j];
+            cc[j] = cn;
+          }
+        }
+        // rows at or past kv_len may hold anything (NaN bit patterns included): P is 0 there, V must be finite
+        if (key0 + kk >= kvl) {
+          *reinterpret_cast<uint4*>(Vb + (lc / 8) * kBlockBytes + sw128(kk, lc % 8)) = make_uint4(0, 0, 0, 0);
+          *reinterpret_cast<uint4*>(Vb + (hc / 8) * kBlockBytes + sw128(kk, hc % 8)) = make_uint4(0, 0, 0, 0);
+        }
+      }
+      fence_async_smem();
+      mbar_arrive(BAR(1, st));
+    }
+  } else if (warp == kLoaderWarp) {
+    // =============================================================== loader warp: lane g loads 16-key group g
+    for (int tile = 0; tile < n_tiles; ++tile) {
+      const int st = tile & 1;
+      if (tile >= 2) {      // stage free once the PV of the tile that used it has completed
+        const int pt = tile - 2;
+        if (!mbar_wait_warp(BAR(4, pt & 1), static_cast<uint32_t>(pt >> 1) & 1u, abort_flag, p.status)) break;
+      }
+      const int key0 = tile * kTileN;
+      const int gkey = key0 + lane * 16;
+      const bool live = lane < 8 && gkey < kvl;
+      int page = 0, pos = 0, slot0 = 0;
+      if (live) {
+        const int e = gkey / p.page_size;
+        slot0 = gkey % p.page_size;
+        page = __ldg(ids + e);
+        pos = __ldg(bases + e) + slot0;
+        if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
+      }
+      if (lane < 8) gbase[st * 8 + lane] = pos;
+      const unsigned live_mask = __ballot_sync(0xffffffffu, live);
+      __syncwarp();
+      if (lane == 0) mbar_expect_tx(BAR(0, st), static_cast<uint32_t>(__popc(live_mask)) * kGroupBytes);
+      __syncwarp();
+      if (live) {
+        const int y = (page * p.n_kv_heads + h) * p.page_size + slot0;     // row of the pool viewed as [rows][D]
+        const uint32_t kdst = smem_u32(Ks + st * NB * kBlockBytes) + static_cast<uint32_t>(lane * 16 * 128);
+        const uint32_t vdst = smem_u32(Vs + st * NB * kBlockBytes) + static_cast<uint32_t>(lane * 16 * 128);
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) {
+          tma_load_2d(kdst + nb * kBlockBytes, &map_k, nb * 64, y, BAR(0, st));
+          tma_load_2d(vdst + nb * kBlockBytes, &map_v, nb * 64, y, BAR(0, st));
+        }
+      }
+    }
+  } else if (warp == kMmaWarp && lane == 0) {
+    // =============================================================== MMA issuer (one thread)
+    const uint32_t q_addr = smem_u32(Qs);
+    for (int j = 0; j <= n_tiles; ++j) {
+      if (j < n_tiles) {
+        const int st = j & 1;
+        if (!mbar_wait(BAR(1, st), static_cast<uint32_t>(j >> 1) & 1u, abort_flag, p.status)) break;
+        tc_fence_after();
+        const uint32_t k_addr = smem_u32(Ks + st * NB * kBlockBytes);
+#pragma unroll
+        for (int ks = 0; ks < D / 16; ++ks) {
+          const uint32_t off = (ks / 4) * kBlockBytes + (ks % 4) * 32;
+          tc_mma(tmem_base + static_cast<uint32_t>(st * 128), smem_desc(q_addr + off, 16, 1024),
+                 smem_desc(k_addr + off, 16, 1024), kIdescQK, ks > 0);
+        }
+        tc_commit(BAR(2, st));
+      }
+      if (j >= 1) {
+        const int i = j - 1, st = i & 1;
+        if (!mbar_wait(BAR(3, st), static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.status)) break;
+        tc_fence_after();
+        const uint32_t p_addr = smem_u32(Ps + st * 2 * kBlockBytes);
+        const uint32_t v_addr = smem_u32(Vs + st * NB * kBlockBytes);
+#pragma unroll
+        for (int ks = 0; ks < kTileN / 16; ++ks) {
+          const uint64_t a = smem_desc(p_addr + (ks / 4) * kBlockBytes + (ks % 4) * 32, 16, 1024);
+          const uint64_t bdesc = smem_desc(v_addr + ks * 2048, kBlockBytes, 1024);
+          tc_mma(tmem_base + 256, a, bdesc, kIdescPV, (i > 0 || ks > 0) ? 1u : 0u);
+        }
+        tc_commit(BAR(4, st));
+      }
+    }
+  }
+
+  // ---- common exit: nothing of this CTA may still be in flight when tensor memory is released
+  if (warp == kLoaderWarp && *abort_flag) {
+    // a wait ran out somewhere: give outstanding TMA copies a bounded chance to land before leaving
+    for (int s = 0; s < 2; ++s)
+      for (int i = 0; i < (1 << 16) && !mbar_try_wait(BAR(0, s), 0) && !mbar_try_wait(BAR(0, s), 1); ++i) {}
   }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
 }
 
-template <int D>
-constexpr size_t prefill_smem_bytes() { return static_cast<size_t>(3 * (D / 64) + 2) * kBlockBytes + 64 + 1024; }
-
 template <int D, int G>
-int32_t launch_prefill(const PrefillParams& p, int n_items, cudaStream_t stream) {
-  constexpr size_t smem = prefill_smem_bytes<D>();
+int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
+  constexpr size_t smem = PrefillSmem<D>::kBytes + 1024;
   cudaError_t e = cudaFuncSetAttribute(mepic_prefill_attn<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("prefill: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   const int chunks_per_row = p.n_kv_heads * D / 8;
   mepic_prefill_commit<<<p.total_rows, 128, 0, stream>>>(p, chunks_per_row);
-  mepic_prefill_attn<D, G><<<n_items, kThreads, smem, stream>>>(p);
+  mepic_prefill_attn<D, G><<<n_items, kThreads, smem, stream>>>(p, map_k, map_v);
   e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("prefill: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   mepic_count_launches(2);
@@ -443,6 +582,40 @@ bool build_items(const mepic_config_t* cfg, int batch, const int32_t* row_offset
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// The driver's tensor-map encoder, looked up through the runtime so that the library links no driver stub.
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static std::mutex mu;
+  static EncodeTiledFn fn = nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  if (!fn) {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult res;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &res) == cudaSuccess &&
+        res == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  }
+  return fn;
+}
+
+// The pool seen as a 2-D bf16 tensor [num_pages * n_kv_heads * page_size rows][D]; box = 64 dims x 16 rows, 128-byte swizzle.
+int32_t make_pool_map(const mepic_config_t* cfg, void* pool, CUtensorMap* out) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) { mepic_set_error("prefill: cuTensorMapEncodeTiled is not available from the driver"); return MEPIC_E_CUDA; }
+  const cuuint64_t rows = static_cast<cuuint64_t>(cfg->num_pages) * cfg->n_kv_heads * cfg->page_size;
+  if (rows > 0x7fffffffull) { mepic_set_error("prefill: pool has too many rows for 32-bit tensor coordinates"); return MEPIC_E_INVAL; }
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cfg->head_dim), rows};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cfg->head_dim) * 2};
+  const cuuint32_t box[2] = {64, 16};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { mepic_set_error("prefill: cuTensorMapEncodeTiled failed with code %d", static_cast<int>(r)); return MEPIC_E_CUDA; }
+  return MEPIC_OK;
+}
+
 }  // namespace
 
 extern "C" size_t mepic_attn_prefill_workspace(const mepic_config_t* cfg, int32_t batch, const int32_t* row_offsets_host) {
@@ -462,12 +635,18 @@ extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_pre
       !aligned16(a->rope_table) || !aligned16(a->out) || !aligned16(a->workspace)) {
     mepic_set_error("prefill: pointers must be 16-byte aligned"); return MEPIC_E_INVAL;
   }
+  if (cfg->max_position < 16) { mepic_set_error("prefill: rope table must cover positions 0..16"); return MEPIC_E_INVAL; }
   if (a->row_offsets_host[0] != 0) { mepic_set_error("prefill: row_offsets[0] must be 0"); return MEPIC_E_INVAL; }
   std::vector<Item> items;
   if (!build_items(cfg, a->batch, a->row_offsets_host, &items)) { mepic_set_error("prefill: row_offsets must be non-decreasing"); return MEPIC_E_INVAL; }
   const int total_rows = a->row_offsets_host[a->batch];
   if (items.empty() || total_rows == 0) return MEPIC_OK;      // nothing to recompute
   if (a->workspace_bytes < items.size() * sizeof(Item)) { mepic_set_error("prefill: workspace too small"); return MEPIC_E_INVAL; }
+  alignas(64) CUtensorMap map_k, map_v;
+  int32_t rc = make_pool_map(cfg, a->k_pool, &map_k);
+  if (rc != MEPIC_OK) return rc;
+  rc = make_pool_map(cfg, a->v_pool, &map_v);
+  if (rc != MEPIC_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e = cudaMemcpyAsync(a->workspace, items.data(), items.size() * sizeof(Item), cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) { mepic_set_error("prefill: work list upload: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
@@ -488,7 +667,7 @@ extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_pre
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
   const int D = cfg->head_dim, G = cfg->n_q_heads / cfg->n_kv_heads;
   const int n_items = static_cast<int>(items.size());
-#define MEPIC_PREFILL_CASE(DD, GG) if (D == DD && G == GG) return launch_prefill<DD, GG>(p, n_items, st);
+#define MEPIC_PREFILL_CASE(DD, GG) if (D == DD && G == GG) return launch_prefill<DD, GG>(p, n_items, map_k, map_v, st);
   MEPIC_PREFILL_CASE(128, 1) MEPIC_PREFILL_CASE(128, 2) MEPIC_PREFILL_CASE(128, 4) MEPIC_PREFILL_CASE(128, 5) MEPIC_PREFILL_CASE(128, 8)
   MEPIC_PREFILL_CASE(64, 1) MEPIC_PREFILL_CASE(64, 2) MEPIC_PREFILL_CASE(64, 4) MEPIC_PREFILL_CASE(64, 5) MEPIC_PREFILL_CASE(64, 8)
 #undef MEPIC_PREFILL_CASE
