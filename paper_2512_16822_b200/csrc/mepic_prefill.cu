@@ -6,10 +6,12 @@
 // Attention kernel.  One CTA per (request, kv head, tile of query positions).  A tile packs
 // QT = 128 / G query positions x the G query heads of the kv head into the 128 rows of one
 // tcgen05 MMA (M = 128), so that one staged K/V tile serves all G heads.  The CTA is warp
-// specialised and pipelines 128-key tiles through two shared-memory stages:
-//   loader warp   : TMA (cp.async.bulk.tensor, 128-byte swizzle) brings the un-rotated K
-//                   rows and the V rows of the tile's pages straight into the layout the
-//                   MMA reads; one 16-row box per 16-token group and 64-dim half.
+// specialised and pipelines 128-key tiles through three-stage K and V rings:
+//   loader warps  : TMA (cp.async.bulk.tensor, 128-byte swizzle) brings the un-rotated K
+//                   rows (one warp) and the V rows (another) of the tile's pages straight
+//                   into the layout the MMA reads; one 16-row box per 16-token group and
+//                   64-dim half.  A K stage is reused as soon as its QK^T has completed, a
+//                   V stage once its PV has.
 //   rotator warps : rotate the K tile IN PLACE in shared memory (fp32 math, bf16 storage).
 //                   A thread walks CH consecutive keys of one 8-pair chunk and advances
 //                   (cos, sin) by one position per key with a complex multiply, starting
@@ -19,8 +21,9 @@
 //                   the next tile's QK^T issued before it waits for this tile's P.
 //   softmax warps : thread r owns row r: tcgen05.ld the scores, causal mask by logical
 //                   slot, online softmax in the log2 domain with a lazily moved reference
-//                   maximum, P -> bf16 -> shared memory; rescales O in tensor memory when
-//                   the reference moved; the epilogue writes O / l as bf16.
+//                   maximum, P -> bf16 -> tensor memory (over the first half of the tile's
+//                   S buffer, from where the PV MMA takes it as its A operand); rescales O
+//                   in tensor memory when the reference moved; the epilogue writes O / l.
 // Q' carries the rotation at the row's own position and sm_scale * log2(e).
 // Every wait is bounded; a wait that runs out raises an abort flag every role checks.
 #include <cuda.h>
@@ -40,8 +43,8 @@ constexpr int kTileN = 128;            // keys per staged tile
 constexpr int kBlockBytes = 128 * 128; // one [128 rows x 64 bf16] swizzled block
 constexpr int kTmemCols = 512;         // S0: 0..127, S1: 128..255, O: 256..256+D-1
 constexpr int kSoftmaxWarps = 4, kRotatorWarps = 4;
-constexpr int kLoaderWarp = 8, kMmaWarp = 9;
-constexpr int kThreads = 320;
+constexpr int kKLoaderWarp = 8, kVLoaderWarp = 9, kMmaWarp = 10;
+constexpr int kThreads = 352;
 constexpr int kSpinLimit = 1 << 22;
 constexpr float kRescaleThreshold = 8.f;   // move the reference maximum only when it lags by 2^8
 
@@ -134,6 +137,11 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t a_desc, uint64_
   asm volatile("{ .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p; }"
                ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// same with A taken from tensor memory (row i of A in lane i, 16-bit elements packed two per column)
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{ .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p; }"
+               ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
 // shared-memory matrix descriptor, 128-byte swizzle (layout type 2), descriptor version 1
 __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
   return static_cast<uint64_t>((addr & 0x3ffffu) >> 4) | (static_cast<uint64_t>(lbo_bytes >> 4) << 16) |
@@ -199,16 +207,26 @@ __global__ void mepic_prefill_commit(const PrefillParams p, int chunks_per_row) 
 }
 
 // ---------------------------------------------------------------- attention
+constexpr int kStages = 3;             // K ring and V ring depth
+
 template <int D>
 struct PrefillSmem {
   static constexpr int NB = D / 64;
   static constexpr int kQ = 0;
-  static constexpr int kK = kQ + NB * kBlockBytes;          // 2 stages
-  static constexpr int kV = kK + 2 * NB * kBlockBytes;      // 2 stages
-  static constexpr int kP = kV + 2 * NB * kBlockBytes;      // 2 buffers of [128 x 128] bf16
-  static constexpr int kBars = kP + 2 * 2 * kBlockBytes;    // mbarriers and small state
-  static constexpr int kBytes = kBars + 256;
+  static constexpr int kK = kQ + NB * kBlockBytes;                // kStages stages
+  static constexpr int kV = kK + kStages * NB * kBlockBytes;      // kStages stages
+  static constexpr int kBars = kV + kStages * NB * kBlockBytes;   // mbarriers and small state
+  static constexpr int kBytes = kBars + 512;
 };
+
+// barrier indices inside the barrier block
+constexpr int kBarKLanded = 0;              // [kStages] TMA bytes of a K stage
+constexpr int kBarVLanded = kBarKLanded + kStages;
+constexpr int kBarKReady = kBarVLanded + kStages;   // [kStages] K stage rotated
+constexpr int kBarSFull = kBarKReady + kStages;     // [2] QK^T of the tile complete (also: its K stage is free)
+constexpr int kBarPFull = kBarSFull + 2;            // [2] P of the tile is in tensor memory
+constexpr int kBarPvDone = kBarPFull + 2;           // [2] PV of the tile complete (its V stage is free, O is stable)
+constexpr int kNumBars = kBarPvDone + 2;
 
 template <int D, int G>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -219,7 +237,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   constexpr int CH = D / 16;              // (lo, hi) chunk pairs per row: chunk c pairs dims [8c,8c+8) with [D/2+8c, ...)
   constexpr uint32_t kIdescQK = instr_desc(128, kTileN, 0, 0);
   constexpr uint32_t kIdescPV = instr_desc(128, D, 0, 1);
-  constexpr uint32_t kGroupBytes = 2u * 16u * D * 2u;   // K and V rows of one 16-token group
+  constexpr uint32_t kGroupBytes = 16u * D * 2u;        // the rows of one 16-token group in one pool
 
   extern __shared__ unsigned char smem_dyn[];
   // 1024-byte alignment: the swizzle pattern is a function of the address bits
@@ -227,14 +245,12 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   unsigned char* Qs = smem + L::kQ;
   unsigned char* Ks = smem + L::kK;
   unsigned char* Vs = smem + L::kV;
-  unsigned char* Ps = smem + L::kP;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBars);
-  // barrier map (index): kv_landed 0,1 | k_ready 2,3 | s_full 4,5 | p_full 6,7 | pv_done 8,9
   const uint32_t bar0 = smem_u32(bars);
-  auto BAR = [&](int which, int slot) { return bar0 + static_cast<uint32_t>((which * 2 + slot) * 8); };
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 10);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 11);
-  volatile int* gbase = reinterpret_cast<volatile int*>(bars + 12);     // [2][8] position of each 16-key group's first key
+  auto BAR = [&](int which, int slot) { return bar0 + static_cast<uint32_t>((which + slot) * 8); };
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kNumBars + 1);
+  volatile int* gbase = reinterpret_cast<volatile int*>(bars + kNumBars + 2);   // [kStages][8] position of each 16-key group's first key
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const Item item = p.items[blockIdx.x];
@@ -246,12 +262,15 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
 
   if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
   if (tid == 32) {
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(BAR(kBarKLanded, s), 1);                     // loader's expect_tx + TMA bytes
+      mbar_init(BAR(kBarVLanded, s), 1);
+      mbar_init(BAR(kBarKReady, s), kRotatorWarps * 32);
+    }
     for (int s = 0; s < 2; ++s) {
-      mbar_init(BAR(0, s), 1);                       // kv_landed: loader's expect_tx + TMA bytes
-      mbar_init(BAR(1, s), kRotatorWarps * 32);      // k_ready
-      mbar_init(BAR(2, s), 1);                       // s_full: tcgen05.commit
-      mbar_init(BAR(3, s), kSoftmaxWarps * 32);      // p_full
-      mbar_init(BAR(4, s), 1);                       // pv_done: tcgen05.commit
+      mbar_init(BAR(kBarSFull, s), 1);                       // tcgen05.commit
+      mbar_init(BAR(kBarPFull, s), kSoftmaxWarps * 32);
+      mbar_init(BAR(kBarPvDone, s), 1);                      // tcgen05.commit
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -314,7 +333,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     for (int tile = 0; tile < n_tiles; ++tile) {
       const int sb = tile & 1;
       const uint32_t ph = static_cast<uint32_t>(tile >> 1) & 1u;
-      if (!mbar_wait_warp(BAR(2, sb), ph, abort_flag, p.status)) { ok = false; break; }
+      if (!mbar_wait_warp(BAR(kBarSFull, sb), ph, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
       uint32_t s[128];
       const uint32_t t_S = t_row + static_cast<uint32_t>(sb * 128);
@@ -324,56 +343,62 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       TMEM_LD32(t_S + 96, s, 96);
       tmem_wait_ld();
       const int n_vis = limit - tile * kTileN + 1;          // columns [0, n_vis) are visible to this row
-      float mx = -INFINITY;
+      if (n_vis < kTileN) {                                 // only the tile(s) on the causal boundary need the mask
 #pragma unroll
-      for (int c = 0; c < 128; ++c) mx = fmaxf(mx, c < n_vis ? __uint_as_float(s[c]) : -INFINITY);
+        for (int c = 0; c < 128; ++c) s[c] = c < n_vis ? s[c] : 0xff800000u;   // -inf
+      }
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+      for (int c = 0; c < 128; c += 4) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(mx4[k], __uint_as_float(s[c + k]));
+      }
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       // move the reference only when it lags by more than the threshold (exponents stay below 2^8 otherwise)
       float alpha = 1.f;
       if (mx > m_ref + kRescaleThreshold) {       // always true on the first tile (m_ref = -inf; key 0 is visible)
         alpha = ex2(m_ref - mx);
         m_ref = mx;
       }
-      float sum = 0.f;
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
       uint32_t pw[64];
 #pragma unroll
-      for (int c = 0; c < 128; c += 2) {
-        const float p0 = c < n_vis ? ex2(__uint_as_float(s[c]) - m_ref) : 0.f;
-        const float p1 = c + 1 < n_vis ? ex2(__uint_as_float(s[c + 1]) - m_ref) : 0.f;
-        sum += p0 + p1;
-        pw[c / 2] = pack_bf16x2(p0, p1);
-      }
-      l_run = l_run * alpha + sum;
-      // O is stable and P buffer `sb` is free once the previous tile's PV has completed
-      if (tile > 0) {
-        const int pt = tile - 1;
-        if (!mbar_wait_warp(BAR(4, pt & 1), static_cast<uint32_t>(pt >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
-        tc_fence_after();
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+      for (int c = 0; c < 128; c += 8) {
 #pragma unroll
-          for (int cb = 0; cb < D; cb += 32) {
-            uint32_t o[32];
-            TMEM_LD32(t_O + cb, o, 0);
-            tmem_wait_ld();
-#pragma unroll
-            for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-            TMEM_ST32(t_O + cb, o, 0);
-          }
-          tmem_wait_st();
+        for (int k = 0; k < 4; ++k) {
+          const float p0 = ex2(__uint_as_float(s[c + 2 * k]) - m_ref);        // 2^(-inf) = 0 for masked columns
+          const float p1 = ex2(__uint_as_float(s[c + 2 * k + 1]) - m_ref);
+          sum4[k] += p0 + p1;
+          pw[c / 2 + k] = pack_bf16x2(p0, p1);
         }
       }
-      unsigned char* Pb = Ps + sb * 2 * kBlockBytes;
+      l_run = l_run * alpha + (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+      // rescale O only when some row of this warp moved its reference; O is stable once the previous PV is complete
+      if (tile > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+        const int pt = tile - 1;
+        if (!mbar_wait_warp(BAR(kBarPvDone, pt & 1), static_cast<uint32_t>(pt >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
 #pragma unroll
-      for (int cc = 0; cc < 16; ++cc)
-        *reinterpret_cast<uint4*>(Pb + (cc / 8) * kBlockBytes + sw128(r, cc % 8)) =
-            make_uint4(pw[4 * cc], pw[4 * cc + 1], pw[4 * cc + 2], pw[4 * cc + 3]);
-      fence_async_smem();
+        for (int cb = 0; cb < D; cb += 32) {
+          uint32_t o[32];
+          TMEM_LD32(t_O + cb, o, 0);
+          tmem_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+          TMEM_ST32(t_O + cb, o, 0);
+        }
+      }
+      // P (bf16 pairs) takes the place of the first 64 columns of this tile's S buffer: the MMA reads it from there
+      TMEM_ST32(t_S + 0, pw, 0);
+      TMEM_ST32(t_S + 32, pw, 32);
+      tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(BAR(3, sb));
+      mbar_arrive(BAR(kBarPFull, sb));
     }
     // ---- epilogue: out = O / l once the last PV has completed
     if (ok) {
       const int lt = n_tiles - 1;
-      ok = mbar_wait_warp(BAR(4, lt & 1), static_cast<uint32_t>(lt >> 1) & 1u, abort_flag, p.status);
+      ok = mbar_wait_warp(BAR(kBarPvDone, lt & 1), static_cast<uint32_t>(lt >> 1) & 1u, abort_flag, p.status);
     }
     if (ok) {
       tc_fence_after();
@@ -414,11 +439,10 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     }
     const int lc = c, hc = CH + c;
     for (int tile = 0; tile < n_tiles; ++tile) {
-      const int st = tile & 1;
-      const uint32_t ph = static_cast<uint32_t>(tile >> 1) & 1u;
-      if (!mbar_wait(BAR(0, st), ph, abort_flag, p.status)) break;
+      const int st = tile % kStages;
+      const uint32_t ph = static_cast<uint32_t>(tile / kStages) & 1u;
+      if (!mbar_wait(BAR(kBarKLanded, st), ph, abort_flag, p.status)) break;
       unsigned char* Kb = Ks + st * NB * kBlockBytes;
-      unsigned char* Vb = Vs + st * NB * kBlockBytes;
       const int key0 = tile * kTileN;
       int pos = gbase[st * 8 + k0 / 16] + (k0 & 15);
       if (pos < 0 || pos > p.max_position) {
@@ -458,22 +482,36 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
             cc[j] = cn;
           }
         }
-        // rows at or past kv_len may hold anything (NaN bit patterns included): P is 0 there, V must be finite
-        if (key0 + kk >= kvl) {
-          *reinterpret_cast<uint4*>(Vb + (lc / 8) * kBlockBytes + sw128(kk, lc % 8)) = make_uint4(0, 0, 0, 0);
-          *reinterpret_cast<uint4*>(Vb + (hc / 8) * kBlockBytes + sw128(kk, hc % 8)) = make_uint4(0, 0, 0, 0);
+      }
+      // rows at or past kv_len may hold anything (NaN bit patterns included): P is 0 there, V must be finite.
+      // Only the request's last tile has such rows; its V stage must have landed before it is patched.
+      if (key0 + kTileN > kvl) {
+        if (!mbar_wait(BAR(kBarVLanded, st), ph, abort_flag, p.status)) break;
+        unsigned char* Vb = Vs + st * NB * kBlockBytes;
+#pragma unroll
+        for (int i = 0; i < CH; ++i) {
+          const int kk = k0 + i;
+          if (key0 + kk >= kvl) {
+            *reinterpret_cast<uint4*>(Vb + (lc / 8) * kBlockBytes + sw128(kk, lc % 8)) = make_uint4(0, 0, 0, 0);
+            *reinterpret_cast<uint4*>(Vb + (hc / 8) * kBlockBytes + sw128(kk, hc % 8)) = make_uint4(0, 0, 0, 0);
+          }
         }
       }
       fence_async_smem();
-      mbar_arrive(BAR(1, st));
+      mbar_arrive(BAR(kBarKReady, st));
     }
-  } else if (warp == kLoaderWarp) {
-    // =============================================================== loader warp: lane g loads 16-key group g
+  } else if (warp == kKLoaderWarp || warp == kVLoaderWarp) {
+    // =============================================================== loader warps: lane g loads 16-key group g
+    const bool is_k = warp == kKLoaderWarp;
+    const CUtensorMap* map = is_k ? &map_k : &map_v;
+    unsigned char* ring = is_k ? Ks : Vs;
     for (int tile = 0; tile < n_tiles; ++tile) {
-      const int st = tile & 1;
-      if (tile >= 2) {      // stage free once the PV of the tile that used it has completed
-        const int pt = tile - 2;
-        if (!mbar_wait_warp(BAR(4, pt & 1), static_cast<uint32_t>(pt >> 1) & 1u, abort_flag, p.status)) break;
+      const int st = tile % kStages;
+      if (tile >= kStages) {
+        // the stage is free once its previous tenant has been consumed: K by that tile's QK^T, V by its PV
+        const int pt = tile - kStages;
+        const uint32_t bar = BAR(is_k ? kBarSFull : kBarPvDone, pt & 1);
+        if (!mbar_wait_warp(bar, static_cast<uint32_t>(pt >> 1) & 1u, abort_flag, p.status)) break;
       }
       const int key0 = tile * kTileN;
       const int gkey = key0 + lane * 16;
@@ -486,20 +524,17 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         pos = __ldg(bases + e) + slot0;
         if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
       }
-      if (lane < 8) gbase[st * 8 + lane] = pos;
+      if (is_k && lane < 8) gbase[st * 8 + lane] = pos;
       const unsigned live_mask = __ballot_sync(0xffffffffu, live);
       __syncwarp();
-      if (lane == 0) mbar_expect_tx(BAR(0, st), static_cast<uint32_t>(__popc(live_mask)) * kGroupBytes);
+      const uint32_t landed = BAR(is_k ? kBarKLanded : kBarVLanded, st);
+      if (lane == 0) mbar_expect_tx(landed, static_cast<uint32_t>(__popc(live_mask)) * kGroupBytes);
       __syncwarp();
       if (live) {
         const int y = (page * p.n_kv_heads + h) * p.page_size + slot0;     // row of the pool viewed as [rows][D]
-        const uint32_t kdst = smem_u32(Ks + st * NB * kBlockBytes) + static_cast<uint32_t>(lane * 16 * 128);
-        const uint32_t vdst = smem_u32(Vs + st * NB * kBlockBytes) + static_cast<uint32_t>(lane * 16 * 128);
+        const uint32_t dst = smem_u32(ring + st * NB * kBlockBytes) + static_cast<uint32_t>(lane * 16 * 128);
 #pragma unroll
-        for (int nb = 0; nb < NB; ++nb) {
-          tma_load_2d(kdst + nb * kBlockBytes, &map_k, nb * 64, y, BAR(0, st));
-          tma_load_2d(vdst + nb * kBlockBytes, &map_v, nb * 64, y, BAR(0, st));
-        }
+        for (int nb = 0; nb < NB; ++nb) tma_load_2d(dst + nb * kBlockBytes, map, nb * 64, y, landed);
       }
     }
   } else if (warp == kMmaWarp && lane == 0) {
@@ -507,40 +542,41 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     const uint32_t q_addr = smem_u32(Qs);
     for (int j = 0; j <= n_tiles; ++j) {
       if (j < n_tiles) {
-        const int st = j & 1;
-        if (!mbar_wait(BAR(1, st), static_cast<uint32_t>(j >> 1) & 1u, abort_flag, p.status)) break;
+        const int st = j % kStages, sb = j & 1;
+        if (!mbar_wait(BAR(kBarKReady, st), static_cast<uint32_t>(j / kStages) & 1u, abort_flag, p.status)) break;
         tc_fence_after();
         const uint32_t k_addr = smem_u32(Ks + st * NB * kBlockBytes);
 #pragma unroll
         for (int ks = 0; ks < D / 16; ++ks) {
           const uint32_t off = (ks / 4) * kBlockBytes + (ks % 4) * 32;
-          tc_mma(tmem_base + static_cast<uint32_t>(st * 128), smem_desc(q_addr + off, 16, 1024),
+          tc_mma(tmem_base + static_cast<uint32_t>(sb * 128), smem_desc(q_addr + off, 16, 1024),
                  smem_desc(k_addr + off, 16, 1024), kIdescQK, ks > 0);
         }
-        tc_commit(BAR(2, st));
+        tc_commit(BAR(kBarSFull, sb));
       }
       if (j >= 1) {
-        const int i = j - 1, st = i & 1;
-        if (!mbar_wait(BAR(3, st), static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.status)) break;
+        const int i = j - 1, st = i % kStages, sb = i & 1;
+        if (!mbar_wait(BAR(kBarPFull, sb), static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.status)) break;
+        if (!mbar_wait(BAR(kBarVLanded, st), static_cast<uint32_t>(i / kStages) & 1u, abort_flag, p.status)) break;
         tc_fence_after();
-        const uint32_t p_addr = smem_u32(Ps + st * 2 * kBlockBytes);
         const uint32_t v_addr = smem_u32(Vs + st * NB * kBlockBytes);
 #pragma unroll
         for (int ks = 0; ks < kTileN / 16; ++ks) {
-          const uint64_t a = smem_desc(p_addr + (ks / 4) * kBlockBytes + (ks % 4) * 32, 16, 1024);
-          const uint64_t bdesc = smem_desc(v_addr + ks * 2048, kBlockBytes, 1024);
-          tc_mma(tmem_base + 256, a, bdesc, kIdescPV, (i > 0 || ks > 0) ? 1u : 0u);
+          // A = P from tensor memory: 16 bf16 per k-step = 8 columns; B = V, MN-major
+          tc_mma_ts(tmem_base + 256, tmem_base + static_cast<uint32_t>(sb * 128 + ks * 8),
+                    smem_desc(v_addr + ks * 2048, kBlockBytes, 1024), kIdescPV, (i > 0 || ks > 0) ? 1u : 0u);
         }
-        tc_commit(BAR(4, st));
+        tc_commit(BAR(kBarPvDone, sb));
       }
     }
   }
 
   // ---- common exit: nothing of this CTA may still be in flight when tensor memory is released
-  if (warp == kLoaderWarp && *abort_flag) {
+  if ((warp == kKLoaderWarp || warp == kVLoaderWarp) && *abort_flag) {
     // a wait ran out somewhere: give outstanding TMA copies a bounded chance to land before leaving
-    for (int s = 0; s < 2; ++s)
-      for (int i = 0; i < (1 << 16) && !mbar_try_wait(BAR(0, s), 0) && !mbar_try_wait(BAR(0, s), 1); ++i) {}
+    const int which = warp == kKLoaderWarp ? kBarKLanded : kBarVLanded;
+    for (int s = 0; s < kStages; ++s)
+      for (int i = 0; i < (1 << 16) && !mbar_try_wait(BAR(which, s), 0) && !mbar_try_wait(BAR(which, s), 1); ++i) {}
   }
   tc_fence_before();
   __syncthreads();
