@@ -3,10 +3,12 @@
 // request's paged context with RoPE applied to K on the way from the page pool to the
 // tensor cores.
 //
-// Attention kernel.  One CTA per (request, kv head, tile of query positions).  A tile packs
-// QT = 128 / G query positions x the G query heads of the kv head into the 128 rows of one
-// tcgen05 MMA (M = 128), so that one staged K/V tile serves all G heads.  The CTA is warp
-// specialised and pipelines 128-key tiles through three-stage K and V rings:
+// Attention kernel.  One CTA per (request, kv head, 2 x 128/G query positions).  An M-tile
+// packs QT = 128 / G query positions x the G query heads of the kv head into the 128 rows
+// of one tcgen05 MMA (M = 128); a CTA carries two M-tiles, so one staged and rotated K/V
+// tile serves 2 x G x QT rows and the tensor core always has the other M-tile's MMAs to
+// run while one M-tile is in its softmax.  The CTA is warp specialised and pipelines
+// 128-key tiles through a three-stage K ring and a two-stage V ring:
 //   loader warps  : TMA (cp.async.bulk.tensor, 128-byte swizzle) brings the un-rotated K
 //                   rows (one warp) and the V rows (another) of the tile's pages straight
 //                   into the layout the MMA reads; one 16-row box per 16-token group and
@@ -16,10 +18,10 @@
 //                   A thread walks CH consecutive keys of one 8-pair chunk and advances
 //                   (cos, sin) by one position per key with a complex multiply, starting
 //                   from the table row of its first key: 8 KB of table per tile, not 64.
-//   MMA warp      : one thread issues S = Q' K'^T (8 x tcgen05.mma 128x128x16 into one of
-//                   two S buffers in tensor memory) and O += P V (8 x 128 x D x 16), with
-//                   the next tile's QK^T issued before it waits for this tile's P.
-//   softmax warps : thread r owns row r: tcgen05.ld the scores, causal mask by logical
+//   MMA warp      : one thread issues, per M-tile, S = Q' K'^T (8 x tcgen05.mma 128x128x16
+//                   into tensor memory) and O += P V (8 x 128 x D x 16), alternating the
+//                   two M-tiles: PV_a(j), QK_a(j+1), PV_b(j), QK_b(j+1).
+//   softmax warps : one warpgroup per M-tile; thread r owns row r: tcgen05.ld the scores, causal mask by logical
 //                   slot, online softmax in the log2 domain with a lazily moved reference
 //                   maximum, P -> bf16 -> tensor memory (over the first half of the tile's
 //                   S buffer, from where the PV MMA takes it as its A operand); rescales O
@@ -41,10 +43,10 @@ namespace {
 
 constexpr int kTileN = 128;            // keys per staged tile
 constexpr int kBlockBytes = 128 * 128; // one [128 rows x 64 bf16] swizzled block
-constexpr int kTmemCols = 512;         // S0: 0..127, S1: 128..255, O: 256..256+D-1
+constexpr int kTmemCols = 512;         // S of M-tile a: 0..127, of b: 128..255; O of a: 256.., of b: 384..
 constexpr int kSoftmaxWarps = 4, kRotatorWarps = 4;
-constexpr int kKLoaderWarp = 8, kVLoaderWarp = 9, kMmaWarp = 10;
-constexpr int kThreads = 352;
+constexpr int kKLoaderWarp = 12, kVLoaderWarp = 13, kMmaWarp = 14;   // warp 15 idles: 16 warps keep the register split even
+constexpr int kThreads = 512;
 constexpr int kSpinLimit = 1 << 22;
 constexpr float kRescaleThreshold = 8.f;   // move the reference maximum only when it lags by 2^8
 
@@ -207,33 +209,37 @@ __global__ void mepic_prefill_commit(const PrefillParams p, int chunks_per_row) 
 }
 
 // ---------------------------------------------------------------- attention
-constexpr int kStages = 3;             // K ring and V ring depth
+constexpr int kKStages = 3;            // K ring depth (rotation runs ahead of the MMA)
+constexpr int kVStages = 2;            // V ring depth
 
 template <int D>
 struct PrefillSmem {
   static constexpr int NB = D / 64;
-  static constexpr int kQ = 0;
-  static constexpr int kK = kQ + NB * kBlockBytes;                // kStages stages
-  static constexpr int kV = kK + kStages * NB * kBlockBytes;      // kStages stages
-  static constexpr int kBars = kV + kStages * NB * kBlockBytes;   // mbarriers and small state
+  static constexpr int kQ = 0;                                     // two M-tiles of Q'
+  static constexpr int kK = kQ + 2 * NB * kBlockBytes;
+  static constexpr int kV = kK + kKStages * NB * kBlockBytes;
+  static constexpr int kBars = kV + kVStages * NB * kBlockBytes;   // mbarriers and small state
   static constexpr int kBytes = kBars + 512;
 };
 
 // barrier indices inside the barrier block
-constexpr int kBarKLanded = 0;              // [kStages] TMA bytes of a K stage
-constexpr int kBarVLanded = kBarKLanded + kStages;
-constexpr int kBarKReady = kBarVLanded + kStages;   // [kStages] K stage rotated
-constexpr int kBarSFull = kBarKReady + kStages;     // [2] QK^T of the tile complete (also: its K stage is free)
-constexpr int kBarPFull = kBarSFull + 2;            // [2] P of the tile is in tensor memory
-constexpr int kBarPvDone = kBarPFull + 2;           // [2] PV of the tile complete (its V stage is free, O is stable)
-constexpr int kNumBars = kBarPvDone + 2;
+constexpr int kBarKLanded = 0;                          // [kKStages] TMA bytes of a K stage
+constexpr int kBarKReady = kBarKLanded + kKStages;      // [kKStages] K stage rotated
+constexpr int kBarKFree = kBarKReady + kKStages;        // [kKStages] every QK^T that reads the stage is complete
+constexpr int kBarVLanded = kBarKFree + kKStages;       // [kVStages] TMA bytes of a V stage
+constexpr int kBarVFree = kBarVLanded + kVStages;       // [kVStages] every PV that reads the stage is complete
+constexpr int kBarSFull = kBarVFree + kVStages;         // [2 M-tiles] S of the current tile is in tensor memory
+constexpr int kBarPFull = kBarSFull + 2;                // [2] P of the current tile is in tensor memory
+constexpr int kBarPvDone = kBarPFull + 2;               // [2] PV of the current tile complete
+constexpr int kBarVPatched = kBarPvDone + 2;            // [1] rows past kv_len of the last V tile zeroed
+constexpr int kNumBars = kBarVPatched + 1;
 
 template <int D, int G>
 __global__ void __launch_bounds__(kThreads, 1)
 mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
   using L = PrefillSmem<D>;
   constexpr int NB = D / 64;              // 64-dim blocks per row
-  constexpr int QT = 128 / G;             // query positions per tile
+  constexpr int QT = 128 / G;             // query positions per M-tile
   constexpr int CH = D / 16;              // (lo, hi) chunk pairs per row: chunk c pairs dims [8c,8c+8) with [D/2+8c, ...)
   constexpr uint32_t kIdescQK = instr_desc(128, kTileN, 0, 0);
   constexpr uint32_t kIdescPV = instr_desc(128, D, 0, 1);
@@ -250,7 +256,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   auto BAR = [&](int which, int slot) { return bar0 + static_cast<uint32_t>((which + slot) * 8); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kNumBars + 1);
-  volatile int* gbase = reinterpret_cast<volatile int*>(bars + kNumBars + 2);   // [kStages][8] position of each 16-key group's first key
+  volatile int* gbase = reinterpret_cast<volatile int*>(bars + kNumBars + 2);   // [kKStages][8] position of each 16-key group's first key
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const Item item = p.items[blockIdx.x];
@@ -262,30 +268,45 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
 
   if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
   if (tid == 32) {
-    for (int s = 0; s < kStages; ++s) {
+    for (int s = 0; s < kKStages; ++s) {
       mbar_init(BAR(kBarKLanded, s), 1);                     // loader's expect_tx + TMA bytes
-      mbar_init(BAR(kBarVLanded, s), 1);
       mbar_init(BAR(kBarKReady, s), kRotatorWarps * 32);
+      mbar_init(BAR(kBarKFree, s), 1);                       // tcgen05.commit
+    }
+    for (int s = 0; s < kVStages; ++s) {
+      mbar_init(BAR(kBarVLanded, s), 1);
+      mbar_init(BAR(kBarVFree, s), 1);                       // tcgen05.commit
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(BAR(kBarSFull, s), 1);                       // tcgen05.commit
-      mbar_init(BAR(kBarPFull, s), kSoftmaxWarps * 32);
+      mbar_init(BAR(kBarPFull, s), 128);                     // the M-tile's softmax warpgroup
       mbar_init(BAR(kBarPvDone, s), 1);                      // tcgen05.commit
     }
+    mbar_init(BAR(kBarVPatched, 0), 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
 
-  const int last_row = item.row0 + item.nq - 1;
-  int max_limit = p.q_slot[last_row];
-  max_limit = max_limit < 0 ? 0 : (max_limit >= kvl ? kvl - 1 : max_limit);
-  const int n_tiles = max_limit / kTileN + 1;
+  // key tiles each M-tile needs: up to the causal limit of its last live row (rows ascend by slot)
+  int lim[2], nt[2];
+#pragma unroll
+  for (int x = 0; x < 2; ++x) {
+    const int last_q = min((x + 1) * QT, item.nq) - 1;            // last live position of M-tile x, or < x*QT when it has none
+    if (last_q < x * QT) { lim[x] = -1; nt[x] = 0; continue; }
+    int l = p.q_slot[item.row0 + last_q];
+    l = l < 0 ? 0 : (l >= kvl ? kvl - 1 : l);
+    lim[x] = l;
+    nt[x] = l / kTileN + 1;
+  }
+  const int n_tiles = nt[1] > nt[0] ? nt[1] : nt[0];
+  const bool last_has_tail = n_tiles * kTileN > kvl;
 
   // ---- stage Q (all threads): rotate each row at its own position, fold in sm_scale*log2e, round to bf16
-  for (int task = tid; task < 128 * CH; task += kThreads) {
-    const int rr = task / CH, c = task % CH;
-    const int qq = rr / G, gg = rr % G;
+  for (int task = tid; task < 256 * CH; task += kThreads) {
+    const int rr2 = task / CH, c = task % CH;
+    const int x = rr2 >> 7, rr = rr2 & 127;
+    const int qq = x * QT + rr / G, gg = rr % G;
     uint32_t lo_w[4] = {0, 0, 0, 0}, hi_w[4] = {0, 0, 0, 0};
     if (rr < QT * G && qq < item.nq) {
       const int row = item.row0 + qq;
@@ -310,8 +331,9 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     }
     // chunk index within the row: lo chunk = c, hi chunk = CH + c ; 8 chunks per 64-dim block
     const int lc = c, hc = CH + c;
-    *reinterpret_cast<uint4*>(Qs + (lc / 8) * kBlockBytes + sw128(rr, lc % 8)) = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
-    *reinterpret_cast<uint4*>(Qs + (hc / 8) * kBlockBytes + sw128(rr, hc % 8)) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
+    unsigned char* Qx = Qs + x * NB * kBlockBytes;
+    *reinterpret_cast<uint4*>(Qx + (lc / 8) * kBlockBytes + sw128(rr, lc % 8)) = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
+    *reinterpret_cast<uint4*>(Qx + (hc / 8) * kBlockBytes + sw128(rr, hc % 8)) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
   }
   fence_async_smem();          // Q is read by the tensor core (async proxy)
   tc_fence_before();
@@ -319,39 +341,44 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp < kSoftmaxWarps) {
-    // =============================================================== softmax warps: thread r = row r
-    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(warp * 32) << 16);
-    const uint32_t t_O = t_row + 256;
-    const int r = tid;
-    const int qi = r / G, g = r % G;
+  if (warp < 2 * kSoftmaxWarps) {
+    // =============================================================== softmax warpgroups: one per M-tile, thread = row
+    const int x = warp / kSoftmaxWarps;
+    const uint32_t t_row = tmem_base + (static_cast<uint32_t>((warp % 4) * 32) << 16);
+    const uint32_t t_S = t_row + static_cast<uint32_t>(x * 128);       // S of this M-tile; P overwrites its first 64 columns
+    const uint32_t t_O = t_row + 256u + static_cast<uint32_t>(x * 128);
+    const int r = tid & 127;
+    const int qi = x * QT + r / G, g = r % G;
     const bool row_live = (r < QT * G) && (qi < item.nq);
-    int limit = p.q_slot[row_live ? item.row0 + qi : last_row];
-    if (limit < 0 || limit >= kvl) { atomicOr(p.status, MEPIC_DEV_BAD_SLOT); limit = limit < 0 ? 0 : kvl - 1; }
+    int limit = lim[x];
+    if (row_live) {
+      limit = p.q_slot[item.row0 + qi];
+      if (limit < 0 || limit >= kvl) { atomicOr(p.status, MEPIC_DEV_BAD_SLOT); limit = limit < 0 ? 0 : kvl - 1; }
+    }
     float m_ref = -INFINITY, l_run = 0.f;
     bool ok = true;
-    for (int tile = 0; tile < n_tiles; ++tile) {
-      const int sb = tile & 1;
-      const uint32_t ph = static_cast<uint32_t>(tile >> 1) & 1u;
-      if (!mbar_wait_warp(BAR(kBarSFull, sb), ph, abort_flag, p.status)) { ok = false; break; }
+    const int my_tiles = nt[x];
+    for (int tile = 0; tile < my_tiles; ++tile) {
+      if (!mbar_wait_warp(BAR(kBarSFull, x), static_cast<uint32_t>(tile) & 1u, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
-      uint32_t s[128];
-      const uint32_t t_S = t_row + static_cast<uint32_t>(sb * 128);
-      TMEM_LD32(t_S + 0, s, 0);
-      TMEM_LD32(t_S + 32, s, 32);
-      TMEM_LD32(t_S + 64, s, 64);
-      TMEM_LD32(t_S + 96, s, 96);
-      tmem_wait_ld();
       const int n_vis = limit - tile * kTileN + 1;          // columns [0, n_vis) are visible to this row
-      if (n_vis < kTileN) {                                 // only the tile(s) on the causal boundary need the mask
-#pragma unroll
-        for (int c = 0; c < 128; ++c) s[c] = c < n_vis ? s[c] : 0xff800000u;   // -inf
-      }
+      const bool boundary = n_vis < kTileN;                 // only the tile(s) on the causal boundary need the mask
+      // ---- pass 1: row maximum
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-      for (int c = 0; c < 128; c += 4) {
+      for (int q = 0; q < 4; ++q) {
+        uint32_t s[32];
+        TMEM_LD32(t_S + 32 * q, s, 0);
+        tmem_wait_ld();
+        if (boundary) {
 #pragma unroll
-        for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(mx4[k], __uint_as_float(s[c + k]));
+          for (int c = 0; c < 32; ++c) s[c] = (32 * q + c) < n_vis ? s[c] : 0xff800000u;   // -inf
+        }
+#pragma unroll
+        for (int c = 0; c < 32; c += 4) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(mx4[k], __uint_as_float(s[c + k]));
+        }
       }
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
       // move the reference only when it lags by more than the threshold (exponents stay below 2^8 otherwise)
@@ -360,24 +387,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         alpha = ex2(m_ref - mx);
         m_ref = mx;
       }
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
-      uint32_t pw[64];
-#pragma unroll
-      for (int c = 0; c < 128; c += 8) {
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float p0 = ex2(__uint_as_float(s[c + 2 * k]) - m_ref);        // 2^(-inf) = 0 for masked columns
-          const float p1 = ex2(__uint_as_float(s[c + 2 * k + 1]) - m_ref);
-          sum4[k] += p0 + p1;
-          pw[c / 2 + k] = pack_bf16x2(p0, p1);
-        }
-      }
-      l_run = l_run * alpha + (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
-      // rescale O only when some row of this warp moved its reference; O is stable once the previous PV is complete
+      // O needs no wait: this tile's S exists, so the previous tile's PV (issued before it) has completed
       if (tile > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
-        const int pt = tile - 1;
-        if (!mbar_wait_warp(BAR(kBarPvDone, pt & 1), static_cast<uint32_t>(pt >> 1) & 1u, abort_flag, p.status)) { ok = false; break; }
-        tc_fence_after();
 #pragma unroll
         for (int cb = 0; cb < D; cb += 32) {
           uint32_t o[32];
@@ -388,43 +399,68 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
           TMEM_ST32(t_O + cb, o, 0);
         }
       }
-      // P (bf16 pairs) takes the place of the first 64 columns of this tile's S buffer: the MMA reads it from there
-      TMEM_ST32(t_S + 0, pw, 0);
-      TMEM_ST32(t_S + 32, pw, 32);
-      tmem_wait_st();
-      tc_fence_before();
-      mbar_arrive(BAR(kBarPFull, sb));
-    }
-    // ---- epilogue: out = O / l once the last PV has completed
-    if (ok) {
-      const int lt = n_tiles - 1;
-      ok = mbar_wait_warp(BAR(kBarPvDone, lt & 1), static_cast<uint32_t>(lt >> 1) & 1u, abort_flag, p.status);
-    }
-    if (ok) {
-      tc_fence_after();
-      const float inv = 1.f / l_run;
-      uint16_t* dst = p.out + (static_cast<size_t>(item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g) * D;
+      // ---- pass 2: P = 2^(S - reference) as bf16 pairs, written over the first 64 columns of S
+      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int cb = 0; cb < D; cb += 32) {
-        uint32_t o[32];
-        TMEM_LD32(t_O + cb, o, 0);
-        tmem_wait_ld();
-        if (row_live) {
+      for (int half = 0; half < 2; ++half) {
+        uint32_t pw[32];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+          uint32_t s[32];
+          const int col0 = 64 * half + 32 * q;
+          TMEM_LD32(t_S + col0, s, 0);
+          tmem_wait_ld();
+          if (boundary) {
+#pragma unroll
+            for (int c = 0; c < 32; ++c) s[c] = (col0 + c) < n_vis ? s[c] : 0xff800000u;
+          }
 #pragma unroll
           for (int c = 0; c < 32; c += 8) {
-            uint4 w;
-            w.x = pack_bf16x2(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
-            w.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
-            w.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
-            w.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
-            *reinterpret_cast<uint4*>(dst + cb + c) = w;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+              const float p0 = ex2(__uint_as_float(s[c + 2 * k]) - m_ref);        // 2^(-inf) = 0 for masked columns
+              const float p1 = ex2(__uint_as_float(s[c + 2 * k + 1]) - m_ref);
+              sum4[k] += p0 + p1;
+              pw[16 * q + c / 2 + k] = pack_bf16x2(p0, p1);
+            }
+          }
+        }
+        TMEM_ST32(t_S + 32 * half, pw, 0);
+      }
+      l_run = l_run * alpha + (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+      tmem_wait_st();
+      tc_fence_before();
+      mbar_arrive(BAR(kBarPFull, x));
+    }
+    // ---- epilogue: out = O / l once the last PV has completed
+    if (ok && my_tiles > 0) {
+      ok = mbar_wait_warp(BAR(kBarPvDone, x), static_cast<uint32_t>(my_tiles - 1) & 1u, abort_flag, p.status);
+      if (ok) {
+        tc_fence_after();
+        const float inv = 1.f / l_run;
+        uint16_t* dst = p.out + (static_cast<size_t>(item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g) * D;
+#pragma unroll
+        for (int cb = 0; cb < D; cb += 32) {
+          uint32_t o[32];
+          TMEM_LD32(t_O + cb, o, 0);
+          tmem_wait_ld();
+          if (row_live) {
+#pragma unroll
+            for (int c = 0; c < 32; c += 8) {
+              uint4 w;
+              w.x = pack_bf16x2(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
+              w.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+              w.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+              w.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+              *reinterpret_cast<uint4*>(dst + cb + c) = w;
+            }
           }
         }
       }
     }
-  } else if (warp < kSoftmaxWarps + kRotatorWarps) {
+  } else if (warp < 2 * kSoftmaxWarps + kRotatorWarps) {
     // =============================================================== rotator warps: K tile, in place
-    const int rt = tid - kSoftmaxWarps * 32;     // 0..127
+    const int rt = tid - 2 * kSoftmaxWarps * 32;     // 0..127
     const int c = rt % CH;                       // chunk pair: dims [8c, 8c+8) and [D/2+8c, ...)
     const int k0 = (rt / CH) * CH;               // first of this thread's CH consecutive keys
     // one-position step of this chunk's 8 pairs: table row 1
@@ -439,8 +475,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     }
     const int lc = c, hc = CH + c;
     for (int tile = 0; tile < n_tiles; ++tile) {
-      const int st = tile % kStages;
-      const uint32_t ph = static_cast<uint32_t>(tile / kStages) & 1u;
+      const int st = tile % kKStages;
+      const uint32_t ph = static_cast<uint32_t>(tile / kKStages) & 1u;
       if (!mbar_wait(BAR(kBarKLanded, st), ph, abort_flag, p.status)) break;
       unsigned char* Kb = Ks + st * NB * kBlockBytes;
       const int key0 = tile * kTileN;
@@ -483,20 +519,6 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
           }
         }
       }
-      // rows at or past kv_len may hold anything (NaN bit patterns included): P is 0 there, V must be finite.
-      // Only the request's last tile has such rows; its V stage must have landed before it is patched.
-      if (key0 + kTileN > kvl) {
-        if (!mbar_wait(BAR(kBarVLanded, st), ph, abort_flag, p.status)) break;
-        unsigned char* Vb = Vs + st * NB * kBlockBytes;
-#pragma unroll
-        for (int i = 0; i < CH; ++i) {
-          const int kk = k0 + i;
-          if (key0 + kk >= kvl) {
-            *reinterpret_cast<uint4*>(Vb + (lc / 8) * kBlockBytes + sw128(kk, lc % 8)) = make_uint4(0, 0, 0, 0);
-            *reinterpret_cast<uint4*>(Vb + (hc / 8) * kBlockBytes + sw128(kk, hc % 8)) = make_uint4(0, 0, 0, 0);
-          }
-        }
-      }
       fence_async_smem();
       mbar_arrive(BAR(kBarKReady, st));
     }
@@ -505,13 +527,14 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     const bool is_k = warp == kKLoaderWarp;
     const CUtensorMap* map = is_k ? &map_k : &map_v;
     unsigned char* ring = is_k ? Ks : Vs;
+    const int depth = is_k ? kKStages : kVStages;
+    bool ok = true;
     for (int tile = 0; tile < n_tiles; ++tile) {
-      const int st = tile % kStages;
-      if (tile >= kStages) {
-        // the stage is free once its previous tenant has been consumed: K by that tile's QK^T, V by its PV
-        const int pt = tile - kStages;
-        const uint32_t bar = BAR(is_k ? kBarSFull : kBarPvDone, pt & 1);
-        if (!mbar_wait_warp(bar, static_cast<uint32_t>(pt >> 1) & 1u, abort_flag, p.status)) break;
+      const int st = tile % depth;
+      if (tile >= depth) {
+        // the stage is free once every MMA that reads its previous tenant has completed
+        const uint32_t bar = BAR(is_k ? kBarKFree : kBarVFree, st);
+        if (!mbar_wait_warp(bar, static_cast<uint32_t>(tile / depth - 1) & 1u, abort_flag, p.status)) { ok = false; break; }
       }
       const int key0 = tile * kTileN;
       const int gkey = key0 + lane * 16;
@@ -537,36 +560,90 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         for (int nb = 0; nb < NB; ++nb) tma_load_2d(dst + nb * kBlockBytes, map, nb * 64, y, landed);
       }
     }
+    // Rows at or past kv_len of the last V tile may hold anything (NaN bit patterns included): P is 0 there,
+    // but 0 x NaN is NaN, so V must be finite.  Zero them once the tile has landed.
+    if (!is_k && ok && last_has_tail) {
+      const int lt = n_tiles - 1, st = lt % kVStages;
+      if (mbar_wait_warp(BAR(kBarVLanded, st), static_cast<uint32_t>(lt / kVStages) & 1u, abort_flag, p.status)) {
+        unsigned char* Vb = Vs + st * NB * kBlockBytes;
+        const int first = kvl - lt * kTileN;       // first row to clear (0 < first < 128)
+        for (int idx = first * 2 * CH + lane; idx < kTileN * 2 * CH; idx += 32) {
+          const int kk = idx / (2 * CH), ch = idx % (2 * CH);
+          *reinterpret_cast<uint4*>(Vb + (ch / 8) * kBlockBytes + sw128(kk, ch % 8)) = make_uint4(0, 0, 0, 0);
+        }
+        fence_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(BAR(kBarVPatched, 0));
+      }
+    }
   } else if (warp == kMmaWarp && lane == 0) {
     // =============================================================== MMA issuer (one thread)
-    const uint32_t q_addr = smem_u32(Qs);
-    for (int j = 0; j <= n_tiles; ++j) {
-      if (j < n_tiles) {
-        const int st = j % kStages, sb = j & 1;
-        if (!mbar_wait(BAR(kBarKReady, st), static_cast<uint32_t>(j / kStages) & 1u, abort_flag, p.status)) break;
-        tc_fence_after();
-        const uint32_t k_addr = smem_u32(Ks + st * NB * kBlockBytes);
+    // Order per key tile j:  PV_a(j), QK_a(j+1), PV_b(j), QK_b(j+1): while one M-tile's softmax runs, the
+    // tensor core works on the other M-tile.  S of an M-tile is reused by its P, so QK_x(j+1) follows PV_x(j).
+    const uint32_t q_addr[2] = {smem_u32(Qs), smem_u32(Qs + NB * kBlockBytes)};
+    bool ok = true;
+    auto issue_qk = [&](int x, int j) {
+      const uint32_t k_addr = smem_u32(Ks + (j % kKStages) * NB * kBlockBytes);
 #pragma unroll
-        for (int ks = 0; ks < D / 16; ++ks) {
-          const uint32_t off = (ks / 4) * kBlockBytes + (ks % 4) * 32;
-          tc_mma(tmem_base + static_cast<uint32_t>(sb * 128), smem_desc(q_addr + off, 16, 1024),
-                 smem_desc(k_addr + off, 16, 1024), kIdescQK, ks > 0);
-        }
-        tc_commit(BAR(kBarSFull, sb));
+      for (int ks = 0; ks < D / 16; ++ks) {
+        const uint32_t off = (ks / 4) * kBlockBytes + (ks % 4) * 32;
+        tc_mma(tmem_base + static_cast<uint32_t>(x * 128), smem_desc(q_addr[x] + off, 16, 1024),
+               smem_desc(k_addr + off, 16, 1024), kIdescQK, ks > 0);
       }
-      if (j >= 1) {
-        const int i = j - 1, st = i % kStages, sb = i & 1;
-        if (!mbar_wait(BAR(kBarPFull, sb), static_cast<uint32_t>(i >> 1) & 1u, abort_flag, p.status)) break;
-        if (!mbar_wait(BAR(kBarVLanded, st), static_cast<uint32_t>(i / kStages) & 1u, abort_flag, p.status)) break;
-        tc_fence_after();
-        const uint32_t v_addr = smem_u32(Vs + st * NB * kBlockBytes);
+      tc_commit(BAR(kBarSFull, x));
+    };
+    auto issue_pv = [&](int x, int j) {
+      const uint32_t v_addr = smem_u32(Vs + (j % kVStages) * NB * kBlockBytes);
 #pragma unroll
-        for (int ks = 0; ks < kTileN / 16; ++ks) {
-          // A = P from tensor memory: 16 bf16 per k-step = 8 columns; B = V, MN-major
-          tc_mma_ts(tmem_base + 256, tmem_base + static_cast<uint32_t>(sb * 128 + ks * 8),
-                    smem_desc(v_addr + ks * 2048, kBlockBytes, 1024), kIdescPV, (i > 0 || ks > 0) ? 1u : 0u);
-        }
-        tc_commit(BAR(kBarPvDone, sb));
+      for (int ks = 0; ks < kTileN / 16; ++ks) {
+        // A = P from tensor memory: 16 bf16 per k-step = 8 columns; B = V, MN-major
+        tc_mma_ts(tmem_base + 256u + static_cast<uint32_t>(x * 128), tmem_base + static_cast<uint32_t>(x * 128 + ks * 8),
+                  smem_desc(v_addr + ks * 2048, kBlockBytes, 1024), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+      }
+      tc_commit(BAR(kBarPvDone, x));
+    };
+    auto wait_k = [&](int j) {
+      const bool w = mbar_wait(BAR(kBarKReady, j % kKStages), static_cast<uint32_t>(j / kKStages) & 1u, abort_flag, p.status);
+      tc_fence_after();
+      return w;
+    };
+    // prologue: S of key tile 0 for both M-tiles
+    ok = wait_k(0);
+    if (ok) {
+      if (nt[0] > 0) issue_qk(0, 0);
+      if (nt[1] > 0) issue_qk(1, 0);
+      tc_commit(BAR(kBarKFree, 0));
+    }
+    for (int j = 0; j < n_tiles && ok; ++j) {
+      bool v_here = false;
+      auto wait_v = [&]() {
+        if (v_here) return true;
+        bool w = mbar_wait(BAR(kBarVLanded, j % kVStages), static_cast<uint32_t>(j / kVStages) & 1u, abort_flag, p.status);
+        if (w && j == n_tiles - 1 && last_has_tail) w = mbar_wait(BAR(kBarVPatched, 0), 0, abort_flag, p.status);
+        v_here = w;
+        return w;
+      };
+      const bool more = j + 1 < n_tiles;
+      // ---- M-tile a
+      if (j < nt[0]) {
+        if (!mbar_wait(BAR(kBarPFull, 0), static_cast<uint32_t>(j) & 1u, abort_flag, p.status) || !wait_v()) { ok = false; break; }
+        tc_fence_after();
+        issue_pv(0, j);
+      }
+      if (more) {
+        if (!wait_k(j + 1)) { ok = false; break; }
+        if (j + 1 < nt[0]) issue_qk(0, j + 1);
+      }
+      // ---- M-tile b
+      if (j < nt[1]) {
+        if (!mbar_wait(BAR(kBarPFull, 1), static_cast<uint32_t>(j) & 1u, abort_flag, p.status) || !wait_v()) { ok = false; break; }
+        tc_fence_after();
+        issue_pv(1, j);
+      }
+      tc_commit(BAR(kBarVFree, j % kVStages));
+      if (more) {
+        if (j + 1 < nt[1]) issue_qk(1, j + 1);
+        tc_commit(BAR(kBarKFree, (j + 1) % kKStages));
       }
     }
   }
@@ -575,7 +652,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   if ((warp == kKLoaderWarp || warp == kVLoaderWarp) && *abort_flag) {
     // a wait ran out somewhere: give outstanding TMA copies a bounded chance to land before leaving
     const int which = warp == kKLoaderWarp ? kBarKLanded : kBarVLanded;
-    for (int s = 0; s < kStages; ++s)
+    const int depth = warp == kKLoaderWarp ? kKStages : kVStages;
+    for (int s = 0; s < depth; ++s)
       for (int i = 0; i < (1 << 16) && !mbar_try_wait(BAR(which, s), 0) && !mbar_try_wait(BAR(which, s), 1); ++i) {}
   }
   tc_fence_before();
@@ -599,7 +677,7 @@ int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& m
 
 // Work items, heaviest first: later tiles of a request see more keys.
 bool build_items(const mepic_config_t* cfg, int batch, const int32_t* row_offsets_host, std::vector<Item>* items) {
-  const int G = cfg->n_q_heads / cfg->n_kv_heads, QT = 128 / G;
+  const int G = cfg->n_q_heads / cfg->n_kv_heads, QT = 2 * (128 / G);   // two M-tiles of query positions per CTA
   int max_tiles = 0;
   for (int b = 0; b < batch; ++b) {
     const int n = row_offsets_host[b + 1] - row_offsets_host[b];
