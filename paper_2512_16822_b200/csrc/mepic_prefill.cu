@@ -76,6 +76,32 @@ __device__ __forceinline__ float ex2(float x) { float y; asm("ex2.approx.ftz.f32
 __device__ __forceinline__ float2 bf16x2_to_float2(uint32_t w) {
   return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
 }
+// packed fp32 pairs (one instruction for two lanes of work)
+__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
+  float2 d;
+  asm("{ .reg .b64 ra, rb, rc, rd;\n mov.b64 ra, {%2,%3};\n mov.b64 rb, {%4,%5};\n mov.b64 rc, {%6,%7};\n"
+      " fma.rn.f32x2 rd, ra, rb, rc;\n mov.b64 {%0,%1}, rd; }"
+      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+  return d;
+}
+__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
+  float2 d;
+  asm("{ .reg .b64 ra, rb, rd;\n mov.b64 ra, {%2,%3};\n mov.b64 rb, {%4,%5};\n mul.rn.f32x2 rd, ra, rb;\n mov.b64 {%0,%1}, rd; }"
+      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+__device__ __forceinline__ float2 sub2(float2 a, float2 b) {
+  float2 d;
+  asm("{ .reg .b64 ra, rb, rd;\n mov.b64 ra, {%2,%3};\n mov.b64 rb, {%4,%5};\n sub.rn.f32x2 rd, ra, rb;\n mov.b64 {%0,%1}, rd; }"
+      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
+__device__ __forceinline__ float2 add2(float2 a, float2 b) {
+  float2 d;
+  asm("{ .reg .b64 ra, rb, rd;\n mov.b64 ra, {%2,%3};\n mov.b64 rb, {%4,%5};\n add.rn.f32x2 rd, ra, rb;\n mov.b64 {%0,%1}, rd; }"
+      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+  return d;
+}
 // (lo, hi) -> packed bf16x2, round to nearest even
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
@@ -178,6 +204,11 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int a_mn_major, 
                  "r"(r[o + 18]), "r"(r[o + 19]), "r"(r[o + 20]), "r"(r[o + 21]), "r"(r[o + 22]), "r"(r[o + 23]),     \
                  "r"(r[o + 24]), "r"(r[o + 25]), "r"(r[o + 26]), "r"(r[o + 27]), "r"(r[o + 28]), "r"(r[o + 29]),     \
                  "r"(r[o + 30]), "r"(r[o + 31]) : "memory")
+
+#define TMEM_ST16(taddr, r)                                                                                          \
+  asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" \
+               ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),  \
+                 "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory")
 
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
@@ -363,33 +394,63 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       tc_fence_after();
       const int n_vis = limit - tile * kTileN + 1;          // columns [0, n_vis) are visible to this row
       const bool boundary = n_vis < kTileN;                 // only the tile(s) on the causal boundary need the mask
-      // ---- pass 1: row maximum
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        uint32_t s[32];
-        TMEM_LD32(t_S + 32 * q, s, 0);
-        tmem_wait_ld();
+      // One 32-column chunk: mask; if its maximum is more than 2^8 above the reference, move the reference
+      // to it (so no exponent ever exceeds 2^8); P = 2^(S - ref) as bf16 pairs; row sum of the chunk.
+      auto chunk = [&](uint32_t (&sv)[32], int col0, float& ref, float& sum_out, uint32_t (&pw)[16]) {
         if (boundary) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) s[c] = (32 * q + c) < n_vis ? s[c] : 0xff800000u;   // -inf
+          for (int c = 0; c < 32; ++c) sv[c] = (col0 + c) < n_vis ? sv[c] : 0xff800000u;   // -inf -> P = 0
         }
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int c = 0; c < 32; c += 4) {
 #pragma unroll
-          for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(mx4[k], __uint_as_float(s[c + k]));
+          for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(mx4[k], __uint_as_float(sv[c + k]));
+        }
+        const float cm = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        if (cm > ref + kRescaleThreshold) ref = cm;      // first chunk of the first tile: ref = -inf, key 0 is visible
+        const float2 ref2 = make_float2(ref, ref);
+        float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+#pragma unroll
+        for (int c = 0; c < 32; c += 4) {
+          const float2 d0 = sub2(make_float2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), ref2);
+          const float2 d1 = sub2(make_float2(__uint_as_float(sv[c + 2]), __uint_as_float(sv[c + 3])), ref2);
+          const float2 p0 = make_float2(ex2(d0.x), ex2(d0.y)), p1 = make_float2(ex2(d1.x), ex2(d1.y));
+          sum2[0] = add2(sum2[0], p0);
+          sum2[1] = add2(sum2[1], p1);
+          pw[c / 2] = pack_bf16x2(p0.x, p0.y);
+          pw[c / 2 + 1] = pack_bf16x2(p1.x, p1.y);
+        }
+        sum_out = (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
+      };
+      // One pass over the tile; loads run one chunk ahead of the arithmetic.  P chunk q goes to columns
+      // [16q, 16q+16) of the S buffer, which by then only holds S columns that have been consumed.
+      float ref = m_ref, ref_at[4], sum_q[4];
+      {
+        uint32_t sa[32], sb[32], pw[16];
+        TMEM_LD32(t_S, sa, 0);
+#pragma unroll
+        for (int hq = 0; hq < 2; ++hq) {
+          tmem_wait_ld();
+          TMEM_LD32(t_S + 64 * hq + 32, sb, 0);
+          chunk(sa, 64 * hq, ref, sum_q[2 * hq], pw);
+          ref_at[2 * hq] = ref;
+          tmem_wait_ld();                         // sb has landed (and every earlier load)
+          if (hq == 0) TMEM_LD32(t_S + 64, sa, 0);
+          TMEM_ST16(t_S + 32 * hq, pw);
+          chunk(sb, 64 * hq + 32, ref, sum_q[2 * hq + 1], pw);
+          ref_at[2 * hq + 1] = ref;
+          TMEM_ST16(t_S + 32 * hq + 16, pw);
         }
       }
-      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      // move the reference only when it lags by more than the threshold (exponents stay below 2^8 otherwise)
-      float alpha = 1.f;
-      if (mx > m_ref + kRescaleThreshold) {       // always true on the first tile (m_ref = -inf; key 0 is visible)
-        alpha = ex2(m_ref - mx);
-        m_ref = mx;
-      }
-      // O needs no wait: this tile's S exists, so the previous tile's PV (issued before it) has completed
-      if (tile > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+      // Bring everything to the final reference.  Common case: the reference did not move and nothing is touched.
+      const float alpha = ex2(m_ref - ref);       // 1 when unchanged; 0 on the first tile (m_ref = -inf)
+      float sum = sum_q[3];
 #pragma unroll
+      for (int q = 0; q < 3; ++q) sum += sum_q[q] * ex2(ref_at[q] - ref);
+      if (tile > 0 && __any_sync(0xffffffffu, ref != m_ref)) {
+        // O holds the sum up to the previous tile, whose PV is complete: this tile's S, issued after it, exists
+#pragma unroll 1
         for (int cb = 0; cb < D; cb += 32) {
           uint32_t o[32];
           TMEM_LD32(t_O + cb, o, 0);
@@ -399,35 +460,27 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
           TMEM_ST32(t_O + cb, o, 0);
         }
       }
-      // ---- pass 2: P = 2^(S - reference) as bf16 pairs, written over the first 64 columns of S
-      float sum4[4] = {0.f, 0.f, 0.f, 0.f};
+      if (__any_sync(0xffffffffu, ref_at[0] != ref)) {
+        // the reference moved inside the tile: P chunks written before the move are scaled down to it
 #pragma unroll
-      for (int half = 0; half < 2; ++half) {
-        uint32_t pw[32];
-#pragma unroll
-        for (int q = 0; q < 2; ++q) {
-          uint32_t s[32];
-          const int col0 = 64 * half + 32 * q;
-          TMEM_LD32(t_S + col0, s, 0);
+        for (int q = 0; q < 3; ++q) {
+          const float f = ex2(ref_at[q] - ref);
+          uint32_t pw[16];
+          asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+                       : "=r"(pw[0]), "=r"(pw[1]), "=r"(pw[2]), "=r"(pw[3]), "=r"(pw[4]), "=r"(pw[5]), "=r"(pw[6]), "=r"(pw[7]),
+                         "=r"(pw[8]), "=r"(pw[9]), "=r"(pw[10]), "=r"(pw[11]), "=r"(pw[12]), "=r"(pw[13]), "=r"(pw[14]), "=r"(pw[15])
+                       : "r"(t_S + 16 * q) : "memory");
           tmem_wait_ld();
-          if (boundary) {
 #pragma unroll
-            for (int c = 0; c < 32; ++c) s[c] = (col0 + c) < n_vis ? s[c] : 0xff800000u;
+          for (int c = 0; c < 16; ++c) {
+            const float2 v = bf16x2_to_float2(pw[c]);
+            pw[c] = pack_bf16x2(v.x * f, v.y * f);
           }
-#pragma unroll
-          for (int c = 0; c < 32; c += 8) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              const float p0 = ex2(__uint_as_float(s[c + 2 * k]) - m_ref);        // 2^(-inf) = 0 for masked columns
-              const float p1 = ex2(__uint_as_float(s[c + 2 * k + 1]) - m_ref);
-              sum4[k] += p0 + p1;
-              pw[16 * q + c / 2 + k] = pack_bf16x2(p0, p1);
-            }
-          }
+          TMEM_ST16(t_S + 16 * q, pw);
         }
-        TMEM_ST32(t_S + 32 * half, pw, 0);
       }
-      l_run = l_run * alpha + (sum4[0] + sum4[1]) + (sum4[2] + sum4[3]);
+      l_run = l_run * alpha + sum;
+      m_ref = ref;
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(BAR(kBarPFull, x));
@@ -463,14 +516,14 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     const int rt = tid - 2 * kSoftmaxWarps * 32;     // 0..127
     const int c = rt % CH;                       // chunk pair: dims [8c, 8c+8) and [D/2+8c, ...)
     const int k0 = (rt / CH) * CH;               // first of this thread's CH consecutive keys
-    // one-position step of this chunk's 8 pairs: table row 1
-    float c1[8], s1[8];
+    // one-position step of this chunk's 8 pairs: table row 1, as packed pairs (cos, sin, -sin)
+    float2 c1[4], s1[4], ns1[4];
     {
       const float4* row1 = reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(1) * D + 16 * c);
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const float4 t = __ldg(row1 + j);
-        c1[2 * j] = t.x; s1[2 * j] = t.y; c1[2 * j + 1] = t.z; s1[2 * j + 1] = t.w;
+        c1[j] = make_float2(t.x, t.z); s1[j] = make_float2(t.y, t.w); ns1[j] = make_float2(-t.y, -t.w);
       }
     }
     const int lc = c, hc = CH + c;
@@ -485,13 +538,13 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         if (key0 + k0 < kvl) atomicOr(p.status, MEPIC_DEV_BAD_POSITION);
         pos = 0;
       }
-      float cc[8], ss[8];
+      float2 cc[4], ss[4];
       {
         const float4* row = reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(pos) * D + 16 * c);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const float4 t = __ldg(row + j);
-          cc[2 * j] = t.x; ss[2 * j] = t.y; cc[2 * j + 1] = t.z; ss[2 * j + 1] = t.w;
+          cc[j] = make_float2(t.x, t.z); ss[j] = make_float2(t.y, t.w);
         }
       }
 #pragma unroll
@@ -505,16 +558,18 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const float2 a = bf16x2_to_float2(lw[j]), bq = bf16x2_to_float2(hw[j]);
-          lo_w[j] = pack_bf16x2(a.x * cc[2 * j] - bq.x * ss[2 * j], a.y * cc[2 * j + 1] - bq.y * ss[2 * j + 1]);
-          hi_w[j] = pack_bf16x2(a.x * ss[2 * j] + bq.x * cc[2 * j], a.y * ss[2 * j + 1] + bq.y * cc[2 * j + 1]);
+          const float2 nl = sub2(mul2(a, cc[j]), mul2(bq, ss[j]));
+          const float2 nh = fma2(a, ss[j], mul2(bq, cc[j]));
+          lo_w[j] = pack_bf16x2(nl.x, nl.y);
+          hi_w[j] = pack_bf16x2(nh.x, nh.y);
         }
         *plo = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
         *phi = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
         if (i + 1 < CH) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j) {          // (cos, sin)(pos+1) = (cos, sin)(pos) x (cos, sin)(1)
-            const float cn = cc[j] * c1[j] - ss[j] * s1[j];
-            ss[j] = ss[j] * c1[j] + cc[j] * s1[j];
+          for (int j = 0; j < 4; ++j) {          // (cos, sin)(pos+1) = (cos, sin)(pos) x (cos, sin)(1)
+            const float2 cn = fma2(ss[j], ns1[j], mul2(cc[j], c1[j]));
+            ss[j] = fma2(ss[j], c1[j], mul2(cc[j], s1[j]));
             cc[j] = cn;
           }
         }
