@@ -425,22 +425,27 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       };
       // One pass over the tile; loads run one chunk ahead of the arithmetic.  P chunk q goes to columns
       // [16q, 16q+16) of the S buffer, which by then only holds S columns that have been consumed.
-      float ref = m_ref, ref_at[4], sum_q[4];
+      float ref = m_ref, ref_at[4] = {0.f, 0.f, 0.f, 0.f}, sum_q[4] = {0.f, 0.f, 0.f, 0.f};
       {
         uint32_t sa[32], sb[32], pw[16];
         TMEM_LD32(t_S, sa, 0);
-#pragma unroll
+#pragma unroll 1
         for (int hq = 0; hq < 2; ++hq) {
+          float sum_a, sum_b;
           tmem_wait_ld();
           TMEM_LD32(t_S + 64 * hq + 32, sb, 0);
-          chunk(sa, 64 * hq, ref, sum_q[2 * hq], pw);
-          ref_at[2 * hq] = ref;
+          chunk(sa, 64 * hq, ref, sum_a, pw);
+          const float ref_a = ref;
           tmem_wait_ld();                         // sb has landed (and every earlier load)
           if (hq == 0) TMEM_LD32(t_S + 64, sa, 0);
           TMEM_ST16(t_S + 32 * hq, pw);
-          chunk(sb, 64 * hq + 32, ref, sum_q[2 * hq + 1], pw);
-          ref_at[2 * hq + 1] = ref;
+          chunk(sb, 64 * hq + 32, ref, sum_b, pw);
           TMEM_ST16(t_S + 32 * hq + 16, pw);
+          // static indices only (the loop is kept rolled to keep the code small): select by hq
+          ref_at[0] = hq == 0 ? ref_a : ref_at[0]; ref_at[1] = hq == 0 ? ref : ref_at[1];
+          ref_at[2] = hq == 1 ? ref_a : ref_at[2]; ref_at[3] = hq == 1 ? ref : ref_at[3];
+          sum_q[0] = hq == 0 ? sum_a : sum_q[0]; sum_q[1] = hq == 0 ? sum_b : sum_q[1];
+          sum_q[2] = hq == 1 ? sum_a : sum_q[2]; sum_q[3] = hq == 1 ? sum_b : sum_q[3];
         }
       }
       // Bring everything to the final reference.  Common case: the reference did not move and nothing is touched.
@@ -547,7 +552,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
           cc[j] = make_float2(t.x, t.z); ss[j] = make_float2(t.y, t.w);
         }
       }
-#pragma unroll
+#pragma unroll 2
       for (int i = 0; i < CH; ++i) {
         const int kk = k0 + i;
         uint4* plo = reinterpret_cast<uint4*>(Kb + (lc / 8) * kBlockBytes + sw128(kk, lc % 8));
