@@ -48,7 +48,7 @@ constexpr int kSoftmaxWarps = 4, kRotatorWarps = 4;
 constexpr int kKLoaderWarp = 12, kVLoaderWarp = 13, kMmaWarp = 14;   // warp 15 idles: 16 warps keep the register split even
 constexpr int kThreads = 512;
 constexpr int kSpinLimit = 1 << 22;
-constexpr float kSumTrigger = 256.f;       // a 32-column chunk whose P sums above this has outgrown the reference
+constexpr float kRescaleThreshold = 8.f;   // move the reference maximum only when it lags by 2^8
 
 struct Item { int32_t b, h, row0, nq; };   // rows row0 .. row0+nq-1 (global row indices) of request b
 
@@ -127,13 +127,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait that also gives up when another role has raised the abort flag.
-// `nap_ns` > 0 puts the warp to sleep between polls: for the roles that run ahead of the critical path, so that
-// their polling does not take issue slots from the warps that are on it.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                          unsigned nap_ns = 0) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
   for (int i = 0; i < kSpinLimit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (nap_ns) __nanosleep(nap_ns);
     if ((i & 1023) == 1023 && *abort_flag) return false;
   }
   *abort_flag = 1;
@@ -141,9 +137,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 // Same, with one verdict for the whole warp (the callers run warp-collective instructions afterwards).
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status,
-                                               unsigned nap_ns = 0) {
-  const bool w = mbar_wait(bar, parity, abort_flag, status, nap_ns);
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
+  const bool w = mbar_wait(bar, parity, abort_flag, status);
   return __all_sync(0xffffffffu, w) != 0;
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
@@ -399,36 +394,34 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       tc_fence_after();
       const int n_vis = limit - tile * kTileN + 1;          // columns [0, n_vis) are visible to this row
       const bool boundary = n_vis < kTileN;                 // only the tile(s) on the causal boundary need the mask
-      // One 32-column chunk: P = 2^(S - ref) as bf16 pairs and the chunk's row sum.  The common path does not
-      // look for the maximum at all: if some score were far above the reference its exponential would be large
-      // (or infinite, as on the very first chunk where ref = -inf), and the chunk sum shows it.  Only then is the
-      // maximum found, the reference moved to it, and the chunk redone from the scores still in registers; so no
-      // P ever exceeds kSumTrigger and none overflows.
+      // One 32-column chunk: mask; if its maximum is more than 2^8 above the reference, move the reference
+      // to it (so no exponent ever exceeds 2^8); P = 2^(S - ref) as bf16 pairs; row sum of the chunk.
       auto chunk = [&](uint32_t (&sv)[32], int col0, float& ref, float& sum_out, uint32_t (&pw)[16]) {
         if (boundary) {
 #pragma unroll
           for (int c = 0; c < 32; ++c) sv[c] = (col0 + c) < n_vis ? sv[c] : 0xff800000u;   // -inf -> P = 0
         }
-        float pr[32];
-        float s4[4] = {0.f, 0.f, 0.f, 0.f};
+        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-          pr[c] = ex2(__uint_as_float(sv[c]) - ref);
-          s4[c & 3] += pr[c];
+        for (int c = 0; c < 32; c += 4) {
+#pragma unroll
+          for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(mx4[k], __uint_as_float(sv[c + k]));
         }
-        float total = (s4[0] + s4[1]) + (s4[2] + s4[3]);
-        if (!(total <= kSumTrigger)) {            // also catches inf and NaN
-          float cm = -INFINITY;
+        const float cm = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+        if (cm > ref + kRescaleThreshold) ref = cm;      // first chunk of the first tile: ref = -inf, key 0 is visible
+        const float2 ref2 = make_float2(ref, ref);
+        float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
 #pragma unroll
-          for (int c = 0; c < 32; ++c) cm = fmaxf(cm, __uint_as_float(sv[c]));
-          if (cm > ref) ref = cm;                 // a fully masked chunk keeps the reference
-          total = 0.f;
-#pragma unroll
-          for (int c = 0; c < 32; ++c) { pr[c] = ex2(__uint_as_float(sv[c]) - ref); total += pr[c]; }
+        for (int c = 0; c < 32; c += 4) {
+          const float2 d0 = sub2(make_float2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), ref2);
+          const float2 d1 = sub2(make_float2(__uint_as_float(sv[c + 2]), __uint_as_float(sv[c + 3])), ref2);
+          const float2 p0 = make_float2(ex2(d0.x), ex2(d0.y)), p1 = make_float2(ex2(d1.x), ex2(d1.y));
+          sum2[0] = add2(sum2[0], p0);
+          sum2[1] = add2(sum2[1], p1);
+          pw[c / 2] = pack_bf16x2(p0.x, p0.y);
+          pw[c / 2 + 1] = pack_bf16x2(p1.x, p1.y);
         }
-#pragma unroll
-        for (int c = 0; c < 32; c += 2) pw[c / 2] = pack_bf16x2(pr[c], pr[c + 1]);
-        sum_out = total;
+        sum_out = (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
       };
       // One pass over the tile; loads run one chunk ahead of the arithmetic.  P chunk q goes to columns
       // [16q, 16q+16) of the S buffer, which by then only holds S columns that have been consumed.
@@ -542,7 +535,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     for (int tile = 0; tile < n_tiles; ++tile) {
       const int st = tile % kKStages;
       const uint32_t ph = static_cast<uint32_t>(tile / kKStages) & 1u;
-      if (!mbar_wait(BAR(kBarKLanded, st), ph, abort_flag, p.status, 200)) break;
+      if (!mbar_wait(BAR(kBarKLanded, st), ph, abort_flag, p.status)) break;
       unsigned char* Kb = Ks + st * NB * kBlockBytes;
       const int key0 = tile * kTileN;
       int pos = gbase[st * 8 + k0 / 16] + (k0 & 15);
@@ -570,16 +563,18 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
           const float2 a = bf16x2_to_float2(lw[j]), bq = bf16x2_to_float2(hw[j]);
-          lo_w[j] = pack_bf16x2(fmaf(a.x, cc[j].x, -(bq.x * ss[j].x)), fmaf(a.y, cc[j].y, -(bq.y * ss[j].y)));
-          hi_w[j] = pack_bf16x2(fmaf(a.x, ss[j].x, bq.x * cc[j].x), fmaf(a.y, ss[j].y, bq.y * cc[j].y));
+          const float2 nl = sub2(mul2(a, cc[j]), mul2(bq, ss[j]));
+          const float2 nh = fma2(a, ss[j], mul2(bq, cc[j]));
+          lo_w[j] = pack_bf16x2(nl.x, nl.y);
+          hi_w[j] = pack_bf16x2(nh.x, nh.y);
         }
         *plo = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
         *phi = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
         if (i + 1 < CH) {
 #pragma unroll
           for (int j = 0; j < 4; ++j) {          // (cos, sin)(pos+1) = (cos, sin)(pos) x (cos, sin)(1)
-            const float2 cn = make_float2(fmaf(ss[j].x, ns1[j].x, cc[j].x * c1[j].x), fmaf(ss[j].y, ns1[j].y, cc[j].y * c1[j].y));
-            ss[j] = make_float2(fmaf(ss[j].x, c1[j].x, cc[j].x * s1[j].x), fmaf(ss[j].y, c1[j].y, cc[j].y * s1[j].y));
+            const float2 cn = fma2(ss[j], ns1[j], mul2(cc[j], c1[j]));
+            ss[j] = fma2(ss[j], c1[j], mul2(cc[j], s1[j]));
             cc[j] = cn;
           }
         }
@@ -599,7 +594,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       if (tile >= depth) {
         // the stage is free once every MMA that reads its previous tenant has completed
         const uint32_t bar = BAR(is_k ? kBarKFree : kBarVFree, st);
-        if (!mbar_wait_warp(bar, static_cast<uint32_t>(tile / depth - 1) & 1u, abort_flag, p.status, 200)) { ok = false; break; }
+        if (!mbar_wait_warp(bar, static_cast<uint32_t>(tile / depth - 1) & 1u, abort_flag, p.status)) { ok = false; break; }
       }
       const int key0 = tile * kTileN;
       const int gkey = key0 + lane * 16;
