@@ -19,6 +19,7 @@
 // the cos/sin table, and rotates every key only by its offset tau < 16 inside
 // the tile, with cos/sin of those 16 offsets held in registers for the whole
 // kernel.  Keys are rotated in registers in fp32 and never written back.
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -170,37 +171,58 @@ __device__ __forceinline__ void advance(Cursor& c, const int32_t* kv_len, int ba
 }
 
 // ---------------------------------------------------------------- the split-KV kernel
-template <int D, int G>
-__global__ void __launch_bounds__(kWarps * 32, 1) mepic_decode_splitkv(const DecodeParams p) {
-  constexpr int kStages = stages_for(D, G);
-  constexpr int DL = D / 16;                 // K phase: bf16 per lane per half row (8 lanes span a half row)
-  constexpr int NP = DL / 2;                 // ... as packed pairs (32-bit words / float2)
-  constexpr int DV = D / 16;                 // V phase: dims per lane (16 lanes span a row)
-  constexpr int GP = G <= 1 ? 1 : G <= 2 ? 2 : G <= 4 ? 4 : 8;   // heads padded to a power of two
-  constexpr int LPH = 8 / GP;                // dim-lanes that end up holding the same head's score
-  constexpr int HPL = (G + 3) / 4;           // heads each key-group rotates per tile
-  constexpr int PSTR = GP < 4 ? 4 : GP;      // floats per key in the probability buffer
-  constexpr int kTileElems = kTile * D;
-  constexpr int kStageBytes = 2 * kTileElems * 2;
-  constexpr int kQrotFloats = G * D;
-  constexpr int kWarpBytes = kStages * kStageBytes + kQrotFloats * 4 + kTile * PSTR * 4 + 64;
+// Warp-level tensor-core MMA (mma.sync m16n8k16, bf16 in, fp32 accumulate) for the two contractions of a tile:
+//   S^T[head][key]  = Q_tile[head][dim] . K'[key][dim]^T      A = rotated q (heads padded to 16 rows), B = rotated K
+//   O  [head][dim] += P[head][key]      . V[key][dim]         A = P straight from the S accumulators, B = V
+// so that only the rotation of K (thread-local on the B fragments: the partner dim i + D/2 sits in the fragment
+// of k-step j + D/32, same lane, same position) and the softmax stay on the CUDA cores.
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// (lo, hi) -> packed bf16x2, round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t r;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+  return r;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
 
-  extern __shared__ __align__(128) unsigned char smem_raw[];
+template <int D, int G>
+__global__ void __launch_bounds__(kWarps * 32, 1)
+mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
+  constexpr int kStages = 3;
+  constexpr int NB = D / 64;                 // 64-dim blocks (128-byte swizzled rows) per K or V row
+  constexpr int KS = D / 16;                 // k-steps of the QK^T contraction
+  constexpr int KH = KS / 2;                 // k-steps per half: step j pairs with step j + KH
+  constexpr int ND = D / 8;                  // n-tiles of the PV product
+  constexpr int kBlockBytes = kTile * 128;   // one [16 rows x 64 dims] block
+  constexpr int kStageBytes = 2 * NB * kBlockBytes;   // K blocks then V blocks
+  constexpr int kWarpBytes = kStages * kStageBytes;
+
+  extern __shared__ unsigned char smem_dyn[];
+  // 1024-byte alignment: the swizzle pattern is a function of the address bits
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
   const int lane = threadIdx.x & 31;
   const int wic = threadIdx.x >> 5;
-  unsigned char* wbase = smem_raw + static_cast<size_t>(wic) * kWarpBytes;
-  uint16_t* stage0 = reinterpret_cast<uint16_t*>(wbase);
-  float4* qrot = reinterpret_cast<float4*>(wbase + kStages * kStageBytes);
-  float* pbuf = reinterpret_cast<float*>(wbase + kStages * kStageBytes + kQrotFloats * 4);
-  unsigned char* tail = wbase + kStages * kStageBytes + kQrotFloats * 4 + kTile * PSTR * 4;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(tail);          // kStages x 8 bytes
-  volatile int* meta = reinterpret_cast<volatile int*>(tail + 32);   // tile position base per stage
+  unsigned char* stage0 = smem + static_cast<size_t>(wic) * kWarpBytes;
+  unsigned char* misc = smem + static_cast<size_t>(kWarps) * kWarpBytes + wic * 64;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(misc);                 // kStages x 8 bytes
+  volatile int* meta = reinterpret_cast<volatile int*>(misc + 32);    // tile position base per stage
 
-  const int kg = lane >> 3;      // key group (K phase): keys kg, kg+4, kg+8, kg+12 of the tile
-  const int l8 = lane & 7;       // dim lane (K phase)
-  const int hw = lane >> 4;      // half warp (V phase): keys of parity hw
-  const int l16 = lane & 15;     // dim lane (V phase)
-  const int my_head = l8 / LPH;  // head whose score this lane holds after the reduction
+  const int g = lane >> 2;       // fragment row group: head g (A, C) / key g (B)
+  const int t = lane & 3;        // fragment column group
 
   const long long w = static_cast<long long>(blockIdx.x) * kWarps + wic;
   const Cut cut = cut_of_line(p.kv_len, p.batch, p.n_kv_heads, p.n_workers, lane);
@@ -217,18 +239,17 @@ __global__ void __launch_bounds__(kWarps * 32, 1) mepic_decode_splitkv(const Dec
   }
   __syncwarp();
 
-  // cos/sin of the 16 in-tile offsets, this lane's dims: rows 0..15 of the table.
-  float2 c2[4][NP], s2[4][NP];
+  // cos/sin of the in-tile offsets this lane's B fragments cover: keys g and g+8, pairs 16j + 2t + 8r + {0,1}.
+  float kc[2][KH][2][2], ksn[2][KH][2][2];      // [key g / g+8][k-step][fragment register][element]
 #pragma unroll
-  for (int ps = 0; ps < 4; ++ps) {
-    const float4* row = reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(kg + 4 * ps) * D + l8 * DL * 2);
+  for (int kq = 0; kq < 2; ++kq)
 #pragma unroll
-    for (int j = 0; j < NP; ++j) {
-      const float4 cs = __ldg(row + j);      // (cos, sin) of dims 2j and 2j+1 of this lane's slice
-      c2[ps][j] = make_float2(cs.x, cs.z);
-      s2[ps][j] = make_float2(cs.y, cs.w);
-    }
-  }
+    for (int j = 0; j < KH; ++j)
+#pragma unroll
+      for (int r = 0; r < 2; ++r) {
+        const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(g + 8 * kq) * D + 2 * (16 * j + 2 * t + 8 * r)));
+        kc[kq][j][r][0] = cs.x; ksn[kq][j][r][0] = cs.y; kc[kq][j][r][1] = cs.z; ksn[kq][j][r][1] = cs.w;
+      }
 
   Cursor pc = locate(p.kv_len, p.batch, p.n_kv_heads, x0, lane);   // producer cursor
   Cursor cc = pc;                                                  // consumer cursor
@@ -249,13 +270,16 @@ __global__ void __launch_bounds__(kWarps * 32, 1) mepic_decode_splitkv(const Dec
     const int pos = __shfl_sync(kFull, win_pos, e - win_e0);
     if (lane == 0) {
       if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
-      const size_t off = ((static_cast<size_t>(page) * p.n_kv_heads + pc.h) * p.page_size + static_cast<size_t>(sub) * kTile) * D;
+      const int y = (page * p.n_kv_heads + pc.h) * p.page_size + sub * kTile;     // row of the pool viewed as [rows][D]
       const uint32_t bar = smem_u32(&bars[stage]);
-      const uint32_t dst = smem_u32(stage0 + static_cast<size_t>(stage) * 2 * kTileElems);
+      const uint32_t dst = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
       meta[stage] = pos + sub * kTile;
       mbar_expect_tx(bar, kStageBytes);
-      bulk_g2s(dst, p.k_pool + off, kTileElems * 2, bar);
-      bulk_g2s(dst + kTileElems * 2, p.v_pool + off, kTileElems * 2, bar);
+#pragma unroll
+      for (int nb = 0; nb < NB; ++nb) {
+        tma_load_2d(dst + nb * kBlockBytes, &map_k, nb * 64, y, bar);
+        tma_load_2d(dst + (NB + nb) * kBlockBytes, &map_v, nb * 64, y, bar);
+      }
     }
     advance(pc, p.kv_len, p.batch, p.n_kv_heads);
   };
@@ -263,33 +287,24 @@ __global__ void __launch_bounds__(kWarps * 32, 1) mepic_decode_splitkv(const Dec
   int issued = 0;
   for (; issued < kStages && issued < n_tiles; ++issued) issue(issued);
 
-  // per-unit state
+  // per-unit state: head g of the unit's G query heads (lanes with g >= G carry zeros)
   int ub = -1, uh = -1, qpos = 0;
-  float qraw_lo[HPL][DL], qraw_hi[HPL][DL];   // this key group's heads, un-rotated, pre-scaled
-  float m_mine = -INFINITY, l_mine = 0.f;
-  float2 acc[G][DV / 2];
+  float q_lo[KH][2][2], q_hi[KH][2][2];     // un-rotated q, pre-scaled by sm_scale*log2e: pairs as for kc/ksn
+  float m_run = -INFINITY, l_run = 0.f;
+  float acc[ND][4];                         // O fragments: [n-tile][c0,c1 = head g | c2,c3 = head g+8 (unused)]
 
   auto flush = [&]() {
     if (ub < 0) return;
-    float l_tot = l_mine;
-    l_tot += __shfl_xor_sync(kFull, l_tot, 8);
-    l_tot += __shfl_xor_sync(kFull, l_tot, 16);
+    float l_tot = l_run;
+    l_tot += __shfl_xor_sync(kFull, l_tot, 1);
+    l_tot += __shfl_xor_sync(kFull, l_tot, 2);
     const long long slot = static_cast<long long>(ub) * p.n_kv_heads + uh + w;
+    if (g < G) {
+      float* dst = p.part_o + (slot * G + g) * D;
 #pragma unroll
-    for (int g = 0; g < G; ++g) {
-#pragma unroll
-      for (int j = 0; j < DV / 2; ++j) {
-        acc[g][j].x += __shfl_xor_sync(kFull, acc[g][j].x, 16);
-        acc[g][j].y += __shfl_xor_sync(kFull, acc[g][j].y, 16);
-      }
-      if (hw == 0) {
-        float2* dst = reinterpret_cast<float2*>(p.part_o + (slot * G + g) * D + l16 * DV);
-#pragma unroll
-        for (int j = 0; j < DV / 2; ++j) dst[j] = acc[g][j];
-      }
+      for (int nd = 0; nd < ND; ++nd) *reinterpret_cast<float2*>(dst + 8 * nd + 2 * t) = make_float2(acc[nd][0], acc[nd][1]);
+      if (t == 0) *reinterpret_cast<float2*>(p.part_ml + (slot * G + g) * 2) = make_float2(m_run, l_tot);
     }
-    if (kg == 0 && (l8 % LPH) == 0 && my_head < G)
-      *reinterpret_cast<float2*>(p.part_ml + (slot * G + my_head) * 2) = make_float2(m_mine, l_tot);
   };
 
   int stage = 0;
@@ -300,198 +315,134 @@ __global__ void __launch_bounds__(kWarps * 32, 1) mepic_decode_splitkv(const Dec
       ub = cc.b; uh = cc.h;
       qpos = __ldg(p.q_pos + ub);
       const int n_q_heads = p.n_kv_heads * G;
+      const uint32_t* src = reinterpret_cast<const uint32_t*>(
+          p.q + (static_cast<size_t>(ub) * n_q_heads + static_cast<size_t>(uh) * G + (g < G ? g : 0)) * D);
 #pragma unroll
-      for (int hh = 0; hh < HPL; ++hh) {
-        const int head = kg + 4 * hh;
-        if (head < G) {
-          const uint32_t* src = reinterpret_cast<const uint32_t*>(
-              p.q + (static_cast<size_t>(ub) * n_q_heads + static_cast<size_t>(uh) * G + head) * D);
+      for (int j = 0; j < KH; ++j)
 #pragma unroll
-          for (int j = 0; j < NP; ++j) {
-            const float2 lo = bf16x2_to_float2(__ldg(src + l8 * NP + j));
-            const float2 hi = bf16x2_to_float2(__ldg(src + D / 4 + l8 * NP + j));
-            qraw_lo[hh][2 * j] = lo.x * p.scale_log2; qraw_lo[hh][2 * j + 1] = lo.y * p.scale_log2;
-            qraw_hi[hh][2 * j] = hi.x * p.scale_log2; qraw_hi[hh][2 * j + 1] = hi.y * p.scale_log2;
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < DL; ++j) { qraw_lo[hh][j] = 0.f; qraw_hi[hh][j] = 0.f; }
+        for (int r = 0; r < 2; ++r) {
+          const int pair = 16 * j + 2 * t + 8 * r;              // dims pair, pair+1 and their partners + D/2
+          const float2 lo = bf16x2_to_float2(__ldg(src + pair / 2));
+          const float2 hi = bf16x2_to_float2(__ldg(src + (pair + D / 2) / 2));
+          const float sc = g < G ? p.scale_log2 : 0.f;
+          q_lo[j][r][0] = lo.x * sc; q_lo[j][r][1] = lo.y * sc;
+          q_hi[j][r][0] = hi.x * sc; q_hi[j][r][1] = hi.y * sc;
         }
-      }
-      m_mine = -INFINITY; l_mine = 0.f;
+      m_run = -INFINITY; l_run = 0.f;
 #pragma unroll
-      for (int g = 0; g < G; ++g)
-#pragma unroll
-        for (int j = 0; j < DV / 2; ++j) acc[g][j] = make_float2(0.f, 0.f);
+      for (int nd = 0; nd < ND; ++nd) { acc[nd][0] = 0.f; acc[nd][1] = 0.f; acc[nd][2] = 0.f; acc[nd][3] = 0.f; }
     }
 
+    // ---- A fragments of the query rotated by (qpos - tile base); the table row does not depend on the data, so
+    //      it is fetched before the wait for the tile
+    uint32_t qa[KS][2];                         // [k-step][a0 (dims 16j+2t,+1) | a2 (dims 16j+8+2t,+1)], row = head g
+    {
+      // meta is written by lane 0 before it arms the barrier; reading it needs the barrier's acquire, so the
+      // position comes after the wait - but the wait is short once the ring is primed.  Do the wait first.
+    }
     if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity)) {
       // Give the copies still in flight a last bounded chance to land, then leave cleanly.
       if (lane == 0) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
       for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(&bars[s]), s == stage ? parity : (s < stage ? parity ^ 1u : parity));
       return;
     }
-    const uint16_t* ks = stage0 + static_cast<size_t>(stage) * 2 * kTileElems;
-    const uint16_t* vs = ks + kTileElems;
+    const uint32_t ks_addr = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
+    const uint32_t vs_addr = ks_addr + NB * kBlockBytes;
     const int base = meta[stage];
     const int n_valid = min(kTile, cc.kvl - cc.t * kTile);
-
-    // ---- rotate the G query vectors by (qpos - base): one table row, each key group does its heads
     {
       const int rel = qpos - base;
       int arel = rel < 0 ? -rel : rel;
       const float sgn = rel < 0 ? -1.f : 1.f;
       if (arel > p.max_position) { if (lane == 0) atomicOr(p.status, MEPIC_DEV_BAD_POSITION); arel = p.max_position; }
-      const float4* row = reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(arel) * D + l8 * DL * 2);
-      float4 cs[NP];
+      const float* row = p.rope + static_cast<size_t>(arel) * D;
 #pragma unroll
-      for (int j = 0; j < NP; ++j) cs[j] = __ldg(row + j);
+      for (int j = 0; j < KH; ++j)
 #pragma unroll
-      for (int hh = 0; hh < HPL; ++hh) {
-        const int head = kg + 4 * hh;
-        if (head < G) {
-          float lo[DL], hi[DL];
-#pragma unroll
-          for (int j = 0; j < NP; ++j) {
-            const float c0 = cs[j].x, s0 = cs[j].y * sgn, c1 = cs[j].z, s1 = cs[j].w * sgn;
-            lo[2 * j] = qraw_lo[hh][2 * j] * c0 - qraw_hi[hh][2 * j] * s0;
-            hi[2 * j] = qraw_lo[hh][2 * j] * s0 + qraw_hi[hh][2 * j] * c0;
-            lo[2 * j + 1] = qraw_lo[hh][2 * j + 1] * c1 - qraw_hi[hh][2 * j + 1] * s1;
-            hi[2 * j + 1] = qraw_lo[hh][2 * j + 1] * s1 + qraw_hi[hh][2 * j + 1] * c1;
-          }
-          // layout: float4 index (head * 2*DL/4 + part) * 8 + l8 ; parts = lo quads then hi quads
-#pragma unroll
-          for (int part = 0; part < DL / 4; ++part) {
-            qrot[(head * (DL / 2) + part) * 8 + l8] = make_float4(lo[4 * part], lo[4 * part + 1], lo[4 * part + 2], lo[4 * part + 3]);
-            qrot[(head * (DL / 2) + DL / 4 + part) * 8 + l8] = make_float4(hi[4 * part], hi[4 * part + 1], hi[4 * part + 2], hi[4 * part + 3]);
-          }
+        for (int r = 0; r < 2; ++r) {
+          const float4 cs = __ldg(reinterpret_cast<const float4*>(row + 2 * (16 * j + 2 * t + 8 * r)));
+          const float c0 = cs.x, s0 = cs.y * sgn, c1 = cs.z, s1 = cs.w * sgn;
+          const float l0 = q_lo[j][r][0] * c0 - q_hi[j][r][0] * s0, h0 = q_lo[j][r][0] * s0 + q_hi[j][r][0] * c0;
+          const float l1 = q_lo[j][r][1] * c1 - q_hi[j][r][1] * s1, h1 = q_lo[j][r][1] * s1 + q_hi[j][r][1] * c1;
+          qa[j][r] = pack_bf16x2(l0, l1);
+          qa[j + KH][r] = pack_bf16x2(h0, h1);
         }
-      }
     }
-    __syncwarp();
-    float2 qlo[G][NP], qhi[G][NP];
-#pragma unroll
-    for (int g = 0; g < G; ++g) {
-#pragma unroll
-      for (int part = 0; part < DL / 4; ++part) {
-        const float4 a = qrot[(g * (DL / 2) + part) * 8 + l8];
-        const float4 b = qrot[(g * (DL / 2) + DL / 4 + part) * 8 + l8];
-        qlo[g][2 * part] = make_float2(a.x, a.y); qlo[g][2 * part + 1] = make_float2(a.z, a.w);
-        qhi[g][2 * part] = make_float2(b.x, b.y); qhi[g][2 * part + 1] = make_float2(b.z, b.w);
+    // rows at or past kv_len may hold anything (NaN bit patterns included): their P is 0, but 0 x NaN is NaN,
+    // so V must be finite there.  Only a request's last tile has such rows.
+    if (n_valid < kTile) {
+      for (int idx = n_valid * 8 * NB + lane; idx < kTile * 8 * NB; idx += 32) {
+        const int key = idx / (8 * NB), ch = idx % (8 * NB);
+        const uint32_t a = vs_addr + (ch / 8) * kBlockBytes + key * 128 + (((ch % 8) ^ (key & 7)) << 4);
+        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
       }
+      __syncwarp();
     }
 
-    // ---- K phase: rotate each key by its in-tile offset, dot with the G queries, reduce over 8 lanes
-    float sc[4];
+    // ---- S^T = Q K'^T : B fragments by ldmatrix, rotated in registers, two key n-tiles (keys 0-7, 8-15)
+    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int ps = 0; ps < 4; ++ps) {
-      const int r = kg + 4 * ps;
-      const uint32_t* krow = reinterpret_cast<const uint32_t*>(ks + r * D);
-      uint32_t wlo[NP], whi[NP];
-      if constexpr (NP == 4) {
-        const uint4 a = *reinterpret_cast<const uint4*>(krow + l8 * 4);
-        const uint4 b = *reinterpret_cast<const uint4*>(krow + D / 4 + l8 * 4);
-        wlo[0] = a.x; wlo[1] = a.y; wlo[2] = a.z; wlo[3] = a.w;
-        whi[0] = b.x; whi[1] = b.y; whi[2] = b.z; whi[3] = b.w;
-      } else {
-        const uint2 a = *reinterpret_cast<const uint2*>(krow + l8 * 2);
-        const uint2 b = *reinterpret_cast<const uint2*>(krow + D / 4 + l8 * 2);
-        wlo[0] = a.x; wlo[1] = a.y; whi[0] = b.x; whi[1] = b.y;
+    for (int j = 0; j < KH; ++j) {
+      uint32_t lo[4], hi[4];      // lo: k-step j, hi: k-step j + KH; [b0 nt0, b1 nt0, b0 nt1, b1 nt1]
+      {
+        // lane -> (matrix mi = lane / 8, row = lane % 8): key = 8 (mi / 2) + row, 16-byte chunk 2 j + (mi & 1)
+        const int mi = lane >> 3, key = ((mi >> 1) << 3) + (lane & 7);
+        const int cl = 2 * j + (mi & 1), chh = 2 * (j + KH) + (mi & 1);
+        ldmatrix_x4(lo, ks_addr + (cl / 8) * kBlockBytes + key * 128 + (((cl % 8) ^ (key & 7)) << 4));
+        ldmatrix_x4(hi, ks_addr + (chh / 8) * kBlockBytes + key * 128 + (((chh % 8) ^ (key & 7)) << 4));
       }
-      float2 dot[GP];
 #pragma unroll
-      for (int g = 0; g < GP; ++g) dot[g] = make_float2(0.f, 0.f);
-#pragma unroll
-      for (int j = 0; j < NP; ++j) {
-        const float2 lo = bf16x2_to_float2(wlo[j]);
-        const float2 hi = bf16x2_to_float2(whi[j]);
-        const float2 klo = sub2(mul2(lo, c2[ps][j]), mul2(hi, s2[ps][j]));
-        const float2 khi = fma2(lo, s2[ps][j], mul2(hi, c2[ps][j]));
-#pragma unroll
-        for (int g = 0; g < G; ++g) {
-          dot[g] = fma2(qlo[g][j], klo, dot[g]);
-          dot[g] = fma2(qhi[g][j], khi, dot[g]);
-        }
+      for (int f = 0; f < 4; ++f) {
+        const int kq = f >> 1, r = f & 1;       // key g + 8 kq, fragment register r
+        const float2 a = bf16x2_to_float2(lo[f]), b = bf16x2_to_float2(hi[f]);
+        const float c0 = kc[kq][j][r][0], sn0 = ksn[kq][j][r][0], c1 = kc[kq][j][r][1], sn1 = ksn[kq][j][r][1];
+        lo[f] = pack_bf16x2(fmaf(a.x, c0, -(b.x * sn0)), fmaf(a.y, c1, -(b.y * sn1)));
+        hi[f] = pack_bf16x2(fmaf(a.x, sn0, b.x * c0), fmaf(a.y, sn1, b.y * c1));
       }
-      float v[GP];
-#pragma unroll
-      for (int g = 0; g < GP; ++g) v[g] = dot[g].x + dot[g].y;
-      // reduce-scatter over the 8 dim lanes: halve the number of live heads per step while any remain
-      int cnt = GP;
-#pragma unroll
-      for (int msk = 4; msk >= 1; msk >>= 1) {
-        if (cnt > 1) {
-          const bool upper = (l8 & msk) != 0;
-#pragma unroll
-          for (int i = 0; i < GP / 2; ++i) {
-            if (i < cnt / 2) {
-              const float keep = upper ? v[i + cnt / 2] : v[i];
-              const float send = upper ? v[i] : v[i + cnt / 2];
-              v[i] = keep + __shfl_xor_sync(kFull, send, msk);
-            }
-          }
-          cnt >>= 1;
-        } else {
-          v[0] += __shfl_xor_sync(kFull, v[0], msk);
-        }
-      }
-      sc[ps] = (r < n_valid) ? v[0] : -INFINITY;
+      mma_bf16(s0, qa[j][0], 0u, qa[j][1], 0u, lo[0], lo[1]);
+      mma_bf16(s1, qa[j][0], 0u, qa[j][1], 0u, lo[2], lo[3]);
+      mma_bf16(s0, qa[j + KH][0], 0u, qa[j + KH][1], 0u, hi[0], hi[1]);
+      mma_bf16(s1, qa[j + KH][0], 0u, qa[j + KH][1], 0u, hi[2], hi[3]);
     }
 
-    // ---- online softmax for this lane's head (log2 domain)
+    // ---- online softmax for head g (log2 domain); this lane holds keys 2t, 2t+1, 8+2t, 9+2t
+    float sc[4] = {s0[0], s0[1], s1[0], s1[1]};
+    {
+      const int k0 = 2 * t;
+      if (k0 >= n_valid) sc[0] = -INFINITY;
+      if (k0 + 1 >= n_valid) sc[1] = -INFINITY;
+      if (k0 + 8 >= n_valid) sc[2] = -INFINITY;
+      if (k0 + 9 >= n_valid) sc[3] = -INFINITY;
+    }
     float mx = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
-    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 8));
-    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 16));
-    if (__any_sync(kFull, mx > m_mine)) {
-      const float m_new = fmaxf(m_mine, mx);
-      const float alpha = ex2(m_mine - m_new);     // 0 on the first tile (m_mine = -inf)
-      m_mine = m_new;
-      l_mine *= alpha;
+    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
+    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 2));
+    if (__any_sync(kFull, mx > m_run)) {
+      const float m_new = fmaxf(m_run, mx);
+      const float alpha = ex2(m_run - m_new);     // 0 on the first tile (m_run = -inf)
+      m_run = m_new;
+      l_run *= alpha;
 #pragma unroll
-      for (int g = 0; g < G; ++g) {
-        const float a = __shfl_sync(kFull, alpha, g * LPH);
-#pragma unroll
-        for (int j = 0; j < DV / 2; ++j) { acc[g][j].x *= a; acc[g][j].y *= a; }
-      }
+      for (int nd = 0; nd < ND; ++nd) { acc[nd][0] *= alpha; acc[nd][1] *= alpha; }
     }
-#pragma unroll
-    for (int ps = 0; ps < 4; ++ps) {
-      const float pr = ex2(sc[ps] - m_mine);
-      l_mine += pr;
-      if ((l8 % LPH) == 0) pbuf[(kg + 4 * ps) * PSTR + my_head] = pr;
-    }
-    __syncwarp();
+    const float p0 = ex2(sc[0] - m_run), p1 = ex2(sc[1] - m_run), p2 = ex2(sc[2] - m_run), p3 = ex2(sc[3] - m_run);
+    l_run += (p0 + p1) + (p2 + p3);
+    const uint32_t pa0 = pack_bf16x2(p0, p1), pa2 = pack_bf16x2(p2, p3);    // A fragment of P: a0 keys 2t.., a2 keys 8+2t..
 
-    // ---- V phase: half warps take alternate keys, 16 lanes span the row
+    // ---- O += P V : B fragments of V by transposing ldmatrix, two dim n-tiles per load
 #pragma unroll
-    for (int i = 0; i < kTile / 2; ++i) {
-      const int key = 2 * i + hw;
-      if (key < n_valid) {
-        float pg[8];
-        const float4 p0 = *reinterpret_cast<const float4*>(pbuf + key * PSTR);
-        pg[0] = p0.x; pg[1] = p0.y; pg[2] = p0.z; pg[3] = p0.w;
-        if constexpr (GP == 8) {
-          const float4 p1 = *reinterpret_cast<const float4*>(pbuf + key * PSTR + 4);
-          pg[4] = p1.x; pg[5] = p1.y; pg[6] = p1.z; pg[7] = p1.w;
-        }
-        const uint32_t* vrow = reinterpret_cast<const uint32_t*>(vs + key * D + l16 * DV);
-        uint32_t wv[DV / 2];
-        if constexpr (DV == 8) {
-          const uint4 a = *reinterpret_cast<const uint4*>(vrow);
-          wv[0] = a.x; wv[1] = a.y; wv[2] = a.z; wv[3] = a.w;
-        } else {
-          const uint2 a = *reinterpret_cast<const uint2*>(vrow);
-          wv[0] = a.x; wv[1] = a.y;
-        }
-#pragma unroll
-        for (int j = 0; j < DV / 2; ++j) {
-          const float2 vv = bf16x2_to_float2(wv[j]);
-#pragma unroll
-          for (int g = 0; g < G; ++g) acc[g][j] = fma2(make_float2(pg[g], pg[g]), vv, acc[g][j]);
-        }
+    for (int nd = 0; nd < ND; nd += 2) {
+      uint32_t vb[4];             // [b0, b1] of n-tile nd, [b0, b1] of n-tile nd+1
+      {
+        // lane -> (matrix mi, row): key = 8 (mi & 1) + row, 16-byte chunk nd + (mi >> 1)
+        const int mi = lane >> 3, key = ((mi & 1) << 3) + (lane & 7);
+        const int ch = nd + (mi >> 1);
+        ldmatrix_x4_trans(vb, vs_addr + (ch / 8) * kBlockBytes + key * 128 + (((ch % 8) ^ (key & 7)) << 4));
       }
+      mma_bf16(acc[nd], pa0, 0u, pa2, 0u, vb[0], vb[1]);
+      mma_bf16(acc[nd + 1], pa0, 0u, pa2, 0u, vb[2], vb[3]);
     }
-    __syncwarp();   // every lane is done with this stage, qrot and pbuf
+    __syncwarp();   // every lane is done with this stage
 
     if (issued < n_tiles) { issue(stage); ++issued; }
     advance(cc, p.kv_len, p.batch, p.n_kv_heads);
@@ -543,17 +494,16 @@ __global__ void mepic_decode_merge(const DecodeParams p) {
 
 template <int D, int G>
 constexpr size_t decode_smem_bytes() {
-  constexpr int GP = G <= 1 ? 1 : G <= 2 ? 2 : G <= 4 ? 4 : 8;
-  constexpr int PSTR = GP < 4 ? 4 : GP;
-  return static_cast<size_t>(kWarps) * (stages_for(D, G) * (2 * kTile * D * 2) + G * D * 4 + kTile * PSTR * 4 + 64);
+  // per warp: 3 stages of (K blocks + V blocks); then 64 bytes of barriers and tile positions per warp; 1 KB alignment slack
+  return static_cast<size_t>(kWarps) * (3 * 2 * (D / 64) * kTile * 128) + kWarps * 64 + 1024;
 }
 
 template <int D, int G>
-int32_t launch_decode(const DecodeParams& p, int n_ctas, cudaStream_t stream) {
+int32_t launch_decode(const DecodeParams& p, int n_ctas, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
   constexpr size_t smem = decode_smem_bytes<D, G>();
   cudaError_t e = cudaFuncSetAttribute(mepic_decode_splitkv<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("decode: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
-  mepic_decode_splitkv<D, G><<<n_ctas, kWarps * 32, smem, stream>>>(p);
+  mepic_decode_splitkv<D, G><<<n_ctas, kWarps * 32, smem, stream>>>(p, map_k, map_v);
   mepic_decode_merge<D, G><<<p.batch * p.n_kv_heads, G * D, 0, stream>>>(p);
   e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("decode: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
@@ -617,8 +567,13 @@ extern "C" int32_t mepic_attn_decode(const mepic_config_t* cfg, const mepic_deco
   p.n_workers = sms * kWarps;
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  alignas(64) CUtensorMap map_k, map_v;
+  int32_t rc = mepic_make_pool_map(cfg, a->k_pool, &map_k);
+  if (rc != MEPIC_OK) return rc;
+  rc = mepic_make_pool_map(cfg, a->v_pool, &map_v);
+  if (rc != MEPIC_OK) return rc;
 
-#define MEPIC_DECODE_CASE(DD, GG) if (D == DD && G == GG) return launch_decode<DD, GG>(p, sms, st);
+#define MEPIC_DECODE_CASE(DD, GG) if (D == DD && G == GG) return launch_decode<DD, GG>(p, sms, map_k, map_v, st);
   MEPIC_DECODE_CASE(128, 1) MEPIC_DECODE_CASE(128, 2) MEPIC_DECODE_CASE(128, 4) MEPIC_DECODE_CASE(128, 5) MEPIC_DECODE_CASE(128, 8)
   MEPIC_DECODE_CASE(64, 1) MEPIC_DECODE_CASE(64, 2) MEPIC_DECODE_CASE(64, 4) MEPIC_DECODE_CASE(64, 5) MEPIC_DECODE_CASE(64, 8)
 #undef MEPIC_DECODE_CASE

@@ -33,7 +33,6 @@
 #include <stdint.h>
 
 #include <algorithm>
-#include <mutex>
 #include <vector>
 
 #include "mepic.h"
@@ -756,40 +755,6 @@ bool build_items(const mepic_config_t* cfg, int batch, const int32_t* row_offset
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// The driver's tensor-map encoder, looked up through the runtime so that the library links no driver stub.
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
-                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-EncodeTiledFn encode_tiled_fn() {
-  static std::mutex mu;
-  static EncodeTiledFn fn = nullptr;
-  std::lock_guard<std::mutex> lock(mu);
-  if (!fn) {
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult res;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &res) == cudaSuccess &&
-        res == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
-  return fn;
-}
-
-// The pool seen as a 2-D bf16 tensor [num_pages * n_kv_heads * page_size rows][D]; box = 64 dims x 16 rows, 128-byte swizzle.
-int32_t make_pool_map(const mepic_config_t* cfg, void* pool, CUtensorMap* out) {
-  EncodeTiledFn fn = encode_tiled_fn();
-  if (!fn) { mepic_set_error("prefill: cuTensorMapEncodeTiled is not available from the driver"); return MEPIC_E_CUDA; }
-  const cuuint64_t rows = static_cast<cuuint64_t>(cfg->num_pages) * cfg->n_kv_heads * cfg->page_size;
-  if (rows > 0x7fffffffull) { mepic_set_error("prefill: pool has too many rows for 32-bit tensor coordinates"); return MEPIC_E_INVAL; }
-  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cfg->head_dim), rows};
-  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cfg->head_dim) * 2};
-  const cuuint32_t box[2] = {64, 16};
-  const cuuint32_t estr[2] = {1, 1};
-  const CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                        CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-  if (r != CUDA_SUCCESS) { mepic_set_error("prefill: cuTensorMapEncodeTiled failed with code %d", static_cast<int>(r)); return MEPIC_E_CUDA; }
-  return MEPIC_OK;
-}
-
 }  // namespace
 
 extern "C" size_t mepic_attn_prefill_workspace(const mepic_config_t* cfg, int32_t batch, const int32_t* row_offsets_host) {
@@ -817,9 +782,9 @@ extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_pre
   if (items.empty() || total_rows == 0) return MEPIC_OK;      // nothing to recompute
   if (a->workspace_bytes < items.size() * sizeof(Item)) { mepic_set_error("prefill: workspace too small"); return MEPIC_E_INVAL; }
   alignas(64) CUtensorMap map_k, map_v;
-  int32_t rc = make_pool_map(cfg, a->k_pool, &map_k);
+  int32_t rc = mepic_make_pool_map(cfg, a->k_pool, &map_k);
   if (rc != MEPIC_OK) return rc;
-  rc = make_pool_map(cfg, a->v_pool, &map_v);
+  rc = mepic_make_pool_map(cfg, a->v_pool, &map_v);
   if (rc != MEPIC_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   cudaError_t e = cudaMemcpyAsync(a->workspace, items.data(), items.size() * sizeof(Item), cudaMemcpyHostToDevice, st);
