@@ -194,6 +194,16 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
+__device__ __forceinline__ uint32_t bf16x2_mul(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
                ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
@@ -239,8 +249,10 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   }
   __syncwarp();
 
-  // cos/sin of the in-tile offsets this lane's B fragments cover: keys g and g+8, pairs 16j + 2t + 8r + {0,1}.
-  float kc[2][KH][2][2], ksn[2][KH][2][2];      // [key g / g+8][k-step][fragment register][element]
+  // cos/sin of the in-tile offsets this lane's B fragments cover: keys g and g+8, pairs 16j + 2t + 8r + {0,1},
+  // kept as packed bf16 pairs (cos, sin, -sin): the rotated K is rounded to bf16 for the MMA anyway, and packed
+  // bf16 arithmetic rotates two elements per instruction without widening them first.
+  uint32_t kc[2][KH][2], ksn[2][KH][2], kns[2][KH][2];      // [key g / g+8][k-step][fragment register]
 #pragma unroll
   for (int kq = 0; kq < 2; ++kq)
 #pragma unroll
@@ -248,7 +260,9 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
 #pragma unroll
       for (int r = 0; r < 2; ++r) {
         const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(g + 8 * kq) * D + 2 * (16 * j + 2 * t + 8 * r)));
-        kc[kq][j][r][0] = cs.x; ksn[kq][j][r][0] = cs.y; kc[kq][j][r][1] = cs.z; ksn[kq][j][r][1] = cs.w;
+        kc[kq][j][r] = pack_bf16x2(cs.x, cs.z);
+        ksn[kq][j][r] = pack_bf16x2(cs.y, cs.w);
+        kns[kq][j][r] = pack_bf16x2(-cs.y, -cs.w);
       }
 
   Cursor pc = locate(p.kv_len, p.batch, p.n_kv_heads, x0, lane);   // producer cursor
@@ -394,10 +408,9 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
 #pragma unroll
       for (int f = 0; f < 4; ++f) {
         const int kq = f >> 1, r = f & 1;       // key g + 8 kq, fragment register r
-        const float2 a = bf16x2_to_float2(lo[f]), b = bf16x2_to_float2(hi[f]);
-        const float c0 = kc[kq][j][r][0], sn0 = ksn[kq][j][r][0], c1 = kc[kq][j][r][1], sn1 = ksn[kq][j][r][1];
-        lo[f] = pack_bf16x2(fmaf(a.x, c0, -(b.x * sn0)), fmaf(a.y, c1, -(b.y * sn1)));
-        hi[f] = pack_bf16x2(fmaf(a.x, sn0, b.x * c0), fmaf(a.y, sn1, b.y * c1));
+        const uint32_t a = lo[f], b = hi[f];
+        lo[f] = bf16x2_fma(a, kc[kq][j][r], bf16x2_mul(b, kns[kq][j][r]));     // lo cos - hi sin
+        hi[f] = bf16x2_fma(a, ksn[kq][j][r], bf16x2_mul(b, kc[kq][j][r]));     // lo sin + hi cos
       }
       mma_bf16(s0, qa[j][0], 0u, qa[j][1], 0u, lo[0], lo[1]);
       mma_bf16(s1, qa[j][0], 0u, qa[j][1], 0u, lo[2], lo[3]);
