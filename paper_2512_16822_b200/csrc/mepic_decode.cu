@@ -227,9 +227,11 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   const int lane = threadIdx.x & 31;
   const int wic = threadIdx.x >> 5;
   unsigned char* stage0 = smem + static_cast<size_t>(wic) * kWarpBytes;
-  unsigned char* misc = smem + static_cast<size_t>(kWarps) * kWarpBytes + wic * 64;
+  // after the K/V rings: per warp, per stage, the cos/sin table row the tile's query rotation needs (D floats)
+  float* rope_rows = reinterpret_cast<float*>(smem + static_cast<size_t>(kWarps) * kWarpBytes) + static_cast<size_t>(wic) * kStages * D;
+  unsigned char* misc = smem + static_cast<size_t>(kWarps) * (kWarpBytes + kStages * D * 4) + wic * 64;
   uint64_t* bars = reinterpret_cast<uint64_t*>(misc);                 // kStages x 8 bytes
-  volatile int* meta = reinterpret_cast<volatile int*>(misc + 32);    // tile position base per stage
+  volatile float* meta = reinterpret_cast<volatile float*>(misc + 32);  // per stage: sign of (query position - tile base)
 
   const int g = lane >> 2;       // fragment row group: head g (A, C) / key g (B)
   const int t = lane & 3;        // fragment column group
@@ -268,11 +270,13 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   Cursor pc = locate(p.kv_len, p.batch, p.n_kv_heads, x0, lane);   // producer cursor
   Cursor cc = pc;                                                  // consumer cursor
   int win_b = -1, win_e0 = 0, win_page = 0, win_pos = 0;           // 32 block-table entries, one per lane
+  int win_qpos = 0;                                                // query position of the window's request
 
   auto issue = [&](int stage) {
     const int e = pc.t >> p.log2_tpp;
     const int sub = pc.t & ((1 << p.log2_tpp) - 1);
     if (pc.b != win_b || e < win_e0 || e >= win_e0 + 32) {
+      if (pc.b != win_b) win_qpos = __ldg(p.q_pos + pc.b);
       win_b = pc.b; win_e0 = e;
       const int n_ent = (pc.kvl + p.page_size - 1) / p.page_size;
       const bool ok = e + lane < n_ent;
@@ -287,13 +291,18 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
       const int y = (page * p.n_kv_heads + pc.h) * p.page_size + sub * kTile;     // row of the pool viewed as [rows][D]
       const uint32_t bar = smem_u32(&bars[stage]);
       const uint32_t dst = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
-      meta[stage] = pos + sub * kTile;
-      mbar_expect_tx(bar, kStageBytes);
+      // the query is rotated by (its position - tile base): that table row travels with the tile
+      const int rel = win_qpos - (pos + sub * kTile);
+      int arel = rel < 0 ? -rel : rel;
+      if (arel > p.max_position) { atomicOr(p.status, MEPIC_DEV_BAD_POSITION); arel = p.max_position; }
+      meta[stage] = rel < 0 ? -1.f : 1.f;
+      mbar_expect_tx(bar, kStageBytes + D * 4);
 #pragma unroll
       for (int nb = 0; nb < NB; ++nb) {
         tma_load_2d(dst + nb * kBlockBytes, &map_k, nb * 64, y, bar);
         tma_load_2d(dst + (NB + nb) * kBlockBytes, &map_v, nb * 64, y, bar);
       }
+      bulk_g2s(smem_u32(rope_rows + stage * D), p.rope + static_cast<size_t>(arel) * D, D * 4, bar);
     }
     advance(pc, p.kv_len, p.batch, p.n_kv_heads);
   };
@@ -302,7 +311,7 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   for (; issued < kStages && issued < n_tiles; ++issued) issue(issued);
 
   // per-unit state: head g of the unit's G query heads (lanes with g >= G carry zeros)
-  int ub = -1, uh = -1, qpos = 0;
+  int ub = -1, uh = -1;
   float q_lo[KH][2][2], q_hi[KH][2][2];     // un-rotated q, pre-scaled by sm_scale*log2e: pairs as for kc/ksn
   float m_run = -INFINITY, l_run = 0.f;
   float acc[ND][4];                         // O fragments: [n-tile][c0,c1 = head g | c2,c3 = head g+8 (unused)]
@@ -327,7 +336,6 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
     if (cc.b != ub || cc.h != uh) {
       flush();
       ub = cc.b; uh = cc.h;
-      qpos = __ldg(p.q_pos + ub);
       const int n_q_heads = p.n_kv_heads * G;
       const uint32_t* src = reinterpret_cast<const uint32_t*>(
           p.q + (static_cast<size_t>(ub) * n_q_heads + static_cast<size_t>(uh) * G + (g < G ? g : 0)) * D);
@@ -347,13 +355,8 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
       for (int nd = 0; nd < ND; ++nd) { acc[nd][0] = 0.f; acc[nd][1] = 0.f; acc[nd][2] = 0.f; acc[nd][3] = 0.f; }
     }
 
-    // ---- A fragments of the query rotated by (qpos - tile base); the table row does not depend on the data, so
-    //      it is fetched before the wait for the tile
+    // ---- A fragments of the query rotated by (qpos - tile base), from the table row that came with the tile
     uint32_t qa[KS][2];                         // [k-step][a0 (dims 16j+2t,+1) | a2 (dims 16j+8+2t,+1)], row = head g
-    {
-      // meta is written by lane 0 before it arms the barrier; reading it needs the barrier's acquire, so the
-      // position comes after the wait - but the wait is short once the ring is primed.  Do the wait first.
-    }
     if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity)) {
       // Give the copies still in flight a last bounded chance to land, then leave cleanly.
       if (lane == 0) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
@@ -362,19 +365,15 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
     }
     const uint32_t ks_addr = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
     const uint32_t vs_addr = ks_addr + NB * kBlockBytes;
-    const int base = meta[stage];
+    const float sgn = meta[stage];
     const int n_valid = min(kTile, cc.kvl - cc.t * kTile);
     {
-      const int rel = qpos - base;
-      int arel = rel < 0 ? -rel : rel;
-      const float sgn = rel < 0 ? -1.f : 1.f;
-      if (arel > p.max_position) { if (lane == 0) atomicOr(p.status, MEPIC_DEV_BAD_POSITION); arel = p.max_position; }
-      const float* row = p.rope + static_cast<size_t>(arel) * D;
+      const float* row = rope_rows + stage * D;
 #pragma unroll
       for (int j = 0; j < KH; ++j)
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
-          const float4 cs = __ldg(reinterpret_cast<const float4*>(row + 2 * (16 * j + 2 * t + 8 * r)));
+          const float4 cs = *reinterpret_cast<const float4*>(row + 2 * (16 * j + 2 * t + 8 * r));
           const float c0 = cs.x, s0 = cs.y * sgn, c1 = cs.z, s1 = cs.w * sgn;
           const float l0 = q_lo[j][r][0] * c0 - q_hi[j][r][0] * s0, h0 = q_lo[j][r][0] * s0 + q_hi[j][r][0] * c0;
           const float l1 = q_lo[j][r][1] * c1 - q_hi[j][r][1] * s1, h1 = q_lo[j][r][1] * s1 + q_hi[j][r][1] * c1;
@@ -507,8 +506,8 @@ __global__ void mepic_decode_merge(const DecodeParams p) {
 
 template <int D, int G>
 constexpr size_t decode_smem_bytes() {
-  // per warp: 3 stages of (K blocks + V blocks); then 64 bytes of barriers and tile positions per warp; 1 KB alignment slack
-  return static_cast<size_t>(kWarps) * (3 * 2 * (D / 64) * kTile * 128) + kWarps * 64 + 1024;
+  // per warp: 3 stages of (K blocks + V blocks), 3 table rows, 64 bytes of barriers and flags; 1 KB alignment slack
+  return static_cast<size_t>(kWarps) * (3 * 2 * (D / 64) * kTile * 128 + 3 * D * 4) + kWarps * 64 + 1024;
 }
 
 template <int D, int G>
