@@ -190,6 +190,47 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def measure_unshared(args, wl, device_index: int):
+    """The same decode batch on a layout WITHOUT chunk sharing: every request owns a private copy of each of its
+    chunks (one page per block-table entry), so no page is read twice and nothing can be served from L2 because a
+    neighbour touched it.  Separates kernel quality from the cache effect of sharing."""
+    import torch
+    import paper_2512_16822_b200 as M
+    from paper_2512_16822_b200 import runtime as RT
+    P = wl.page_size
+    ents = [sum(-(-(len(wl.chunks[v]) if k == 0 else v) // P) for k, v in r.segments) for r in wl.decode_requests]
+    lens = [sum((len(wl.chunks[v]) if k == 0 else v) for k, v in r.segments) for r in wl.decode_requests]
+    num_pages = int(sum(ents))
+    cfg = M.Config(P, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, num_pages, wl.max_position, wl.rope_theta, wl.pad_token_id)
+    B, stride = len(ents), max(ents)
+    page_ids = np.zeros((B, stride), dtype=np.int32); pos_base = np.zeros((B, stride), dtype=np.int32)
+    perm = np.random.default_rng([0, wl.index, 99]).permutation(num_pages).astype(np.int32)
+    at = 0
+    for b, e in enumerate(ents):
+        page_ids[b, :e] = perm[at:at + e]; at += e
+        pos_base[b, :e] = np.arange(e) * P
+    kv_len = np.asarray(lens, dtype=np.int32)
+    q_pos = kv_len - 1
+    dev = RT.Device(cfg, device=f"cuda:{device_index}")
+    dev.k_pool.normal_(); dev.v_pool.normal_()             # values do not matter for timing; drawn on the device
+    batch = RT.DecodeBatch(dev, page_ids, pos_base, kv_len, q_pos, wl.decode_q())
+    stream = torch.cuda.current_stream()
+    flush_buf = torch.empty(512 << 20, dtype=torch.uint8, device=dev.device)
+    for _ in range(3):
+        batch.run(wl.sm_scale, stream)
+    steps = max(5, min(args.steps, 50))
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        flush_buf.fill_(1)
+        a.record(stream); batch.run(wl.sm_scale, stream); b.record(stream)
+    torch.cuda.synchronize()
+    assert dev.read_status() == 0
+    ms = sum(a.elapsed_time(b) for a, b in evs) / steps
+    nbytes = int(kv_len.astype(np.int64).sum()) * kv_bytes_per_token(wl)
+    return {"value": nbytes / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms, "pages_held": num_pages,
+            "note": "no chunk sharing: logical bytes = unique bytes; L2 flushed between steps"}
+
+
 def measure_prefill(args, device_index: int):
     """Config 3 (first-block recompute prefill): one step = one mepic_attn_prefill call (commit + attention)."""
     import torch
@@ -331,9 +372,11 @@ def run_ours(args):
         return float(t.item())
 
     tot, tot_warm, tot_e2e = agg(ms), agg(ms_warm), agg(ms_e2e)
-    prefill = None
+    prefill = unshared = None
     if rank == 0 and world == 1 and not args.no_prefill:
         prefill = measure_prefill(args, local_rank)
+    if rank == 0 and world == 1 and not args.no_unshared:
+        unshared = measure_unshared(args, wl, local_rank)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -366,6 +409,7 @@ def run_ours(args):
                   "unshared_equivalent": stats["unshared_equivalent_pages"], "dedup_hits": stats["dedup_hits"]},
         "table_build_ms": table_build_ms,
         "prefill": prefill,
+        "unshared_layout": unshared,
     }
     if not args.no_cpu_baseline and world == 1:
         s = oracle_decode_sample(wl, args.cpu_budget)
@@ -390,6 +434,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true", help="skip the config-3 prefill measurement")
+    ap.add_argument("--no-unshared", action="store_true", help="skip the decode run on the layout without sharing")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
