@@ -39,8 +39,8 @@ from mepic_inputs import make_workload  # noqa: E402
 
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one mepic_decode_splitkv launch (ncu, see profiles/);
-# None until a capture of that workload exists.
-NCU_TRAFFIC_BYTES = {2: None}
+# config 2: 358.9 MB read + 4.1 MB written (profiles/decode_splitkv_config2.md).
+NCU_TRAFFIC_BYTES = {2: 362_957_000}
 
 
 def kv_bytes_per_token(wl) -> int:
