@@ -101,6 +101,21 @@ __device__ __forceinline__ float2 add2(float2 a, float2 b) {
       : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
   return d;
 }
+__device__ __forceinline__ uint32_t bf16x2_mul(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf16x2_sub(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
 // (lo, hi) -> packed bf16x2, round to nearest even
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
@@ -561,11 +576,11 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         uint32_t lo_w[4], hi_w[4];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-          const float2 a = bf16x2_to_float2(lw[j]), bq = bf16x2_to_float2(hw[j]);
-          const float2 nl = sub2(mul2(a, cc[j]), mul2(bq, ss[j]));
-          const float2 nh = fma2(a, ss[j], mul2(bq, cc[j]));
-          lo_w[j] = pack_bf16x2(nl.x, nl.y);
-          hi_w[j] = pack_bf16x2(nh.x, nh.y);
+          // packed bf16 arithmetic: the result is rounded to bf16 for the MMA anyway, and two elements rotate per
+          // instruction without being widened first; cos/sin are carried in fp32 and rounded once per key
+          const uint32_t cb = pack_bf16x2(cc[j].x, cc[j].y), sb = pack_bf16x2(ss[j].x, ss[j].y);
+          lo_w[j] = bf16x2_sub(bf16x2_mul(lw[j], cb), bf16x2_mul(hw[j], sb));      // lo cos - hi sin
+          hi_w[j] = bf16x2_fma(lw[j], sb, bf16x2_mul(hw[j], cb));                  // lo sin + hi cos
         }
         *plo = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
         *phi = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
