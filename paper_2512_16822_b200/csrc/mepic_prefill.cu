@@ -43,9 +43,10 @@ namespace {
 constexpr int kTileN = 128;            // keys per staged tile
 constexpr int kBlockBytes = 128 * 128; // one [128 rows x 64 bf16] swizzled block
 constexpr int kTmemCols = 512;         // S of M-tile a: 0..127, of b: 128..255; O of a: 256.., of b: 384..
-constexpr int kSoftmaxWarps = 4, kRotatorWarps = 4;
-constexpr int kKLoaderWarp = 12, kVLoaderWarp = 13, kMmaWarp = 14;   // warp 15 idles: 16 warps keep the register split even
-constexpr int kThreads = 512;
+constexpr int kSoftmaxWarps = 16;       // 2 M-tiles x 2 column halves x 4 lane quadrants: two threads share a row
+constexpr int kRotatorWarps = 4;
+constexpr int kKLoaderWarp = 20, kVLoaderWarp = 21, kMmaWarp = 22;   // warp 23 idles
+constexpr int kThreads = 768;
 constexpr int kSpinLimit = 1 << 22;
 constexpr float kRescaleThreshold = 8.f;   // move the reference maximum only when it lags by 2^8
 
@@ -263,7 +264,8 @@ struct PrefillSmem {
   static constexpr int kQ = 0;                                     // two M-tiles of Q'
   static constexpr int kK = kQ + 2 * NB * kBlockBytes;
   static constexpr int kV = kK + kKStages * NB * kBlockBytes;
-  static constexpr int kBars = kV + kVStages * NB * kBlockBytes;   // mbarriers and small state
+  static constexpr int kXchg = kV + kVStages * NB * kBlockBytes;   // float [2 M-tiles][2 halves][128 rows]: row-half exchange
+  static constexpr int kBars = kXchg + 2 * 2 * 128 * 4;            // mbarriers and small state
   static constexpr int kBytes = kBars + 512;
 };
 
@@ -277,7 +279,8 @@ constexpr int kBarSFull = kBarVFree + kVStages;         // [2 M-tiles] S of the 
 constexpr int kBarPFull = kBarSFull + 2;                // [2] P of the current tile is in tensor memory
 constexpr int kBarPvDone = kBarPFull + 2;               // [2] PV of the current tile complete
 constexpr int kBarVPatched = kBarPvDone + 2;            // [1] rows past kv_len of the last V tile zeroed
-constexpr int kNumBars = kBarVPatched + 1;
+constexpr int kBarPair = kBarVPatched + 1;              // [2 M-tiles][4 quadrants] the two warps that share 32 rows
+constexpr int kNumBars = kBarPair + 8;
 
 template <int D, int G>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -290,12 +293,13 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   constexpr uint32_t kIdescPV = instr_desc(128, D, 0, 1);
   constexpr uint32_t kGroupBytes = 16u * D * 2u;        // the rows of one 16-token group in one pool
 
-  extern __shared__ unsigned char smem_dyn[];
-  // 1024-byte alignment: the swizzle pattern is a function of the address bits
-  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~static_cast<uintptr_t>(1023));
+  // 1024-byte alignment: the swizzle pattern is a function of the address bits (checked below; there is no slack left)
+  extern __shared__ __align__(1024) unsigned char smem_dyn[];
+  unsigned char* smem = smem_dyn;
   unsigned char* Qs = smem + L::kQ;
   unsigned char* Ks = smem + L::kK;
   unsigned char* Vs = smem + L::kV;
+  float* xchg = reinterpret_cast<float*>(smem + L::kXchg);
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::kBars);
   const uint32_t bar0 = smem_u32(bars);
   auto BAR = [&](int which, int slot) { return bar0 + static_cast<uint32_t>((which + slot) * 8); };
@@ -311,6 +315,10 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   const int32_t* bases = p.pos_base + static_cast<size_t>(b) * p.table_stride;
   const int n_q_heads = p.n_kv_heads * G;
 
+  if ((smem_u32(smem) & 1023u) != 0) {       // cannot happen with the alignment requested above; never run misaligned
+    if (tid == 0) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
+    return;
+  }
   if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
   if (tid == 32) {
     for (int s = 0; s < kKStages; ++s) {
@@ -324,10 +332,11 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(BAR(kBarSFull, s), 1);                       // tcgen05.commit
-      mbar_init(BAR(kBarPFull, s), 128);                     // the M-tile's softmax warpgroup
+      mbar_init(BAR(kBarPFull, s), 256);                     // the M-tile's two softmax warpgroups
       mbar_init(BAR(kBarPvDone, s), 1);                      // tcgen05.commit
     }
     mbar_init(BAR(kBarVPatched, 0), 1);
+    for (int s = 0; s < 8; ++s) mbar_init(BAR(kBarPair, s), 64);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -386,13 +395,18 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  if (warp < 2 * kSoftmaxWarps) {
-    // =============================================================== softmax warpgroups: one per M-tile, thread = row
-    const int x = warp / kSoftmaxWarps;
-    const uint32_t t_row = tmem_base + (static_cast<uint32_t>((warp % 4) * 32) << 16);
-    const uint32_t t_S = t_row + static_cast<uint32_t>(x * 128);       // S of this M-tile; P overwrites its first 64 columns
-    const uint32_t t_O = t_row + 256u + static_cast<uint32_t>(x * 128);
-    const int r = tid & 127;
+  if (warp < kSoftmaxWarps) {
+    // =============================================================== softmax warps
+    // Row r of M-tile x is shared by two threads (same tensor-memory lane, warps w and w + 4 of the M-tile's
+    // eight): one takes the scores of keys 0..63 of the tile, the other keys 64..127.  They agree on the row's
+    // reference maximum through shared memory once per tile; everything else is private.
+    const int x = warp >> 3;                      // M-tile
+    const int ch = (warp >> 2) & 1;               // column half
+    const int q4 = warp & 3;                      // lane quadrant of tensor memory
+    const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q4 * 32) << 16);
+    const uint32_t t_H = t_row + static_cast<uint32_t>(x * 128 + ch * 64);     // my 64 score columns; P goes over the first 32
+    const uint32_t t_O = t_row + 256u + static_cast<uint32_t>(x * 128 + ch * (D / 2));   // my half of the row's O columns
+    const int r = q4 * 32 + lane;
     const int qi = x * QT + r / G, g = r % G;
     const bool row_live = (r < QT * G) && (qi < item.nq);
     int limit = lim[x];
@@ -400,31 +414,78 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       limit = p.q_slot[item.row0 + qi];
       if (limit < 0 || limit >= kvl) { atomicOr(p.status, MEPIC_DEV_BAD_SLOT); limit = limit < 0 ? 0 : kvl - 1; }
     }
+    float* mine = xchg + (x * 2 + ch) * 128 + r;
+    const float* theirs = xchg + (x * 2 + (ch ^ 1)) * 128 + r;
+    const uint32_t pair_bar = BAR(kBarPair, x * 4 + q4);
+    uint32_t pair_ph = 0;
+    // publish `v`, wait for the partner warp, return the partner's value of the same row
+    auto swap_with_partner = [&](float v, bool& ok_io) {
+      *mine = v;
+      mbar_arrive(pair_bar);
+      if (!mbar_wait_warp(pair_bar, pair_ph, abort_flag, p.status)) ok_io = false;
+      pair_ph ^= 1u;
+      return *theirs;
+    };
     float m_ref = -INFINITY, l_run = 0.f;
     bool ok = true;
     const int my_tiles = nt[x];
     for (int tile = 0; tile < my_tiles; ++tile) {
       if (!mbar_wait_warp(BAR(kBarSFull, x), static_cast<uint32_t>(tile) & 1u, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
-      const int n_vis = limit - tile * kTileN + 1;          // columns [0, n_vis) are visible to this row
-      const bool boundary = n_vis < kTileN;                 // only the tile(s) on the causal boundary need the mask
-      // One 32-column chunk: mask; if its maximum is more than 2^8 above the reference, move the reference
-      // to it (so no exponent ever exceeds 2^8); P = 2^(S - ref) as bf16 pairs; row sum of the chunk.
-      auto chunk = [&](uint32_t (&sv)[32], int col0, float& ref, float& sum_out, uint32_t (&pw)[16]) {
+      const int n_vis = limit - tile * kTileN + 1 - 64 * ch;     // my columns [0, n_vis) are visible to this row
+      const bool boundary = n_vis < 64;                          // only the tile(s) on the causal boundary need the mask
+      // ---- pass 1: maximum of my 64 scores
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll 1
+      for (int q = 0; q < 2; ++q) {
+        uint32_t sv[32];
+        TMEM_LD32(t_H + 32 * q, sv, 0);
+        tmem_wait_ld();
         if (boundary) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) sv[c] = (col0 + c) < n_vis ? sv[c] : 0xff800000u;   // -inf -> P = 0
+          for (int c = 0; c < 32; ++c) sv[c] = (32 * q + c) < n_vis ? sv[c] : 0xff800000u;   // -inf
         }
-        float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
         for (int c = 0; c < 32; c += 4) {
 #pragma unroll
           for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(mx4[k], __uint_as_float(sv[c + k]));
         }
-        const float cm = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-        if (cm > ref + kRescaleThreshold) ref = cm;      // first chunk of the first tile: ref = -inf, key 0 is visible
-        const float2 ref2 = make_float2(ref, ref);
-        float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      }
+      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
+      mx = fmaxf(mx, swap_with_partner(mx, ok));
+      if (!ok) break;
+      // move the reference only when it lags by more than the threshold (both threads of the row decide alike);
+      // always true on the first tile: m_ref = -inf and key 0 is visible to every row
+      float alpha = 1.f;
+      if (mx > m_ref + kRescaleThreshold) {
+        alpha = ex2(m_ref - mx);
+        m_ref = mx;
+      }
+      // O holds every earlier tile's PV, all complete: this tile's S was issued after them.  Each thread of the
+      // row rescales its own half of the O columns.
+      if (tile > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+        for (int cb = 0; cb < D / 2; cb += 32) {
+          uint32_t o[32];
+          TMEM_LD32(t_O + cb, o, 0);
+          tmem_wait_ld();
+#pragma unroll
+          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
+          TMEM_ST32(t_O + cb, o, 0);
+        }
+      }
+      // ---- pass 2: P = 2^(S - reference) as bf16 pairs over the first 32 of my 64 columns
+      float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
+      const float2 ref2 = make_float2(m_ref, m_ref);
+#pragma unroll 1
+      for (int q = 0; q < 2; ++q) {
+        uint32_t sv[32], pw[16];
+        TMEM_LD32(t_H + 32 * q, sv, 0);
+        tmem_wait_ld();
+        if (boundary) {
+#pragma unroll
+          for (int c = 0; c < 32; ++c) sv[c] = (32 * q + c) < n_vis ? sv[c] : 0xff800000u;   // -inf -> P = 0
+        }
 #pragma unroll
         for (int c = 0; c < 32; c += 4) {
           const float2 d0 = sub2(make_float2(__uint_as_float(sv[c]), __uint_as_float(sv[c + 1])), ref2);
@@ -435,84 +496,23 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
           pw[c / 2] = pack_bf16x2(p0.x, p0.y);
           pw[c / 2 + 1] = pack_bf16x2(p1.x, p1.y);
         }
-        sum_out = (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
-      };
-      // One pass over the tile; loads run one chunk ahead of the arithmetic.  P chunk q goes to columns
-      // [16q, 16q+16) of the S buffer, which by then only holds S columns that have been consumed.
-      float ref = m_ref, ref_at[4] = {0.f, 0.f, 0.f, 0.f}, sum_q[4] = {0.f, 0.f, 0.f, 0.f};
-      {
-        uint32_t sa[32], sb[32], pw[16];
-        TMEM_LD32(t_S, sa, 0);
-#pragma unroll 1
-        for (int hq = 0; hq < 2; ++hq) {
-          float sum_a, sum_b;
-          tmem_wait_ld();
-          TMEM_LD32(t_S + 64 * hq + 32, sb, 0);
-          chunk(sa, 64 * hq, ref, sum_a, pw);
-          const float ref_a = ref;
-          tmem_wait_ld();                         // sb has landed (and every earlier load)
-          if (hq == 0) TMEM_LD32(t_S + 64, sa, 0);
-          TMEM_ST16(t_S + 32 * hq, pw);
-          chunk(sb, 64 * hq + 32, ref, sum_b, pw);
-          TMEM_ST16(t_S + 32 * hq + 16, pw);
-          // static indices only (the loop is kept rolled to keep the code small): select by hq
-          ref_at[0] = hq == 0 ? ref_a : ref_at[0]; ref_at[1] = hq == 0 ? ref : ref_at[1];
-          ref_at[2] = hq == 1 ? ref_a : ref_at[2]; ref_at[3] = hq == 1 ? ref : ref_at[3];
-          sum_q[0] = hq == 0 ? sum_a : sum_q[0]; sum_q[1] = hq == 0 ? sum_b : sum_q[1];
-          sum_q[2] = hq == 1 ? sum_a : sum_q[2]; sum_q[3] = hq == 1 ? sum_b : sum_q[3];
-        }
+        TMEM_ST16(t_H + 16 * q, pw);      // chunk q's P over columns that hold only consumed scores
       }
-      // Bring everything to the final reference.  Common case: the reference did not move and nothing is touched.
-      const float alpha = ex2(m_ref - ref);       // 1 when unchanged; 0 on the first tile (m_ref = -inf)
-      float sum = sum_q[3];
-#pragma unroll
-      for (int q = 0; q < 3; ++q) sum += sum_q[q] * ex2(ref_at[q] - ref);
-      if (tile > 0 && __any_sync(0xffffffffu, ref != m_ref)) {
-        // O holds the sum up to the previous tile, whose PV is complete: this tile's S, issued after it, exists
-#pragma unroll 1
-        for (int cb = 0; cb < D; cb += 32) {
-          uint32_t o[32];
-          TMEM_LD32(t_O + cb, o, 0);
-          tmem_wait_ld();
-#pragma unroll
-          for (int c = 0; c < 32; ++c) o[c] = __float_as_uint(__uint_as_float(o[c]) * alpha);
-          TMEM_ST32(t_O + cb, o, 0);
-        }
-      }
-      if (__any_sync(0xffffffffu, ref_at[0] != ref)) {
-        // the reference moved inside the tile: P chunks written before the move are scaled down to it
-#pragma unroll
-        for (int q = 0; q < 3; ++q) {
-          const float f = ex2(ref_at[q] - ref);
-          uint32_t pw[16];
-          asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-                       : "=r"(pw[0]), "=r"(pw[1]), "=r"(pw[2]), "=r"(pw[3]), "=r"(pw[4]), "=r"(pw[5]), "=r"(pw[6]), "=r"(pw[7]),
-                         "=r"(pw[8]), "=r"(pw[9]), "=r"(pw[10]), "=r"(pw[11]), "=r"(pw[12]), "=r"(pw[13]), "=r"(pw[14]), "=r"(pw[15])
-                       : "r"(t_S + 16 * q) : "memory");
-          tmem_wait_ld();
-#pragma unroll
-          for (int c = 0; c < 16; ++c) {
-            const float2 v = bf16x2_to_float2(pw[c]);
-            pw[c] = pack_bf16x2(v.x * f, v.y * f);
-          }
-          TMEM_ST16(t_S + 16 * q, pw);
-        }
-      }
-      l_run = l_run * alpha + sum;
-      m_ref = ref;
+      l_run = l_run * alpha + (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(BAR(kBarPFull, x));
     }
-    // ---- epilogue: out = O / l once the last PV has completed
+    // ---- epilogue: out = O / l once the last PV has completed; each thread of the row writes half of it
     if (ok && my_tiles > 0) {
-      ok = mbar_wait_warp(BAR(kBarPvDone, x), static_cast<uint32_t>(my_tiles - 1) & 1u, abort_flag, p.status);
+      const float l_tot = l_run + swap_with_partner(l_run, ok);
+      if (ok) ok = mbar_wait_warp(BAR(kBarPvDone, x), static_cast<uint32_t>(my_tiles - 1) & 1u, abort_flag, p.status);
       if (ok) {
         tc_fence_after();
-        const float inv = 1.f / l_run;
-        uint16_t* dst = p.out + (static_cast<size_t>(item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g) * D;
-#pragma unroll
-        for (int cb = 0; cb < D; cb += 32) {
+        const float inv = 1.f / l_tot;
+        uint16_t* dst = p.out + (static_cast<size_t>(item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g) * D + ch * (D / 2);
+#pragma unroll 1
+        for (int cb = 0; cb < D / 2; cb += 32) {
           uint32_t o[32];
           TMEM_LD32(t_O + cb, o, 0);
           tmem_wait_ld();
@@ -530,9 +530,9 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         }
       }
     }
-  } else if (warp < 2 * kSoftmaxWarps + kRotatorWarps) {
+  } else if (warp < kSoftmaxWarps + kRotatorWarps) {
     // =============================================================== rotator warps: K tile, in place
-    const int rt = tid - 2 * kSoftmaxWarps * 32;     // 0..127
+    const int rt = tid - kSoftmaxWarps * 32;     // 0..127
     const int c = rt % CH;                       // chunk pair: dims [8c, 8c+8) and [D/2+8c, ...)
     const int k0 = (rt / CH) * CH;               // first of this thread's CH consecutive keys
     // one-position step of this chunk's 8 pairs: table row 1, as packed pairs (cos, sin, -sin)
@@ -670,8 +670,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       const uint32_t v_addr = smem_u32(Vs + (j % kVStages) * NB * kBlockBytes);
 #pragma unroll
       for (int ks = 0; ks < kTileN / 16; ++ks) {
-        // A = P from tensor memory: 16 bf16 per k-step = 8 columns; B = V, MN-major
-        tc_mma_ts(tmem_base + 256u + static_cast<uint32_t>(x * 128), tmem_base + static_cast<uint32_t>(x * 128 + ks * 8),
+        // A = P from tensor memory: 16 bf16 per k-step = 8 columns, keys 0..63 at columns 0.., keys 64..127 at 64..; B = V, MN-major
+        tc_mma_ts(tmem_base + 256u + static_cast<uint32_t>(x * 128), tmem_base + static_cast<uint32_t>(x * 128 + (ks / 4) * 64 + (ks % 4) * 8),
                   smem_desc(v_addr + ks * 2048, kBlockBytes, 1024), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
       }
       tc_commit(BAR(kBarPvDone, x));
@@ -737,7 +737,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
 
 template <int D, int G>
 int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
-  constexpr size_t smem = PrefillSmem<D>::kBytes + 1024;
+  constexpr size_t smem = PrefillSmem<D>::kBytes;
   cudaError_t e = cudaFuncSetAttribute(mepic_prefill_attn<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("prefill: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   const int chunks_per_row = p.n_kv_heads * D / 8;
