@@ -6,19 +6,22 @@
 // the (request, kv head, tile) triples of the whole batch are laid on one line
 // in that order and cut into equal contiguous pieces, one per WARP of a
 // persistent grid (one CTA per SM, 8 warps).  A warp is a self-contained
-// worker: it owns a ring of shared-memory stages that bulk-async copies
-// (cp.async.bulk + mbarrier complete_tx) fill with the 16 x D K tile and V tile
-// of its next tiles, and it keeps one online-softmax state per query head of
-// the kv head it is on.  When its piece crosses into another (request, head)
-// unit, or ends, it writes a partial (max, sum, weighted V) for the unit; a
-// second kernel merges the partials of each unit.  Equal pieces balance the
-// ragged batches; no warp ever waits on another warp.
+// worker: it owns a ring of shared-memory stages that TMA tensor copies
+// (cp.async.bulk.tensor + mbarrier complete_tx, 128-byte swizzle) fill with the
+// K tile and V tile of its next tiles, together with the one row of the cos/sin
+// table the tile's query rotation needs, and it keeps one online-softmax state
+// per query head of the kv head it is on.  When its piece crosses into another
+// (request, head) unit, or ends, it writes a partial (max, sum, weighted V) for
+// the unit; a second kernel merges the partials of each unit.  Equal pieces
+// balance ragged batches; no warp ever waits on another warp.
 //
-// Rotation.  <R(qpos) q, R(base+tau) k> = <R(qpos-base) q, R(tau) k>: per tile
-// the warp rotates the G query vectors by (qpos - tile base) from one row of
-// the cos/sin table, and rotates every key only by its offset tau < 16 inside
-// the tile, with cos/sin of those 16 offsets held in registers for the whole
-// kernel.  Keys are rotated in registers in fp32 and never written back.
+// Arithmetic.  <R(qpos) q, R(base+tau) k> = <R(qpos-base) q, R(tau) k>: per tile
+// the G query vectors are rotated by (qpos - tile base) in fp32 and rounded to
+// bf16, and every key only by its offset tau < 16 inside the tile, with cos/sin
+// of those 16 offsets held in registers for the whole kernel.  Both contractions
+// of a tile run on the tensor cores (mma.sync m16n8k16, fp32 accumulate); the K
+// rotation is applied to the MMA's B fragments in registers (packed bf16), so
+// rotated keys never touch shared or global memory.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -32,8 +35,6 @@ namespace {
 
 constexpr int kTile = 16;      // tokens per staged tile
 constexpr int kWarps = 8;      // workers per CTA
-// ring depth per worker: 3 stages, 2 where the per-warp buffers of a large group would not fit
-__host__ __device__ constexpr int stages_for(int D, int G) { return G * D > 640 ? 2 : 3; }
 constexpr int kMinPiece = 4;   // never cut the line into pieces shorter than this many tiles
 constexpr unsigned kFull = 0xffffffffu;
 constexpr int kSpinLimit = 1 << 22;
@@ -58,25 +59,6 @@ struct DecodeParams {
 // ---------------------------------------------------------------- small PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
 
-__device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
-  float2 d;
-  asm("{ .reg .b64 ra, rb, rc, rd;\n mov.b64 ra, {%2,%3};\n mov.b64 rb, {%4,%5};\n mov.b64 rc, {%6,%7};\n"
-      " fma.rn.f32x2 rd, ra, rb, rc;\n mov.b64 {%0,%1}, rd; }"
-      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
-  return d;
-}
-__device__ __forceinline__ float2 mul2(float2 a, float2 b) {
-  float2 d;
-  asm("{ .reg .b64 ra, rb, rd;\n mov.b64 ra, {%2,%3};\n mov.b64 rb, {%4,%5};\n mul.rn.f32x2 rd, ra, rb;\n mov.b64 {%0,%1}, rd; }"
-      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
-  return d;
-}
-__device__ __forceinline__ float2 sub2(float2 a, float2 b) {
-  float2 d;
-  asm("{ .reg .b64 ra, rb, rd;\n mov.b64 ra, {%2,%3};\n mov.b64 rb, {%4,%5};\n sub.rn.f32x2 rd, ra, rb;\n mov.b64 {%0,%1}, rd; }"
-      : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
-  return d;
-}
 // two bf16 packed in a 32-bit word (low half = even element) -> two floats, exactly
 __device__ __forceinline__ float2 bf16x2_to_float2(uint32_t w) {
   return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
