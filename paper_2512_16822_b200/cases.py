@@ -1,0 +1,71 @@
+"""Run one benchmark configuration through the public binding and print the device time.
+
+    python -m paper_2512_16822_b200.cases decode  --config 2 [--scale 1.0] [--iters 10]
+    python -m paper_2512_16822_b200.cases prefill --config 3 [--scale 0.5] [--iters 4]
+
+A small driver for profiling (a fixed, short sequence of calls that a profiler can capture) and for trying the
+library on the synthetic workloads.  Inputs come from ``mepic_inputs``; nothing here checks results (the tests do).
+"""
+from __future__ import annotations
+
+import argparse
+import os
+import sys
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+
+def _setup(index: int, scale: float, which: str):
+    import paper_2512_16822_b200 as M
+    from paper_2512_16822_b200 import runtime as RT
+    from mepic_inputs import make_workload
+    wl = make_workload(index, scale=scale)
+    cfg = M.Config(wl.page_size, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.num_pages, wl.max_position,
+                   wl.rope_theta, wl.pad_token_id)
+    kp, vp = wl.kv_pool()
+    with M.Store(cfg) as st:
+        dec = RT.build_tables(st, wl.chunks, wl.decode_requests) if wl.decode_requests else []
+        pre = RT.build_tables(st, wl.chunks, wl.prefill_requests) if wl.prefill_requests else []
+    dev = RT.Device(cfg, kp, vp)
+    if which == "decode":
+        if not dec:
+            raise SystemExit(f"config {index} has no decode requests")
+        page_ids, pos_base, kv_len, q_pos = RT.pack_tables(dec, wl.page_size)
+        return wl, dev, RT.DecodeBatch(dev, page_ids, pos_base, kv_len, q_pos, wl.decode_q())
+    if not pre:
+        raise SystemExit(f"config {index} has no prefill requests")
+    page_ids, pos_base, kv_len, _ = RT.pack_tables(pre, wl.page_size)
+    slots = [t.recompute_slots for t in pre]
+    rows = [wl.prefill_rows(i, len(s)) for i, s in enumerate(slots)]
+    ro = np.concatenate([[0], np.cumsum([len(s) for s in slots])]).astype(np.int32)
+    batch = RT.PrefillBatch(dev, page_ids, pos_base, kv_len, ro, np.concatenate(slots).astype(np.int32),
+                            np.concatenate([r.q_new for r in rows]), np.concatenate([r.k_new for r in rows]),
+                            np.concatenate([r.v_new for r in rows]))
+    return wl, dev, batch
+
+
+def main() -> None:
+    import torch
+    ap = argparse.ArgumentParser()
+    ap.add_argument("which", choices=["decode", "prefill"])
+    ap.add_argument("--config", type=int, default=None)
+    ap.add_argument("--scale", type=float, default=1.0)
+    ap.add_argument("--iters", type=int, default=4)
+    args = ap.parse_args()
+    index = args.config if args.config is not None else (2 if args.which == "decode" else 3)
+    wl, dev, batch = _setup(index, args.scale, args.which)
+    for _ in range(max(args.iters - 1, 1)):
+        batch.run(wl.sm_scale)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(); batch.run(wl.sm_scale); e1.record()
+    torch.cuda.synchronize()
+    print(f"{args.which} config {index} scale {args.scale}: {e0.elapsed_time(e1):.4f} ms, device status {dev.read_status()}")
+
+
+if __name__ == "__main__":
+    main()
