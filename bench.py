@@ -277,6 +277,21 @@ def measure_prefill(args, device_index: int):
                          "kernel": "mepic_prefill_attn (+ commit kernel: the C-ABI call is timed as a whole)"}}
 
 
+def max_over_ranks(total_ms: float, world: int, device) -> float:
+    """The slowest rank's time: every multi-GPU number is the job's bytes over this."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([total_ms], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_gbs(world: int, steps: int, bytes_per_rank_step: int, total_ms: float) -> float:
+    """Whole-job throughput: all ranks' bytes (replicas, weak scaling) over the slowest rank's time."""
+    return world * steps * bytes_per_rank_step / (total_ms * 1e-3) / 1e9
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -366,10 +381,7 @@ def run_ours(args):
     assert dev.read_status() == 0, "device status word is not clean"
 
     def agg(xs):
-        t = torch.tensor([sum(xs)], dtype=torch.float64, device=dev.device)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return max_over_ranks(sum(xs), world, dev.device)
 
     tot, tot_warm, tot_e2e = agg(ms), agg(ms_warm), agg(ms_e2e)
     prefill = unshared = None
@@ -381,7 +393,7 @@ def run_ours(args):
         if world > 1:
             dist.destroy_process_group()
         return
-    gbs = lambda total_ms: world * args.steps * logical_bytes / (total_ms * 1e-3) / 1e9
+    gbs = lambda total_ms: aggregate_gbs(world, args.steps, logical_bytes, total_ms)
     peak, peak_src, _ = measured_peaks()
     per_launch_ms = sum(ms) / len(ms)
     achieved = logical_bytes / (per_launch_ms * 1e-3) / 1e9

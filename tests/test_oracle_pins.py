@@ -437,3 +437,36 @@ def test_negative_controls_exceed_tolerance_on_benchmark_statistics():
     zero_base = O.decode_attention_one(q[0], kp, vp, t.page_ids, [0] * len(t.pos_base), t.kv_len, qp, 1.0, 5e5)
     wrong_qpos = O.decode_attention_one(q[0], kp, vp, t.page_ids, t.pos_base, t.kv_len, 0, 1.0, 5e5)
     assert exceeds(no_rope) and exceeds(zero_base) and exceeds(wrong_qpos)
+
+
+def test_pairing_convention_matters_interleaved_differs_beyond_tolerance():
+    """The paper gives no RoPE pairing; the specification fixes split-half (i, i + D/2).  An interleaved
+    (2i, 2i+1) rotation of the same inputs is a different function: the tolerance tells them apart, so a kernel
+    built on the other convention could not pass."""
+    wl = make_custom(2, n_q_heads=8, n_kv_heads=2, head_dim=128, page_size=16, rope_theta=5e5, sm_scale=1.0,
+                     q_std=1 / math.sqrt(128), n_pool_chunks=4, chunk_tokens=512, zipf_s=1.1,
+                     decode_chunks_per_request=[4], decode_question=64, salt=7)
+    kp, vp = wl.kv_pool(); q = wl.decode_q()
+    st = O.OracleStore(16, wl.num_pages)
+    r = wl.decode_requests[0]
+    segs = [(k, st.register_chunk(wl.chunks[v])[0]) if k == O.KIND_CHUNK else (k, v) for k, v in r.segments]
+    t = st.build_block_table(0, segs)
+    good = O.decode_attention_one(q[0], kp, vp, t.page_ids, t.pos_base, t.kv_len, t.kv_len - 1, 1.0, 5e5)
+    # interleaved pairing, written out independently with complex numbers on (x[2i], x[2i+1])
+    D, P, L, theta = 128, 16, t.kv_len, 5e5
+    inv = np.array([theta ** (-(2.0 * i) / D) for i in range(D // 2)])
+    def rot_il(x, pos):
+        z = (x[..., 0::2] + 1j * x[..., 1::2]) * np.exp(1j * np.asarray(pos, dtype=np.float64)[..., None] * inv)
+        y = np.empty_like(x); y[..., 0::2] = z.real; y[..., 1::2] = z.imag
+        return y
+    K = bf16_bits_to_f64(O.gather_pages(kp, t.page_ids, L)); V = bf16_bits_to_f64(O.gather_pages(vp, t.page_ids, L))
+    pos = O.slot_positions(t.pos_base, L, P)
+    Kr = rot_il(K, pos[:, None] * np.ones((1, K.shape[1])))
+    qr = rot_il(bf16_bits_to_f64(q[0]), np.full(q.shape[1], L - 1.0))
+    other = np.empty_like(good)
+    for h in range(q.shape[1]):
+        s = Kr[:, h // 4, :] @ qr[h]
+        w = np.exp(s - s.max()); w /= w.sum()
+        other[h] = w @ V[:, h // 4, :]
+    d = np.abs(other - good)
+    assert d.max() > 2e-2 or d.mean() > 2e-3
