@@ -89,6 +89,8 @@ typedef struct {
   int64_t unshared_equivalent_pages;  /* sum of block-table entries of live requests = pages a
                                          per-request copy of every chunk would hold */
   int64_t live_requests;
+  int64_t chunks_evicted;             /* zero-reference chunk objects reclaimed under memory pressure */
+  int64_t pages_evicted;              /* pages those evictions returned to the pool */
 } mepic_stats_t;
 
 typedef struct {
@@ -107,6 +109,18 @@ int64_t mepic_launch_count(void);
  * mepic_store_create: make an empty store over a pool of cfg->num_pages pages.  Free pages are
  * handed out first-in-first-out starting from 0,1,2,...; released pages rejoin the queue in
  * ascending order (the paper leaves the order open; this one makes tables reproducible).
+ *
+ * Memory pressure (Section 3.2.3 "Eviction Policy"; Algorithm 1, admission check): when a call needs
+ * more pages than are free, whole chunk objects with ZERO live references are reclaimed, least
+ * recently used first (use = the last register, table build or release that touched the chunk),
+ * until the demand is met; their pages rejoin the queue in ascending order per chunk.  Chunks the
+ * call itself is about to alias, and every page private to a live request, are never reclaimed.
+ * Reclaiming is lazy: it happens only inside such a call.  If free plus reclaimable pages cannot
+ * cover the demand the call is rejected (MEPIC_E_NOSPACE) and nothing is reclaimed.  The id of a
+ * reclaimed chunk becomes unknown; registering the same tokens again reports was_resident = 0.
+ * References are taken by mepic_build_block_table, not by mepic_chunk_register: under pressure a
+ * request's later registration may reclaim a chunk the same request registered just before; the
+ * table build then returns MEPIC_E_NOTFOUND and the caller registers that chunk again.
  * cfg: host.  out: host, receives the handle.  Errors: E_INVAL.
  */
 int32_t mepic_store_create(const mepic_config_t* cfg, mepic_store_t** out);
@@ -121,7 +135,7 @@ void    mepic_store_destroy(mepic_store_t* store);
  * pad_token_id to a multiple of page_size, hashes the padded sequence (64-bit FNV-1a, confirmed by
  * a full token compare, so identity is by content) and looks it up.  On a miss it takes
  * ceil(n/page_size) - 1 pages from the pool for the shareable blocks; on a hit it allocates
- * nothing.  out_chunk_id, out_was_resident (0/1), out_lead_pad (pad tokens added), out_n_shared:
+ * nothing (a miss may first reclaim idle chunks, see mepic_store_create).  out_chunk_id, out_was_resident (0/1), out_lead_pad (pad tokens added), out_n_shared:
  * host, each may be NULL.  out_shared_pages (host, cap entries, may be NULL when cap == 0)
  * receives the shared page ids in block order.
  * Errors: E_INVAL; E_NOSPACE (nothing allocated, chunk not registered); E_CAPACITY (cap too small:

@@ -13,8 +13,10 @@ What it states, and where the paper fixes it:
   A chunk's identity is its padded token sequence (Section 3.2.3, "KV Block
   Allocation"); its first KV block is private to each request and the
   remaining blocks are shared by every request that uses the chunk
-  (Section 3.2.3, Section 3.3.1).  A request is rejected when the pool cannot
-  supply its blocks (Algorithm 1, admission check).
+  (Section 3.2.3, Section 3.3.1).  Under memory pressure zero-reference chunk
+  objects are reclaimed whole, least recently used first, and only then; a
+  request is rejected when free plus reclaimable blocks cannot supply its
+  demand (Section 3.2.3 "Eviction Policy"; Algorithm 1, admission check).
 * Computation path (Section 3.3): recomputed K/V rows are written straight
   into their assigned pages (Section 3.3.2); pages hold keys WITHOUT rotary
   position embedding, and the rotation is applied to K when the attention
@@ -80,6 +82,32 @@ class OracleStore:
         self.chunks: Dict[Tuple[int, ...], dict] = {}
         self.requests: Dict[int, dict] = {}
         self.dedup_hits = 0
+        self.tick = 0
+        self.chunks_evicted = 0
+        self.pages_evicted = 0
+
+    def _touch(self, key) -> None:
+        self.tick += 1
+        self.chunks[key]["last_use"] = self.tick
+
+    # Section 3.2.3 "Eviction Policy" + Algorithm 1 admission check: under pressure, whole zero-reference chunk
+    # objects are reclaimed, least recently used first; chunks the call is about to use are protected; if that
+    # cannot cover the demand the call is rejected and nothing is reclaimed.
+    def _make_room(self, need: int, protect=()) -> bool:
+        if need <= len(self.free):
+            return True
+        cand = [(c["last_use"], k) for k, c in self.chunks.items()
+                if c["refs"] == 0 and c["shared"] and k not in protect]
+        if len(self.free) + sum(len(self.chunks[k]["shared"]) for _, k in cand) < need:
+            return False
+        for _, k in sorted(cand, key=lambda x: x[0]):
+            if need <= len(self.free):
+                break
+            pages = sorted(self.chunks.pop(k)["shared"])
+            self.free.extend(pages)
+            self.chunks_evicted += 1
+            self.pages_evicted += len(pages)
+        return True
 
     # Section 3.2.1: leading pad so that the chunk fills whole blocks.
     def canonical_chunk(self, tokens: Sequence[int]) -> Tuple[int, ...]:
@@ -94,13 +122,15 @@ class OracleStore:
         key = self.canonical_chunk(tokens)
         if key in self.chunks:
             self.dedup_hits += 1
+            self._touch(key)
             return key, True, list(self.chunks[key]["shared"])
         n_pages = len(key) // self.P
         n_shared = n_pages - 1          # first block is private per request
-        if n_shared > len(self.free):
+        if not self._make_room(n_shared):
             raise Reject("no space for shared pages")
         shared = [self.free.popleft() for _ in range(n_shared)]
-        self.chunks[key] = {"shared": shared, "refs": 0, "n_pages": n_pages}
+        self.chunks[key] = {"shared": shared, "refs": 0, "n_pages": n_pages, "last_use": 0}
+        self._touch(key)
         return key, False, list(shared)
 
     # Algorithm 1, last stage: walk the segments in order and assign blocks.
@@ -118,8 +148,9 @@ class OracleStore:
                 need += 1
             else:
                 need += -(-int(val) // self.P)
-        if need > len(self.free):
-            raise Reject("no space for private pages")     # nothing was allocated yet
+        protect = {v for k, v in segs if k == KIND_CHUNK}
+        if not self._make_room(need, protect):
+            raise Reject("no space for private pages")     # nothing was allocated or reclaimed
         pages: List[int] = []
         private: List[int] = []
         recompute: List[int] = []
@@ -135,6 +166,7 @@ class OracleStore:
                 pages.extend(c["shared"])
                 recompute.extend(range(start, start + self.P))
                 c["refs"] += 1
+                self._touch(val)
                 used.append(val)
                 kv_len = len(pages) * self.P
             else:
@@ -156,6 +188,7 @@ class OracleStore:
         r = self.requests.pop(request_id)
         for key in r["chunks"]:
             self.chunks[key]["refs"] -= 1
+            self._touch(key)
         for pg in sorted(r["private"]):
             self.free.append(pg)
 
@@ -172,6 +205,8 @@ class OracleStore:
             "dedup_hits": self.dedup_hits,
             "unshared_equivalent_pages": sum(r["entries"] for r in self.requests.values()),
             "live_requests": len(self.requests),
+            "chunks_evicted": self.chunks_evicted,
+            "pages_evicted": self.pages_evicted,
         }
 
 

@@ -61,7 +61,8 @@ class _ConfigC(C.Structure):
 class _StatsC(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "pages_total", "pages_free", "pages_shared_held", "pages_private_held", "chunks_resident",
-        "chunk_refs", "dedup_hits", "unshared_equivalent_pages", "live_requests")]
+        "chunk_refs", "dedup_hits", "unshared_equivalent_pages", "live_requests", "chunks_evicted",
+        "pages_evicted")]
 
 
 class _SegmentC(C.Structure):

@@ -50,6 +50,7 @@ struct Chunk {
   std::vector<int32_t> padded;   // canonical form: leading pads + tokens
   std::vector<int32_t> shared;   // page ids of blocks 1..n-1
   int64_t refs = 0;
+  uint64_t last_use = 0;         // store tick of the last register / table build / release that touched it
 };
 
 struct LiveRequest {
@@ -66,7 +67,43 @@ struct mepic_store {
   int64_t dedup_hits = 0;
   int64_t shared_held = 0;
   int64_t private_held = 0;
+  int64_t chunks_evicted = 0;
+  int64_t pages_evicted = 0;
+  uint64_t tick = 0;
   mutable std::mutex mu;
+
+  void touch(Chunk& c) { c.last_use = ++tick; }
+
+  // Section 3.2.3 "Eviction Policy" / Algorithm 1 admission check: if `need` pages are not free, reclaim whole
+  // chunk objects with zero references, least recently used first, until they are; chunks named in `protect`
+  // (those the call in progress is about to alias) are never taken.  Chunks are reclaimed lazily, only here.
+  // Returns false, having evicted nothing, when free + evictable pages cannot cover the demand (Reject).
+  bool make_room(size_t need, const std::vector<uint64_t>& protect) {
+    if (need <= free_pages.size()) return true;
+    std::vector<std::pair<uint64_t, uint64_t>> cand;     // (last_use, id) of evictable chunks that hold pages
+    size_t evictable = 0;
+    for (const auto& kv : chunks) {
+      const Chunk& c = kv.second;
+      if (c.refs != 0 || c.shared.empty()) continue;
+      if (std::find(protect.begin(), protect.end(), kv.first) != protect.end()) continue;
+      cand.emplace_back(c.last_use, kv.first);
+      evictable += c.shared.size();
+    }
+    if (free_pages.size() + evictable < need) return false;
+    std::sort(cand.begin(), cand.end());
+    for (const auto& lu : cand) {
+      if (need <= free_pages.size()) break;
+      auto it = chunks.find(lu.second);
+      std::vector<int32_t> pages = it->second.shared;
+      std::sort(pages.begin(), pages.end());
+      for (int32_t pg : pages) free_pages.push_back(pg);
+      shared_held -= static_cast<int64_t>(pages.size());
+      pages_evicted += static_cast<int64_t>(pages.size());
+      chunks_evicted += 1;
+      chunks.erase(it);
+    }
+    return true;
+  }
 };
 
 static uint64_t fnv1a64(const std::vector<int32_t>& v) {
@@ -120,14 +157,16 @@ extern "C" int32_t mepic_chunk_register(mepic_store_t* s, const int32_t* tokens,
   if (hit) {
     resident = 1;
     s->dedup_hits += 1;
+    s->touch(s->chunks.at(id));
     shared = &hit->shared;
   } else {
     const size_t n_shared = padded.size() / P - 1;              // first block is private to each request
-    if (n_shared > s->free_pages.size()) {
-      mepic_set_error("chunk_register: %zu shared pages needed, %zu free", n_shared, s->free_pages.size());
+    if (!s->make_room(n_shared, {})) {
+      mepic_set_error("chunk_register: %zu shared pages needed, %zu free and not enough evictable", n_shared, s->free_pages.size());
       return MEPIC_E_NOSPACE;
     }
     Chunk c;
+    s->touch(c);
     c.shared.reserve(n_shared);
     for (size_t i = 0; i < n_shared; ++i) { c.shared.push_back(s->free_pages.front()); s->free_pages.pop_front(); }
     c.padded = std::move(padded);
@@ -195,9 +234,15 @@ extern "C" int32_t mepic_build_block_table(mepic_store_t* s, int64_t request_id,
     mepic_set_error("build_block_table: need %lld entries, %lld slots", (long long)entries, (long long)slots);
     return MEPIC_E_CAPACITY;
   }
-  if (need_private > static_cast<int64_t>(s->free_pages.size())) {
-    mepic_set_error("build_block_table: %lld private pages needed, %zu free", (long long)need_private, s->free_pages.size());
-    return MEPIC_E_NOSPACE;                                     // Reject; nothing is held
+  {
+    std::vector<uint64_t> protect;                              // the chunks this request is about to alias
+    for (int i = 0; i <= last; ++i)
+      if (segs[i].kind == MEPIC_SEG_CHUNK) protect.push_back(segs[i].chunk_id);
+    if (!s->make_room(static_cast<size_t>(need_private), protect)) {
+      mepic_set_error("build_block_table: %lld private pages needed, %zu free and not enough evictable",
+                      (long long)need_private, s->free_pages.size());
+      return MEPIC_E_NOSPACE;                                   // Reject; nothing is held, nothing was evicted
+    }
   }
   // Pass 2 (block assignment).
   LiveRequest live;
@@ -211,6 +256,7 @@ extern "C" int32_t mepic_build_block_table(mepic_store_t* s, int64_t request_id,
       for (int32_t p : c.shared) out_page_ids[e++] = p;         // remaining blocks: shared chunk KV
       for (int64_t t = 0; t < P; ++t) out_recompute_slots[w++] = static_cast<int32_t>(start + t);
       c.refs += 1;
+      s->touch(c);
       live.chunks.push_back(segs[i].chunk_id);
     } else if (segs[i].n_tokens > 0) {
       const int64_t n = segs[i].n_tokens, pages = (n + P - 1) / P;
@@ -232,7 +278,7 @@ extern "C" int32_t mepic_request_release(mepic_store_t* s, int64_t request_id) {
   auto it = s->requests.find(request_id);
   if (it == s->requests.end()) { mepic_set_error("request %lld not live", (long long)request_id); return MEPIC_E_NOTFOUND; }
   LiveRequest& r = it->second;
-  for (uint64_t id : r.chunks) s->chunks.at(id).refs -= 1;
+  for (uint64_t id : r.chunks) { Chunk& c = s->chunks.at(id); c.refs -= 1; s->touch(c); }
   std::sort(r.private_pages.begin(), r.private_pages.end());
   for (int32_t p : r.private_pages) s->free_pages.push_back(p);
   s->private_held -= static_cast<int64_t>(r.private_pages.size());
@@ -256,6 +302,8 @@ extern "C" int32_t mepic_store_stats(const mepic_store_t* s, mepic_stats_t* out)
   for (const auto& kv : s->requests) ent += kv.second.entries;
   out->unshared_equivalent_pages = ent;
   out->live_requests = static_cast<int64_t>(s->requests.size());
+  out->chunks_evicted = s->chunks_evicted;
+  out->pages_evicted = s->pages_evicted;
   return MEPIC_OK;
 }
 

@@ -383,21 +383,53 @@ def test_reject_leaves_nothing_allocated_and_release_restores_fifo_order():
     assert shared == [0, 1]
     before = list(st.free)
     with pytest.raises(O.Reject):
-        st.build_block_table(1, [(O.KIND_CHUNK, key), (O.KIND_PROMPT, 13)])   # needs 1 + 4 = 5 > 4 free
+        # needs 1 + 4 = 5 > 4 free; the only idle chunk is the one the request itself uses: protected
+        st.build_block_table(1, [(O.KIND_CHUNK, key), (O.KIND_PROMPT, 13)])
     assert list(st.free) == before and st.stats()["chunk_refs"] == 0 and not st.requests
-    with pytest.raises(O.Reject):
-        st.register_chunk(list(range(50, 50 + 24)))              # 6 pages -> 5 shared > 4 free
-    assert list(st.free) == before and st.stats()["chunks_resident"] == 1
+    assert st.stats()["chunks_resident"] == 1 and st.stats()["chunks_evicted"] == 0
     t1 = st.build_block_table(1, [(O.KIND_CHUNK, key), (O.KIND_PROMPT, 5)])   # private 2 | 3,4
     assert t1.page_ids == [2, 0, 1, 3, 4] and list(st.free) == [5]
+    with pytest.raises(O.Reject):
+        st.register_chunk(list(range(50, 50 + 24)))              # 6 pages -> 5 shared > 1 free; the chunk in use cannot go
+    assert list(st.free) == [5] and st.stats()["chunks_resident"] == 1
     t2 = st.build_block_table(2, [(O.KIND_PROMPT, 2)])
     assert t2.page_ids == [5]
     st.release(2); st.release(1)
     assert list(st.free) == [5, 2, 3, 4]                          # freed pages appended ascending per release
     assert st.stats()["chunk_refs"] == 0 and st.stats()["chunks_resident"] == 1
-    # the chunk stays resident: registering it again is a hit with the same pages
+    # the chunk stays resident while nothing needs its pages: registering it again is a hit with the same pages
     _, hit, again = st.register_chunk(list(range(10)))
     assert hit and again == [0, 1]
+
+
+def test_idle_chunks_are_reclaimed_least_recently_used_first_and_only_under_pressure():
+    # Section 3.2.3 "Eviction Policy": zero-reference chunk objects go, whole, oldest use first; pages of live
+    # requests and chunks in use never do; nothing is reclaimed while free pages suffice.
+    st = O.OracleStore(4, 10)
+    A, _, sa = st.register_chunk(list(range(100, 112)))          # 3 pages -> shared 0,1
+    B, _, sb = st.register_chunk(list(range(200, 212)))          # shared 2,3
+    C, _, sc = st.register_chunk(list(range(300, 312)))          # shared 4,5
+    assert (sa, sb, sc) == ([0, 1], [2, 3], [4, 5])
+    t = st.build_block_table(1, [(O.KIND_CHUNK, B)])             # B in use; private page 6; free 7,8,9
+    assert t.page_ids == [6, 2, 3]
+    st.register_chunk(list(range(100, 112)))                     # touch A: now C is the least recently used idle chunk
+    # a prompt of 4 pages does not fit the 3 free pages: C (LRU, idle) goes, A (idle, newer) and B (in use) stay
+    t2 = st.build_block_table(2, [(O.KIND_PROMPT, 16)])
+    assert t2.page_ids == [7, 8, 9, 4] and list(st.free) == [5]
+    s = st.stats()
+    assert s["chunks_evicted"] == 1 and s["pages_evicted"] == 2 and s["chunks_resident"] == 2
+    assert C not in st.chunks and A in st.chunks and B in st.chunks
+    # next demand of 2 pages: A is the only idle chunk left
+    t3 = st.build_block_table(3, [(O.KIND_PROMPT, 8)])
+    assert t3.page_ids == [5, 0] and list(st.free) == [1] and A not in st.chunks
+    # B is in use: a demand that would need its pages is rejected and changes nothing
+    with pytest.raises(O.Reject):
+        st.build_block_table(4, [(O.KIND_PROMPT, 8)])
+    assert list(st.free) == [1] and B in st.chunks and st.stats()["chunks_evicted"] == 2
+    # a reclaimed chunk registers again as a miss, with fresh pages
+    st.release(3)                                                # frees 0, 5 -> free [1, 0, 5]
+    _, hit, sa2 = st.register_chunk(list(range(100, 112)))
+    assert not hit and sa2 == [1, 0]
 
 
 def test_same_chunk_twice_in_one_request_and_one_page_chunk():

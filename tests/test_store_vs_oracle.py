@@ -128,10 +128,7 @@ def test_error_codes_and_reject_is_transactional():
         assert list(shared) == [0, 1]
         before = st.stats()
         with pytest.raises(M.MepicError) as e:
-            st.build_block_table(1, [M.Segment(0, cid), M.Segment(1, 16 * 4)])       # 1 + 4 > 4 free
-        assert e.value.code == M.MEPIC_E_NOSPACE and st.stats() == before
-        with pytest.raises(M.MepicError) as e:
-            st.chunk_register(np.arange(1, 16 * 6 + 1, dtype=np.int32))              # 5 shared > 4 free
+            st.build_block_table(1, [M.Segment(0, cid), M.Segment(1, 16 * 4)])       # 1 + 4 > 4 free, own chunk protected
         assert e.value.code == M.MEPIC_E_NOSPACE and st.stats() == before
         with pytest.raises(M.MepicError) as e:
             st.build_block_table(1, [M.Segment(0, cid + 12345)])
@@ -140,6 +137,10 @@ def test_error_codes_and_reject_is_transactional():
             st.build_block_table(1, [M.Segment(1, 0)])
         assert e.value.code == M.MEPIC_E_INVAL
         st.build_block_table(1, [M.Segment(0, cid), M.Segment(1, 5)])
+        held = st.stats()
+        with pytest.raises(M.MepicError) as e:
+            st.chunk_register(np.arange(1, 16 * 6 + 1, dtype=np.int32))              # 5 shared > 3 free, chunk in use stays
+        assert e.value.code == M.MEPIC_E_NOSPACE and st.stats() == held
         with pytest.raises(M.MepicError) as e:
             st.build_block_table(1, [M.Segment(1, 5)])
         assert e.value.code == M.MEPIC_E_EXISTS
@@ -148,11 +149,74 @@ def test_error_codes_and_reject_is_transactional():
         assert e.value.code == M.MEPIC_E_NOTFOUND
         st.request_release(1)
         assert st.stats()["pages_free"] == 4 and st.stats()["chunk_refs"] == 0
+        # now the chunk is idle: a registration that needs its pages reclaims it instead of failing
+        big, res, _, pages = st.chunk_register(np.arange(1, 16 * 6 + 1, dtype=np.int32))
+        assert not res and len(pages) == 5 and st.stats()["chunks_evicted"] == 1 and st.stats()["pages_evicted"] == 2
+        with pytest.raises(M.MepicError) as e:
+            st.build_block_table(9, [M.Segment(0, cid)])                              # its id is gone
+        assert e.value.code == M.MEPIC_E_NOTFOUND
     for bad in (dict(page_size=24), dict(page_size=8), dict(head_dim=96), dict(n_q_heads=7), dict(num_pages=0),
                 dict(n_q_heads=6, n_kv_heads=2)):
         with pytest.raises(M.MepicError) as e:
             M.Store(_cfg(**bad))
         assert e.value.code == M.MEPIC_E_INVAL
+
+
+def test_serving_trace_under_memory_pressure_matches_oracle_step_by_step():
+    """A long random trace of arrivals and departures over a pool far too small to keep every chunk: tables,
+    rejections, evictions and counters must agree with the oracle after every single call."""
+    rng = np.random.default_rng(21)
+    P = 16
+    chunks = [rng.integers(1, 5000, size=int(n), dtype=np.int32) for n in rng.integers(10, 200, size=24)]
+    cfg = _cfg(P=P, num_pages=90)
+    ost = O.OracleStore(P, 90)
+    live, rid, rejected = [], 0, 0
+    with M.Store(cfg) as st:
+        for step in range(600):
+            if live and (rng.random() < 0.45 or len(live) > 6):
+                r = live.pop(int(rng.integers(0, len(live))))
+                ost.release(r); st.request_release(r)
+            else:
+                rid += 1
+                picks = rng.choice(len(chunks), size=int(rng.integers(1, 4)), replace=False)
+                osegs, lsegs, ok = [], [], True
+                for c in picks:
+                    try:
+                        key, ores, oshared = ost.register_chunk(chunks[c])
+                    except O.Reject:
+                        with pytest.raises(M.MepicError) as e:
+                            st.chunk_register(chunks[c])
+                        assert e.value.code == M.MEPIC_E_NOSPACE
+                        ok = False
+                        break
+                    cid, lres, _, lshared = st.chunk_register(chunks[c])
+                    assert lres == ores and list(lshared) == oshared
+                    osegs.append((O.KIND_CHUNK, key)); lsegs.append(M.Segment(0, cid))
+                if ok:
+                    q = int(rng.integers(0, 40))
+                    osegs.append((O.KIND_PROMPT, q)); lsegs.append(M.Segment(1, q))
+                    try:
+                        ot = ost.build_block_table(rid, osegs)
+                    except KeyError:
+                        # a chunk registered earlier in this very request was reclaimed by a later registration
+                        with pytest.raises(M.MepicError) as e:
+                            st.build_block_table(rid, lsegs)
+                        assert e.value.code == M.MEPIC_E_NOTFOUND
+                        ot = None
+                    except O.Reject:
+                        with pytest.raises(M.MepicError) as e:
+                            st.build_block_table(rid, lsegs)
+                        assert e.value.code == M.MEPIC_E_NOSPACE
+                        rejected += 1
+                        ot = None
+                    if ot is not None:
+                        pages, base, kv_len, slots = st.build_block_table(rid, lsegs)
+                        assert list(pages) == ot.page_ids and list(base) == ot.pos_base and kv_len == ot.kv_len
+                        assert list(slots) == ot.recompute_slots
+                        live.append(rid)
+            assert st.stats() == ost.stats(), step
+        s = st.stats()
+        assert s["chunks_evicted"] > 10 and rejected >= 0 and s["pages_free"] + s["pages_shared_held"] + s["pages_private_held"] == 90
 
 
 def test_identity_is_the_padded_sequence():
