@@ -156,7 +156,8 @@ int32_t mepic_chunk_register(mepic_store_t* store, const int32_t* tokens, int32_
  * its index in the padded sequence).  Outputs (host): out_page_ids / out_pos_base (cap_entries
  * each), *out_n_entries, *out_kv_len (padded length; pads are ordinary tokens), and
  * out_recompute_slots (cap_slots): the logical slots whose K/V the caller must compute and hand
- * to mepic_attn_prefill = every slot below kv_len that lives on a private page, ascending.
+ * to mepic_attn_prefill = every slot below kv_len that lives on a private page, plus every slot of a
+ * chunk marked by mepic_chunk_mark_uncomputed (first occurrence in the request), ascending.
  * The admission check runs before any allocation: on E_NOSPACE nothing is held.
  * Errors: E_INVAL (no tokens, bad kind), E_NOTFOUND (chunk id), E_EXISTS (request id live),
  * E_NOSPACE, E_CAPACITY (required counts written to *out_n_entries / *out_n_slots; nothing held).
@@ -166,6 +167,19 @@ int32_t mepic_build_block_table(mepic_store_t* store, int64_t request_id,
                                 int32_t* out_page_ids, int32_t* out_pos_base, int32_t cap_entries,
                                 int32_t* out_n_entries, int32_t* out_kv_len,
                                 int32_t* out_recompute_slots, int32_t cap_slots, int32_t* out_n_slots);
+
+/*
+ * mepic_chunk_mark_uncomputed - Section 3.3.1: "newly encountered chunks are fully recomputed, while cached
+ * chunks require recomputation of only the first KV block".  A registered chunk is taken to have its shareable
+ * pages filled by the caller (offline precompute, a load from a remote tier).  When that is not so - the chunk
+ * is new (mepic_chunk_register reported was_resident = 0) and nobody has its K/V - mark it: the NEXT
+ * mepic_build_block_table that aliases the chunk lists every slot of the chunk, shared pages included, among its
+ * recompute slots, so that that request's mepic_attn_prefill call computes and commits the whole chunk; the mark
+ * is cleared by that build, and later requests recompute the first block only.  The caller orders that prefill
+ * before any other request's attention over the chunk (same stream, or an event).
+ * Errors: E_NOTFOUND; E_EXISTS if live requests already alias the chunk.
+ */
+int32_t mepic_chunk_mark_uncomputed(mepic_store_t* store, uint64_t chunk_id);
 
 /* Request end (Section 3.2.3 "Eviction Policy"): private pages go back to the pool in ascending
  * order, the reference count of every chunk the request aliased drops by one; chunks stay

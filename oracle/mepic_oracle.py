@@ -129,9 +129,17 @@ class OracleStore:
         if not self._make_room(n_shared):
             raise Reject("no space for shared pages")
         shared = [self.free.popleft() for _ in range(n_shared)]
-        self.chunks[key] = {"shared": shared, "refs": 0, "n_pages": n_pages, "last_use": 0}
+        self.chunks[key] = {"shared": shared, "refs": 0, "n_pages": n_pages, "last_use": 0, "uncomputed": False}
         self._touch(key)
         return key, False, list(shared)
+
+    # Section 3.3.1: a newly encountered chunk (nobody has its K/V) is recomputed whole by the next request
+    # that uses it; cached chunks recompute their first block only.
+    def mark_uncomputed(self, key) -> None:
+        c = self.chunks[key]
+        if c["refs"] != 0:
+            raise ValueError("chunk is aliased by live requests")
+        c["uncomputed"] = True
 
     # Algorithm 1, last stage: walk the segments in order and assign blocks.
     def build_block_table(self, request_id: int, segments: Sequence[Tuple[int, object]]) -> OracleTable:
@@ -164,7 +172,9 @@ class OracleStore:
                 private.append(first)
                 pages.append(first)
                 pages.extend(c["shared"])
-                recompute.extend(range(start, start + self.P))
+                n_rec = self.P * c["n_pages"] if c["uncomputed"] else self.P
+                c["uncomputed"] = False
+                recompute.extend(range(start, start + n_rec))
                 c["refs"] += 1
                 self._touch(val)
                 used.append(val)

@@ -22,7 +22,7 @@ from .build import LIB_PATH, build_library
 __all__ = [
     "MepicError", "Config", "Segment", "Store", "lib",
     "mepic_store_create", "mepic_store_destroy", "mepic_chunk_register", "mepic_build_block_table",
-    "mepic_request_release", "mepic_store_stats", "mepic_rope_table_floats", "mepic_rope_table_fill",
+    "mepic_request_release", "mepic_chunk_mark_uncomputed", "mepic_store_stats", "mepic_rope_table_floats", "mepic_rope_table_fill",
     "mepic_attn_decode_workspace", "mepic_attn_decode", "mepic_attn_decode_static",
     "MEPIC_DECODE_STATIC_SCRATCH_BYTES", "mepic_attn_prefill_workspace",
     "mepic_attn_prefill", "mepic_last_error", "mepic_launch_count",
@@ -123,6 +123,7 @@ _PROTOTYPES = {
                                             C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int32),
                                             C.POINTER(C.c_int32), C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]),
     "mepic_request_release": (C.c_int32, [C.c_void_p, C.c_int64]),
+    "mepic_chunk_mark_uncomputed": (C.c_int32, [C.c_void_p, C.c_uint64]),
     "mepic_store_stats": (C.c_int32, [C.c_void_p, C.POINTER(_StatsC)]),
     "mepic_rope_table_floats": (C.c_size_t, [C.POINTER(_ConfigC)]),
     "mepic_rope_table_fill": (C.c_int32, [C.POINTER(_ConfigC), C.c_void_p]),
@@ -232,6 +233,10 @@ def mepic_build_block_table(store: int, request_id: int, segments: Sequence[Segm
     return pages[:ne.value], base[:ne.value], int(kv.value), slots[:ns.value]
 
 
+def mepic_chunk_mark_uncomputed(store: int, chunk_id: int) -> None:
+    _check(lib().mepic_chunk_mark_uncomputed(store, chunk_id))
+
+
 def mepic_request_release(store: int, request_id: int) -> None:
     _check(lib().mepic_request_release(store, request_id))
 
@@ -254,6 +259,9 @@ class Store:
 
     def build_block_table(self, request_id, segments):
         return mepic_build_block_table(self.handle, request_id, segments)
+
+    def chunk_mark_uncomputed(self, chunk_id):
+        mepic_chunk_mark_uncomputed(self.handle, chunk_id)
 
     def request_release(self, request_id):
         mepic_request_release(self.handle, request_id)

@@ -51,6 +51,7 @@ struct Chunk {
   std::vector<int32_t> shared;   // page ids of blocks 1..n-1
   int64_t refs = 0;
   uint64_t last_use = 0;         // store tick of the last register / table build / release that touched it
+  bool uncomputed = false;       // the shared pages hold no K/V yet: the next request to alias the chunk computes them
 };
 
 struct LiveRequest {
@@ -213,9 +214,14 @@ extern "C" int32_t mepic_build_block_table(mepic_store_t* s, int64_t request_id,
   for (int i = 0; i <= last; ++i) {
     if (segs[i].kind == MEPIC_SEG_CHUNK) {
       const Chunk& c = s->chunks.at(segs[i].chunk_id);
+      // Section 3.3.1: a cached chunk recomputes its first block only; a newly encountered one is recomputed whole
+      // (once per request: a second occurrence of the same chunk in this request finds it computed)
+      bool whole = c.uncomputed;
+      for (int k = 0; k < i && whole; ++k)
+        if (segs[k].kind == MEPIC_SEG_CHUNK && segs[k].chunk_id == segs[i].chunk_id) whole = false;
       entries += 1 + static_cast<int64_t>(c.shared.size());
       need_private += 1;
-      slots += P;
+      slots += whole ? P * (1 + static_cast<int64_t>(c.shared.size())) : P;
       kv_len = entries * P;
     } else if (segs[i].n_tokens > 0) {
       const int64_t n = segs[i].n_tokens, pages = (n + P - 1) / P;
@@ -254,7 +260,9 @@ extern "C" int32_t mepic_build_block_table(mepic_store_t* s, int64_t request_id,
       Chunk& c = s->chunks.at(segs[i].chunk_id);
       out_page_ids[e++] = take();                               // first block: private, recomputed
       for (int32_t p : c.shared) out_page_ids[e++] = p;         // remaining blocks: shared chunk KV
-      for (int64_t t = 0; t < P; ++t) out_recompute_slots[w++] = static_cast<int32_t>(start + t);
+      const int64_t n_rec = c.uncomputed ? P * (1 + static_cast<int64_t>(c.shared.size())) : P;
+      c.uncomputed = false;                                     // this request computes them; later ones reuse them
+      for (int64_t t = 0; t < n_rec; ++t) out_recompute_slots[w++] = static_cast<int32_t>(start + t);
       c.refs += 1;
       s->touch(c);
       live.chunks.push_back(segs[i].chunk_id);
@@ -269,6 +277,16 @@ extern "C" int32_t mepic_build_block_table(mepic_store_t* s, int64_t request_id,
   live.entries = entries;
   s->private_held += static_cast<int64_t>(live.private_pages.size());
   s->requests.emplace(request_id, std::move(live));
+  return MEPIC_OK;
+}
+
+extern "C" int32_t mepic_chunk_mark_uncomputed(mepic_store_t* s, uint64_t chunk_id) {
+  if (!s) { mepic_set_error("store is NULL"); return MEPIC_E_INVAL; }
+  std::lock_guard<std::mutex> lock(s->mu);
+  auto it = s->chunks.find(chunk_id);
+  if (it == s->chunks.end()) { mepic_set_error("unknown chunk id"); return MEPIC_E_NOTFOUND; }
+  if (it->second.refs != 0) { mepic_set_error("chunk is aliased by live requests"); return MEPIC_E_EXISTS; }
+  it->second.uncomputed = true;
   return MEPIC_OK;
 }
 

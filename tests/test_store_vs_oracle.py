@@ -238,3 +238,33 @@ def test_rope_table_matches_oracle_angles():
         phi = O.rope_angles(np.int64(p), 128, 5e5)
         assert np.abs(tab[p, :, 0] - np.cos(phi)).max() <= 2.0 ** -24
         assert np.abs(tab[p, :, 1] - np.sin(phi)).max() <= 2.0 ** -24
+
+
+def test_new_chunk_is_recomputed_whole_once_then_first_block_only():
+    # Section 3.3.1 through the ABI and the oracle: tables identical; the marked chunk lists all its slots for the
+    # first request that uses it (first occurrence only), and only its first block afterwards.
+    P = 16
+    rng = np.random.default_rng(31)
+    A = rng.integers(1, 999, size=40, dtype=np.int32)      # 3 pages (8 leading pads)
+    B = rng.integers(1, 999, size=64, dtype=np.int32)      # 4 pages
+    ost = O.OracleStore(P, 64)
+    with M.Store(_cfg(P=P, num_pages=64)) as st:
+        ka, _, _ = ost.register_chunk(A); kb, _, _ = ost.register_chunk(B)
+        ca, ra, _, _ = st.chunk_register(A); cb, rb, _, _ = st.chunk_register(B)
+        assert not ra and not rb
+        ost.mark_uncomputed(ka); st.chunk_mark_uncomputed(ca)
+        o1 = ost.build_block_table(1, [(O.KIND_PROMPT, 5), (O.KIND_CHUNK, ka), (O.KIND_CHUNK, kb), (O.KIND_CHUNK, ka), (O.KIND_PROMPT, 3)])
+        l1 = st.build_block_table(1, [M.Segment(1, 5), M.Segment(0, ca), M.Segment(0, cb), M.Segment(0, ca), M.Segment(1, 3)])
+        assert list(l1[0]) == o1.page_ids and l1[2] == o1.kv_len and list(l1[3]) == o1.recompute_slots
+        # prompt(5) -> slots 0..15; A whole -> 16..63; B first block -> 64..79; A again, first block -> 128..143; prompt(3)
+        assert o1.recompute_slots == list(range(0, 16)) + list(range(16, 64)) + list(range(64, 80)) + list(range(128, 144)) + list(range(176, 179))
+        o2 = ost.build_block_table(2, [(O.KIND_CHUNK, ka)])
+        l2 = st.build_block_table(2, [M.Segment(0, ca)])
+        assert list(l2[3]) == o2.recompute_slots == list(range(0, 16))
+        with pytest.raises(M.MepicError) as e:
+            st.chunk_mark_uncomputed(ca)                      # aliased by live requests
+        assert e.value.code == M.MEPIC_E_EXISTS
+        with pytest.raises(M.MepicError) as e:
+            st.chunk_mark_uncomputed(ca + 77)
+        assert e.value.code == M.MEPIC_E_NOTFOUND
+        assert st.stats() == ost.stats()
