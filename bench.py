@@ -400,7 +400,7 @@ def run_ours(args):
     line = {
         "metric": "rope_fused_paged_decode_effective_hbm_bandwidth", "value": gbs(tot), "unit": "GB/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": tot / args.steps,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16 in, fp32 math",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": f"config{args.config}:{wl.name}", "batch": len(tables), "n_q_heads": wl.n_q_heads,
                    "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "page_size": wl.page_size,

@@ -70,7 +70,7 @@ typedef struct mepic_store mepic_store_t;
 typedef struct {
   int32_t page_size;     /* tokens per KV block ("page"); power of two, >= 16 */
   int32_t n_q_heads;
-  int32_t n_kv_heads;    /* divides n_q_heads; group size n_q_heads/n_kv_heads in {1,2,4,5,8} */
+  int32_t n_kv_heads;    /* divides n_q_heads; group size n_q_heads/n_kv_heads in 1..8 */
   int32_t head_dim;      /* 64 or 128 */
   int32_t num_pages;     /* pages in the pool */
   int32_t pad_token_id;  /* token used for canonical padding; part of the hashed sequence */

@@ -568,8 +568,8 @@ extern "C" int32_t mepic_attn_decode(const mepic_config_t* cfg, const mepic_deco
   if (rc != MEPIC_OK) return rc;
 
 #define MEPIC_DECODE_CASE(DD, GG) if (D == DD && G == GG) return launch_decode<DD, GG>(p, sms, map_k, map_v, st);
-  MEPIC_DECODE_CASE(128, 1) MEPIC_DECODE_CASE(128, 2) MEPIC_DECODE_CASE(128, 4) MEPIC_DECODE_CASE(128, 5) MEPIC_DECODE_CASE(128, 8)
-  MEPIC_DECODE_CASE(64, 1) MEPIC_DECODE_CASE(64, 2) MEPIC_DECODE_CASE(64, 4) MEPIC_DECODE_CASE(64, 5) MEPIC_DECODE_CASE(64, 8)
+  MEPIC_DECODE_CASE(128, 1) MEPIC_DECODE_CASE(128, 2) MEPIC_DECODE_CASE(128, 3) MEPIC_DECODE_CASE(128, 4) MEPIC_DECODE_CASE(128, 5) MEPIC_DECODE_CASE(128, 6) MEPIC_DECODE_CASE(128, 7) MEPIC_DECODE_CASE(128, 8)
+  MEPIC_DECODE_CASE(64, 1) MEPIC_DECODE_CASE(64, 2) MEPIC_DECODE_CASE(64, 3) MEPIC_DECODE_CASE(64, 4) MEPIC_DECODE_CASE(64, 5) MEPIC_DECODE_CASE(64, 6) MEPIC_DECODE_CASE(64, 7) MEPIC_DECODE_CASE(64, 8)
 #undef MEPIC_DECODE_CASE
   mepic_set_error("decode: unsupported head_dim %d / group size %d", D, G);
   return MEPIC_E_INVAL;

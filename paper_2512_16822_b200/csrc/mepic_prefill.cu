@@ -822,8 +822,8 @@ extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_pre
   const int D = cfg->head_dim, G = cfg->n_q_heads / cfg->n_kv_heads;
   const int n_items = static_cast<int>(items.size());
 #define MEPIC_PREFILL_CASE(DD, GG) if (D == DD && G == GG) return launch_prefill<DD, GG>(p, n_items, map_k, map_v, st);
-  MEPIC_PREFILL_CASE(128, 1) MEPIC_PREFILL_CASE(128, 2) MEPIC_PREFILL_CASE(128, 4) MEPIC_PREFILL_CASE(128, 5) MEPIC_PREFILL_CASE(128, 8)
-  MEPIC_PREFILL_CASE(64, 1) MEPIC_PREFILL_CASE(64, 2) MEPIC_PREFILL_CASE(64, 4) MEPIC_PREFILL_CASE(64, 5) MEPIC_PREFILL_CASE(64, 8)
+  MEPIC_PREFILL_CASE(128, 1) MEPIC_PREFILL_CASE(128, 2) MEPIC_PREFILL_CASE(128, 3) MEPIC_PREFILL_CASE(128, 4) MEPIC_PREFILL_CASE(128, 5) MEPIC_PREFILL_CASE(128, 6) MEPIC_PREFILL_CASE(128, 7) MEPIC_PREFILL_CASE(128, 8)
+  MEPIC_PREFILL_CASE(64, 1) MEPIC_PREFILL_CASE(64, 2) MEPIC_PREFILL_CASE(64, 3) MEPIC_PREFILL_CASE(64, 4) MEPIC_PREFILL_CASE(64, 5) MEPIC_PREFILL_CASE(64, 6) MEPIC_PREFILL_CASE(64, 7) MEPIC_PREFILL_CASE(64, 8)
 #undef MEPIC_PREFILL_CASE
   mepic_set_error("prefill: unsupported head_dim %d / group size %d", D, G);
   return MEPIC_E_INVAL;

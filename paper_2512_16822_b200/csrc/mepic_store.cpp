@@ -39,7 +39,7 @@ bool mepic_config_ok(const mepic_config_t* c) {
     mepic_set_error("n_q_heads %d must be a positive multiple of n_kv_heads %d", c->n_q_heads, c->n_kv_heads); return false;
   }
   const int g = c->n_q_heads / c->n_kv_heads;
-  if (!(g == 1 || g == 2 || g == 4 || g == 5 || g == 8)) { mepic_set_error("group size %d not in {1,2,4,5,8}", g); return false; }
+  if (g < 1 || g > 8) { mepic_set_error("group size %d not in 1..8", g); return false; }
   if (c->num_pages < 1) { mepic_set_error("num_pages %d < 1", c->num_pages); return false; }
   if (c->max_position < c->page_size - 1) { mepic_set_error("max_position %d < page_size-1", c->max_position); return false; }
   if (!(c->rope_theta > 1.0f)) { mepic_set_error("rope_theta must exceed 1"); return false; }

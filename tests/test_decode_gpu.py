@@ -136,7 +136,7 @@ def _run_manual(case):
 
 @pytest.mark.parametrize("Hq,Hkv,D,P", [
     (8, 2, 64, 16), (8, 2, 128, 16), (5, 1, 128, 16), (10, 2, 128, 32), (4, 4, 128, 16), (4, 2, 64, 64),
-    (8, 1, 128, 16), (16, 2, 64, 16), (2, 2, 64, 16), (10, 2, 64, 16)])
+    (8, 1, 128, 16), (16, 2, 64, 16), (2, 2, 64, 16), (10, 2, 64, 16), (3, 1, 128, 16), (12, 2, 64, 32), (7, 1, 128, 16)])
 def test_group_sizes_head_dims_page_sizes_ragged_lengths(Hq, Hkv, D, P):
     # lengths: one token, a page minus one, exact pages, several tiles plus ragged tails
     _run_manual(_manual_case(100 + Hq + D + P, Hq=Hq, Hkv=Hkv, D=D, P=P,

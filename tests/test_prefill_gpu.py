@@ -106,7 +106,8 @@ def test_single_tile_and_multi_tile_small():
 
 
 @pytest.mark.parametrize("Hq,Hkv,D,P", [(8, 2, 64, 16), (5, 1, 128, 16), (2, 2, 128, 64), (4, 2, 64, 32),
-                                        (8, 1, 128, 16), (10, 2, 64, 16), (4, 1, 128, 16)])
+                                        (8, 1, 128, 16), (10, 2, 64, 16), (4, 1, 128, 16), (3, 1, 128, 16),
+                                        (6, 1, 64, 16), (7, 1, 128, 32)])
 def test_group_sizes_head_dims_page_sizes(Hq, Hkv, D, P):
     G = Hq // Hkv
     QT = 128 // G

@@ -156,7 +156,7 @@ def test_error_codes_and_reject_is_transactional():
             st.build_block_table(9, [M.Segment(0, cid)])                              # its id is gone
         assert e.value.code == M.MEPIC_E_NOTFOUND
     for bad in (dict(page_size=24), dict(page_size=8), dict(head_dim=96), dict(n_q_heads=7), dict(num_pages=0),
-                dict(n_q_heads=6, n_kv_heads=2)):
+                dict(n_q_heads=18, n_kv_heads=2)):
         with pytest.raises(M.MepicError) as e:
             M.Store(_cfg(**bad))
         assert e.value.code == M.MEPIC_E_INVAL
