@@ -287,7 +287,9 @@ int32_t mepic_attn_decode_static(const mepic_config_t* cfg, const mepic_decode_a
  * the request's PRIVATE pages (shared pages are never written by a correct caller; the library
  * cannot tell).  All struct pointers are DEVICE pointers except row_offsets_host (host copy of
  * row_offsets, batch+1 entries, read during the call for launch sizing).
- * workspace: mepic_attn_prefill_workspace() bytes, 16-byte aligned.  Errors as for decode.
+ * workspace: mepic_attn_prefill_workspace() bytes, 16-byte aligned (a token amount: each CTA derives its share
+ * of the work on the device from row_offsets, nothing is built or uploaded by the call, which only enqueues two
+ * kernels).  Errors as for decode.
  */
 typedef struct {
   const void*    q_new;        /* bf16 [rows][n_q_heads][head_dim], un-rotated */

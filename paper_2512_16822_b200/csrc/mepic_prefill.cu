@@ -33,7 +33,6 @@
 #include <stdint.h>
 
 #include <algorithm>
-#include <vector>
 
 #include "mepic.h"
 #include "mepic_internal.h"
@@ -65,9 +64,9 @@ struct PrefillParams {
   const int32_t* kv_len;
   const float* rope;
   uint16_t* out;
-  const Item* items;
   int32_t* status;
   int table_stride, batch, n_kv_heads, page_size, num_pages, max_position, total_rows;
+  int max_q_tiles;      // most CTA-sized tiles of query positions any request has (launch sizing, from the host copy)
   float scale_log2;
 };
 
@@ -254,6 +253,46 @@ __global__ void mepic_prefill_commit(const PrefillParams p, int chunks_per_row) 
   }
 }
 
+// The work item of CTA `i`, derived on the device from row_offsets alone (no list to build or upload).  Items are
+// ordered heaviest first: level t = index of the tile of query positions inside its request, highest level first
+// (later tiles see more keys); inside a level by request, then kv head.  Executed by one full warp.
+__device__ __forceinline__ Item item_of_cta(const int32_t* row_offsets, int batch, int n_kv_heads, int qt, int max_q_tiles, int i, int lane) {
+  Item it{0, 0, 0, 0};
+  int before = 0;                                   // items of the levels above
+  for (int t = max_q_tiles - 1; t >= 0; --t) {
+    int cnt = 0;                                    // requests that have a tile at this level
+    for (int b0 = 0; b0 < batch; b0 += 32) {
+      const int b = b0 + lane;
+      const int n = b < batch ? row_offsets[b + 1] - row_offsets[b] : 0;
+      cnt += __popc(__ballot_sync(0xffffffffu, n > t * qt));
+    }
+    if (i < before + cnt * n_kv_heads) {
+      const int j = i - before, want = j / n_kv_heads;      // the want-th such request, kv head j % n_kv_heads
+      int seen = 0;
+      for (int b0 = 0; b0 < batch; b0 += 32) {
+        const int b = b0 + lane;
+        const int n = b < batch ? row_offsets[b + 1] - row_offsets[b] : 0;
+        const unsigned m = __ballot_sync(0xffffffffu, n > t * qt);
+        const int here = __popc(m);
+        if (want < seen + here) {
+          unsigned mm = m;
+          for (int k = 0; k < want - seen; ++k) mm &= mm - 1;     // drop the lower set bits
+          const int src = __ffs(mm) - 1;
+          const int bb = b0 + src;
+          const int nn = __shfl_sync(0xffffffffu, n, src);
+          it.b = bb; it.h = j % n_kv_heads;
+          it.row0 = __shfl_sync(0xffffffffu, b < batch ? row_offsets[b] : 0, src) + t * qt;
+          it.nq = min(qt, nn - t * qt);
+          return it;
+        }
+        seen += here;
+      }
+    }
+    before += cnt * n_kv_heads;
+  }
+  return it;       // not reached for i < number of items; nq = 0 makes the CTA do nothing
+}
+
 // ---------------------------------------------------------------- attention
 constexpr int kKStages = 3;            // K ring depth (rotation runs ahead of the MMA)
 constexpr int kVStages = 2;            // V ring depth
@@ -308,7 +347,14 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   volatile int* gbase = reinterpret_cast<volatile int*>(bars + kNumBars + 2);   // [kKStages][8] position of each 16-key group's first key
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const Item item = p.items[blockIdx.x];
+  Item* item_slot = reinterpret_cast<Item*>(bars + kNumBars + 16);
+  if (warp == 1) {
+    const Item it = item_of_cta(p.row_offsets, p.batch, p.n_kv_heads, 2 * QT, p.max_q_tiles, blockIdx.x, lane);
+    if (lane == 0) *item_slot = it;
+  }
+  __syncthreads();
+  const Item item = *item_slot;
+  if (item.nq <= 0) return;
   const int b = item.b, h = item.h;
   const int kvl = p.kv_len[b];
   const int32_t* ids = p.page_ids + static_cast<size_t>(b) * p.table_stride;
@@ -749,22 +795,21 @@ int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& m
   return MEPIC_OK;
 }
 
-// Work items, heaviest first: later tiles of a request see more keys.
-bool build_items(const mepic_config_t* cfg, int batch, const int32_t* row_offsets_host, std::vector<Item>* items) {
+// Launch sizing from the host copy of row_offsets: number of CTAs and the deepest level (see item_of_cta).
+bool count_items(const mepic_config_t* cfg, int batch, const int32_t* row_offsets_host, int* n_items, int* max_q_tiles) {
   const int G = cfg->n_q_heads / cfg->n_kv_heads, QT = 2 * (128 / G);   // two M-tiles of query positions per CTA
-  int max_tiles = 0;
+  long long items = 0;
+  int deepest = 0;
   for (int b = 0; b < batch; ++b) {
     const int n = row_offsets_host[b + 1] - row_offsets_host[b];
     if (n < 0) return false;
-    max_tiles = std::max(max_tiles, (n + QT - 1) / QT);
+    const int tiles = (n + QT - 1) / QT;
+    items += static_cast<long long>(tiles) * cfg->n_kv_heads;
+    deepest = std::max(deepest, tiles);
   }
-  for (int t = max_tiles - 1; t >= 0; --t)
-    for (int b = 0; b < batch; ++b) {
-      const int n = row_offsets_host[b + 1] - row_offsets_host[b];
-      if (t * QT >= n) continue;
-      for (int h = 0; h < cfg->n_kv_heads; ++h)
-        items->push_back(Item{b, h, row_offsets_host[b] + t * QT, std::min(QT, n - t * QT)});
-    }
+  if (items > 0x7fffffffLL) return false;
+  *n_items = static_cast<int>(items);
+  *max_q_tiles = deepest;
   return true;
 }
 
@@ -774,9 +819,9 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 extern "C" size_t mepic_attn_prefill_workspace(const mepic_config_t* cfg, int32_t batch, const int32_t* row_offsets_host) {
   if (!mepic_config_ok(cfg) || batch < 1 || !row_offsets_host) { if (cfg) mepic_set_error("prefill_workspace: bad argument"); return 0; }
-  std::vector<Item> items;
-  if (!build_items(cfg, batch, row_offsets_host, &items)) { mepic_set_error("prefill_workspace: row_offsets must be non-decreasing"); return 0; }
-  return std::max<size_t>(items.size(), 1) * sizeof(Item);
+  int n_items = 0, deepest = 0;
+  if (!count_items(cfg, batch, row_offsets_host, &n_items, &deepest)) { mepic_set_error("prefill_workspace: row_offsets must be non-decreasing"); return 0; }
+  return 16;       // the kernels derive their work on the device; a token amount keeps the argument meaningful
 }
 
 extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_prefill_args_t* a, void* cuda_stream) {
@@ -791,19 +836,16 @@ extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_pre
   }
   if (cfg->max_position < 16) { mepic_set_error("prefill: rope table must cover positions 0..16"); return MEPIC_E_INVAL; }
   if (a->row_offsets_host[0] != 0) { mepic_set_error("prefill: row_offsets[0] must be 0"); return MEPIC_E_INVAL; }
-  std::vector<Item> items;
-  if (!build_items(cfg, a->batch, a->row_offsets_host, &items)) { mepic_set_error("prefill: row_offsets must be non-decreasing"); return MEPIC_E_INVAL; }
+  int n_items = 0, max_q_tiles = 0;
+  if (!count_items(cfg, a->batch, a->row_offsets_host, &n_items, &max_q_tiles)) { mepic_set_error("prefill: row_offsets must be non-decreasing"); return MEPIC_E_INVAL; }
   const int total_rows = a->row_offsets_host[a->batch];
-  if (items.empty() || total_rows == 0) return MEPIC_OK;      // nothing to recompute
-  if (a->workspace_bytes < items.size() * sizeof(Item)) { mepic_set_error("prefill: workspace too small"); return MEPIC_E_INVAL; }
+  if (n_items == 0 || total_rows == 0) return MEPIC_OK;      // nothing to recompute
   alignas(64) CUtensorMap map_k, map_v;
   int32_t rc = mepic_make_pool_map(cfg, a->k_pool, &map_k);
   if (rc != MEPIC_OK) return rc;
   rc = mepic_make_pool_map(cfg, a->v_pool, &map_v);
   if (rc != MEPIC_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
-  cudaError_t e = cudaMemcpyAsync(a->workspace, items.data(), items.size() * sizeof(Item), cudaMemcpyHostToDevice, st);
-  if (e != cudaSuccess) { mepic_set_error("prefill: work list upload: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
 
   PrefillParams p;
   p.q_new = static_cast<const uint16_t*>(a->q_new);
@@ -814,13 +856,12 @@ extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_pre
   p.page_ids = a->page_ids; p.pos_base = a->pos_base; p.kv_len = a->kv_len;
   p.rope = a->rope_table;
   p.out = static_cast<uint16_t*>(a->out);
-  p.items = static_cast<const Item*>(a->workspace);
   p.status = a->status;
   p.table_stride = a->table_stride; p.batch = a->batch; p.n_kv_heads = cfg->n_kv_heads; p.page_size = cfg->page_size;
   p.num_pages = cfg->num_pages; p.max_position = cfg->max_position; p.total_rows = total_rows;
+  p.max_q_tiles = max_q_tiles;
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
   const int D = cfg->head_dim, G = cfg->n_q_heads / cfg->n_kv_heads;
-  const int n_items = static_cast<int>(items.size());
 #define MEPIC_PREFILL_CASE(DD, GG) if (D == DD && G == GG) return launch_prefill<DD, GG>(p, n_items, map_k, map_v, st);
   MEPIC_PREFILL_CASE(128, 1) MEPIC_PREFILL_CASE(128, 2) MEPIC_PREFILL_CASE(128, 3) MEPIC_PREFILL_CASE(128, 4) MEPIC_PREFILL_CASE(128, 5) MEPIC_PREFILL_CASE(128, 6) MEPIC_PREFILL_CASE(128, 7) MEPIC_PREFILL_CASE(128, 8)
   MEPIC_PREFILL_CASE(64, 1) MEPIC_PREFILL_CASE(64, 2) MEPIC_PREFILL_CASE(64, 3) MEPIC_PREFILL_CASE(64, 4) MEPIC_PREFILL_CASE(64, 5) MEPIC_PREFILL_CASE(64, 6) MEPIC_PREFILL_CASE(64, 7) MEPIC_PREFILL_CASE(64, 8)
