@@ -1,6 +1,6 @@
 """Run one benchmark configuration through the public binding and print the device time.
 
-    python -m paper_2512_16822_b200.cases decode  --config 2 [--scale 1.0] [--iters 10]
+    python -m paper_2512_16822_b200.cases decode  --config 2 [--scale 1.0] [--iters 10] [--unshared]
     python -m paper_2512_16822_b200.cases prefill --config 3 [--scale 0.5] [--iters 4]
 
 A small driver for profiling (a fixed, short sequence of calls that a profiler can capture) and for trying the
@@ -17,6 +17,31 @@ import numpy as np
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
+
+
+def _setup_unshared_decode(index: int, scale: float):
+    """The decode batch on a layout without chunk sharing: every request owns private copies of its chunks."""
+    import torch
+    import paper_2512_16822_b200 as M
+    from paper_2512_16822_b200 import runtime as RT
+    from mepic_inputs import make_workload
+    wl = make_workload(index, scale=scale)
+    P = wl.page_size
+    ents = [sum(-(-(len(wl.chunks[v]) if k == 0 else v) // P) for k, v in r.segments) for r in wl.decode_requests]
+    lens = [sum((len(wl.chunks[v]) if k == 0 else v) for k, v in r.segments) for r in wl.decode_requests]
+    num_pages = int(sum(ents))
+    cfg = M.Config(P, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, num_pages, wl.max_position, wl.rope_theta, wl.pad_token_id)
+    B, stride = len(ents), max(ents)
+    page_ids = np.zeros((B, stride), dtype=np.int32); pos_base = np.zeros((B, stride), dtype=np.int32)
+    perm = np.random.default_rng([0, wl.index, 99]).permutation(num_pages).astype(np.int32)
+    at = 0
+    for b, e in enumerate(ents):
+        page_ids[b, :e] = perm[at:at + e]; at += e
+        pos_base[b, :e] = np.arange(e) * P
+    kv_len = np.asarray(lens, dtype=np.int32)
+    dev = RT.Device(cfg)
+    dev.k_pool.normal_(); dev.v_pool.normal_()
+    return wl, dev, RT.DecodeBatch(dev, page_ids, pos_base, kv_len, kv_len - 1, wl.decode_q())
 
 
 def _setup(index: int, scale: float, which: str):
@@ -55,9 +80,13 @@ def main() -> None:
     ap.add_argument("--config", type=int, default=None)
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--iters", type=int, default=4)
+    ap.add_argument("--unshared", action="store_true", help="decode only: no chunk sharing, one page per table entry")
     args = ap.parse_args()
     index = args.config if args.config is not None else (2 if args.which == "decode" else 3)
-    wl, dev, batch = _setup(index, args.scale, args.which)
+    if args.unshared and args.which == "decode":
+        wl, dev, batch = _setup_unshared_decode(index, args.scale)
+    else:
+        wl, dev, batch = _setup(index, args.scale, args.which)
     for _ in range(max(args.iters - 1, 1)):
         batch.run(wl.sm_scale)
     torch.cuda.synchronize()
