@@ -61,6 +61,7 @@ extern "C" {
 #define MEPIC_DEV_WAIT_EXPIRED  0x2 /* a bounded wait on an on-chip barrier ran out */
 #define MEPIC_DEV_BAD_POSITION  0x4 /* a position fell outside the rope table */
 #define MEPIC_DEV_BAD_SLOT      0x8 /* a new row's logical slot fell outside its request */
+#define MEPIC_DEV_BAD_PLAN      0x10 /* a grouped-decode plan no longer matches kv_len (a request gained or lost a page) */
 
 #define MEPIC_SEG_CHUNK  0
 #define MEPIC_SEG_PROMPT 1
@@ -270,6 +271,62 @@ int32_t mepic_attn_decode(const mepic_config_t* cfg, const mepic_decode_args_t* 
  */
 #define MEPIC_DECODE_STATIC_SCRATCH_BYTES (8u << 20)
 int32_t mepic_attn_decode_static(const mepic_config_t* cfg, const mepic_decode_args_t* args, void* cuda_stream);
+
+/* ---------------------------------------------------------------- grouped decode (host plan + device)
+ *
+ * The same decode, aware of chunk sharing.  MEPIC lets many requests alias the physical pages of a
+ * chunk (Section 3.2.2); mepic_attn_decode still reads such a page once per request.  The paper's
+ * related-work section (operator-level acceleration: shared-prefix / shared-KV attention kernels)
+ * names kernels that serve all the requests sharing a piece of context from one pass over it as the
+ * layer to put under MEPIC; this pair of calls is that layer.  The result is the one
+ * mepic_attn_decode defines (same formula, same tolerance); only the order of the work differs.
+ *
+ * mepic_decode_plan_build (HOST pointers, host work only, no device call when n_sms > 0) regroups
+ * the block tables: every (request, table entry) pair is put in exactly one item = a group of at
+ * most R = min(16 / G, 8) requests plus the pages all of them alias; pages nobody else uses, a
+ * set's remainder of one request and a request's partly filled last page go to the request's own
+ * single-request item.  The (item, kv head, 16-token tile) triples are laid on one line and cut in
+ * equal pieces for n_sms * 8 workers (n_sms = 0: the SM count of the current device).  The plan is a
+ * flat int32 buffer the caller treats as opaque, copies to the device as is, and also keeps on the
+ * host.  It bakes in page ids, position bases and the number of table entries of every request; it
+ * stays valid while kv_len grows inside each request's last page and must be rebuilt when a request
+ * gains a page or the batch changes (the device sets MEPIC_DEV_BAD_PLAN otherwise and the result is
+ * then undefined but the call does not fault).  mepic_decode_plan_max_ints bounds the buffer size
+ * for any tables of that shape.  Errors: E_INVAL (bad argument, kv_len < 1, entries > stride),
+ * E_CAPACITY (buffer too small: *out_ints holds the need; or a batch beyond the plan's 32-bit
+ * fields), E_CUDA (n_sms = 0 without a device).
+ *
+ * mepic_attn_decode_grouped: all pointers DEVICE pointers except plan_host (the host copy of the
+ * same plan; its header is read during the call).  q, kv_len, q_pos, out, status, rope_table and the
+ * pools are as for mepic_attn_decode; the block tables are not passed: the plan replaces them.
+ * The rope table must cover position 16 (max_position >= 16).  workspace: at least
+ * mepic_attn_decode_grouped_workspace() bytes, 16-byte aligned, contents overwritten; plan: 16-byte
+ * aligned.  Errors as for mepic_attn_decode, plus E_INVAL for a plan built for another config/batch.
+ */
+size_t  mepic_decode_plan_max_ints(const mepic_config_t* cfg, int32_t batch, int32_t table_stride, int32_t n_sms);
+int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int32_t* page_ids_host, const int32_t* pos_base_host,
+                                const int32_t* kv_len_host, int32_t batch, int32_t table_stride, int32_t n_sms,
+                                int32_t* out_plan_host, size_t cap_ints, size_t* out_ints);
+
+typedef struct {
+  const void*    q;            /* bf16 [batch][n_q_heads][head_dim], un-rotated */
+  const void*    k_pool;
+  const void*    v_pool;
+  const int32_t* plan;         /* device copy of the plan */
+  const int32_t* plan_host;    /* host copy of the same plan */
+  const int32_t* kv_len;       /* [batch] */
+  const int32_t* q_pos;        /* [batch] */
+  const float*   rope_table;
+  void*          out;          /* bf16 [batch][n_q_heads][head_dim] */
+  void*          workspace;
+  size_t         workspace_bytes;
+  int32_t*       status;
+  int32_t        batch;
+  float          sm_scale;
+} mepic_decode_grouped_args_t;
+
+size_t  mepic_attn_decode_grouped_workspace(const mepic_config_t* cfg, const int32_t* plan_host);
+int32_t mepic_attn_decode_grouped(const mepic_config_t* cfg, const mepic_decode_grouped_args_t* args, void* cuda_stream);
 
 /* ---------------------------------------------------------------- prefill (device)
  *

@@ -24,6 +24,8 @@ __all__ = [
     "mepic_store_create", "mepic_store_destroy", "mepic_chunk_register", "mepic_build_block_table",
     "mepic_request_release", "mepic_chunk_mark_uncomputed", "mepic_store_stats", "mepic_rope_table_floats", "mepic_rope_table_fill",
     "mepic_attn_decode_workspace", "mepic_attn_decode", "mepic_attn_decode_static",
+    "mepic_decode_plan_max_ints", "mepic_decode_plan_build", "mepic_attn_decode_grouped_workspace",
+    "mepic_attn_decode_grouped",
     "MEPIC_DECODE_STATIC_SCRATCH_BYTES", "mepic_attn_prefill_workspace",
     "mepic_attn_prefill", "mepic_last_error", "mepic_launch_count",
     "MEPIC_OK", "MEPIC_E_INVAL", "MEPIC_E_NOSPACE", "MEPIC_E_NOTFOUND", "MEPIC_E_CAPACITY",
@@ -87,6 +89,13 @@ class _PrefillArgsC(C.Structure):
                 ("sm_scale", C.c_float)]
 
 
+class _DecodeGroupedArgsC(C.Structure):
+    _fields_ = [("q", C.c_void_p), ("k_pool", C.c_void_p), ("v_pool", C.c_void_p), ("plan", C.c_void_p),
+                ("plan_host", C.c_void_p), ("kv_len", C.c_void_p), ("q_pos", C.c_void_p), ("rope_table", C.c_void_p),
+                ("out", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+                ("status", C.c_void_p), ("batch", C.c_int32), ("sm_scale", C.c_float)]
+
+
 @dataclass(frozen=True)
 class Config:
     page_size: int
@@ -130,6 +139,11 @@ _PROTOTYPES = {
     "mepic_attn_decode_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32]),
     "mepic_attn_decode": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeArgsC), C.c_void_p]),
     "mepic_attn_decode_static": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeArgsC), C.c_void_p]),
+    "mepic_decode_plan_max_ints": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32, C.c_int32, C.c_int32]),
+    "mepic_decode_plan_build": (C.c_int32, [C.POINTER(_ConfigC), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                            C.c_int32, C.c_int32, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]),
+    "mepic_attn_decode_grouped_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_void_p]),
+    "mepic_attn_decode_grouped": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeGroupedArgsC), C.c_void_p]),
     "mepic_attn_prefill_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32, C.c_void_p]),
     "mepic_attn_prefill": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_PrefillArgsC), C.c_void_p]),
 }
@@ -335,6 +349,49 @@ def mepic_attn_decode_static(cfg: Config, *, q, k_pool, v_pool, page_ids, pos_ba
                      _ptr(q_pos), _ptr(rope_table), _ptr(out), None, 0, _ptr(status), table_stride, batch, sm_scale)
     c = cfg.c()
     _check(lib().mepic_attn_decode_static(C.byref(c), C.byref(a), _stream_ptr(stream)))
+
+
+def mepic_decode_plan_max_ints(cfg: Config, batch: int, table_stride: int, n_sms: int = 0) -> int:
+    c = cfg.c()
+    n = int(lib().mepic_decode_plan_max_ints(C.byref(c), batch, table_stride, n_sms))
+    if n == 0:
+        raise MepicError(MEPIC_E_INVAL, mepic_last_error())
+    return n
+
+
+def mepic_decode_plan_build(cfg: Config, page_ids: np.ndarray, pos_base: np.ndarray, kv_len: np.ndarray,
+                            n_sms: int = 0) -> np.ndarray:
+    """Host block tables -> the grouped-decode plan (int32 array, opaque).  n_sms = 0: current device."""
+    ids = np.ascontiguousarray(page_ids, dtype=np.int32)
+    base = np.ascontiguousarray(pos_base, dtype=np.int32)
+    lens = np.ascontiguousarray(kv_len, dtype=np.int32)
+    batch, stride = ids.shape
+    assert base.shape == ids.shape and lens.shape == (batch,)
+    cap = mepic_decode_plan_max_ints(cfg, batch, stride, n_sms)
+    out = np.empty(cap, dtype=np.int32)
+    used = C.c_size_t(0)
+    c = cfg.c()
+    _check(lib().mepic_decode_plan_build(C.byref(c), ids.ctypes.data, base.ctypes.data, lens.ctypes.data, batch, stride,
+                                         n_sms, out.ctypes.data, cap, C.byref(used)))
+    return out[:used.value].copy()
+
+
+def mepic_attn_decode_grouped_workspace(cfg: Config, plan_host: np.ndarray) -> int:
+    c = cfg.c()
+    n = int(lib().mepic_attn_decode_grouped_workspace(C.byref(c), plan_host.ctypes.data))
+    if n == 0:
+        raise MepicError(MEPIC_E_INVAL, mepic_last_error())
+    return n
+
+
+def mepic_attn_decode_grouped(cfg: Config, *, q, k_pool, v_pool, plan, plan_host: np.ndarray, kv_len, q_pos, rope_table,
+                              out, workspace, workspace_bytes: int, status, batch: int, sm_scale: float,
+                              stream=None) -> None:
+    a = _DecodeGroupedArgsC(_ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(plan), plan_host.ctypes.data, _ptr(kv_len),
+                            _ptr(q_pos), _ptr(rope_table), _ptr(out), _ptr(workspace), workspace_bytes, _ptr(status),
+                            batch, sm_scale)
+    c = cfg.c()
+    _check(lib().mepic_attn_decode_grouped(C.byref(c), C.byref(a), _stream_ptr(stream)))
 
 
 def mepic_attn_prefill_workspace(cfg: Config, batch: int, row_offsets_host: np.ndarray) -> int:

@@ -17,7 +17,8 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(HERE, "libmepic.so")
 
-SOURCES = ["mepic_store.cpp", "mepic_tensor_map.cu", "mepic_decode.cu", "mepic_prefill.cu"]
+SOURCES = ["mepic_store.cpp", "mepic_tensor_map.cu", "mepic_decode.cu", "mepic_decode_grouped.cu", "mepic_plan.cpp",
+           "mepic_prefill.cu"]
 
 
 def _nvcc() -> str:

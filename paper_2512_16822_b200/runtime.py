@@ -12,6 +12,7 @@ import numpy as np
 import torch
 
 from . import (Config, Segment, Store, MEPIC_SEG_CHUNK, MEPIC_SEG_PROMPT, mepic_attn_decode,
+               mepic_decode_plan_build, mepic_attn_decode_grouped, mepic_attn_decode_grouped_workspace,
                mepic_attn_decode_workspace, mepic_attn_prefill, mepic_attn_prefill_workspace,
                mepic_rope_table_fill)
 
@@ -125,6 +126,36 @@ class DecodeBatch:
                           rope_table=self.dev.rope, out=self.out, workspace=self.workspace,
                           workspace_bytes=self.ws_bytes, status=self.dev.status, table_stride=self.stride,
                           batch=self.batch, sm_scale=sm_scale, stream=s)
+        return self.out
+
+
+class GroupedDecodeBatch:
+    """One decode batch run through the sharing-aware path: host plan + its device copy, output, workspace."""
+
+    def __init__(self, dev: Device, page_ids: np.ndarray, pos_base: np.ndarray, kv_len: np.ndarray,
+                 q_pos: np.ndarray, q_bits: Optional[np.ndarray] = None, n_sms: int = 0):
+        cfg = dev.cfg
+        self.dev = dev
+        self.batch = page_ids.shape[0]
+        d = dev.device
+        with torch.cuda.device(d):
+            self.plan_host = mepic_decode_plan_build(cfg, page_ids, pos_base, kv_len, n_sms)
+        self.plan = torch.from_numpy(self.plan_host).to(d)
+        self.kv_len = torch.from_numpy(np.ascontiguousarray(kv_len, dtype=np.int32)).to(d)
+        self.q_pos = torch.from_numpy(np.ascontiguousarray(q_pos, dtype=np.int32)).to(d)
+        qshape = (self.batch, cfg.n_q_heads, cfg.head_dim)
+        self.q = bf16_tensor(q_bits, d) if q_bits is not None else torch.empty(qshape, dtype=torch.bfloat16, device=d)
+        self.out = torch.empty(qshape, dtype=torch.bfloat16, device=d)
+        self.ws_bytes = mepic_attn_decode_grouped_workspace(cfg, self.plan_host)
+        self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=d)
+
+    def run(self, sm_scale: float, stream=None) -> torch.Tensor:
+        s = stream if stream is not None else torch.cuda.current_stream(self.dev.device)
+        mepic_attn_decode_grouped(self.dev.cfg, q=self.q, k_pool=self.dev.k_pool, v_pool=self.dev.v_pool,
+                                  plan=self.plan, plan_host=self.plan_host, kv_len=self.kv_len, q_pos=self.q_pos,
+                                  rope_table=self.dev.rope, out=self.out, workspace=self.workspace,
+                                  workspace_bytes=self.ws_bytes, status=self.dev.status, batch=self.batch,
+                                  sm_scale=sm_scale, stream=s)
         return self.out
 
 
