@@ -208,6 +208,40 @@ class L2Flush:
         torch.sum(self.r, dim=0, out=self.acc)
 
 
+def measure_grouped(args, wl, dev, page_ids, pos_base, kv_len, q_pos, q_bits, logical_bytes: int):
+    """The same decode batch through mepic_attn_decode_grouped: requests that alias a page are scored against it
+    together.  Rate = the logical bytes a per-request decode must read / time, so it can exceed the HBM roofline."""
+    import torch
+    from paper_2512_16822_b200 import runtime as RT
+    t0 = time.perf_counter()
+    batch = RT.GroupedDecodeBatch(dev, page_ids, pos_base, kv_len, q_pos, q_bits)
+    setup_ms = 1e3 * (time.perf_counter() - t0)
+    t0 = time.perf_counter()
+    import paper_2512_16822_b200 as M
+    M.mepic_decode_plan_build(dev.cfg, page_ids, pos_base, kv_len)
+    plan_ms = 1e3 * (time.perf_counter() - t0)
+    stream = torch.cuda.current_stream()
+    flush = L2Flush(dev.device)
+    for _ in range(3):
+        batch.run(wl.sm_scale, stream)
+    steps = max(5, min(args.steps, 50))
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        flush()
+        a.record(stream); batch.run(wl.sm_scale, stream); b.record(stream)
+    torch.cuda.synchronize()
+    assert dev.read_status() == 0
+    ms = sum(a.elapsed_time(b) for a, b in evs) / steps
+    entries = int(sum(-(-int(k) // wl.page_size) for k in kv_len))
+    staged = int(batch.plan_host[12])
+    page_bytes = wl.page_size * kv_bytes_per_token(wl)
+    return {"value": logical_bytes / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms, "steps": steps,
+            "table_entries": entries, "pages_staged": staged, "staged_bytes_per_step": staged * page_bytes,
+            "staged_gbs": staged * page_bytes / (ms * 1e-3) / 1e9, "plan_build_ms": plan_ms, "plan_ints": int(len(batch.plan_host)),
+            "note": "sharing-aware decode (host plan + mepic_attn_decode_grouped); value = logical bytes of the per-request "
+                    "decode / time; L2 flushed between steps"}
+
+
 def measure_unshared(args, wl, device_index: int):
     """The same decode batch on a layout WITHOUT chunk sharing: every request owns a private copy of each of its
     chunks (one page per block-table entry), so no page is read twice and nothing can be served from L2 because a
@@ -402,7 +436,9 @@ def run_ours(args):
         return max_over_ranks(sum(xs), world, dev.device)
 
     tot, tot_warm, tot_e2e = agg(ms), agg(ms_warm), agg(ms_e2e)
-    prefill = unshared = None
+    prefill = unshared = grouped = None
+    if rank == 0 and world == 1 and not args.no_grouped:
+        grouped = measure_grouped(args, wl, dev, page_ids, pos_base, kv_len, q_pos, q_bits, logical_bytes)
     if rank == 0 and world == 1 and not args.no_prefill:
         prefill = measure_prefill(args, local_rank)
     if rank == 0 and world == 1 and not args.no_unshared:
@@ -441,6 +477,7 @@ def run_ours(args):
         "table_build_ms": table_build_ms,
         "prefill": prefill,
         "unshared_layout": unshared,
+        "grouped_decode": grouped,
     }
     if not args.no_cpu_baseline and world == 1:
         s = oracle_decode_sample(wl, args.cpu_budget)
@@ -466,6 +503,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true", help="skip the config-3 prefill measurement")
     ap.add_argument("--no-unshared", action="store_true", help="skip the decode run on the layout without sharing")
+    ap.add_argument("--no-grouped", action="store_true", help="skip the sharing-aware (grouped) decode run")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

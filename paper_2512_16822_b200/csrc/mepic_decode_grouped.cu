@@ -45,7 +45,7 @@ struct GroupedParams {
   int32_t* status;
   int n_kv_heads, page_size, log2_tpp, num_pages, max_position, batch;
   int n_items, piece, total;
-  int off_items, off_records, off_workers, off_req_off, off_req_items, off_req_ent;
+  int off_items, off_records, off_workers, off_req_ent, off_slot_base, off_part_off;
   float scale_log2;   // sm_scale * log2(e)
 };
 
@@ -170,7 +170,7 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
   __syncwarp();
 
   // per-unit state of the lane's two rows
-  int ui = -1, uh = -1, u_tail = -1, u_kvl = 0;
+  int ui = -1, uh = -1, u_tail = -1, u_kvl = 0, u_ts = 0;
   int reqA = -1, reqB = -1, qposA = 0, qposB = 0, angA = INT_MIN, angB = INT_MIN;
   float qlA[KH][2][2], qhA[KH][2][2], qlB[KH][2][2], qhB[KH][2][2];   // rotated, pre-scaled q: halves lo / hi
   float mA = -INFINITY, lA = 0.f, mB = -INFINITY, lB = 0.f;
@@ -181,18 +181,22 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
     float la = lA, lb = lB;
     la += __shfl_xor_sync(kFull, la, 1); la += __shfl_xor_sync(kFull, la, 2);
     lb += __shfl_xor_sync(kFull, lb, 1); lb += __shfl_xor_sync(kFull, lb, 2);
-    const long long slot0 = (static_cast<long long>(ui) * p.n_kv_heads + uh + w) * R;
+    // this worker is the k-th whose piece overlaps the unit
+    const long long k = w - (static_cast<long long>(u_ts) * p.n_kv_heads + static_cast<long long>(uh) * c_nt) / p.piece;
+    const int32_t* sb = p.plan + p.off_slot_base + (static_cast<size_t>(ui) * p.n_kv_heads + uh) * R;
     if (reqA >= 0) {
-      float* dst = p.part_o + ((slot0 + jA) * G + hA) * D;
+      const long long slot = __ldg(sb + jA) + k;
+      float* dst = p.part_o + (slot * G + hA) * D;
 #pragma unroll
       for (int nd = 0; nd < ND; ++nd) *reinterpret_cast<float2*>(dst + 8 * nd + 2 * t) = make_float2(acc[nd][0], acc[nd][1]);
-      if (t == 0) *reinterpret_cast<float2*>(p.part_ml + ((slot0 + jA) * G + hA) * 2) = make_float2(mA, la);
+      if (t == 0) *reinterpret_cast<float2*>(p.part_ml + (slot * G + hA) * 2) = make_float2(mA, la);
     }
     if (reqB >= 0) {
-      float* dst = p.part_o + ((slot0 + jB) * G + hB) * D;
+      const long long slot = __ldg(sb + jB) + k;
+      float* dst = p.part_o + (slot * G + hB) * D;
 #pragma unroll
       for (int nd = 0; nd < ND; ++nd) *reinterpret_cast<float2*>(dst + 8 * nd + 2 * t) = make_float2(acc[nd][2], acc[nd][3]);
-      if (t == 0) *reinterpret_cast<float2*>(p.part_ml + ((slot0 + jB) * G + hB) * 2) = make_float2(mB, lb);
+      if (t == 0) *reinterpret_cast<float2*>(p.part_ml + (slot * G + hB) * 2) = make_float2(mB, lb);
     }
   };
 
@@ -242,6 +246,7 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
         const int n_req = __ldg(hd + kPiReq);
         c_nt = __ldg(hd + kPiEnt) << p.log2_tpp;
         u_tail = __ldg(hd + kPiTail);
+        u_ts = __ldg(hd + kPiTileStart);
         reqA = jA < n_req ? __ldg(hd + kPiReqIds + jA) : -1;
         reqB = (jB < R && jB < n_req) ? __ldg(hd + kPiReqIds + jB) : -1;
         if (static_cast<unsigned>(reqA) >= static_cast<unsigned>(p.batch)) reqA = -1;
@@ -265,12 +270,6 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
       for (int nd = 0; nd < ND; ++nd) { acc[nd][0] = 0.f; acc[nd][1] = 0.f; acc[nd][2] = 0.f; acc[nd][3] = 0.f; }
     }
 
-    if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity)) {
-      // Give the copies still in flight a last bounded chance to land, then leave cleanly.
-      if (lane == 0) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
-      for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(&bars[s]), s == stage ? parity : (s < stage ? parity ^ 1u : parity));
-      return;
-    }
     const uint32_t ks_addr = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
     const uint32_t vs_addr = ks_addr + NB * kBlockBytes;
     // only the partly filled last page of a request (always in its single-request item) has invalid slots
@@ -278,9 +277,18 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
     if (u_tail >= 0 && (ct >> p.log2_tpp) == (c_nt >> p.log2_tpp) - 1)
       n_valid = min(kTile, u_kvl - u_tail - (ct & ((1 << p.log2_tpp) - 1)) * kTile);
 
+    // the query rows need only the tile's base positions (written when the stage was issued), not its data
     if (n_valid > 0) {
       if (reqA >= 0) rotate_row(qlA, qhA, angA, qposA - meta[stage * 8 + jA], reqA, hA);
       if (reqB >= 0) rotate_row(qlB, qhB, angB, qposB - meta[stage * 8 + (jB < R ? jB : 0)], reqB, hB);
+    }
+    if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity)) {
+      // Give the copies still in flight a last bounded chance to land, then leave cleanly.
+      if (lane == 0) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
+      for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(&bars[s]), s == stage ? parity : (s < stage ? parity ^ 1u : parity));
+      return;
+    }
+    if (n_valid > 0) {
 
       // slots at or past kv_len may hold anything (NaN bit patterns included): their P is 0, but 0 x NaN is NaN,
       // so V must be finite there.
@@ -376,41 +384,31 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
 }
 
 // ---------------------------------------------------------------- merge
-// One CTA per (request, kv head); thread (g, d) folds in every partial the plan says the pair has: for each
-// (item, row-request) the request takes part in, one partial per worker whose piece overlaps the unit.
+// One CTA per (request, kv head); thread (g, d) folds in the pair's partials, which the plan laid out as one
+// contiguous run of slots: m* = max m, l* = sum l 2^(m - m*), out = sum o 2^(m - m*) / l*  -> bf16.
 template <int D, int G>
 __global__ void mepic_decode_grouped_merge(const GroupedParams p) {
-  constexpr int R = plan_group_requests(G);
-  constexpr int kItemInts = kItemFixed + R;
   const int b = blockIdx.x / p.n_kv_heads, h = blockIdx.x % p.n_kv_heads;
   const int g = threadIdx.x / D, d = threadIdx.x % D;
   if (h == 0 && threadIdx.x == 0) {
     const int kvl = p.kv_len[b];
     if ((kvl + p.page_size - 1) / p.page_size != p.plan[p.off_req_ent + b]) atomicOr(p.status, MEPIC_DEV_BAD_PLAN);
   }
-  const int32_t* items = p.plan + p.off_items;
-  float m_run = -INFINITY, l_run = 0.f, o_run = 0.f;
-  const int i0 = p.plan[p.off_req_off + b], i1 = p.plan[p.off_req_off + b + 1];
-  for (int i = i0; i < i1; ++i) {
-    const int v = p.plan[p.off_req_items + i];
-    const int item = v >> 4, j = v & 15;
-    const long long nt = static_cast<long long>(items[static_cast<size_t>(item) * kItemInts + kPiEnt]) << p.log2_tpp;
-    const long long start = static_cast<long long>(items[static_cast<size_t>(item) * kItemInts + kPiTileStart]) * p.n_kv_heads + h * nt;
-    const long long w_first = start / p.piece, w_last = (start + nt - 1) / p.piece;
-    const long long unit = static_cast<long long>(item) * p.n_kv_heads + h;
-    for (long long wk = w_first; wk <= w_last; ++wk) {
-      const long long row = ((unit + wk) * R + j) * G + g;
-      const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + row * 2);
-      if (!(ml.y > 0.f)) continue;                       // a piece that saw no valid slot of this row
-      const float m_new = fmaxf(m_run, ml.x);
-      const float f_old = ex2(m_run - m_new), f_new = ex2(ml.x - m_new);
-      l_run = l_run * f_old + ml.y * f_new;
-      o_run = o_run * f_old + p.part_o[row * D + d] * f_new;
-      m_run = m_new;
-    }
+  const int k0 = __ldg(p.plan + p.off_part_off + blockIdx.x), k1 = __ldg(p.plan + p.off_part_off + blockIdx.x + 1);
+  // a piece that saw no valid slot of the row left (max, sum) = (-inf, 0): it drops out of both passes
+  float m_star = -INFINITY;
+  for (int k = k0; k < k1; ++k) m_star = fmaxf(m_star, p.part_ml[(static_cast<size_t>(k) * G + g) * 2]);
+  float l_star = 0.f, o_star = 0.f;
+#pragma unroll 4
+  for (int k = k0; k < k1; ++k) {
+    const size_t row = static_cast<size_t>(k) * G + g;
+    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + row * 2);
+    const float wgt = ml.y > 0.f ? ex2(ml.x - m_star) : 0.f;
+    l_star += ml.y * wgt;
+    o_star += p.part_o[row * D + d] * wgt;
   }
   const size_t o_at = (static_cast<size_t>(b) * p.n_kv_heads * G + static_cast<size_t>(h) * G + g) * D + d;
-  p.out[o_at] = l_run > 0.f ? f32_to_bf16_bits(o_run / l_run) : static_cast<uint16_t>(0);
+  p.out[o_at] = l_star > 0.f ? f32_to_bf16_bits(o_star / l_star) : static_cast<uint16_t>(0);
 }
 
 template <int D, int G>
@@ -436,15 +434,13 @@ bool plan_header_ok(const mepic_config_t* cfg, const int32_t* h, int32_t batch) 
   if (!h || h[kPhMagic] != kPlanMagic) { mepic_set_error("decode_grouped: plan_host is not a plan"); return false; }
   const int G = cfg->n_q_heads / cfg->n_kv_heads;
   if (h[kPhR] != plan_group_requests(G) || h[kPhPageSize] != cfg->page_size || (batch >= 0 && h[kPhBatch] != batch) ||
-      h[kPhWorkers] < kWarps || h[kPhWorkers] % kWarps != 0 || h[kPhPiece] < 1 || h[kPhItems] < 1) {
+      h[kPhKvHeads] != cfg->n_kv_heads || h[kPhWorkers] < kWarps || h[kPhWorkers] % kWarps != 0 || h[kPhPiece] < 1 || h[kPhItems] < 1) {
     mepic_set_error("decode_grouped: the plan was built for another config or batch"); return false;
   }
   return true;
 }
 
-size_t grouped_slots(const mepic_config_t* cfg, const int32_t* h) {
-  return (static_cast<size_t>(h[kPhItems]) * cfg->n_kv_heads + h[kPhWorkers]) * h[kPhR];
-}
+size_t grouped_slots(const mepic_config_t*, const int32_t* h) { return static_cast<size_t>(h[kPhSlots]) + 1; }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -484,7 +480,7 @@ extern "C" int32_t mepic_attn_decode_grouped(const mepic_config_t* cfg, const me
   p.num_pages = cfg->num_pages; p.max_position = cfg->max_position; p.batch = a->batch;
   p.n_items = h[kPhItems]; p.piece = h[kPhPiece]; p.total = h[kPhTotal];
   p.off_items = h[kPhOffItems]; p.off_records = h[kPhOffRecords]; p.off_workers = h[kPhOffWorkers];
-  p.off_req_off = h[kPhOffReqOff]; p.off_req_items = h[kPhOffReqItems]; p.off_req_ent = h[kPhOffReqEnt];
+  p.off_req_ent = h[kPhOffReqEnt]; p.off_slot_base = h[kPhOffSlotBase]; p.off_part_off = h[kPhOffPartOff];
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   alignas(64) CUtensorMap map_k, map_v;

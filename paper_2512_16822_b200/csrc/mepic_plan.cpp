@@ -49,7 +49,7 @@ extern "C" size_t mepic_decode_plan_max_ints(const mepic_config_t* cfg, int32_t 
   const int R = plan_group_requests(cfg->n_q_heads / cfg->n_kv_heads);
   const size_t E = static_cast<size_t>(batch) * table_stride;     // every entry is one record of one item at most
   return kPlanHeaderInts + E * (kItemFixed + R) + E * (1 + R) + static_cast<size_t>(sms) * kPlanWarps * 3 +
-         (batch + 1) + E + batch;
+         (batch + 1) + E + batch + E * cfg->n_kv_heads * R + static_cast<size_t>(batch) * cfg->n_kv_heads + 1;
 }
 
 extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int32_t* page_ids, const int32_t* pos_base,
@@ -132,7 +132,9 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
   const size_t off_req_off = off_workers + static_cast<size_t>(n_workers) * 3;
   const size_t off_req_items = off_req_off + batch + 1;
   const size_t off_req_ent = off_req_items + n_req_items;
-  const size_t ints = off_req_ent + batch;
+  const size_t off_slot_base = off_req_ent + batch;
+  const size_t off_part_off = off_slot_base + items.size() * Hkv * R;
+  const size_t ints = off_part_off + static_cast<size_t>(batch) * Hkv + 1;
   *out_ints = ints;
   if (ints > cap_ints) { mepic_set_error("decode_plan: plan needs %zu ints, buffer holds %zu", ints, cap_ints); return MEPIC_E_CAPACITY; }
 
@@ -143,6 +145,9 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
   h[kPhOffWorkers] = static_cast<int32_t>(off_workers); h[kPhOffReqOff] = static_cast<int32_t>(off_req_off);
   h[kPhOffReqItems] = static_cast<int32_t>(off_req_items); h[kPhBatch] = batch; h[kPhRecords] = static_cast<int32_t>(n_records);
   h[kPhInts] = static_cast<int32_t>(ints); h[kPhOffReqEnt] = static_cast<int32_t>(off_req_ent); h[kPhPageSize] = P;
+  h[kPhOffSlotBase] = static_cast<int32_t>(off_slot_base); h[kPhOffPartOff] = static_cast<int32_t>(off_part_off);
+  h[kPhKvHeads] = Hkv;
+  for (int k = kPhKvHeads + 1; k < kPlanHeaderInts; ++k) h[k] = 0;
 
   std::vector<std::vector<int32_t>> req_items(batch);
   int32_t rec = 0, tile_start = 0;
@@ -187,5 +192,37 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
     out_plan[off_req_ent + r] = n_ent[r];
   }
   out_plan[off_req_off + batch] = at;
+
+  // partial slots: a unit (item, kv head) is overlapped by the pieces w_first..w_last of the line; each of its rows gets
+  // one slot per piece, and the slots of a (request, kv head) pair are contiguous so that the merge reads one run
+  std::vector<long long> count(static_cast<size_t>(batch) * Hkv + 1, 0);
+  auto pieces_of = [&](size_t i, int hd) {
+    const long long nt = static_cast<long long>(items[i].ent.size()) * tpp;
+    const long long start = static_cast<long long>(out_plan[off_items + i * (kItemFixed + R) + kPiTileStart]) * Hkv + hd * nt;
+    return (start + nt - 1) / piece - start / piece + 1;
+  };
+  for (size_t i = 0; i < items.size(); ++i)
+    for (int hd = 0; hd < Hkv; ++hd)
+      for (int32_t r : items[i].req) count[static_cast<size_t>(r) * Hkv + hd] += pieces_of(i, hd);
+  long long run = 0;
+  for (size_t u = 0; u < static_cast<size_t>(batch) * Hkv; ++u) {
+    out_plan[off_part_off + u] = static_cast<int32_t>(run);
+    const long long c = count[u]; count[u] = run; run += c;
+  }
+  if (run >= (1ll << 31)) { mepic_set_error("decode_plan: too many partials for the plan's 32-bit fields"); return MEPIC_E_CAPACITY; }
+  out_plan[off_part_off + static_cast<size_t>(batch) * Hkv] = static_cast<int32_t>(run);
+  h[kPhSlots] = static_cast<int32_t>(run);
+  for (size_t i = 0; i < items.size(); ++i)
+    for (int hd = 0; hd < Hkv; ++hd) {
+      const long long c = pieces_of(i, hd);
+      for (int j = 0; j < R; ++j) {
+        int32_t v = 0;
+        if (j < static_cast<int>(items[i].req.size())) {
+          long long& cur = count[static_cast<size_t>(items[i].req[j]) * Hkv + hd];
+          v = static_cast<int32_t>(cur); cur += c;
+        }
+        out_plan[off_slot_base + (i * Hkv + hd) * R + j] = v;
+      }
+    }
   return MEPIC_OK;
 }

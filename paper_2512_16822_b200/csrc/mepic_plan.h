@@ -9,6 +9,9 @@
 //   req_off  [batch + 1]                 CSR over req_items
 //   req_items[...]                       item * 16 + j for every (item, row-request j) a request takes part in
 //   req_ent  [batch]                     table entries each request had when the plan was built
+//   slot_base[n_items][n_kv_heads][R]    first partial slot of (item, kv head, row-request): the worker whose piece is
+//                                        the k-th to overlap the unit writes slot_base + k
+//   part_off [batch * n_kv_heads + 1]    the partial slots of (request, kv head) are part_off[u] .. part_off[u+1]-1
 //
 // R = requests per group.  The line is item-major, then kv head, then tile; an item's tile count
 // per head is n_ent * (page_size / 16); tile_start is the sum of the tile counts of the items
@@ -19,11 +22,12 @@
 #include <stdint.h>
 
 constexpr int32_t kPlanMagic = 0x4d504c31;   // "MPL1"
-constexpr int kPlanHeaderInts = 16;
+constexpr int kPlanHeaderInts = 24;
 constexpr int kItemFixed = 5;
 enum PlanHeader {
   kPhMagic = 0, kPhItems, kPhWorkers, kPhPiece, kPhTotal, kPhR, kPhOffItems, kPhOffRecords, kPhOffWorkers,
-  kPhOffReqOff, kPhOffReqItems, kPhBatch, kPhRecords, kPhInts, kPhOffReqEnt, kPhPageSize
+  kPhOffReqOff, kPhOffReqItems, kPhBatch, kPhRecords, kPhInts, kPhOffReqEnt, kPhPageSize,
+  kPhOffSlotBase, kPhOffPartOff, kPhSlots, kPhKvHeads
 };
 enum PlanItem { kPiReq = 0, kPiRecOff, kPiEnt, kPiTail, kPiTileStart, kPiReqIds };
 

@@ -15,7 +15,7 @@ import paper_2512_16822_b200 as M
 from paper_2512_16822_b200 import runtime as RT
 from mepic_inputs import make_workload
 
-HEADER, ITEM_FIXED = 16, 5
+HEADER, ITEM_FIXED = 24, 5
 MAGIC = 0x4d504c31
 
 
@@ -31,7 +31,12 @@ def _parse(plan, Hkv, P):
     req_off = plan[off_req_off:off_req_off + batch + 1]
     req_items = plan[off_req_items:off_req_items + req_off[-1]]
     req_ent = plan[off_req_ent:off_req_ent + batch]
-    return dict(n_items=n_items, n_workers=n_workers, piece=piece, total=total, R=R, items=items, recs=recs,
+    off_slot_base, off_part_off, n_slots = int(h[16]), int(h[17]), int(h[18])
+    assert int(h[19]) == Hkv
+    slot_base = plan[off_slot_base:off_slot_base + n_items * Hkv * R].reshape(n_items, Hkv, R)
+    part_off = plan[off_part_off:off_part_off + batch * Hkv + 1]
+    assert part_off[0] == 0 and part_off[-1] == n_slots and (np.diff(part_off) >= 1).all()
+    return dict(slot_base=slot_base, part_off=part_off, n_items=n_items, n_workers=n_workers, piece=piece, total=total, R=R, items=items, recs=recs,
                 workers=workers, req_off=req_off, req_items=req_items, req_ent=req_ent, batch=batch)
 
 
@@ -89,6 +94,18 @@ def _check_plan(cfg, page_ids, pos_base, kv_len, n_sms=148):
         it = pl["items"][item]
         nt = int(it[2]) * tpp
         assert 0 <= head < Hkv and 0 <= tile < nt and int(it[4]) * Hkv + head * nt + tile == x
+    # partial slots: unit (item, head) overlaps pieces w_first..w_last; its rows' slots tile each (request, head) run exactly
+    taken = np.zeros(int(pl["part_off"][-1]), dtype=np.int32)
+    for i, it in enumerate(pl["items"]):
+        nt = int(it[2]) * tpp
+        for hd in range(Hkv):
+            start = int(it[4]) * Hkv + hd * nt
+            cnt = (start + nt - 1) // pl["piece"] - start // pl["piece"] + 1
+            for j in range(int(it[0])):
+                r = int(it[ITEM_FIXED + j]); s0 = int(pl["slot_base"][i, hd, j])
+                assert pl["part_off"][r * Hkv + hd] <= s0 and s0 + cnt <= pl["part_off"][r * Hkv + hd + 1]
+                taken[s0:s0 + cnt] += 1
+    assert (taken == 1).all()
     # per-request index of (item, row)
     for r in range(len(kv_len)):
         mine = [int(v) for v in pl["req_items"][pl["req_off"][r]:pl["req_off"][r + 1]]]
