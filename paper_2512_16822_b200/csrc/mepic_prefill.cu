@@ -700,25 +700,30 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     // =============================================================== MMA issuer (one thread)
     // Order per key tile j:  PV_a(j), QK_a(j+1), PV_b(j), QK_b(j+1): while one M-tile's softmax runs, the
     // tensor core works on the other M-tile.  S of an M-tile is reused by its P, so QK_x(j+1) follows PV_x(j).
-    const uint32_t q_addr[2] = {smem_u32(Qs), smem_u32(Qs + NB * kBlockBytes)};
+    // The issuing thread shares its scheduler with softmax and rotator warps and the tensor pipe waits on it between
+    // an M-tile's P and its next S, so the issue loops carry as few instructions as possible: every descriptor is a
+    // base computed once plus a compile-time constant in its 16-byte-unit address field.
+    const uint64_t q_desc[2] = {smem_desc(smem_u32(Qs), 16, 1024), smem_desc(smem_u32(Qs + NB * kBlockBytes), 16, 1024)};
+    const uint64_t k_desc0 = smem_desc(smem_u32(Ks), 16, 1024);
+    const uint64_t v_desc0 = smem_desc(smem_u32(Vs), kBlockBytes, 1024);
+    constexpr uint64_t kStageUnits = (NB * kBlockBytes) >> 4;
     bool ok = true;
     auto issue_qk = [&](int x, int j) {
-      const uint32_t k_addr = smem_u32(Ks + (j % kKStages) * NB * kBlockBytes);
+      const uint64_t kd = k_desc0 + static_cast<uint64_t>(j % kKStages) * kStageUnits;
 #pragma unroll
       for (int ks = 0; ks < D / 16; ++ks) {
-        const uint32_t off = (ks / 4) * kBlockBytes + (ks % 4) * 32;
-        tc_mma(tmem_base + static_cast<uint32_t>(x * 128), smem_desc(q_addr[x] + off, 16, 1024),
-               smem_desc(k_addr + off, 16, 1024), kIdescQK, ks > 0);
+        const uint64_t off = static_cast<uint64_t>(((ks / 4) * kBlockBytes + (ks % 4) * 32) >> 4);
+        tc_mma(tmem_base + static_cast<uint32_t>(x * 128), q_desc[x] + off, kd + off, kIdescQK, ks > 0);
       }
       tc_commit(BAR(kBarSFull, x));
     };
     auto issue_pv = [&](int x, int j) {
-      const uint32_t v_addr = smem_u32(Vs + (j % kVStages) * NB * kBlockBytes);
+      const uint64_t vd = v_desc0 + static_cast<uint64_t>(j % kVStages) * kStageUnits;
 #pragma unroll
       for (int ks = 0; ks < kTileN / 16; ++ks) {
         // A = P from tensor memory: 16 bf16 per k-step = 8 columns, keys 0..63 at columns 0.., keys 64..127 at 64..; B = V, MN-major
         tc_mma_ts(tmem_base + 256u + static_cast<uint32_t>(x * 128), tmem_base + static_cast<uint32_t>(x * 128 + (ks / 4) * 64 + (ks % 4) * 8),
-                  smem_desc(v_addr + ks * 2048, kBlockBytes, 1024), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
+                  vd + static_cast<uint64_t>((ks * 2048) >> 4), kIdescPV, (j > 0 || ks > 0) ? 1u : 0u);
       }
       tc_commit(BAR(kBarPvDone, x));
     };
