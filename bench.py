@@ -411,16 +411,17 @@ def run_ours(args):
     ms_warm = timed(args.steps, step, flush=False)
 
     # end to end: the step's inputs come from pinned host memory, the result goes back to the host
-    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
-    h_q = pin(q_bits.view(np.int16)); h_ids = pin(page_ids); h_base = pin(pos_base); h_len = pin(kv_len); h_qpos = pin(q_pos)
+    # one pinned mirror of the step's inputs (q + block tables + lengths + positions): one copy in, one copy out
+    h_in, hv = batch.host_mirror()
+    hv["q"].copy_(torch.from_numpy(np.ascontiguousarray(q_bits).view(np.int16)))
+    hv["page_ids"].copy_(torch.from_numpy(page_ids)); hv["pos_base"].copy_(torch.from_numpy(pos_base))
+    hv["kv_len"].copy_(torch.from_numpy(kv_len)); hv["q_pos"].copy_(torch.from_numpy(q_pos))
     h_out = torch.empty(batch.out.shape, dtype=torch.bfloat16).pin_memory()
-    h2d = sum(int(t.numel() * t.element_size()) for t in (h_q, h_ids, h_base, h_len, h_qpos))
+    h2d = int(h_in.numel())
     d2h = int(h_out.numel() * h_out.element_size())
 
     def e2e_step():
-        batch.q.view(torch.int16).copy_(h_q, non_blocking=True)
-        batch.page_ids.copy_(h_ids, non_blocking=True); batch.pos_base.copy_(h_base, non_blocking=True)
-        batch.kv_len.copy_(h_len, non_blocking=True); batch.q_pos.copy_(h_qpos, non_blocking=True)
+        batch.upload(h_in)
         batch.run(wl.sm_scale, stream)
         h_out.copy_(batch.out, non_blocking=True)
 

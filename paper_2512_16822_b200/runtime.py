@@ -109,12 +109,26 @@ class DecodeBatch:
         self.dev = dev
         self.batch, self.stride = page_ids.shape
         d = dev.device
-        self.page_ids = torch.from_numpy(np.ascontiguousarray(page_ids, dtype=np.int32)).to(d)
-        self.pos_base = torch.from_numpy(np.ascontiguousarray(pos_base, dtype=np.int32)).to(d)
-        self.kv_len = torch.from_numpy(np.ascontiguousarray(kv_len, dtype=np.int32)).to(d)
-        self.q_pos = torch.from_numpy(np.ascontiguousarray(q_pos, dtype=np.int32)).to(d)
+        # The per-step inputs (q and the tables) are views of ONE device buffer, so that a serving loop can bring a
+        # step's inputs over with a single host-to-device copy from a pinned mirror (see host_mirror / upload).
         qshape = (self.batch, cfg.n_q_heads, cfg.head_dim)
-        self.q = bf16_tensor(q_bits, d) if q_bits is not None else torch.empty(qshape, dtype=torch.bfloat16, device=d)
+        parts = [("q", qshape, torch.bfloat16), ("page_ids", (self.batch, self.stride), torch.int32),
+                 ("pos_base", (self.batch, self.stride), torch.int32), ("kv_len", (self.batch,), torch.int32),
+                 ("q_pos", (self.batch,), torch.int32)]
+        self._layout, at = [], 0
+        for name, shape, dt in parts:
+            n = int(np.prod(shape)) * torch.empty((), dtype=dt).element_size()
+            self._layout.append((name, shape, dt, at, n))
+            at += -(-n // 256) * 256                                   # every view starts 256-byte aligned
+        self.step_inputs = torch.empty(at, dtype=torch.uint8, device=d)
+        for name, shape, dt, off, n in self._layout:
+            setattr(self, name, self.step_inputs[off:off + n].view(dt).view(shape))
+        self.page_ids.copy_(torch.from_numpy(np.ascontiguousarray(page_ids, dtype=np.int32)))
+        self.pos_base.copy_(torch.from_numpy(np.ascontiguousarray(pos_base, dtype=np.int32)))
+        self.kv_len.copy_(torch.from_numpy(np.ascontiguousarray(kv_len, dtype=np.int32)))
+        self.q_pos.copy_(torch.from_numpy(np.ascontiguousarray(q_pos, dtype=np.int32)))
+        if q_bits is not None:
+            self.q.view(torch.int16).copy_(torch.from_numpy(np.ascontiguousarray(q_bits).view(np.int16)))
         self.out = torch.empty(qshape, dtype=torch.bfloat16, device=d)
         self.ws_bytes = mepic_attn_decode_workspace(cfg, self.batch)
         self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=d)
@@ -127,6 +141,19 @@ class DecodeBatch:
                           workspace_bytes=self.ws_bytes, status=self.dev.status, table_stride=self.stride,
                           batch=self.batch, sm_scale=sm_scale, stream=s)
         return self.out
+
+    def host_mirror(self):
+        """Pinned host buffer with the layout of ``step_inputs`` and named views into it (q as int16 bit patterns)."""
+        host = torch.empty(self.step_inputs.numel(), dtype=torch.uint8).pin_memory()
+        views = {}
+        for name, shape, dt, off, n in self._layout:
+            hdt = torch.int16 if dt == torch.bfloat16 else dt
+            views[name] = host[off:off + n].view(hdt).view(shape)
+        return host, views
+
+    def upload(self, host: torch.Tensor) -> None:
+        """One asynchronous host-to-device copy of a whole step's inputs (on the current stream)."""
+        self.step_inputs.copy_(host, non_blocking=True)
 
 
 class GroupedDecodeBatch:
