@@ -92,6 +92,10 @@ typedef struct {
   int64_t live_requests;
   int64_t chunks_evicted;             /* zero-reference chunk objects reclaimed under memory pressure */
   int64_t pages_evicted;              /* pages those evictions returned to the pool */
+  int64_t chunks_spilled;             /* evicted chunks whose pages were copied to the remote tier */
+  int64_t chunks_fetched;             /* registrations served from the remote tier */
+  int64_t remote_chunks;              /* chunks the remote tier holds now */
+  int64_t remote_pages;               /* page slots of the remote tier in use */
 } mepic_stats_t;
 
 typedef struct {
@@ -136,7 +140,8 @@ void    mepic_store_destroy(mepic_store_t* store);
  * pad_token_id to a multiple of page_size, hashes the padded sequence (64-bit FNV-1a, confirmed by
  * a full token compare, so identity is by content) and looks it up.  On a miss it takes
  * ceil(n/page_size) - 1 pages from the pool for the shareable blocks; on a hit it allocates
- * nothing (a miss may first reclaim idle chunks, see mepic_store_create).  out_chunk_id, out_was_resident (0/1), out_lead_pad (pad tokens added), out_n_shared:
+ * nothing (a miss may first reclaim idle chunks, see mepic_store_create).  out_chunk_id, out_was_resident
+ * (0 = new, 1 = resident, 2 = brought back from the remote tier, see mepic_store_attach_remote), out_lead_pad (pad tokens added), out_n_shared:
  * host, each may be NULL.  out_shared_pages (host, cap entries, may be NULL when cap == 0)
  * receives the shared page ids in block order.
  * Errors: E_INVAL; E_NOSPACE (nothing allocated, chunk not registered); E_CAPACITY (cap too small:
@@ -189,6 +194,30 @@ int32_t mepic_request_release(mepic_store_t* store, int64_t request_id);
 
 /* Snapshot of the pool ("HBM usage" of Section 4 in units of pages).  out: host. */
 int32_t mepic_store_stats(const mepic_store_t* store, mepic_stats_t* out);
+
+/*
+ * mepic_store_attach_remote - a second tier behind the HBM pool for chunk KV, standing in for the
+ * remote chunk store of the paper's serving stack (Section 3.1; Algorithm 1 "resolve HBM residency
+ * and remote availability"; Section 3.2.3 eviction).  capacity_pages page slots of host memory are
+ * allocated (page-locked when the pools are device memory).  From then on
+ *   - a computed chunk reclaimed under memory pressure (Section 3.2.3) first has its shareable pages
+ *     copied, K and V, into the tier; the tier drops its own least recently used chunks to make room,
+ *     and a chunk larger than the whole tier is not kept;
+ *   - mepic_chunk_register of a chunk that is not resident but is in the tier allocates its pages as
+ *     for a miss and copies the K/V back into them: *out_was_resident = 2, the pages need no
+ *     recomputation (only the first block does, per request, as for any cached chunk).  The tier keeps
+ *     its copy.
+ * k_pool / v_pool: the pools the kernels read, [num_pages][n_kv_heads][page_size][head_dim] bf16.
+ * pools_on_host = 0: DEVICE pointers; copies are cudaMemcpyAsync on cuda_stream, so they are ordered
+ * with the caller's kernels only if those run on the same stream (or the caller synchronises), and a
+ * page handed out by a call may still be the source of a copy enqueued by that call.
+ * pools_on_host = 1: HOST pointers and plain memcpy (no CUDA call at all; cuda_stream ignored) - for
+ * host-only use and tests.  One tier per store; E_EXISTS if already attached, E_INVAL for bad
+ * arguments, E_CUDA if page-locked memory cannot be had or (later, from the call that triggered it)
+ * a copy cannot be enqueued.  The tier is freed by mepic_store_destroy.
+ */
+int32_t mepic_store_attach_remote(mepic_store_t* store, void* k_pool, void* v_pool, int32_t pools_on_host,
+                                  int64_t capacity_pages, void* cuda_stream);
 
 /* ---------------------------------------------------------------- rope table (host, set-up)
  *

@@ -85,6 +85,30 @@ class OracleStore:
         self.tick = 0
         self.chunks_evicted = 0
         self.pages_evicted = 0
+        self.remote = None              # see attach_remote
+
+    # Algorithm 1 "resolve HBM residency and remote availability" / Section 3.2.3 eviction: a second tier that
+    # keeps the K/V of evicted chunks (here: copies of the page arrays) and gives them back on the next use.
+    def attach_remote(self, k_pool: np.ndarray, v_pool: np.ndarray, capacity_pages: int) -> None:
+        if self.remote is not None:
+            raise ValueError("already attached")
+        self.remote = {"k": k_pool, "v": v_pool, "cap": int(capacity_pages), "used": 0, "chunks": {}, "tick": 0,
+                       "spilled": 0, "fetched": 0}
+
+    def _spill(self, key, pages) -> None:
+        r = self.remote
+        r["tick"] += 1
+        if key in r["chunks"]:
+            r["chunks"][key]["last_use"] = r["tick"]        # shared pages never change once computed
+            return
+        if len(pages) > r["cap"]:
+            return
+        while r["cap"] - r["used"] < len(pages):            # the tier drops its own least recently used chunks
+            victim = min(r["chunks"], key=lambda k: r["chunks"][k]["last_use"])
+            r["used"] -= len(r["chunks"].pop(victim)["kv"])
+        r["chunks"][key] = {"kv": [(r["k"][p].copy(), r["v"][p].copy()) for p in pages], "last_use": r["tick"]}
+        r["used"] += len(pages)
+        r["spilled"] += 1
 
     def _touch(self, key) -> None:
         self.tick += 1
@@ -103,7 +127,10 @@ class OracleStore:
         for _, k in sorted(cand, key=lambda x: x[0]):
             if need <= len(self.free):
                 break
-            pages = sorted(self.chunks.pop(k)["shared"])
+            gone = self.chunks.pop(k)
+            if self.remote is not None and not gone["uncomputed"]:
+                self._spill(k, gone["shared"])
+            pages = sorted(gone["shared"])
             self.free.extend(pages)
             self.chunks_evicted += 1
             self.pages_evicted += len(pages)
@@ -123,7 +150,7 @@ class OracleStore:
         if key in self.chunks:
             self.dedup_hits += 1
             self._touch(key)
-            return key, True, list(self.chunks[key]["shared"])
+            return key, 1, list(self.chunks[key]["shared"])
         n_pages = len(key) // self.P
         n_shared = n_pages - 1          # first block is private per request
         if not self._make_room(n_shared):
@@ -131,7 +158,16 @@ class OracleStore:
         shared = [self.free.popleft() for _ in range(n_shared)]
         self.chunks[key] = {"shared": shared, "refs": 0, "n_pages": n_pages, "last_use": 0, "uncomputed": False}
         self._touch(key)
-        return key, False, list(shared)
+        r = self.remote
+        if r is not None and shared and key in r["chunks"]:      # not in HBM, but a remote copy exists: bring it back
+            r["tick"] += 1
+            r["chunks"][key]["last_use"] = r["tick"]
+            for p, (kpage, vpage) in zip(shared, r["chunks"][key]["kv"]):
+                r["k"][p] = kpage
+                r["v"][p] = vpage
+            r["fetched"] += 1
+            return key, 2, list(shared)
+        return key, 0, list(shared)
 
     # Section 3.3.1: a newly encountered chunk (nobody has its K/V) is recomputed whole by the next request
     # that uses it; cached chunks recompute their first block only.
@@ -217,6 +253,10 @@ class OracleStore:
             "live_requests": len(self.requests),
             "chunks_evicted": self.chunks_evicted,
             "pages_evicted": self.pages_evicted,
+            "chunks_spilled": self.remote["spilled"] if self.remote else 0,
+            "chunks_fetched": self.remote["fetched"] if self.remote else 0,
+            "remote_chunks": len(self.remote["chunks"]) if self.remote else 0,
+            "remote_pages": self.remote["used"] if self.remote else 0,
         }
 
 

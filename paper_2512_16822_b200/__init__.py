@@ -22,7 +22,7 @@ from .build import LIB_PATH, build_library
 __all__ = [
     "MepicError", "Config", "Segment", "Store", "lib",
     "mepic_store_create", "mepic_store_destroy", "mepic_chunk_register", "mepic_build_block_table",
-    "mepic_request_release", "mepic_chunk_mark_uncomputed", "mepic_store_stats", "mepic_rope_table_floats", "mepic_rope_table_fill",
+    "mepic_request_release", "mepic_chunk_mark_uncomputed", "mepic_store_stats", "mepic_store_attach_remote", "mepic_rope_table_floats", "mepic_rope_table_fill",
     "mepic_attn_decode_workspace", "mepic_attn_decode", "mepic_attn_decode_static",
     "mepic_decode_plan_max_ints", "mepic_decode_plan_build", "mepic_attn_decode_grouped_workspace",
     "mepic_attn_decode_grouped",
@@ -64,7 +64,7 @@ class _StatsC(C.Structure):
     _fields_ = [(n, C.c_int64) for n in (
         "pages_total", "pages_free", "pages_shared_held", "pages_private_held", "chunks_resident",
         "chunk_refs", "dedup_hits", "unshared_equivalent_pages", "live_requests", "chunks_evicted",
-        "pages_evicted")]
+        "pages_evicted", "chunks_spilled", "chunks_fetched", "remote_chunks", "remote_pages")]
 
 
 class _SegmentC(C.Structure):
@@ -134,6 +134,7 @@ _PROTOTYPES = {
     "mepic_request_release": (C.c_int32, [C.c_void_p, C.c_int64]),
     "mepic_chunk_mark_uncomputed": (C.c_int32, [C.c_void_p, C.c_uint64]),
     "mepic_store_stats": (C.c_int32, [C.c_void_p, C.POINTER(_StatsC)]),
+    "mepic_store_attach_remote": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_void_p]),
     "mepic_rope_table_floats": (C.c_size_t, [C.POINTER(_ConfigC)]),
     "mepic_rope_table_fill": (C.c_int32, [C.POINTER(_ConfigC), C.c_void_p]),
     "mepic_attn_decode_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32]),
@@ -213,14 +214,14 @@ def mepic_store_destroy(store: int) -> None:
 
 
 def mepic_chunk_register(store: int, tokens: np.ndarray) -> Tuple[int, bool, int, np.ndarray]:
-    """-> (chunk_id, was_resident, lead_pad, shared_pages int32[])."""
+    """-> (chunk_id, was_resident, lead_pad, shared_pages int32[]); was_resident: 0 new, 1 resident, 2 from the remote tier."""
     tok = np.ascontiguousarray(tokens, dtype=np.int32)
     cid, res, lead, n = C.c_uint64(), C.c_int32(), C.c_int32(), C.c_int32()
     cap = max(int(tok.size), 1)          # a chunk never has more pages than tokens
     pages = np.empty(cap, dtype=np.int32)
     _check(lib().mepic_chunk_register(store, tok.ctypes.data, int(tok.size), C.byref(cid), C.byref(res),
                                       C.byref(lead), pages.ctypes.data, cap, C.byref(n)))
-    return int(cid.value), bool(res.value), int(lead.value), pages[:n.value].copy()
+    return int(cid.value), int(res.value), int(lead.value), pages[:n.value].copy()
 
 
 def mepic_build_block_table(store: int, request_id: int, segments: Sequence[Segment]
@@ -261,6 +262,17 @@ def mepic_store_stats(store: int) -> dict:
     return {name: int(getattr(st, name)) for name, _ in _StatsC._fields_}
 
 
+def mepic_store_attach_remote(store: int, k_pool, v_pool, capacity_pages: int, stream=None) -> None:
+    """Attach the remote tier.  numpy pools: host mode (plain memcpy); torch CUDA tensors: device mode."""
+    on_host = isinstance(k_pool, np.ndarray)
+    if on_host:
+        assert k_pool.flags["C_CONTIGUOUS"] and v_pool.flags["C_CONTIGUOUS"]
+        kp, vp, st = k_pool.ctypes.data, v_pool.ctypes.data, None
+    else:
+        kp, vp, st = _ptr(k_pool), _ptr(v_pool), _stream_ptr(stream)
+    _check(lib().mepic_store_attach_remote(store, kp, vp, 1 if on_host else 0, int(capacity_pages), st))
+
+
 class Store:
     """Owns one ``mepic_store_t`` handle (context manager; same calls as the C ABI)."""
 
@@ -282,6 +294,10 @@ class Store:
 
     def stats(self):
         return mepic_store_stats(self.handle)
+
+    def attach_remote(self, k_pool, v_pool, capacity_pages, stream=None):
+        self._remote_pools = (k_pool, v_pool)          # the store keeps raw pointers: keep the arrays alive
+        mepic_store_attach_remote(self.handle, k_pool, v_pool, capacity_pages, stream)
 
     def close(self):
         if self.handle:

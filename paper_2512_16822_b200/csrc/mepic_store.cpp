@@ -4,6 +4,8 @@
 // resident chunks (identity = hash of the canonically padded token sequence,
 // Section 3.2.3) and the private pages of every live request.  No device
 // memory is touched here; the K/V bytes live in buffers the caller owns.
+#include <cuda_runtime.h>
+
 #include "mepic.h"
 #include "mepic_internal.h"
 
@@ -11,6 +13,8 @@
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
+#include <cstdint>
+#include <cstdlib>
 #include <cstring>
 #include <deque>
 #include <mutex>
@@ -60,8 +64,98 @@ struct LiveRequest {
   int64_t entries = 0;
 };
 
+static uint64_t fnv1a64(const std::vector<int32_t>& v);
+
+// The tier behind the HBM pool: evicted chunk KV kept in host memory, keyed by content.
+struct RemoteChunk {
+  std::vector<int32_t> padded;
+  std::vector<int64_t> slots;    // one page slot of the tier per shareable block
+  uint64_t last_use = 0;
+};
+
+struct RemoteTier {
+  bool on = false, host_pools = false, failed = false;
+  unsigned char* k_pool = nullptr;
+  unsigned char* v_pool = nullptr;
+  unsigned char* buf = nullptr;            // [capacity][K page | V page]
+  int64_t capacity = 0;
+  size_t page_bytes = 0;
+  std::vector<int64_t> free_slots;
+  std::unordered_map<uint64_t, RemoteChunk> chunks;   // key = hash of the padded tokens, bumped on collision
+  cudaStream_t stream = nullptr;
+  int64_t spilled = 0, fetched = 0;
+  uint64_t tick = 0;
+
+  ~RemoteTier() {
+    if (!buf) return;
+    if (host_pools) std::free(buf); else cudaFreeHost(buf);
+  }
+  // key of `padded` in the tier, or of the free probe position when it is not there
+  uint64_t find(const std::vector<int32_t>& padded, bool* found) const {
+    uint64_t id = fnv1a64(padded);
+    for (;; ++id) {
+      auto it = chunks.find(id);
+      if (it == chunks.end()) { *found = false; return id; }
+      if (it->second.padded == padded) { *found = true; return id; }
+    }
+  }
+  void copy(void* dst, const void* src, bool to_tier) {
+    if (host_pools) { std::memcpy(dst, src, page_bytes); return; }
+    const cudaError_t e = cudaMemcpyAsync(dst, src, page_bytes, to_tier ? cudaMemcpyDeviceToHost : cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) { failed = true; mepic_set_error("remote tier: cudaMemcpyAsync: %s", cudaGetErrorString(e)); }
+  }
+  void drop(uint64_t key) {
+    auto it = chunks.find(key);
+    for (int64_t sl : it->second.slots) free_slots.push_back(sl);
+    // keep probe chains intact: re-insert the entries that follow in the chain
+    std::vector<RemoteChunk> chain;
+    chunks.erase(it);
+    for (uint64_t k = key + 1;; ++k) {
+      auto nx = chunks.find(k);
+      if (nx == chunks.end()) break;
+      chain.push_back(std::move(nx->second));
+      chunks.erase(nx);
+    }
+    for (RemoteChunk& c : chain) { bool f; const uint64_t k = find(c.padded, &f); chunks.emplace(k, std::move(c)); }
+  }
+  // Keep the K/V of an evicted chunk.  The tier gives up its own least recently used chunks for room.
+  void spill(const std::vector<int32_t>& padded, const std::vector<int32_t>& pages) {
+    bool found;
+    uint64_t key = find(padded, &found);
+    if (found) { chunks[key].last_use = ++tick; return; }        // shared pages never change once computed
+    if (static_cast<int64_t>(pages.size()) > capacity) return;
+    while (free_slots.size() < pages.size()) {
+      uint64_t victim = 0, oldest = UINT64_MAX;
+      for (const auto& kv : chunks) if (kv.second.last_use < oldest) { oldest = kv.second.last_use; victim = kv.first; }
+      drop(victim);
+    }
+    key = find(padded, &found);
+    RemoteChunk rc;
+    rc.padded = padded;
+    rc.last_use = ++tick;
+    for (int32_t pg : pages) {
+      const int64_t sl = free_slots.back(); free_slots.pop_back();
+      rc.slots.push_back(sl);
+      copy(buf + static_cast<size_t>(sl) * 2 * page_bytes, k_pool + static_cast<size_t>(pg) * page_bytes, true);
+      copy(buf + static_cast<size_t>(sl) * 2 * page_bytes + page_bytes, v_pool + static_cast<size_t>(pg) * page_bytes, true);
+    }
+    chunks.emplace(key, std::move(rc));
+    spilled += 1;
+  }
+  void fetch(uint64_t key, const std::vector<int32_t>& pages) {
+    RemoteChunk& rc = chunks.at(key);
+    rc.last_use = ++tick;
+    for (size_t i = 0; i < pages.size(); ++i) {
+      copy(k_pool + static_cast<size_t>(pages[i]) * page_bytes, buf + static_cast<size_t>(rc.slots[i]) * 2 * page_bytes, false);
+      copy(v_pool + static_cast<size_t>(pages[i]) * page_bytes, buf + static_cast<size_t>(rc.slots[i]) * 2 * page_bytes + page_bytes, false);
+    }
+    fetched += 1;
+  }
+};
+
 struct mepic_store {
   mepic_config_t cfg;
+  RemoteTier remote;
   std::deque<int32_t> free_pages;
   std::unordered_map<uint64_t, Chunk> chunks;          // id -> chunk; id = hash, bumped on collision
   std::unordered_map<int64_t, LiveRequest> requests;
@@ -95,6 +189,7 @@ struct mepic_store {
     for (const auto& lu : cand) {
       if (need <= free_pages.size()) break;
       auto it = chunks.find(lu.second);
+      if (remote.on && !it->second.uncomputed) remote.spill(it->second.padded, it->second.shared);
       std::vector<int32_t> pages = it->second.shared;
       std::sort(pages.begin(), pages.end());
       for (int32_t pg : pages) free_pages.push_back(pg);
@@ -170,10 +265,18 @@ extern "C" int32_t mepic_chunk_register(mepic_store_t* s, const int32_t* tokens,
     s->touch(c);
     c.shared.reserve(n_shared);
     for (size_t i = 0; i < n_shared; ++i) { c.shared.push_back(s->free_pages.front()); s->free_pages.pop_front(); }
+    if (s->remote.on && n_shared > 0) {
+      // Algorithm 1, residency resolution: not in HBM, but is there a remote copy?  (Looked up after make_room: the
+      // evictions it caused may have made the tier drop this very chunk.)
+      bool found;
+      const uint64_t key = s->remote.find(padded, &found);
+      if (found) { s->remote.fetch(key, c.shared); resident = 2; }
+    }
     c.padded = std::move(padded);
     s->shared_held += static_cast<int64_t>(n_shared);
     shared = &s->chunks.emplace(id, std::move(c)).first->second.shared;
   }
+  if (s->remote.failed) { s->remote.failed = false; return MEPIC_E_CUDA; }
   if (out_chunk_id) *out_chunk_id = id;
   if (out_was_resident) *out_was_resident = resident;
   if (out_lead_pad) *out_lead_pad = lead;
@@ -249,6 +352,7 @@ extern "C" int32_t mepic_build_block_table(mepic_store_t* s, int64_t request_id,
                       (long long)need_private, s->free_pages.size());
       return MEPIC_E_NOSPACE;                                   // Reject; nothing is held, nothing was evicted
     }
+    if (s->remote.failed) { s->remote.failed = false; return MEPIC_E_CUDA; }
   }
   // Pass 2 (block assignment).
   LiveRequest live;
@@ -322,6 +426,38 @@ extern "C" int32_t mepic_store_stats(const mepic_store_t* s, mepic_stats_t* out)
   out->live_requests = static_cast<int64_t>(s->requests.size());
   out->chunks_evicted = s->chunks_evicted;
   out->pages_evicted = s->pages_evicted;
+  out->chunks_spilled = s->remote.spilled;
+  out->chunks_fetched = s->remote.fetched;
+  out->remote_chunks = static_cast<int64_t>(s->remote.chunks.size());
+  out->remote_pages = s->remote.on ? s->remote.capacity - static_cast<int64_t>(s->remote.free_slots.size()) : 0;
+  return MEPIC_OK;
+}
+
+extern "C" int32_t mepic_store_attach_remote(mepic_store_t* s, void* k_pool, void* v_pool, int32_t pools_on_host,
+                                             int64_t capacity_pages, void* cuda_stream) {
+  if (!s || !k_pool || !v_pool || capacity_pages < 1) { mepic_set_error("attach_remote: bad argument"); return MEPIC_E_INVAL; }
+  std::lock_guard<std::mutex> lock(s->mu);
+  RemoteTier& r = s->remote;
+  if (r.on) { mepic_set_error("attach_remote: the store already has a remote tier"); return MEPIC_E_EXISTS; }
+  r.page_bytes = static_cast<size_t>(s->cfg.n_kv_heads) * s->cfg.page_size * s->cfg.head_dim * 2;
+  const size_t bytes = static_cast<size_t>(capacity_pages) * 2 * r.page_bytes;
+  if (pools_on_host) {
+    r.buf = static_cast<unsigned char*>(std::malloc(bytes));
+    if (!r.buf) { mepic_set_error("attach_remote: out of host memory"); return MEPIC_E_INVAL; }
+  } else {
+    void* ptr = nullptr;
+    const cudaError_t e = cudaHostAlloc(&ptr, bytes, cudaHostAllocDefault);
+    if (e != cudaSuccess) { mepic_set_error("attach_remote: cudaHostAlloc(%zu): %s", bytes, cudaGetErrorString(e)); return MEPIC_E_CUDA; }
+    r.buf = static_cast<unsigned char*>(ptr);
+  }
+  r.host_pools = pools_on_host != 0;
+  r.k_pool = static_cast<unsigned char*>(k_pool);
+  r.v_pool = static_cast<unsigned char*>(v_pool);
+  r.capacity = capacity_pages;
+  r.stream = static_cast<cudaStream_t>(cuda_stream);
+  r.free_slots.reserve(static_cast<size_t>(capacity_pages));
+  for (int64_t i = capacity_pages - 1; i >= 0; --i) r.free_slots.push_back(i);    // slot 0 is handed out first
+  r.on = true;
   return MEPIC_OK;
 }
 
