@@ -316,8 +316,11 @@ def decode_attention_one(q_bits: np.ndarray, k_pool: np.ndarray, v_pool: np.ndar
     attention; q head h reads KV head h // (Hq / Hkv).
     """
     P = k_pool.shape[2]
-    K = bf16_bits_to_f64(gather_pages(k_pool, page_ids, kv_len))        # [L, Hkv, D]
-    V = bf16_bits_to_f64(gather_pages(v_pool, page_ids, kv_len))
+    K = gather_pages(k_pool, page_ids, kv_len)                          # [L, Hkv, D]
+    V = gather_pages(v_pool, page_ids, kv_len)
+    # pools are bf16 bit patterns, or already values (float64: de-quantised fp8 pages)
+    K = bf16_bits_to_f64(K) if K.dtype == np.uint16 else K.astype(np.float64)
+    V = bf16_bits_to_f64(V) if V.dtype == np.uint16 else V.astype(np.float64)
     q = bf16_bits_to_f64(q_bits)                                        # [Hq, D]
     if rotate:
         pos = slot_positions(pos_base, kv_len, P)
@@ -386,6 +389,69 @@ def prefill_attention_one(q_new: np.ndarray, k_new: np.ndarray, v_new: np.ndarra
             p = _softmax_rows(s[None, :])[0]
             out[j, h] = p @ V[:slot + 1, kh, :]
     return out
+
+
+# --------------------------------------------------------------------------- fp8 (e4m3) pages
+# The paper's related-work section names KV-cache quantisation as complementary and fixes no format.  This build's
+# reading: OCP 8-bit floating point E4M3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities; the
+# all-ones exponent with all-ones mantissa is NaN; largest finite value 448), one scale per (page, kv head) and pool:
+#     scale = max|x| / 448 (1 if the block is all zero), code = E4M3(x / scale) rounded to nearest, ties to even,
+#     saturating; x~ = value(code) * scale.   All of it in float32, as the device does it.
+E4M3_MAX = 448.0
+
+
+def e4m3_values() -> np.ndarray:
+    """The value of each of the 256 codes, from the format's definition (NaN for 0x7f and 0xff)."""
+    out = np.empty(256, dtype=np.float64)
+    for code in range(256):
+        sign = -1.0 if code & 0x80 else 1.0
+        e, m = (code >> 3) & 0xF, code & 0x7
+        if e == 0xF and m == 0x7:
+            out[code] = np.nan
+        elif e == 0:
+            out[code] = sign * (m / 8.0) * 2.0 ** -6              # subnormal
+        else:
+            out[code] = sign * (1.0 + m / 8.0) * 2.0 ** (e - 7)
+    return out
+
+
+def e4m3_encode(x: np.ndarray) -> np.ndarray:
+    """float32 -> code: round to nearest representable value, ties to the even mantissa, saturate at +-448."""
+    x = np.asarray(x, dtype=np.float32)
+    a = np.abs(x).astype(np.float64)
+    sign = (np.signbit(x)).astype(np.uint8) << 7
+    a = np.minimum(a, E4M3_MAX)
+    # exponent of the binade; values below the smallest normal (2^-6) use the subnormal step 2^-9
+    with np.errstate(divide="ignore"):
+        e = np.floor(np.log2(np.where(a > 0, a, 1.0)))
+    e = np.clip(e, -6, 8)
+    step = 2.0 ** (e - 3)
+    q = np.rint(a / step)                 # numpy rounds halves to even; a/step is exact (a has at most 24 bits)
+    val = q * step                        # may have carried into the next binade: still representable
+    val = np.minimum(val, E4M3_MAX)
+    # value -> code
+    with np.errstate(divide="ignore"):
+        e2 = np.floor(np.log2(np.where(val > 0, val, 1.0)))
+    e2 = np.clip(e2, -6, 8)
+    normal = val >= 2.0 ** -6
+    mant = np.where(normal, val / 2.0 ** e2 - 1.0, val / 2.0 ** -6) * 8.0
+    code = np.where(normal, ((e2 + 7).astype(np.int64) << 3), 0) | np.rint(mant).astype(np.int64)
+    code = code.astype(np.uint8) | sign
+    return np.where(np.isnan(x), np.uint8(0x7F), code).astype(np.uint8)
+
+
+def quantize_pages(pool_bits: np.ndarray):
+    """bf16 pool ``[N, Hkv, P, D]`` -> (codes uint8 same shape, scales float32 ``[N, Hkv]``)."""
+    x = bf16_bits_to_f64(pool_bits).astype(np.float32)                 # bf16 is exact in float32
+    amax = np.abs(x).max(axis=(2, 3))
+    scale = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+    y = (x / scale[:, :, None, None]).astype(np.float32)
+    return e4m3_encode(y), scale
+
+
+def dequantize_pages(codes: np.ndarray, scale: np.ndarray) -> np.ndarray:
+    """-> float64 pool of the values the attention reads: value(code) * scale (the product in float64)."""
+    return e4m3_values()[codes] * scale.astype(np.float64)[:, :, None, None]
 
 
 def merge_partials(m: np.ndarray, l: np.ndarray, o: np.ndarray) -> np.ndarray:

@@ -9,5 +9,6 @@ bool mepic_config_ok(const mepic_config_t* cfg);
 void mepic_count_launches(int n);
 // Fills a 128-byte, 64-byte-aligned CUtensorMap describing a K or V pool (see mepic_tensor_map.cu).
 int32_t mepic_make_pool_map(const mepic_config_t* cfg, const void* pool, void* out_map);
+int32_t mepic_make_pool_map_u8(const mepic_config_t* cfg, const void* pool, void* out_map);
 
 #endif

@@ -51,3 +51,22 @@ int32_t mepic_make_pool_map(const mepic_config_t* cfg, const void* pool, void* o
   if (r != CUDA_SUCCESS) { mepic_set_error("cuTensorMapEncodeTiled failed with code %d", static_cast<int>(r)); return MEPIC_E_CUDA; }
   return MEPIC_OK;
 }
+
+// The same for a pool of 8-bit elements (fp8 pages, head_dim = 128): rows of 128 bytes, one box = a whole
+// 16-token group (16 rows x 128 bytes).
+int32_t mepic_make_pool_map_u8(const mepic_config_t* cfg, const void* pool, void* out_map) {
+  EncodeTiledFn fn = encode_tiled_fn();
+  if (!fn) { mepic_set_error("cuTensorMapEncodeTiled is not available from the driver"); return MEPIC_E_CUDA; }
+  if (cfg->head_dim != 128) { mepic_set_error("8-bit pools need head_dim 128"); return MEPIC_E_INVAL; }
+  const cuuint64_t rows = static_cast<cuuint64_t>(cfg->num_pages) * cfg->n_kv_heads * cfg->page_size;
+  if (rows > 0x7fffffffull) { mepic_set_error("pool has too many rows for 32-bit tensor coordinates"); return MEPIC_E_INVAL; }
+  const cuuint64_t dims[2] = {128, rows};
+  const cuuint64_t strides[1] = {128};
+  const cuuint32_t box[2] = {128, 16};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = fn(static_cast<CUtensorMap*>(out_map), CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(pool), dims, strides,
+                        box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) { mepic_set_error("cuTensorMapEncodeTiled failed with code %d", static_cast<int>(r)); return MEPIC_E_CUDA; }
+  return MEPIC_OK;
+}

@@ -502,3 +502,61 @@ def test_pairing_convention_matters_interleaved_differs_beyond_tolerance():
         other[h] = w @ V[:, h // 4, :]
     d = np.abs(other - good)
     assert d.max() > 2e-2 or d.mean() > 2e-3
+
+
+# --------------------------------------------------------------------------- fp8 (e4m3) pages
+def test_e4m3_codes_roundtrip_and_known_values():
+    v = O.e4m3_values()
+    assert np.isnan(v[0x7F]) and np.isnan(v[0xFF]) and v[0x7E] == 448.0 and v[0xFE] == -448.0
+    assert v[0x38] == 1.0 and v[0x40] == 2.0 and v[0x01] == 2.0 ** -9 and v[0x08] == 2.0 ** -6 and v[0x00] == 0.0
+    finite = [c for c in range(256) if not np.isnan(v[c]) and c != 0x80]            # -0 encodes as 0x80 too; skip it here
+    assert list(O.e4m3_encode(v[finite].astype(np.float32))) == finite
+    # halves go to the even mantissa; out-of-range saturates; half the smallest subnormal goes to zero
+    x = np.array([1.0625, 1.1875, 1000.0, -1000.0, 2.0 ** -10, 3 * 2.0 ** -10, 464.0, 0.0], dtype=np.float32)
+    assert list(O.e4m3_encode(x)) == [0x38, 0x3A, 0x7E, 0xFE, 0x00, 0x02, 0x7E, 0x00]
+
+
+def test_e4m3_encode_is_nearest_value_by_brute_force():
+    v = O.e4m3_values()
+    pos = np.array([c for c in range(128) if not np.isnan(v[c])])
+    rng = np.random.default_rng(5)
+    x = np.concatenate([rng.standard_normal(4000) * s for s in (1e-3, 0.05, 1.0, 30.0, 400.0)]).astype(np.float32)
+    codes = O.e4m3_encode(x)
+    for xi, ci in zip(x, codes):
+        d = np.abs(v[pos] - min(abs(float(xi)), 448.0))
+        best = pos[np.flatnonzero(d == d.min())]
+        want = best[0] if len(best) == 1 else [c for c in best if c % 2 == 0][0]   # a tie: the even mantissa
+        assert (ci & 0x7F) == want and (ci >> 7) == int(np.signbit(xi)), (xi, ci, want)
+
+
+def test_quantize_pages_scale_and_error_bound():
+    rng = np.random.default_rng(6)
+    pool = f32_to_bf16_bits((rng.standard_normal((5, 2, 16, 64)) * rng.uniform(0.01, 20, size=(5, 2, 1, 1))).astype(np.float32))
+    pool[3, 1] = 0                                                                  # an all-zero block
+    codes, scale = O.quantize_pages(pool)
+    x = bf16_bits_to_f64(pool)
+    amax = np.abs(x).max(axis=(2, 3))
+    assert np.array_equal(scale[amax > 0], (amax[amax > 0].astype(np.float32) / np.float32(448.0)))
+    assert scale[3, 1] == 1.0 and not codes[3, 1].any()
+    # every non-zero block uses the top code for its largest element
+    assert all((codes[i, j] & 0x7F).max() == 0x7E for i in range(5) for j in range(2) if amax[i, j] > 0)
+    back = O.dequantize_pages(codes, scale)
+    # half a unit in the last place of a 3-bit mantissa, or half a subnormal step, in units of the block's scale;
+    # plus the float32 rounding of x / scale
+    bound = np.maximum(np.abs(x) * 2.0 ** -4, scale[:, :, None, None] * 2.0 ** -10) * (1 + 1e-6)
+    assert (np.abs(back - x) <= bound).all()
+
+
+def test_decode_over_value_pools_equals_decode_over_bf16_pools():
+    # values that e4m3 represents exactly with scale 1: the fp8 route and the bf16 route must then agree to the last bit
+    rng = np.random.default_rng(8)
+    v = O.e4m3_values()
+    codes_k = rng.integers(0, 0x78, size=(6, 2, 16, 64)).astype(np.uint8) | (rng.integers(0, 2, size=(6, 2, 16, 64)).astype(np.uint8) << 7)
+    codes_v = rng.integers(0, 0x78, size=(6, 2, 16, 64)).astype(np.uint8)
+    ones = np.ones((6, 2), dtype=np.float32)
+    kf, vf = O.dequantize_pages(codes_k, ones), O.dequantize_pages(codes_v, ones)
+    kb, vb = f32_to_bf16_bits(kf.astype(np.float32)), f32_to_bf16_bits(vf.astype(np.float32))
+    assert np.array_equal(bf16_bits_to_f64(kb), kf)                                 # exactly representable in bf16 too
+    q = f32_to_bf16_bits(rng.standard_normal((4, 64)).astype(np.float32))
+    args = ([4, 1, 3, 0, 5], [0, 16, 40, 56, 72], 70, 85, 0.05, 1e4)
+    assert np.array_equal(O.decode_attention_one(q, kf, vf, *args), O.decode_attention_one(q, kb, vb, *args))
