@@ -357,6 +357,32 @@ typedef struct {
 size_t  mepic_attn_decode_grouped_workspace(const mepic_config_t* cfg, const int32_t* plan_host);
 int32_t mepic_attn_decode_grouped(const mepic_config_t* cfg, const mepic_decode_grouped_args_t* args, void* cuda_stream);
 
+/* ---------------------------------------------------------------- fp8 (e4m3) pages (device)
+ *
+ * KV-cache quantisation is named by the paper's related-work section as complementary and no format
+ * is given; this is this build's: a pool of 8-bit pages [num_pages][n_kv_heads][page_size][head_dim]
+ * of OCP E4M3 codes (1-4-3, bias 7, no infinities, largest finite value 448) plus one fp32 scale per
+ * (page, kv head) block [num_pages][n_kv_heads], for K and for V separately.  Keys stay un-rotated.
+ *
+ * mepic_pages_quantize: for every page listed in pages (DEVICE int32[n_pages]) and every kv head,
+ *     scale = max|x| / 448 over the block (1 if the block is all zero),
+ *     code  = E4M3(x / scale), rounded to nearest, ties to even, saturating (NaN -> the NaN code),
+ * computed in fp32 from the bf16 pool src_pool (DEVICE) into dst_pool and scales (DEVICE).  Call it
+ * once for the K pools and once for the V pools.  A page id outside the pool sets MEPIC_DEV_BAD_PAGE
+ * in *status and that block is skipped.  Errors: E_INVAL, E_CUDA.
+ *
+ * mepic_attn_decode_fp8: mepic_attn_decode over such pools: args->k_pool / v_pool are the 8-bit pools,
+ * k_scales / v_scales (DEVICE) their scales; every other field, the workspace size included, is as for
+ * mepic_attn_decode.  What is computed is that call's formula with K_t, V_t replaced by
+ * value(code) * scale; the tolerance against the fp64 oracle evaluated on the same codes and scales
+ * is that call's.  head_dim must be 128.  The queries are carried in fp16 after rotation and scaling
+ * (|q| * sm_scale * log2(e) must stay below 65504).
+ */
+int32_t mepic_pages_quantize(const mepic_config_t* cfg, const void* src_pool, void* dst_pool, float* scales,
+                             const int32_t* pages, int32_t n_pages, int32_t* status, void* cuda_stream);
+int32_t mepic_attn_decode_fp8(const mepic_config_t* cfg, const mepic_decode_args_t* args, const float* k_scales,
+                              const float* v_scales, void* cuda_stream);
+
 /* ---------------------------------------------------------------- prefill (device)
  *
  * mepic_attn_prefill - Sections 3.3.1-3.3.3 for the rows a request recomputes (the first block of

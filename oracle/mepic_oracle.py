@@ -395,7 +395,7 @@ def prefill_attention_one(q_new: np.ndarray, k_new: np.ndarray, v_new: np.ndarra
 # The paper's related-work section names KV-cache quantisation as complementary and fixes no format.  This build's
 # reading: OCP 8-bit floating point E4M3 (1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities; the
 # all-ones exponent with all-ones mantissa is NaN; largest finite value 448), one scale per (page, kv head) and pool:
-#     scale = max|x| / 448 (1 if the block is all zero), code = E4M3(x / scale) rounded to nearest, ties to even,
+#     scale = max|x| / 448 over the block's non-NaN elements (1 if that maximum is zero), code = E4M3(x / scale) rounded to nearest, ties to even,
 #     saturating; x~ = value(code) * scale.   All of it in float32, as the device does it.
 E4M3_MAX = 448.0
 
@@ -418,7 +418,7 @@ def e4m3_values() -> np.ndarray:
 def e4m3_encode(x: np.ndarray) -> np.ndarray:
     """float32 -> code: round to nearest representable value, ties to the even mantissa, saturate at +-448."""
     x = np.asarray(x, dtype=np.float32)
-    a = np.abs(x).astype(np.float64)
+    a = np.where(np.isnan(x), 0.0, np.abs(x)).astype(np.float64)        # NaN gets its code at the end
     sign = (np.signbit(x)).astype(np.uint8) << 7
     a = np.minimum(a, E4M3_MAX)
     # exponent of the binade; values below the smallest normal (2^-6) use the subnormal step 2^-9
@@ -443,7 +443,7 @@ def e4m3_encode(x: np.ndarray) -> np.ndarray:
 def quantize_pages(pool_bits: np.ndarray):
     """bf16 pool ``[N, Hkv, P, D]`` -> (codes uint8 same shape, scales float32 ``[N, Hkv]``)."""
     x = bf16_bits_to_f64(pool_bits).astype(np.float32)                 # bf16 is exact in float32
-    amax = np.abs(x).max(axis=(2, 3))
+    amax = np.where(np.isnan(x), np.float32(0), np.abs(x)).max(axis=(2, 3))       # NaN elements do not set the scale
     scale = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
     y = (x / scale[:, :, None, None]).astype(np.float32)
     return e4m3_encode(y), scale

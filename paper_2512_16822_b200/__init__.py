@@ -24,7 +24,7 @@ __all__ = [
     "mepic_store_create", "mepic_store_destroy", "mepic_chunk_register", "mepic_build_block_table",
     "mepic_request_release", "mepic_chunk_mark_uncomputed", "mepic_store_stats", "mepic_store_attach_remote", "mepic_rope_table_floats", "mepic_rope_table_fill",
     "mepic_attn_decode_workspace", "mepic_attn_decode", "mepic_attn_decode_static",
-    "mepic_decode_plan_max_ints", "mepic_decode_plan_build", "mepic_attn_decode_grouped_workspace",
+    "mepic_pages_quantize", "mepic_attn_decode_fp8", "mepic_decode_plan_max_ints", "mepic_decode_plan_build", "mepic_attn_decode_grouped_workspace",
     "mepic_attn_decode_grouped",
     "MEPIC_DECODE_STATIC_SCRATCH_BYTES", "mepic_attn_prefill_workspace",
     "mepic_attn_prefill", "mepic_last_error", "mepic_launch_count",
@@ -140,6 +140,9 @@ _PROTOTYPES = {
     "mepic_attn_decode_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32]),
     "mepic_attn_decode": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeArgsC), C.c_void_p]),
     "mepic_attn_decode_static": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeArgsC), C.c_void_p]),
+    "mepic_pages_quantize": (C.c_int32, [C.POINTER(_ConfigC), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                         C.c_void_p, C.c_void_p]),
+    "mepic_attn_decode_fp8": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeArgsC), C.c_void_p, C.c_void_p, C.c_void_p]),
     "mepic_decode_plan_max_ints": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32, C.c_int32, C.c_int32]),
     "mepic_decode_plan_build": (C.c_int32, [C.POINTER(_ConfigC), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                             C.c_int32, C.c_int32, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]),
@@ -365,6 +368,23 @@ def mepic_attn_decode_static(cfg: Config, *, q, k_pool, v_pool, page_ids, pos_ba
                      _ptr(q_pos), _ptr(rope_table), _ptr(out), None, 0, _ptr(status), table_stride, batch, sm_scale)
     c = cfg.c()
     _check(lib().mepic_attn_decode_static(C.byref(c), C.byref(a), _stream_ptr(stream)))
+
+
+def mepic_pages_quantize(cfg: Config, *, src_pool, dst_pool, scales, pages, n_pages: int, status, stream=None) -> None:
+    """bf16 pool -> e4m3 codes + one scale per (page, kv head) for the listed pages (all device tensors)."""
+    c = cfg.c()
+    _check(lib().mepic_pages_quantize(C.byref(c), _ptr(src_pool), _ptr(dst_pool), _ptr(scales), _ptr(pages), n_pages,
+                                      _ptr(status), _stream_ptr(stream)))
+
+
+def mepic_attn_decode_fp8(cfg: Config, *, q, k_pool, v_pool, k_scales, v_scales, page_ids, pos_base, kv_len, q_pos,
+                          rope_table, out, workspace, workspace_bytes: int, status, table_stride: int, batch: int,
+                          sm_scale: float, stream=None) -> None:
+    a = _DecodeArgsC(_ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(page_ids), _ptr(pos_base), _ptr(kv_len),
+                     _ptr(q_pos), _ptr(rope_table), _ptr(out), _ptr(workspace), workspace_bytes, _ptr(status),
+                     table_stride, batch, sm_scale)
+    c = cfg.c()
+    _check(lib().mepic_attn_decode_fp8(C.byref(c), C.byref(a), _ptr(k_scales), _ptr(v_scales), _stream_ptr(stream)))
 
 
 def mepic_decode_plan_max_ints(cfg: Config, batch: int, table_stride: int, n_sms: int = 0) -> int:

@@ -17,7 +17,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB_PATH = os.path.join(HERE, "libmepic.so")
 
-SOURCES = ["mepic_store.cpp", "mepic_tensor_map.cu", "mepic_decode.cu", "mepic_decode_grouped.cu", "mepic_plan.cpp",
+SOURCES = ["mepic_store.cpp", "mepic_tensor_map.cu", "mepic_decode.cu", "mepic_decode_fp8.cu", "mepic_decode_grouped.cu", "mepic_plan.cpp",
            "mepic_prefill.cu"]
 
 

@@ -1,6 +1,6 @@
 """Run one benchmark configuration through the public binding and print the device time.
 
-    python -m paper_2512_16822_b200.cases decode  --config 2 [--scale 1.0] [--iters 10] [--unshared] [--grouped]
+    python -m paper_2512_16822_b200.cases decode  --config 2 [--scale 1.0] [--iters 10] [--unshared] [--grouped] [--fp8]
     python -m paper_2512_16822_b200.cases prefill --config 3 [--scale 0.5] [--iters 4]
 
 A small driver for profiling (a fixed, short sequence of calls that a profiler can capture) and for trying the
@@ -44,7 +44,7 @@ def _setup_unshared_decode(index: int, scale: float):
     return wl, dev, RT.DecodeBatch(dev, page_ids, pos_base, kv_len, kv_len - 1, wl.decode_q())
 
 
-def _setup(index: int, scale: float, which: str, grouped: bool = False):
+def _setup(index: int, scale: float, which: str, grouped: bool = False, fp8: bool = False):
     import paper_2512_16822_b200 as M
     from paper_2512_16822_b200 import runtime as RT
     from mepic_inputs import make_workload
@@ -60,6 +60,8 @@ def _setup(index: int, scale: float, which: str, grouped: bool = False):
         if not dec:
             raise SystemExit(f"config {index} has no decode requests")
         page_ids, pos_base, kv_len, q_pos = RT.pack_tables(dec, wl.page_size)
+        if fp8:
+            return wl, dev, RT.Fp8DecodeBatch(RT.Fp8Pools(dev), page_ids, pos_base, kv_len, q_pos, wl.decode_q())
         kind = RT.GroupedDecodeBatch if grouped else RT.DecodeBatch
         return wl, dev, kind(dev, page_ids, pos_base, kv_len, q_pos, wl.decode_q())
     if not pre:
@@ -83,12 +85,13 @@ def main() -> None:
     ap.add_argument("--iters", type=int, default=4)
     ap.add_argument("--unshared", action="store_true", help="decode only: no chunk sharing, one page per table entry")
     ap.add_argument("--grouped", action="store_true", help="decode only: the sharing-aware path (host plan + grouped kernel)")
+    ap.add_argument("--fp8", action="store_true", help="decode only: 8-bit (e4m3) pages made from the bf16 pool by the library's quantiser")
     args = ap.parse_args()
     index = args.config if args.config is not None else (2 if args.which == "decode" else 3)
     if args.unshared and args.which == "decode":
         wl, dev, batch = _setup_unshared_decode(index, args.scale)
     else:
-        wl, dev, batch = _setup(index, args.scale, args.which, args.grouped)
+        wl, dev, batch = _setup(index, args.scale, args.which, args.grouped, args.fp8)
     for _ in range(max(args.iters - 1, 1)):
         batch.run(wl.sm_scale)
     torch.cuda.synchronize()

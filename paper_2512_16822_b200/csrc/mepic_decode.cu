@@ -31,126 +31,11 @@
 #include "mepic.h"
 #include "mepic_internal.h"
 
+#include "mepic_decode_line.cuh"
+
 namespace {
 
-constexpr int kTile = 16;      // tokens per staged tile
-constexpr int kWarps = 8;      // workers per CTA
-constexpr int kMinPiece = 4;   // never cut the line into pieces shorter than this many tiles
-constexpr unsigned kFull = 0xffffffffu;
-constexpr int kSpinLimit = 1 << 22;
-
-struct DecodeParams {
-  const uint16_t* q;
-  const uint16_t* k_pool;
-  const uint16_t* v_pool;
-  const int32_t* page_ids;
-  const int32_t* pos_base;
-  const int32_t* kv_len;
-  const int32_t* q_pos;
-  const float* rope;
-  float* part_o;    // [slots][G][D]
-  float* part_ml;   // [slots][G][2] = (max in log2 units, sum)
-  uint16_t* out;
-  int32_t* status;
-  int table_stride, batch, n_kv_heads, page_size, log2_tpp, num_pages, max_position, n_workers;
-  float scale_log2;   // sm_scale * log2(e)
-};
-
-// ---------------------------------------------------------------- small PTX helpers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-// two bf16 packed in a 32-bit word (low half = even element) -> two floats, exactly
-__device__ __forceinline__ float2 bf16x2_to_float2(uint32_t w) {
-  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-}
-__device__ __forceinline__ float ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{ .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p; }"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait: gives up after kSpinLimit polls instead of hanging the SM.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (int i = 0; i < kSpinLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ int warp_sum(int v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
-  return v;
-}
-__device__ __forceinline__ int tiles_of(int kv_len) { return kv_len > 0 ? (kv_len + kTile - 1) / kTile : 0; }
-
-// The cut of the tile line, recomputed by every warp from kv_len (no host mirror, no plan upload).
-struct Cut { long long total; long long piece; };
-__device__ __forceinline__ Cut cut_of_line(const int32_t* kv_len, int batch, int n_kv_heads, int n_workers, int lane) {
-  long long tiles = 0;
-  for (int b0 = 0; b0 < batch; b0 += 32) {
-    const int n = (b0 + lane < batch) ? tiles_of(kv_len[b0 + lane]) : 0;
-    tiles += warp_sum(n);
-  }
-  Cut c;
-  c.total = tiles * n_kv_heads;
-  long long piece = (c.total + n_workers - 1) / n_workers;
-  c.piece = piece < kMinPiece ? kMinPiece : piece;
-  return c;
-}
-
-// Position on the line: request b, kv head h, tile t of the request's nt tiles.
-struct Cursor { int b, h, t, nt, kvl; };
-
-__device__ __forceinline__ Cursor locate(const int32_t* kv_len, int batch, int n_kv_heads, long long x, int lane) {
-  Cursor c{batch, 0, 0, 0, 0};
-  long long before = 0;   // tiles of the requests before the 32 under inspection
-  for (int b0 = 0; b0 < batch; b0 += 32) {
-    const int kvl = (b0 + lane < batch) ? kv_len[b0 + lane] : 0;
-    const int n = tiles_of(kvl);
-    int incl = n;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(kFull, incl, o); if (lane >= o) incl += y; }
-    const bool past = (before + incl) * n_kv_heads > x;
-    const unsigned m = __ballot_sync(kFull, past);
-    if (m) {
-      const int l = __ffs(m) - 1;
-      const long long pre = before + __shfl_sync(kFull, incl - n, l);
-      c.b = b0 + l;
-      c.nt = __shfl_sync(kFull, n, l);
-      c.kvl = __shfl_sync(kFull, kvl, l);
-      const long long r = x - pre * n_kv_heads;
-      c.h = static_cast<int>(r / c.nt);
-      c.t = static_cast<int>(r % c.nt);
-      return c;
-    }
-    before += __shfl_sync(kFull, incl, 31);
-  }
-  return c;
-}
-
-__device__ __forceinline__ void advance(Cursor& c, const int32_t* kv_len, int batch, int n_kv_heads) {
-  if (++c.t < c.nt) return;
-  c.t = 0;
-  if (++c.h < n_kv_heads) return;
-  c.h = 0;
-  do {
-    ++c.b;
-    c.kvl = (c.b < batch) ? kv_len[c.b] : 0;
-    c.nt = tiles_of(c.kvl);
-  } while (c.b < batch && c.nt == 0);
-}
+using namespace mepic_dev;
 
 // ---------------------------------------------------------------- the split-KV kernel
 // Warp-level tensor-core MMA (mma.sync m16n8k16, bf16 in, fp32 accumulate) for the two contractions of a tile:
@@ -158,39 +43,6 @@ __device__ __forceinline__ void advance(Cursor& c, const int32_t* kv_len, int ba
 //   O  [head][dim] += P[head][key]      . V[key][dim]         A = P straight from the S accumulators, B = V
 // so that only the rotation of K (thread-local on the B fragments: the partner dim i + D/2 sits in the fragment
 // of k-step j + D/32, same lane, same position) and the softmax stay on the CUDA cores.
-__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
-}
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr) {
-  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
-}
-__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-               : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3]) : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-// (lo, hi) -> packed bf16x2, round to nearest even
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
-__device__ __forceinline__ uint32_t bf16x2_mul(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
-__device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t d;
-  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-
 template <int D, int G>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
@@ -445,47 +297,6 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   flush();
 }
 
-// ---------------------------------------------------------------- merge of the partials of each unit
-// One CTA per (request, kv head); thread (g, d) combines the unit's partials:
-// m* = max m, l* = sum l 2^(m - m*), out = sum o 2^(m - m*) / l*  -> bf16.
-template <int D, int G>
-__global__ void mepic_decode_merge(const DecodeParams p) {
-  const int b = blockIdx.x / p.n_kv_heads, h = blockIdx.x % p.n_kv_heads;
-  const int lane = threadIdx.x & 31;
-  __shared__ long long sh[3];
-  if (threadIdx.x < 32) {
-    const Cut cut = cut_of_line(p.kv_len, p.batch, p.n_kv_heads, p.n_workers, lane);
-    long long before = 0;
-    for (int b0 = 0; b0 < b; b0 += 32) {
-      const int n = (b0 + lane < b) ? tiles_of(p.kv_len[b0 + lane]) : 0;
-      before += warp_sum(n);
-    }
-    if (lane == 0) { sh[0] = cut.piece; sh[1] = before; sh[2] = tiles_of(p.kv_len[b]); }
-  }
-  __syncthreads();
-  const long long piece = sh[0], nt = sh[2];
-  const int g = threadIdx.x / D, d = threadIdx.x % D;
-  const size_t o_at = (static_cast<size_t>(b) * p.n_kv_heads * G + static_cast<size_t>(h) * G + g) * D + d;
-  if (nt == 0) { p.out[o_at] = 0; return; }
-  const long long u0 = sh[1] * p.n_kv_heads + static_cast<long long>(h) * nt;
-  const long long w_first = u0 / piece, w_last = (u0 + nt - 1) / piece;
-  const long long unit = static_cast<long long>(b) * p.n_kv_heads + h;
-  float m_star = -INFINITY;
-  for (long long wk = w_first; wk <= w_last; ++wk) m_star = fmaxf(m_star, p.part_ml[((unit + wk) * G + g) * 2]);
-  float l_star = 0.f, o_star = 0.f;
-  for (long long wk = w_first; wk <= w_last; ++wk) {
-    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + ((unit + wk) * G + g) * 2);
-    const float wgt = ex2(ml.x - m_star);
-    l_star += ml.y * wgt;
-    o_star += p.part_o[((unit + wk) * G + g) * D + d] * wgt;
-  }
-  const float r = o_star / l_star;
-  // fp32 -> bf16, round to nearest even
-  uint32_t u = __float_as_uint(r);
-  u += 0x7fffu + ((u >> 16) & 1u);
-  p.out[o_at] = (r != r) ? 0x7fc0 : static_cast<uint16_t>(u >> 16);
-}
-
 template <int D, int G>
 constexpr size_t decode_smem_bytes() {
   // per warp: 3 stages of (K blocks + V blocks), 3 table rows, 64 bytes of barriers and flags; 1 KB alignment slack
@@ -549,6 +360,7 @@ extern "C" int32_t mepic_attn_decode(const mepic_config_t* cfg, const mepic_deco
   p.v_pool = static_cast<const uint16_t*>(a->v_pool);
   p.page_ids = a->page_ids; p.pos_base = a->pos_base; p.kv_len = a->kv_len; p.q_pos = a->q_pos;
   p.rope = a->rope_table;
+  p.k_scales = nullptr; p.v_scales = nullptr;
   p.part_o = static_cast<float*>(a->workspace);
   p.part_ml = p.part_o + slots * G * D;
   p.out = static_cast<uint16_t*>(a->out);

@@ -1,0 +1,141 @@
+// The tile line of the per-request decode kernels and what they share: launch parameters, the cut of the line
+// into equal pieces, the cursor that walks it, and the kernel that merges the partials of each unit.
+#ifndef MEPIC_DECODE_LINE_CUH_
+#define MEPIC_DECODE_LINE_CUH_
+
+#include "mepic.h"
+#include "mepic_decode_common.cuh"
+
+namespace mepic_dev {
+
+constexpr int kTile = 16;      // tokens per staged tile
+constexpr int kWarps = 8;      // workers per CTA
+constexpr int kMinPiece = 4;   // never cut the line into pieces shorter than this many tiles
+
+struct DecodeParams {
+  const uint16_t* q;
+  const uint16_t* k_pool;
+  const uint16_t* v_pool;
+  const int32_t* page_ids;
+  const int32_t* pos_base;
+  const int32_t* kv_len;
+  const int32_t* q_pos;
+  const float* rope;
+  const float* k_scales;   // fp8 pools only: [num_pages][n_kv_heads] scale of each (page, kv head) block of K
+  const float* v_scales;   // ... and of V
+  float* part_o;    // [slots][G][D]
+  float* part_ml;   // [slots][G][2] = (max in log2 units, sum)
+  uint16_t* out;
+  int32_t* status;
+  int table_stride, batch, n_kv_heads, page_size, log2_tpp, num_pages, max_position, n_workers;
+  float scale_log2;   // sm_scale * log2(e)
+};
+
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(kFull, v, o);
+  return v;
+}
+__device__ __forceinline__ int tiles_of(int kv_len) { return kv_len > 0 ? (kv_len + kTile - 1) / kTile : 0; }
+
+// The cut of the tile line, recomputed by every warp from kv_len (no host mirror, no plan upload).
+struct Cut { long long total; long long piece; };
+__device__ __forceinline__ Cut cut_of_line(const int32_t* kv_len, int batch, int n_kv_heads, int n_workers, int lane) {
+  long long tiles = 0;
+  for (int b0 = 0; b0 < batch; b0 += 32) {
+    const int n = (b0 + lane < batch) ? tiles_of(kv_len[b0 + lane]) : 0;
+    tiles += warp_sum(n);
+  }
+  Cut c;
+  c.total = tiles * n_kv_heads;
+  long long piece = (c.total + n_workers - 1) / n_workers;
+  c.piece = piece < kMinPiece ? kMinPiece : piece;
+  return c;
+}
+
+// Position on the line: request b, kv head h, tile t of the request's nt tiles.
+struct Cursor { int b, h, t, nt, kvl; };
+
+__device__ __forceinline__ Cursor locate(const int32_t* kv_len, int batch, int n_kv_heads, long long x, int lane) {
+  Cursor c{batch, 0, 0, 0, 0};
+  long long before = 0;   // tiles of the requests before the 32 under inspection
+  for (int b0 = 0; b0 < batch; b0 += 32) {
+    const int kvl = (b0 + lane < batch) ? kv_len[b0 + lane] : 0;
+    const int n = tiles_of(kvl);
+    int incl = n;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) { const int y = __shfl_up_sync(kFull, incl, o); if (lane >= o) incl += y; }
+    const bool past = (before + incl) * n_kv_heads > x;
+    const unsigned m = __ballot_sync(kFull, past);
+    if (m) {
+      const int l = __ffs(m) - 1;
+      const long long pre = before + __shfl_sync(kFull, incl - n, l);
+      c.b = b0 + l;
+      c.nt = __shfl_sync(kFull, n, l);
+      c.kvl = __shfl_sync(kFull, kvl, l);
+      const long long r = x - pre * n_kv_heads;
+      c.h = static_cast<int>(r / c.nt);
+      c.t = static_cast<int>(r % c.nt);
+      return c;
+    }
+    before += __shfl_sync(kFull, incl, 31);
+  }
+  return c;
+}
+
+__device__ __forceinline__ void advance(Cursor& c, const int32_t* kv_len, int batch, int n_kv_heads) {
+  if (++c.t < c.nt) return;
+  c.t = 0;
+  if (++c.h < n_kv_heads) return;
+  c.h = 0;
+  do {
+    ++c.b;
+    c.kvl = (c.b < batch) ? kv_len[c.b] : 0;
+    c.nt = tiles_of(c.kvl);
+  } while (c.b < batch && c.nt == 0);
+}
+
+// ---------------------------------------------------------------- merge of the partials of each unit
+// One CTA per (request, kv head); thread (g, d) combines the unit's partials:
+// m* = max m, l* = sum l 2^(m - m*), out = sum o 2^(m - m*) / l*  -> bf16.
+template <int D, int G>
+__global__ void mepic_decode_merge(const DecodeParams p) {
+  const int b = blockIdx.x / p.n_kv_heads, h = blockIdx.x % p.n_kv_heads;
+  const int lane = threadIdx.x & 31;
+  __shared__ long long sh[3];
+  if (threadIdx.x < 32) {
+    const Cut cut = cut_of_line(p.kv_len, p.batch, p.n_kv_heads, p.n_workers, lane);
+    long long before = 0;
+    for (int b0 = 0; b0 < b; b0 += 32) {
+      const int n = (b0 + lane < b) ? tiles_of(p.kv_len[b0 + lane]) : 0;
+      before += warp_sum(n);
+    }
+    if (lane == 0) { sh[0] = cut.piece; sh[1] = before; sh[2] = tiles_of(p.kv_len[b]); }
+  }
+  __syncthreads();
+  const long long piece = sh[0], nt = sh[2];
+  const int g = threadIdx.x / D, d = threadIdx.x % D;
+  const size_t o_at = (static_cast<size_t>(b) * p.n_kv_heads * G + static_cast<size_t>(h) * G + g) * D + d;
+  if (nt == 0) { p.out[o_at] = 0; return; }
+  const long long u0 = sh[1] * p.n_kv_heads + static_cast<long long>(h) * nt;
+  const long long w_first = u0 / piece, w_last = (u0 + nt - 1) / piece;
+  const long long unit = static_cast<long long>(b) * p.n_kv_heads + h;
+  float m_star = -INFINITY;
+  for (long long wk = w_first; wk <= w_last; ++wk) m_star = fmaxf(m_star, p.part_ml[((unit + wk) * G + g) * 2]);
+  float l_star = 0.f, o_star = 0.f;
+  for (long long wk = w_first; wk <= w_last; ++wk) {
+    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + ((unit + wk) * G + g) * 2);
+    const float wgt = ex2(ml.x - m_star);
+    l_star += ml.y * wgt;
+    o_star += p.part_o[((unit + wk) * G + g) * D + d] * wgt;
+  }
+  const float r = o_star / l_star;
+  // fp32 -> bf16, round to nearest even
+  uint32_t u = __float_as_uint(r);
+  u += 0x7fffu + ((u >> 16) & 1u);
+  p.out[o_at] = (r != r) ? 0x7fc0 : static_cast<uint16_t>(u >> 16);
+}
+
+}  // namespace mepic_dev
+
+#endif

@@ -13,6 +13,7 @@ import torch
 
 from . import (Config, Segment, Store, MEPIC_SEG_CHUNK, MEPIC_SEG_PROMPT, mepic_attn_decode,
                mepic_decode_plan_build, mepic_attn_decode_grouped, mepic_attn_decode_grouped_workspace,
+               mepic_pages_quantize, mepic_attn_decode_fp8,
                mepic_attn_decode_workspace, mepic_attn_prefill, mepic_attn_prefill_workspace,
                mepic_rope_table_fill)
 
@@ -154,6 +155,46 @@ class DecodeBatch:
     def upload(self, host: torch.Tensor) -> None:
         """One asynchronous host-to-device copy of a whole step's inputs (on the current stream)."""
         self.step_inputs.copy_(host, non_blocking=True)
+
+
+class Fp8Pools:
+    """8-bit (e4m3) copies of a device's K/V pools with one scale per (page, kv head), made by the library's quantiser."""
+
+    def __init__(self, dev: Device, pages: Optional[np.ndarray] = None):
+        cfg = dev.cfg
+        self.dev = dev
+        d = dev.device
+        shape = (cfg.num_pages, cfg.n_kv_heads, cfg.page_size, cfg.head_dim)
+        self.k_codes = torch.zeros(shape, dtype=torch.uint8, device=d)
+        self.v_codes = torch.zeros(shape, dtype=torch.uint8, device=d)
+        self.k_scales = torch.ones((cfg.num_pages, cfg.n_kv_heads), dtype=torch.float32, device=d)
+        self.v_scales = torch.ones((cfg.num_pages, cfg.n_kv_heads), dtype=torch.float32, device=d)
+        self.quantize(np.arange(cfg.num_pages, dtype=np.int32) if pages is None else pages)
+
+    def quantize(self, pages: np.ndarray, stream=None) -> None:
+        lst = torch.from_numpy(np.ascontiguousarray(pages, dtype=np.int32)).to(self.dev.device)
+        s = stream if stream is not None else torch.cuda.current_stream(self.dev.device)
+        for src, dst, sc in ((self.dev.k_pool, self.k_codes, self.k_scales), (self.dev.v_pool, self.v_codes, self.v_scales)):
+            mepic_pages_quantize(self.dev.cfg, src_pool=src, dst_pool=dst, scales=sc, pages=lst, n_pages=int(lst.numel()),
+                                 status=self.dev.status, stream=s)
+
+
+class Fp8DecodeBatch(DecodeBatch):
+    """A decode batch that reads the 8-bit pools."""
+
+    def __init__(self, pools: Fp8Pools, page_ids, pos_base, kv_len, q_pos, q_bits=None):
+        super().__init__(pools.dev, page_ids, pos_base, kv_len, q_pos, q_bits)
+        self.pools = pools
+
+    def run(self, sm_scale: float, stream=None) -> torch.Tensor:
+        s = stream if stream is not None else torch.cuda.current_stream(self.dev.device)
+        mepic_attn_decode_fp8(self.dev.cfg, q=self.q, k_pool=self.pools.k_codes, v_pool=self.pools.v_codes,
+                              k_scales=self.pools.k_scales, v_scales=self.pools.v_scales, page_ids=self.page_ids,
+                              pos_base=self.pos_base, kv_len=self.kv_len, q_pos=self.q_pos, rope_table=self.dev.rope,
+                              out=self.out, workspace=self.workspace, workspace_bytes=self.ws_bytes,
+                              status=self.dev.status, table_stride=self.stride, batch=self.batch, sm_scale=sm_scale,
+                              stream=s)
+        return self.out
 
 
 class GroupedDecodeBatch:
