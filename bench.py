@@ -242,6 +242,32 @@ def measure_grouped(args, wl, dev, page_ids, pos_base, kv_len, q_pos, q_bits, lo
                     "decode / time; L2 flushed between steps"}
 
 
+def measure_fp8(args, wl, dev, page_ids, pos_base, kv_len, q_pos, q_bits):
+    """The same decode batch over 8-bit (e4m3) copies of the pools (library quantiser, one scale per page and head)."""
+    import torch
+    from paper_2512_16822_b200 import runtime as RT
+    pools = RT.Fp8Pools(dev)
+    batch = RT.Fp8DecodeBatch(pools, page_ids, pos_base, kv_len, q_pos, q_bits)
+    stream = torch.cuda.current_stream()
+    flush = L2Flush(dev.device)
+    for _ in range(3):
+        batch.run(wl.sm_scale, stream)
+    steps = max(5, min(args.steps, 50))
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in evs:
+        flush()
+        a.record(stream); batch.run(wl.sm_scale, stream); b.record(stream)
+    torch.cuda.synchronize()
+    assert dev.read_status() == 0
+    ms = sum(a.elapsed_time(b) for a, b in evs) / steps
+    tokens = int(kv_len.astype(np.int64).sum())
+    bytes_per_token = kv_bytes_per_token(wl) // 2
+    return {"ms_per_step": ms, "steps": steps, "context_tokens_per_s": tokens / (ms * 1e-3),
+            "kv_bytes_per_token": bytes_per_token, "value": tokens * bytes_per_token / (ms * 1e-3) / 1e9, "unit": "GB/s",
+            "note": "e4m3 pages + fp32 scale per (page, kv head): half the K/V bytes of bf16 per context token; "
+                    "value = 8-bit bytes / time; L2 flushed between steps"}
+
+
 def measure_unshared(args, wl, device_index: int):
     """The same decode batch on a layout WITHOUT chunk sharing: every request owns a private copy of each of its
     chunks (one page per block-table entry), so no page is read twice and nothing can be served from L2 because a
@@ -437,7 +463,9 @@ def run_ours(args):
         return max_over_ranks(sum(xs), world, dev.device)
 
     tot, tot_warm, tot_e2e = agg(ms), agg(ms_warm), agg(ms_e2e)
-    prefill = unshared = grouped = None
+    prefill = unshared = grouped = fp8 = None
+    if rank == 0 and world == 1 and not args.no_fp8 and wl.head_dim == 128:
+        fp8 = measure_fp8(args, wl, dev, page_ids, pos_base, kv_len, q_pos, q_bits)
     if rank == 0 and world == 1 and not args.no_grouped:
         grouped = measure_grouped(args, wl, dev, page_ids, pos_base, kv_len, q_pos, q_bits, logical_bytes)
     if rank == 0 and world == 1 and not args.no_prefill:
@@ -479,6 +507,7 @@ def run_ours(args):
         "prefill": prefill,
         "unshared_layout": unshared,
         "grouped_decode": grouped,
+        "fp8_decode": fp8,
     }
     if not args.no_cpu_baseline and world == 1:
         s = oracle_decode_sample(wl, args.cpu_budget)
@@ -505,6 +534,7 @@ def main():
     ap.add_argument("--no-prefill", action="store_true", help="skip the config-3 prefill measurement")
     ap.add_argument("--no-unshared", action="store_true", help="skip the decode run on the layout without sharing")
     ap.add_argument("--no-grouped", action="store_true", help="skip the sharing-aware (grouped) decode run")
+    ap.add_argument("--no-fp8", action="store_true", help="skip the decode run over 8-bit pages")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
