@@ -39,8 +39,8 @@ from mepic_inputs import make_workload  # noqa: E402
 
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one mepic_decode_splitkv launch (ncu, see profiles/);
-# config 2: 358.9 MB read + 4.1 MB written (profiles/decode_splitkv_config2.md).
-NCU_TRAFFIC_BYTES = {2: 362_957_000}
+# config 2: 356.9 MB read + 3.9 MB written (profiles/decode_splitkv_config2.md).
+NCU_TRAFFIC_BYTES = {2: 360_870_000}
 
 
 def kv_bytes_per_token(wl) -> int:
@@ -199,7 +199,7 @@ class L2Flush:
     def __init__(self, device):
         import torch
         self.w = torch.empty(512 << 20, dtype=torch.uint8, device=device)
-        self.r = torch.zeros(128 << 20, dtype=torch.int32, device=device)
+        self.r = torch.zeros(64 << 20, dtype=torch.int64, device=device)       # 512 MiB, summed without a widening copy
         self.acc = torch.zeros((), dtype=torch.int64, device=device)
 
     def __call__(self):

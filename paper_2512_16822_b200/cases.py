@@ -98,7 +98,7 @@ def main() -> None:
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev.device)
     times = []
     for _ in range(5):
-        flush.fill_(1); flush.view(torch.int32).sum()                 # L2 flushed, dirty lines pushed out
+        flush.fill_(1); flush.view(torch.int64).sum()                 # L2 flushed, dirty lines pushed out
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(); batch.run(wl.sm_scale); e1.record()
         torch.cuda.synchronize()
