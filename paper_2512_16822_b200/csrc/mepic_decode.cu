@@ -70,6 +70,7 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   const int g = lane >> 2;       // fragment row group: head g (A, C) / key g (B)
   const int t = lane & 3;        // fragment column group
 
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the merge kernel may move in as CTAs of this one retire
   const long long w = static_cast<long long>(blockIdx.x) * kWarps + wic;
   const Cut cut = cut_of_line(p.kv_len, p.batch, p.n_kv_heads, p.n_workers, lane);
   const long long x0 = w * cut.piece;
@@ -309,8 +310,8 @@ int32_t launch_decode(const DecodeParams& p, int n_ctas, const CUtensorMap& map_
   cudaError_t e = cudaFuncSetAttribute(mepic_decode_splitkv<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("decode: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   mepic_decode_splitkv<D, G><<<n_ctas, kWarps * 32, smem, stream>>>(p, map_k, map_v);
-  mepic_decode_merge<D, G><<<p.batch * p.n_kv_heads, G * D, 0, stream>>>(p);
-  e = cudaGetLastError();
+  e = launch_dependent(mepic_decode_merge<D, G>, dim3(p.batch * p.n_kv_heads), dim3(G * D), stream, p);
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("decode: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   mepic_count_launches(2);
   return MEPIC_OK;

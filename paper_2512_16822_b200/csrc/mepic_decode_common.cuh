@@ -82,6 +82,19 @@ __device__ __forceinline__ uint16_t f32_to_bf16_bits(float r) {
   return (r != r) ? 0x7fc0 : static_cast<uint16_t>(u >> 16);
 }
 
+// Launches `kernel` so that it may become resident while the previous kernel on the stream is still running
+// (programmatic dependent launch); the kernel itself waits with griddepcontrol.wait before touching that kernel's output.
+template <typename Kernel, typename... Args>
+cudaError_t launch_dependent(Kernel kernel, dim3 grid, dim3 block, cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
 }  // namespace mepic_dev
 
 #endif

@@ -123,6 +123,7 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
   // keys behind row g of the two key n-tiles
   const int key0 = 4 * (g >> 1) + (g & 1), key1 = key0 + 2;
 
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const long long w = static_cast<long long>(blockIdx.x) * kWarps + wic;
   const Cut cut = cut_of_line(p.kv_len, p.batch, p.n_kv_heads, p.n_workers, lane);
   const long long x0 = w * cut.piece;
@@ -369,8 +370,8 @@ int32_t launch_fp8(const DecodeParams& p, int n_ctas, const CUtensorMap& map_k, 
   cudaError_t e = cudaFuncSetAttribute(mepic_decode_splitkv_fp8<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("decode_fp8: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   mepic_decode_splitkv_fp8<G><<<n_ctas, kWarps * 32, smem, stream>>>(p, map_k, map_v);
-  mepic_decode_merge<128, G><<<p.batch * p.n_kv_heads, G * 128, 0, stream>>>(p);
-  e = cudaGetLastError();
+  e = launch_dependent(mepic_decode_merge<128, G>, dim3(p.batch * p.n_kv_heads), dim3(G * 128), stream, p);
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("decode_fp8: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   mepic_count_launches(2);
   return MEPIC_OK;

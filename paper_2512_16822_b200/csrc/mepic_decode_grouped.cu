@@ -76,6 +76,7 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
   uint64_t* bars = reinterpret_cast<uint64_t*>(misc);                       // kStages x 8 bytes
   volatile int32_t* meta = reinterpret_cast<volatile int32_t*>(misc + 32);  // [kStages][8]
 
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the merge kernel may move in as CTAs of this one retire
   for (int i = threadIdx.x; i < D; i += kWarps * 32) step16[i] = __ldg(p.rope + static_cast<size_t>(kTile) * D + i);
   __syncthreads();
 
@@ -395,6 +396,8 @@ __global__ void mepic_decode_grouped_merge(const GroupedParams p) {
     if ((kvl + p.page_size - 1) / p.page_size != p.plan[p.off_req_ent + b]) atomicOr(p.status, MEPIC_DEV_BAD_PLAN);
   }
   const int k0 = __ldg(p.plan + p.off_part_off + blockIdx.x), k1 = __ldg(p.plan + p.off_part_off + blockIdx.x + 1);
+  // launched as a programmatic dependent of the grouped kernel: its partials are complete and visible after this
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   // a piece that saw no valid slot of the row left (max, sum) = (-inf, 0): it drops out of both passes
   float m_star = -INFINITY;
   for (int k = k0; k < k1; ++k) m_star = fmaxf(m_star, p.part_ml[(static_cast<size_t>(k) * G + g) * 2]);
@@ -423,8 +426,8 @@ int32_t launch_grouped(const GroupedParams& p, int n_ctas, const CUtensorMap& ma
   cudaError_t e = cudaFuncSetAttribute(mepic_decode_grouped<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("decode_grouped: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   mepic_decode_grouped<D, G><<<n_ctas, kWarps * 32, smem, stream>>>(p, map_k, map_v);
-  mepic_decode_grouped_merge<D, G><<<p.batch * p.n_kv_heads, G * D, 0, stream>>>(p);
-  e = cudaGetLastError();
+  e = launch_dependent(mepic_decode_grouped_merge<D, G>, dim3(p.batch * p.n_kv_heads), dim3(G * D), stream, p);
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("decode_grouped: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   mepic_count_launches(2);
   return MEPIC_OK;

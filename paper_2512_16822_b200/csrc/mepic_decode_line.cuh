@@ -113,6 +113,10 @@ __global__ void mepic_decode_merge(const DecodeParams p) {
     if (lane == 0) { sh[0] = cut.piece; sh[1] = before; sh[2] = tiles_of(p.kv_len[b]); }
   }
   __syncthreads();
+  // Everything above read only the call's inputs.  The partials come from the split-KV kernel launched just before
+  // on the same stream: with programmatic dependent launch this kernel may already be resident, so wait for that
+  // kernel's completion (and the visibility of its writes) here rather than at launch.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const long long piece = sh[0], nt = sh[2];
   const int g = threadIdx.x / D, d = threadIdx.x % D;
   const size_t o_at = (static_cast<size_t>(b) * p.n_kv_heads * G + static_cast<size_t>(h) * G + g) * D + d;
