@@ -19,7 +19,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
-def _setup_unshared_decode(index: int, scale: float):
+def _setup_unshared_decode(index: int, scale: float, fp8: bool = False):
     """The decode batch on a layout without chunk sharing: every request owns private copies of its chunks."""
     import torch
     import paper_2512_16822_b200 as M
@@ -41,6 +41,8 @@ def _setup_unshared_decode(index: int, scale: float):
     kv_len = np.asarray(lens, dtype=np.int32)
     dev = RT.Device(cfg)
     dev.k_pool.normal_(); dev.v_pool.normal_()
+    if fp8:
+        return wl, dev, RT.Fp8DecodeBatch(RT.Fp8Pools(dev), page_ids, pos_base, kv_len, kv_len - 1, wl.decode_q())
     return wl, dev, RT.DecodeBatch(dev, page_ids, pos_base, kv_len, kv_len - 1, wl.decode_q())
 
 
@@ -89,7 +91,7 @@ def main() -> None:
     args = ap.parse_args()
     index = args.config if args.config is not None else (2 if args.which == "decode" else 3)
     if args.unshared and args.which == "decode":
-        wl, dev, batch = _setup_unshared_decode(index, args.scale)
+        wl, dev, batch = _setup_unshared_decode(index, args.scale, args.fp8)
     else:
         wl, dev, batch = _setup(index, args.scale, args.which, args.grouped, args.fp8)
     for _ in range(max(args.iters - 1, 1)):
