@@ -1,6 +1,6 @@
 """Run one benchmark configuration through the public binding and print the device time.
 
-    python -m paper_2512_16822_b200.cases decode  --config 2 [--scale 1.0] [--iters 10] [--unshared] [--grouped] [--fp8]
+    python -m paper_2512_16822_b200.cases decode  --config 2 [--scale 1.0] [--iters 10] [--unshared] [--grouped] [--fp8] [--graph]
     python -m paper_2512_16822_b200.cases prefill --config 3 [--scale 0.5] [--iters 4]
 
 A small driver for profiling (a fixed, short sequence of calls that a profiler can capture) and for trying the
@@ -87,6 +87,7 @@ def main() -> None:
     ap.add_argument("--iters", type=int, default=4)
     ap.add_argument("--unshared", action="store_true", help="decode only: no chunk sharing, one page per table entry")
     ap.add_argument("--grouped", action="store_true", help="decode only: the sharing-aware path (host plan + grouped kernel)")
+    ap.add_argument("--graph", action="store_true", help="capture the call in a CUDA graph and time replays (no L2 flush: launch latency)")
     ap.add_argument("--fp8", action="store_true", help="decode only: 8-bit (e4m3) pages made from the bf16 pool by the library's quantiser")
     args = ap.parse_args()
     index = args.config if args.config is not None else (2 if args.which == "decode" else 3)
@@ -97,6 +98,23 @@ def main() -> None:
     for _ in range(max(args.iters - 1, 1)):
         batch.run(wl.sm_scale)
     torch.cuda.synchronize()
+    if args.graph:
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            batch.run(wl.sm_scale, torch.cuda.current_stream())
+        for name, fn in (("direct calls", lambda: batch.run(wl.sm_scale)), ("graph replays", graph.replay)):
+            for _ in range(5):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(200):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            print(f"{args.which} config {index}: {name}: {e0.elapsed_time(e1) / 200 * 1e3:.2f} us per call back to back, device status {dev.read_status()}")
+        return
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev.device)
     times = []
     for _ in range(5):

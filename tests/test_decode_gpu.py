@@ -221,3 +221,37 @@ def test_argument_validation():
                             kv_len=b.kv_len, q_pos=b.q_pos, rope_table=dev.rope, out=b.out, workspace=b.workspace,
                             workspace_bytes=b.ws_bytes, status=dev.status, table_stride=b.stride, batch=1, sm_scale=1.0)
     assert e.value.code == M.MEPIC_E_INVAL
+
+
+def test_decode_call_can_be_captured_in_a_cuda_graph_and_replayed():
+    # The call only enqueues kernels on the caller's stream (tensor maps are encoded on the host and passed by value),
+    # so a serving loop may capture it once and replay it with new q / tables written into the same buffers.
+    wl = make_workload(1)
+    cfg = _config_of(wl)
+    kp, vp = wl.kv_pool()
+    with M.Store(cfg) as st:
+        tables = RT.build_tables(st, wl.chunks, wl.decode_requests)
+    page_ids, pos_base, kv_len, q_pos = RT.pack_tables(tables, wl.page_size)
+    dev = RT.Device(cfg, kp, vp)
+    batch = RT.DecodeBatch(dev, page_ids, pos_base, kv_len, q_pos, wl.decode_q())
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        batch.run(wl.sm_scale, side)                      # first call outside capture (function attributes, entry points)
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        batch.run(wl.sm_scale, torch.cuda.current_stream())
+    rng = np.random.default_rng(3)
+    for _ in range(2):
+        q = f32_to_bf16_bits(rng.standard_normal((len(tables), wl.n_q_heads, wl.head_dim)).astype(np.float32))
+        batch.q.view(torch.int16).copy_(torch.from_numpy(q.view(np.int16)))
+        batch.out.zero_()
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert dev.read_status() == 0
+        got = RT.bf16_bits(batch.out)
+        for b, t in enumerate(tables):
+            want = O.decode_attention_one(q[b], kp, vp, list(t.page_ids), list(t.pos_base), t.kv_len, int(q_pos[b]),
+                                          wl.sm_scale, wl.rope_theta)
+            _check(got[b], want, f"request {b}")
