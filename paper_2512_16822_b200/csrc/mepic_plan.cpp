@@ -12,7 +12,7 @@
 // the request's own single-request item.  Items are laid on one line of (item, kv head, 16-token
 // tile) triples which is cut into equal pieces, one per worker.
 #include <algorithm>
-#include <map>
+#include <cstdint>
 #include <unordered_map>
 #include <vector>
 
@@ -28,7 +28,8 @@ struct Use { int32_t r, e; };
 
 struct Item {
   std::vector<int32_t> req;                 // requests of the group (a request may appear twice)
-  std::vector<std::vector<int32_t>> ent;    // per page of the item: entry index in each request's table
+  std::vector<int32_t> ent;                 // per page of the item, n_req entries: the entry index in each request's table
+  size_t pages() const { return ent.size() / req.size(); }
   int32_t tail_slot_start = -1;
 };
 
@@ -65,43 +66,69 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
   const int R = plan_group_requests(cfg->n_q_heads / Hkv);
   const int tpp = P / kPlanTile;
 
-  // users of every page, in (request, entry) order; a request's partly filled last page stays private
+  // users of every page, in (request, entry) order (a counting sort over page ids); a request's partly filled last
+  // page stays private, and so does an entry whose page id is outside the pool (the kernel reports it)
   std::vector<int32_t> n_ent(batch);
-  std::unordered_map<int32_t, std::vector<Use>> users;
-  std::vector<int32_t> page_order;                       // pages in order of first appearance
   std::vector<std::vector<int32_t>> own(batch);          // entries of a request that no group takes
+  const int32_t NP = cfg->num_pages;
+  std::vector<int32_t> first_use(static_cast<size_t>(NP) + 1, 0);   // becomes the offset of each page's users
+  size_t n_full = 0;
   for (int32_t r = 0; r < batch; ++r) {
     if (kv_len[r] < 1) { mepic_set_error("decode_plan: kv_len[%d] = %d < 1", r, kv_len[r]); return MEPIC_E_INVAL; }
     n_ent[r] = (kv_len[r] + P - 1) / P;
     if (n_ent[r] > table_stride) { mepic_set_error("decode_plan: request %d needs %d entries > stride", r, n_ent[r]); return MEPIC_E_INVAL; }
-    for (int32_t e = 0; e < n_ent[r]; ++e) {
-      const bool full = (e + 1) * P <= kv_len[r];
-      if (!full) { own[r].push_back(e); continue; }
+    const int32_t n_whole = kv_len[r] / P;                // entries 0 .. n_whole-1 are full pages
+    for (int32_t e = 0; e < n_whole; ++e) {
       const int32_t page = page_ids[static_cast<size_t>(r) * table_stride + e];
-      auto it = users.find(page);
-      if (it == users.end()) { page_order.push_back(page); it = users.emplace(page, std::vector<Use>()).first; }
-      it->second.push_back(Use{r, e});
+      if (static_cast<uint32_t>(page) >= static_cast<uint32_t>(NP)) { own[r].push_back(e); continue; }
+      ++first_use[page + 1]; ++n_full;
+    }
+    if (n_whole < n_ent[r]) own[r].push_back(n_whole);
+  }
+  for (int32_t pg = 0; pg < NP; ++pg) first_use[pg + 1] += first_use[pg];
+  std::vector<Use> uses(n_full);
+  std::vector<int32_t> page_order;                       // pages in order of first appearance
+  {
+    std::vector<int32_t> fill(first_use.begin(), first_use.end() - 1);
+    for (int32_t r = 0; r < batch; ++r) {
+      const int32_t n_whole = kv_len[r] / P;
+      for (int32_t e = 0; e < n_whole; ++e) {
+        const int32_t page = page_ids[static_cast<size_t>(r) * table_stride + e];
+        if (static_cast<uint32_t>(page) >= static_cast<uint32_t>(NP)) continue;
+        if (fill[page] == first_use[page]) page_order.push_back(page);
+        uses[fill[page]++] = Use{r, e};
+      }
     }
   }
 
-  // pages with the same user requests form a set; each set is cut into groups of R requests
-  std::map<std::vector<int32_t>, size_t> item_of_group;
+  // pages with the same user requests form a set; each set is cut into groups of R requests; a group's pages
+  // accumulate in one item (found through a hash of its request list, confirmed by comparing the list)
+  std::unordered_map<uint64_t, std::vector<size_t>> item_of_group;
   std::vector<Item> shared_items;
   for (int32_t page : page_order) {
-    const std::vector<Use>& u = users[page];
-    if (u.size() == 1) { own[u[0].r].push_back(u[0].e); continue; }
-    for (size_t at = 0; at < u.size(); at += R) {
-      const size_t n = std::min<size_t>(R, u.size() - at);
+    const Use* u = uses.data() + first_use[page];
+    const size_t n_users = static_cast<size_t>(first_use[page + 1] - first_use[page]);
+    if (n_users == 1) { own[u[0].r].push_back(u[0].e); continue; }
+    for (size_t at = 0; at < n_users; at += R) {
+      const size_t n = std::min<size_t>(R, n_users - at);
       if (n == 1) { own[u[at].r].push_back(u[at].e); continue; }
-      std::vector<int32_t> key(n), ent(n);
-      for (size_t j = 0; j < n; ++j) { key[j] = u[at + j].r; ent[j] = u[at + j].e; }
-      auto it = item_of_group.find(key);
-      if (it == item_of_group.end()) {
-        it = item_of_group.emplace(key, shared_items.size()).first;
-        shared_items.emplace_back();
-        shared_items.back().req = key;
+      uint64_t hsh = 0xcbf29ce484222325ULL;
+      for (size_t j = 0; j < n; ++j) { hsh ^= static_cast<uint64_t>(static_cast<uint32_t>(u[at + j].r)) + 1; hsh *= 0x100000001b3ULL; }
+      std::vector<size_t>& cands = item_of_group[hsh];
+      size_t idx = SIZE_MAX;
+      for (size_t c : cands) {
+        const std::vector<int32_t>& rq = shared_items[c].req;
+        bool same = rq.size() == n;
+        for (size_t j = 0; same && j < n; ++j) same = rq[j] == u[at + j].r;
+        if (same) { idx = c; break; }
       }
-      shared_items[it->second].ent.push_back(ent);
+      if (idx == SIZE_MAX) {
+        idx = shared_items.size();
+        cands.push_back(idx);
+        shared_items.emplace_back();
+        for (size_t j = 0; j < n; ++j) shared_items.back().req.push_back(u[at + j].r);
+      }
+      for (size_t j = 0; j < n; ++j) shared_items[idx].ent.push_back(u[at + j].e);
     }
   }
   std::vector<Item> items;
@@ -112,7 +139,7 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
     std::sort(own[r].begin(), own[r].end());
     Item it;
     it.req = {r};
-    for (int32_t e : own[r]) it.ent.push_back({e});
+    it.ent = own[r];
     if (own[r].back() == n_ent[r] - 1) it.tail_slot_start = (n_ent[r] - 1) * P;
     items.push_back(std::move(it));
   }
@@ -120,7 +147,7 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
   // sizes and offsets
   size_t n_records = 0, n_req_items = 0;
   long long tiles_per_head = 0;
-  for (const Item& it : items) { n_records += it.ent.size(); n_req_items += it.req.size(); tiles_per_head += static_cast<long long>(it.ent.size()) * tpp; }
+  for (const Item& it : items) { n_records += it.pages(); n_req_items += it.req.size(); tiles_per_head += static_cast<long long>(it.pages()) * tpp; }
   const long long total = tiles_per_head * Hkv;
   if (total >= (1ll << 31) || items.size() >= (1u << 27)) { mepic_set_error("decode_plan: batch too large for the plan's 32-bit fields"); return MEPIC_E_CAPACITY; }
   const int n_workers = sms * kPlanWarps;
@@ -154,18 +181,20 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
   for (size_t i = 0; i < items.size(); ++i) {
     const Item& it = items[i];
     int32_t* d = out_plan + off_items + i * (kItemFixed + R);
-    d[kPiReq] = static_cast<int32_t>(it.req.size()); d[kPiRecOff] = rec; d[kPiEnt] = static_cast<int32_t>(it.ent.size());
+    d[kPiReq] = static_cast<int32_t>(it.req.size()); d[kPiRecOff] = rec; d[kPiEnt] = static_cast<int32_t>(it.pages());
     d[kPiTail] = it.tail_slot_start; d[kPiTileStart] = tile_start;
     for (int j = 0; j < R; ++j) d[kPiReqIds + j] = j < static_cast<int>(it.req.size()) ? it.req[j] : -1;
     for (size_t j = 0; j < it.req.size(); ++j) req_items[it.req[j]].push_back(static_cast<int32_t>(i) * 16 + static_cast<int32_t>(j));
-    for (const std::vector<int32_t>& ent : it.ent) {
+    const int nr = static_cast<int>(it.req.size());
+    for (size_t k = 0; k < it.pages(); ++k) {
+      const int32_t* ent = it.ent.data() + k * nr;
       int32_t* q = out_plan + off_records + static_cast<size_t>(rec) * (1 + R);
       q[0] = page_ids[static_cast<size_t>(it.req[0]) * table_stride + ent[0]];
       for (int j = 0; j < R; ++j)
-        q[1 + j] = j < static_cast<int>(ent.size()) ? pos_base[static_cast<size_t>(it.req[j]) * table_stride + ent[j]] : 0;
+        q[1 + j] = j < nr ? pos_base[static_cast<size_t>(it.req[j]) * table_stride + ent[j]] : 0;
       ++rec;
     }
-    tile_start += static_cast<int32_t>(it.ent.size()) * tpp;
+    tile_start += static_cast<int32_t>(it.pages()) * tpp;
   }
   // where each worker's piece begins
   {
@@ -175,7 +204,7 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
       const long long x = static_cast<long long>(w) * piece;
       if (x >= total) { d[0] = static_cast<int32_t>(items.size()); d[1] = 0; d[2] = 0; continue; }
       while (true) {
-        const long long nt = static_cast<long long>(items[i].ent.size()) * tpp;
+        const long long nt = static_cast<long long>(items[i].pages()) * tpp;
         const long long start = static_cast<long long>(out_plan[off_items + i * (kItemFixed + R) + kPiTileStart]) * Hkv;
         if (x < start + nt * Hkv) {
           d[0] = static_cast<int32_t>(i); d[1] = static_cast<int32_t>((x - start) / nt); d[2] = static_cast<int32_t>((x - start) % nt);
@@ -197,7 +226,7 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
   // one slot per piece, and the slots of a (request, kv head) pair are contiguous so that the merge reads one run
   std::vector<long long> count(static_cast<size_t>(batch) * Hkv + 1, 0);
   auto pieces_of = [&](size_t i, int hd) {
-    const long long nt = static_cast<long long>(items[i].ent.size()) * tpp;
+    const long long nt = static_cast<long long>(items[i].pages()) * tpp;
     const long long start = static_cast<long long>(out_plan[off_items + i * (kItemFixed + R) + kPiTileStart]) * Hkv + hd * nt;
     return (start + nt - 1) / piece - start / piece + 1;
   };
