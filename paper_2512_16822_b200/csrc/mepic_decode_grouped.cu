@@ -385,33 +385,58 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
 }
 
 // ---------------------------------------------------------------- merge
-// One CTA per (request, kv head); thread (g, d) folds in the pair's partials, which the plan laid out as one
-// contiguous run of slots: m* = max m, l* = sum l 2^(m - m*), out = sum o 2^(m - m*) / l*  -> bf16.
+// One CTA of four warps per (request, kv head, query head): the row's partials, which the plan laid out as one
+// contiguous run of slots, are dealt round-robin to the warps; a lane owns four output dims.  Two passes
+// (m* = max m; l* = sum l 2^(m - m*), o* = sum o 2^(m - m*)), the warps' results combined through shared memory,
+// out = o* / l* -> bf16.  Many small CTAs with short load chains: the kernel is pure latency.
 template <int D, int G>
-__global__ void mepic_decode_grouped_merge(const GroupedParams p) {
-  const int b = blockIdx.x / p.n_kv_heads, h = blockIdx.x % p.n_kv_heads;
-  const int g = threadIdx.x / D, d = threadIdx.x % D;
-  if (h == 0 && threadIdx.x == 0) {
+__global__ void __launch_bounds__(128) mepic_decode_grouped_merge(const GroupedParams p) {
+  const int unit = blockIdx.x / G, g = blockIdx.x % G;          // unit = request * n_kv_heads + kv head
+  const int b = unit / p.n_kv_heads, h = unit % p.n_kv_heads;
+  const int wv = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __shared__ float sh_m[4], sh_l[4];
+  __shared__ float4 sh_o[4][D / 4];
+  if (h == 0 && g == 0 && threadIdx.x == 0) {
     const int kvl = p.kv_len[b];
     if ((kvl + p.page_size - 1) / p.page_size != p.plan[p.off_req_ent + b]) atomicOr(p.status, MEPIC_DEV_BAD_PLAN);
   }
-  const int k0 = __ldg(p.plan + p.off_part_off + blockIdx.x), k1 = __ldg(p.plan + p.off_part_off + blockIdx.x + 1);
+  const int k0 = __ldg(p.plan + p.off_part_off + unit), k1 = __ldg(p.plan + p.off_part_off + unit + 1);
   // launched as a programmatic dependent of the grouped kernel: its partials are complete and visible after this
   asm volatile("griddepcontrol.wait;" ::: "memory");
   // a piece that saw no valid slot of the row left (max, sum) = (-inf, 0): it drops out of both passes
-  float m_star = -INFINITY;
-  for (int k = k0; k < k1; ++k) m_star = fmaxf(m_star, p.part_ml[(static_cast<size_t>(k) * G + g) * 2]);
-  float l_star = 0.f, o_star = 0.f;
-#pragma unroll 4
-  for (int k = k0; k < k1; ++k) {
+  float m_mine = -INFINITY;
+  for (int k = k0 + wv; k < k1; k += 4) m_mine = fmaxf(m_mine, p.part_ml[(static_cast<size_t>(k) * G + g) * 2]);
+  if (lane == 0) sh_m[wv] = m_mine;
+  __syncthreads();
+  const float m_star = fmaxf(fmaxf(sh_m[0], sh_m[1]), fmaxf(sh_m[2], sh_m[3]));
+  float l_mine = 0.f;
+  float4 o_mine = make_float4(0.f, 0.f, 0.f, 0.f);
+  const bool has_dims = lane < D / 4;
+#pragma unroll 2
+  for (int k = k0 + wv; k < k1; k += 4) {
     const size_t row = static_cast<size_t>(k) * G + g;
     const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + row * 2);
     const float wgt = ml.y > 0.f ? ex2(ml.x - m_star) : 0.f;
-    l_star += ml.y * wgt;
-    o_star += p.part_o[row * D + d] * wgt;
+    l_mine += ml.y * wgt;
+    if (has_dims) {
+      const float4 o = *reinterpret_cast<const float4*>(p.part_o + row * D + 4 * lane);
+      o_mine.x += o.x * wgt; o_mine.y += o.y * wgt; o_mine.z += o.z * wgt; o_mine.w += o.w * wgt;
+    }
   }
-  const size_t o_at = (static_cast<size_t>(b) * p.n_kv_heads * G + static_cast<size_t>(h) * G + g) * D + d;
-  p.out[o_at] = l_star > 0.f ? f32_to_bf16_bits(o_star / l_star) : static_cast<uint16_t>(0);
+  if (lane == 0) sh_l[wv] = l_mine;
+  if (has_dims) sh_o[wv][lane] = o_mine;
+  __syncthreads();
+  if (wv == 0 && has_dims) {
+    const float l_star = (sh_l[0] + sh_l[1]) + (sh_l[2] + sh_l[3]);
+    float4 o = sh_o[0][lane];
+#pragma unroll
+    for (int k = 1; k < 4; ++k) { const float4 x = sh_o[k][lane]; o.x += x.x; o.y += x.y; o.z += x.z; o.w += x.w; }
+    const float inv = l_star > 0.f ? 1.f / l_star : 0.f;
+    const size_t o_at = (static_cast<size_t>(b) * p.n_kv_heads * G + static_cast<size_t>(h) * G + g) * D + 4 * lane;
+    const uint32_t lo = static_cast<uint32_t>(f32_to_bf16_bits(o.x * inv)) | (static_cast<uint32_t>(f32_to_bf16_bits(o.y * inv)) << 16);
+    const uint32_t hi = static_cast<uint32_t>(f32_to_bf16_bits(o.z * inv)) | (static_cast<uint32_t>(f32_to_bf16_bits(o.w * inv)) << 16);
+    *reinterpret_cast<uint2*>(p.out + o_at) = make_uint2(lo, hi);
+  }
 }
 
 template <int D, int G>
@@ -426,7 +451,7 @@ int32_t launch_grouped(const GroupedParams& p, int n_ctas, const CUtensorMap& ma
   cudaError_t e = cudaFuncSetAttribute(mepic_decode_grouped<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("decode_grouped: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   mepic_decode_grouped<D, G><<<n_ctas, kWarps * 32, smem, stream>>>(p, map_k, map_v);
-  e = launch_dependent(mepic_decode_grouped_merge<D, G>, dim3(p.batch * p.n_kv_heads), dim3(G * D), stream, p);
+  e = launch_dependent(mepic_decode_grouped_merge<D, G>, dim3(p.batch * p.n_kv_heads * G), dim3(128), stream, p);
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("decode_grouped: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   mepic_count_launches(2);
