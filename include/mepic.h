@@ -17,9 +17,10 @@
  *    mepic_last_error() returns thread-local text for the last failure.
  *  - "host" / "device" is stated for every pointer.  The CALLER owns every
  *    device buffer and the CUDA stream; the library owns only the host
- *    metadata inside mepic_store_t.  The library never allocates or frees
- *    device memory and never synchronises the stream: kernels are enqueued
- *    and the call returns.
+ *    metadata inside mepic_store_t (and, when a remote tier is attached, that
+ *    tier's page-locked HOST buffer).  The library never allocates or frees
+ *    device memory and never synchronises the stream: kernels and copies are
+ *    enqueued and the call returns.
  *  - Device-side problems (a page id outside the pool, a bounded wait that ran
  *    out) never fault or hang the GPU: the kernel records a code in the device
  *    status word the caller passes and carries on with safe values.  Read the

@@ -21,11 +21,14 @@
 //   MMA warp      : one thread issues, per M-tile, S = Q' K'^T (8 x tcgen05.mma 128x128x16
 //                   into tensor memory) and O += P V (8 x 128 x D x 16), alternating the
 //                   two M-tiles: PV_a(j), QK_a(j+1), PV_b(j), QK_b(j+1).
-//   softmax warps : one warpgroup per M-tile; thread r owns row r: tcgen05.ld the scores, causal mask by logical
+//   softmax warps : two warpgroups per M-tile; row r is shared by two threads, one per half of
+//                   the tile's 128 score columns: tcgen05.ld the scores, causal mask by logical
 //                   slot, online softmax in the log2 domain with a lazily moved reference
-//                   maximum, P -> bf16 -> tensor memory (over the first half of the tile's
-//                   S buffer, from where the PV MMA takes it as its A operand); rescales O
-//                   in tensor memory when the reference moved; the epilogue writes O / l.
+//                   maximum that the two threads agree on through shared memory once per tile,
+//                   P -> bf16 -> tensor memory (over the first columns of each half of the S
+//                   buffer, from where the PV MMA takes it as its A operand); each rescales its
+//                   half of the O columns in tensor memory when the reference moved; the
+//                   epilogue writes O / l.
 // Q' carries the rotation at the row's own position and sm_scale * log2(e).
 // Every wait is bounded; a wait that runs out raises an abort flag every role checks.
 #include <cuda.h>
