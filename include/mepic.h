@@ -400,9 +400,12 @@ int32_t mepic_attn_decode_fp8(const mepic_config_t* cfg, const mepic_decode_args
  * the request's PRIVATE pages (shared pages are never written by a correct caller; the library
  * cannot tell).  All struct pointers are DEVICE pointers except row_offsets_host (host copy of
  * row_offsets, batch+1 entries, read during the call for launch sizing).
- * workspace: mepic_attn_prefill_workspace() bytes, 16-byte aligned (a token amount: each CTA derives its share
- * of the work on the device from row_offsets, nothing is built or uploaded by the call, which only enqueues two
- * kernels).  Errors as for decode.
+ * workspace: mepic_attn_prefill_workspace() bytes, 16-byte aligned.  Each CTA derives its share of the work on the
+ * device from row_offsets; nothing is built or uploaded by the call, which only enqueues kernels.  When the work
+ * items fill at least one wave of the GPU that amount is 16 bytes.  When they do not (one request, say), each item's
+ * key range is cut into up to four shares, one CTA each, whose per-row partials (reference, sum, unnormalised
+ * output: 4 (head_dim + 2) bytes per row, q head and share) go to the workspace and are merged by a third kernel;
+ * given a smaller workspace the call runs one CTA per item instead.  Errors as for decode.
  */
 typedef struct {
   const void*    q_new;        /* bf16 [rows][n_q_heads][head_dim], un-rotated */

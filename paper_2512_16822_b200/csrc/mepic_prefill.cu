@@ -70,6 +70,9 @@ struct PrefillParams {
   int32_t* status;
   int table_stride, batch, n_kv_heads, page_size, num_pages, max_position, total_rows;
   int max_q_tiles;      // most CTA-sized tiles of query positions any request has (launch sizing, from the host copy)
+  int n_splits;         // CTAs per work item: each takes a contiguous share of the item's key tiles (1 = no split)
+  float* part_o;        // n_splits > 1: [split][row][q head][D] unnormalised O of the share
+  float* part_ml;       // n_splits > 1: [split][row][q head][2] = (reference maximum in log2 units, sum)
   float scale_log2;
 };
 
@@ -352,7 +355,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   Item* item_slot = reinterpret_cast<Item*>(bars + kNumBars + 16);
   if (warp == 1) {
-    const Item it = item_of_cta(p.row_offsets, p.batch, p.n_kv_heads, 2 * QT, p.max_q_tiles, blockIdx.x, lane);
+    const Item it = item_of_cta(p.row_offsets, p.batch, p.n_kv_heads, 2 * QT, p.max_q_tiles, blockIdx.x / p.n_splits, lane);
     if (lane == 0) *item_slot = it;
   }
   __syncthreads();
@@ -402,8 +405,18 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     lim[x] = l;
     nt[x] = l / kTileN + 1;
   }
-  const int n_tiles = nt[1] > nt[0] ? nt[1] : nt[0];
-  const bool last_has_tail = n_tiles * kTileN > kvl;
+  // With few work items (a single request, say) each item is cut into n_splits CTAs so that the grid still fills
+  // the GPU: this CTA takes key tiles [tile_base, tile_base + n_tiles) of the item's n_all and leaves a partial
+  // (reference, sum, unnormalised O) per row that a second kernel merges.  From here on nt[] and n_tiles count
+  // this CTA's tiles.
+  const int n_all = nt[1] > nt[0] ? nt[1] : nt[0];
+  const int split = blockIdx.x % p.n_splits;
+  const int tile_base = static_cast<int>(static_cast<long long>(n_all) * split / p.n_splits);
+  const int tile_end = static_cast<int>(static_cast<long long>(n_all) * (split + 1) / p.n_splits);
+#pragma unroll
+  for (int x = 0; x < 2; ++x) nt[x] = min(max(nt[x], tile_base), tile_end) - tile_base;
+  const int n_tiles = tile_end - tile_base;
+  const bool last_has_tail = n_tiles > 0 && tile_end == n_all && n_all * kTileN > kvl;
 
   // ---- stage Q (all threads): rotate each row at its own position, fold in sm_scale*log2e, round to bf16
   for (int task = tid; task < 256 * CH; task += kThreads) {
@@ -481,7 +494,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     for (int tile = 0; tile < my_tiles; ++tile) {
       if (!mbar_wait_warp(BAR(kBarSFull, x), static_cast<uint32_t>(tile) & 1u, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
-      const int n_vis = limit - tile * kTileN + 1 - 64 * ch;     // my columns [0, n_vis) are visible to this row
+      const int n_vis = limit - (tile_base + tile) * kTileN + 1 - 64 * ch;     // my columns [0, n_vis) are visible to this row
       const bool boundary = n_vis < 64;                          // only the tile(s) on the causal boundary need the mask
       // ---- pass 1: maximum of my 64 scores
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -525,7 +538,10 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       }
       // ---- pass 2: P = 2^(S - reference) as bf16 pairs over the first 32 of my 64 columns
       float2 sum2[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};
-      const float2 ref2 = make_float2(m_ref, m_ref);
+      // a row none of whose keys lies in this CTA's share so far still has m_ref = -inf: every score is masked
+      // (-inf) and must give P = 0, not 2^(-inf + inf)
+      const float m_use = m_ref == -INFINITY ? 0.f : m_ref;
+      const float2 ref2 = make_float2(m_use, m_use);
 #pragma unroll 1
       for (int q = 0; q < 2; ++q) {
         uint32_t sv[32], pw[16];
@@ -552,28 +568,50 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       tc_fence_before();
       mbar_arrive(BAR(kBarPFull, x));
     }
-    // ---- epilogue: out = O / l once the last PV has completed; each thread of the row writes half of it
+    // ---- epilogue once the last PV has completed; each thread of the row writes its half of the head dims:
+    // out = O / l, or (when the item is split) this share's unnormalised O with its reference and sum
+    if (p.n_splits > 1 && my_tiles == 0 && row_live && ch == 0) {
+      const size_t at = (static_cast<size_t>(split) * p.total_rows + item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g;
+      *reinterpret_cast<float2*>(p.part_ml + at * 2) = make_float2(-INFINITY, 0.f);      // nothing of this row in the share
+    }
     if (ok && my_tiles > 0) {
       const float l_tot = l_run + swap_with_partner(l_run, ok);
       if (ok) ok = mbar_wait_warp(BAR(kBarPvDone, x), static_cast<uint32_t>(my_tiles - 1) & 1u, abort_flag, p.status);
       if (ok) {
         tc_fence_after();
-        const float inv = 1.f / l_tot;
-        uint16_t* dst = p.out + (static_cast<size_t>(item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g) * D + ch * (D / 2);
+        const size_t rh = static_cast<size_t>(item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g;
+        if (p.n_splits == 1) {
+          const float inv = 1.f / l_tot;
+          uint16_t* dst = p.out + rh * D + ch * (D / 2);
 #pragma unroll 1
-        for (int cb = 0; cb < D / 2; cb += 32) {
-          uint32_t o[32];
-          TMEM_LD32(t_O + cb, o, 0);
-          tmem_wait_ld();
-          if (row_live) {
+          for (int cb = 0; cb < D / 2; cb += 32) {
+            uint32_t o[32];
+            TMEM_LD32(t_O + cb, o, 0);
+            tmem_wait_ld();
+            if (row_live) {
 #pragma unroll
-            for (int c = 0; c < 32; c += 8) {
-              uint4 w;
-              w.x = pack_bf16x2(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
-              w.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
-              w.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
-              w.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
-              *reinterpret_cast<uint4*>(dst + cb + c) = w;
+              for (int c = 0; c < 32; c += 8) {
+                uint4 w;
+                w.x = pack_bf16x2(__uint_as_float(o[c + 0]) * inv, __uint_as_float(o[c + 1]) * inv);
+                w.y = pack_bf16x2(__uint_as_float(o[c + 2]) * inv, __uint_as_float(o[c + 3]) * inv);
+                w.z = pack_bf16x2(__uint_as_float(o[c + 4]) * inv, __uint_as_float(o[c + 5]) * inv);
+                w.w = pack_bf16x2(__uint_as_float(o[c + 6]) * inv, __uint_as_float(o[c + 7]) * inv);
+                *reinterpret_cast<uint4*>(dst + cb + c) = w;
+              }
+            }
+          }
+        } else {
+          const size_t at = static_cast<size_t>(split) * p.total_rows * n_q_heads + rh;
+          float* dst = p.part_o + at * D + ch * (D / 2);
+          if (row_live && ch == 0) *reinterpret_cast<float2*>(p.part_ml + at * 2) = make_float2(m_ref, l_tot);
+#pragma unroll 1
+          for (int cb = 0; cb < D / 2; cb += 32) {
+            uint32_t o[32];
+            TMEM_LD32(t_O + cb, o, 0);
+            tmem_wait_ld();
+            if (row_live) {
+#pragma unroll
+              for (int c = 0; c < 32; c += 4) *reinterpret_cast<uint4*>(dst + cb + c) = make_uint4(o[c], o[c + 1], o[c + 2], o[c + 3]);
             }
           }
         }
@@ -600,7 +638,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       const uint32_t ph = static_cast<uint32_t>(tile / kKStages) & 1u;
       if (!mbar_wait(BAR(kBarKLanded, st), ph, abort_flag, p.status)) break;
       unsigned char* Kb = Ks + st * NB * kBlockBytes;
-      const int key0 = tile * kTileN;
+      const int key0 = (tile_base + tile) * kTileN;
       int pos = gbase[st * 8 + k0 / 16] + (k0 & 15);
       if (pos < 0 || pos > p.max_position) {
         if (key0 + k0 < kvl) atomicOr(p.status, MEPIC_DEV_BAD_POSITION);
@@ -659,7 +697,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         const uint32_t bar = BAR(is_k ? kBarKFree : kBarVFree, st);
         if (!mbar_wait_warp(bar, static_cast<uint32_t>(tile / depth - 1) & 1u, abort_flag, p.status)) { ok = false; break; }
       }
-      const int key0 = tile * kTileN;
+      const int key0 = (tile_base + tile) * kTileN;
       const int gkey = key0 + lane * 16;
       const bool live = lane < 8 && gkey < kvl;
       int page = 0, pos = 0, slot0 = 0;
@@ -689,7 +727,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       const int lt = n_tiles - 1, st = lt % kVStages;
       if (mbar_wait_warp(BAR(kBarVLanded, st), static_cast<uint32_t>(lt / kVStages) & 1u, abort_flag, p.status)) {
         unsigned char* Vb = Vs + st * NB * kBlockBytes;
-        const int first = kvl - lt * kTileN;       // first row to clear (0 < first < 128)
+        const int first = kvl - (tile_base + lt) * kTileN;       // first row to clear (0 < first < 128)
         for (int idx = first * 2 * CH + lane; idx < kTileN * 2 * CH; idx += 32) {
           const int kk = idx / (2 * CH), ch = idx % (2 * CH);
           *reinterpret_cast<uint4*>(Vb + (ch / 8) * kBlockBytes + sw128(kk, ch % 8)) = make_uint4(0, 0, 0, 0);
@@ -736,7 +774,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       return w;
     };
     // prologue: S of key tile 0 for both M-tiles
-    ok = wait_k(0);
+    ok = n_tiles > 0 && wait_k(0);
     if (ok) {
       if (nt[0] > 0) issue_qk(0, 0);
       if (nt[1] > 0) issue_qk(1, 0);
@@ -789,6 +827,37 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
 }
 
+// Merge of the shares of a split item: one warp per (row, q head), a lane per four head dims.
+template <int D>
+__global__ void __launch_bounds__(128) mepic_prefill_merge(const PrefillParams p, int n_q_heads) {
+  const long long pair = static_cast<long long>(blockIdx.x) * 4 + (threadIdx.x >> 5);
+  const long long n_pairs = static_cast<long long>(p.total_rows) * n_q_heads;
+  const int lane = threadIdx.x & 31;
+  if (pair >= n_pairs) return;
+  float m_star = -INFINITY;
+  for (int s = 0; s < p.n_splits; ++s) {
+    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + (static_cast<size_t>(s) * n_pairs + pair) * 2);
+    if (ml.y > 0.f) m_star = fmaxf(m_star, ml.x);
+  }
+  float l_star = 0.f;
+  float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < p.n_splits; ++s) {
+    const size_t at = static_cast<size_t>(s) * n_pairs + pair;
+    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + at * 2);
+    if (!(ml.y > 0.f)) continue;                     // the share held none of this row's keys
+    const float wgt = ex2(ml.x - m_star);
+    l_star += ml.y * wgt;
+    if (lane < D / 4) {
+      const float4 x = *reinterpret_cast<const float4*>(p.part_o + at * D + 4 * lane);
+      o.x += x.x * wgt; o.y += x.y * wgt; o.z += x.z * wgt; o.w += x.w * wgt;
+    }
+  }
+  if (lane < D / 4) {
+    const float inv = l_star > 0.f ? 1.f / l_star : 0.f;
+    *reinterpret_cast<uint2*>(p.out + pair * D + 4 * lane) = make_uint2(pack_bf16x2(o.x * inv, o.y * inv), pack_bf16x2(o.z * inv, o.w * inv));
+  }
+}
+
 template <int D, int G>
 int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
   constexpr size_t smem = PrefillSmem<D>::kBytes;
@@ -796,10 +865,14 @@ int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& m
   if (e != cudaSuccess) { mepic_set_error("prefill: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   const int chunks_per_row = p.n_kv_heads * D / 8;
   mepic_prefill_commit<<<p.total_rows, 128, 0, stream>>>(p, chunks_per_row);
-  mepic_prefill_attn<D, G><<<n_items, kThreads, smem, stream>>>(p, map_k, map_v);
+  mepic_prefill_attn<D, G><<<n_items * p.n_splits, kThreads, smem, stream>>>(p, map_k, map_v);
+  if (p.n_splits > 1) {
+    const long long n_pairs = static_cast<long long>(p.total_rows) * p.n_kv_heads * G;
+    mepic_prefill_merge<D><<<static_cast<unsigned>((n_pairs + 3) / 4), 128, 0, stream>>>(p, p.n_kv_heads * G);
+  }
   e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("prefill: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
-  mepic_count_launches(2);
+  mepic_count_launches(p.n_splits > 1 ? 3 : 2);
   return MEPIC_OK;
 }
 
@@ -823,13 +896,30 @@ bool count_items(const mepic_config_t* cfg, int batch, const int32_t* row_offset
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// How many CTAs share a work item: 1 when the items fill at least one wave of the GPU, else enough for about three
+// waves of shares (at most kMaxSplits).  Depends on the SM count of the current device; 1 without a device.
+constexpr int kMaxSplits = 4;
+int splits_for(int n_items) {
+  int dev = 0, sms = 0;
+  if (n_items <= 0 || cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+    return 1;
+  if (n_items >= sms) return 1;                  // a full wave or more: a share's fixed cost (Q staging, pipeline fill, partials) outweighs the balance
+  return std::max(1, std::min(kMaxSplits, (3 * sms + n_items - 1) / n_items));
+}
+size_t split_workspace_bytes(const mepic_config_t* cfg, long long total_rows, int splits) {
+  if (splits <= 1) return 16;
+  return 16 + static_cast<size_t>(splits) * static_cast<size_t>(total_rows) * cfg->n_q_heads * (cfg->head_dim + 2) * sizeof(float);
+}
+
 }  // namespace
 
 extern "C" size_t mepic_attn_prefill_workspace(const mepic_config_t* cfg, int32_t batch, const int32_t* row_offsets_host) {
   if (!mepic_config_ok(cfg) || batch < 1 || !row_offsets_host) { if (cfg) mepic_set_error("prefill_workspace: bad argument"); return 0; }
   int n_items = 0, deepest = 0;
   if (!count_items(cfg, batch, row_offsets_host, &n_items, &deepest)) { mepic_set_error("prefill_workspace: row_offsets must be non-decreasing"); return 0; }
-  return 16;       // the kernels derive their work on the device; a token amount keeps the argument meaningful
+  // 16 bytes when the items fill the GPU by themselves (the kernels derive their work on the device; nothing is
+  // staged); else room for the partials of the items' key-range shares
+  return split_workspace_bytes(cfg, row_offsets_host[batch], splits_for(n_items));
 }
 
 extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_prefill_args_t* a, void* cuda_stream) {
@@ -868,6 +958,10 @@ extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_pre
   p.table_stride = a->table_stride; p.batch = a->batch; p.n_kv_heads = cfg->n_kv_heads; p.page_size = cfg->page_size;
   p.num_pages = cfg->num_pages; p.max_position = cfg->max_position; p.total_rows = total_rows;
   p.max_q_tiles = max_q_tiles;
+  p.n_splits = splits_for(n_items);
+  if (a->workspace_bytes < split_workspace_bytes(cfg, total_rows, p.n_splits)) p.n_splits = 1;     // no room for partials: one CTA per item
+  p.part_o = reinterpret_cast<float*>(static_cast<unsigned char*>(a->workspace) + 16);
+  p.part_ml = p.part_o + static_cast<size_t>(p.n_splits) * total_rows * cfg->n_q_heads * cfg->head_dim;
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
   const int D = cfg->head_dim, G = cfg->n_q_heads / cfg->n_kv_heads;
 #define MEPIC_PREFILL_CASE(DD, GG) if (D == DD && G == GG) return launch_prefill<DD, GG>(p, n_items, map_k, map_v, st);

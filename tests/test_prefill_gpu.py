@@ -177,3 +177,24 @@ def test_bad_slot_and_bad_page_are_reported_not_faulted():
                     rows[0].v_new).run(0.1)
     torch.cuda.synchronize()
     assert dev2.read_status() & M.MEPIC_DEV_BAD_SLOT
+
+
+def test_small_grids_split_the_key_range_and_agree_with_the_unsplit_run():
+    # one request: 8 work items for 148 SMs, so each item is cut into key-range shares whose partials a second kernel
+    # merges; with a 16-byte workspace the same call runs one CTA per item.  Both against the oracle, and each other.
+    L = 9 * 128 + 77
+    new = sorted(set(list(range(0, 16)) + list(range(512, 528)) + list(range(1024, 1040)) + list(range(L - 90, L))))
+    cfg, kp, vp, ids, base, kvl, slots, rows = _manual(31, Hq=8, Hkv=2, D=128, P=16, specs=[(L, new)], theta=5e5)
+    dev, batch = _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 0.1, 5e5)
+    assert batch.ws_bytes > 16, "this grid is expected to be split"
+    split_out = RT.bf16_bits(batch.out).copy()
+    launches = M.mepic_launch_count()
+    batch.ws_bytes = 16                                     # no room for partials: the library must fall back to one CTA per item
+    out = batch.run(0.1)
+    torch.cuda.synchronize()
+    assert dev.read_status() == 0 and M.mepic_launch_count() - launches == 2
+    ok, ov = kp.copy(), vp.copy()
+    want = O.prefill_attention_one(rows[0].q_new, rows[0].k_new, rows[0].v_new, list(slots[0]), ok, ov, list(ids[0, :-(-L // 16)]),
+                                   list(base[0, :-(-L // 16)]), L, 0.1, 5e5)
+    _check(RT.bf16_bits(out), want, "unsplit")
+    assert np.abs(bf16_bits_to_f64(RT.bf16_bits(out)) - bf16_bits_to_f64(split_out)).max() <= 8e-3
