@@ -236,6 +236,7 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 // ---------------------------------------------------------------- commit (Section 3.3.2)
 // One CTA per new row: its K and V bits go, un-rotated, to (page, slot) of the pools.
 __global__ void mepic_prefill_commit(const PrefillParams p, int chunks_per_row) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the attention kernel may stage its queries meanwhile
   const int row = blockIdx.x;
   __shared__ int sh_b;
   if (threadIdx.x == 0) {
@@ -690,6 +691,9 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     unsigned char* ring = is_k ? Ks : Vs;
     const int depth = is_k ? kKStages : kVStages;
     bool ok = true;
+    // This kernel is launched as a programmatic dependent of the commit kernel: everything up to here read only
+    // the call's inputs; the pools may be read once that kernel has completed and its writes are visible.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     for (int tile = 0; tile < n_tiles; ++tile) {
       const int st = tile % depth;
       if (tile >= depth) {
@@ -834,6 +838,7 @@ __global__ void __launch_bounds__(128) mepic_prefill_merge(const PrefillParams p
   const long long n_pairs = static_cast<long long>(p.total_rows) * n_q_heads;
   const int lane = threadIdx.x & 31;
   if (pair >= n_pairs) return;
+  asm volatile("griddepcontrol.wait;" ::: "memory");              // launched as a programmatic dependent of the attention kernel
   float m_star = -INFINITY;
   for (int s = 0; s < p.n_splits; ++s) {
     const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + (static_cast<size_t>(s) * n_pairs + pair) * 2);
@@ -865,12 +870,21 @@ int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& m
   if (e != cudaSuccess) { mepic_set_error("prefill: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   const int chunks_per_row = p.n_kv_heads * D / 8;
   mepic_prefill_commit<<<p.total_rows, 128, 0, stream>>>(p, chunks_per_row);
-  mepic_prefill_attn<D, G><<<n_items * p.n_splits, kThreads, smem, stream>>>(p, map_k, map_v);
-  if (p.n_splits > 1) {
+  // each kernel may become resident while its predecessor drains (programmatic dependent launch); it waits with
+  // griddepcontrol.wait before it touches what the predecessor writes
+  cudaLaunchAttribute pdl[1];
+  pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  pdl[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(static_cast<unsigned>(n_items * p.n_splits)); lc.blockDim = dim3(kThreads); lc.dynamicSmemBytes = smem; lc.stream = stream;
+  lc.attrs = pdl; lc.numAttrs = 1;
+  e = cudaLaunchKernelEx(&lc, mepic_prefill_attn<D, G>, p, map_k, map_v);
+  if (e == cudaSuccess && p.n_splits > 1) {
     const long long n_pairs = static_cast<long long>(p.total_rows) * p.n_kv_heads * G;
-    mepic_prefill_merge<D><<<static_cast<unsigned>((n_pairs + 3) / 4), 128, 0, stream>>>(p, p.n_kv_heads * G);
+    lc.gridDim = dim3(static_cast<unsigned>((n_pairs + 3) / 4)); lc.blockDim = dim3(128); lc.dynamicSmemBytes = 0;
+    e = cudaLaunchKernelEx(&lc, mepic_prefill_merge<D>, p, p.n_kv_heads * G);
   }
-  e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("prefill: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   mepic_count_launches(p.n_splits > 1 ? 3 : 2);
   return MEPIC_OK;
