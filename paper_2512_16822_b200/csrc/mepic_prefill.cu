@@ -326,7 +326,8 @@ constexpr int kBarPFull = kBarSFull + 2;                // [2] P of the current 
 constexpr int kBarPvDone = kBarPFull + 2;               // [2] PV of the current tile complete
 constexpr int kBarVPatched = kBarPvDone + 2;            // [1] rows past kv_len of the last V tile zeroed
 constexpr int kBarPair = kBarVPatched + 1;              // [2 M-tiles][4 quadrants] the two warps that share 32 rows
-constexpr int kNumBars = kBarPair + 8;
+constexpr int kBarQReady = kBarPair + 8;                // [1] Q' of both M-tiles is staged
+constexpr int kNumBars = kBarQReady + 1;
 
 template <int D, int G>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -390,6 +391,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     }
     mbar_init(BAR(kBarVPatched, 0), 1);
     for (int s = 0; s < 8; ++s) mbar_init(BAR(kBarPair, s), 64);
+    mbar_init(BAR(kBarQReady, 0), kSoftmaxWarps * 32);      // the softmax warps stage Q'
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -419,8 +421,15 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   const int n_tiles = tile_end - tile_base;
   const bool last_has_tail = n_tiles > 0 && tile_end == n_all && n_all * kTileN > kvl;
 
-  // ---- stage Q (all threads): rotate each row at its own position, fold in sm_scale*log2e, round to bf16
-  for (int task = tid; task < 256 * CH; task += kThreads) {
+  tc_fence_before();
+  __syncthreads();             // barriers initialised, tensor memory allocated
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  // ---- stage Q (the softmax warps; meanwhile the loaders and rotators already work on the first key tiles):
+  // rotate each row at its own position, fold in sm_scale*log2e, round to bf16
+  if (warp < kSoftmaxWarps) {
+  for (int task = tid; task < 256 * CH; task += kSoftmaxWarps * 32) {
     const int rr2 = task / CH, c = task % CH;
     const int x = rr2 >> 7, rr = rr2 & 127;
     const int qq = x * QT + rr / G, gg = rr % G;
@@ -453,10 +462,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     *reinterpret_cast<uint4*>(Qx + (hc / 8) * kBlockBytes + sw128(rr, hc % 8)) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
   }
   fence_async_smem();          // Q is read by the tensor core (async proxy)
-  tc_fence_before();
-  __syncthreads();
-  tc_fence_after();
-  const uint32_t tmem_base = *tmem_slot;
+  mbar_arrive(BAR(kBarQReady, 0));
+  }
 
   if (warp < kSoftmaxWarps) {
     // =============================================================== softmax warps
@@ -778,7 +785,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       return w;
     };
     // prologue: S of key tile 0 for both M-tiles
-    ok = n_tiles > 0 && wait_k(0);
+    ok = n_tiles > 0 && mbar_wait(BAR(kBarQReady, 0), 0, abort_flag, p.status) && wait_k(0);
     if (ok) {
       if (nt[0] > 0) issue_qk(0, 0);
       if (nt[1] > 0) issue_qk(1, 0);
