@@ -266,11 +266,14 @@ __global__ void mepic_prefill_commit(const PrefillParams p, int chunks_per_row) 
 __device__ __forceinline__ Item item_of_cta(const int32_t* row_offsets, int batch, int n_kv_heads, int qt, int max_q_tiles, int i, int lane) {
   Item it{0, 0, 0, 0};
   int before = 0;                                   // items of the levels above
+  // row counts of the first 32 requests stay in registers: the level loop below would otherwise reload them
+  const int r_first = lane < batch ? __ldg(row_offsets + lane) : 0;
+  const int n_first = lane < batch ? __ldg(row_offsets + lane + 1) - r_first : 0;
   for (int t = max_q_tiles - 1; t >= 0; --t) {
     int cnt = 0;                                    // requests that have a tile at this level
     for (int b0 = 0; b0 < batch; b0 += 32) {
       const int b = b0 + lane;
-      const int n = b < batch ? row_offsets[b + 1] - row_offsets[b] : 0;
+      const int n = b0 == 0 ? n_first : (b < batch ? row_offsets[b + 1] - row_offsets[b] : 0);
       cnt += __popc(__ballot_sync(0xffffffffu, n > t * qt));
     }
     if (i < before + cnt * n_kv_heads) {
@@ -278,7 +281,7 @@ __device__ __forceinline__ Item item_of_cta(const int32_t* row_offsets, int batc
       int seen = 0;
       for (int b0 = 0; b0 < batch; b0 += 32) {
         const int b = b0 + lane;
-        const int n = b < batch ? row_offsets[b + 1] - row_offsets[b] : 0;
+        const int n = b0 == 0 ? n_first : (b < batch ? row_offsets[b + 1] - row_offsets[b] : 0);
         const unsigned m = __ballot_sync(0xffffffffu, n > t * qt);
         const int here = __popc(m);
         if (want < seen + here) {
@@ -288,7 +291,7 @@ __device__ __forceinline__ Item item_of_cta(const int32_t* row_offsets, int batc
           const int bb = b0 + src;
           const int nn = __shfl_sync(0xffffffffu, n, src);
           it.b = bb; it.h = j % n_kv_heads;
-          it.row0 = __shfl_sync(0xffffffffu, b < batch ? row_offsets[b] : 0, src) + t * qt;
+          it.row0 = __shfl_sync(0xffffffffu, b0 == 0 ? r_first : (b < batch ? row_offsets[b] : 0), src) + t * qt;
           it.nq = min(qt, nn - t * qt);
           return it;
         }
