@@ -191,3 +191,13 @@ def test_argument_errors():
                                     kv_len=gb.kv_len, q_pos=gb.q_pos, rope_table=dev.rope, out=gb.out, workspace=gb.workspace,
                                     workspace_bytes=gb.ws_bytes - 16, status=dev.status, batch=2, sm_scale=1.0)
     assert e.value.code == M.MEPIC_E_INVAL
+
+
+def test_more_than_32_requests():
+    n_req = 70
+    rng = np.random.default_rng(5)
+    uses = [sorted(rng.choice(6, size=int(rng.integers(1, 4)), replace=False).tolist()) for _ in range(n_req)]
+    tails = [int(x) for x in rng.integers(1, 50, size=n_req)]
+    args = _shared_case(55, Hq=8, Hkv=2, D=128, P=16, n_req=n_req, chunk_pages=[7, 5, 9, 3, 4, 6], uses=uses,
+                        tail_tokens=tails, jitter=False)
+    _run(*args, 1.0 / np.sqrt(128), 1e4, sample=list(range(0, n_req, 7)))

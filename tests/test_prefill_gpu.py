@@ -198,3 +198,16 @@ def test_small_grids_split_the_key_range_and_agree_with_the_unsplit_run():
                                    list(base[0, :-(-L // 16)]), L, 0.1, 5e5)
     _check(RT.bf16_bits(out), want, "unsplit")
     assert np.abs(bf16_bits_to_f64(RT.bf16_bits(out)) - bf16_bits_to_f64(split_out)).max() <= 8e-3
+
+
+def test_more_than_32_requests_in_one_call():
+    # the device-side work-item lookup scans requests 32 at a time: 45 requests of 1-3 query tiles each
+    rng = np.random.default_rng(41)
+    specs = []
+    for b in range(45):
+        L = int(rng.integers(40, 400))
+        n_new = int(rng.integers(1, min(L, 150)))
+        new = sorted(rng.choice(L, size=n_new, replace=False).tolist())
+        specs.append((L, new))
+    cfg, kp, vp, ids, base, kvl, slots, rows = _manual(42, Hq=8, Hkv=2, D=128, P=16, specs=specs, jitter=True)
+    _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 1.0 / np.sqrt(128), 1e4, sample_rows=lambda R: [0, R // 2, R - 1])
