@@ -2,6 +2,7 @@
 
     python -m paper_2512_16822_b200.cases decode  --config 2 [--scale 1.0] [--iters 10] [--unshared] [--grouped] [--fp8] [--graph]
     python -m paper_2512_16822_b200.cases prefill --config 3 [--scale 0.5] [--iters 4]
+    python -m paper_2512_16822_b200.cases mixed   --config 5            # decode and prefill of one pool on two streams
 
 A small driver for profiling (a fixed, short sequence of calls that a profiler can capture) and for trying the
 library on the synthetic workloads.  Inputs come from ``mepic_inputs``; nothing here checks results (the tests do).
@@ -58,30 +59,65 @@ def _setup(index: int, scale: float, which: str, grouped: bool = False, fp8: boo
         dec = RT.build_tables(st, wl.chunks, wl.decode_requests) if wl.decode_requests else []
         pre = RT.build_tables(st, wl.chunks, wl.prefill_requests) if wl.prefill_requests else []
     dev = RT.Device(cfg, kp, vp)
-    if which == "decode":
+    dbatch = pbatch = None
+    if which in ("decode", "both"):
         if not dec:
             raise SystemExit(f"config {index} has no decode requests")
         page_ids, pos_base, kv_len, q_pos = RT.pack_tables(dec, wl.page_size)
         if fp8:
             return wl, dev, RT.Fp8DecodeBatch(RT.Fp8Pools(dev), page_ids, pos_base, kv_len, q_pos, wl.decode_q())
         kind = RT.GroupedDecodeBatch if grouped else RT.DecodeBatch
-        return wl, dev, kind(dev, page_ids, pos_base, kv_len, q_pos, wl.decode_q())
+        dbatch = kind(dev, page_ids, pos_base, kv_len, q_pos, wl.decode_q())
+        if which == "decode":
+            return wl, dev, dbatch
     if not pre:
         raise SystemExit(f"config {index} has no prefill requests")
     page_ids, pos_base, kv_len, _ = RT.pack_tables(pre, wl.page_size)
     slots = [t.recompute_slots for t in pre]
     rows = [wl.prefill_rows(i, len(s)) for i, s in enumerate(slots)]
     ro = np.concatenate([[0], np.cumsum([len(s) for s in slots])]).astype(np.int32)
-    batch = RT.PrefillBatch(dev, page_ids, pos_base, kv_len, ro, np.concatenate(slots).astype(np.int32),
-                            np.concatenate([r.q_new for r in rows]), np.concatenate([r.k_new for r in rows]),
-                            np.concatenate([r.v_new for r in rows]))
-    return wl, dev, batch
+    pbatch = RT.PrefillBatch(dev, page_ids, pos_base, kv_len, ro, np.concatenate(slots).astype(np.int32),
+                             np.concatenate([r.q_new for r in rows]), np.concatenate([r.k_new for r in rows]),
+                             np.concatenate([r.v_new for r in rows]))
+    return wl, dev, ((dbatch, pbatch) if which == "both" else pbatch)
+
+
+def _mixed(index: int, scale: float) -> None:
+    """A serving step of a config that has both kinds of request: the decode batch and the prefill requests over one
+    pool, each call alone and then both enqueued on two streams (device time from the fork to the join)."""
+    import torch
+    wl, dev, (db, pb) = _setup(index, scale, "both")
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    main_s = torch.cuda.current_stream()
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev.device)
+
+    def both():
+        fork = torch.cuda.Event(); fork.record(main_s)
+        s1.wait_event(fork); s2.wait_event(fork)
+        pb.run(wl.sm_scale, s2)
+        db.run(wl.sm_scale, s1)
+        j1, j2 = torch.cuda.Event(), torch.cuda.Event()
+        j1.record(s1); j2.record(s2)
+        main_s.wait_event(j1); main_s.wait_event(j2)
+
+    for name, fn in (("decode alone", lambda: db.run(wl.sm_scale)), ("prefill alone", lambda: pb.run(wl.sm_scale)),
+                     ("both, two streams", both)):
+        times = []
+        for it in range(8):
+            flush.fill_(1); flush.view(torch.int64).sum()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(); fn(); e1.record()
+            torch.cuda.synchronize()
+            if it >= 3:
+                times.append(e0.elapsed_time(e1))
+        print(f"mixed config {index} scale {scale}: {name}: {sorted(times)[len(times) // 2]:.4f} ms median, {min(times):.4f} min "
+              f"(L2 flushed), device status {dev.read_status()}")
 
 
 def main() -> None:
     import torch
     ap = argparse.ArgumentParser()
-    ap.add_argument("which", choices=["decode", "prefill"])
+    ap.add_argument("which", choices=["decode", "prefill", "mixed"])
     ap.add_argument("--config", type=int, default=None)
     ap.add_argument("--scale", type=float, default=1.0)
     ap.add_argument("--iters", type=int, default=4)
@@ -90,7 +126,10 @@ def main() -> None:
     ap.add_argument("--graph", action="store_true", help="capture the call in a CUDA graph and time replays (no L2 flush: launch latency)")
     ap.add_argument("--fp8", action="store_true", help="decode only: 8-bit (e4m3) pages made from the bf16 pool by the library's quantiser")
     args = ap.parse_args()
-    index = args.config if args.config is not None else (2 if args.which == "decode" else 3)
+    index = args.config if args.config is not None else {"decode": 2, "prefill": 3, "mixed": 5}[args.which]
+    if args.which == "mixed":
+        _mixed(index, args.scale)
+        return
     if args.unshared and args.which == "decode":
         wl, dev, batch = _setup_unshared_decode(index, args.scale, args.fp8)
     else:
