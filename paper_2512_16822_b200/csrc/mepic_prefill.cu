@@ -492,12 +492,12 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     const uint32_t pair_bar = BAR(kBarPair, x * 4 + q4);
     uint32_t pair_ph = 0;
     // publish `v`, wait for the partner warp, return the partner's value of the same row
-    auto swap_with_partner = [&](float v, bool& ok_io) {
-      *mine = v;
+    auto swap_with_partner = [&](float v, bool& ok_io, float* dst, const float* src) {
+      *dst = v;
       mbar_arrive(pair_bar);
       if (!mbar_wait_warp(pair_bar, pair_ph, abort_flag, p.status)) ok_io = false;
       pair_ph ^= 1u;
-      return *theirs;
+      return *src;
     };
     float m_ref = -INFINITY, l_run = 0.f;
     bool ok = true;
@@ -525,7 +525,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         }
       }
       float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      mx = fmaxf(mx, swap_with_partner(mx, ok));
+      mx = fmaxf(mx, swap_with_partner(mx, ok, mine, theirs));
       if (!ok) break;
       // move the reference only when it lags by more than the threshold (both threads of the row decide alike);
       // always true on the first tile: m_ref = -inf and key 0 is visible to every row
@@ -586,7 +586,11 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       *reinterpret_cast<float2*>(p.part_ml + at * 2) = make_float2(-INFINITY, 0.f);      // nothing of this row in the share
     }
     if (ok && my_tiles > 0) {
-      const float l_tot = l_run + swap_with_partner(l_run, ok);
+      // The row sums go through a second pair of slots: the partner may not have read this thread's last maximum yet
+      // (nothing orders that read before this write, unlike inside the loop, where the next write follows a QK^T that
+      // was issued after both threads handed P over).  The M-tile's Q' block is free by now: its last QK^T has completed.
+      float* ep = reinterpret_cast<float*>(Qs + x * NB * kBlockBytes);
+      const float l_tot = l_run + swap_with_partner(l_run, ok, ep + ch * 128 + r, ep + (ch ^ 1) * 128 + r);
       if (ok) ok = mbar_wait_warp(BAR(kBarPvDone, x), static_cast<uint32_t>(my_tiles - 1) & 1u, abort_flag, p.status);
       if (ok) {
         tc_fence_after();
