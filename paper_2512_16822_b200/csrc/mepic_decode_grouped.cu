@@ -24,7 +24,7 @@
 #include "mepic.h"
 #include "mepic_internal.h"
 #include "mepic_plan.h"
-#include "mepic_decode_common.cuh"
+#include "mepic_ptx.cuh"
 
 namespace {
 

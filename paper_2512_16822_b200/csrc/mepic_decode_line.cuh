@@ -4,7 +4,7 @@
 #define MEPIC_DECODE_LINE_CUH_
 
 #include "mepic.h"
-#include "mepic_decode_common.cuh"
+#include "mepic_ptx.cuh"
 
 namespace mepic_dev {
 

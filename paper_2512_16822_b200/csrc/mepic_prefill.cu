@@ -39,8 +39,11 @@
 
 #include "mepic.h"
 #include "mepic_internal.h"
+#include "mepic_ptx.cuh"
 
 namespace {
+
+using namespace mepic_dev;
 
 constexpr int kTileN = 128;            // keys per staged tile
 constexpr int kBlockBytes = 128 * 128; // one [128 rows x 64 bf16] swizzled block
@@ -49,7 +52,6 @@ constexpr int kSoftmaxWarps = 16;       // 2 M-tiles x 2 column halves x 4 lane 
 constexpr int kRotatorWarps = 4;
 constexpr int kKLoaderWarp = 20, kVLoaderWarp = 21, kMmaWarp = 22;   // warp 23 idles
 constexpr int kThreads = 768;
-constexpr int kSpinLimit = 1 << 22;
 constexpr float kRescaleThreshold = 8.f;   // move the reference maximum only when it lags by 2^8
 
 struct Item { int32_t b, h, row0, nq; };   // rows row0 .. row0+nq-1 (global row indices) of request b
@@ -76,11 +78,6 @@ struct PrefillParams {
   float scale_log2;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ float ex2(float x) { float y; asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x)); return y; }
-__device__ __forceinline__ float2 bf16x2_to_float2(uint32_t w) {
-  return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-}
 // packed fp32 pairs (one instruction for two lanes of work)
 __device__ __forceinline__ float2 fma2(float2 a, float2 b, float2 c) {
   float2 d;
@@ -107,44 +104,16 @@ __device__ __forceinline__ float2 add2(float2 a, float2 b) {
       : "=f"(d.x), "=f"(d.y) : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
   return d;
 }
-__device__ __forceinline__ uint32_t bf16x2_mul(uint32_t a, uint32_t b) {
-  uint32_t d;
-  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
-  return d;
-}
 __device__ __forceinline__ uint32_t bf16x2_sub(uint32_t a, uint32_t b) {
   uint32_t d;
   asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
   return d;
 }
-__device__ __forceinline__ uint32_t bf16x2_fma(uint32_t a, uint32_t b, uint32_t c) {
-  uint32_t d;
-  asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-  return d;
-}
-// (lo, hi) -> packed bf16x2, round to nearest even
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
-  uint32_t r;
-  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
-  return r;
-}
 // byte offset of 16-byte chunk `chunk` of row `row` inside a [rows x 128 B] block with the 128-byte swizzle
 __device__ __forceinline__ uint32_t sw128(int row, int chunk) { return static_cast<uint32_t>(row * 128 + ((chunk ^ (row & 7)) << 4)); }
 
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{ .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p; }"
-               : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-  return ok != 0;
 }
 // Bounded wait that also gives up when another role has raised the abort flag.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
@@ -161,11 +130,6 @@ __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, vo
   const bool w = mbar_wait(bar, parity, abort_flag, status);
   return __all_sync(0xffffffffu, w) != 0;
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-               ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-
 // ---- tcgen05 wrappers
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_slot, uint32_t cols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(cols) : "memory");

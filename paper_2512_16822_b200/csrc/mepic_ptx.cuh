@@ -1,7 +1,7 @@
-// PTX wrappers shared by the decode kernels: mbarrier + TMA staging, ldmatrix, warp-level
-// tensor-core MMA (mma.sync m16n8k16, bf16 in, fp32 accumulate) and packed-bf16 arithmetic.
-#ifndef MEPIC_DECODE_COMMON_CUH_
-#define MEPIC_DECODE_COMMON_CUH_
+// PTX wrappers shared by the kernels: mbarrier + TMA staging, ldmatrix, warp-level tensor-core MMA
+// (mma.sync m16n8k16, bf16 in, fp32 accumulate), packed-bf16 arithmetic, programmatic dependent launch.
+#ifndef MEPIC_PTX_CUH_
+#define MEPIC_PTX_CUH_
 
 #include <cuda.h>
 #include <cuda_runtime.h>
