@@ -406,6 +406,8 @@ int32_t mepic_attn_decode_fp8(const mepic_config_t* cfg, const mepic_decode_args
  * key range is cut into up to four shares, one CTA each, whose per-row partials (reference, sum, unnormalised
  * output: 4 (head_dim + 2) bytes per row, q head and share) go to the workspace and are merged by a third kernel;
  * given a smaller workspace the call runs one CTA per item instead.  Errors as for decode.
+ * A request may have no rows (row_offsets[b] == row_offsets[b+1]).  A call with no rows at all returns MEPIC_OK
+ * without launching anything or reading any pointer but row_offsets_host.
  */
 typedef struct {
   const void*    q_new;        /* bf16 [rows][n_q_heads][head_dim], un-rotated */

@@ -916,10 +916,13 @@ extern "C" size_t mepic_attn_prefill_workspace(const mepic_config_t* cfg, int32_
 
 extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_prefill_args_t* a, void* cuda_stream) {
   if (!mepic_config_ok(cfg)) return MEPIC_E_INVAL;
-  if (!a || !a->q_new || !a->k_new || !a->v_new || !a->row_offsets || !a->q_slot || !a->k_pool || !a->v_pool ||
-      !a->page_ids || !a->pos_base || !a->kv_len || !a->rope_table || !a->out || !a->workspace || !a->status ||
-      !a->row_offsets_host) { mepic_set_error("prefill: NULL pointer argument"); return MEPIC_E_INVAL; }
+  if (!a || !a->row_offsets_host) { mepic_set_error("prefill: NULL pointer argument"); return MEPIC_E_INVAL; }
   if (a->batch < 1 || a->table_stride < 1) { mepic_set_error("prefill: batch and table_stride must be positive"); return MEPIC_E_INVAL; }
+  if (a->row_offsets_host[0] == 0 && a->row_offsets_host[a->batch] == 0) return MEPIC_OK;   // no rows at all: the row buffers may be absent
+  if (!a->q_new || !a->k_new || !a->v_new || !a->row_offsets || !a->q_slot || !a->k_pool || !a->v_pool ||
+      !a->page_ids || !a->pos_base || !a->kv_len || !a->rope_table || !a->out || !a->workspace || !a->status) {
+    mepic_set_error("prefill: NULL pointer argument"); return MEPIC_E_INVAL;
+  }
   if (!aligned16(a->q_new) || !aligned16(a->k_new) || !aligned16(a->v_new) || !aligned16(a->k_pool) || !aligned16(a->v_pool) ||
       !aligned16(a->rope_table) || !aligned16(a->out) || !aligned16(a->workspace)) {
     mepic_set_error("prefill: pointers must be 16-byte aligned"); return MEPIC_E_INVAL;

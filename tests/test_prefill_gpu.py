@@ -54,6 +54,8 @@ def _run_prefill(cfg, kp, vp, page_ids, pos_base, kv_len, q_slots, rows, sm_scal
     ok, ov = kp.copy(), vp.copy()
     P = cfg.page_size
     for b in range(B):
+        if len(q_slots[b]) == 0:
+            continue
         n = -(-int(kv_len[b]) // P)
         sel = None
         if sample_rows is not None:
@@ -211,3 +213,20 @@ def test_more_than_32_requests_in_one_call():
         specs.append((L, new))
     cfg, kp, vp, ids, base, kvl, slots, rows = _manual(42, Hq=8, Hkv=2, D=128, P=16, specs=specs, jitter=True)
     _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 1.0 / np.sqrt(128), 1e4, sample_rows=lambda R: [0, R // 2, R - 1])
+
+
+def test_request_without_new_rows_and_call_without_any():
+    # A request whose K/V is entirely cached contributes no query rows: it sits in the batch with an empty row range.
+    specs = [(300, list(range(0, 16)) + [299]), (200, []), (150, list(range(140, 150)))]
+    cfg, kp, vp, ids, base, kvl, slots, rows = _manual(77, Hq=8, Hkv=2, D=128, P=16, specs=specs)
+    _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 1.0 / np.sqrt(128), 1e4)
+    # No rows in the whole call: nothing is launched, the pools keep their bits, the status word stays clear.
+    dev = RT.Device(cfg, kp, vp)
+    empty = np.zeros((0, 8, 128), dtype=np.uint16)
+    batch = RT.PrefillBatch(dev, ids, base, kvl, np.zeros(4, dtype=np.int32), np.zeros(0, dtype=np.int32),
+                            empty, np.zeros((0, 2, 128), dtype=np.uint16), np.zeros((0, 2, 128), dtype=np.uint16))
+    before = M.mepic_launch_count()
+    batch.run(1.0)
+    torch.cuda.synchronize()
+    assert dev.read_status() == 0 and M.mepic_launch_count() == before
+    assert np.array_equal(RT.bf16_bits(dev.k_pool), kp) and np.array_equal(RT.bf16_bits(dev.v_pool), vp)
