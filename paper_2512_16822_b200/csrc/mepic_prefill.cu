@@ -292,8 +292,7 @@ constexpr int kBarSFull = kBarVFree + kVStages;         // [2 M-tiles] S of the 
 constexpr int kBarPFull = kBarSFull + 2;                // [2] P of the current tile is in tensor memory
 constexpr int kBarPvDone = kBarPFull + 2;               // [2] PV of the current tile complete
 constexpr int kBarVPatched = kBarPvDone + 2;            // [1] rows past kv_len of the last V tile zeroed
-constexpr int kBarPair = kBarVPatched + 1;              // [2 M-tiles][4 quadrants] the two warps that share 32 rows
-constexpr int kBarQReady = kBarPair + 8;                // [1] Q' of both M-tiles is staged
+constexpr int kBarQReady = kBarVPatched + 1;                // [1] Q' of both M-tiles is staged
 constexpr int kNumBars = kBarQReady + 1;
 
 template <int D, int G>
@@ -357,7 +356,6 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       mbar_init(BAR(kBarPvDone, s), 1);                      // tcgen05.commit
     }
     mbar_init(BAR(kBarVPatched, 0), 1);
-    for (int s = 0; s < 8; ++s) mbar_init(BAR(kBarPair, s), 64);
     mbar_init(BAR(kBarQReady, 0), kSoftmaxWarps * 32);      // the softmax warps stage Q'
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -453,14 +451,15 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     }
     float* mine = xchg + (x * 2 + ch) * 128 + r;
     const float* theirs = xchg + (x * 2 + (ch ^ 1)) * 128 + r;
-    const uint32_t pair_bar = BAR(kBarPair, x * 4 + q4);
-    uint32_t pair_ph = 0;
-    // publish `v`, wait for the partner warp, return the partner's value of the same row
+    const int pair_id = 1 + x * 4 + q4;         // hardware barrier of the two warps that share these 32 rows (0 is the CTA's)
+    // publish `v`, meet the partner warp, return the partner's value of the same row.  The meeting point is a
+    // hardware barrier (a waiting warp takes no issue slots and wakes at once); it has no time limit of its own, so
+    // a warp that leaves this role early after a lost wait arrives on it once (below) and every warp looks at the
+    // abort flag, which is raised before that arrival, as soon as it is through.
     auto swap_with_partner = [&](float v, bool& ok_io, float* dst, const float* src) {
       *dst = v;
-      mbar_arrive(pair_bar);
-      if (!mbar_wait_warp(pair_bar, pair_ph, abort_flag, p.status)) ok_io = false;
-      pair_ph ^= 1u;
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_id) : "memory");
+      if (*abort_flag) ok_io = false;
       return *src;
     };
     float m_ref = -INFINITY, l_run = 0.f;
@@ -596,6 +595,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         }
       }
     }
+    if (!ok) asm volatile("bar.arrive %0, 64;" ::"r"(pair_id) : "memory");   // never leave the partner at the barrier
   } else if (warp < kSoftmaxWarps + kRotatorWarps) {
     // =============================================================== rotator warps: K tile, in place
     const int rt = tid - kSoftmaxWarps * 32;     // 0..127
