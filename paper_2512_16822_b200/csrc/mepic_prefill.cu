@@ -24,13 +24,15 @@
 //   softmax warps : two warpgroups per M-tile; row r is shared by two threads, one per half of
 //                   the tile's 128 score columns: tcgen05.ld the scores, causal mask by logical
 //                   slot, online softmax in the log2 domain with a lazily moved reference
-//                   maximum that the two threads agree on through shared memory once per tile,
+//                   maximum that the two threads agree on once per tile (values through shared
+//                   memory, the meeting on a hardware barrier of their two warps),
 //                   P -> bf16 -> tensor memory (over the first columns of each half of the S
 //                   buffer, from where the PV MMA takes it as its A operand); each rescales its
 //                   half of the O columns in tensor memory when the reference moved; the
 //                   epilogue writes O / l.
 // Q' carries the rotation at the row's own position and sm_scale * log2(e).
-// Every wait is bounded; a wait that runs out raises an abort flag every role checks.
+// Every mbarrier wait is bounded; a wait that runs out raises an abort flag every role checks, and a softmax warp
+// that leaves early releases its partner from the hardware barrier.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
