@@ -474,17 +474,17 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       const bool boundary = n_vis < 64;                          // only the tile(s) on the causal boundary need the mask
       // ---- pass 1: maximum of my 64 scores
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-#pragma unroll 1
-      for (int q = 0; q < 2; ++q) {
-        uint32_t sv[32];
-        TMEM_LD32(t_H + 32 * q, sv, 0);
+      {
+        uint32_t sv[64];                  // both loads in flight at once: one wait
+        TMEM_LD32(t_H, sv, 0);
+        TMEM_LD32(t_H + 32, sv, 32);
         tmem_wait_ld();
         if (boundary) {
 #pragma unroll
-          for (int c = 0; c < 32; ++c) sv[c] = (32 * q + c) < n_vis ? sv[c] : 0xff800000u;   // -inf
+          for (int c = 0; c < 64; ++c) sv[c] = c < n_vis ? sv[c] : 0xff800000u;   // -inf
         }
 #pragma unroll
-        for (int c = 0; c < 32; c += 4) {
+        for (int c = 0; c < 64; c += 4) {
 #pragma unroll
           for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(mx4[k], __uint_as_float(sv[c + k]));
         }
