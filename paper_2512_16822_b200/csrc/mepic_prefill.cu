@@ -811,6 +811,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
 }
 
+constexpr int kMaxSplits = 4;           // most shares a work item's key range is cut into
+
 // Merge of the shares of a split item: one warp per (row, q head), a lane per four head dims.
 template <int D>
 __global__ void __launch_bounds__(128) mepic_prefill_merge(const PrefillParams p, int n_q_heads) {
@@ -819,23 +821,31 @@ __global__ void __launch_bounds__(128) mepic_prefill_merge(const PrefillParams p
   const int lane = threadIdx.x & 31;
   if (pair >= n_pairs) return;
   asm volatile("griddepcontrol.wait;" ::: "memory");              // launched as a programmatic dependent of the attention kernel
-  float m_star = -INFINITY;
-  for (int s = 0; s < p.n_splits; ++s) {
-    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + (static_cast<size_t>(s) * n_pairs + pair) * 2);
-    if (ml.y > 0.f) m_star = fmaxf(m_star, ml.x);
+  // every load of the pair is issued before the first use (the share count is at most kMaxSplits)
+  float2 ml[kMaxSplits];
+  float4 x[kMaxSplits];
+#pragma unroll
+  for (int s = 0; s < kMaxSplits; ++s) {
+    ml[s] = make_float2(-INFINITY, 0.f);
+    x[s] = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (s < p.n_splits) {
+      const size_t at = static_cast<size_t>(s) * n_pairs + pair;
+      ml[s] = *reinterpret_cast<const float2*>(p.part_ml + at * 2);
+      if (lane < D / 4) x[s] = *reinterpret_cast<const float4*>(p.part_o + at * D + 4 * lane);
+    }
   }
+  float m_star = -INFINITY;
+#pragma unroll
+  for (int s = 0; s < kMaxSplits; ++s)
+    if (ml[s].y > 0.f) m_star = fmaxf(m_star, ml[s].x);
   float l_star = 0.f;
   float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (int s = 0; s < p.n_splits; ++s) {
-    const size_t at = static_cast<size_t>(s) * n_pairs + pair;
-    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + at * 2);
-    if (!(ml.y > 0.f)) continue;                     // the share held none of this row's keys
-    const float wgt = ex2(ml.x - m_star);
-    l_star += ml.y * wgt;
-    if (lane < D / 4) {
-      const float4 x = *reinterpret_cast<const float4*>(p.part_o + at * D + 4 * lane);
-      o.x += x.x * wgt; o.y += x.y * wgt; o.z += x.z * wgt; o.w += x.w * wgt;
-    }
+#pragma unroll
+  for (int s = 0; s < kMaxSplits; ++s) {
+    if (!(ml[s].y > 0.f)) continue;                  // the share held none of this row's keys (or does not exist)
+    const float wgt = ex2(ml[s].x - m_star);
+    l_star += ml[s].y * wgt;
+    o.x += x[s].x * wgt; o.y += x[s].y * wgt; o.z += x[s].z * wgt; o.w += x[s].w * wgt;
   }
   if (lane < D / 4) {
     const float inv = l_star > 0.f ? 1.f / l_star : 0.f;
@@ -892,7 +902,6 @@ bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) ==
 
 // How many CTAs share a work item: 1 when the items fill at least one wave of the GPU, else enough for about three
 // waves of shares (at most kMaxSplits).  Depends on the SM count of the current device; 1 without a device.
-constexpr int kMaxSplits = 4;
 int splits_for(int n_items) {
   int dev = 0, sms = 0;
   if (n_items <= 0 || cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
