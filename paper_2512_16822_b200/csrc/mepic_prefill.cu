@@ -774,16 +774,15 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         return w;
       };
       const bool more = j + 1 < n_tiles;
-      // ---- M-tile a
+      // ---- M-tile a.  The next K tile was rotated long ago (the rotators run ahead): its wait comes first so that
+      // nothing stands between the issue of PV_a and of QK_a(next) and the pipe's queue does not run dry.
+      if (more && !wait_k(j + 1)) { ok = false; break; }
       if (j < nt[0]) {
         if (!mbar_wait(BAR(kBarPFull, 0), static_cast<uint32_t>(j) & 1u, abort_flag, p.status) || !wait_v()) { ok = false; break; }
         tc_fence_after();
         issue_pv(0, j);
       }
-      if (more) {
-        if (!wait_k(j + 1)) { ok = false; break; }
-        if (j + 1 < nt[0]) issue_qk(0, j + 1);
-      }
+      if (more && j + 1 < nt[0]) issue_qk(0, j + 1);
       // ---- M-tile b
       if (j < nt[1]) {
         if (!mbar_wait(BAR(kBarPFull, 1), static_cast<uint32_t>(j) & 1u, abort_flag, p.status) || !wait_v()) { ok = false; break; }
