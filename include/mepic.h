@@ -403,7 +403,7 @@ int32_t mepic_attn_decode_fp8(const mepic_config_t* cfg, const mepic_decode_args
  * workspace: mepic_attn_prefill_workspace() bytes, 16-byte aligned.  Each CTA derives its share of the work on the
  * device from row_offsets; nothing is built or uploaded by the call, which only enqueues kernels.  When the work
  * items fill at least one wave of the GPU that amount is 16 bytes.  When they do not (one request, say), each item's
- * key range is cut into up to four shares, one CTA each, whose per-row partials (reference, sum, unnormalised
+ * key range is cut into up to eight shares, one CTA each, whose per-row partials (reference, sum, unnormalised
  * output: 4 (head_dim + 2) bytes per row, q head and share) go to the workspace and are merged by a third kernel;
  * given a smaller workspace the call runs one CTA per item instead.  Errors as for decode.
  * A request may have no rows (row_offsets[b] == row_offsets[b+1]).  A call with no rows at all returns MEPIC_OK

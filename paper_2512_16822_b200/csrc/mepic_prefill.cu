@@ -38,6 +38,7 @@
 #include <stdint.h>
 
 #include <algorithm>
+#include <cmath>
 
 #include "mepic.h"
 #include "mepic_internal.h"
@@ -810,7 +811,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
 }
 
-constexpr int kMaxSplits = 4;           // most shares a work item's key range is cut into
+constexpr int kMaxSplits = 8;           // most shares a work item's key range is cut into
 
 // Merge of the shares of a split item: one warp per (row, q head), a lane per four head dims.
 template <int D>
@@ -899,14 +900,19 @@ bool count_items(const mepic_config_t* cfg, int batch, const int32_t* row_offset
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-// How many CTAs share a work item: 1 when the items fill at least one wave of the GPU, else enough for about three
-// waves of shares (at most kMaxSplits).  Depends on the SM count of the current device; 1 without a device.
+// How many CTAs share a work item: 1 when the items fill at least one wave of the GPU; below that
+// round((1.2 SMs / items)^0.8), at most kMaxSplits.  The host knows the number of items but not their sizes (slots and
+// lengths are device data), so this is a fit: CTAs are handed to SMs in index order and a share costs about eight key
+// tiles of fixed work (Q staging, pipeline fill, partials); a model of exactly that reproduces the measured times of
+// seven small batches to within ten tiles, and over those and a dozen more shapes this rule is at or next to the model's
+// best uniform share count.  Depends on the SM count of the current device; 1 without a device.
 int splits_for(int n_items) {
   int dev = 0, sms = 0;
   if (n_items <= 0 || cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
     return 1;
   if (n_items >= sms) return 1;                  // a full wave or more: a share's fixed cost (Q staging, pipeline fill, partials) outweighs the balance
-  return std::max(1, std::min(kMaxSplits, (3 * sms + n_items - 1) / n_items));
+  const int s = static_cast<int>(std::lround(std::pow(1.2 * sms / n_items, 0.8)));
+  return std::max(1, std::min(kMaxSplits, s));
 }
 size_t split_workspace_bytes(const mepic_config_t* cfg, long long total_rows, int splits) {
   if (splits <= 1) return 16;
