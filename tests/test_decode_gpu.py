@@ -255,3 +255,21 @@ def test_decode_call_can_be_captured_in_a_cuda_graph_and_replayed():
             want = O.decode_attention_one(q[b], kp, vp, list(t.page_ids), list(t.pos_base), t.kv_len, int(q_pos[b]),
                                           wl.sm_scale, wl.rope_theta)
             _check(got[b], want, f"request {b}")
+
+
+def test_one_dominant_key_late_in_the_context_moves_the_reference_far():
+    # One key whose score lies ~80 nats above all others, deep inside the context: the running maximum jumps when its
+    # tile arrives (everything accumulated before is scaled to nothing) and the output is that key's V row.  The big
+    # components sit in the slowest-rotating pair (63, 127 at D = 128), so their product barely depends on the positions.
+    case = list(_manual_case(31, Hq=8, Hkv=2, D=128, P=16, kv_lens=[700, 2500], theta=1e4))
+    cfg, kp, vp, page_ids, pos_base, kv_len, q_pos, q, sm, theta = case
+    big = f32_to_bf16_bits(np.array([30.0], dtype=np.float32))[0]
+    q[:, :, 63] = big
+    star = [450, 1777]
+    for b, t in enumerate(star):
+        kp[page_ids[b, t // 16], :, t % 16, 63] = big
+    got = _run_manual(tuple(case))
+    for b, t in enumerate(star):
+        v_star = bf16_bits_to_f64(vp[page_ids[b, t // 16], :, t % 16, :])            # [Hkv, D]
+        want = np.repeat(v_star, 4, axis=0)                                          # q head h reads kv head h // 4
+        assert np.abs(bf16_bits_to_f64(got[b]) - want).max() <= 2e-2

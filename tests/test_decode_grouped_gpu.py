@@ -201,3 +201,25 @@ def test_more_than_32_requests():
     args = _shared_case(55, Hq=8, Hkv=2, D=128, P=16, n_req=n_req, chunk_pages=[7, 5, 9, 3, 4, 6], uses=uses,
                         tail_tokens=tails, jitter=False)
     _run(*args, 1.0 / np.sqrt(128), 1e4, sample=list(range(0, n_req, 7)))
+
+
+def test_one_dominant_key_inside_a_shared_chunk():
+    # A key ~80 nats above all others sits in a page three requests alias: every request's running maximum jumps when
+    # that page is reached, whatever was accumulated before scales to nothing, and the output is that key's V row.
+    # The big components sit in the slowest-rotating pair (63, 127 at D = 128): the score barely depends on positions.
+    cfg, kp, vp, page_ids, pos_base, kv_len, q_pos, q = _shared_case(
+        23, Hq=8, Hkv=2, D=128, P=16, n_req=4, chunk_pages=[20, 12], uses=[[1, 0], [0], [1, 0, 1], [1]],
+        tail_tokens=[40, 7, 100, 300], jitter=False)
+    big = f32_to_bf16_bits(np.array([30.0], dtype=np.float32))[0]
+    q[:, :, 63] = big
+    # chunk 0's shared pages follow a private page in every request that uses it; take its 10th shared page, slot 5
+    r0 = 1
+    page = page_ids[r0, 1 + 9]
+    kp[page, :, 5, 63] = big
+    dev, gb = _run(cfg, kp, vp, page_ids, pos_base, kv_len, q_pos, q, 1.0 / np.sqrt(128), 1e4)
+    got = bf16_bits_to_f64(RT.bf16_bits(gb.out))
+    v_star = np.repeat(bf16_bits_to_f64(vp[page, :, 5, :]), 4, axis=0)
+    for r in (0, 1, 2):                                   # the requests that alias chunk 0; request 3 does not
+        assert (page_ids[r] == page).any()
+        assert np.abs(got[r] - v_star).max() <= 2e-2, r
+    assert not (page_ids[3] == page).any()

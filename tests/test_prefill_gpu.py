@@ -230,3 +230,20 @@ def test_request_without_new_rows_and_call_without_any():
     torch.cuda.synchronize()
     assert dev.read_status() == 0 and M.mepic_launch_count() == before
     assert np.array_equal(RT.bf16_bits(dev.k_pool), kp) and np.array_equal(RT.bf16_bits(dev.v_pool), vp)
+
+
+def test_one_dominant_key_in_a_late_tile_rescales_everything_accumulated_before():
+    # A key ~80 nats above all others in the fourth 128-key tile: the rows' reference jumps there, O and the row sums
+    # of the first three tiles are multiplied down to nothing, later tiles leave the reference alone.  The big
+    # components sit in the slowest-rotating pair (63, 127), so the score barely depends on the positions.
+    specs = [(1000, list(range(0, 16)) + list(range(900, 1000)))]
+    cfg, kp, vp, ids, base, kvl, slots, rows = _manual(41, Hq=8, Hkv=2, D=128, P=16, specs=specs)
+    big = f32_to_bf16_bits(np.array([30.0], dtype=np.float32))[0]
+    rows[0].q_new[:, :, 63] = big
+    t = 450
+    kp[ids[0, t // 16], :, t % 16, 63] = big
+    dev, batch = _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 1.0 / np.sqrt(128), 1e4)
+    got = bf16_bits_to_f64(RT.bf16_bits(batch.out))                                  # [116, 8, 128]
+    v_star = np.repeat(bf16_bits_to_f64(vp[ids[0, t // 16], :, t % 16, :]), 4, axis=0)
+    late = got[16:]                                                                  # rows at slots 900..999 see the key
+    assert np.abs(late - v_star[None]).max() <= 2e-2
