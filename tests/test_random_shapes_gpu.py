@@ -49,3 +49,14 @@ def test_random_case(i):
         specs[0] = (specs[0][0], [0])
     pc = TP._manual(3000 + i, Hq=Hq, Hkv=Hkv, D=D, P=P, specs=specs, jitter=bool(rng.integers(0, 2)))
     TP._run_prefill(*pc, 1.0 / np.sqrt(D), 1e4)
+
+
+@pytest.mark.parametrize("i", range(8))
+def test_random_case_over_8bit_pages(i):
+    import test_decode_fp8_gpu as TF
+    TD.build_library()
+    rng = np.random.default_rng([2512, 100 + i])
+    G = int(rng.integers(1, 9)); Hkv = int(rng.integers(1, 4)); P = int(rng.choice([16, 32, 64]))
+    lens = [int(x) for x in rng.integers(1, int(rng.choice([40, 300, 2500])), size=int(rng.integers(1, 10)))]
+    args = TF._manual(500 + i, Hq=G * Hkv, Hkv=Hkv, P=P, kv_lens=lens, jitter=bool(rng.integers(0, 2)), spread=bool(rng.integers(0, 2)))
+    TF._run(*args, 1.0 / np.sqrt(128), 1e4)
