@@ -176,8 +176,8 @@ int32_t mepic_build_block_table(mepic_store_t* store, int64_t request_id,
                                 int32_t* out_recompute_slots, int32_t cap_slots, int32_t* out_n_slots);
 
 /*
- * mepic_chunk_mark_uncomputed - Section 3.3.1: "newly encountered chunks are fully recomputed, while cached
- * chunks require recomputation of only the first KV block".  A registered chunk is taken to have its shareable
+ * mepic_chunk_mark_uncomputed - Section 3.3.1: a chunk seen for the first time is recomputed whole, a cached
+ * one only in its first KV block.  A registered chunk is taken to have its shareable
  * pages filled by the caller (offline precompute, a load from a remote tier).  When that is not so - the chunk
  * is new (mepic_chunk_register reported was_resident = 0) and nobody has its K/V - mark it: the NEXT
  * mepic_build_block_table that aliases the chunk lists every slot of the chunk, shared pages included, among its
@@ -222,7 +222,7 @@ int32_t mepic_store_attach_remote(mepic_store_t* store, void* k_pool, void* v_po
 
 /* ---------------------------------------------------------------- rope table (host, set-up)
  *
- * Section 3.3.3 applies "the appropriate rotary offsets" without giving the formula; the table
+ * Section 3.3.3 has the kernel apply each block's rotary offset but gives no formula; the table
  * holds (cos, sin)(p * rope_theta^(-2i/head_dim)) for p in [0, max_position], i < head_dim/2,
  * computed in double precision and rounded to fp32.  The caller uploads it once and passes the
  * device copy to the attention calls.  mepic_rope_table_floats returns the float count
@@ -366,8 +366,11 @@ int32_t mepic_attn_decode_grouped(const mepic_config_t* cfg, const mepic_decode_
  * (page, kv head) block [num_pages][n_kv_heads], for K and for V separately.  Keys stay un-rotated.
  *
  * mepic_pages_quantize: for every page listed in pages (DEVICE int32[n_pages]) and every kv head,
- *     scale = max|x| / 448 over the block (1 if the block is all zero),
- *     code  = E4M3(x / scale), rounded to nearest, ties to even, saturating (NaN -> the NaN code),
+ *     scale = max|x| / 448 over the block's elements that are not NaN (1 if that maximum is zero: a block of
+ *             zeros, of NaN, or of both),
+ *     code  = E4M3(x / scale), rounded to nearest, ties to even, saturating; a NaN element -> the NaN code 0x7F
+ *             whatever its sign, -0 -> 0x80; an infinite element makes the scale infinite, so the block's finite
+ *             elements encode to zero and the infinite ones to the NaN code,
  * computed in fp32 from the bf16 pool src_pool (DEVICE) into dst_pool and scales (DEVICE).  Call it
  * once for the K pools and once for the V pools.  A page id outside the pool sets MEPIC_DEV_BAD_PAGE
  * in *status and that block is skipped.  Errors: E_INVAL, E_CUDA.

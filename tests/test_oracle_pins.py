@@ -560,3 +560,40 @@ def test_decode_over_value_pools_equals_decode_over_bf16_pools():
     q = f32_to_bf16_bits(rng.standard_normal((4, 64)).astype(np.float32))
     args = ([4, 1, 3, 0, 5], [0, 16, 40, 56, 72], 70, 85, 0.05, 1e4)
     assert np.array_equal(O.decode_attention_one(q, kf, vf, *args), O.decode_attention_one(q, kb, vb, *args))
+
+
+def test_quantize_pages_nan_zero_and_infinity_rules_by_hand():
+    """The codec's corner rules (the design notes' reading R24), with every expected byte worked out by hand from the
+    format's definition (1-4-3, bias 7, 448 = 0x7E, NaN = 0x7F) rather than by calling the codec:
+    a NaN element takes the NaN code and does not take part in the block's maximum; a block whose finite maximum
+    is zero (all zero, all NaN, or a mix of both) has scale 1; -0 keeps its sign bit; an infinite element makes
+    the scale infinite, after which finite elements encode to zero and the infinite ones (inf/inf) to the NaN code."""
+    def bf16(x):
+        return int(f32_to_bf16_bits(np.array([x], dtype=np.float32))[0])
+    pool = np.zeros((5, 1, 16, 64), dtype=np.uint16)
+    # block 0: largest finite |x| = 3.5 -> scale = 3.5 / 448 = 2^-7 exactly
+    row = [3.5, float("nan"), -1.75, -0.0, 2.0 ** -7, 2.0 ** -16, 2.0 ** -17, 3.0 * 2.0 ** -17, 0.4375]
+    for j, x in enumerate(row):
+        pool[0, 0, 0, j] = bf16(x)
+    pool[0, 0, 5, 9] = 0xFFC0                      # a NaN with its sign bit set
+    # x / 2^-7:          448   NaN  -224  -0    1     2^-9   2^-10 (tie -> even = 0)   3 * 2^-10 (tie -> 2 steps)   56
+    want0 = [0x7E, 0x7F, 0xF6, 0x80, 0x38, 0x01, 0x00, 0x02, 0x66]
+    pool[1, 0] = 0x7FC0                            # block 1: nothing but NaN
+    pool[2, 0, 3, 3] = 0x7FC0                      # block 2: zeros and one NaN
+    pool[3, 0, 0, 0] = bf16(float("inf")); pool[3, 0, 0, 1] = bf16(-2.0); pool[3, 0, 0, 2] = bf16(float("-inf"))
+    # block 4 stays all zero
+    codes, scale = O.quantize_pages(pool)
+    assert scale[0, 0] == np.float32(2.0 ** -7)
+    assert list(codes[0, 0, 0, :9]) == want0 and codes[0, 0, 5, 9] == 0x7F
+    rest = codes[0, 0].copy(); rest[0, :9] = 0; rest[5, 9] = 0
+    assert not rest.any()
+    assert scale[1, 0] == 1.0 and (codes[1, 0] == 0x7F).all()
+    assert scale[2, 0] == 1.0 and codes[2, 0, 3, 3] == 0x7F and np.count_nonzero(codes[2, 0]) == 1
+    assert np.isinf(scale[3, 0]) and list(codes[3, 0, 0, :3]) == [0x7F, 0x80, 0x7F] and not codes[3, 0, 1:].any()
+    assert scale[4, 0] == 1.0 and not codes[4, 0].any()
+    # the encoder alone: NaN of either sign -> 0x7F; the zeros keep their sign
+    nan_neg = np.array([0xFFC00000], dtype=np.uint32).view(np.float32)[0]
+    assert list(O.e4m3_encode(np.array([np.nan, nan_neg, 0.0, -0.0], dtype=np.float32))) == [0x7F, 0x7F, 0x00, 0x80]
+    # what the attention reads back: value(code) * scale, NaN stays NaN
+    back = O.dequantize_pages(codes, scale)
+    assert list(back[0, 0, 0, [0, 2, 4, 8]]) == [3.5, -1.75, 2.0 ** -7, 0.4375] and np.isnan(back[0, 0, 0, 1])
