@@ -220,6 +220,17 @@ int32_t mepic_store_stats(const mepic_store_t* store, mepic_stats_t* out);
 int32_t mepic_store_attach_remote(mepic_store_t* store, void* k_pool, void* v_pool, int32_t pools_on_host,
                                   int64_t capacity_pages, void* cuda_stream);
 
+/*
+ * mepic_store_test_hooks - host-side fault injection for the store's rare paths (the paper has no counterpart;
+ * no GPU is involved).  hash_mask: chunk ids are taken from (hash & hash_mask), so a mask of a few bits makes
+ * different chunks collide and exercises the probing that keeps identity by content (may only change while no
+ * chunk is resident; ~0 = normal).  fail_copies: the next fail_copies page copies to or from the remote tier
+ * report failure without copying, as a failed cudaMemcpyAsync would.  What a failed copy leaves behind: a spill
+ * that failed keeps no record of the chunk in the tier (the eviction itself stands), a fetch that failed returns
+ * the pages and registers nothing; the call that triggered it returns MEPIC_E_CUDA.  Errors: E_INVAL, E_EXISTS.
+ */
+int32_t mepic_store_test_hooks(mepic_store_t* store, uint64_t hash_mask, int32_t fail_copies);
+
 /* ---------------------------------------------------------------- rope table (host, set-up)
  *
  * Section 3.3.3 has the kernel apply each block's rotary offset but gives no formula; the table
@@ -282,8 +293,12 @@ int32_t mepic_attn_decode(const mepic_config_t* cfg, const mepic_decode_args_t* 
  * process forbids device allocation after start-up, or when the page pool has already been given
  * all the free device memory - and therefore cannot produce the workspace mepic_attn_decode asks
  * for.  Here the split-KV partials go to an array built into the library instead:
- * MEPIC_DECODE_STATIC_SCRATCH_BYTES bytes of device memory that every GPU which loads the library
- * holds from load until the process exits.
+ * MEPIC_DECODE_STATIC_SCRATCH_BYTES bytes of device memory that every GPU which uses the library's
+ * decode module holds until the process exits.  The CUDA runtime loads a module lazily by default,
+ * so the array comes into existence on a device when the first decode call of any kind
+ * (mepic_attn_decode, mepic_attn_decode_static) is made there, not when the library is loaded: a
+ * caller that is about to hand all remaining device memory to its page pool makes one such call
+ * first (a one-request warm-up will do), or that first call fails with MEPIC_E_CUDA later.
  *
  * Arguments are those of mepic_attn_decode; args->workspace and args->workspace_bytes are ignored.
  * The call allocates nothing and frees nothing, on the host's device allocator or through any

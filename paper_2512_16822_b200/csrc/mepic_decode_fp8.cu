@@ -276,6 +276,8 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
         const uint32_t a = vs_addr + key * 128 + ((ch ^ (key & 7)) << 4);
         asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
       }
+      // these generic-proxy stores must be ordered before the TMA (async proxy) write that refills this stage
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
     }
 

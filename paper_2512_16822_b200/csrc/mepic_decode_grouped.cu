@@ -299,6 +299,8 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
           const uint32_t a = vs_addr + (chk / 8) * kBlockBytes + key * 128 + (((chk % 8) ^ (key & 7)) << 4);
           asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
         }
+        // these generic-proxy stores must be ordered before the TMA (async proxy) write that refills this stage
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
       }
 

@@ -20,6 +20,7 @@
 #include <mutex>
 #include <new>
 #include <unordered_map>
+#include <unordered_set>
 #include <vector>
 
 namespace {
@@ -85,6 +86,7 @@ struct RemoteTier {
   cudaStream_t stream = nullptr;
   int64_t spilled = 0, fetched = 0;
   uint64_t tick = 0;
+  int fail_next = 0;                       // test hook: this many of the next page copies report failure
 
   ~RemoteTier() {
     if (!buf) return;
@@ -100,6 +102,7 @@ struct RemoteTier {
     }
   }
   void copy(void* dst, const void* src, bool to_tier) {
+    if (fail_next > 0) { --fail_next; failed = true; mepic_set_error("remote tier: page copy failed (injected)"); return; }
     if (host_pools) { std::memcpy(dst, src, page_bytes); return; }
     const cudaError_t e = cudaMemcpyAsync(dst, src, page_bytes, to_tier ? cudaMemcpyDeviceToHost : cudaMemcpyHostToDevice, stream);
     if (e != cudaSuccess) { failed = true; mepic_set_error("remote tier: cudaMemcpyAsync: %s", cudaGetErrorString(e)); }
@@ -132,24 +135,33 @@ struct RemoteTier {
     key = find(padded, &found);
     RemoteChunk rc;
     rc.padded = padded;
-    rc.last_use = ++tick;
     for (int32_t pg : pages) {
       const int64_t sl = free_slots.back(); free_slots.pop_back();
       rc.slots.push_back(sl);
       copy(buf + static_cast<size_t>(sl) * 2 * page_bytes, k_pool + static_cast<size_t>(pg) * page_bytes, true);
       copy(buf + static_cast<size_t>(sl) * 2 * page_bytes + page_bytes, v_pool + static_cast<size_t>(pg) * page_bytes, true);
     }
+    if (failed) {
+      // a copy could not be made: the tier must not claim K/V it does not hold.  Give the slots back (in the order
+      // they were taken, so that the next spill sees the same slots) and keep no record of the chunk.
+      for (auto it = rc.slots.rbegin(); it != rc.slots.rend(); ++it) free_slots.push_back(*it);
+      return;
+    }
+    rc.last_use = ++tick;
     chunks.emplace(key, std::move(rc));
     spilled += 1;
   }
-  void fetch(uint64_t key, const std::vector<int32_t>& pages) {
+  // false (and nothing counted) when a copy failed: the caller's pages then hold no valid K/V
+  bool fetch(uint64_t key, const std::vector<int32_t>& pages) {
     RemoteChunk& rc = chunks.at(key);
-    rc.last_use = ++tick;
     for (size_t i = 0; i < pages.size(); ++i) {
       copy(k_pool + static_cast<size_t>(pages[i]) * page_bytes, buf + static_cast<size_t>(rc.slots[i]) * 2 * page_bytes, false);
       copy(v_pool + static_cast<size_t>(pages[i]) * page_bytes, buf + static_cast<size_t>(rc.slots[i]) * 2 * page_bytes + page_bytes, false);
     }
+    if (failed) return false;
+    rc.last_use = ++tick;
     fetched += 1;
+    return true;
   }
 };
 
@@ -158,6 +170,8 @@ struct mepic_store {
   RemoteTier remote;
   std::deque<int32_t> free_pages;
   std::unordered_map<uint64_t, Chunk> chunks;          // id -> chunk; id = hash, bumped on collision
+  std::unordered_set<uint64_t> erased;                 // ids of reclaimed chunks that other ids were probed past
+  uint64_t hash_mask = ~0ull;                          // test hook: fewer hash bits, so that ids collide
   std::unordered_map<int64_t, LiveRequest> requests;
   int64_t dedup_hits = 0;
   int64_t shared_held = 0;
@@ -196,9 +210,33 @@ struct mepic_store {
       shared_held -= static_cast<int64_t>(pages.size());
       pages_evicted += static_cast<int64_t>(pages.size());
       chunks_evicted += 1;
-      chunks.erase(it);
+      forget(it);
     }
     return true;
+  }
+
+  // Ids are handed out by linear probing from the hash (a chunk whose hash is taken by other content gets the next
+  // free id), and callers hold ids, so an id can never move.  A lookup stops at the first id nobody holds; when a
+  // chunk that others were probed past goes away its id is therefore remembered as erased and lookups walk on over it.
+  // Only a chunk with a successor in its chain leaves such a mark, i.e. only after a 64-bit hash collision.
+  void forget(std::unordered_map<uint64_t, Chunk>::iterator it) {
+    const uint64_t id = it->first;
+    chunks.erase(it);
+    if (chunks.count(id + 1) || erased.count(id + 1)) erased.insert(id);
+    else for (uint64_t k = id - 1; erased.count(k); --k) erased.erase(k);      // the chain now ends earlier: marks at its end go
+  }
+  // The id of `padded` if resident (*hit set), else the id a new chunk with this content gets: the first erased id
+  // of its chain, else the chain's end.
+  uint64_t locate(const std::vector<int32_t>& padded, const Chunk** hit) {
+    *hit = nullptr;
+    uint64_t id = fnv1a64(padded) & hash_mask;
+    bool have_gap = false; uint64_t gap = 0;
+    for (;; ++id) {
+      auto it = chunks.find(id);
+      if (it != chunks.end()) { if (it->second.padded == padded) { *hit = &it->second; return id; } continue; }
+      if (erased.count(id)) { if (!have_gap) { have_gap = true; gap = id; } continue; }
+      return have_gap ? gap : id;
+    }
   }
 };
 
@@ -241,13 +279,8 @@ extern "C" int32_t mepic_chunk_register(mepic_store_t* s, const int32_t* tokens,
   const int32_t lead = (P - n_tokens % P) % P;                 // Section 3.2.1: chunks are padded at the FRONT
   std::vector<int32_t> padded(static_cast<size_t>(lead) + n_tokens, s->cfg.pad_token_id);
   std::copy(tokens, tokens + n_tokens, padded.begin() + lead);
-  uint64_t id = fnv1a64(padded);
   const Chunk* hit = nullptr;
-  for (;; ++id) {                                               // identity is by content: confirm, else probe on
-    auto it = s->chunks.find(id);
-    if (it == s->chunks.end()) break;
-    if (it->second.padded == padded) { hit = &it->second; break; }
-  }
+  uint64_t id = s->locate(padded, &hit);                        // identity is by content: hash, confirm, else probe on
   int32_t resident = 0;
   const std::vector<int32_t>* shared = nullptr;
   if (hit) {
@@ -261,8 +294,11 @@ extern "C" int32_t mepic_chunk_register(mepic_store_t* s, const int32_t* tokens,
       mepic_set_error("chunk_register: %zu shared pages needed, %zu free and not enough evictable", n_shared, s->free_pages.size());
       return MEPIC_E_NOSPACE;
     }
+    // a spill made for room could not be copied out: the evicted chunks are gone from HBM and the tier kept no
+    // record of the one that failed, so the state is consistent; report it before anything is allocated
+    if (s->remote.failed) { s->remote.failed = false; return MEPIC_E_CUDA; }
+    id = s->locate(padded, &hit);                               // the evictions may have freed an earlier id of the chain
     Chunk c;
-    s->touch(c);
     c.shared.reserve(n_shared);
     for (size_t i = 0; i < n_shared; ++i) { c.shared.push_back(s->free_pages.front()); s->free_pages.pop_front(); }
     if (s->remote.on && n_shared > 0) {
@@ -270,13 +306,22 @@ extern "C" int32_t mepic_chunk_register(mepic_store_t* s, const int32_t* tokens,
       // evictions it caused may have made the tier drop this very chunk.)
       bool found;
       const uint64_t key = s->remote.find(padded, &found);
-      if (found) { s->remote.fetch(key, c.shared); resident = 2; }
+      if (found) {
+        if (!s->remote.fetch(key, c.shared)) {
+          // the pages hold no valid K/V: hand them back where they came from and register nothing
+          for (auto it = c.shared.rbegin(); it != c.shared.rend(); ++it) s->free_pages.push_front(*it);
+          s->remote.failed = false;
+          return MEPIC_E_CUDA;
+        }
+        resident = 2;
+      }
     }
+    s->touch(c);
     c.padded = std::move(padded);
     s->shared_held += static_cast<int64_t>(n_shared);
+    s->erased.erase(id);
     shared = &s->chunks.emplace(id, std::move(c)).first->second.shared;
   }
-  if (s->remote.failed) { s->remote.failed = false; return MEPIC_E_CUDA; }
   if (out_chunk_id) *out_chunk_id = id;
   if (out_was_resident) *out_was_resident = resident;
   if (out_lead_pad) *out_lead_pad = lead;
@@ -458,6 +503,15 @@ extern "C" int32_t mepic_store_attach_remote(mepic_store_t* s, void* k_pool, voi
   r.free_slots.reserve(static_cast<size_t>(capacity_pages));
   for (int64_t i = capacity_pages - 1; i >= 0; --i) r.free_slots.push_back(i);    // slot 0 is handed out first
   r.on = true;
+  return MEPIC_OK;
+}
+
+extern "C" int32_t mepic_store_test_hooks(mepic_store_t* s, uint64_t hash_mask, int32_t fail_copies) {
+  if (!s || fail_copies < 0) { mepic_set_error("test_hooks: bad argument"); return MEPIC_E_INVAL; }
+  std::lock_guard<std::mutex> lock(s->mu);
+  if (hash_mask != s->hash_mask && !s->chunks.empty()) { mepic_set_error("test_hooks: the hash mask can only change while no chunk is resident"); return MEPIC_E_EXISTS; }
+  s->hash_mask = hash_mask;
+  s->remote.fail_next = fail_copies;
   return MEPIC_OK;
 }
 

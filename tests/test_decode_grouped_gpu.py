@@ -171,7 +171,7 @@ def test_stale_plan_sets_the_status_bit_without_faulting():
     # ... gaining a page does not: request 0 filled its last page and now needs another entry
     gb.kv_len[0] += 1
     gb.run(0.125); torch.cuda.synchronize()
-    assert dev.read_status() & 0x10
+    assert dev.read_status() & M.MEPIC_DEV_BAD_PLAN
     dev.status.zero_()
 
 
