@@ -1,23 +1,28 @@
 #!/usr/bin/env python
-"""Benchmark of the MEPIC hot path on B200: RoPE-fused paged-attention decode (HBM GB/s).
+"""Benchmark of the MEPIC hot path on B200: RoPE-fused paged-attention decode (HBM GB/s) and
+first-block-recompute prefill (TFLOP/s), on the five synthetic configurations.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config 2]
+    python bench.py --leg prefill --config 3 --scale 0.5 --steps 2 --warmup 1     # one leg alone (profiling)
 
-One "step" is one pass of the decode hot path over one batch: a call of
-``mepic_attn_decode`` (split-KV kernel + merge kernel) on the configuration the
-metric is quoted on (config 2, the Llama-3-8B-shaped decode layer).  ``value``
-is the effective bandwidth = logical K/V bytes the batch must read / device
-time, with every input already resident in HBM and the L2 flushed between
-timed steps.  ``e2e`` is the same call with the step's inputs (q and the block
-tables) coming from pinned host memory and the result read back, copies inside
-the timed region; the K/V pool is the cache itself and stays resident.
+Headline.  One "step" is one pass of the decode hot path over one batch: a call of ``mepic_attn_decode``
+(split-KV kernel + merge kernel) on the configuration the metric is quoted on (config 2, the Llama-3-8B-shaped
+decode layer).  ``value`` is the effective bandwidth = logical K/V bytes the batch must read / device time, with
+every input already resident in HBM and the L2 flushed between timed steps.  ``e2e`` is the same call with the
+step's inputs (q and the block tables) coming from pinned host memory and the result read back, copies inside the
+timed region; the K/V pool is the cache itself and stays resident.  Exactly K steps are timed for the headline; a
+second, longer run of the same step (at least half a second of device time) gives the clock sampler something to
+see and a median / minimum per step.
 
-Under torchrun every rank runs its own replica of the batch on its own GPU
-(requests are independent: no data-path collective); the aggregate is all
-ranks' bytes over the slowest rank's time.
+``configs`` holds the other configurations through the same C-ABI calls: decode on configs 1, 4 and 5 (shared and
+unshared layout, end to end, error against an oracle sample, one negative control), prefill on configs 3 and 5,
+and config 5 as one serving step (decode and prefill together).
 
-``--impl reference`` times the CPU oracle, as it stands, on the host cores
-(rank 0 only) on a bounded sample of the same workload.
+Under torchrun every rank runs its own replica of the headline batch on its own GPU (requests are independent: no
+data-path collective); the aggregate is all ranks' bytes over the slowest rank's time.
+
+``--impl reference`` times the CPU oracle, as it stands, on the host cores (rank 0 only) on a bounded sample of
+the same workload.
 """
 from __future__ import annotations
 
@@ -38,9 +43,13 @@ sys.path.insert(0, ROOT)
 from mepic_inputs import make_workload  # noqa: E402
 
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one mepic_decode_splitkv launch (ncu, see profiles/);
-# config 2: 356.9 MB read + 3.9 MB written (profiles/decode_splitkv_config2.md).
-NCU_TRAFFIC_BYTES = {2: 360_870_000}
+FALLBACK_BF16_TFLOPS = 1590.0
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_BF16_TFLOPS = 2250.0
+MAX_ABS, MEAN_ABS = 2e-2, 2e-3
+METRIC = "rope_fused_paged_decode_effective_hbm_bandwidth"
+L2_NOTE = ("flushed between timed steps (512 MiB written, then 512 MiB of another buffer read so no dirty line is "
+           "left to write back inside the timed region); value_no_flush is the same loop without it")
 
 
 def kv_bytes_per_token(wl) -> int:
@@ -54,85 +63,170 @@ def measured_peaks():
         with open(path) as f:
             d = json.load(f)
         return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)", d
-    return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)", {}
+    return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, an earlier measurement)", {}
 
 
+def ncu_traffic(kernel: str, workload: str):
+    """DRAM bytes per launch of ``kernel`` on ``workload`` from the tracked ncu summary (profiles/traffic.json),
+    with the capture it came from; None when there is no capture of that pair."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    try:
+        with open(path) as f:
+            for row in json.load(f)["captures"]:
+                if row["kernel"] == kernel and row["workload"] == workload:
+                    return row
+    except Exception:
+        pass
+    return None
+
+
+def config_dict(index: int, wl, kv_len, world: int) -> dict:
+    """The ``config`` object of the JSON line; both arms print the same keys and values."""
+    kv = np.asarray(kv_len, dtype=np.int64)
+    return {"workload": f"config{index}:{wl.name}", "batch": int(len(kv)), "n_q_heads": wl.n_q_heads,
+            "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "page_size": wl.page_size,
+            "kv_len_mean": float(kv.mean()), "logical_kv_bytes_per_step": int(kv.sum()) * kv_bytes_per_token(wl),
+            "l2": L2_NOTE, "parallelism": "replicas" if world > 1 else "single"}
+
+
+# ---------------------------------------------------------------- clocks during the timed regions
 class ClockSampler:
-    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
-              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons every few milliseconds through NVML (read-only queries) while the timed
+    regions run; falls back to polling nvidia-smi.  Only samples taken inside a marked window count."""
+    PERIOD_S = 0.002
 
     def __init__(self, gpu_index: int):
         self.gpu = gpu_index
-        self.rows = []
-        self.proc = None
+        self.rows = []              # (time, sm_mhz, sm_max_mhz, reasons bitmask or list)
+        self.windows = []
+        self._stop = threading.Event()
+        self.thread = None
+        self.how = None
+
+    def _nvml_loop(self, nv, h):
+        smax = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or nv.nvmlDeviceGetCurrentClocksThrottleReasons
+        while not self._stop.is_set():
+            try:
+                self.rows.append((time.time(), float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)), float(smax),
+                                  int(get_reasons(h))))
+            except Exception:
+                pass
+            time.sleep(self.PERIOD_S)
+
+    def _smi_loop(self):
+        fields = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+                  "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+        proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={fields}", "--format=csv,noheader,nounits",
+                                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        self._proc = proc
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in proc.stdout:
+            r = [x.strip() for x in line.split(",")]
+            try:
+                self.rows.append((time.time(), float(r[0]), float(r[1]),
+                                  [n for n, v in zip(names, r[2:6]) if v.lower().startswith("active")]))
+            except Exception:
+                continue
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
+            import pynvml as nv
+            nv.nvmlInit()
+            # the CUDA device of this rank, found in NVML by its PCI address (NVML's indices need not match CUDA's)
+            h = None
+            try:
+                import torch
+                pr = torch.cuda.get_device_properties(self.gpu)
+                h = nv.nvmlDeviceGetHandleByPciBusId(f"{pr.pci_domain_id:08X}:{pr.pci_bus_id:02X}:{pr.pci_device_id:02X}.0".encode())
+            except Exception:
+                h = None
+            if h is None:
+                h = nv.nvmlDeviceGetHandleByIndex(self.gpu)
+            nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
+            self.how = "nvml, every 2 ms"
+            self._nv = nv
+            self.thread = threading.Thread(target=self._nvml_loop, args=(nv, h), daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            pass
+        try:
+            self.how = "nvidia-smi -lms 20"
+            self.thread = threading.Thread(target=self._smi_loop, daemon=True)
             self.thread.start()
         except Exception:
-            self.proc = None
-
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+            self.how = None
 
     def wait_first_sample(self, timeout_s: float = 5.0):
         t0 = time.time()
-        while self.proc is not None and not self.rows and time.time() - t0 < timeout_s:
-            time.sleep(0.05)
+        while self.how and not self.rows and time.time() - t0 < timeout_s:
+            time.sleep(0.01)
 
-    def mark(self):
-        """Start of the region whose samples count."""
-        self.t_begin = time.time()
+    def window(self, name: str):
+        sampler = self
+
+        class _W:
+            def __enter__(self_w):
+                self_w.t0 = time.time()
+
+            def __exit__(self_w, *exc):
+                sampler.windows.append((name, self_w.t0, time.time()))
+        return _W()
 
     def stop(self) -> dict:
-        t_end = time.time()
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
-        sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ts, r in self.rows:
-            if ts < getattr(self, "t_begin", 0.0) or ts > t_end + 0.2:
-                continue
-            try:
-                sm.append(float(r[0])); smax.append(float(r[1]))
-                for name, val in zip(names, r[4:8]):
-                    if val.lower().startswith("active"):
-                        reasons.add(name)
-            except Exception:
-                continue
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        self._stop.set()
+        proc = getattr(self, "_proc", None)
+        if proc is not None:
+            proc.terminate()
+        if self.how is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no clock source available"], "samples": 0}
+        bits = {"hw_slowdown": 0x8, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40, "sw_power_cap": 0x4}
+        sm, smax, reasons, per_window = [], [], set(), {}
+        for ts, mhz, mx, rs in list(self.rows):
+            for name, t0, t1 in self.windows:
+                if t0 <= ts <= t1:
+                    sm.append(mhz); smax.append(mx)
+                    per_window[name] = per_window.get(name, 0) + 1
+                    if isinstance(rs, int):
+                        reasons.update(n for n, b in bits.items() if rs & b)
+                    else:
+                        reasons.update(rs)
+                    break
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None, "reasons": sorted(reasons), "samples": len(sm),
+                "samples_per_region": per_window, "source": self.how}
+
+
+# ---------------------------------------------------------------- the oracle legs (CPU)
+def oracle_tables(wl, requests):
+    from oracle import mepic_oracle as O
+    st = O.OracleStore(wl.page_size, wl.num_pages, wl.pad_token_id)
+    tables = []
+    for r in requests:
+        segs = [(k, st.register_chunk(wl.chunks[v])[0]) if k == O.KIND_CHUNK else (k, v) for k, v in r.segments]
+        tables.append(st.build_block_table(r.request_id, segs))
+    return tables
+
+
+def oracle_decode_one(wl, kp, vp, q, t, b, **kw):
+    from oracle import mepic_oracle as O
+    last = t.kv_len - 1
+    q_pos = t.pos_base[last // wl.page_size] + last % wl.page_size
+    return O.decode_attention_one(q[b], kp, vp, t.page_ids, t.pos_base, t.kv_len, q_pos, wl.sm_scale, wl.rope_theta, **kw)
 
 
 def oracle_decode_sample(wl, budget_s: float):
     """Time the oracle (tables + attention) on whole requests of ``wl`` until ~budget_s is spent."""
-    from oracle import mepic_oracle as O
     kp, vp = wl.kv_pool()
     q = wl.decode_q()
     t0 = time.perf_counter()
-    st = O.OracleStore(wl.page_size, wl.num_pages, wl.pad_token_id)
-    tables = []
-    for r in wl.decode_requests:
-        segs = [(k, st.register_chunk(wl.chunks[v])[0]) if k == O.KIND_CHUNK else (k, v) for k, v in r.segments]
-        tables.append(st.build_block_table(r.request_id, segs))
+    tables = oracle_tables(wl, wl.decode_requests)
     t_tables = time.perf_counter() - t0
     done, tokens, t_attn = 0, 0, 0.0
     for b, t in enumerate(tables):
         t1 = time.perf_counter()
-        O.decode_attention_one(q[b], kp, vp, t.page_ids, t.pos_base, t.kv_len, t.pos_base[(t.kv_len - 1) // wl.page_size]
-                               + (t.kv_len - 1) % wl.page_size, wl.sm_scale, wl.rope_theta)
+        oracle_decode_one(wl, kp, vp, q, t, b)
         t_attn += time.perf_counter() - t1
         done += 1; tokens += t.kv_len
         if t_attn >= budget_s:
@@ -160,47 +254,44 @@ def run_reference(args):
     # one step = one whole request of the batch through the oracle (a bounded sample of the workload)
     per_step = []
     total_tokens = 0
-    from oracle import mepic_oracle as O
     kp, vp = wl.kv_pool(); q = wl.decode_q()
-    st = O.OracleStore(wl.page_size, wl.num_pages, wl.pad_token_id)
-    tables = []
-    for r in wl.decode_requests:
-        segs = [(k, st.register_chunk(wl.chunks[v])[0]) if k == O.KIND_CHUNK else (k, v) for k, v in r.segments]
-        tables.append(st.build_block_table(r.request_id, segs))
+    tables = oracle_tables(wl, wl.decode_requests)
     for i in range(args.warmup + args.steps):
         b = i % len(tables)
-        t = tables[b]
         t1 = time.perf_counter()
-        O.decode_attention_one(q[b], kp, vp, t.page_ids, t.pos_base, t.kv_len,
-                               t.pos_base[(t.kv_len - 1) // wl.page_size] + (t.kv_len - 1) % wl.page_size,
-                               wl.sm_scale, wl.rope_theta)
+        oracle_decode_one(wl, kp, vp, q, tables[b], b)
         dt = time.perf_counter() - t1
         if i >= args.warmup:
-            per_step.append(dt); total_tokens += t.kv_len
+            per_step.append(dt); total_tokens += tables[b].kv_len
     secs = sum(per_step)
     value = total_tokens * bpt / secs / 1e9
     cores = cpu_threads()
     sample = f"{args.steps} steps, each one whole request of the batch ({tables[0].kv_len} context tokens) in fp64"
-    line = {"impl": "reference", "metric": "rope_fused_paged_decode_effective_hbm_bandwidth", "value": value, "unit": "GB/s",
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s",
             "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * secs / len(per_step),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"config{args.config}:{wl.name}", "sample": sample},
+            "config": config_dict(args.config, wl, [t.kv_len for t in tables], 1),
             "cpu_baseline": {"value": value, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------- GPU set-up shared by every leg
 class L2Flush:
     """Evicts the 126 MB L2 between timed steps: writes a 512 MiB buffer, then reads a second one.
 
     The read pass pushes the dirty lines of the write pass out to HBM before the start event, so
     their write-back is not charged to the kernel being timed."""
+    _cache = {}
 
     def __init__(self, device):
         import torch
-        self.w = torch.empty(512 << 20, dtype=torch.uint8, device=device)
-        self.r = torch.zeros(64 << 20, dtype=torch.int64, device=device)       # 512 MiB, summed without a widening copy
-        self.acc = torch.zeros((), dtype=torch.int64, device=device)
+        key = str(device)
+        if key not in L2Flush._cache:
+            L2Flush._cache[key] = (torch.empty(512 << 20, dtype=torch.uint8, device=device),
+                                   torch.zeros(64 << 20, dtype=torch.int64, device=device),   # 512 MiB, summed in place
+                                   torch.zeros((), dtype=torch.int64, device=device))
+        self.w, self.r, self.acc = L2Flush._cache[key]
 
     def __call__(self):
         import torch
@@ -208,78 +299,56 @@ class L2Flush:
         torch.sum(self.r, dim=0, out=self.acc)
 
 
-def measure_grouped(args, wl, dev, page_ids, pos_base, kv_len, q_pos, q_bits, logical_bytes: int):
-    """The same decode batch through mepic_attn_decode_grouped: requests that alias a page are scored against it
-    together.  Rate = the logical bytes a per-request decode must read / time, so it can exceed the HBM roofline."""
+def time_steps(step_fn, steps: int, flush, stream):
+    """CUDA events on the launching stream around each step; the flush runs outside the events."""
     import torch
-    from paper_2512_16822_b200 import runtime as RT
-    t0 = time.perf_counter()
-    batch = RT.GroupedDecodeBatch(dev, page_ids, pos_base, kv_len, q_pos, q_bits)
-    setup_ms = 1e3 * (time.perf_counter() - t0)
-    t0 = time.perf_counter()
-    import paper_2512_16822_b200 as M
-    M.mepic_decode_plan_build(dev.cfg, page_ids, pos_base, kv_len)
-    plan_ms = 1e3 * (time.perf_counter() - t0)
-    stream = torch.cuda.current_stream()
-    flush = L2Flush(dev.device)
-    for _ in range(3):
-        batch.run(wl.sm_scale, stream)
-    steps = max(5, min(args.steps, 50))
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     for a, b in evs:
-        flush()
-        a.record(stream); batch.run(wl.sm_scale, stream); b.record(stream)
+        if flush is not None:
+            flush()
+        a.record(stream); step_fn(); b.record(stream)
     torch.cuda.synchronize()
-    assert dev.read_status() == 0
-    ms = sum(a.elapsed_time(b) for a, b in evs) / steps
-    entries = int(sum(-(-int(k) // wl.page_size) for k in kv_len))
-    staged = int(batch.plan_host[12])
-    page_bytes = wl.page_size * kv_bytes_per_token(wl)
-    return {"value": logical_bytes / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms, "steps": steps,
-            "table_entries": entries, "pages_staged": staged, "staged_bytes_per_step": staged * page_bytes,
-            "staged_gbs": staged * page_bytes / (ms * 1e-3) / 1e9, "plan_build_ms": plan_ms, "plan_ints": int(len(batch.plan_host)),
-            "note": "sharing-aware decode (host plan + mepic_attn_decode_grouped); value = logical bytes of the per-request "
-                    "decode / time; L2 flushed between steps"}
+    return [a.elapsed_time(b) for a, b in evs]
 
 
-def measure_fp8(args, wl, dev, page_ids, pos_base, kv_len, q_pos, q_bits):
-    """The same decode batch over 8-bit (e4m3) copies of the pools (library quantiser, one scale per page and head)."""
-    import torch
-    from paper_2512_16822_b200 import runtime as RT
-    pools = RT.Fp8Pools(dev)
-    batch = RT.Fp8DecodeBatch(pools, page_ids, pos_base, kv_len, q_pos, q_bits)
-    stream = torch.cuda.current_stream()
-    flush = L2Flush(dev.device)
-    for _ in range(3):
-        batch.run(wl.sm_scale, stream)
-    steps = max(5, min(args.steps, 50))
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-    for a, b in evs:
-        flush()
-        a.record(stream); batch.run(wl.sm_scale, stream); b.record(stream)
-    torch.cuda.synchronize()
-    assert dev.read_status() == 0
-    ms = sum(a.elapsed_time(b) for a, b in evs) / steps
-    tokens = int(kv_len.astype(np.int64).sum())
-    bytes_per_token = kv_bytes_per_token(wl) // 2
-    return {"ms_per_step": ms, "steps": steps, "context_tokens_per_s": tokens / (ms * 1e-3),
-            "kv_bytes_per_token": bytes_per_token, "value": tokens * bytes_per_token / (ms * 1e-3) / 1e9, "unit": "GB/s",
-            "note": "e4m3 pages + fp32 scale per (page, kv head): half the K/V bytes of bf16 per context token; "
-                    "value = 8-bit bytes / time; L2 flushed between steps"}
+def summary(ms):
+    return {"ms_per_step": sum(ms) / len(ms), "ms_median": statistics.median(ms), "ms_min": min(ms), "steps": len(ms)}
 
 
-def measure_unshared(args, wl, device_index: int):
-    """The same decode batch on a layout WITHOUT chunk sharing: every request owns a private copy of each of its
-    chunks (one page per block-table entry), so no page is read twice and nothing can be served from L2 because a
-    neighbour touched it.  Separates kernel quality from the cache effect of sharing."""
-    import torch
+def make_config(wl, num_pages=None):
     import paper_2512_16822_b200 as M
+    return M.Config(wl.page_size, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.num_pages if num_pages is None else num_pages,
+                    wl.max_position, wl.rope_theta, wl.pad_token_id)
+
+
+def shared_layout(wl, device: str):
+    """Store -> block tables of the workload's requests; pools filled from the workload's seeded K/V."""
+    import paper_2512_16822_b200 as M
+    from paper_2512_16822_b200 import runtime as RT
+    cfg = make_config(wl)
+    t0 = time.perf_counter()
+    with M.Store(cfg) as st:
+        dec = RT.build_tables(st, wl.chunks, wl.decode_requests) if wl.decode_requests else []
+        pre = RT.build_tables(st, wl.chunks, wl.prefill_requests) if wl.prefill_requests else []
+        stats = st.stats()
+    build_ms = 1e3 * (time.perf_counter() - t0)
+    kp, vp = wl.kv_pool()
+    dev = RT.Device(cfg, kp, vp, device=device)
+    return {"cfg": cfg, "dev": dev, "decode_tables": dec, "prefill_tables": pre, "stats": stats, "table_build_ms": build_ms,
+            "kp": kp, "vp": vp}
+
+
+def unshared_layout(wl, device: str):
+    """The decode batch on a layout WITHOUT chunk sharing: every request owns a private copy of each of its chunks
+    (one page per block-table entry), so no page is read twice and nothing can be served from L2 because a
+    neighbour touched it.  Separates kernel quality from the cache effect of sharing.  Pool values are drawn on the
+    device (they do not matter for timing)."""
     from paper_2512_16822_b200 import runtime as RT
     P = wl.page_size
     ents = [sum(-(-(len(wl.chunks[v]) if k == 0 else v) // P) for k, v in r.segments) for r in wl.decode_requests]
     lens = [sum((len(wl.chunks[v]) if k == 0 else v) for k, v in r.segments) for r in wl.decode_requests]
     num_pages = int(sum(ents))
-    cfg = M.Config(P, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, num_pages, wl.max_position, wl.rope_theta, wl.pad_token_id)
+    cfg = make_config(wl, num_pages)
     B, stride = len(ents), max(ents)
     page_ids = np.zeros((B, stride), dtype=np.int32); pos_base = np.zeros((B, stride), dtype=np.int32)
     perm = np.random.default_rng([0, wl.index, 99]).permutation(num_pages).astype(np.int32)
@@ -288,73 +357,289 @@ def measure_unshared(args, wl, device_index: int):
         page_ids[b, :e] = perm[at:at + e]; at += e
         pos_base[b, :e] = np.arange(e) * P
     kv_len = np.asarray(lens, dtype=np.int32)
-    q_pos = kv_len - 1
-    dev = RT.Device(cfg, device=f"cuda:{device_index}")
-    dev.k_pool.normal_(); dev.v_pool.normal_()             # values do not matter for timing; drawn on the device
-    batch = RT.DecodeBatch(dev, page_ids, pos_base, kv_len, q_pos, wl.decode_q())
-    stream = torch.cuda.current_stream()
-    flush = L2Flush(dev.device)
-    for _ in range(3):
-        batch.run(wl.sm_scale, stream)
-    steps = max(5, min(args.steps, 50))
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-    for a, b in evs:
-        flush()
-        a.record(stream); batch.run(wl.sm_scale, stream); b.record(stream)
-    torch.cuda.synchronize()
-    assert dev.read_status() == 0
-    ms = sum(a.elapsed_time(b) for a, b in evs) / steps
-    nbytes = int(kv_len.astype(np.int64).sum()) * kv_bytes_per_token(wl)
-    return {"value": nbytes / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms, "pages_held": num_pages,
-            "note": "no chunk sharing: logical bytes = unique bytes; L2 flushed between steps"}
+    dev = RT.Device(cfg, device=device)
+    dev.k_pool.normal_(); dev.v_pool.normal_()
+    return dev, page_ids, pos_base, kv_len, (kv_len - 1).astype(np.int32)
 
 
-def measure_prefill(args, device_index: int):
-    """Config 3 (first-block recompute prefill): one step = one mepic_attn_prefill call (commit + attention)."""
-    import torch
-    import paper_2512_16822_b200 as M
+def decode_batch(kind: str, dev, page_ids, pos_base, kv_len, q_pos, q_bits):
     from paper_2512_16822_b200 import runtime as RT
-    wl = make_workload(3)
-    cfg = M.Config(wl.page_size, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.num_pages, wl.max_position,
-                   wl.rope_theta, wl.pad_token_id)
-    kp, vp = wl.kv_pool()
-    with M.Store(cfg) as st:
-        tables = RT.build_tables(st, wl.chunks, wl.prefill_requests)
+    if kind == "fp8":
+        return RT.Fp8DecodeBatch(RT.Fp8Pools(dev), page_ids, pos_base, kv_len, q_pos, q_bits)
+    if kind == "grouped":
+        return RT.GroupedDecodeBatch(dev, page_ids, pos_base, kv_len, q_pos, q_bits)
+    return RT.DecodeBatch(dev, page_ids, pos_base, kv_len, q_pos, q_bits)
+
+
+def prefill_batch(wl, dev, tables):
+    from paper_2512_16822_b200 import runtime as RT
     page_ids, pos_base, kv_len, _ = RT.pack_tables(tables, wl.page_size)
-    q_slots = [t.recompute_slots for t in tables]
-    rows = [wl.prefill_rows(i, len(t.recompute_slots)) for i, t in enumerate(tables)]
+    q_slots = [np.asarray(t.recompute_slots) for t in tables]
+    rows = [wl.prefill_rows(i, len(s)) for i, s in enumerate(q_slots)]
     row_offsets = np.concatenate([[0], np.cumsum([len(s) for s in q_slots])]).astype(np.int32)
-    dev = RT.Device(cfg, kp, vp, device=f"cuda:{device_index}")
     pb = RT.PrefillBatch(dev, page_ids, pos_base, kv_len, row_offsets, np.concatenate(q_slots).astype(np.int32),
                          np.concatenate([r.q_new for r in rows]), np.concatenate([r.k_new for r in rows]),
                          np.concatenate([r.v_new for r in rows]))
-    stream = torch.cuda.current_stream()
     # unmasked (row, key) pairs only: QK^T and PV, 2 flops per multiply-add
     pairs = sum(int((s.astype(np.int64) + 1).sum()) for s in q_slots)
     flops = 4 * wl.head_dim * wl.n_q_heads * pairs
+    return pb, flops, q_slots, rows, (page_ids, pos_base, kv_len, row_offsets)
+
+
+def rates_gbs(nbytes: int, ms: float, peak: float) -> dict:
+    g = nbytes / (ms * 1e-3) / 1e9
+    return {"value": g, "unit": "GB/s", "frac_of_measured": g / peak, "frac_of_nominal_8TBs": g / NOMINAL_HBM_GBS}
+
+
+def error_figures(got, want) -> dict:
+    d = np.abs(got - want)
+    return {"max_abs": float(d.max()), "mean_abs": float(d.mean()),
+            "rel_l2": float(np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30))}
+
+
+# ---------------------------------------------------------------- decode on one configuration
+def decode_error(wl, lay, out_bits, sample) -> dict:
+    """Measured error of the GPU result against the oracle on whole sampled requests, plus one negative control:
+    the oracle without rotation must be further from the GPU result than the tolerance allows."""
+    from mepic_inputs import bf16_bits_to_f64
+    got = bf16_bits_to_f64(out_bits)
+    q = wl.decode_q()
+    tables = oracle_tables(wl, wl.decode_requests)
+    g, w, nr = [], [], []
+    for b in sample:
+        g.append(got[b]); w.append(oracle_decode_one(wl, lay["kp"], lay["vp"], q, tables[b], b))
+        nr.append(oracle_decode_one(wl, lay["kp"], lay["vp"], q, tables[b], b, rotate=False))
+    g, w, nr = np.stack(g), np.stack(w), np.stack(nr)
+    e = error_figures(g, w)
+    neg = error_figures(g, nr)
+    e.update({"sample": f"requests {list(sample)} of {len(tables)} against the fp64 oracle, all heads and dims",
+              "within_tolerance": bool(e["max_abs"] <= MAX_ABS and e["mean_abs"] <= MEAN_ABS),
+              "negative_control": {"what": "oracle with the rotation left out", "max_abs": neg["max_abs"],
+                                   "mean_abs": neg["mean_abs"], "rel_l2": neg["rel_l2"],
+                                   "fails_tolerance": bool(neg["max_abs"] > MAX_ABS or neg["mean_abs"] > MEAN_ABS)}})
+    return e
+
+
+def decode_legs(index: int, args, device: str, peak: float, *, scale=1.0, kinds=("plain", "unshared", "e2e", "error")):
+    """Decode of one configuration through mepic_attn_decode: shared layout (flushed / not), unshared layout, end to
+    end, error figures.  Returns the per-config object."""
+    import torch
+    import paper_2512_16822_b200 as M
+    from paper_2512_16822_b200 import runtime as RT
+    wl = make_workload(index, scale=scale)
+    lay = shared_layout(wl, device)
+    dev = lay["dev"]
+    page_ids, pos_base, kv_len, q_pos = RT.pack_tables(lay["decode_tables"], wl.page_size)
+    q_bits = wl.decode_q()
+    batch = RT.DecodeBatch(dev, page_ids, pos_base, kv_len, q_pos, q_bits)
+    stream = torch.cuda.current_stream()
+    flush = L2Flush(dev.device)
+    nbytes = int(kv_len.astype(np.int64).sum()) * kv_bytes_per_token(wl)
+    steps = max(5, min(args.steps, 50))
+    step = lambda: batch.run(wl.sm_scale, stream)
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    assert dev.read_status() == 0, "device status word is not clean"
+    out = {"workload": f"config{index}:{wl.name}", "batch": len(kv_len), "kv_len_mean": float(kv_len.mean()),
+           "kv_len_max": int(kv_len.max()), "logical_kv_bytes_per_step": nbytes,
+           "pages": {"held": lay["stats"]["pages_shared_held"] + lay["stats"]["pages_private_held"],
+                     "unshared_equivalent": lay["stats"]["unshared_equivalent_pages"]},
+           "table_build_ms": lay["table_build_ms"]}
+    ms = time_steps(step, steps, flush, stream)
+    d = summary(ms); d.update(rates_gbs(nbytes, d["ms_per_step"], peak))
+    d["note"] = "shared layout: effective rate (logical bytes; repeats of shared pages may come from L2)"
+    out["decode"] = d
+    ms = time_steps(step, steps, None, stream)
+    out["decode"]["ms_per_step_no_flush"] = sum(ms) / len(ms)
+    if "e2e" in kinds:
+        h_in, hv = batch.host_mirror()
+        hv["q"].copy_(torch.from_numpy(np.ascontiguousarray(q_bits).view(np.int16)))
+        hv["page_ids"].copy_(torch.from_numpy(page_ids)); hv["pos_base"].copy_(torch.from_numpy(pos_base))
+        hv["kv_len"].copy_(torch.from_numpy(kv_len)); hv["q_pos"].copy_(torch.from_numpy(q_pos))
+        h_out = torch.empty(batch.out.shape, dtype=torch.bfloat16).pin_memory()
+
+        def e2e_step():
+            batch.upload(h_in)
+            batch.run(wl.sm_scale, stream)
+            h_out.copy_(batch.out, non_blocking=True)
+        for _ in range(3):
+            e2e_step()
+        ms = time_steps(e2e_step, steps, flush, stream)
+        d = summary(ms); d.update(rates_gbs(nbytes, d["ms_per_step"], peak))
+        d.update({"h2d_bytes_per_step": int(h_in.numel()), "d2h_bytes_per_step": int(h_out.numel() * h_out.element_size())})
+        out["e2e"] = d
+    if "error" in kinds:
+        batch.run(wl.sm_scale, stream); torch.cuda.synchronize()
+        B = len(kv_len)
+        sample = sorted({0, B // 2, B - 1}) if index != 4 else [0, B - 1]
+        out["error"] = decode_error(wl, lay, RT.bf16_bits(batch.out), sample)
+    assert dev.read_status() == 0, "device status word is not clean"
+    del batch, dev, lay
+    torch.cuda.empty_cache()
+    if "unshared" in kinds:
+        udev, uids, ubase, ukv, uqpos = unshared_layout(wl, device)
+        ub = RT.DecodeBatch(udev, uids, ubase, ukv, uqpos, q_bits)
+        ustep = lambda: ub.run(wl.sm_scale, stream)
+        for _ in range(3):
+            ustep()
+        ms = time_steps(ustep, steps, flush, stream)
+        assert udev.read_status() == 0
+        d = summary(ms); d.update(rates_gbs(nbytes, d["ms_per_step"], peak))
+        d.update({"pages_held": int(udev.cfg.num_pages),
+                  "note": "no chunk sharing: logical bytes = unique bytes, every byte comes from DRAM; L2 flushed between steps"})
+        out["unshared_layout"] = d
+        del ub, udev
+        torch.cuda.empty_cache()
+    return out
+
+
+# ---------------------------------------------------------------- prefill on one configuration
+def prefill_error(wl, lay, pb, q_slots, rows, tabs, n_rows=12) -> dict:
+    """Error of sampled rows of request 0 against the oracle, the committed pages bit for bit, and one negative
+    control (oracle with every position base zeroed)."""
+    from mepic_inputs import bf16_bits_to_f64
+    from oracle import mepic_oracle as O
+    from paper_2512_16822_b200 import runtime as RT
+    page_ids, pos_base, kv_len, row_offsets = tabs
+    R = len(q_slots[0])
+    pick = sorted(set(np.linspace(0, R - 1, n_rows).astype(int).tolist()))
+    okp, ovp = lay["kp"].copy(), lay["vp"].copy()
+    ne = -(-int(kv_len[0]) // wl.page_size)
+    args = (rows[0].q_new, rows[0].k_new, rows[0].v_new, list(q_slots[0]), okp, ovp, list(page_ids[0][:ne]))
+    want = O.prefill_attention_one(*args, list(pos_base[0][:ne]), int(kv_len[0]), wl.sm_scale, wl.rope_theta, rows=pick)
+    wrong = O.prefill_attention_one(*args, [0] * ne, int(kv_len[0]), wl.sm_scale, wl.rope_theta, rows=pick)
+    got = bf16_bits_to_f64(RT.bf16_bits(pb.out[:R]))[pick]
+    e = error_figures(got, want)
+    neg = error_figures(got, wrong)
+    touched = sorted({int(page_ids[0][s // wl.page_size]) for s in q_slots[0]})
+    kbits, vbits = RT.bf16_bits(pb.dev.k_pool[touched]), RT.bf16_bits(pb.dev.v_pool[touched])
+    e.update({"sample": f"{len(pick)} of the {R} rows of request 0 (first to last), all heads and dims, against the fp64 oracle",
+              "within_tolerance": bool(e["max_abs"] <= MAX_ABS and e["mean_abs"] <= MEAN_ABS),
+              "committed_pages_bit_exact": bool(np.array_equal(kbits, okp[touched]) and np.array_equal(vbits, ovp[touched])),
+              "negative_control": {"what": "oracle with every position base set to zero", "max_abs": neg["max_abs"],
+                                   "mean_abs": neg["mean_abs"], "rel_l2": neg["rel_l2"],
+                                   "fails_tolerance": bool(neg["max_abs"] > MAX_ABS or neg["mean_abs"] > MEAN_ABS)}})
+    return e
+
+
+def prefill_leg(index: int, args, device: str, *, scale=1.0, error=True, lay=None):
+    """One step = one mepic_attn_prefill call (commit + attention) over the configuration's prefill requests."""
+    import torch
+    wl = make_workload(index, scale=scale)
+    lay = lay or shared_layout(wl, device)
+    dev = lay["dev"]
+    pb, flops, q_slots, rows, tabs = prefill_batch(wl, dev, lay["prefill_tables"])
+    stream = torch.cuda.current_stream()
     for _ in range(3):
         pb.run(wl.sm_scale, stream)
     torch.cuda.synchronize()
     assert dev.read_status() == 0, "device status word is not clean"
     steps = max(5, min(args.steps, 20))
-    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-    for a, b in evs:
-        a.record(stream); pb.run(wl.sm_scale, stream); b.record(stream)
-    torch.cuda.synchronize()
-    ms = [a.elapsed_time(b) for a, b in evs]
-    mean_ms = sum(ms) / len(ms)
+    ms = time_steps(lambda: pb.run(wl.sm_scale, stream), steps, None, stream)
     _, _, peaks = measured_peaks()
-    peak = float(peaks.get("bf16_tflops", 1590.0))
-    achieved = flops / (mean_ms * 1e-3) / 1e12
-    return {"workload": f"config3:{wl.name}", "metric": "first_block_recompute_prefill_tflops", "value": achieved,
-            "unit": "TFLOP/s", "ms_per_step": mean_ms, "ms_min": min(ms), "steps": steps, "flops_per_step": flops,
-            "rows": int(row_offsets[-1]), "kv_len": int(kv_len[0]), "dtype": "bf16 MMA, fp32 accumulate",
-            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                         "frac": achieved / peak, "traffic": None,
-                         "peak_source": "measured burst bf16 (MEASURED_PEAKS.json bf16_tflops)" if peaks else "fallback 1590",
-                         "kernel": "mepic_prefill_attn (+ commit kernel: the C-ABI call is timed as a whole)"}}
+    burst = float(peaks.get("bf16_tflops", FALLBACK_BF16_TFLOPS))
+    sustained = float(peaks.get("bf16_tflops_sustained", 0.0)) or None
+    d = summary(ms)
+    achieved = flops / (d["ms_per_step"] * 1e-3) / 1e12
+    tr = ncu_traffic("mepic_prefill_attn", f"config{index}")
+    d.update({"workload": f"config{index}:{wl.name}", "metric": "first_block_recompute_prefill_tflops", "value": achieved,
+              "unit": "TFLOP/s", "flops_per_step": flops, "rows": int(tabs[3][-1]), "requests": len(q_slots),
+              "kv_len": int(tabs[2][0]), "dtype": "bf16 MMA, fp32 accumulate",
+              "l2": "not flushed: a step reads far more than L2 holds only through the shared pages; the bound is the tensor pipe",
+              "roofline": {"bound": "tensor", "achieved": achieved, "peak": burst, "unit": "TFLOP/s",
+                           "frac": achieved / burst, "frac_of_sustained": achieved / sustained if sustained else None,
+                           "frac_of_nominal_2250": achieved / NOMINAL_BF16_TFLOPS,
+                           "traffic": tr["dram_bytes_per_launch"] if tr else None, "traffic_source": tr,
+                           "peak_source": "measured burst bf16 (MEASURED_PEAKS.json bf16_tflops)" if peaks else "fallback 1590",
+                           "kernel": "mepic_prefill_attn (+ commit kernel: the C-ABI call is timed as a whole)"}})
+    if error:
+        d["error"] = prefill_error(wl, lay, pb, q_slots, rows, tabs)
+    return d, lay, pb
 
 
+# ---------------------------------------------------------------- the other decode paths on the headline batch
+def measure_variant(kind: str, args, wl, dev, tabs, q_bits, logical_bytes: int, peak: float):
+    """The headline batch through mepic_attn_decode_grouped ("grouped") or mepic_attn_decode_fp8 ("fp8")."""
+    import torch
+    import paper_2512_16822_b200 as M
+    page_ids, pos_base, kv_len, q_pos = tabs
+    batch = decode_batch(kind, dev, page_ids, pos_base, kv_len, q_pos, q_bits)
+    stream = torch.cuda.current_stream()
+    flush = L2Flush(dev.device)
+    for _ in range(3):
+        batch.run(wl.sm_scale, stream)
+    steps = max(5, min(args.steps, 50))
+    ms = time_steps(lambda: batch.run(wl.sm_scale, stream), steps, flush, stream)
+    assert dev.read_status() == 0
+    d = summary(ms)
+    tokens = int(kv_len.astype(np.int64).sum())
+    if kind == "grouped":
+        t0 = time.perf_counter()
+        M.mepic_decode_plan_build(dev.cfg, page_ids, pos_base, kv_len)
+        plan_ms = 1e3 * (time.perf_counter() - t0)
+        staged = int(batch.plan_host[12])
+        page_bytes = wl.page_size * kv_bytes_per_token(wl)
+        d.update({"value": logical_bytes / (d["ms_per_step"] * 1e-3) / 1e9, "unit": "GB/s",
+                  "table_entries": int(sum(-(-int(k) // wl.page_size) for k in kv_len)), "pages_staged": staged,
+                  "staged_bytes_per_step": staged * page_bytes,
+                  "staged_gbs": staged * page_bytes / (d["ms_per_step"] * 1e-3) / 1e9,
+                  "staged_frac_of_measured": staged * page_bytes / (d["ms_per_step"] * 1e-3) / 1e9 / peak,
+                  "plan_build_ms": plan_ms, "plan_ints": int(len(batch.plan_host)),
+                  "note": "sharing-aware decode (host plan + mepic_attn_decode_grouped); value = logical bytes of the "
+                          "per-request decode / time; staged = bytes the kernel actually brings on chip; L2 flushed between steps"})
+    else:
+        bpt = kv_bytes_per_token(wl) // 2
+        d.update({"context_tokens_per_s": tokens / (d["ms_per_step"] * 1e-3), "kv_bytes_per_token": bpt,
+                  "value": tokens * bpt / (d["ms_per_step"] * 1e-3) / 1e9, "unit": "GB/s",
+                  "frac_of_measured": tokens * bpt / (d["ms_per_step"] * 1e-3) / 1e9 / peak,
+                  "pages_per_GB": int(1e9 // (wl.page_size * bpt + 2 * wl.n_kv_heads * 4)),
+                  "pages_per_GB_bf16": int(1e9 // (wl.page_size * kv_bytes_per_token(wl))),
+                  "note": "e4m3 pages + fp32 scale per (page, kv head): half the K/V bytes of bf16 per context token; "
+                          "value = 8-bit bytes / time; L2 flushed between steps"})
+    del batch
+    return d
+
+
+def measure_mixed(args, device: str):
+    """Config 5 as one serving step: its decode batch and its prefill requests over one pool, each call alone and
+    both enqueued on two streams (device time from the fork to the join)."""
+    import torch
+    from paper_2512_16822_b200 import runtime as RT
+    wl = make_workload(5)
+    lay = shared_layout(wl, device)
+    dev = lay["dev"]
+    page_ids, pos_base, kv_len, q_pos = RT.pack_tables(lay["decode_tables"], wl.page_size)
+    db = RT.DecodeBatch(dev, page_ids, pos_base, kv_len, q_pos, wl.decode_q())
+    pb, flops, _, _, _ = prefill_batch(wl, dev, lay["prefill_tables"])
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    main_s = torch.cuda.current_stream()
+    flush = L2Flush(dev.device)
+
+    def both():
+        fork = torch.cuda.Event(); fork.record(main_s)
+        s1.wait_event(fork); s2.wait_event(fork)
+        pb.run(wl.sm_scale, s2)
+        db.run(wl.sm_scale, s1)
+        j1, j2 = torch.cuda.Event(), torch.cuda.Event()
+        j1.record(s1); j2.record(s2)
+        main_s.wait_event(j1); main_s.wait_event(j2)
+
+    out = {}
+    steps = max(5, min(args.steps, 10))
+    for name, fn in (("decode_alone", lambda: db.run(wl.sm_scale, main_s)), ("prefill_alone", lambda: pb.run(wl.sm_scale, main_s)),
+                     ("together_two_streams", both)):
+        for _ in range(2):
+            fn()
+        out[name] = summary(time_steps(fn, steps, flush, main_s))
+    assert dev.read_status() == 0
+    s = out["decode_alone"]["ms_median"] + out["prefill_alone"]["ms_median"]
+    out["together_over_sum"] = out["together_two_streams"]["ms_median"] / s
+    out["note"] = "medians; L2 flushed before each measurement"
+    return out
+
+
+# ---------------------------------------------------------------- multi-rank plumbing
 def max_over_ranks(total_ms: float, world: int, device) -> float:
     """The slowest rank's time: every multi-GPU number is the job's bytes over this."""
     import torch
@@ -368,6 +653,65 @@ def max_over_ranks(total_ms: float, world: int, device) -> float:
 def aggregate_gbs(world: int, steps: int, bytes_per_rank_step: int, total_ms: float) -> float:
     """Whole-job throughput: all ranks' bytes (replicas, weak scaling) over the slowest rank's time."""
     return world * steps * bytes_per_rank_step / (total_ms * 1e-3) / 1e9
+
+
+def run_leg(args):
+    """One leg alone on (possibly scaled) inputs: a short, fixed sequence of calls for a profiler to capture."""
+    import torch
+    from paper_2512_16822_b200 import runtime as RT
+    from paper_2512_16822_b200.build import build_library
+    build_library()
+    device = "cuda:0"
+    peak, _, _ = measured_peaks()
+    if args.leg == "prefill":
+        d, _, _ = prefill_leg(args.config if args.config in (3, 5) else 3, args, device, scale=args.scale, error=False)
+        print(json.dumps(d), flush=True)
+        return
+    if args.leg == "mixed":
+        print(json.dumps(measure_mixed(args, device)), flush=True)
+        return
+    wl = make_workload(args.config, scale=args.scale)
+    stream = torch.cuda.current_stream()
+    if args.leg == "unshared":
+        dev, page_ids, pos_base, kv_len, q_pos = unshared_layout(wl, device)
+        kind = "plain"
+    else:
+        lay = shared_layout(wl, device)
+        dev = lay["dev"]
+        page_ids, pos_base, kv_len, q_pos = RT.pack_tables(lay["decode_tables"], wl.page_size)
+        kind = {"decode": "plain", "graph": "plain"}.get(args.leg, args.leg)
+    if args.leg == "unshared-fp8":
+        dev, page_ids, pos_base, kv_len, q_pos = unshared_layout(wl, device)
+        kind = "fp8"
+    batch = decode_batch(kind, dev, page_ids, pos_base, kv_len, q_pos, wl.decode_q())
+    step = lambda: batch.run(wl.sm_scale, stream)
+    for _ in range(max(args.warmup, 1)):
+        step()
+    torch.cuda.synchronize()
+    nbytes = int(kv_len.astype(np.int64).sum()) * kv_bytes_per_token(wl) // (2 if kind == "fp8" else 1)
+    if args.leg == "graph":
+        side = torch.cuda.Stream()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            batch.run(wl.sm_scale, torch.cuda.current_stream())
+        res = {}
+        for name, fn in (("direct_calls_us", step), ("graph_replays_us", graph.replay)):
+            for _ in range(5):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(200):
+                fn()
+            e1.record(); torch.cuda.synchronize()
+            res[name] = e0.elapsed_time(e1) / 200 * 1e3
+        res["note"] = "per call, back to back, no L2 flush: launch latency of a tiny batch"
+        print(json.dumps(res), flush=True)
+        return
+    ms = time_steps(step, args.steps, L2Flush(dev.device), stream)
+    d = summary(ms); d.update(rates_gbs(nbytes, d["ms_per_step"], peak))
+    d.update({"leg": args.leg, "workload": f"config{args.config}:{wl.name}", "scale": args.scale, "status": dev.read_status()})
+    print(json.dumps(d), flush=True)
 
 
 def run_ours(args):
@@ -386,40 +730,27 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
     build_library()
+    device = f"cuda:{local_rank}"
 
     wl = make_workload(args.config)
-    cfg = M.Config(wl.page_size, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.num_pages, wl.max_position,
-                   wl.rope_theta, wl.pad_token_id)
-    kp, vp = wl.kv_pool()
+    lay = shared_layout(wl, device)
+    cfg, dev, tables, stats = lay["cfg"], lay["dev"], lay["decode_tables"], lay["stats"]
+    table_build_ms = lay["table_build_ms"]
     q_bits = wl.decode_q()
-    t0 = time.perf_counter()
-    with M.Store(cfg) as st:
-        tables = RT.build_tables(st, wl.chunks, wl.decode_requests)
-        stats = st.stats()
-    table_build_ms = 1e3 * (time.perf_counter() - t0)
     page_ids, pos_base, kv_len, q_pos = RT.pack_tables(tables, wl.page_size)
-    dev = RT.Device(cfg, kp, vp, device=f"cuda:{local_rank}")
     batch = RT.DecodeBatch(dev, page_ids, pos_base, kv_len, q_pos, q_bits)
     logical_bytes = int(kv_len.astype(np.int64).sum()) * kv_bytes_per_token(wl)
     stream = torch.cuda.current_stream()
     l2_flush = L2Flush(dev.device)
+    warmup = max(args.warmup, 3)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    def timed(steps, step_fn, flush):
-        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-        for a, b in evs:
-            if flush:
-                l2_flush()
-            a.record(stream); step_fn(); b.record(stream)
-        torch.cuda.synchronize()
-        return [a.elapsed_time(b) for a, b in evs]
-
     step = lambda: batch.run(wl.sm_scale, stream)
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(warmup):
         step()
     torch.cuda.synchronize()
     assert dev.read_status() == 0, "device status word is not clean"
@@ -428,16 +759,21 @@ def run_ours(args):
     if rank == 0:
         sampler.start()
         sampler.wait_first_sample()
-        sampler.mark()
     launches0 = M.mepic_launch_count()
     barrier()
-    ms = timed(args.steps, step, flush=True)
-    barrier()
+    with sampler.window("headline"):
+        ms = time_steps(step, args.steps, l2_flush, stream)
+        barrier()
     launches = M.mepic_launch_count() - launches0
-    ms_warm = timed(args.steps, step, flush=False)
+    ms_warm = time_steps(step, args.steps, None, stream)
+    # the same step, for at least half a second of device time (flushed): enough samples of the clocks, and a
+    # median / minimum that do not rest on a handful of launches
+    n_long = int(min(max(0.5 / (1e-3 * sum(ms) / len(ms)), args.steps), 4000))
+    with sampler.window("sustained"):
+        ms_long = time_steps(step, n_long, l2_flush, stream)
 
-    # end to end: the step's inputs come from pinned host memory, the result goes back to the host
-    # one pinned mirror of the step's inputs (q + block tables + lengths + positions): one copy in, one copy out
+    # end to end: one pinned mirror of the step's inputs (q + block tables + lengths + positions): one copy in,
+    # the kernels, one copy out, all inside the timed region
     h_in, hv = batch.host_mirror()
     hv["q"].copy_(torch.from_numpy(np.ascontiguousarray(q_bits).view(np.int16)))
     hv["page_ids"].copy_(torch.from_numpy(page_ids)); hv["pos_base"].copy_(torch.from_numpy(pos_base))
@@ -454,60 +790,108 @@ def run_ours(args):
     for _ in range(3):
         e2e_step()
     barrier()
-    ms_e2e = timed(args.steps, e2e_step, flush=True)
-    barrier()
-    clocks = sampler.stop() if rank == 0 else None
+    with sampler.window("e2e"):
+        ms_e2e = time_steps(e2e_step, args.steps, l2_flush, stream)
+        barrier()
     assert dev.read_status() == 0, "device status word is not clean"
 
     def agg(xs):
         return max_over_ranks(sum(xs), world, dev.device)
 
     tot, tot_warm, tot_e2e = agg(ms), agg(ms_warm), agg(ms_e2e)
-    prefill = unshared = grouped = fp8 = None
-    if rank == 0 and world == 1 and not args.no_fp8 and wl.head_dim == 128:
-        fp8 = measure_fp8(args, wl, dev, page_ids, pos_base, kv_len, q_pos, q_bits)
-    if rank == 0 and world == 1 and not args.no_grouped:
-        grouped = measure_grouped(args, wl, dev, page_ids, pos_base, kv_len, q_pos, q_bits, logical_bytes)
-    if rank == 0 and world == 1 and not args.no_prefill:
-        prefill = measure_prefill(args, local_rank)
-    if rank == 0 and world == 1 and not args.no_unshared:
-        unshared = measure_unshared(args, wl, local_rank)
+    peak, peak_src, peaks = measured_peaks()
+    extras = rank == 0 and world == 1
+    error = grouped = fp8 = unshared = None
+    configs = {}
+    tabs = (page_ids, pos_base, kv_len, q_pos)
+    if extras and not args.quick:
+        B = len(kv_len)
+        error = decode_error(wl, lay, RT.bf16_bits(batch.out), sorted({0, B // 2, B - 1}))
+        if wl.head_dim == 128:
+            with sampler.window("fp8"):
+                fp8 = measure_variant("fp8", args, wl, dev, tabs, q_bits, logical_bytes, peak)
+        with sampler.window("grouped"):
+            grouped = measure_variant("grouped", args, wl, dev, tabs, q_bits, logical_bytes, peak)
+    del batch
+    if extras:
+        # the same batch without sharing: every byte from DRAM
+        udev, uids, ubase, ukv, uqpos = unshared_layout(wl, device)
+        ub = RT.DecodeBatch(udev, uids, ubase, ukv, uqpos, q_bits)
+        for _ in range(3):
+            ub.run(wl.sm_scale, stream)
+        with sampler.window("unshared"):
+            ums = time_steps(lambda: ub.run(wl.sm_scale, stream), max(5, min(args.steps, 50)), l2_flush, stream)
+        assert udev.read_status() == 0
+        unshared = summary(ums); unshared.update(rates_gbs(logical_bytes, unshared["ms_per_step"], peak))
+        unshared.update({"pages_held": int(udev.cfg.num_pages),
+                         "note": "no chunk sharing: logical bytes = unique bytes, every byte comes from DRAM; L2 flushed between steps"})
+        del ub, udev
+        torch.cuda.empty_cache()
+    if extras and not args.quick:
+        del dev, lay
+        torch.cuda.empty_cache()
+        with sampler.window("other_configs"):
+            for idx in (1, 4, 5):
+                if idx != args.config:
+                    configs[f"config{idx}"] = decode_legs(idx, args, device, peak)
+            pre3, _, _ = prefill_leg(3, args, device)
+            configs["config3"] = {"prefill": pre3}
+            torch.cuda.empty_cache()
+            pre5, _, _ = prefill_leg(5, args, device)
+            configs.setdefault("config5", {})["prefill"] = pre5
+            torch.cuda.empty_cache()
+            configs["config5"]["serving_step"] = measure_mixed(args, device)
+    clocks = sampler.stop() if rank == 0 else None
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
     gbs = lambda total_ms: aggregate_gbs(world, args.steps, logical_bytes, total_ms)
-    peak, peak_src, _ = measured_peaks()
     per_launch_ms = sum(ms) / len(ms)
-    achieved = logical_bytes / (per_launch_ms * 1e-3) / 1e9
+    effective = logical_bytes / (per_launch_ms * 1e-3) / 1e9
+    tr = ncu_traffic("mepic_decode_splitkv", f"config{args.config}")
+    roofline = {"bound": "hbm", "peak": peak, "unit": "GB/s", "peak_source": peak_src,
+                "kernel": "mepic_decode_splitkv (+ its merge kernel: the C-ABI call is timed as a whole)",
+                "algorithmic_bytes_per_launch": logical_bytes,
+                "traffic": tr["dram_bytes_per_launch"] if tr else None, "traffic_source": tr,
+                "effective": {"achieved": effective, "frac": effective / peak, "frac_of_nominal_8TBs": effective / NOMINAL_HBM_GBS,
+                              "what": "this line's value: logical bytes / time on the shared layout; includes L2 hits on shared pages"}}
+    if unshared is not None:
+        # the DRAM-honest figure: the same kernel and the same logical bytes on the layout where no byte can come from L2
+        roofline.update({"achieved": unshared["value"], "frac": unshared["value"] / peak,
+                         "frac_of_nominal_8TBs": unshared["value"] / NOMINAL_HBM_GBS,
+                         "what": "unshared layout of the same batch (unshared_layout.ms_per_step): every byte comes from DRAM"})
+    else:
+        roofline.update({"achieved": effective, "frac": effective / peak, "frac_of_nominal_8TBs": effective / NOMINAL_HBM_GBS,
+                         "what": "shared layout (effective): the unshared-layout run is made at 1 GPU only"})
     line = {
-        "metric": "rope_fused_paged_decode_effective_hbm_bandwidth", "value": gbs(tot), "unit": "GB/s",
-        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": tot / args.steps,
+        "metric": METRIC, "value": gbs(tot), "unit": "GB/s",
+        "n_gpus": world, "steps": args.steps, "warmup": warmup, "ms_per_step": tot / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": f"config{args.config}:{wl.name}", "batch": len(tables), "n_q_heads": wl.n_q_heads,
-                   "n_kv_heads": wl.n_kv_heads, "head_dim": wl.head_dim, "page_size": wl.page_size,
-                   "kv_len_mean": float(kv_len.mean()), "logical_kv_bytes_per_step": logical_bytes,
-                   "l2": "flushed between timed steps (512 MiB written, then 512 MiB of another buffer read so no dirty "
-                         "line is left to write back inside the timed region); value_no_flush is the same loop without it",
-                   "parallelism": "replicas" if world > 1 else "single"},
+        "config": config_dict(args.config, wl, kv_len, world),
         "value_no_flush": gbs(tot_warm), "ms_per_step_no_flush": tot_warm / args.steps,
+        "sustained": dict(summary(ms_long), **rates_gbs(logical_bytes, sum(ms_long) / len(ms_long), peak)),
         "e2e": {"value": gbs(tot_e2e), "unit": "GB/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": tot_e2e / args.steps},
         "gpu_launches": int(launches),
         "clocks": clocks,
-        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": NCU_TRAFFIC_BYTES.get(args.config), "peak_source": peak_src,
-                     "kernel": "mepic_decode_splitkv (+ its merge kernel: the C-ABI call is timed as a whole)",
-                     "algorithmic_bytes_per_launch": logical_bytes, "frac_of_nominal_8TBs": achieved / 8000.0},
+        "roofline": roofline,
         "pages": {"held": stats["pages_shared_held"] + stats["pages_private_held"],
                   "shared": stats["pages_shared_held"], "private": stats["pages_private_held"],
                   "unshared_equivalent": stats["unshared_equivalent_pages"], "dedup_hits": stats["dedup_hits"]},
         "table_build_ms": table_build_ms,
-        "prefill": prefill,
+        "error": error,
+        "prefill": configs.get("config3", {}).get("prefill"),
         "unshared_layout": unshared,
         "grouped_decode": grouped,
         "fp8_decode": fp8,
+        "configs": configs,
+        "targets": {"decode": ">= 70 % of HBM bandwidth", "prefill": ">= 50 % of dense bf16 peak",
+                    "denominators": {"hbm_gbs_measured": peak, "hbm_gbs_nominal": NOMINAL_HBM_GBS,
+                                     "bf16_tflops_burst": peaks.get("bf16_tflops"),
+                                     "bf16_tflops_sustained": peaks.get("bf16_tflops_sustained"),
+                                     "bf16_tflops_nominal": NOMINAL_BF16_TFLOPS}},
     }
     if not args.no_cpu_baseline and world == 1:
         s = oracle_decode_sample(wl, args.cpu_budget)
@@ -525,20 +909,26 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 4, 5])
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5])
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-prefill", action="store_true", help="skip the config-3 prefill measurement")
-    ap.add_argument("--no-unshared", action="store_true", help="skip the decode run on the layout without sharing")
-    ap.add_argument("--no-grouped", action="store_true", help="skip the sharing-aware (grouped) decode run")
-    ap.add_argument("--no-fp8", action="store_true", help="skip the decode run over 8-bit pages")
+    ap.add_argument("--quick", action="store_true", help="headline and unshared layout only: no other configs, no variants")
+    ap.add_argument("--leg", default=None, choices=["decode", "unshared", "grouped", "fp8", "unshared-fp8", "prefill", "mixed", "graph"],
+                    help="run one leg alone (a short fixed sequence of calls, e.g. for a profiler) and print its line")
+    ap.add_argument("--scale", type=float, default=1.0, help="with --leg: shrink the configuration (1.0 = as specified)")
     args = ap.parse_args()
     if args.impl == "reference":
+        if args.config == 3:
+            raise SystemExit("--impl reference times the decode metric: --config 1, 2, 4 or 5")
         run_reference(args)
+    elif args.leg:
+        run_leg(args)
     else:
+        if args.config == 3:
+            raise SystemExit("the headline metric is a decode rate: --config 1, 2, 4 or 5 (config 3 is in `configs`)")
         run_ours(args)
 
 
