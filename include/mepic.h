@@ -231,6 +231,19 @@ int32_t mepic_store_attach_remote(mepic_store_t* store, void* k_pool, void* v_po
  */
 int32_t mepic_store_test_hooks(mepic_store_t* store, uint64_t hash_mask, int32_t fail_copies);
 
+/*
+ * mepic_kernel_test_hooks - lets a test make a kernel's bounded wait run out, in the one form that harms nothing
+ * (the paper has no counterpart).  Every wait of the kernels on an on-chip barrier polls a limited number of times
+ * and then gives up: the kernel ORs MEPIC_DEV_WAIT_EXPIRED into the status word, lets whatever it still has in
+ * flight land, releases what it holds and returns; the results of that call are undefined, the GPU and the
+ * context stay usable.  spin_limit > 0 replaces the built-in poll limit (about a second) for calls made from now
+ * on, 0 restores it.  skip_tile >= 0 makes the first worker of every such call (warp 0 of CTA 0 in the decode
+ * kernels, the K loader of CTA 0 in the prefill kernel) leave out the staged copy of its tile with that index, so
+ * that the barrier that copy would complete is a flag nothing sets and the wait on it expires; -1 restores normal
+ * operation.  Process-wide; not for production use.  Errors: E_INVAL.
+ */
+int32_t mepic_kernel_test_hooks(int32_t spin_limit, int32_t skip_tile);
+
 /* ---------------------------------------------------------------- rope table (host, set-up)
  *
  * Section 3.3.3 has the kernel apply each block's rotary offset but gives no formula; the table

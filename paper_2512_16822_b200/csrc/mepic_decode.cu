@@ -107,6 +107,7 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   int win_b = -1, win_e0 = 0, win_page = 0, win_pos = 0;           // 32 block-table entries, one per lane
   int win_qpos = 0;                                                // query position of the window's request
 
+  int issued = 0;     // tiles handed to the ring so far = index of the tile issue() is called for
   auto issue = [&](int stage) {
     const int e = pc.t >> p.log2_tpp;
     const int sub = pc.t & ((1 << p.log2_tpp) - 1);
@@ -121,7 +122,7 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
     }
     int page = __shfl_sync(kFull, win_page, e - win_e0);
     const int pos = __shfl_sync(kFull, win_pos, e - win_e0);
-    if (lane == 0) {
+    if (lane == 0 && !(w == 0 && issued == p.skip_tile)) {     // (test hook: one copy that never comes)
       if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
       const int y = (page * p.n_kv_heads + pc.h) * p.page_size + sub * kTile;     // row of the pool viewed as [rows][D]
       const uint32_t bar = smem_u32(&bars[stage]);
@@ -142,7 +143,6 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
     advance(pc, p.kv_len, p.batch, p.n_kv_heads);
   };
 
-  int issued = 0;
   for (; issued < kStages && issued < n_tiles; ++issued) issue(issued);
 
   // per-unit state: head g of the unit's G query heads (lanes with g >= G carry zeros)
@@ -192,10 +192,10 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
 
     // ---- A fragments of the query rotated by (qpos - tile base), from the table row that came with the tile
     uint32_t qa[KS][2];                         // [k-step][a0 (dims 16j+2t,+1) | a2 (dims 16j+8+2t,+1)], row = head g
-    if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity)) {
+    if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity, p.spin_limit)) {
       // Give the copies still in flight a last bounded chance to land, then leave cleanly.
       if (lane == 0) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
-      for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(&bars[s]), s == stage ? parity : (s < stage ? parity ^ 1u : parity));
+      for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(&bars[s]), s == stage ? parity : (s < stage ? parity ^ 1u : parity), p.spin_limit);
       return;
     }
     const uint32_t ks_addr = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
@@ -375,6 +375,7 @@ extern "C" int32_t mepic_attn_decode(const mepic_config_t* cfg, const mepic_deco
   p.num_pages = cfg->num_pages; p.max_position = cfg->max_position;
   p.n_workers = sms * kWarps;
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
+  p.spin_limit = mepic_test_spin_limit(kSpinLimit); p.skip_tile = mepic_test_skip_tile();
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   alignas(64) CUtensorMap map_k, map_v;
   int32_t rc = mepic_make_pool_map(cfg, a->k_pool, &map_k);

@@ -159,6 +159,7 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
   float win_ks = 1.f, win_vs = 1.f;                                // and the scales of their (page, head) blocks
   int win_qpos = 0;
 
+  int issued = 0;     // tiles handed to the ring so far = index of the tile issue() is called for
   auto issue = [&](int stage) {
     const int e = pc.t >> p.log2_tpp;
     const int sub = pc.t & ((1 << p.log2_tpp) - 1);
@@ -177,7 +178,7 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
     int page = __shfl_sync(kFull, win_page, e - win_e0);
     const int pos = __shfl_sync(kFull, win_pos, e - win_e0);
     const float ks = __shfl_sync(kFull, win_ks, e - win_e0), vs = __shfl_sync(kFull, win_vs, e - win_e0);
-    if (lane == 0) {
+    if (lane == 0 && !(w == 0 && issued == p.skip_tile)) {     // (test hook: one copy that never comes)
       if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
       const int y = (page * p.n_kv_heads + pc.h) * p.page_size + sub * kTile;     // row of the pool viewed as [rows][128 bytes]
       const uint32_t bar = smem_u32(&bars[stage]);
@@ -196,7 +197,6 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
     advance(pc, p.kv_len, p.batch, p.n_kv_heads);
   };
 
-  int issued = 0;
   for (; issued < kStages && issued < n_tiles; ++issued) issue(issued);
   __syncwarp();
 
@@ -244,9 +244,9 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
       for (int nd = 0; nd < ND; ++nd) { acc[nd][0] = 0.f; acc[nd][1] = 0.f; acc[nd][2] = 0.f; acc[nd][3] = 0.f; }
     }
 
-    if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity)) {
+    if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity, p.spin_limit)) {
       if (lane == 0) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
-      for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(&bars[s]), s == stage ? parity : (s < stage ? parity ^ 1u : parity));
+      for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(&bars[s]), s == stage ? parity : (s < stage ? parity ^ 1u : parity), p.spin_limit);
       return;
     }
     const uint32_t ks_addr = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
@@ -443,6 +443,7 @@ extern "C" int32_t mepic_attn_decode_fp8(const mepic_config_t* cfg, const mepic_
   p.num_pages = cfg->num_pages; p.max_position = cfg->max_position;
   p.n_workers = sms * kWarps;
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
+  p.spin_limit = mepic_test_spin_limit(kSpinLimit); p.skip_tile = mepic_test_skip_tile();
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   alignas(64) CUtensorMap map_k, map_v;
   int32_t rc = mepic_make_pool_map_u8(cfg, a->k_pool, &map_k);

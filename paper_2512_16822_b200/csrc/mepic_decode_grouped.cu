@@ -46,6 +46,8 @@ struct GroupedParams {
   int n_kv_heads, page_size, log2_tpp, num_pages, max_position, batch;
   int n_items, piece, total;
   int off_items, off_records, off_workers, off_req_ent, off_slot_base, off_part_off;
+  int spin_limit;   // polls before a bounded wait gives up
+  int skip_tile;    // test hook: worker 0 leaves out the staged copy of its tile with this index (-1: none)
   float scale_log2;   // sm_scale * log2(e)
 };
 
@@ -131,6 +133,7 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
 
   int win_item = -1, win_e0 = 0, win_page = 0, win_pos[R];   // 32 records of the producer's item, one per lane
 
+  int issued = 0;     // tiles handed to the ring so far = index of the tile issue() is called for
   auto issue = [&](int stage) {
     const int e = pt >> p.log2_tpp;
     const int sub = pt & ((1 << p.log2_tpp) - 1);
@@ -147,12 +150,14 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
 #pragma unroll
     for (int j = 0; j < R; ++j) pos[j] = __shfl_sync(kFull, win_pos[j], e - win_e0);
     if (lane == 0) {
+#pragma unroll
+      for (int j = 0; j < R; ++j) meta[stage * 8 + j] = pos[j] + sub * kTile;
+    }
+    if (lane == 0 && !(w == 0 && issued == p.skip_tile)) {     // (test hook: one copy that never comes)
       if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
       const int y = (page * p.n_kv_heads + ph) * p.page_size + sub * kTile;     // row of the pool viewed as [rows][D]
       const uint32_t bar = smem_u32(&bars[stage]);
       const uint32_t dst = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
-#pragma unroll
-      for (int j = 0; j < R; ++j) meta[stage * 8 + j] = pos[j] + sub * kTile;
       mbar_expect_tx(bar, kStageBytes);
 #pragma unroll
       for (int nb = 0; nb < NB; ++nb) {
@@ -166,7 +171,6 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
     }
   };
 
-  int issued = 0;
   for (; issued < kStages && issued < n_tiles; ++issued) issue(issued);
   __syncwarp();
 
@@ -283,10 +287,10 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
       if (reqA >= 0) rotate_row(qlA, qhA, angA, qposA - meta[stage * 8 + jA], reqA, hA);
       if (reqB >= 0) rotate_row(qlB, qhB, angB, qposB - meta[stage * 8 + (jB < R ? jB : 0)], reqB, hB);
     }
-    if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity)) {
+    if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity, p.spin_limit)) {
       // Give the copies still in flight a last bounded chance to land, then leave cleanly.
       if (lane == 0) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
-      for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(&bars[s]), s == stage ? parity : (s < stage ? parity ^ 1u : parity));
+      for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(&bars[s]), s == stage ? parity : (s < stage ? parity ^ 1u : parity), p.spin_limit);
       return;
     }
     if (n_valid > 0) {
@@ -512,6 +516,7 @@ extern "C" int32_t mepic_attn_decode_grouped(const mepic_config_t* cfg, const me
   p.off_items = h[kPhOffItems]; p.off_records = h[kPhOffRecords]; p.off_workers = h[kPhOffWorkers];
   p.off_req_ent = h[kPhOffReqEnt]; p.off_slot_base = h[kPhOffSlotBase]; p.off_part_off = h[kPhOffPartOff];
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
+  p.spin_limit = mepic_test_spin_limit(kSpinLimit); p.skip_tile = mepic_test_skip_tile();
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   alignas(64) CUtensorMap map_k, map_v;
   int32_t rc = mepic_make_pool_map(cfg, a->k_pool, &map_k);

@@ -28,6 +28,8 @@ struct DecodeParams {
   uint16_t* out;
   int32_t* status;
   int table_stride, batch, n_kv_heads, page_size, log2_tpp, num_pages, max_position, n_workers;
+  int spin_limit;   // polls before a bounded wait gives up
+  int skip_tile;    // test hook: worker 0 leaves out the staged copy of its tile with this index (-1: none)
   float scale_log2;   // sm_scale * log2(e)
 };
 

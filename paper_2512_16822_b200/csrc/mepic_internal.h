@@ -11,4 +11,9 @@ void mepic_count_launches(int n);
 int32_t mepic_make_pool_map(const mepic_config_t* cfg, const void* pool, void* out_map);
 int32_t mepic_make_pool_map_u8(const mepic_config_t* cfg, const void* pool, void* out_map);
 
+// Test hooks for the kernels' give-up paths (see mepic_kernel_test_hooks in mepic.h): the poll limit of every bounded
+// wait (the built-in limit when no test changed it) and the index of the one staged copy that is left out (-1: none).
+int mepic_test_spin_limit(int built_in);
+int mepic_test_skip_tile();
+
 #endif

@@ -79,6 +79,8 @@ struct PrefillParams {
   float* part_o;        // n_splits > 1: [split][row][q head][D] unnormalised O of the share
   float* part_ml;       // n_splits > 1: [split][row][q head][2] = (reference maximum in log2 units, sum)
   float scale_log2;
+  int spin_limit;       // polls before a bounded wait gives up
+  int skip_tile;        // test hook: CTA 0's K loader leaves out the copies of its key tile with this index (-1: none)
 };
 
 // packed fp32 pairs (one instruction for two lanes of work)
@@ -119,8 +121,8 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // Bounded wait that also gives up when another role has raised the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  for (int i = 0; i < kSpinLimit; ++i) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int limit) {
+  for (int i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((i & 1023) == 1023 && *abort_flag) return false;
   }
@@ -129,8 +131,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 // Same, with one verdict for the whole warp (the callers run warp-collective instructions afterwards).
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status) {
-  const bool w = mbar_wait(bar, parity, abort_flag, status);
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int limit) {
+  const bool w = mbar_wait(bar, parity, abort_flag, status, limit);
   return __all_sync(0xffffffffu, w) != 0;
 }
 // ---- tcgen05 wrappers
@@ -296,7 +298,8 @@ constexpr int kBarPFull = kBarSFull + 2;                // [2] P of the current 
 constexpr int kBarPvDone = kBarPFull + 2;               // [2] PV of the current tile complete
 constexpr int kBarVPatched = kBarPvDone + 2;            // [1] rows past kv_len of the last V tile zeroed
 constexpr int kBarQReady = kBarVPatched + 1;                // [1] Q' of both M-tiles is staged
-constexpr int kNumBars = kBarQReady + 1;
+constexpr int kBarDrain = kBarQReady + 1;                   // [1] after a lost wait: every MMA issued so far has completed
+constexpr int kNumBars = kBarDrain + 1;
 
 template <int D, int G>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -360,6 +363,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     }
     mbar_init(BAR(kBarVPatched, 0), 1);
     mbar_init(BAR(kBarQReady, 0), kSoftmaxWarps * 32);      // the softmax warps stage Q'
+    mbar_init(BAR(kBarDrain, 0), 1);                         // tcgen05.commit
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -469,7 +473,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     bool ok = true;
     const int my_tiles = nt[x];
     for (int tile = 0; tile < my_tiles; ++tile) {
-      if (!mbar_wait_warp(BAR(kBarSFull, x), static_cast<uint32_t>(tile) & 1u, abort_flag, p.status)) { ok = false; break; }
+      if (!mbar_wait_warp(BAR(kBarSFull, x), static_cast<uint32_t>(tile) & 1u, abort_flag, p.status, p.spin_limit)) { ok = false; break; }
       tc_fence_after();
       const int n_vis = limit - (tile_base + tile) * kTileN + 1 - 64 * ch;     // my columns [0, n_vis) are visible to this row
       const bool boundary = n_vis < 64;                          // only the tile(s) on the causal boundary need the mask
@@ -557,7 +561,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       // was issued after both threads handed P over).  The M-tile's Q' block is free by now: its last QK^T has completed.
       float* ep = reinterpret_cast<float*>(Qs + x * NB * kBlockBytes);
       const float l_tot = l_run + swap_with_partner(l_run, ok, ep + ch * 128 + r, ep + (ch ^ 1) * 128 + r);
-      if (ok) ok = mbar_wait_warp(BAR(kBarPvDone, x), static_cast<uint32_t>(my_tiles - 1) & 1u, abort_flag, p.status);
+      if (ok) ok = mbar_wait_warp(BAR(kBarPvDone, x), static_cast<uint32_t>(my_tiles - 1) & 1u, abort_flag, p.status, p.spin_limit);
       if (ok) {
         tc_fence_after();
         const size_t rh = static_cast<size_t>(item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g;
@@ -618,7 +622,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     for (int tile = 0; tile < n_tiles; ++tile) {
       const int st = tile % kKStages;
       const uint32_t ph = static_cast<uint32_t>(tile / kKStages) & 1u;
-      if (!mbar_wait(BAR(kBarKLanded, st), ph, abort_flag, p.status)) break;
+      if (!mbar_wait(BAR(kBarKLanded, st), ph, abort_flag, p.status, p.spin_limit)) break;
       unsigned char* Kb = Ks + st * NB * kBlockBytes;
       const int key0 = (tile_base + tile) * kTileN;
       int pos = gbase[st * 8 + k0 / 16] + (k0 & 15);
@@ -680,7 +684,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       if (tile >= depth) {
         // the stage is free once every MMA that reads its previous tenant has completed
         const uint32_t bar = BAR(is_k ? kBarKFree : kBarVFree, st);
-        if (!mbar_wait_warp(bar, static_cast<uint32_t>(tile / depth - 1) & 1u, abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait_warp(bar, static_cast<uint32_t>(tile / depth - 1) & 1u, abort_flag, p.status, p.spin_limit)) { ok = false; break; }
       }
       const int key0 = (tile_base + tile) * kTileN;
       const int gkey = key0 + lane * 16;
@@ -697,6 +701,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       const unsigned live_mask = __ballot_sync(0xffffffffu, live);
       __syncwarp();
       const uint32_t landed = BAR(is_k ? kBarKLanded : kBarVLanded, st);
+      if (is_k && blockIdx.x == 0 && tile == p.skip_tile) continue;      // (test hook: a K tile that never comes)
       if (lane == 0) mbar_expect_tx(landed, static_cast<uint32_t>(__popc(live_mask)) * kGroupBytes);
       __syncwarp();
       if (live) {
@@ -710,7 +715,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     // but 0 x NaN is NaN, so V must be finite.  Zero them once the tile has landed.
     if (!is_k && ok && last_has_tail) {
       const int lt = n_tiles - 1, st = lt % kVStages;
-      if (mbar_wait_warp(BAR(kBarVLanded, st), static_cast<uint32_t>(lt / kVStages) & 1u, abort_flag, p.status)) {
+      if (mbar_wait_warp(BAR(kBarVLanded, st), static_cast<uint32_t>(lt / kVStages) & 1u, abort_flag, p.status, p.spin_limit)) {
         unsigned char* Vb = Vs + st * NB * kBlockBytes;
         const int first = kvl - (tile_base + lt) * kTileN;       // first row to clear (0 < first < 128)
         for (int idx = first * 2 * CH + lane; idx < kTileN * 2 * CH; idx += 32) {
@@ -754,12 +759,12 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       tc_commit(BAR(kBarPvDone, x));
     };
     auto wait_k = [&](int j) {
-      const bool w = mbar_wait(BAR(kBarKReady, j % kKStages), static_cast<uint32_t>(j / kKStages) & 1u, abort_flag, p.status);
+      const bool w = mbar_wait(BAR(kBarKReady, j % kKStages), static_cast<uint32_t>(j / kKStages) & 1u, abort_flag, p.status, p.spin_limit);
       tc_fence_after();
       return w;
     };
     // prologue: S of key tile 0 for both M-tiles
-    ok = n_tiles > 0 && mbar_wait(BAR(kBarQReady, 0), 0, abort_flag, p.status) && wait_k(0);
+    ok = n_tiles > 0 && mbar_wait(BAR(kBarQReady, 0), 0, abort_flag, p.status, p.spin_limit) && wait_k(0);
     if (ok) {
       if (nt[0] > 0) issue_qk(0, 0);
       if (nt[1] > 0) issue_qk(1, 0);
@@ -769,8 +774,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       bool v_here = false;
       auto wait_v = [&]() {
         if (v_here) return true;
-        bool w = mbar_wait(BAR(kBarVLanded, j % kVStages), static_cast<uint32_t>(j / kVStages) & 1u, abort_flag, p.status);
-        if (w && j == n_tiles - 1 && last_has_tail) w = mbar_wait(BAR(kBarVPatched, 0), 0, abort_flag, p.status);
+        bool w = mbar_wait(BAR(kBarVLanded, j % kVStages), static_cast<uint32_t>(j / kVStages) & 1u, abort_flag, p.status, p.spin_limit);
+        if (w && j == n_tiles - 1 && last_has_tail) w = mbar_wait(BAR(kBarVPatched, 0), 0, abort_flag, p.status, p.spin_limit);
         v_here = w;
         return w;
       };
@@ -779,14 +784,14 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       // nothing stands between the issue of PV_a and of QK_a(next) and the pipe's queue does not run dry.
       if (more && !wait_k(j + 1)) { ok = false; break; }
       if (j < nt[0]) {
-        if (!mbar_wait(BAR(kBarPFull, 0), static_cast<uint32_t>(j) & 1u, abort_flag, p.status) || !wait_v()) { ok = false; break; }
+        if (!mbar_wait(BAR(kBarPFull, 0), static_cast<uint32_t>(j) & 1u, abort_flag, p.status, p.spin_limit) || !wait_v()) { ok = false; break; }
         tc_fence_after();
         issue_pv(0, j);
       }
       if (more && j + 1 < nt[0]) issue_qk(0, j + 1);
       // ---- M-tile b
       if (j < nt[1]) {
-        if (!mbar_wait(BAR(kBarPFull, 1), static_cast<uint32_t>(j) & 1u, abort_flag, p.status) || !wait_v()) { ok = false; break; }
+        if (!mbar_wait(BAR(kBarPFull, 1), static_cast<uint32_t>(j) & 1u, abort_flag, p.status, p.spin_limit) || !wait_v()) { ok = false; break; }
         tc_fence_after();
         issue_pv(1, j);
       }
@@ -795,6 +800,11 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         if (j + 1 < nt[1]) issue_qk(1, j + 1);
         tc_commit(BAR(kBarKFree, (j + 1) % kKStages));
       }
+    }
+    if (!ok) {
+      // a wait was lost: the MMAs issued so far still run; tensor memory may only be released once they are done
+      tc_commit(BAR(kBarDrain, 0));
+      for (int i = 0; i < p.spin_limit && !mbar_try_wait(BAR(kBarDrain, 0), 0); ++i) {}
     }
   }
 
@@ -974,6 +984,7 @@ extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_pre
   p.part_o = reinterpret_cast<float*>(static_cast<unsigned char*>(a->workspace) + 16);
   p.part_ml = p.part_o + static_cast<size_t>(p.n_splits) * total_rows * cfg->n_q_heads * cfg->head_dim;
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
+  p.spin_limit = mepic_test_spin_limit(kSpinLimit); p.skip_tile = mepic_test_skip_tile();
   const int D = cfg->head_dim, G = cfg->n_q_heads / cfg->n_kv_heads;
 #define MEPIC_PREFILL_CASE(DD, GG) if (D == DD && G == GG) return launch_prefill<DD, GG>(p, n_items, map_k, map_v, st);
   MEPIC_PREFILL_CASE(128, 1) MEPIC_PREFILL_CASE(128, 2) MEPIC_PREFILL_CASE(128, 3) MEPIC_PREFILL_CASE(128, 4) MEPIC_PREFILL_CASE(128, 5) MEPIC_PREFILL_CASE(128, 6) MEPIC_PREFILL_CASE(128, 7) MEPIC_PREFILL_CASE(128, 8)

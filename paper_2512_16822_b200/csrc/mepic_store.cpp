@@ -10,6 +10,7 @@
 #include "mepic_internal.h"
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -537,8 +538,18 @@ extern "C" int32_t mepic_rope_table_fill(const mepic_config_t* cfg, float* out) 
   return MEPIC_OK;
 }
 
+// ---------------------------------------------------------------- kernel test hooks
+static std::atomic<int> g_spin_limit{0}, g_skip_tile{-1};
+int mepic_test_spin_limit(int built_in) { const int v = g_spin_limit.load(std::memory_order_relaxed); return v > 0 ? v : built_in; }
+int mepic_test_skip_tile() { return g_skip_tile.load(std::memory_order_relaxed); }
+extern "C" int32_t mepic_kernel_test_hooks(int32_t spin_limit, int32_t skip_tile) {
+  if (spin_limit < 0 || skip_tile < -1) { mepic_set_error("kernel_test_hooks: bad argument"); return MEPIC_E_INVAL; }
+  g_spin_limit.store(spin_limit, std::memory_order_relaxed);
+  g_skip_tile.store(skip_tile, std::memory_order_relaxed);
+  return MEPIC_OK;
+}
+
 // ---------------------------------------------------------------- launch counter
-#include <atomic>
 static std::atomic<int64_t> g_launches{0};
 void mepic_count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
 extern "C" int64_t mepic_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
