@@ -364,16 +364,22 @@ def prefill_attention_one(q_new: np.ndarray, k_new: np.ndarray, v_new: np.ndarra
                           rows: Optional[Sequence[int]] = None) -> np.ndarray:
     """Selective-recompute prefill for one request (Sections 3.3.1-3.3.3).
 
-    Commits ``k_new/v_new`` (uint16 ``[R, Hkv, D]``) into the pools IN PLACE,
-    then lets every new row i attend, causally by logical slot, over slots
+    Commits ``k_new/v_new`` (uint16 ``[R, Hkv, D]``) into the pools IN PLACE
+    (bf16 pools; for float64 value pools see the comment below), then lets every new row i attend, causally by logical slot, over slots
     ``0..q_slot[i]`` of the paged context with K rotated at its position and
     the row's q rotated at the position of its own slot.  Returns fp64
     ``[R, Hq, D]`` (or only the listed ``rows``).
     """
     P = k_pool.shape[2]
-    commit_rows(k_pool, v_pool, page_ids, q_slot, k_new, v_new)
-    K = bf16_bits_to_f64(gather_pages(k_pool, page_ids, kv_len))
-    V = bf16_bits_to_f64(gather_pages(v_pool, page_ids, kv_len))
+    if k_pool.dtype == np.uint16:
+        commit_rows(k_pool, v_pool, page_ids, q_slot, k_new, v_new)
+        K = bf16_bits_to_f64(gather_pages(k_pool, page_ids, kv_len))
+        V = bf16_bits_to_f64(gather_pages(v_pool, page_ids, kv_len))
+    else:
+        # value pools (float64: de-quantised 8-bit pages).  The commit into 8-bit pages is a separate step with
+        # its own rule (commit_rows_fp8); the caller has made it and de-quantised, so the new rows are already in.
+        K = gather_pages(k_pool, page_ids, kv_len).astype(np.float64)
+        V = gather_pages(v_pool, page_ids, kv_len).astype(np.float64)
     pos = slot_positions(pos_base, kv_len, P)
     K = rope_rotate(K, pos[:, None], theta)
     sel = list(range(len(q_slot))) if rows is None else list(rows)
@@ -452,6 +458,35 @@ def quantize_pages(pool_bits: np.ndarray):
 def dequantize_pages(codes: np.ndarray, scale: np.ndarray) -> np.ndarray:
     """-> float64 pool of the values the attention reads: value(code) * scale (the product in float64)."""
     return e4m3_values()[codes] * scale.astype(np.float64)[:, :, None, None]
+
+
+def commit_rows_fp8(k_codes: np.ndarray, k_scale: np.ndarray, v_codes: np.ndarray, v_scale: np.ndarray,
+                    page_ids: Sequence[int], q_slot: Sequence[int], k_new: np.ndarray, v_new: np.ndarray) -> None:
+    """Section 3.3.2 for 8-bit pages: write the new rows (bf16 bits ``[R, Hkv, D]``) into the code pools. In place.
+
+    The paper commits recomputed K/V straight into the assigned pages and names quantisation only as something that
+    can be combined with it, so the rule for a page whose scale is a property of the whole (page, kv head) block is
+    this build's reading: pages fill from slot 0 upwards, so a call whose rows for a block include the block's slot 0
+    STARTS that block and sets its scale from the rows it writes there (largest non-NaN magnitude / 448, 1 if that is
+    zero, as for whole pages); a call whose rows for a block do not include slot 0 APPENDS to it: the block keeps its
+    scale and the new codes saturate at +-448 times that scale.  Codes are E4M3(x / scale), all in float32.
+    """
+    P = k_codes.shape[2]
+    by_page: Dict[int, List[Tuple[int, int]]] = {}
+    for i, slot in enumerate(q_slot):
+        by_page.setdefault(int(page_ids[int(slot) // P]), []).append((int(slot) % P, i))
+    for codes, scale, new in ((k_codes, k_scale, k_new), (v_codes, v_scale, v_new)):
+        x = bf16_bits_to_f64(new).astype(np.float32)                                  # [R, Hkv, D]
+        for pg, rows in by_page.items():
+            idx = [i for _, i in rows]
+            if any(s == 0 for s, _ in rows):
+                amax = np.where(np.isnan(x[idx]), np.float32(0), np.abs(x[idx])).max(axis=(0, 2))      # per kv head
+                scale[pg] = np.where(amax > 0, amax / np.float32(E4M3_MAX), np.float32(1.0)).astype(np.float32)
+            with np.errstate(invalid="ignore", over="ignore"):
+                y = (x[idx] / scale[pg][None, :, None]).astype(np.float32)
+            c = e4m3_encode(y)
+            for (s, _), ci in zip(rows, c):
+                codes[pg, :, s, :] = ci
 
 
 def merge_partials(m: np.ndarray, l: np.ndarray, o: np.ndarray) -> np.ndarray:

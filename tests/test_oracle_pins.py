@@ -599,3 +599,67 @@ def test_quantize_pages_nan_zero_and_infinity_rules_by_hand():
     with np.errstate(invalid="ignore"):
         back = O.dequantize_pages(codes, scale)
     assert list(back[0, 0, 0, [0, 2, 4, 8]]) == [3.5, -1.75, 2.0 ** -7, 0.4375] and np.isnan(back[0, 0, 0, 1])
+
+
+def test_commit_into_8bit_pages_by_hand_and_against_the_whole_page_codec():
+    """Commit rule for 8-bit pages (the design notes' reading R25), bytes worked out by hand: a call that writes a
+    block's slot 0 sets the block's scale from the rows it writes; a later call that appends keeps the scale and
+    saturates.  A commit of a whole page must equal the whole-page codec on the same values (two routes, one format)."""
+    def bf16(x):
+        return int(f32_to_bf16_bits(np.array([x], dtype=np.float32))[0])
+    P, Hkv, D = 4, 2, 8
+    kc = np.full((3, Hkv, P, D), 0x55, dtype=np.uint8); vc = kc.copy()
+    ks = np.full((3, Hkv), 7.0, dtype=np.float32); vs = ks.copy()
+    page_ids = [2, 0]                                   # logical slots 0-3 live on page 2, slots 4-7 on page 0
+    k_new = np.zeros((3, Hkv, D), dtype=np.uint16); v_new = np.zeros((3, Hkv, D), dtype=np.uint16)
+    # rows for slots 4 and 5 (page 0, in-page slots 0 and 1: the block starts here) and slot 2 (page 2, slot 2: an append)
+    k_new[0, 0, :3] = [bf16(7.0), bf16(-3.5), bf16(0.875)]      # head 0: block maximum 7 -> scale 7/448 = 2^-6
+    k_new[1, 0, 0] = bf16(1.75)
+    k_new[0, 1, 0] = bf16(float("nan"))                          # head 1 sees only NaN and zeros: scale 1
+    k_new[2, 0, :2] = [bf16(4000.0), bf16(-14.0)]                # the append: page 2 keeps scale 7
+    v_new[0, 0, 0] = bf16(448.0)                                 # V head 0: scale 1
+    O.commit_rows_fp8(kc, ks, vc, vs, page_ids, [4, 5, 2], k_new, v_new)
+    assert ks[0, 0] == np.float32(2.0 ** -6) and ks[0, 1] == 1.0 and ks[2, 0] == 7.0 and ks[1, 0] == 7.0
+    # x / 2^-6: 448 -> 0x7E ; -224 -> 0xF6 ; 56 -> 0x66 ; second row 112 = 1.75 * 2^6 -> e = 13, m = 6 -> 0x6E
+    assert list(kc[0, 0, 0, :4]) == [0x7E, 0xF6, 0x66, 0x00] and list(kc[0, 0, 1, :2]) == [0x6E, 0x00]
+    assert kc[0, 1, 0, 0] == 0x7F and not kc[0, 1, 0, 1:].any() and not kc[0, 1, 1].any()
+    assert (kc[0, :, 2:] == 0x55).all() and (kc[1] == 0x55).all()           # slots and pages not written keep their bytes
+    # the append under scale 7: 4000/7 = 571 saturates to 448 (0x7E); -14/7 = -2 -> 0xC0; other slots untouched
+    assert list(kc[2, 0, 2, :3]) == [0x7E, 0xC0, 0x00] and (kc[2, 0, [0, 1, 3]] == 0x55).all()
+    assert vs[0, 0] == 1.0 and vc[0, 0, 0, 0] == 0x7E and vs[2, 0] == 7.0
+    # a whole page through the commit = the whole-page codec
+    rng = np.random.default_rng(11)
+    page = f32_to_bf16_bits((rng.standard_normal((1, Hkv, P, D)) * 3).astype(np.float32))
+    want_c, want_s = O.quantize_pages(page)
+    c2 = np.zeros((1, Hkv, P, D), dtype=np.uint8); s2 = np.zeros((1, Hkv), dtype=np.float32)
+    rows = np.ascontiguousarray(np.transpose(page[0], (1, 0, 2)))            # [P, Hkv, D]
+    O.commit_rows_fp8(c2, s2, c2.copy(), s2.copy(), [0], [0, 1, 2, 3], rows, rows)
+    assert np.array_equal(c2, want_c) and np.array_equal(s2, want_s)
+
+
+def test_prefill_over_value_pools_equals_prefill_over_bf16_pools():
+    # values that e4m3 holds exactly with scale 1: the route through 8-bit pages and the bf16 route give the same
+    # bits, including the rows committed by the call
+    rng = np.random.default_rng(12)
+    P, Hkv, Hq, D, L = 4, 2, 4, 8, 14
+    codes = lambda shape: rng.integers(0, 0x70, size=shape).astype(np.uint8) | (rng.integers(0, 2, size=shape).astype(np.uint8) << 7)
+    kc, vc = codes((5, Hkv, P, D)), codes((5, Hkv, P, D))
+    ones = np.ones((5, Hkv), dtype=np.float32)
+    page_ids, pos_base = [3, 0, 4, 1], [0, 4, 20, 24]
+    slots = [0, 1, 2, 3, 12, 13]
+    vals = O.e4m3_values()
+    new_c = codes((len(slots), Hkv, D)); new_cv = codes((len(slots), Hkv, D))
+    k_new = f32_to_bf16_bits(vals[new_c].astype(np.float32)); v_new = f32_to_bf16_bits(vals[new_cv].astype(np.float32))
+    # keep every block's maximum at 448 so that the commit's fresh scale is exactly 1 as well
+    k_new[0, :, 0] = f32_to_bf16_bits(np.array([448.0], dtype=np.float32))[0]; v_new[0, :, 0] = k_new[0, 0, 0]
+    k_new[4, :, 0] = k_new[0, 0, 0]; v_new[4, :, 0] = k_new[0, 0, 0]
+    q_new = f32_to_bf16_bits(rng.standard_normal((len(slots), Hq, D)).astype(np.float32))
+    kb = f32_to_bf16_bits(vals[kc].astype(np.float32)); vb = f32_to_bf16_bits(vals[vc].astype(np.float32))
+    want = O.prefill_attention_one(q_new, k_new, v_new, slots, kb, vb, page_ids, pos_base, L, 0.3, 1e4)
+    ks, vs = ones.copy(), ones.copy()
+    O.commit_rows_fp8(kc, ks, vc, vs, page_ids, slots, k_new, v_new)
+    assert (ks[[3, 1]] == 1.0).all() and (vs[[3, 1]] == 1.0).all()
+    got = O.prefill_attention_one(q_new, k_new, v_new, slots, O.dequantize_pages(kc, ks), O.dequantize_pages(vc, vs),
+                                  page_ids, pos_base, L, 0.3, 1e4)
+    assert np.array_equal(got, want)
+    assert np.array_equal(O.dequantize_pages(kc, ks), bf16_bits_to_f64(kb))        # the committed pool is the same pool
