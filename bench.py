@@ -523,13 +523,27 @@ def prefill_error(wl, lay, pb, q_slots, rows, tabs, n_rows=12) -> dict:
     return e
 
 
-def prefill_leg(index: int, args, device: str, *, scale=1.0, error=True, lay=None):
-    """One step = one mepic_attn_prefill call (commit + attention) over the configuration's prefill requests."""
+def prefill_leg(index: int, args, device: str, *, scale=1.0, error=True, lay=None, fp8=False):
+    """One step = one mepic_attn_prefill call (commit + attention) over the configuration's prefill requests.
+    fp8: the same requests over 8-bit (e4m3) pools made from the workload's pool by the library's quantiser, the
+    bf16 pools freed before the run (mepic_attn_prefill_fp8: commits codes, attends over codes)."""
     import torch
+    from paper_2512_16822_b200 import runtime as RT
     wl = make_workload(index, scale=scale)
     lay = lay or shared_layout(wl, device)
     dev = lay["dev"]
     pb, flops, q_slots, rows, tabs = prefill_batch(wl, dev, lay["prefill_tables"])
+    if fp8:
+        pools = RT.Fp8Pools(dev)
+        torch.cuda.synchronize()
+        dev.k_pool = dev.v_pool = None                   # from here on the 8-bit pools are the only pools
+        torch.cuda.empty_cache()
+        pb8 = RT.Fp8PrefillBatch(pools, *tabs[:3], tabs[3], np.concatenate(q_slots).astype(np.int32),
+                                 np.concatenate([r.q_new for r in rows]), np.concatenate([r.k_new for r in rows]),
+                                 np.concatenate([r.v_new for r in rows]))
+        del pb
+        pb = pb8
+        error = False
     stream = torch.cuda.current_stream()
     for _ in range(3):
         pb.run(wl.sm_scale, stream)
@@ -553,6 +567,15 @@ def prefill_leg(index: int, args, device: str, *, scale=1.0, error=True, lay=Non
                            "traffic": tr["dram_bytes_per_launch"] if tr else None, "traffic_source": tr,
                            "peak_source": "measured burst bf16 (MEASURED_PEAKS.json bf16_tflops)" if peaks else "fallback 1590",
                            "kernel": "mepic_prefill_attn (+ commit kernel: the C-ABI call is timed as a whole)"}})
+    if fp8:
+        bpt = kv_bytes_per_token(wl) // 2
+        d.update({"metric": "first_block_recompute_prefill_tflops_8bit_pages",
+                  "pages_per_GB": int(1e9 // (wl.page_size * bpt + 2 * wl.n_kv_heads * 4)),
+                  "pages_per_GB_bf16": int(1e9 // (wl.page_size * kv_bytes_per_token(wl))),
+                  "note": "e4m3 pages + one fp32 scale per (page, kv head); no bf16 copy of the pool on the device; "
+                          "parity of this path is the GPU test suite's (tests/test_fp8_end_to_end_gpu.py)"})
+        d["roofline"]["kernel"] = "mepic_prefill_attn, 8-bit pages (+ commit kernel: the C-ABI call is timed as a whole)"
+        d["roofline"]["traffic"] = None; d["roofline"]["traffic_source"] = None
     if error:
         d["error"] = prefill_error(wl, lay, pb, q_slots, rows, tabs)
     return d, lay, pb
@@ -663,8 +686,9 @@ def run_leg(args):
     build_library()
     device = "cuda:0"
     peak, _, _ = measured_peaks()
-    if args.leg == "prefill":
-        d, _, _ = prefill_leg(args.config if args.config in (3, 5) else 3, args, device, scale=args.scale, error=False)
+    if args.leg in ("prefill", "prefill-fp8"):
+        d, _, _ = prefill_leg(args.config if args.config in (3, 5) else 3, args, device, scale=args.scale, error=False,
+                              fp8=args.leg == "prefill-fp8")
         print(json.dumps(d), flush=True)
         return
     if args.leg == "mixed":
@@ -837,6 +861,8 @@ def run_ours(args):
             pre3, _, _ = prefill_leg(3, args, device)
             configs["config3"] = {"prefill": pre3}
             torch.cuda.empty_cache()
+            configs["config3"]["prefill_8bit_pages"], _, _ = prefill_leg(3, args, device, fp8=True)
+            torch.cuda.empty_cache()
             pre5, _, _ = prefill_leg(5, args, device)
             configs.setdefault("config5", {})["prefill"] = pre5
             torch.cuda.empty_cache()
@@ -916,7 +942,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true", help="headline and unshared layout only: no other configs, no variants")
-    ap.add_argument("--leg", default=None, choices=["decode", "unshared", "grouped", "fp8", "unshared-fp8", "prefill", "mixed", "graph"],
+    ap.add_argument("--leg", default=None, choices=["decode", "unshared", "grouped", "fp8", "unshared-fp8", "prefill", "prefill-fp8", "mixed", "graph"],
                     help="run one leg alone (a short fixed sequence of calls, e.g. for a profiler) and print its line")
     ap.add_argument("--scale", type=float, default=1.0, help="with --leg: shrink the configuration (1.0 = as specified)")
     args = ap.parse_args()

@@ -465,6 +465,24 @@ typedef struct {
 size_t  mepic_attn_prefill_workspace(const mepic_config_t* cfg, int32_t batch, const int32_t* row_offsets_host);
 int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_prefill_args_t* args, void* cuda_stream);
 
+/*
+ * mepic_attn_prefill_fp8 - mepic_attn_prefill over 8-bit (e4m3) pools: Sections 3.3.1-3.3.3 with the KV-cache
+ * quantisation the paper's related-work section calls combinable.  args->k_pool / v_pool are the 8-bit pools
+ * (format above), k_scales / v_scales (DEVICE, [num_pages][n_kv_heads] fp32) their scales; both are read and
+ * WRITTEN; q_new / k_new / v_new / out stay bf16.  No bf16 copy of the pool is needed anywhere.
+ * Step 1 (commit): row i's k_new / v_new go to page page_ids[b][q_slot[i]/P], slot q_slot[i]%P as codes.  A block's
+ * scale belongs to the whole (page, kv head) block and pages fill from slot 0 upwards, so: if the call's rows for a
+ * block include the block's slot 0 the call STARTS the block and sets its scale to the largest non-NaN magnitude of
+ * the rows it writes there / 448 (1 if that is zero); otherwise it APPENDS: the block keeps its scale and the codes
+ * saturate at +-448 x scale.  code = E4M3(x / scale), to nearest even, in fp32.  (The paper commits rows as they
+ * are, Section 3.3.2; this rule is this library's.)  Step 2: the attention of mepic_attn_prefill with K_t, V_t
+ * replaced by value(code) x scale, committed rows included; same tolerance against the fp64 oracle evaluated on the
+ * same codes and scales.  head_dim must be 128.  Everything else (row grouping, workspace, splitting of small
+ * grids, errors) is as for mepic_attn_prefill.
+ */
+int32_t mepic_attn_prefill_fp8(const mepic_config_t* cfg, const mepic_prefill_args_t* args, float* k_scales, float* v_scales,
+                               void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

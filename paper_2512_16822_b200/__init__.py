@@ -27,7 +27,7 @@ __all__ = [
     "mepic_pages_quantize", "mepic_attn_decode_fp8", "mepic_decode_plan_max_ints", "mepic_decode_plan_build", "mepic_attn_decode_grouped_workspace",
     "mepic_attn_decode_grouped",
     "MEPIC_DECODE_STATIC_SCRATCH_BYTES", "mepic_attn_prefill_workspace",
-    "mepic_attn_prefill", "mepic_last_error", "mepic_launch_count",
+    "mepic_attn_prefill", "mepic_attn_prefill_fp8", "mepic_last_error", "mepic_launch_count",
     "MEPIC_OK", "MEPIC_E_INVAL", "MEPIC_E_NOSPACE", "MEPIC_E_NOTFOUND", "MEPIC_E_CAPACITY",
     "MEPIC_E_CUDA", "MEPIC_E_EXISTS", "MEPIC_SEG_CHUNK", "MEPIC_SEG_PROMPT",
 ]
@@ -153,6 +153,7 @@ _PROTOTYPES = {
     "mepic_attn_decode_grouped": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeGroupedArgsC), C.c_void_p]),
     "mepic_attn_prefill_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32, C.c_void_p]),
     "mepic_attn_prefill": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_PrefillArgsC), C.c_void_p]),
+    "mepic_attn_prefill_fp8": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_PrefillArgsC), C.c_void_p, C.c_void_p, C.c_void_p]),
 }
 
 
@@ -461,3 +462,17 @@ def mepic_attn_prefill(cfg: Config, *, q_new, k_new, v_new, row_offsets, q_slot,
                       sm_scale)
     c = cfg.c()
     _check(lib().mepic_attn_prefill(C.byref(c), C.byref(a), _stream_ptr(stream)))
+
+
+def mepic_attn_prefill_fp8(cfg: Config, *, q_new, k_new, v_new, row_offsets, q_slot, k_pool, v_pool, k_scales, v_scales,
+                           page_ids, pos_base, kv_len, rope_table, out, workspace, workspace_bytes: int, status,
+                           row_offsets_host: np.ndarray, table_stride: int, batch: int, sm_scale: float,
+                           stream=None) -> None:
+    """Prefill over 8-bit pools: k_pool / v_pool are uint8 code pools, k_scales / v_scales their fp32 scales."""
+    ro = np.ascontiguousarray(row_offsets_host, dtype=np.int32)
+    a = _PrefillArgsC(_ptr(q_new), _ptr(k_new), _ptr(v_new), _ptr(row_offsets), _ptr(q_slot), _ptr(k_pool),
+                      _ptr(v_pool), _ptr(page_ids), _ptr(pos_base), _ptr(kv_len), _ptr(rope_table), _ptr(out),
+                      _ptr(workspace), workspace_bytes, _ptr(status), ro.ctypes.data, table_stride, batch,
+                      sm_scale)
+    c = cfg.c()
+    _check(lib().mepic_attn_prefill_fp8(C.byref(c), C.byref(a), _ptr(k_scales), _ptr(v_scales), _stream_ptr(stream)))

@@ -34,11 +34,13 @@
 // Every mbarrier wait is bounded; a wait that runs out raises an abort flag every role checks, and a softmax warp
 // that leaves early releases its partner from the hardware barrier.
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
 #include <algorithm>
 #include <cmath>
+#include <cstring>
 
 #include "mepic.h"
 #include "mepic_internal.h"
@@ -79,6 +81,8 @@ struct PrefillParams {
   float* part_o;        // n_splits > 1: [split][row][q head][D] unnormalised O of the share
   float* part_ml;       // n_splits > 1: [split][row][q head][2] = (reference maximum in log2 units, sum)
   float scale_log2;
+  float* k_scales;      // 8-bit pools only: [num_pages][n_kv_heads] scale of each (page, kv head) block of K (the commit writes them)
+  float* v_scales;      // ... and of V
   int spin_limit;       // polls before a bounded wait gives up
   int skip_tile;        // test hook: CTA 0's K loader leaves out the copies of its key tile with this index (-1: none)
 };
@@ -229,6 +233,96 @@ __global__ void mepic_prefill_commit(const PrefillParams p, int chunks_per_row) 
   }
 }
 
+// The same commit into 8-bit (e4m3) pages.  A block's scale belongs to the whole (page, kv head) block and pages fill
+// from slot 0 upwards: a call whose rows for a block include its slot 0 starts the block and sets the scale from the rows
+// it writes there (largest non-NaN magnitude / 448, 1 if zero); otherwise the call appends, the block keeps its scale
+// and the codes saturate.  One CTA per new row; the first row of each run of rows that share a page does the run's work
+// (a request's slots ascend, so a page's rows are neighbours), the others leave at once.
+__device__ __forceinline__ uint32_t e4m3x4_of(float a, float b, float c, float d) {     // byte i = element i
+  uint16_t lo, hi;
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(lo) : "f"(b), "f"(a));
+  asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(hi) : "f"(d), "f"(c));
+  return static_cast<uint32_t>(lo) | (static_cast<uint32_t>(hi) << 16);
+}
+__global__ void __launch_bounds__(256) mepic_prefill_commit_fp8(const PrefillParams p, int head_dim) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int row = blockIdx.x;
+  __shared__ int sh_b;
+  __shared__ unsigned sh_amax[2][8];         // [K | V][kv head], bit patterns of non-negative floats order like integers
+  __shared__ float sh_scale[2][8];
+  if (threadIdx.x == 0) {
+    int b = 0;
+    while (b + 1 < p.batch && row >= p.row_offsets[b + 1]) ++b;
+    sh_b = b;
+  }
+  if (threadIdx.x < 16) sh_amax[threadIdx.x >> 3][threadIdx.x & 7] = 0u;
+  __syncthreads();
+  const int b = sh_b, P = p.page_size, kvl = p.kv_len[b];
+  const int slot = p.q_slot[row];
+  if (slot < 0 || slot >= kvl) { if (threadIdx.x == 0) atomicOr(p.status, MEPIC_DEV_BAD_SLOT); return; }
+  const int e = slot / P;
+  if (row > p.row_offsets[b]) {
+    const int prev = p.q_slot[row - 1];
+    if (prev >= 0 && prev < kvl && prev / P == e) return;         // not the first row of its page's run
+  }
+  const int page = p.page_ids[static_cast<size_t>(b) * p.table_stride + e];
+  if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { if (threadIdx.x == 0) atomicOr(p.status, MEPIC_DEV_BAD_PAGE); return; }
+  int n = 1;                                                      // rows of the run (at most one page's worth)
+  const int row_end = p.row_offsets[b + 1];
+  while (row + n < row_end && n < P) {
+    const int s2 = p.q_slot[row + n];
+    if (s2 < 0 || s2 >= kvl || s2 / P != e) break;
+    ++n;
+  }
+  const bool fresh = slot % P == 0;
+  const int H = p.n_kv_heads, D8 = head_dim / 8;                  // 16-byte chunks (8 bf16) per head row
+  const int chunks = n * H * D8;
+  const uint16_t* srcs[2] = {p.k_new, p.v_new};
+  unsigned char* dsts[2] = {reinterpret_cast<unsigned char*>(p.k_pool), reinterpret_cast<unsigned char*>(p.v_pool)};
+  float* scl[2] = {p.k_scales, p.v_scales};
+  if (fresh) {
+    for (int w = 0; w < 2; ++w)
+      for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+        const int r = c / (H * D8), h = (c / D8) % H;
+        const uint4 v = *reinterpret_cast<const uint4*>(srcs[w] + (static_cast<size_t>(row + r) * H + h) * head_dim + 8 * (c % D8));
+        const uint32_t ww[4] = {v.x, v.y, v.z, v.w};
+        float amax = 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float2 f = bf16x2_to_float2(ww[k]);
+          amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y)));       // fmaxf drops NaN operands: a NaN element does not set the scale
+        }
+        atomicMax(&sh_amax[w][h], __float_as_uint(amax));
+      }
+  }
+  __syncthreads();
+  if (threadIdx.x < 2 * H) {
+    const int w = threadIdx.x / H, h = threadIdx.x % H;
+    float sc;
+    if (fresh) {
+      const float amax = __uint_as_float(sh_amax[w][h]);
+      sc = amax > 0.f ? __fdiv_rn(amax, 448.f) : 1.f;
+      scl[w][static_cast<size_t>(page) * H + h] = sc;
+    } else {
+      sc = scl[w][static_cast<size_t>(page) * H + h];
+    }
+    sh_scale[w][h] = sc;
+  }
+  __syncthreads();
+  for (int w = 0; w < 2; ++w)
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+      const int r = c / (H * D8), h = (c / D8) % H, cc = c % D8;
+      const uint4 v = *reinterpret_cast<const uint4*>(srcs[w] + (static_cast<size_t>(row + r) * H + h) * head_dim + 8 * cc);
+      const float sc = sh_scale[w][h];
+      const float2 f0 = bf16x2_to_float2(v.x), f1 = bf16x2_to_float2(v.y), f2 = bf16x2_to_float2(v.z), f3 = bf16x2_to_float2(v.w);
+      uint2 out;
+      out.x = e4m3x4_of(__fdiv_rn(f0.x, sc), __fdiv_rn(f0.y, sc), __fdiv_rn(f1.x, sc), __fdiv_rn(f1.y, sc));
+      out.y = e4m3x4_of(__fdiv_rn(f2.x, sc), __fdiv_rn(f2.y, sc), __fdiv_rn(f3.x, sc), __fdiv_rn(f3.y, sc));
+      const int in_page = p.q_slot[row + r] % P;
+      *reinterpret_cast<uint2*>(dsts[w] + ((static_cast<size_t>(page) * H + h) * P + in_page) * head_dim + 8 * cc) = out;
+    }
+}
+
 // The work item of CTA `i`, derived on the device from row_offsets alone (no list to build or upload).  Items are
 // ordered heaviest first: level t = index of the tile of query positions inside its request, highest level first
 // (later tiles see more keys); inside a level by request, then kv head.  Executed by one full warp.
@@ -299,9 +393,15 @@ constexpr int kBarPvDone = kBarPFull + 2;               // [2] PV of the current
 constexpr int kBarVPatched = kBarPvDone + 2;            // [1] rows past kv_len of the last V tile zeroed
 constexpr int kBarQReady = kBarVPatched + 1;                // [1] Q' of both M-tiles is staged
 constexpr int kBarDrain = kBarQReady + 1;                   // [1] after a lost wait: every MMA issued so far has completed
-constexpr int kNumBars = kBarDrain + 1;
+constexpr int kBarVReady = kBarDrain + 1;                   // [kVStages] 8-bit pages only: the V stage has been widened to bf16
+constexpr int kNumBars = kBarVReady + kVStages;
 
-template <int D, int G>
+// FP8 = the pools hold e4m3 codes with one scale per (page, kv head) block: no TMA then (the tensor cores need bf16
+// operands in the swizzled layout, and shared memory has no room for a second, 8-bit copy of the rings): the loader warps
+// only publish where each 16-key group of the tile lives, and the rotator warps fetch the codes from global memory
+// themselves, widen them exactly, fold the block's scale into the rotation constants (K) or the widening (V) and write
+// the bf16 stage the MMA reads.  Everything downstream of the stages is unchanged.
+template <int D, int G, bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
   using L = PrefillSmem<D>;
@@ -325,6 +425,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kNumBars + 1);
   volatile int* gbase = reinterpret_cast<volatile int*>(bars + kNumBars + 2);   // [kKStages][8] position of each 16-key group's first key
+  volatile int* krow = reinterpret_cast<volatile int*>(bars + kNumBars + 18);   // 8-bit pages: [kKStages][8] pool row of each group's first key (-1: no such keys)
+  volatile int* vrow = reinterpret_cast<volatile int*>(bars + kNumBars + 30);   // ... and [kVStages][8] for the V stages
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   Item* item_slot = reinterpret_cast<Item*>(bars + kNumBars + 16);
@@ -364,6 +466,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     mbar_init(BAR(kBarVPatched, 0), 1);
     mbar_init(BAR(kBarQReady, 0), kSoftmaxWarps * 32);      // the softmax warps stage Q'
     mbar_init(BAR(kBarDrain, 0), 1);                         // tcgen05.commit
+    for (int s = 0; s < kVStages; ++s) mbar_init(BAR(kBarVReady, s), kRotatorWarps * 32);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
@@ -619,6 +722,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       }
     }
     const int lc = c, hc = CH + c;
+    if (FP8) asm volatile("griddepcontrol.wait;" ::: "memory");   // this role reads the pools itself: after the commit kernel
     for (int tile = 0; tile < n_tiles; ++tile) {
       const int st = tile % kKStages;
       const uint32_t ph = static_cast<uint32_t>(tile / kKStages) & 1u;
@@ -638,6 +742,87 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
           const float4 t = __ldg(row + j);
           cc[j] = make_float2(t.x, t.z); ss[j] = make_float2(t.y, t.w);
         }
+      }
+      if constexpr (FP8) {
+        // ---- 8-bit pages: codes from global memory, widened exactly, rotated in fp32 with the block's scale folded
+        // into (cos, sin) (the one-position step is a pure rotation, so the factor rides along), rounded to bf16 once
+        const int r0 = krow[st * 8 + k0 / 16];
+        const bool have = r0 >= 0;
+        const unsigned char* src0 = reinterpret_cast<const unsigned char*>(p.k_pool) + static_cast<size_t>(have ? r0 + (k0 & 15) : 0) * D;
+        if (have) {
+          const float sc = __ldg(p.k_scales + r0 / p.page_size);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) { cc[j].x *= sc; cc[j].y *= sc; ss[j].x *= sc; ss[j].y *= sc; }
+        }
+#pragma unroll 1
+        for (int i0 = 0; i0 < CH; i0 += 4) {
+          uint2 lo8[4], hi8[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            lo8[u] = have ? __ldg(reinterpret_cast<const uint2*>(src0 + static_cast<size_t>(i0 + u) * D + 8 * c)) : make_uint2(0, 0);
+            hi8[u] = have ? __ldg(reinterpret_cast<const uint2*>(src0 + static_cast<size_t>(i0 + u) * D + D / 2 + 8 * c)) : make_uint2(0, 0);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int kk = k0 + i0 + u;
+            const uint32_t lw[2] = {lo8[u].x, lo8[u].y}, hw[2] = {hi8[u].x, hi8[u].y};
+            uint32_t lo_w[4], hi_w[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {          // pairs 8c + 2j, 8c + 2j + 1 = bytes 2j, 2j + 1 of the 8
+              const uint16_t lb = static_cast<uint16_t>(lw[j >> 1] >> (16 * (j & 1))), hb = static_cast<uint16_t>(hw[j >> 1] >> (16 * (j & 1)));
+              uint32_t lh, hh;
+              asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(lh) : "h"(lb));
+              asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(hh) : "h"(hb));
+              const float2 a = __half22float2(*reinterpret_cast<const __half2*>(&lh)), bq = __half22float2(*reinterpret_cast<const __half2*>(&hh));
+              const float2 l = fma2(a, cc[j], mul2(bq, make_float2(-ss[j].x, -ss[j].y)));      // lo cos - hi sin
+              const float2 hgh = fma2(a, ss[j], mul2(bq, cc[j]));                                // lo sin + hi cos
+              lo_w[j] = pack_bf16x2(l.x, l.y);
+              hi_w[j] = pack_bf16x2(hgh.x, hgh.y);
+            }
+            *reinterpret_cast<uint4*>(Kb + (lc / 8) * kBlockBytes + sw128(kk, lc % 8)) = make_uint4(lo_w[0], lo_w[1], lo_w[2], lo_w[3]);
+            *reinterpret_cast<uint4*>(Kb + (hc / 8) * kBlockBytes + sw128(kk, hc % 8)) = make_uint4(hi_w[0], hi_w[1], hi_w[2], hi_w[3]);
+            if (i0 + u + 1 < CH) {
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const float2 cn = fma2(ss[j], ns1[j], mul2(cc[j], c1[j]));
+                ss[j] = fma2(ss[j], c1[j], mul2(cc[j], s1[j]));
+                cc[j] = cn;
+              }
+            }
+          }
+        }
+        fence_async_smem();
+        mbar_arrive(BAR(kBarKReady, st));
+        // ---- the V tile of the same index: widen, scale, store; rows at or past kv_len become zero (P is 0 there,
+        // but 0 x NaN is NaN)
+        const int vst = tile % kVStages;
+        if (!mbar_wait(BAR(kBarVLanded, vst), static_cast<uint32_t>(tile / kVStages) & 1u, abort_flag, p.status, p.spin_limit)) break;
+        unsigned char* Vb = Vs + vst * NB * kBlockBytes;
+#pragma unroll 2
+        for (int i = 0; i < 8; ++i) {
+          const int idx = rt + 128 * i;              // 16-byte chunk of codes: key idx / 8, dims [16 (idx % 8), +16)
+          const int kk = idx >> 3, c16 = idx & 7;
+          const int vr = vrow[vst * 8 + (kk >> 4)];
+          uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+          if (vr >= 0 && key0 + kk < kvl) {
+            const uint4 cd = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(p.v_pool) + static_cast<size_t>(vr + (kk & 15)) * D + 16 * c16));
+            const float sc = __ldg(p.v_scales + vr / p.page_size);
+            const uint32_t cw[4] = {cd.x, cd.y, cd.z, cd.w};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+              uint32_t hh;
+              asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(hh) : "h"(static_cast<uint16_t>(cw[j >> 1] >> (16 * (j & 1)))));
+              const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hh));
+              w[j] = pack_bf16x2(f.x * sc, f.y * sc);
+            }
+          }
+          const int ch0 = 2 * c16;                   // bf16 chunk (8 dims) index within the row
+          *reinterpret_cast<uint4*>(Vb + (ch0 / 8) * kBlockBytes + sw128(kk, ch0 % 8)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(Vb + (ch0 / 8) * kBlockBytes + sw128(kk, ch0 % 8 + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+        fence_async_smem();
+        mbar_arrive(BAR(kBarVReady, vst));
+        continue;
       }
 #pragma unroll 2
       for (int i = 0; i < CH; ++i) {
@@ -698,10 +883,16 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
       }
       if (is_k && lane < 8) gbase[st * 8 + lane] = pos;
+      if (FP8 && lane < 8) (is_k ? krow : vrow)[st * 8 + lane] = live ? (page * p.n_kv_heads + h) * p.page_size + slot0 : -1;
       const unsigned live_mask = __ballot_sync(0xffffffffu, live);
       __syncwarp();
       const uint32_t landed = BAR(is_k ? kBarKLanded : kBarVLanded, st);
       if (is_k && blockIdx.x == 0 && tile == p.skip_tile) continue;      // (test hook: a K tile that never comes)
+      if constexpr (FP8) {
+        // nothing to copy: the stage is free and its groups' pool rows are published; the rotators do the rest
+        if (lane == 0) mbar_arrive(landed);
+        continue;
+      }
       if (lane == 0) mbar_expect_tx(landed, static_cast<uint32_t>(__popc(live_mask)) * kGroupBytes);
       __syncwarp();
       if (live) {
@@ -713,7 +904,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     }
     // Rows at or past kv_len of the last V tile may hold anything (NaN bit patterns included): P is 0 there,
     // but 0 x NaN is NaN, so V must be finite.  Zero them once the tile has landed.
-    if (!is_k && ok && last_has_tail) {
+    if (!FP8 && !is_k && ok && last_has_tail) {
       const int lt = n_tiles - 1, st = lt % kVStages;
       if (mbar_wait_warp(BAR(kBarVLanded, st), static_cast<uint32_t>(lt / kVStages) & 1u, abort_flag, p.status, p.spin_limit)) {
         unsigned char* Vb = Vs + st * NB * kBlockBytes;
@@ -774,8 +965,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       bool v_here = false;
       auto wait_v = [&]() {
         if (v_here) return true;
-        bool w = mbar_wait(BAR(kBarVLanded, j % kVStages), static_cast<uint32_t>(j / kVStages) & 1u, abort_flag, p.status, p.spin_limit);
-        if (w && j == n_tiles - 1 && last_has_tail) w = mbar_wait(BAR(kBarVPatched, 0), 0, abort_flag, p.status, p.spin_limit);
+        bool w = mbar_wait(BAR(FP8 ? kBarVReady : kBarVLanded, j % kVStages), static_cast<uint32_t>(j / kVStages) & 1u, abort_flag, p.status, p.spin_limit);
+        if (!FP8 && w && j == n_tiles - 1 && last_has_tail) w = mbar_wait(BAR(kBarVPatched, 0), 0, abort_flag, p.status, p.spin_limit);
         v_here = w;
         return w;
       };
@@ -809,7 +1000,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   }
 
   // ---- common exit: nothing of this CTA may still be in flight when tensor memory is released
-  if ((warp == kKLoaderWarp || warp == kVLoaderWarp) && *abort_flag) {
+  if (!FP8 && (warp == kKLoaderWarp || warp == kVLoaderWarp) && *abort_flag) {
     // a wait ran out somewhere: give outstanding TMA copies a bounded chance to land before leaving
     const int which = warp == kKLoaderWarp ? kBarKLanded : kBarVLanded;
     const int depth = warp == kKLoaderWarp ? kKStages : kVStages;
@@ -863,13 +1054,14 @@ __global__ void __launch_bounds__(128) mepic_prefill_merge(const PrefillParams p
   }
 }
 
-template <int D, int G>
+template <int D, int G, bool FP8>
 int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
   constexpr size_t smem = PrefillSmem<D>::kBytes;
-  cudaError_t e = cudaFuncSetAttribute(mepic_prefill_attn<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  cudaError_t e = cudaFuncSetAttribute(mepic_prefill_attn<D, G, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("prefill: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   const int chunks_per_row = p.n_kv_heads * D / 8;
-  mepic_prefill_commit<<<p.total_rows, 128, 0, stream>>>(p, chunks_per_row);
+  if (FP8) mepic_prefill_commit_fp8<<<p.total_rows, 256, 0, stream>>>(p, D);
+  else mepic_prefill_commit<<<p.total_rows, 128, 0, stream>>>(p, chunks_per_row);
   // each kernel may become resident while its predecessor drains (programmatic dependent launch); it waits with
   // griddepcontrol.wait before it touches what the predecessor writes
   cudaLaunchAttribute pdl[1];
@@ -878,7 +1070,7 @@ int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& m
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(static_cast<unsigned>(n_items * p.n_splits)); lc.blockDim = dim3(kThreads); lc.dynamicSmemBytes = smem; lc.stream = stream;
   lc.attrs = pdl; lc.numAttrs = 1;
-  e = cudaLaunchKernelEx(&lc, mepic_prefill_attn<D, G>, p, map_k, map_v);
+  e = cudaLaunchKernelEx(&lc, mepic_prefill_attn<D, G, FP8>, p, map_k, map_v);
   if (e == cudaSuccess && p.n_splits > 1) {
     const long long n_pairs = static_cast<long long>(p.total_rows) * p.n_kv_heads * G;
     lc.gridDim = dim3(static_cast<unsigned>((n_pairs + 3) / 4)); lc.blockDim = dim3(128); lc.dynamicSmemBytes = 0;
@@ -940,8 +1132,9 @@ extern "C" size_t mepic_attn_prefill_workspace(const mepic_config_t* cfg, int32_
   return split_workspace_bytes(cfg, row_offsets_host[batch], splits_for(n_items));
 }
 
-extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_prefill_args_t* a, void* cuda_stream) {
+static int32_t prefill_call(const mepic_config_t* cfg, const mepic_prefill_args_t* a, float* k_scales, float* v_scales, bool fp8, void* cuda_stream) {
   if (!mepic_config_ok(cfg)) return MEPIC_E_INVAL;
+  if (fp8 && cfg->head_dim != 128) { mepic_set_error("prefill_fp8: head_dim %d: 8-bit pages are built for head_dim 128", cfg->head_dim); return MEPIC_E_INVAL; }
   if (!a || !a->row_offsets_host) { mepic_set_error("prefill: NULL pointer argument"); return MEPIC_E_INVAL; }
   if (a->batch < 1 || a->table_stride < 1) { mepic_set_error("prefill: batch and table_stride must be positive"); return MEPIC_E_INVAL; }
   if (a->row_offsets_host[0] == 0 && a->row_offsets_host[a->batch] == 0) return MEPIC_OK;   // no rows at all: the row buffers may be absent
@@ -959,14 +1152,20 @@ extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_pre
   if (!count_items(cfg, a->batch, a->row_offsets_host, &n_items, &max_q_tiles)) { mepic_set_error("prefill: row_offsets must be non-decreasing"); return MEPIC_E_INVAL; }
   const int total_rows = a->row_offsets_host[a->batch];
   if (n_items == 0 || total_rows == 0) return MEPIC_OK;      // nothing to recompute
+  if (fp8 && (!k_scales || !v_scales)) { mepic_set_error("prefill_fp8: NULL scale pointer"); return MEPIC_E_INVAL; }
   alignas(64) CUtensorMap map_k, map_v;
-  int32_t rc = mepic_make_pool_map(cfg, a->k_pool, &map_k);
-  if (rc != MEPIC_OK) return rc;
-  rc = mepic_make_pool_map(cfg, a->v_pool, &map_v);
-  if (rc != MEPIC_OK) return rc;
+  if (fp8) {
+    memset(&map_k, 0, sizeof(map_k)); memset(&map_v, 0, sizeof(map_v));        // the 8-bit kernel does not use TMA
+  } else {
+    int32_t rc = mepic_make_pool_map(cfg, a->k_pool, &map_k);
+    if (rc != MEPIC_OK) return rc;
+    rc = mepic_make_pool_map(cfg, a->v_pool, &map_v);
+    if (rc != MEPIC_OK) return rc;
+  }
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
   PrefillParams p;
+  p.k_scales = k_scales; p.v_scales = v_scales;
   p.q_new = static_cast<const uint16_t*>(a->q_new);
   p.k_new = static_cast<const uint16_t*>(a->k_new);
   p.v_new = static_cast<const uint16_t*>(a->v_new);
@@ -986,10 +1185,24 @@ extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_pre
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
   p.spin_limit = mepic_test_spin_limit(kSpinLimit); p.skip_tile = mepic_test_skip_tile();
   const int D = cfg->head_dim, G = cfg->n_q_heads / cfg->n_kv_heads;
-#define MEPIC_PREFILL_CASE(DD, GG) if (D == DD && G == GG) return launch_prefill<DD, GG>(p, n_items, map_k, map_v, st);
+  if (fp8) {
+#define MEPIC_PREFILL_FP8_CASE(GG) if (G == GG) return launch_prefill<128, GG, true>(p, n_items, map_k, map_v, st);
+    MEPIC_PREFILL_FP8_CASE(1) MEPIC_PREFILL_FP8_CASE(2) MEPIC_PREFILL_FP8_CASE(3) MEPIC_PREFILL_FP8_CASE(4) MEPIC_PREFILL_FP8_CASE(5) MEPIC_PREFILL_FP8_CASE(6) MEPIC_PREFILL_FP8_CASE(7) MEPIC_PREFILL_FP8_CASE(8)
+#undef MEPIC_PREFILL_FP8_CASE
+  }
+#define MEPIC_PREFILL_CASE(DD, GG) if (D == DD && G == GG) return launch_prefill<DD, GG, false>(p, n_items, map_k, map_v, st);
   MEPIC_PREFILL_CASE(128, 1) MEPIC_PREFILL_CASE(128, 2) MEPIC_PREFILL_CASE(128, 3) MEPIC_PREFILL_CASE(128, 4) MEPIC_PREFILL_CASE(128, 5) MEPIC_PREFILL_CASE(128, 6) MEPIC_PREFILL_CASE(128, 7) MEPIC_PREFILL_CASE(128, 8)
   MEPIC_PREFILL_CASE(64, 1) MEPIC_PREFILL_CASE(64, 2) MEPIC_PREFILL_CASE(64, 3) MEPIC_PREFILL_CASE(64, 4) MEPIC_PREFILL_CASE(64, 5) MEPIC_PREFILL_CASE(64, 6) MEPIC_PREFILL_CASE(64, 7) MEPIC_PREFILL_CASE(64, 8)
 #undef MEPIC_PREFILL_CASE
   mepic_set_error("prefill: unsupported head_dim %d / group size %d", D, G);
   return MEPIC_E_INVAL;
+}
+
+extern "C" int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_prefill_args_t* a, void* cuda_stream) {
+  return prefill_call(cfg, a, nullptr, nullptr, false, cuda_stream);
+}
+
+extern "C" int32_t mepic_attn_prefill_fp8(const mepic_config_t* cfg, const mepic_prefill_args_t* a, float* k_scales, float* v_scales,
+                                          void* cuda_stream) {
+  return prefill_call(cfg, a, k_scales, v_scales, true, cuda_stream);
 }

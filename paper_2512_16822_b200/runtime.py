@@ -14,7 +14,7 @@ import torch
 from . import (Config, Segment, Store, MEPIC_SEG_CHUNK, MEPIC_SEG_PROMPT, mepic_attn_decode,
                mepic_decode_plan_build, mepic_attn_decode_grouped, mepic_attn_decode_grouped_workspace,
                mepic_pages_quantize, mepic_attn_decode_fp8,
-               mepic_attn_decode_workspace, mepic_attn_prefill, mepic_attn_prefill_workspace,
+               mepic_attn_decode_workspace, mepic_attn_prefill, mepic_attn_prefill_fp8, mepic_attn_prefill_workspace,
                mepic_rope_table_fill)
 
 
@@ -81,13 +81,15 @@ class Device:
     """The buffers one pool needs on a GPU: K/V pools, rope table, status word."""
 
     def __init__(self, cfg: Config, k_bits: Optional[np.ndarray] = None, v_bits: Optional[np.ndarray] = None,
-                 device: str = "cuda:0"):
+                 device: str = "cuda:0", bf16_pools: bool = True):
         if not torch.cuda.is_available():
             raise RuntimeError("the MEPIC kernels need a CUDA device; there is no CPU path")
         self.cfg = cfg
         self.device = torch.device(device)
         shape = (cfg.num_pages, cfg.n_kv_heads, cfg.page_size, cfg.head_dim)
-        if k_bits is not None:
+        if not bf16_pools:
+            self.k_pool = self.v_pool = None           # a device whose only pools are 8-bit (see Fp8Pools)
+        elif k_bits is not None:
             assert k_bits.shape == shape and v_bits.shape == shape
             self.k_pool = bf16_tensor(k_bits, self.device)
             self.v_pool = bf16_tensor(v_bits, self.device)
@@ -169,7 +171,8 @@ class Fp8Pools:
         self.v_codes = torch.zeros(shape, dtype=torch.uint8, device=d)
         self.k_scales = torch.ones((cfg.num_pages, cfg.n_kv_heads), dtype=torch.float32, device=d)
         self.v_scales = torch.ones((cfg.num_pages, cfg.n_kv_heads), dtype=torch.float32, device=d)
-        self.quantize(np.arange(cfg.num_pages, dtype=np.int32) if pages is None else pages)
+        if dev.k_pool is not None:                     # pools without a bf16 original start empty: prefill fills them
+            self.quantize(np.arange(cfg.num_pages, dtype=np.int32) if pages is None else pages)
 
     def quantize(self, pages: np.ndarray, stream=None) -> None:
         lst = torch.from_numpy(np.ascontiguousarray(pages, dtype=np.int32)).to(self.dev.device)
@@ -255,4 +258,24 @@ class PrefillBatch:
                            workspace_bytes=self.ws_bytes, status=self.dev.status,
                            row_offsets_host=self.row_offsets_host, table_stride=self.stride, batch=self.batch,
                            sm_scale=sm_scale, stream=s)
+        return self.out
+
+
+class Fp8PrefillBatch(PrefillBatch):
+    """A prefill batch that commits into, and attends over, the 8-bit pools."""
+
+    def __init__(self, pools: Fp8Pools, page_ids, pos_base, kv_len, row_offsets, q_slot, q_bits, k_bits, v_bits):
+        super().__init__(pools.dev, page_ids, pos_base, kv_len, row_offsets, q_slot, q_bits, k_bits, v_bits)
+        self.pools = pools
+
+    def run(self, sm_scale: float, stream=None) -> torch.Tensor:
+        s = stream if stream is not None else torch.cuda.current_stream(self.dev.device)
+        mepic_attn_prefill_fp8(self.dev.cfg, q_new=self.q_new, k_new=self.k_new, v_new=self.v_new,
+                               row_offsets=self.row_offsets, q_slot=self.q_slot, k_pool=self.pools.k_codes,
+                               v_pool=self.pools.v_codes, k_scales=self.pools.k_scales, v_scales=self.pools.v_scales,
+                               page_ids=self.page_ids, pos_base=self.pos_base, kv_len=self.kv_len,
+                               rope_table=self.dev.rope, out=self.out, workspace=self.workspace,
+                               workspace_bytes=self.ws_bytes, status=self.dev.status,
+                               row_offsets_host=self.row_offsets_host, table_stride=self.stride, batch=self.batch,
+                               sm_scale=sm_scale, stream=s)
         return self.out

@@ -79,7 +79,8 @@ def test_decode_wait_runs_out_status_is_set_and_the_next_call_is_clean(kind):
             assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS, (b, d.max())
 
 
-def test_prefill_wait_runs_out_every_role_leaves_and_the_next_call_is_clean():
+@pytest.mark.parametrize("fp8", [False, True])
+def test_prefill_wait_runs_out_every_role_leaves_and_the_next_call_is_clean(fp8):
     # one work item, one CTA (a 16-byte workspace keeps the call from cutting the item into shares): 600 keys = 5 key tiles
     cfg, kp, vp, ids, base, kvl, _, _ = _case(2, [600])
     rng = np.random.default_rng(3)
@@ -89,7 +90,11 @@ def test_prefill_wait_runs_out_every_role_leaves_and_the_next_call_is_clean():
     ro = np.array([0, 32], dtype=np.int32)
     sm = 1.0 / np.sqrt(D)
     dev = RT.Device(cfg, kp.copy(), vp.copy())
-    pb = RT.PrefillBatch(dev, ids, base, kvl, ro, slots, qn, kn, vn)
+    if fp8:
+        pools = RT.Fp8Pools(dev)
+        pb = RT.Fp8PrefillBatch(pools, ids, base, kvl, ro, slots, qn, kn, vn)
+    else:
+        pb = RT.PrefillBatch(dev, ids, base, kvl, ro, slots, qn, kn, vn)
     pb.ws_bytes = 16
     for skip in (0, 2):                               # the very first key tile; one in the middle of the pipeline
         try:
@@ -102,6 +107,15 @@ def test_prefill_wait_runs_out_every_role_leaves_and_the_next_call_is_clean():
         dev.status.zero_()
     out = pb.run(sm); torch.cuda.synchronize()
     assert dev.read_status() == 0
+    if fp8:
+        kc, ks = O.quantize_pages(kp); vc, vs = O.quantize_pages(vp)
+        O.commit_rows_fp8(kc, ks, vc, vs, list(ids[0]), list(slots), kn, vn)
+        want = O.prefill_attention_one(qn, kn, vn, list(slots), O.dequantize_pages(kc, ks), O.dequantize_pages(vc, vs),
+                                       list(ids[0]), list(base[0]), 600, sm, THETA)
+        d = np.abs(bf16_bits_to_f64(RT.bf16_bits(out)) - want)
+        assert d.max() <= MAX_ABS and d.mean() <= MEAN_ABS
+        assert np.array_equal(pools.k_codes.cpu().numpy(), kc) and np.array_equal(pools.k_scales.cpu().numpy(), ks)
+        return
     okp, ovp = kp.copy(), vp.copy()
     want = O.prefill_attention_one(qn, kn, vn, list(slots), okp, ovp, list(ids[0]), list(base[0]), 600, sm, THETA)
     d = np.abs(bf16_bits_to_f64(RT.bf16_bits(out)) - want)
