@@ -624,6 +624,110 @@ def measure_variant(kind: str, args, wl, dev, tabs, q_bits, logical_bytes: int, 
     return d
 
 
+def measure_decode_loop(args, device: str, index: int = 2, n_steps: int = 64):
+    """A decode loop as a serving system runs it: n_steps consecutive steps of the batch, every request one token
+    longer each step (page gains included), the step's inputs from pinned host memory, the result read back and
+    waited for before the next step.  Once through mepic_attn_decode (q, lengths, positions every step; the block
+    tables again whenever a request gained a page) and once through the sharing-aware path (the plan built once
+    before the loop, patched with mepic_decode_plan_patch at every page gain, only the changed stretches uploaded).
+    Wall-clock time per step: host work (table update, plan patch) counts."""
+    import torch
+    from paper_2512_16822_b200 import runtime as RT
+    wl = make_workload(index)
+    P = wl.page_size
+    import paper_2512_16822_b200 as M
+    B = len(wl.decode_requests)
+    spare = -(-n_steps // P) + 1
+    cfg0 = make_config(wl)
+    with M.Store(cfg0) as st:
+        tables = RT.build_tables(st, wl.chunks, wl.decode_requests)
+    ids0, base0, kvl0, _ = RT.pack_tables(tables, P)
+    stride = ids0.shape[1] + spare
+    cfg = M.Config(P, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.num_pages + B * spare, wl.max_position + (spare + 1) * P,
+                   wl.rope_theta, wl.pad_token_id)
+    kp, vp = wl.kv_pool()
+    pad = np.zeros((B * spare,) + kp.shape[1:], dtype=np.uint16)        # the pages the loop will hand out (values do not matter)
+    dev = RT.Device(cfg, np.concatenate([kp, pad]), np.concatenate([vp, pad]), device=device)
+    q_bits = wl.decode_q()
+    stream = torch.cuda.current_stream()
+    out = {}
+    for path in ("per_request", "grouped"):
+        ids = np.zeros((B, stride), dtype=np.int32); base = np.zeros((B, stride), dtype=np.int32)
+        ids[:, :ids0.shape[1]] = ids0; base[:, :ids0.shape[1]] = base0
+        kvl = kvl0.copy()
+        q_pos = (kvl - 1).astype(np.int32)
+        if path == "per_request":
+            batch = RT.DecodeBatch(dev, ids, base, kvl, q_pos, q_bits)
+            h_in, hv = batch.host_mirror()
+            hv["q"].copy_(torch.from_numpy(np.ascontiguousarray(q_bits).view(np.int16)))
+            h_ids, h_base, h_kvl, h_qpos = hv["page_ids"].numpy(), hv["pos_base"].numpy(), hv["kv_len"].numpy(), hv["q_pos"].numpy()
+            h_q = hv["q"].view(torch.bfloat16)
+        else:
+            batch = RT.GroupedDecodeBatch(dev, ids, base, kvl, q_pos, q_bits)
+            h_q = torch.from_numpy(np.ascontiguousarray(q_bits).view(np.int16)).view(torch.bfloat16).pin_memory()
+            h_kvl_t = torch.empty(B, dtype=torch.int32).pin_memory(); h_qpos_t = torch.empty(B, dtype=torch.int32).pin_memory()
+            h_kvl, h_qpos = h_kvl_t.numpy(), h_qpos_t.numpy()
+        h_out = torch.empty(batch.out.shape, dtype=torch.bfloat16).pin_memory()
+        next_page = wl.num_pages
+        for rep in range(2):                       # the first pass warms up (and checks the status word); the second is timed
+            ids[:, ids0.shape[1]:] = 0; kvl[:] = kvl0
+            if rep == 1 and path == "grouped":
+                batch = RT.GroupedDecodeBatch(dev, ids, base, kvl, (kvl - 1).astype(np.int32), q_bits)   # a fresh plan (built outside the timed loop)
+            if path == "per_request":
+                h_ids[:] = ids; h_base[:] = base
+                batch.upload(h_in)
+            next_page = wl.num_pages
+            gains = uploaded = 0
+            host_s = 0.0
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for step in range(n_steps):
+                th = time.perf_counter()
+                gained = False
+                for r in range(B):
+                    if kvl[r] % P == 0:
+                        e = kvl[r] // P
+                        ids[r, e] = next_page; next_page += 1
+                        base[r, e] = base[r, e - 1] + P
+                        gained = True; gains += 1
+                    kvl[r] += 1
+                h_kvl[:] = kvl; h_qpos[:] = kvl - 1
+                if path == "per_request":
+                    if gained:
+                        h_ids[:] = ids; h_base[:] = base
+                        host_s += time.perf_counter() - th
+                        batch.upload(h_in); uploaded += int(h_in.numel())
+                    else:
+                        host_s += time.perf_counter() - th
+                        batch.q.copy_(h_q, non_blocking=True); batch.kv_len.copy_(hv["kv_len"], non_blocking=True)
+                        batch.q_pos.copy_(hv["q_pos"], non_blocking=True)
+                        uploaded += int(h_q.numel() * 2 + 8 * B)
+                else:
+                    if gained:
+                        uploaded += batch.patch(ids, base, kvl)
+                    host_s += time.perf_counter() - th
+                    batch.q.copy_(h_q, non_blocking=True); batch.kv_len.copy_(h_kvl_t, non_blocking=True)
+                    batch.q_pos.copy_(h_qpos_t, non_blocking=True)
+                    uploaded += int(h_q.numel() * 2 + 8 * B)
+                batch.run(wl.sm_scale, stream)
+                h_out.copy_(batch.out, non_blocking=True)
+                stream.synchronize()
+            wall = time.perf_counter() - t0
+            assert dev.read_status() == 0, "device status word is not clean"
+        tokens = int(kvl0.astype(np.int64).sum()) + B * (n_steps + 1) // 2
+        out[path] = {"ms_per_step": 1e3 * wall / n_steps, "steps": n_steps, "page_gains": gains,
+                     "host_ms_per_step": 1e3 * host_s / n_steps, "h2d_bytes_per_step": uploaded / n_steps,
+                     "d2h_bytes_per_step": int(h_out.numel() * 2),
+                     "value": tokens * kv_bytes_per_token(wl) / (wall / n_steps) / 1e9, "unit": "GB/s"}
+        if path == "grouped":
+            out[path]["plan_ints"] = int(len(batch.plan_host))
+        del batch
+    out["grouped_over_per_request"] = out["per_request"]["ms_per_step"] / out["grouped"]["ms_per_step"]
+    out["note"] = (f"config {index}, {n_steps} consecutive decode steps, kv_len + 1 per step and request; wall clock per step with the "
+                   "result awaited every step; value = mean logical K/V bytes per step / time; no L2 flush (a serving loop has none)")
+    return out
+
+
 def measure_mixed(args, device: str):
     """Config 5 as one serving step: its decode batch and its prefill requests over one pool, each call alone and
     both enqueued on two streams (device time from the fork to the join)."""
@@ -693,6 +797,9 @@ def run_leg(args):
         return
     if args.leg == "mixed":
         print(json.dumps(measure_mixed(args, device)), flush=True)
+        return
+    if args.leg == "loop":
+        print(json.dumps(measure_decode_loop(args, device, args.config if args.config != 3 else 2)), flush=True)
         return
     wl = make_workload(args.config, scale=args.scale)
     stream = torch.cuda.current_stream()
@@ -867,6 +974,10 @@ def run_ours(args):
             configs.setdefault("config5", {})["prefill"] = pre5
             torch.cuda.empty_cache()
             configs["config5"]["serving_step"] = measure_mixed(args, device)
+            torch.cuda.empty_cache()
+            loop = measure_decode_loop(args, device)
+        if grouped is not None:
+            grouped["e2e"] = loop
     clocks = sampler.stop() if rank == 0 else None
     if rank != 0:
         if world > 1:
@@ -942,7 +1053,7 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=12.0, help="seconds of oracle time for cpu_baseline")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--quick", action="store_true", help="headline and unshared layout only: no other configs, no variants")
-    ap.add_argument("--leg", default=None, choices=["decode", "unshared", "grouped", "fp8", "unshared-fp8", "prefill", "prefill-fp8", "mixed", "graph"],
+    ap.add_argument("--leg", default=None, choices=["decode", "unshared", "grouped", "fp8", "unshared-fp8", "prefill", "prefill-fp8", "mixed", "graph", "loop"],
                     help="run one leg alone (a short fixed sequence of calls, e.g. for a profiler) and print its line")
     ap.add_argument("--scale", type=float, default=1.0, help="with --leg: shrink the configuration (1.0 = as specified)")
     args = ap.parse_args()

@@ -347,9 +347,9 @@ int32_t mepic_attn_decode_static(const mepic_config_t* cfg, const mepic_decode_a
  * equal pieces for n_sms * 8 workers (n_sms = 0: the SM count of the current device).  The plan is a
  * flat int32 buffer the caller treats as opaque, copies to the device as is, and also keeps on the
  * host.  It bakes in page ids, position bases and the number of table entries of every request; it
- * stays valid while kv_len grows inside each request's last page and must be rebuilt when a request
- * gains a page or the batch changes (the device sets MEPIC_DEV_BAD_PLAN otherwise and the result is
- * then undefined but the call does not fault).  mepic_decode_plan_max_ints bounds the buffer size
+ * stays valid while kv_len grows inside each request's last page; when a request gains a page it is
+ * patched (mepic_decode_plan_patch) or rebuilt, when the batch changes it is rebuilt (the device sets
+ * MEPIC_DEV_BAD_PLAN otherwise and the result is then undefined but the call does not fault).  mepic_decode_plan_max_ints bounds the buffer size
  * for any tables of that shape.  Errors: E_INVAL (bad argument, kv_len < 1, entries > stride),
  * E_CAPACITY (buffer too small: *out_ints holds the need; or a batch beyond the plan's 32-bit
  * fields), E_CUDA (n_sms = 0 without a device).
@@ -365,6 +365,23 @@ size_t  mepic_decode_plan_max_ints(const mepic_config_t* cfg, int32_t batch, int
 int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int32_t* page_ids_host, const int32_t* pos_base_host,
                                 const int32_t* kv_len_host, int32_t batch, int32_t table_stride, int32_t n_sms,
                                 int32_t* out_plan_host, size_t cap_ints, size_t* out_ints);
+
+/*
+ * mepic_decode_plan_patch - keeps a plan alive across a page gain (the paper has no counterpart; a plan is this
+ * library's).  In a decode loop every request gains a table entry each page_size tokens; instead of regrouping every
+ * entry again, the request's new pages are appended to its own single-request item (the plan reserves room for 16
+ * more pages per request, as far as table_stride lets the request grow) and everything that follows from the items'
+ * sizes (places on the line, the cut, the workers' starts, the partial slots) is written again: host work of
+ * O(items + workers).  plan_host (HOST, in/out): the plan as built; page_ids_host / pos_base_host / kv_len_host (HOST):
+ * the tables as they are NOW (entries that existed at build time must be unchanged).  On MEPIC_OK out_ranges (HOST,
+ * 4 x int64) holds *out_n_ranges (0 or 2) pairs {first int, number of ints} of plan_host that changed: copy exactly
+ * those to the device copy.  The workspace the plan needs may have grown (mepic_attn_decode_grouped_workspace).
+ * Errors: E_INVAL (bad argument, another config or batch, a request that lost pages), E_CAPACITY (a request has no
+ * own item or its reserve is used up: build a new plan; nothing was changed).
+ */
+int32_t mepic_decode_plan_patch(const mepic_config_t* cfg, int32_t* plan_host, const int32_t* page_ids_host,
+                                const int32_t* pos_base_host, const int32_t* kv_len_host, int32_t batch, int32_t table_stride,
+                                int64_t* out_ranges, int32_t* out_n_ranges);
 
 typedef struct {
   const void*    q;            /* bf16 [batch][n_q_heads][head_dim], un-rotated */

@@ -24,7 +24,7 @@ __all__ = [
     "mepic_store_create", "mepic_store_destroy", "mepic_chunk_register", "mepic_build_block_table",
     "mepic_request_release", "mepic_chunk_mark_uncomputed", "mepic_store_stats", "mepic_store_attach_remote", "mepic_store_test_hooks", "mepic_kernel_test_hooks", "mepic_rope_table_floats", "mepic_rope_table_fill",
     "mepic_attn_decode_workspace", "mepic_attn_decode", "mepic_attn_decode_static",
-    "mepic_pages_quantize", "mepic_attn_decode_fp8", "mepic_decode_plan_max_ints", "mepic_decode_plan_build", "mepic_attn_decode_grouped_workspace",
+    "mepic_pages_quantize", "mepic_attn_decode_fp8", "mepic_decode_plan_max_ints", "mepic_decode_plan_build", "mepic_decode_plan_patch", "mepic_attn_decode_grouped_workspace",
     "mepic_attn_decode_grouped",
     "MEPIC_DECODE_STATIC_SCRATCH_BYTES", "mepic_attn_prefill_workspace",
     "mepic_attn_prefill", "mepic_attn_prefill_fp8", "mepic_last_error", "mepic_launch_count",
@@ -149,6 +149,8 @@ _PROTOTYPES = {
     "mepic_decode_plan_max_ints": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32, C.c_int32, C.c_int32]),
     "mepic_decode_plan_build": (C.c_int32, [C.POINTER(_ConfigC), C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                             C.c_int32, C.c_int32, C.c_void_p, C.c_size_t, C.POINTER(C.c_size_t)]),
+    "mepic_decode_plan_patch": (C.c_int32, [C.POINTER(_ConfigC), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                            C.c_int32, C.c_void_p, C.POINTER(C.c_int32)]),
     "mepic_attn_decode_grouped_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_void_p]),
     "mepic_attn_decode_grouped": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeGroupedArgsC), C.c_void_p]),
     "mepic_attn_prefill_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32, C.c_void_p]),
@@ -422,6 +424,22 @@ def mepic_decode_plan_build(cfg: Config, page_ids: np.ndarray, pos_base: np.ndar
     _check(lib().mepic_decode_plan_build(C.byref(c), ids.ctypes.data, base.ctypes.data, lens.ctypes.data, batch, stride,
                                          n_sms, out.ctypes.data, cap, C.byref(used)))
     return out[:used.value].copy()
+
+
+def mepic_decode_plan_patch(cfg: Config, plan_host: np.ndarray, page_ids: np.ndarray, pos_base: np.ndarray,
+                            kv_len: np.ndarray):
+    """Patch ``plan_host`` in place after requests gained pages -> list of (first int, count) ranges that changed."""
+    ids = np.ascontiguousarray(page_ids, dtype=np.int32)
+    base = np.ascontiguousarray(pos_base, dtype=np.int32)
+    lens = np.ascontiguousarray(kv_len, dtype=np.int32)
+    batch, stride = ids.shape
+    assert plan_host.dtype == np.int32 and plan_host.flags["C_CONTIGUOUS"]
+    ranges = np.zeros(4, dtype=np.int64)
+    n = C.c_int32(0)
+    c = cfg.c()
+    _check(lib().mepic_decode_plan_patch(C.byref(c), plan_host.ctypes.data, ids.ctypes.data, base.ctypes.data, lens.ctypes.data,
+                                         batch, stride, ranges.ctypes.data, C.byref(n)))
+    return [(int(ranges[2 * k]), int(ranges[2 * k + 1])) for k in range(n.value)]
 
 
 def mepic_attn_decode_grouped_workspace(cfg: Config, plan_host: np.ndarray) -> int:

@@ -41,6 +41,81 @@ int sm_count_or(int n_sms) {
   return sms;
 }
 
+// Everything in the plan that follows from the items and their page counts: each item's place on the line, the cut of
+// the line into pieces, where each worker's piece begins, and the partial slots.  Written at build time and again after
+// a patch (a request that gained pages moves every later item along the line).
+int32_t derive_plan(int32_t* plan) {
+  int32_t* h = plan;
+  const int n_items = h[kPhItems], R = h[kPhR], Hkv = h[kPhKvHeads], batch = h[kPhBatch], n_workers = h[kPhWorkers];
+  const int tpp = h[kPhPageSize] / kPlanTile;
+  const size_t stride = kItemFixed + R;
+  int32_t* items = plan + h[kPhOffItems];
+  long long tiles_per_head = 0;
+  for (int i = 0; i < n_items; ++i) {
+    if (tiles_per_head >= (1ll << 31)) break;
+    items[i * stride + kPiTileStart] = static_cast<int32_t>(tiles_per_head);
+    tiles_per_head += static_cast<long long>(items[i * stride + kPiEnt]) * tpp;
+  }
+  const long long total = tiles_per_head * Hkv;
+  if (total >= (1ll << 31)) { mepic_set_error("decode_plan: batch too large for the plan's 32-bit fields"); return MEPIC_E_CAPACITY; }
+  long long piece = (total + n_workers - 1) / n_workers;
+  if (piece < kPlanMinPiece) piece = kPlanMinPiece;
+  h[kPhPiece] = static_cast<int32_t>(piece); h[kPhTotal] = static_cast<int32_t>(total);
+  // where each worker's piece begins
+  {
+    int i = 0;
+    for (int w = 0; w < n_workers; ++w) {
+      int32_t* d = plan + h[kPhOffWorkers] + static_cast<size_t>(w) * 3;
+      const long long x = static_cast<long long>(w) * piece;
+      if (x >= total) { d[0] = n_items; d[1] = 0; d[2] = 0; continue; }
+      while (true) {
+        const long long nt = static_cast<long long>(items[i * stride + kPiEnt]) * tpp;
+        const long long start = static_cast<long long>(items[i * stride + kPiTileStart]) * Hkv;
+        if (x < start + nt * Hkv) {
+          d[0] = i; d[1] = static_cast<int32_t>((x - start) / nt); d[2] = static_cast<int32_t>((x - start) % nt);
+          break;
+        }
+        ++i;
+      }
+    }
+  }
+  // partial slots: a unit (item, kv head) is overlapped by the pieces w_first..w_last of the line; each of its rows gets
+  // one slot per piece, and the slots of a (request, kv head) pair are contiguous so that the merge reads one run
+  std::vector<long long> count(static_cast<size_t>(batch) * Hkv + 1, 0);
+  auto pieces_of = [&](int i, int hd) {
+    const long long nt = static_cast<long long>(items[i * stride + kPiEnt]) * tpp;
+    const long long start = static_cast<long long>(items[i * stride + kPiTileStart]) * Hkv + hd * nt;
+    return (start + nt - 1) / piece - start / piece + 1;
+  };
+  for (int i = 0; i < n_items; ++i)
+    for (int hd = 0; hd < Hkv; ++hd)
+      for (int j = 0; j < items[i * stride + kPiReq]; ++j)
+        count[static_cast<size_t>(items[i * stride + kPiReqIds + j]) * Hkv + hd] += pieces_of(i, hd);
+  int32_t* part_off = plan + h[kPhOffPartOff];
+  long long run = 0;
+  for (size_t u = 0; u < static_cast<size_t>(batch) * Hkv; ++u) {
+    part_off[u] = static_cast<int32_t>(run);
+    const long long c = count[u]; count[u] = run; run += c;
+  }
+  if (run >= (1ll << 31)) { mepic_set_error("decode_plan: too many partials for the plan's 32-bit fields"); return MEPIC_E_CAPACITY; }
+  part_off[static_cast<size_t>(batch) * Hkv] = static_cast<int32_t>(run);
+  h[kPhSlots] = static_cast<int32_t>(run);
+  int32_t* slot_base = plan + h[kPhOffSlotBase];
+  for (int i = 0; i < n_items; ++i)
+    for (int hd = 0; hd < Hkv; ++hd) {
+      const long long c = pieces_of(i, hd);
+      for (int j = 0; j < R; ++j) {
+        int32_t v = 0;
+        if (j < items[i * stride + kPiReq]) {
+          long long& cur = count[static_cast<size_t>(items[i * stride + kPiReqIds + j]) * Hkv + hd];
+          v = static_cast<int32_t>(cur); cur += c;
+        }
+        slot_base[(static_cast<size_t>(i) * Hkv + hd) * R + j] = v;
+      }
+    }
+  return MEPIC_OK;
+}
+
 }  // namespace
 
 extern "C" size_t mepic_decode_plan_max_ints(const mepic_config_t* cfg, int32_t batch, int32_t table_stride, int32_t n_sms) {
@@ -49,8 +124,9 @@ extern "C" size_t mepic_decode_plan_max_ints(const mepic_config_t* cfg, int32_t 
   if (sms <= 0) { mepic_set_error("decode_plan: no CUDA device and no SM count given"); return 0; }
   const int R = plan_group_requests(cfg->n_q_heads / cfg->n_kv_heads);
   const size_t E = static_cast<size_t>(batch) * table_stride;     // every entry is one record of one item at most
-  return kPlanHeaderInts + E * (kItemFixed + R) + E * (1 + R) + static_cast<size_t>(sms) * kPlanWarps * 3 +
-         (batch + 1) + E + batch + E * cfg->n_kv_heads * R + static_cast<size_t>(batch) * cfg->n_kv_heads + 1;
+  return kPlanHeaderInts + E * (kItemFixed + R) + (E + static_cast<size_t>(batch) * kPlanReservePages) * (1 + R) +
+         static_cast<size_t>(sms) * kPlanWarps * 3 + (batch + 1) + E + batch + batch + E + E * cfg->n_kv_heads * R +
+         static_cast<size_t>(batch) * cfg->n_kv_heads + 1;
 }
 
 extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int32_t* page_ids, const int32_t* pos_base,
@@ -133,6 +209,7 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
   }
   std::vector<Item> items;
   items.reserve(shared_items.size() + batch);
+  const size_t n_shared_items = shared_items.size();          // the items after these are the requests' own ones
   for (Item& it : shared_items) items.push_back(std::move(it));
   for (int32_t r = 0; r < batch; ++r) {
     if (own[r].empty()) continue;
@@ -144,75 +221,66 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
     items.push_back(std::move(it));
   }
 
-  // sizes and offsets
+  // sizes and offsets.  The run of records of a request's own item has room for kPlanReservePages more pages (as far as
+  // the table's stride lets the request grow), so that a page gain can be patched in (mepic_decode_plan_patch).
+  std::vector<int32_t> cap(items.size());
   size_t n_records = 0, n_req_items = 0;
-  long long tiles_per_head = 0;
-  for (const Item& it : items) { n_records += it.pages(); n_req_items += it.req.size(); tiles_per_head += static_cast<long long>(it.pages()) * tpp; }
-  const long long total = tiles_per_head * Hkv;
-  if (total >= (1ll << 31) || items.size() >= (1u << 27)) { mepic_set_error("decode_plan: batch too large for the plan's 32-bit fields"); return MEPIC_E_CAPACITY; }
+  for (size_t i = 0; i < items.size(); ++i) {
+    const Item& it = items[i];
+    int32_t c = static_cast<int32_t>(it.pages());
+    if (i >= n_shared_items) c += std::min<int32_t>(kPlanReservePages, table_stride - n_ent[it.req[0]]);
+    cap[i] = c;
+    n_records += static_cast<size_t>(c); n_req_items += it.req.size();
+  }
+  if (items.size() >= (1u << 27)) { mepic_set_error("decode_plan: batch too large for the plan's 32-bit fields"); return MEPIC_E_CAPACITY; }
   const int n_workers = sms * kPlanWarps;
-  long long piece = (total + n_workers - 1) / n_workers;
-  if (piece < kPlanMinPiece) piece = kPlanMinPiece;
   const size_t off_items = kPlanHeaderInts;
-  const size_t off_records = off_items + items.size() * (kItemFixed + R);
-  const size_t off_workers = off_records + n_records * (1 + R);
+  const size_t off_workers = off_items + items.size() * (kItemFixed + R);
   const size_t off_req_off = off_workers + static_cast<size_t>(n_workers) * 3;
   const size_t off_req_items = off_req_off + batch + 1;
   const size_t off_req_ent = off_req_items + n_req_items;
-  const size_t off_slot_base = off_req_ent + batch;
+  const size_t off_own_item = off_req_ent + batch;
+  const size_t off_rec_cap = off_own_item + batch;
+  const size_t off_slot_base = off_rec_cap + items.size();
   const size_t off_part_off = off_slot_base + items.size() * Hkv * R;
-  const size_t ints = off_part_off + static_cast<size_t>(batch) * Hkv + 1;
+  const size_t off_records = off_part_off + static_cast<size_t>(batch) * Hkv + 1;
+  const size_t ints = off_records + n_records * (1 + R);
   *out_ints = ints;
+  if (ints >= (1ull << 31)) { mepic_set_error("decode_plan: batch too large for the plan's 32-bit fields"); return MEPIC_E_CAPACITY; }
   if (ints > cap_ints) { mepic_set_error("decode_plan: plan needs %zu ints, buffer holds %zu", ints, cap_ints); return MEPIC_E_CAPACITY; }
 
   int32_t* h = out_plan;
-  h[kPhMagic] = kPlanMagic; h[kPhItems] = static_cast<int32_t>(items.size()); h[kPhWorkers] = n_workers;
-  h[kPhPiece] = static_cast<int32_t>(piece); h[kPhTotal] = static_cast<int32_t>(total); h[kPhR] = R;
+  for (int k = 0; k < kPlanHeaderInts; ++k) h[k] = 0;
+  h[kPhMagic] = kPlanMagic; h[kPhItems] = static_cast<int32_t>(items.size()); h[kPhWorkers] = n_workers; h[kPhR] = R;
   h[kPhOffItems] = static_cast<int32_t>(off_items); h[kPhOffRecords] = static_cast<int32_t>(off_records);
   h[kPhOffWorkers] = static_cast<int32_t>(off_workers); h[kPhOffReqOff] = static_cast<int32_t>(off_req_off);
   h[kPhOffReqItems] = static_cast<int32_t>(off_req_items); h[kPhBatch] = batch; h[kPhRecords] = static_cast<int32_t>(n_records);
   h[kPhInts] = static_cast<int32_t>(ints); h[kPhOffReqEnt] = static_cast<int32_t>(off_req_ent); h[kPhPageSize] = P;
   h[kPhOffSlotBase] = static_cast<int32_t>(off_slot_base); h[kPhOffPartOff] = static_cast<int32_t>(off_part_off);
-  h[kPhKvHeads] = Hkv;
-  for (int k = kPhKvHeads + 1; k < kPlanHeaderInts; ++k) h[k] = 0;
+  h[kPhKvHeads] = Hkv; h[kPhOffOwnItem] = static_cast<int32_t>(off_own_item); h[kPhOffRecCap] = static_cast<int32_t>(off_rec_cap);
 
   std::vector<std::vector<int32_t>> req_items(batch);
-  int32_t rec = 0, tile_start = 0;
+  for (int32_t r = 0; r < batch; ++r) out_plan[off_own_item + r] = -1;
+  int32_t rec = 0;
   for (size_t i = 0; i < items.size(); ++i) {
     const Item& it = items[i];
     int32_t* d = out_plan + off_items + i * (kItemFixed + R);
     d[kPiReq] = static_cast<int32_t>(it.req.size()); d[kPiRecOff] = rec; d[kPiEnt] = static_cast<int32_t>(it.pages());
-    d[kPiTail] = it.tail_slot_start; d[kPiTileStart] = tile_start;
+    d[kPiTail] = it.tail_slot_start; d[kPiTileStart] = 0;
     for (int j = 0; j < R; ++j) d[kPiReqIds + j] = j < static_cast<int>(it.req.size()) ? it.req[j] : -1;
     for (size_t j = 0; j < it.req.size(); ++j) req_items[it.req[j]].push_back(static_cast<int32_t>(i) * 16 + static_cast<int32_t>(j));
+    if (i >= n_shared_items) out_plan[off_own_item + it.req[0]] = static_cast<int32_t>(i);
+    out_plan[off_rec_cap + i] = cap[i];
     const int nr = static_cast<int>(it.req.size());
-    for (size_t k = 0; k < it.pages(); ++k) {
-      const int32_t* ent = it.ent.data() + k * nr;
-      int32_t* q = out_plan + off_records + static_cast<size_t>(rec) * (1 + R);
+    for (int32_t k = 0; k < cap[i]; ++k) {
+      int32_t* q = out_plan + off_records + static_cast<size_t>(rec + k) * (1 + R);
+      for (int j = 0; j <= R; ++j) q[j] = 0;                      // (the unused part of a run reads as page 0)
+      if (static_cast<size_t>(k) >= it.pages()) continue;
+      const int32_t* ent = it.ent.data() + static_cast<size_t>(k) * nr;
       q[0] = page_ids[static_cast<size_t>(it.req[0]) * table_stride + ent[0]];
-      for (int j = 0; j < R; ++j)
-        q[1 + j] = j < nr ? pos_base[static_cast<size_t>(it.req[j]) * table_stride + ent[j]] : 0;
-      ++rec;
+      for (int j = 0; j < nr; ++j) q[1 + j] = pos_base[static_cast<size_t>(it.req[j]) * table_stride + ent[j]];
     }
-    tile_start += static_cast<int32_t>(it.pages()) * tpp;
-  }
-  // where each worker's piece begins
-  {
-    size_t i = 0;
-    for (int w = 0; w < n_workers; ++w) {
-      int32_t* d = out_plan + off_workers + static_cast<size_t>(w) * 3;
-      const long long x = static_cast<long long>(w) * piece;
-      if (x >= total) { d[0] = static_cast<int32_t>(items.size()); d[1] = 0; d[2] = 0; continue; }
-      while (true) {
-        const long long nt = static_cast<long long>(items[i].pages()) * tpp;
-        const long long start = static_cast<long long>(out_plan[off_items + i * (kItemFixed + R) + kPiTileStart]) * Hkv;
-        if (x < start + nt * Hkv) {
-          d[0] = static_cast<int32_t>(i); d[1] = static_cast<int32_t>((x - start) / nt); d[2] = static_cast<int32_t>((x - start) % nt);
-          break;
-        }
-        ++i;
-      }
-    }
+    rec += cap[i];
   }
   int32_t at = 0;
   for (int32_t r = 0; r < batch; ++r) {
@@ -221,37 +289,67 @@ extern "C" int32_t mepic_decode_plan_build(const mepic_config_t* cfg, const int3
     out_plan[off_req_ent + r] = n_ent[r];
   }
   out_plan[off_req_off + batch] = at;
+  return derive_plan(out_plan);
+}
 
-  // partial slots: a unit (item, kv head) is overlapped by the pieces w_first..w_last of the line; each of its rows gets
-  // one slot per piece, and the slots of a (request, kv head) pair are contiguous so that the merge reads one run
-  std::vector<long long> count(static_cast<size_t>(batch) * Hkv + 1, 0);
-  auto pieces_of = [&](size_t i, int hd) {
-    const long long nt = static_cast<long long>(items[i].pages()) * tpp;
-    const long long start = static_cast<long long>(out_plan[off_items + i * (kItemFixed + R) + kPiTileStart]) * Hkv + hd * nt;
-    return (start + nt - 1) / piece - start / piece + 1;
-  };
-  for (size_t i = 0; i < items.size(); ++i)
-    for (int hd = 0; hd < Hkv; ++hd)
-      for (int32_t r : items[i].req) count[static_cast<size_t>(r) * Hkv + hd] += pieces_of(i, hd);
-  long long run = 0;
-  for (size_t u = 0; u < static_cast<size_t>(batch) * Hkv; ++u) {
-    out_plan[off_part_off + u] = static_cast<int32_t>(run);
-    const long long c = count[u]; count[u] = run; run += c;
+// A request gained table entries since the plan was built (its kv_len moved into new pages): its own item takes the new
+// pages, everything derived from the items' sizes is written again, and the caller uploads the two stretches that
+// changed.  Host work is O(items + workers), not the regrouping of every table entry.
+extern "C" int32_t mepic_decode_plan_patch(const mepic_config_t* cfg, int32_t* plan, const int32_t* page_ids, const int32_t* pos_base,
+                                           const int32_t* kv_len, int32_t batch, int32_t table_stride,
+                                           int64_t* out_ranges, int32_t* out_n_ranges) {
+  if (!mepic_config_ok(cfg)) return MEPIC_E_INVAL;
+  if (!plan || !page_ids || !pos_base || !kv_len || !out_ranges || !out_n_ranges || batch < 1 || table_stride < 1) {
+    mepic_set_error("decode_plan_patch: bad argument"); return MEPIC_E_INVAL;
   }
-  if (run >= (1ll << 31)) { mepic_set_error("decode_plan: too many partials for the plan's 32-bit fields"); return MEPIC_E_CAPACITY; }
-  out_plan[off_part_off + static_cast<size_t>(batch) * Hkv] = static_cast<int32_t>(run);
-  h[kPhSlots] = static_cast<int32_t>(run);
-  for (size_t i = 0; i < items.size(); ++i)
-    for (int hd = 0; hd < Hkv; ++hd) {
-      const long long c = pieces_of(i, hd);
-      for (int j = 0; j < R; ++j) {
-        int32_t v = 0;
-        if (j < static_cast<int>(items[i].req.size())) {
-          long long& cur = count[static_cast<size_t>(items[i].req[j]) * Hkv + hd];
-          v = static_cast<int32_t>(cur); cur += c;
-        }
-        out_plan[off_slot_base + (i * Hkv + hd) * R + j] = v;
-      }
+  int32_t* h = plan;
+  const int R = plan_group_requests(cfg->n_q_heads / cfg->n_kv_heads);
+  if (h[kPhMagic] != kPlanMagic || h[kPhBatch] != batch || h[kPhR] != R || h[kPhPageSize] != cfg->page_size ||
+      h[kPhKvHeads] != cfg->n_kv_heads) { mepic_set_error("decode_plan_patch: the plan was built for another config or batch"); return MEPIC_E_INVAL; }
+  const int32_t P = cfg->page_size;
+  const size_t stride = kItemFixed + R;
+  int32_t* items = plan + h[kPhOffItems];
+  int32_t* req_ent = plan + h[kPhOffReqEnt];
+  const int32_t* own_item = plan + h[kPhOffOwnItem];
+  const int32_t* rec_cap = plan + h[kPhOffRecCap];
+  // first pass: can every grown request be served?  (nothing is changed before that is known)
+  bool any = false;
+  for (int32_t r = 0; r < batch; ++r) {
+    if (kv_len[r] < 1) { mepic_set_error("decode_plan_patch: kv_len[%d] = %d < 1", r, kv_len[r]); return MEPIC_E_INVAL; }
+    const int32_t now = (kv_len[r] + P - 1) / P;
+    if (now > table_stride) { mepic_set_error("decode_plan_patch: request %d needs %d entries > stride", r, now); return MEPIC_E_INVAL; }
+    if (now < req_ent[r]) { mepic_set_error("decode_plan_patch: request %d lost pages: build a new plan", r); return MEPIC_E_INVAL; }
+    if (now == req_ent[r]) continue;
+    any = true;
+    const int32_t i = own_item[r];
+    if (i < 0 || items[i * stride + kPiEnt] + (now - req_ent[r]) > rec_cap[i]) {
+      mepic_set_error("decode_plan_patch: no room left for request %d's new pages: build a new plan", r);
+      return MEPIC_E_CAPACITY;
     }
+  }
+  *out_n_ranges = 0;
+  if (!any) return MEPIC_OK;
+  int64_t rec_lo = INT64_MAX, rec_hi = 0;      // the stretch of the buffer (in ints) that holds the new records
+  for (int32_t r = 0; r < batch; ++r) {
+    const int32_t now = (kv_len[r] + P - 1) / P;
+    if (now == req_ent[r]) continue;
+    int32_t* it = items + static_cast<size_t>(own_item[r]) * stride;
+    for (int32_t e = req_ent[r]; e < now; ++e) {
+      const int64_t at = h[kPhOffRecords] + static_cast<int64_t>(it[kPiRecOff] + it[kPiEnt]) * (1 + R);
+      int32_t* q = plan + at;
+      q[0] = page_ids[static_cast<size_t>(r) * table_stride + e];
+      q[1] = pos_base[static_cast<size_t>(r) * table_stride + e];
+      for (int j = 1; j < R; ++j) q[1 + j] = 0;
+      it[kPiEnt] += 1;
+      rec_lo = std::min(rec_lo, at); rec_hi = std::max<int64_t>(rec_hi, at + 1 + R);
+    }
+    it[kPiTail] = (now - 1) * P;               // the request's last page now lives in its own item
+    req_ent[r] = now;
+  }
+  const int32_t rc = derive_plan(plan);
+  if (rc != MEPIC_OK) return rc;
+  out_ranges[0] = 0; out_ranges[1] = h[kPhOffRecords];
+  out_ranges[2] = rec_lo; out_ranges[3] = rec_hi - rec_lo;
+  *out_n_ranges = 2;
   return MEPIC_OK;
 }

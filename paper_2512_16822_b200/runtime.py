@@ -12,7 +12,7 @@ import numpy as np
 import torch
 
 from . import (Config, Segment, Store, MEPIC_SEG_CHUNK, MEPIC_SEG_PROMPT, mepic_attn_decode,
-               mepic_decode_plan_build, mepic_attn_decode_grouped, mepic_attn_decode_grouped_workspace,
+               mepic_decode_plan_build, mepic_decode_plan_patch, mepic_attn_decode_grouped, mepic_attn_decode_grouped_workspace,
                mepic_pages_quantize, mepic_attn_decode_fp8,
                mepic_attn_decode_workspace, mepic_attn_prefill, mepic_attn_prefill_fp8, mepic_attn_prefill_workspace,
                mepic_rope_table_fill)
@@ -210,8 +210,13 @@ class GroupedDecodeBatch:
         self.batch = page_ids.shape[0]
         d = dev.device
         with torch.cuda.device(d):
-            self.plan_host = mepic_decode_plan_build(cfg, page_ids, pos_base, kv_len, n_sms)
-        self.plan = torch.from_numpy(self.plan_host).to(d)
+            built = mepic_decode_plan_build(cfg, page_ids, pos_base, kv_len, n_sms)
+        # the host copy lives in page-locked memory: a patch uploads stretches of it without a staging copy
+        self._plan_pinned = torch.empty(len(built), dtype=torch.int32).pin_memory()
+        self.plan_host = self._plan_pinned.numpy()
+        self.plan_host[:] = built
+        self.plan = torch.from_numpy(built).to(d)
+        self._uploaded = None
         self.kv_len = torch.from_numpy(np.ascontiguousarray(kv_len, dtype=np.int32)).to(d)
         self.q_pos = torch.from_numpy(np.ascontiguousarray(q_pos, dtype=np.int32)).to(d)
         qshape = (self.batch, cfg.n_q_heads, cfg.head_dim)
@@ -228,6 +233,24 @@ class GroupedDecodeBatch:
                                   workspace_bytes=self.ws_bytes, status=self.dev.status, batch=self.batch,
                                   sm_scale=sm_scale, stream=s)
         return self.out
+
+    def patch(self, page_ids: np.ndarray, pos_base: np.ndarray, kv_len: np.ndarray) -> int:
+        """Requests gained pages: patch the host plan in place and upload only what changed (on the current stream).
+        Returns the bytes uploaded.  kv_len itself is the caller's per-step input and is not touched here."""
+        if self._uploaded is not None:
+            self._uploaded.synchronize()              # the previous patch's copies have read the host buffer
+        ranges = mepic_decode_plan_patch(self.dev.cfg, self.plan_host, page_ids, pos_base, kv_len)
+        sent = 0
+        for lo, n in ranges:
+            self.plan[lo:lo + n].copy_(self._plan_pinned[lo:lo + n], non_blocking=True)
+            sent += 4 * n
+        if ranges:
+            self._uploaded = torch.cuda.Event(); self._uploaded.record()
+            need = mepic_attn_decode_grouped_workspace(self.dev.cfg, self.plan_host)
+            if need > self.ws_bytes:                  # more partial slots than before: a larger workspace (rare)
+                self.ws_bytes = need + need // 8
+                self.workspace = torch.empty(self.ws_bytes, dtype=torch.uint8, device=self.dev.device)
+        return sent
 
 
 class PrefillBatch:

@@ -223,3 +223,53 @@ def test_one_dominant_key_inside_a_shared_chunk():
         assert (page_ids[r] == page).any()
         assert np.abs(got[r] - v_star).max() <= 2e-2, r
     assert not (page_ids[3] == page).any()
+
+
+def test_plan_patched_through_a_decode_loop_stays_parity_green():
+    """A serving loop: every request grows by one token per step and gains a page now and then.  The plan is built once
+    and patched (mepic_decode_plan_patch: only the changed stretches are uploaded); after every page gain, and on some
+    steps in between, the grouped result is compared with the fp64 oracle on the tables as they are then."""
+    P, Hq, Hkv, D = 16, 8, 2, 128
+    cfg, kp, vp, ids, base, kvl, q_pos, q = _shared_case(61, Hq=Hq, Hkv=Hkv, D=D, P=P, n_req=5, chunk_pages=[6, 4, 5],
+                                                         uses=[[0, 1], [1, 0], [2], [0, 2, 1], [1]], tail_tokens=[16, 5, 32, 9, 1], jitter=False)
+    rng = np.random.default_rng(62)
+    B, stride0 = ids.shape
+    steps, spare_per_req = 37, 4
+    # the tokens to come: their K/V is already in the pool (random numbers instead of the NaN poison), in pages nobody uses yet
+    for pool in (kp, vp):
+        bad = pool == 0x7FC0
+        pool[bad] = f32_to_bf16_bits(rng.standard_normal(int(bad.sum())).astype(np.float32))
+    n0 = cfg.num_pages
+    extra = lambda: f32_to_bf16_bits(rng.standard_normal((B * spare_per_req, Hkv, P, D)).astype(np.float32))
+    kp, vp = np.concatenate([kp, extra()]), np.concatenate([vp, extra()])
+    cfg = M.Config(P, Hq, Hkv, D, n0 + B * spare_per_req, cfg.max_position + (spare_per_req + 1) * P, 1e4)
+    stride = stride0 + spare_per_req
+    ids2 = np.zeros((B, stride), dtype=np.int32); base2 = np.zeros((B, stride), dtype=np.int32)
+    ids2[:, :stride0] = np.maximum(ids, 0); base2[:, :stride0] = base
+    dev = RT.Device(cfg, kp, vp)
+    gb = RT.GroupedDecodeBatch(dev, ids2, base2, kvl, q_pos, q)
+    kvl = kvl.copy()
+    next_page, gains, uploaded = n0, 0, 0
+    for step in range(steps):
+        gained = False
+        for r in range(B):
+            if kvl[r] % P == 0:
+                e = kvl[r] // P
+                ids2[r, e] = next_page; next_page += 1
+                base2[r, e] = base2[r, e - 1] + P
+                gained = True; gains += 1
+            kvl[r] += 1
+        last = kvl - 1
+        q_pos = (base2[np.arange(B), last // P] + last % P).astype(np.int32)
+        if gained:
+            uploaded += gb.patch(ids2, base2, kvl)
+        gb.kv_len.copy_(torch.from_numpy(kvl)); gb.q_pos.copy_(torch.from_numpy(q_pos))
+        out = gb.run(0.09); torch.cuda.synchronize()
+        assert dev.read_status() == 0, step
+        if gained or step % 7 == 0:
+            got = RT.bf16_bits(out)
+            for r in range(B):
+                ne = -(-int(kvl[r]) // P)
+                want = O.decode_attention_one(q[r], kp, vp, list(ids2[r, :ne]), list(base2[r, :ne]), int(kvl[r]), int(q_pos[r]), 0.09, 1e4)
+                _check(got[r], want, f"step {step} request {r}")
+    assert gains >= 2 * B and 0 < uploaded < gains * 4 * len(gb.plan_host)      # patches were made, and they were partial uploads

@@ -40,10 +40,11 @@ def _parse(plan, Hkv, P):
                 workers=workers, req_off=req_off, req_items=req_items, req_ent=req_ent, batch=batch)
 
 
-def _check_plan(cfg, page_ids, pos_base, kv_len, n_sms=148):
+def _check_plan(cfg, page_ids, pos_base, kv_len, n_sms=148, plan=None):
     P, Hkv = cfg.page_size, cfg.n_kv_heads
     G = cfg.n_q_heads // Hkv
-    plan = M.mepic_decode_plan_build(cfg, page_ids, pos_base, kv_len, n_sms)
+    if plan is None:
+        plan = M.mepic_decode_plan_build(cfg, page_ids, pos_base, kv_len, n_sms)
     pl = _parse(plan, Hkv, P)
     R, tpp = pl["R"], P // 16
     assert R == min(16 // G, 8) and pl["n_workers"] == n_sms * 8 and pl["batch"] == len(kv_len)
@@ -207,3 +208,72 @@ def test_errors():
     rc = M.lib().mepic_decode_plan_build(C.byref(c), ids.ctypes.data, base.ctypes.data, kvl.ctypes.data, 2, 4, 4,
                                          out.ctypes.data, 8, C.byref(used))
     assert rc == M.MEPIC_E_CAPACITY and used.value == len(M.mepic_decode_plan_build(cfg, ids, base, kvl, 4))
+
+
+def test_patched_plan_satisfies_every_invariant_of_a_fresh_one_step_after_step():
+    """A decode loop: every request grows by one token per step, gaining a page now and then (some requests start on a
+    full page, some in the middle of one).  After every step the plan is patched, not rebuilt, and must still cover
+    the tables as they are now exactly once, keep the tail rule, the cut and the partial slots consistent; the ranges
+    the patch reports are exactly where the buffer changed."""
+    cfg, ids, base, kvl = _tables_of(2, scale=0.25)
+    P = cfg.page_size
+    B, stride0 = ids.shape
+    grow = 40                                                           # tokens per request: 2-3 page gains each
+    stride = stride0 + 4
+    ids2 = np.zeros((B, stride), dtype=np.int32); base2 = np.zeros((B, stride), dtype=np.int32)
+    ids2[:, :stride0] = ids; base2[:, :stride0] = base
+    kvl = kvl.copy(); kvl[1] -= 5; kvl[2] -= P - 1                      # ragged starts
+    cfg = M.Config(P, cfg.n_q_heads, cfg.n_kv_heads, cfg.head_dim, cfg.num_pages + 4 * B, cfg.max_position + 4 * P, cfg.rope_theta)
+    plan = M.mepic_decode_plan_build(cfg, ids2, base2, kvl, 148)
+    _check_plan(cfg, ids2, base2, kvl, plan=plan)
+    next_page = cfg.num_pages - 4 * B
+    gains = 0
+    for step in range(grow):
+        before = plan.copy()
+        for r in range(B):
+            if kvl[r] % P == 0:                                         # the last page is full: the new token opens a page
+                e = kvl[r] // P
+                ids2[r, e] = next_page; next_page += 1
+                base2[r, e] = base2[r, e - 1] + P
+                gains += 1
+            kvl[r] += 1
+        ranges = M.mepic_decode_plan_patch(cfg, plan, ids2, base2, kvl)
+        changed = np.flatnonzero(plan != before)
+        if len(changed):
+            assert len(ranges) == 2
+            covered = np.zeros(len(plan), dtype=bool)
+            for lo, n in ranges:
+                covered[lo:lo + n] = True
+            assert covered[changed].all()
+            assert ranges[0] == (0, int(plan[7])) and ranges[1][0] >= int(plan[7])     # the derived prefix, then records
+        else:
+            assert ranges == []
+        _check_plan(cfg, ids2, base2, kvl, plan=plan)
+    assert gains >= 2 * B
+    # the patched plan stages the same pages as a plan built from scratch on the final tables
+    fresh = _parse(M.mepic_decode_plan_build(cfg, ids2, base2, kvl, 148), cfg.n_kv_heads, P)
+    mine = _parse(plan, cfg.n_kv_heads, P)
+    assert mine["total"] == fresh["total"] and mine["piece"] == fresh["piece"]
+
+
+def test_patch_refuses_what_it_cannot_do_and_changes_nothing_then():
+    cfg, ids, base, kvl = _tables_of(1)
+    P = cfg.page_size
+    B, stride0 = ids.shape
+    stride = stride0 + 40
+    ids2 = np.zeros((B, stride), dtype=np.int32); base2 = np.zeros((B, stride), dtype=np.int32)
+    ids2[:, :stride0] = ids; base2[:, :stride0] = base
+    base2[:, stride0:] = (np.arange(stride0, stride) * P)[None, :]
+    plan = M.mepic_decode_plan_build(cfg, ids2, base2, kvl, 148)
+    keep = plan.copy()
+    shrunk = kvl.copy(); shrunk[0] -= 2 * P
+    with pytest.raises(M.MepicError) as e:
+        M.mepic_decode_plan_patch(cfg, plan, ids2, base2, shrunk)
+    assert e.value.code == M.MEPIC_E_INVAL and np.array_equal(plan, keep)
+    far = kvl.copy(); far[1] += 17 * P                                  # more pages than the reserve of 16
+    with pytest.raises(M.MepicError) as e:
+        M.mepic_decode_plan_patch(cfg, plan, ids2, base2, far)
+    assert e.value.code == M.MEPIC_E_CAPACITY and np.array_equal(plan, keep)
+    ok = kvl.copy(); ok[1] += 16 * P                                    # exactly the reserve
+    assert len(M.mepic_decode_plan_patch(cfg, plan, ids2, base2, ok)) == 2
+    _check_plan(cfg, ids2, base2, ok, plan=plan)
