@@ -752,16 +752,31 @@ def measure_mixed(args, device: str):
         j1.record(s1); j2.record(s2)
         main_s.wait_event(j1); main_s.wait_event(j2)
 
+    # the same with the prefill enqueued first on a high-priority stream and the decode behind it on a low-priority one:
+    # the decode's CTAs then move in as the prefill's last wave leaves SMs idle
+    lo_p, hi_p = torch.cuda.Stream.priority_range() if hasattr(torch.cuda.Stream, "priority_range") else (0, -1)
+    s_hi, s_lo = torch.cuda.Stream(priority=hi_p), torch.cuda.Stream(priority=lo_p)
+
+    def prefill_first():
+        fork = torch.cuda.Event(); fork.record(main_s)
+        s_hi.wait_event(fork); s_lo.wait_event(fork)
+        pb.run(wl.sm_scale, s_hi)
+        db.run(wl.sm_scale, s_lo)
+        j1, j2 = torch.cuda.Event(), torch.cuda.Event()
+        j1.record(s_hi); j2.record(s_lo)
+        main_s.wait_event(j1); main_s.wait_event(j2)
+
     out = {}
     steps = max(5, min(args.steps, 10))
     for name, fn in (("decode_alone", lambda: db.run(wl.sm_scale, main_s)), ("prefill_alone", lambda: pb.run(wl.sm_scale, main_s)),
-                     ("together_two_streams", both)):
+                     ("together_two_streams", both), ("together_prefill_first_decode_low_priority", prefill_first)):
         for _ in range(2):
             fn()
         out[name] = summary(time_steps(fn, steps, flush, main_s))
     assert dev.read_status() == 0
     s = out["decode_alone"]["ms_median"] + out["prefill_alone"]["ms_median"]
-    out["together_over_sum"] = out["together_two_streams"]["ms_median"] / s
+    best = min(out["together_two_streams"]["ms_median"], out["together_prefill_first_decode_low_priority"]["ms_median"])
+    out["together_over_sum"] = best / s
     out["note"] = "medians; L2 flushed before each measurement"
     return out
 

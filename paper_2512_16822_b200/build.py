@@ -46,6 +46,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
            "-I", INCLUDE, "-I", CSRC, "-o", LIB_PATH + ".tmp"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
+    cmd += os.environ.get("MEPIC_NVCC_FLAGS", "").split()      # extra flags for experiments (e.g. -DMEPIC_DECODE_STAGES=2)
     cmd += srcs      # libcuda is NOT linked: the library must load on a machine without a driver
     proc = subprocess.run(cmd, capture_output=True, text=True)
     if proc.returncode != 0:

@@ -39,18 +39,25 @@ using namespace mepic_dev;
 
 // ---------------------------------------------------------------- the split-KV kernel
 // Warp-level tensor-core MMA (mma.sync m16n8k16, bf16 in, fp32 accumulate) for the two contractions of a tile:
-//   S^T[head][key]  = Q_tile[head][dim] . K'[key][dim]^T      A = rotated q (heads padded to 16 rows), B = rotated K
-//   O  [head][dim] += P[head][key]      . V[key][dim]         A = P straight from the S accumulators, B = V
-// so that only the rotation of K (thread-local on the B fragments: the partner dim i + D/2 sits in the fragment
-// of k-step j + D/32, same lane, same position) and the softmax stay on the CUDA cores.
+//   S^T[key][head]  = K'[key][dim] . Q^T[dim][head]           A = rotated K (16 keys = the M rows), B = rotated q (heads = N <= 8)
+//   O^T[dim][head] += V^T[dim][key] . P^T[key][head]          A = V^T by transposing ldmatrix, B = P^T (movmatrix of the S fragments)
+// The keys and the head dims fill the 16 M rows completely and the G <= 8 query heads sit in the 8 N columns, so a tile
+// costs 8 + 8 MMAs and 32 output accumulators per lane at D = 128 (with the heads as M rows, padded to 16, it was 16 + 16
+// and 64).  Only the rotation of K (thread-local on the A fragments: the partner dim i + D/2 sits in the fragment of
+// k-step j + D/32, same lane, same position) and the softmax stay on the CUDA cores.
+#ifndef MEPIC_DECODE_STAGES
+#define MEPIC_DECODE_STAGES 2
+#endif
+constexpr int kDecodeStages = MEPIC_DECODE_STAGES;     // depth of each warp's ring of staged tiles
+
 template <int D, int G>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
-  constexpr int kStages = 3;
+  constexpr int kStages = kDecodeStages;
   constexpr int NB = D / 64;                 // 64-dim blocks (128-byte swizzled rows) per K or V row
   constexpr int KS = D / 16;                 // k-steps of the QK^T contraction
   constexpr int KH = KS / 2;                 // k-steps per half: step j pairs with step j + KH
-  constexpr int ND = D / 8;                  // n-tiles of the PV product
+  constexpr int NV = D / 16;                 // 16-dim blocks of the output (M tiles of the PV product)
   constexpr int kBlockBytes = kTile * 128;   // one [16 rows x 64 dims] block
   constexpr int kStageBytes = 2 * NB * kBlockBytes;   // K blocks then V blocks
   constexpr int kWarpBytes = kStages * kStageBytes;
@@ -145,23 +152,30 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
 
   for (; issued < kStages && issued < n_tiles; ++issued) issue(issued);
 
-  // per-unit state: head g of the unit's G query heads (lanes with g >= G carry zeros)
+  // per-unit state.  The keys are the M rows of both MMAs (S^T = K' Q^T and O^T = V^T P^T), the query heads the N
+  // columns: this lane's B fragments of Q^T hold head g (lanes with g >= G carry zeros); its accumulators hold heads
+  // 2t and 2t+1 (columns) for keys g, g+8 (scores) and for dims g, g+8 of every 16-dim block (output).
   int ub = -1, uh = -1;
-  float q_lo[KH][2][2], q_hi[KH][2][2];     // un-rotated q, pre-scaled by sm_scale*log2e: pairs as for kc/ksn
-  float m_run = -INFINITY, l_run = 0.f;
-  float acc[ND][4];                         // O fragments: [n-tile][c0,c1 = head g | c2,c3 = head g+8 (unused)]
+  float q_lo[KH][2][2], q_hi[KH][2][2];     // un-rotated q of head g, pre-scaled by sm_scale*log2e: pairs as for kc/ksn
+  float m_run[2] = {-INFINITY, -INFINITY};  // running maximum of heads 2t, 2t+1 (the same in the 8 lanes that share t)
+  float l_run[2] = {0.f, 0.f};              // this lane's share (keys g, g+8 of every tile) of the two heads' sums
+  float acc[NV][4];                         // O^T fragments: [16-dim block][dim g: head 2t, 2t+1 | dim g+8: head 2t, 2t+1]
 
   auto flush = [&]() {
     if (ub < 0) return;
-    float l_tot = l_run;
-    l_tot += __shfl_xor_sync(kFull, l_tot, 1);
-    l_tot += __shfl_xor_sync(kFull, l_tot, 2);
-    const long long slot = static_cast<long long>(ub) * p.n_kv_heads + uh + w;
-    if (g < G) {
-      float* dst = p.part_o + (slot * G + g) * D;
+    float l0 = l_run[0], l1 = l_run[1];
 #pragma unroll
-      for (int nd = 0; nd < ND; ++nd) *reinterpret_cast<float2*>(dst + 8 * nd + 2 * t) = make_float2(acc[nd][0], acc[nd][1]);
-      if (t == 0) *reinterpret_cast<float2*>(p.part_ml + (slot * G + g) * 2) = make_float2(m_run, l_tot);
+    for (int o = 4; o < 32; o <<= 1) { l0 += __shfl_xor_sync(kFull, l0, o); l1 += __shfl_xor_sync(kFull, l1, o); }
+    const long long slot = static_cast<long long>(ub) * p.n_kv_heads + uh + w;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      const int hh = 2 * t + c;
+      if (hh < G) {
+        float* dst = p.part_o + (slot * G + hh) * D;
+#pragma unroll
+        for (int db = 0; db < NV; ++db) { dst[16 * db + g] = acc[db][c]; dst[16 * db + 8 + g] = acc[db][2 + c]; }
+        if (g == 0) *reinterpret_cast<float2*>(p.part_ml + (slot * G + hh) * 2) = make_float2(m_run[c], c ? l1 : l0);
+      }
     }
   };
 
@@ -185,13 +199,11 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
           q_lo[j][r][0] = lo.x * sc; q_lo[j][r][1] = lo.y * sc;
           q_hi[j][r][0] = hi.x * sc; q_hi[j][r][1] = hi.y * sc;
         }
-      m_run = -INFINITY; l_run = 0.f;
+      m_run[0] = m_run[1] = -INFINITY; l_run[0] = l_run[1] = 0.f;
 #pragma unroll
-      for (int nd = 0; nd < ND; ++nd) { acc[nd][0] = 0.f; acc[nd][1] = 0.f; acc[nd][2] = 0.f; acc[nd][3] = 0.f; }
+      for (int db = 0; db < NV; ++db) { acc[db][0] = 0.f; acc[db][1] = 0.f; acc[db][2] = 0.f; acc[db][3] = 0.f; }
     }
 
-    // ---- A fragments of the query rotated by (qpos - tile base), from the table row that came with the tile
-    uint32_t qa[KS][2];                         // [k-step][a0 (dims 16j+2t,+1) | a2 (dims 16j+8+2t,+1)], row = head g
     if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity, p.spin_limit)) {
       // Give the copies still in flight a last bounded chance to land, then leave cleanly.
       if (lane == 0) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
@@ -202,6 +214,8 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
     const uint32_t vs_addr = ks_addr + NB * kBlockBytes;
     const float sgn = meta[stage];
     const int n_valid = min(kTile, cc.kvl - cc.t * kTile);
+    // ---- B fragments of Q^T: head g rotated by (qpos - tile base), from the table row that came with the tile
+    uint32_t qa[KS][2];                         // [k-step][b0 (dims 16j+2t,+1) | b1 (dims 16j+8+2t,+1)], column = head g
     {
       const float* row = rope_rows + stage * D;
 #pragma unroll
@@ -229,67 +243,64 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
       __syncwarp();
     }
 
-    // ---- S^T = Q K'^T : B fragments by ldmatrix, rotated in registers, two key n-tiles (keys 0-7, 8-15)
-    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+    // ---- S^T = K' Q^T : A fragments of K by ldmatrix (keys g, g+8 x 16 dims), rotated in registers; two
+    // accumulators so that the MMAs of the lower and the upper half of the head dimension do not wait on each other
+    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int j = 0; j < KH; ++j) {
-      uint32_t lo[4], hi[4];      // lo: k-step j, hi: k-step j + KH; [b0 nt0, b1 nt0, b0 nt1, b1 nt1]
+      uint32_t lo[4], hi[4];      // lo: k-step j, hi: k-step j + KH; [a0 key g, a1 key g+8 | a2 key g, a3 key g+8 (dims + 8)]
       {
-        // lane -> (matrix mi = lane / 8, row = lane % 8): key = 8 (mi / 2) + row, 16-byte chunk 2 j + (mi & 1)
-        const int mi = lane >> 3, key = ((mi >> 1) << 3) + (lane & 7);
-        const int cl = 2 * j + (mi & 1), chh = 2 * (j + KH) + (mi & 1);
+        // lane -> (matrix mi = lane / 8, row = lane % 8): key = 8 (mi & 1) + row, 16-byte chunk 2 j + (mi >> 1)
+        const int mi = lane >> 3, key = ((mi & 1) << 3) + (lane & 7);
+        const int cl = 2 * j + (mi >> 1), chh = 2 * (j + KH) + (mi >> 1);
         ldmatrix_x4(lo, ks_addr + (cl / 8) * kBlockBytes + key * 128 + (((cl % 8) ^ (key & 7)) << 4));
         ldmatrix_x4(hi, ks_addr + (chh / 8) * kBlockBytes + key * 128 + (((chh % 8) ^ (key & 7)) << 4));
       }
 #pragma unroll
       for (int f = 0; f < 4; ++f) {
-        const int kq = f >> 1, r = f & 1;       // key g + 8 kq, fragment register r
+        const int kq = f & 1, r = f >> 1;       // key g + 8 kq, column half r
         const uint32_t a = lo[f], b = hi[f];
         lo[f] = bf16x2_fma(a, kc[kq][j][r], bf16x2_mul(b, kns[kq][j][r]));     // lo cos - hi sin
         hi[f] = bf16x2_fma(a, ksn[kq][j][r], bf16x2_mul(b, kc[kq][j][r]));     // lo sin + hi cos
       }
-      mma_bf16(s0, qa[j][0], 0u, qa[j][1], 0u, lo[0], lo[1]);
-      mma_bf16(s1, qa[j][0], 0u, qa[j][1], 0u, lo[2], lo[3]);
-      mma_bf16(s0, qa[j + KH][0], 0u, qa[j + KH][1], 0u, hi[0], hi[1]);
-      mma_bf16(s1, qa[j + KH][0], 0u, qa[j + KH][1], 0u, hi[2], hi[3]);
+      mma_bf16(sa, lo[0], lo[1], lo[2], lo[3], qa[j][0], qa[j][1]);
+      mma_bf16(sb, hi[0], hi[1], hi[2], hi[3], qa[j + KH][0], qa[j + KH][1]);
     }
 
-    // ---- online softmax for head g (log2 domain); this lane holds keys 2t, 2t+1, 8+2t, 9+2t
-    float sc[4] = {s0[0], s0[1], s1[0], s1[1]};
-    {
-      const int k0 = 2 * t;
-      if (k0 >= n_valid) sc[0] = -INFINITY;
-      if (k0 + 1 >= n_valid) sc[1] = -INFINITY;
-      if (k0 + 8 >= n_valid) sc[2] = -INFINITY;
-      if (k0 + 9 >= n_valid) sc[3] = -INFINITY;
+    // ---- online softmax (log2 domain): this lane holds keys g (c0, c1) and g+8 (c2, c3) of heads 2t (c0, c2), 2t+1 (c1, c3)
+    float sc[4] = {sa[0] + sb[0], sa[1] + sb[1], sa[2] + sb[2], sa[3] + sb[3]};
+    if (n_valid < kTile) {
+      if (g >= n_valid) { sc[0] = -INFINITY; sc[1] = -INFINITY; }
+      if (g + 8 >= n_valid) { sc[2] = -INFINITY; sc[3] = -INFINITY; }
     }
-    float mx = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
-    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
-    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 2));
-    if (__any_sync(kFull, mx > m_run)) {
-      const float m_new = fmaxf(m_run, mx);
-      const float alpha = ex2(m_run - m_new);     // 0 on the first tile (m_run = -inf)
-      m_run = m_new;
-      l_run *= alpha;
+    float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
+    // the running maximum moves only if some lane saw a larger score: only then is the tile's maximum worked out
+    if (__any_sync(kFull, mx0 > m_run[0] || mx1 > m_run[1])) {
 #pragma unroll
-      for (int nd = 0; nd < ND; ++nd) { acc[nd][0] *= alpha; acc[nd][1] *= alpha; }
+      for (int o = 4; o < 32; o <<= 1) { mx0 = fmaxf(mx0, __shfl_xor_sync(kFull, mx0, o)); mx1 = fmaxf(mx1, __shfl_xor_sync(kFull, mx1, o)); }
+      const float n0 = fmaxf(m_run[0], mx0), n1 = fmaxf(m_run[1], mx1);
+      const float a0 = ex2(m_run[0] - n0), a1 = ex2(m_run[1] - n1);     // 0 on the first tile (m_run = -inf)
+      m_run[0] = n0; m_run[1] = n1;
+      l_run[0] *= a0; l_run[1] *= a1;
+#pragma unroll
+      for (int db = 0; db < NV; ++db) { acc[db][0] *= a0; acc[db][1] *= a1; acc[db][2] *= a0; acc[db][3] *= a1; }
     }
-    const float p0 = ex2(sc[0] - m_run), p1 = ex2(sc[1] - m_run), p2 = ex2(sc[2] - m_run), p3 = ex2(sc[3] - m_run);
-    l_run += (p0 + p1) + (p2 + p3);
-    const uint32_t pa0 = pack_bf16x2(p0, p1), pa2 = pack_bf16x2(p2, p3);    // A fragment of P: a0 keys 2t.., a2 keys 8+2t..
+    const float p0 = ex2(sc[0] - m_run[0]), p1 = ex2(sc[1] - m_run[1]), p2 = ex2(sc[2] - m_run[0]), p3 = ex2(sc[3] - m_run[1]);
+    l_run[0] += p0 + p2; l_run[1] += p1 + p3;
+    // B fragments of P^T (keys x heads) = the transposes of the two 8 x 8 blocks this warp holds as (key row, head columns)
+    const uint32_t pb0 = movmatrix_trans(pack_bf16x2(p0, p1)), pb1 = movmatrix_trans(pack_bf16x2(p2, p3));
 
-    // ---- O += P V : B fragments of V by transposing ldmatrix, two dim n-tiles per load
+    // ---- O^T += V^T P^T : A fragments of V^T by transposing ldmatrix, one 16-dim block per MMA
 #pragma unroll
-    for (int nd = 0; nd < ND; nd += 2) {
-      uint32_t vb[4];             // [b0, b1] of n-tile nd, [b0, b1] of n-tile nd+1
+    for (int db = 0; db < NV; ++db) {
+      uint32_t va[4];             // a0 dims g x keys 0-7, a1 dims g+8 x keys 0-7, a2 dims g x keys 8-15, a3 dims g+8 x keys 8-15
       {
-        // lane -> (matrix mi, row): key = 8 (mi & 1) + row, 16-byte chunk nd + (mi >> 1)
-        const int mi = lane >> 3, key = ((mi & 1) << 3) + (lane & 7);
-        const int ch = nd + (mi >> 1);
-        ldmatrix_x4_trans(vb, vs_addr + (ch / 8) * kBlockBytes + key * 128 + (((ch % 8) ^ (key & 7)) << 4));
+        // lane -> (matrix mi, row): key = 8 (mi >> 1) + row, 16-byte chunk 2 db + (mi & 1)
+        const int mi = lane >> 3, key = ((mi >> 1) << 3) + (lane & 7);
+        const int ch = 2 * db + (mi & 1);
+        ldmatrix_x4_trans(va, vs_addr + (ch / 8) * kBlockBytes + key * 128 + (((ch % 8) ^ (key & 7)) << 4));
       }
-      mma_bf16(acc[nd], pa0, 0u, pa2, 0u, vb[0], vb[1]);
-      mma_bf16(acc[nd + 1], pa0, 0u, pa2, 0u, vb[2], vb[3]);
+      mma_bf16(acc[db], va[0], va[1], va[2], va[3], pb0, pb1);
     }
     __syncwarp();   // every lane is done with this stage
 
@@ -303,7 +314,7 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
 template <int D, int G>
 constexpr size_t decode_smem_bytes() {
   // per warp: 3 stages of (K blocks + V blocks), 3 table rows, 64 bytes of barriers and flags; 1 KB alignment slack
-  return static_cast<size_t>(kWarps) * (3 * 2 * (D / 64) * kTile * 128 + 3 * D * 4) + kWarps * 64 + 1024;
+  return static_cast<size_t>(kWarps) * (kDecodeStages * 2 * (D / 64) * kTile * 128 + kDecodeStages * D * 4) + kWarps * 64 + 1024;
 }
 
 template <int D, int G>

@@ -103,7 +103,7 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
   constexpr int D = 128;
   constexpr int kStages = 4;
   constexpr int KH = D / 32;                 // k-steps per half: 16-dim block j pairs with block j + KH
-  constexpr int ND = D / 8;                  // n-tiles of the PV product
+  constexpr int NV = D / 16;                 // 16-dim blocks of the output (M tiles of the PV product)
   constexpr int kBlockBytes = kTile * 128;   // one tile of one pool: 16 rows x 128 bytes
   constexpr int kStageBytes = 2 * kBlockBytes;
   constexpr int kWarpBytes = kStages * kStageBytes;
@@ -200,22 +200,30 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
   for (; issued < kStages && issued < n_tiles; ++issued) issue(issued);
   __syncwarp();
 
+  // The keys are the M rows of both MMAs (S^T = K' Q^T, O^T = V^T P^T) and the query heads the N columns: this lane's B
+  // fragments of Q^T hold head g; its accumulators hold heads 2t, 2t+1 for the keys key0 / key1 (scores) and for dims g,
+  // g+8 of every 16-dim block (output).
   int ub = -1, uh = -1;
-  float q_lo[KH][2][2], q_hi[KH][2][2];     // un-rotated q, pre-scaled by sm_scale*log2e: pairs as for kc/ksn
-  float m_run = -INFINITY, l_run = 0.f;
-  float acc[ND][4];                         // O fragments: [n-tile][c0,c1 = head g | c2,c3 unused]
+  float q_lo[KH][2][2], q_hi[KH][2][2];     // un-rotated q of head g, pre-scaled by sm_scale*log2e: pairs as for kc/ksn
+  float m_run[2] = {-INFINITY, -INFINITY};  // running maximum of heads 2t, 2t+1 (the same in the 8 lanes that share t)
+  float l_run[2] = {0.f, 0.f};              // this lane's share (its two keys of every tile) of the two heads' sums
+  float acc[NV][4];                         // O^T fragments: [16-dim block][dim g: head 2t, 2t+1 | dim g+8: head 2t, 2t+1]
 
   auto flush = [&]() {
     if (ub < 0) return;
-    float l_tot = l_run;
-    l_tot += __shfl_xor_sync(kFull, l_tot, 1);
-    l_tot += __shfl_xor_sync(kFull, l_tot, 2);
-    const long long slot = static_cast<long long>(ub) * p.n_kv_heads + uh + w;
-    if (g < G) {
-      float* dst = p.part_o + (slot * G + g) * D;
+    float l0 = l_run[0], l1 = l_run[1];
 #pragma unroll
-      for (int nd = 0; nd < ND; ++nd) *reinterpret_cast<float2*>(dst + 8 * nd + 2 * t) = make_float2(acc[nd][0], acc[nd][1]);
-      if (t == 0) *reinterpret_cast<float2*>(p.part_ml + (slot * G + g) * 2) = make_float2(m_run, l_tot);
+    for (int o = 4; o < 32; o <<= 1) { l0 += __shfl_xor_sync(kFull, l0, o); l1 += __shfl_xor_sync(kFull, l1, o); }
+    const long long slot = static_cast<long long>(ub) * p.n_kv_heads + uh + w;
+#pragma unroll
+    for (int c = 0; c < 2; ++c) {
+      const int hh = 2 * t + c;
+      if (hh < G) {
+        float* dst = p.part_o + (slot * G + hh) * D;
+#pragma unroll
+        for (int db = 0; db < NV; ++db) { dst[16 * db + g] = acc[db][c]; dst[16 * db + 8 + g] = acc[db][2 + c]; }
+        if (g == 0) *reinterpret_cast<float2*>(p.part_ml + (slot * G + hh) * 2) = make_float2(m_run[c], c ? l1 : l0);
+      }
     }
   };
 
@@ -239,9 +247,9 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
           q_lo[j][r][0] = lo.x * sc; q_lo[j][r][1] = lo.y * sc;
           q_hi[j][r][0] = hi.x * sc; q_hi[j][r][1] = hi.y * sc;
         }
-      m_run = -INFINITY; l_run = 0.f;
+      m_run[0] = m_run[1] = -INFINITY; l_run[0] = l_run[1] = 0.f;
 #pragma unroll
-      for (int nd = 0; nd < ND; ++nd) { acc[nd][0] = 0.f; acc[nd][1] = 0.f; acc[nd][2] = 0.f; acc[nd][3] = 0.f; }
+      for (int db = 0; db < NV; ++db) { acc[db][0] = 0.f; acc[db][1] = 0.f; acc[db][2] = 0.f; acc[db][3] = 0.f; }
     }
 
     if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity, p.spin_limit)) {
@@ -281,75 +289,75 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
       __syncwarp();
     }
 
-    // ---- S^T = Q K'^T: one ldmatrix per k-step pair brings, for both key n-tiles, 16 dims of the lower half and
-    // their partners of the upper half; widened to fp16 and rotated in registers
-    float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+    // ---- S^T = K' Q^T: one ldmatrix per k-step pair brings, for both key sets (M rows 0-7 and 8-15), 16 dims of the
+    // lower half and their partners of the upper half; widened to fp16 and rotated in registers.  Two accumulators so
+    // that the MMAs of the two halves do not wait on each other.
+    float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int j = 0; j < KH; ++j) {
-      uint32_t raw[4];            // [n-tile 0 lower, n-tile 1 lower, n-tile 0 upper, n-tile 1 upper], 4 dims each
+      uint32_t raw[4];            // [key set 0 lower, key set 1 lower, key set 0 upper, key set 1 upper], 4 dims each
       {
-        // lane -> (matrix mi = lane / 8, row = lane % 8): key of that row in n-tile (mi & 1), 16-byte chunk j (+ KH)
+        // lane -> (matrix mi = lane / 8, row = lane % 8): key of that row in key set (mi & 1), 16-byte chunk j (+ KH)
         const int mi = lane >> 3, rr = lane & 7;
         const int key = 4 * (rr >> 1) + (rr & 1) + 2 * (mi & 1);
         const int ch = j + KH * (mi >> 1);
         ldmatrix_x4(raw, ks_addr + key * 128 + ((ch ^ (key & 7)) << 4));
       }
-      uint32_t lo[4], hi[4];      // [b0 nt0, b1 nt0, b0 nt1, b1 nt1] of k-step j / j + KH
+      uint32_t lo[4], hi[4];      // [key0: dims 4t,+1 | key0: dims 4t+2,+3 | key1: ... | key1: ...] of k-step j / j + KH
       e4m3x4_to_f16x2x2(raw[0], lo[0], lo[1]);
       e4m3x4_to_f16x2x2(raw[1], lo[2], lo[3]);
       e4m3x4_to_f16x2x2(raw[2], hi[0], hi[1]);
       e4m3x4_to_f16x2x2(raw[3], hi[2], hi[3]);
 #pragma unroll
       for (int f = 0; f < 4; ++f) {
-        const int kq = f >> 1, r = f & 1;       // key of n-tile kq, fragment register r
+        const int kq = f >> 1, r = f & 1;       // key of set kq, column pair r
         const uint32_t a = lo[f], b = hi[f];
         lo[f] = f16x2_fma(a, kc[kq][j][r], f16x2_mul(b, kns[kq][j][r]));     // lo cos - hi sin
         hi[f] = f16x2_fma(a, ksn[kq][j][r], f16x2_mul(b, kc[kq][j][r]));     // lo sin + hi cos
       }
-      mma_f16(s0, qa[j][0], 0u, qa[j][1], 0u, lo[0], lo[1]);
-      mma_f16(s1, qa[j][0], 0u, qa[j][1], 0u, lo[2], lo[3]);
-      mma_f16(s0, qa[j + KH][0], 0u, qa[j + KH][1], 0u, hi[0], hi[1]);
-      mma_f16(s1, qa[j + KH][0], 0u, qa[j + KH][1], 0u, hi[2], hi[3]);
+      // A = (row g: key0, row g+8: key1) x (k columns 2t,+1 <-> dims 4t,+1 ; k columns 2t+8,+9 <-> dims 4t+2,+3)
+      mma_f16(sa, lo[0], lo[2], lo[1], lo[3], qa[j][0], qa[j][1]);
+      mma_f16(sb, hi[0], hi[2], hi[1], hi[3], qa[j + KH][0], qa[j + KH][1]);
     }
 
-    // ---- online softmax for head g (log2 domain); this lane holds keys 4t, 4t+1 (n-tile 0) and 4t+2, 4t+3 (n-tile 1)
-    float sc[4] = {s0[0] * k_scale, s0[1] * k_scale, s1[0] * k_scale, s1[1] * k_scale};
-    {
-      const int k0 = 4 * t;
-      if (k0 >= n_valid) sc[0] = -INFINITY;
-      if (k0 + 1 >= n_valid) sc[1] = -INFINITY;
-      if (k0 + 2 >= n_valid) sc[2] = -INFINITY;
-      if (k0 + 3 >= n_valid) sc[3] = -INFINITY;
+    // ---- online softmax (log2 domain): this lane holds key0 (c0, c1) and key1 (c2, c3) of heads 2t (c0, c2), 2t+1 (c1, c3)
+    float sc[4] = {(sa[0] + sb[0]) * k_scale, (sa[1] + sb[1]) * k_scale, (sa[2] + sb[2]) * k_scale, (sa[3] + sb[3]) * k_scale};
+    if (n_valid < kTile) {
+      if (key0 >= n_valid) { sc[0] = -INFINITY; sc[1] = -INFINITY; }
+      if (key1 >= n_valid) { sc[2] = -INFINITY; sc[3] = -INFINITY; }
     }
-    float mx = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
-    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 1));
-    mx = fmaxf(mx, __shfl_xor_sync(kFull, mx, 2));
-    if (__any_sync(kFull, mx > m_run)) {
-      const float m_new = fmaxf(m_run, mx);
-      const float alpha = ex2(m_run - m_new);     // 0 on the first tile (m_run = -inf)
-      m_run = m_new;
-      l_run *= alpha;
+    float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
+    // the running maximum moves only if some lane saw a larger score: only then is the tile's maximum worked out
+    if (__any_sync(kFull, mx0 > m_run[0] || mx1 > m_run[1])) {
 #pragma unroll
-      for (int nd = 0; nd < ND; ++nd) { acc[nd][0] *= alpha; acc[nd][1] *= alpha; }
+      for (int o = 4; o < 32; o <<= 1) { mx0 = fmaxf(mx0, __shfl_xor_sync(kFull, mx0, o)); mx1 = fmaxf(mx1, __shfl_xor_sync(kFull, mx1, o)); }
+      const float n0 = fmaxf(m_run[0], mx0), n1 = fmaxf(m_run[1], mx1);
+      const float a0 = ex2(m_run[0] - n0), a1 = ex2(m_run[1] - n1);     // 0 on the first tile (m_run = -inf)
+      m_run[0] = n0; m_run[1] = n1;
+      l_run[0] *= a0; l_run[1] *= a1;
+#pragma unroll
+      for (int db = 0; db < NV; ++db) { acc[db][0] *= a0; acc[db][1] *= a1; acc[db][2] *= a0; acc[db][3] *= a1; }
     }
-    const float p0 = ex2(sc[0] - m_run), p1 = ex2(sc[1] - m_run), p2 = ex2(sc[2] - m_run), p3 = ex2(sc[3] - m_run);
-    l_run += (p0 + p1) + (p2 + p3);
-    // A fragment of P, carrying the V scale of the tile: a0 = keys 4t, 4t+1 ; a2 = keys 4t+2, 4t+3
-    const uint32_t pa0 = pack_f16x2(p0 * v_scale, p1 * v_scale), pa2 = pack_f16x2(p2 * v_scale, p3 * v_scale);
+    const float p0 = ex2(sc[0] - m_run[0]), p1 = ex2(sc[1] - m_run[1]), p2 = ex2(sc[2] - m_run[0]), p3 = ex2(sc[3] - m_run[1]);
+    l_run[0] += p0 + p2; l_run[1] += p1 + p3;
+    // B fragments of P^T carrying the V scale of the tile: the transposes of the two 8 x 8 blocks (key row, head columns);
+    // row r of block 0 is key 4 (r / 2) + r % 2 and of block 1 that key + 2, so b0 = keys 4t, 4t+1 and b1 = keys 4t+2, 4t+3
+    const uint32_t pb0 = movmatrix_trans(pack_f16x2(p0 * v_scale, p1 * v_scale)), pb1 = movmatrix_trans(pack_f16x2(p2 * v_scale, p3 * v_scale));
 
-    // ---- O += P V: the transposing 8-bit ldmatrix hands this lane keys 4t..4t+3 of dims g and g + 8 of a 16-dim block
+    // ---- O^T += V^T P^T: the transposing 8-bit ldmatrix hands this lane keys 4t..4t+3 of dims g and g + 8 of a 16-dim block
 #pragma unroll
-    for (int c = 0; c < D / 16; c += 2) {
+    for (int c = 0; c < NV; c += 2) {
       uint32_t raw[4];            // [block c: dim g, dim g + 8 | block c + 1: dim g, dim g + 8]
       {
         const int key = lane & 15, ch = c + (lane >> 4);
         ldmatrix_b8_trans_x2(raw, vs_addr + key * 128 + ((ch ^ (key & 7)) << 4));
       }
 #pragma unroll
-      for (int m = 0; m < 4; ++m) {
-        uint32_t b0, b1;
-        e4m3x4_to_f16x2x2(raw[m], b0, b1);
-        mma_f16(acc[2 * c + m], pa0, 0u, pa2, 0u, b0, b1);
+      for (int k = 0; k < 2; ++k) {
+        uint32_t a0, a2, a1, a3;  // dim g: keys 4t,+1 | keys 4t+2,+3 ; dim g + 8: the same
+        e4m3x4_to_f16x2x2(raw[2 * k], a0, a2);
+        e4m3x4_to_f16x2x2(raw[2 * k + 1], a1, a3);
+        mma_f16(acc[c + k], a0, a1, a2, a3, pb0, pb1);
       }
     }
     __syncwarp();   // every lane is done with this stage

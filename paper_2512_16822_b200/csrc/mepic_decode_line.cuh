@@ -9,7 +9,10 @@
 namespace mepic_dev {
 
 constexpr int kTile = 16;      // tokens per staged tile
-constexpr int kWarps = 8;      // workers per CTA
+#ifndef MEPIC_DECODE_WARPS
+#define MEPIC_DECODE_WARPS 8
+#endif
+constexpr int kWarps = MEPIC_DECODE_WARPS;      // workers per CTA
 constexpr int kMinPiece = 4;   // never cut the line into pieces shorter than this many tiles
 
 struct DecodeParams {
