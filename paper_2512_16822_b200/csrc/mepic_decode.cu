@@ -5,7 +5,7 @@
 // Work decomposition.  The context of request b is cut into tiles of 16 tokens;
 // the (request, kv head, tile) triples of the whole batch are laid on one line
 // in that order and cut into equal contiguous pieces, one per WARP of a
-// persistent grid (one CTA per SM, 8 warps).  A warp is a self-contained
+// persistent grid (one CTA per SM, 8 or 12 warps).  A warp is a self-contained
 // worker: it owns a ring of shared-memory stages that TMA tensor copies
 // (cp.async.bulk.tensor + mbarrier complete_tx, 128-byte swizzle) fill with the
 // K tile and V tile of its next tiles, together with the one row of the cos/sin
@@ -19,9 +19,9 @@
 // the G query vectors are rotated by (qpos - tile base) in fp32 and rounded to
 // bf16, and every key only by its offset tau < 16 inside the tile, with cos/sin
 // of those 16 offsets held in registers for the whole kernel.  Both contractions
-// of a tile run on the tensor cores (mma.sync m16n8k16, fp32 accumulate); the K
-// rotation is applied to the MMA's B fragments in registers (packed bf16), so
-// rotated keys never touch shared or global memory.
+// of a tile run on the tensor cores (mma.sync m16n8k16, fp32 accumulate) with the
+// keys as the M rows; the K rotation is applied to the MMA's A fragments in
+// registers (packed bf16), so rotated keys never touch shared or global memory.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -50,8 +50,9 @@ using namespace mepic_dev;
 #endif
 constexpr int kDecodeStages = MEPIC_DECODE_STAGES;     // depth of each warp's ring of staged tiles
 
-template <int D, int G>
-__global__ void __launch_bounds__(kWarps * 32, 1)
+// W = warps per CTA (12); how many of them take part (8 or 12) is decided on the device, see cut_of_line.
+template <int D, int G, int W>
+__global__ void __launch_bounds__(W * 32, 1)
 mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
   constexpr int kStages = kDecodeStages;
   constexpr int NB = D / 64;                 // 64-dim blocks (128-byte swizzled rows) per K or V row
@@ -69,8 +70,8 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   const int wic = threadIdx.x >> 5;
   unsigned char* stage0 = smem + static_cast<size_t>(wic) * kWarpBytes;
   // after the K/V rings: per warp, per stage, the cos/sin table row the tile's query rotation needs (D floats)
-  float* rope_rows = reinterpret_cast<float*>(smem + static_cast<size_t>(kWarps) * kWarpBytes) + static_cast<size_t>(wic) * kStages * D;
-  unsigned char* misc = smem + static_cast<size_t>(kWarps) * (kWarpBytes + kStages * D * 4) + wic * 64;
+  float* rope_rows = reinterpret_cast<float*>(smem + static_cast<size_t>(W) * kWarpBytes) + static_cast<size_t>(wic) * kStages * D;
+  unsigned char* misc = smem + static_cast<size_t>(W) * (kWarpBytes + kStages * D * 4) + wic * 64;
   uint64_t* bars = reinterpret_cast<uint64_t*>(misc);                 // kStages x 8 bytes
   volatile float* meta = reinterpret_cast<volatile float*>(misc + 32);  // per stage: sign of (query position - tile base)
 
@@ -78,8 +79,10 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   const int t = lane & 3;        // fragment column group
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the merge kernel may move in as CTAs of this one retire
-  const long long w = static_cast<long long>(blockIdx.x) * kWarps + wic;
-  const Cut cut = cut_of_line(p.kv_len, p.batch, p.n_kv_heads, p.n_workers, lane);
+  const Cut cut = cut_of_line(p, lane);
+  const int w_active = cut.workers / static_cast<int>(gridDim.x);     // warps of this CTA that take part (8 or all 12)
+  if (wic >= w_active) return;
+  const long long w = static_cast<long long>(blockIdx.x) * w_active + wic;
   const long long x0 = w * cut.piece;
   if (x0 >= cut.total) return;
   const long long x1 = (x0 + cut.piece < cut.total) ? x0 + cut.piece : cut.total;
@@ -96,7 +99,7 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   // cos/sin of the in-tile offsets this lane's B fragments cover: keys g and g+8, pairs 16j + 2t + 8r + {0,1},
   // kept as packed bf16 pairs (cos, sin, -sin): the rotated K is rounded to bf16 for the MMA anyway, and packed
   // bf16 arithmetic rotates two elements per instruction without widening them first.
-  uint32_t kc[2][KH][2], ksn[2][KH][2], kns[2][KH][2];      // [key g / g+8][k-step][fragment register]
+  uint32_t kc[2][KH][2], ksn[2][KH][2];      // [key g / g+8][k-step][fragment register]
 #pragma unroll
   for (int kq = 0; kq < 2; ++kq)
 #pragma unroll
@@ -106,7 +109,6 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
         const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(g + 8 * kq) * D + 2 * (16 * j + 2 * t + 8 * r)));
         kc[kq][j][r] = pack_bf16x2(cs.x, cs.z);
         ksn[kq][j][r] = pack_bf16x2(cs.y, cs.w);
-        kns[kq][j][r] = pack_bf16x2(-cs.y, -cs.w);
       }
 
   Cursor pc = locate(p.kv_len, p.batch, p.n_kv_heads, x0, lane);   // producer cursor
@@ -156,7 +158,7 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   // columns: this lane's B fragments of Q^T hold head g (lanes with g >= G carry zeros); its accumulators hold heads
   // 2t and 2t+1 (columns) for keys g, g+8 (scores) and for dims g, g+8 of every 16-dim block (output).
   int ub = -1, uh = -1;
-  float q_lo[KH][2][2], q_hi[KH][2][2];     // un-rotated q of head g, pre-scaled by sm_scale*log2e: pairs as for kc/ksn
+  uint32_t q_lo[KH][2], q_hi[KH][2];        // un-rotated q of head g as packed bf16 pairs, pre-scaled by sm_scale*log2e: pairs as for kc/ksn
   float m_run[2] = {-INFINITY, -INFINITY};  // running maximum of heads 2t, 2t+1 (the same in the 8 lanes that share t)
   float l_run[2] = {0.f, 0.f};              // this lane's share (keys g, g+8 of every tile) of the two heads' sums
   float acc[NV][4];                         // O^T fragments: [16-dim block][dim g: head 2t, 2t+1 | dim g+8: head 2t, 2t+1]
@@ -196,8 +198,8 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
           const float2 lo = bf16x2_to_float2(__ldg(src + pair / 2));
           const float2 hi = bf16x2_to_float2(__ldg(src + (pair + D / 2) / 2));
           const float sc = g < G ? p.scale_log2 : 0.f;
-          q_lo[j][r][0] = lo.x * sc; q_lo[j][r][1] = lo.y * sc;
-          q_hi[j][r][0] = hi.x * sc; q_hi[j][r][1] = hi.y * sc;
+          q_lo[j][r] = pack_bf16x2(lo.x * sc, lo.y * sc);
+          q_hi[j][r] = pack_bf16x2(hi.x * sc, hi.y * sc);
         }
       m_run[0] = m_run[1] = -INFINITY; l_run[0] = l_run[1] = 0.f;
 #pragma unroll
@@ -212,7 +214,7 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
     }
     const uint32_t ks_addr = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
     const uint32_t vs_addr = ks_addr + NB * kBlockBytes;
-    const float sgn = meta[stage];
+    const uint32_t sgn_bits = meta[stage] < 0.f ? 0x80008000u : 0u;      // a negative angle flips the sines
     const int n_valid = min(kTile, cc.kvl - cc.t * kTile);
     // ---- B fragments of Q^T: head g rotated by (qpos - tile base), from the table row that came with the tile
     uint32_t qa[KS][2];                         // [k-step][b0 (dims 16j+2t,+1) | b1 (dims 16j+8+2t,+1)], column = head g
@@ -222,12 +224,11 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
       for (int j = 0; j < KH; ++j)
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
+          // packed bf16 arithmetic, as for the keys: the rotated query is rounded to bf16 for the MMA anyway
           const float4 cs = *reinterpret_cast<const float4*>(row + 2 * (16 * j + 2 * t + 8 * r));
-          const float c0 = cs.x, s0 = cs.y * sgn, c1 = cs.z, s1 = cs.w * sgn;
-          const float l0 = q_lo[j][r][0] * c0 - q_hi[j][r][0] * s0, h0 = q_lo[j][r][0] * s0 + q_hi[j][r][0] * c0;
-          const float l1 = q_lo[j][r][1] * c1 - q_hi[j][r][1] * s1, h1 = q_lo[j][r][1] * s1 + q_hi[j][r][1] * c1;
-          qa[j][r] = pack_bf16x2(l0, l1);
-          qa[j + KH][r] = pack_bf16x2(h0, h1);
+          const uint32_t c2 = pack_bf16x2(cs.x, cs.z), s2 = pack_bf16x2(cs.y, cs.w) ^ sgn_bits;
+          qa[j][r] = bf16x2_fma(q_lo[j][r], c2, bf16x2_neg(bf16x2_mul(q_hi[j][r], s2)));      // lo cos - hi sin
+          qa[j + KH][r] = bf16x2_fma(q_lo[j][r], s2, bf16x2_mul(q_hi[j][r], c2));            // lo sin + hi cos
         }
     }
     // rows at or past kv_len may hold anything (NaN bit patterns included): their P is 0, but 0 x NaN is NaN,
@@ -260,7 +261,7 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
       for (int f = 0; f < 4; ++f) {
         const int kq = f & 1, r = f >> 1;       // key g + 8 kq, column half r
         const uint32_t a = lo[f], b = hi[f];
-        lo[f] = bf16x2_fma(a, kc[kq][j][r], bf16x2_mul(b, kns[kq][j][r]));     // lo cos - hi sin
+        lo[f] = bf16x2_fma(a, kc[kq][j][r], bf16x2_neg(bf16x2_mul(b, ksn[kq][j][r])));     // lo cos - hi sin
         hi[f] = bf16x2_fma(a, ksn[kq][j][r], bf16x2_mul(b, kc[kq][j][r]));     // lo sin + hi cos
       }
       mma_bf16(sa, lo[0], lo[1], lo[2], lo[3], qa[j][0], qa[j][1]);
@@ -311,23 +312,28 @@ mepic_decode_splitkv(const DecodeParams p, const __grid_constant__ CUtensorMap m
   flush();
 }
 
-template <int D, int G>
+template <int D, int G, int W>
 constexpr size_t decode_smem_bytes() {
-  // per warp: 3 stages of (K blocks + V blocks), 3 table rows, 64 bytes of barriers and flags; 1 KB alignment slack
-  return static_cast<size_t>(kWarps) * (kDecodeStages * 2 * (D / 64) * kTile * 128 + kDecodeStages * D * 4) + kWarps * 64 + 1024;
+  // per warp: the stages of (K blocks + V blocks) and their table rows, 64 bytes of barriers and flags; 1 KB alignment slack
+  return static_cast<size_t>(W) * (kDecodeStages * 2 * (D / 64) * kTile * 128 + kDecodeStages * D * 4) + W * 64 + 1024;
 }
 
-template <int D, int G>
-int32_t launch_decode(const DecodeParams& p, int n_ctas, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
-  constexpr size_t smem = decode_smem_bytes<D, G>();
-  cudaError_t e = cudaFuncSetAttribute(mepic_decode_splitkv<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+template <int D, int G, int W>
+int32_t launch_decode_w(const DecodeParams& p, int n_ctas, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
+  constexpr size_t smem = decode_smem_bytes<D, G, W>();
+  cudaError_t e = cudaFuncSetAttribute(mepic_decode_splitkv<D, G, W>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("decode: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
-  mepic_decode_splitkv<D, G><<<n_ctas, kWarps * 32, smem, stream>>>(p, map_k, map_v);
+  mepic_decode_splitkv<D, G, W><<<n_ctas, W * 32, smem, stream>>>(p, map_k, map_v);
   e = launch_dependent(mepic_decode_merge<D, G>, dim3(p.batch * p.n_kv_heads), dim3(G * D), stream, p);
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("decode: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   mepic_count_launches(2);
   return MEPIC_OK;
+}
+
+template <int D, int G>
+int32_t launch_decode(const DecodeParams& p, int n_ctas, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
+  return launch_decode_w<D, G, kWarpsShared>(p, n_ctas, map_k, map_v, stream);
 }
 
 int sm_count_of_current_device() {
@@ -338,7 +344,7 @@ int sm_count_of_current_device() {
 }
 
 size_t decode_slots(const mepic_config_t* cfg, int batch, int sms) {
-  return static_cast<size_t>(batch) * cfg->n_kv_heads + static_cast<size_t>(sms) * kWarps;
+  return static_cast<size_t>(batch) * cfg->n_kv_heads + static_cast<size_t>(sms) * kMaxWarps;
 }
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -384,7 +390,7 @@ extern "C" int32_t mepic_attn_decode(const mepic_config_t* cfg, const mepic_deco
   int l2 = 0; while ((kTile << l2) < cfg->page_size) ++l2;
   p.log2_tpp = l2;
   p.num_pages = cfg->num_pages; p.max_position = cfg->max_position;
-  p.n_workers = sms * kWarps;
+  p.n_workers = sms * kWarpsShared; p.n_workers_dram = sms * kWarps;
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
   p.spin_limit = mepic_test_spin_limit(kSpinLimit); p.skip_tile = mepic_test_skip_tile();
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

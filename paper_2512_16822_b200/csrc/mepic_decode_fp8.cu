@@ -11,12 +11,15 @@
 //   * E4M3 values are exact in fp16, so codes are widened with cvt.f16x2.e4m3x2 and both
 //     contractions run as fp16 MMAs (fp32 accumulate); the scales are applied to the fp32 scores
 //     (K) and to P before it is packed (V), never to the 8-bit data;
-//   * ldmatrix (16-bit elements) on 8-bit rows hands a lane FOUR consecutive dims of a key where the
-//     bf16 layout hands it two, and the transposing 8-bit ldmatrix (m16n16) hands it four consecutive
-//     KEYS of a dim.  The MMA does not care which physical index sits at which k position as long
-//     as A and B agree, so the query fragments use the same dim order (pairs 16j + 4t + 2r), and the
-//     rows of the two key n-tiles are loaded in the order {0,1,4,5,8,9,12,13} / {2,3,6,7,10,11,14,15}
-//     so that a lane's four scores are keys 4t..4t+3 - the four keys its V fragments carry.
+//   * the keys are the M rows of both MMAs (S^T = K' Q^T, O^T = V^T P^T), the query heads the N columns, as in the
+//     bf16 kernel.  ldmatrix (16-bit elements) on 8-bit rows hands a lane FOUR consecutive dims of a key where the
+//     bf16 layout hands it two, and the transposing 8-bit ldmatrix (m16n16) hands it four consecutive KEYS of a dim.
+//     The MMA does not care which physical index sits at which k position as long as A and B agree, so the query
+//     fragments use the same dim order (pairs 16j + 4t + 2r), and the M rows of the score MMA are the keys in the
+//     order {0,1,4,5,8,9,12,13} / {2,3,6,7,10,11,14,15}: after the movmatrix transposition of the probabilities a
+//     lane's P^T fragments are keys 4t..4t+3 - the four keys its V^T fragments carry;
+//   * the query rotation runs in packed fp16 (the rotated query is rounded to fp16 for the MMA anyway), which with
+//     the halved accumulators leaves a thread at 168 registers: 12 warps per SM with a 3-stage ring each.
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -83,6 +86,7 @@ __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
   asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
+__device__ __forceinline__ uint32_t f16x2_neg(uint32_t a) { uint32_t d; asm("neg.f16x2 %0, %1;" : "=r"(d) : "r"(a)); return d; }
 __device__ __forceinline__ uint32_t f16x2_mul(uint32_t a, uint32_t b) { uint32_t d; asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b)); return d; }
 __device__ __forceinline__ uint32_t f16x2_fma(uint32_t a, uint32_t b, uint32_t c) { uint32_t d; asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c)); return d; }
 // four e4m3 codes (byte i = element i) -> two fp16 pairs, exactly
@@ -97,11 +101,16 @@ __device__ __forceinline__ void ldmatrix_b8_trans_x2(uint32_t (&r)[4], uint32_t 
                : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr) : "memory");
 }
 
+#ifndef MEPIC_FP8_STAGES
+#define MEPIC_FP8_STAGES 3
+#endif
+constexpr int kFp8Stages = MEPIC_FP8_STAGES;               // depth of each warp's ring of staged tiles
+
 template <int G>
-__global__ void __launch_bounds__(kWarps * 32, 1)
+__global__ void __launch_bounds__(kWarpsFp8 * 32, 1)
 mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
   constexpr int D = 128;
-  constexpr int kStages = 4;
+  constexpr int kStages = kFp8Stages;
   constexpr int KH = D / 32;                 // k-steps per half: 16-dim block j pairs with block j + KH
   constexpr int NV = D / 16;                 // 16-dim blocks of the output (M tiles of the PV product)
   constexpr int kBlockBytes = kTile * 128;   // one tile of one pool: 16 rows x 128 bytes
@@ -113,8 +122,8 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
   const int lane = threadIdx.x & 31;
   const int wic = threadIdx.x >> 5;
   unsigned char* stage0 = smem + static_cast<size_t>(wic) * kWarpBytes;
-  float* rope_rows = reinterpret_cast<float*>(smem + static_cast<size_t>(kWarps) * kWarpBytes) + static_cast<size_t>(wic) * kStages * D;
-  unsigned char* misc = smem + static_cast<size_t>(kWarps) * (kWarpBytes + kStages * D * 4) + wic * 128;
+  float* rope_rows = reinterpret_cast<float*>(smem + static_cast<size_t>(kWarpsFp8) * kWarpBytes) + static_cast<size_t>(wic) * kStages * D;
+  unsigned char* misc = smem + static_cast<size_t>(kWarpsFp8) * (kWarpBytes + kStages * D * 4) + wic * 128;
   uint64_t* bars = reinterpret_cast<uint64_t*>(misc);                   // kStages x 8 bytes
   volatile float* meta = reinterpret_cast<volatile float*>(misc + 32);  // per stage: sign of (q position - tile base), K scale, V scale
 
@@ -124,8 +133,8 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
   const int key0 = 4 * (g >> 1) + (g & 1), key1 = key0 + 2;
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  const long long w = static_cast<long long>(blockIdx.x) * kWarps + wic;
-  const Cut cut = cut_of_line(p.kv_len, p.batch, p.n_kv_heads, p.n_workers, lane);
+  const long long w = static_cast<long long>(blockIdx.x) * kWarpsFp8 + wic;
+  const Cut cut = cut_of_line(p, lane);
   const long long x0 = w * cut.piece;
   if (x0 >= cut.total) return;
   const long long x1 = (x0 + cut.piece < cut.total) ? x0 + cut.piece : cut.total;
@@ -139,8 +148,8 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
   }
   __syncwarp();
 
-  // cos/sin of the in-tile offsets of this lane's two keys, pairs 16j + 4t + 2r + {0,1}, as packed fp16 (cos, sin, -sin)
-  uint32_t kc[2][KH][2], ksn[2][KH][2], kns[2][KH][2];      // [n-tile][k-step][fragment register]
+  // cos/sin of the in-tile offsets of this lane's two keys, pairs 16j + 4t + 2r + {0,1}, as packed fp16 (cos, sin)
+  uint32_t kc[2][KH][2], ksn[2][KH][2];      // [key set][k-step][column pair]
 #pragma unroll
   for (int kq = 0; kq < 2; ++kq)
 #pragma unroll
@@ -150,7 +159,6 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
         const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(kq ? key1 : key0) * D + 2 * (16 * j + 4 * t + 2 * r)));
         kc[kq][j][r] = pack_f16x2(cs.x, cs.z);
         ksn[kq][j][r] = pack_f16x2(cs.y, cs.w);
-        kns[kq][j][r] = pack_f16x2(-cs.y, -cs.w);
       }
 
   Cursor pc = locate(p.kv_len, p.batch, p.n_kv_heads, x0, lane);   // producer cursor
@@ -204,7 +212,7 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
   // fragments of Q^T hold head g; its accumulators hold heads 2t, 2t+1 for the keys key0 / key1 (scores) and for dims g,
   // g+8 of every 16-dim block (output).
   int ub = -1, uh = -1;
-  float q_lo[KH][2][2], q_hi[KH][2][2];     // un-rotated q of head g, pre-scaled by sm_scale*log2e: pairs as for kc/ksn
+  uint32_t q_lo[KH][2], q_hi[KH][2];        // un-rotated q of head g as packed fp16 pairs, pre-scaled by sm_scale*log2e: pairs as for kc/ksn
   float m_run[2] = {-INFINITY, -INFINITY};  // running maximum of heads 2t, 2t+1 (the same in the 8 lanes that share t)
   float l_run[2] = {0.f, 0.f};              // this lane's share (its two keys of every tile) of the two heads' sums
   float acc[NV][4];                         // O^T fragments: [16-dim block][dim g: head 2t, 2t+1 | dim g+8: head 2t, 2t+1]
@@ -227,71 +235,37 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
     }
   };
 
+  // ---- the pieces of one tile's work, as functions of the ring stage
+  // bounded wait for a stage; on expiry the status bit is set and the other stages get one more bounded wait each
   int stage = 0;
   uint32_t parity = 0;
-  for (int it = 0; it < n_tiles; ++it) {
-    if (cc.b != ub || cc.h != uh) {
-      flush();
-      ub = cc.b; uh = cc.h;
-      const int n_q_heads = p.n_kv_heads * G;
-      const uint32_t* src = reinterpret_cast<const uint32_t*>(
-          p.q + (static_cast<size_t>(ub) * n_q_heads + static_cast<size_t>(uh) * G + (g < G ? g : 0)) * D);
+  auto landed = [&](int st, uint32_t par) {
+    if (mbar_wait_bounded(smem_u32(&bars[st]), par, p.spin_limit)) return true;
+    if (lane == 0) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
+    for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(&bars[s]), s == stage ? parity : (s < stage ? parity ^ 1u : parity), p.spin_limit);
+    return false;
+  };
+  // S^T of the tile in stage st (log2 domain, K scale applied): sc = {key0: head 2t, 2t+1 | key1: head 2t, 2t+1}
+  auto scores = [&](int st, float (&sc)[4]) {
+    const uint32_t ks_addr = smem_u32(stage0 + static_cast<size_t>(st) * kStageBytes);
+    const uint32_t sgn_bits = meta[st * 4] < 0.f ? 0x80008000u : 0u;     // a negative angle flips the sines
+    const float k_scale = meta[st * 4 + 1];
+    // B fragments of Q^T: head g rotated by (qpos - tile base), fp16, from the table row that came with the tile
+    uint32_t qa[2 * KH][2];                     // [k-step][b0 (dims 16j+4t,+1) | b1 (dims 16j+4t+2,+3)], column = head g
+    const float* row = rope_rows + st * D;
 #pragma unroll
-      for (int j = 0; j < KH; ++j)
+    for (int j = 0; j < KH; ++j)
 #pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          const int pair = 16 * j + 4 * t + 2 * r;              // dims pair, pair+1 and their partners + D/2
-          const float2 lo = bf16x2_to_float2(__ldg(src + pair / 2));
-          const float2 hi = bf16x2_to_float2(__ldg(src + (pair + D / 2) / 2));
-          const float sc = g < G ? p.scale_log2 : 0.f;
-          q_lo[j][r][0] = lo.x * sc; q_lo[j][r][1] = lo.y * sc;
-          q_hi[j][r][0] = hi.x * sc; q_hi[j][r][1] = hi.y * sc;
-        }
-      m_run[0] = m_run[1] = -INFINITY; l_run[0] = l_run[1] = 0.f;
-#pragma unroll
-      for (int db = 0; db < NV; ++db) { acc[db][0] = 0.f; acc[db][1] = 0.f; acc[db][2] = 0.f; acc[db][3] = 0.f; }
-    }
-
-    if (!mbar_wait_bounded(smem_u32(&bars[stage]), parity, p.spin_limit)) {
-      if (lane == 0) atomicOr(p.status, MEPIC_DEV_WAIT_EXPIRED);
-      for (int s = 0; s < kStages; ++s) mbar_wait_bounded(smem_u32(&bars[s]), s == stage ? parity : (s < stage ? parity ^ 1u : parity), p.spin_limit);
-      return;
-    }
-    const uint32_t ks_addr = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
-    const uint32_t vs_addr = ks_addr + kBlockBytes;
-    const float sgn = meta[stage * 4], k_scale = meta[stage * 4 + 1], v_scale = meta[stage * 4 + 2];
-    const int n_valid = min(kTile, cc.kvl - cc.t * kTile);
-    // ---- A fragments of the query rotated by (qpos - tile base), fp16
-    uint32_t qa[2 * KH][2];                     // [k-step][a0 (dims 16j+4t,+1) | a2 (dims 16j+4t+2,+3)], row = head g
-    {
-      const float* row = rope_rows + stage * D;
-#pragma unroll
-      for (int j = 0; j < KH; ++j)
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-          const float4 cs = *reinterpret_cast<const float4*>(row + 2 * (16 * j + 4 * t + 2 * r));
-          const float c0 = cs.x, s0 = cs.y * sgn, c1 = cs.z, s1 = cs.w * sgn;
-          const float l0 = q_lo[j][r][0] * c0 - q_hi[j][r][0] * s0, h0 = q_lo[j][r][0] * s0 + q_hi[j][r][0] * c0;
-          const float l1 = q_lo[j][r][1] * c1 - q_hi[j][r][1] * s1, h1 = q_lo[j][r][1] * s1 + q_hi[j][r][1] * c1;
-          qa[j][r] = pack_f16x2(l0, l1);
-          qa[j + KH][r] = pack_f16x2(h0, h1);
-        }
-    }
-    // slots at or past kv_len may hold any code (NaN included): P is 0 there, but 0 x NaN is NaN, so V must be finite
-    if (n_valid < kTile) {
-      for (int idx = n_valid * 8 + lane; idx < kTile * 8; idx += 32) {
-        const int key = idx / 8, ch = idx % 8;
-        const uint32_t a = vs_addr + key * 128 + ((ch ^ (key & 7)) << 4);
-        asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
+      for (int r = 0; r < 2; ++r) {
+        // packed fp16 arithmetic: the rotated query is rounded to fp16 for the MMA anyway
+        const float4 cs = *reinterpret_cast<const float4*>(row + 2 * (16 * j + 4 * t + 2 * r));
+        const uint32_t c2 = pack_f16x2(cs.x, cs.z), s2 = pack_f16x2(cs.y, cs.w) ^ sgn_bits;
+        qa[j][r] = f16x2_fma(q_lo[j][r], c2, f16x2_neg(f16x2_mul(q_hi[j][r], s2)));       // lo cos - hi sin
+        qa[j + KH][r] = f16x2_fma(q_lo[j][r], s2, f16x2_mul(q_hi[j][r], c2));             // lo sin + hi cos
       }
-      // these generic-proxy stores must be ordered before the TMA (async proxy) write that refills this stage
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncwarp();
-    }
-
-    // ---- S^T = K' Q^T: one ldmatrix per k-step pair brings, for both key sets (M rows 0-7 and 8-15), 16 dims of the
-    // lower half and their partners of the upper half; widened to fp16 and rotated in registers.  Two accumulators so
-    // that the MMAs of the two halves do not wait on each other.
+    // one ldmatrix per k-step pair brings, for both key sets (M rows 0-7 and 8-15), 16 dims of the lower half and their
+    // partners of the upper half; widened to fp16 and rotated in registers.  Two accumulators so that the MMAs of the
+    // two halves do not wait on each other.
     float sa[4] = {0.f, 0.f, 0.f, 0.f}, sb[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
     for (int j = 0; j < KH; ++j) {
@@ -312,39 +286,39 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
       for (int f = 0; f < 4; ++f) {
         const int kq = f >> 1, r = f & 1;       // key of set kq, column pair r
         const uint32_t a = lo[f], b = hi[f];
-        lo[f] = f16x2_fma(a, kc[kq][j][r], f16x2_mul(b, kns[kq][j][r]));     // lo cos - hi sin
-        hi[f] = f16x2_fma(a, ksn[kq][j][r], f16x2_mul(b, kc[kq][j][r]));     // lo sin + hi cos
+        lo[f] = f16x2_fma(a, kc[kq][j][r], f16x2_neg(f16x2_mul(b, ksn[kq][j][r])));     // lo cos - hi sin
+        hi[f] = f16x2_fma(a, ksn[kq][j][r], f16x2_mul(b, kc[kq][j][r]));                // lo sin + hi cos
       }
       // A = (row g: key0, row g+8: key1) x (k columns 2t,+1 <-> dims 4t,+1 ; k columns 2t+8,+9 <-> dims 4t+2,+3)
       mma_f16(sa, lo[0], lo[2], lo[1], lo[3], qa[j][0], qa[j][1]);
       mma_f16(sb, hi[0], hi[2], hi[1], hi[3], qa[j + KH][0], qa[j + KH][1]);
     }
-
-    // ---- online softmax (log2 domain): this lane holds key0 (c0, c1) and key1 (c2, c3) of heads 2t (c0, c2), 2t+1 (c1, c3)
-    float sc[4] = {(sa[0] + sb[0]) * k_scale, (sa[1] + sb[1]) * k_scale, (sa[2] + sb[2]) * k_scale, (sa[3] + sb[3]) * k_scale};
-    if (n_valid < kTile) {
-      if (key0 >= n_valid) { sc[0] = -INFINITY; sc[1] = -INFINITY; }
-      if (key1 >= n_valid) { sc[2] = -INFINITY; sc[3] = -INFINITY; }
-    }
-    float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
-    // the running maximum moves only if some lane saw a larger score: only then is the tile's maximum worked out
-    if (__any_sync(kFull, mx0 > m_run[0] || mx1 > m_run[1])) {
 #pragma unroll
-      for (int o = 4; o < 32; o <<= 1) { mx0 = fmaxf(mx0, __shfl_xor_sync(kFull, mx0, o)); mx1 = fmaxf(mx1, __shfl_xor_sync(kFull, mx1, o)); }
-      const float n0 = fmaxf(m_run[0], mx0), n1 = fmaxf(m_run[1], mx1);
-      const float a0 = ex2(m_run[0] - n0), a1 = ex2(m_run[1] - n1);     // 0 on the first tile (m_run = -inf)
-      m_run[0] = n0; m_run[1] = n1;
-      l_run[0] *= a0; l_run[1] *= a1;
-#pragma unroll
-      for (int db = 0; db < NV; ++db) { acc[db][0] *= a0; acc[db][1] *= a1; acc[db][2] *= a0; acc[db][3] *= a1; }
+    for (int k = 0; k < 4; ++k) sc[k] = (sa[k] + sb[k]) * k_scale;
+  };
+  // slots at or past kv_len may hold any code (NaN included): P is 0 there, but 0 x NaN is NaN, so V must be finite;
+  // their scores are masked
+  auto tail = [&](int st, int n_valid, float (&sc)[4]) {
+    const uint32_t vs_addr = smem_u32(stage0 + static_cast<size_t>(st) * kStageBytes) + kBlockBytes;
+    for (int idx = n_valid * 8 + lane; idx < kTile * 8; idx += 32) {
+      const int key = idx / 8, ch = idx % 8;
+      const uint32_t a = vs_addr + key * 128 + ((ch ^ (key & 7)) << 4);
+      asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
     }
-    const float p0 = ex2(sc[0] - m_run[0]), p1 = ex2(sc[1] - m_run[1]), p2 = ex2(sc[2] - m_run[0]), p3 = ex2(sc[3] - m_run[1]);
-    l_run[0] += p0 + p2; l_run[1] += p1 + p3;
+    // these generic-proxy stores must be ordered before the TMA (async proxy) write that refills this stage
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    __syncwarp();
+    if (key0 >= n_valid) { sc[0] = -INFINITY; sc[1] = -INFINITY; }
+    if (key1 >= n_valid) { sc[2] = -INFINITY; sc[3] = -INFINITY; }
+  };
+  // O^T += V^T P^T for the tile in stage st; p = the tile's four probabilities of this lane (V scale not yet applied)
+  auto pv = [&](int st, float p0, float p1, float p2, float p3) {
+    const uint32_t vs_addr = smem_u32(stage0 + static_cast<size_t>(st) * kStageBytes) + kBlockBytes;
+    const float v_scale = meta[st * 4 + 2];
     // B fragments of P^T carrying the V scale of the tile: the transposes of the two 8 x 8 blocks (key row, head columns);
     // row r of block 0 is key 4 (r / 2) + r % 2 and of block 1 that key + 2, so b0 = keys 4t, 4t+1 and b1 = keys 4t+2, 4t+3
     const uint32_t pb0 = movmatrix_trans(pack_f16x2(p0 * v_scale, p1 * v_scale)), pb1 = movmatrix_trans(pack_f16x2(p2 * v_scale, p3 * v_scale));
-
-    // ---- O^T += V^T P^T: the transposing 8-bit ldmatrix hands this lane keys 4t..4t+3 of dims g and g + 8 of a 16-dim block
+    // the transposing 8-bit ldmatrix hands this lane keys 4t..4t+3 of dims g and g + 8 of a 16-dim block
 #pragma unroll
     for (int c = 0; c < NV; c += 2) {
       uint32_t raw[4];            // [block c: dim g, dim g + 8 | block c + 1: dim g, dim g + 8]
@@ -360,18 +334,66 @@ mepic_decode_splitkv_fp8(const DecodeParams p, const __grid_constant__ CUtensorM
         mma_f16(acc[c + k], a0, a1, a2, a3, pb0, pb1);
       }
     }
-    __syncwarp();   // every lane is done with this stage
+  };
+  // the running maxima move only if some lane saw a larger score: only then is the maximum over the lanes worked out
+  auto raise = [&](float mx0, float mx1) {
+    if (!__any_sync(kFull, mx0 > m_run[0] || mx1 > m_run[1])) return;
+#pragma unroll
+    for (int o = 4; o < 32; o <<= 1) { mx0 = fmaxf(mx0, __shfl_xor_sync(kFull, mx0, o)); mx1 = fmaxf(mx1, __shfl_xor_sync(kFull, mx1, o)); }
+    const float n0 = fmaxf(m_run[0], mx0), n1 = fmaxf(m_run[1], mx1);
+    const float a0 = ex2(m_run[0] - n0), a1 = ex2(m_run[1] - n1);     // 0 on the first tile (m_run = -inf)
+    m_run[0] = n0; m_run[1] = n1;
+    l_run[0] *= a0; l_run[1] *= a1;
+#pragma unroll
+    for (int db = 0; db < NV; ++db) { acc[db][0] *= a0; acc[db][1] *= a1; acc[db][2] *= a0; acc[db][3] *= a1; }
+  };
 
-    if (issued < n_tiles) { issue(stage); ++issued; }
-    advance(cc, p.kv_len, p.batch, p.n_kv_heads);
-    if (++stage == kStages) { stage = 0; parity ^= 1u; }
+  int it = 0;
+  while (it < n_tiles) {
+    if (cc.b != ub || cc.h != uh) {
+      flush();
+      ub = cc.b; uh = cc.h;
+      const int n_q_heads = p.n_kv_heads * G;
+      const uint32_t* src = reinterpret_cast<const uint32_t*>(
+          p.q + (static_cast<size_t>(ub) * n_q_heads + static_cast<size_t>(uh) * G + (g < G ? g : 0)) * D);
+#pragma unroll
+      for (int j = 0; j < KH; ++j)
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+          const int pair = 16 * j + 4 * t + 2 * r;              // dims pair, pair+1 and their partners + D/2
+          const float2 lo = bf16x2_to_float2(__ldg(src + pair / 2));
+          const float2 hi = bf16x2_to_float2(__ldg(src + (pair + D / 2) / 2));
+          const float sc = g < G ? p.scale_log2 : 0.f;
+          q_lo[j][r] = pack_f16x2(lo.x * sc, lo.y * sc);
+          q_hi[j][r] = pack_f16x2(hi.x * sc, hi.y * sc);
+        }
+      m_run[0] = m_run[1] = -INFINITY; l_run[0] = l_run[1] = 0.f;
+#pragma unroll
+      for (int db = 0; db < NV; ++db) { acc[db][0] = 0.f; acc[db][1] = 0.f; acc[db][2] = 0.f; acc[db][3] = 0.f; }
+    }
+    if (!landed(stage, parity)) return;
+    {
+      float sA[4];
+      scores(stage, sA);
+      const int n_valid = min(kTile, cc.kvl - cc.t * kTile);
+      if (n_valid < kTile) tail(stage, n_valid, sA);
+      raise(fmaxf(sA[0], sA[2]), fmaxf(sA[1], sA[3]));
+      const float a0 = ex2(sA[0] - m_run[0]), a1 = ex2(sA[1] - m_run[1]), a2 = ex2(sA[2] - m_run[0]), a3 = ex2(sA[3] - m_run[1]);
+      l_run[0] += a0 + a2; l_run[1] += a1 + a3;
+      pv(stage, a0, a1, a2, a3);
+      __syncwarp();   // every lane is done with this stage
+      if (issued < n_tiles) { issue(stage); ++issued; }
+      advance(cc, p.kv_len, p.batch, p.n_kv_heads);
+      it += 1;
+      if (++stage == kStages) { stage = 0; parity ^= 1u; }
+    }
   }
   flush();
 }
 
 constexpr size_t fp8_smem_bytes() {
   // per warp: 4 stages of (K tile + V tile), 4 table rows, 128 bytes of barriers and per-stage scalars; 1 KB alignment slack
-  return static_cast<size_t>(kWarps) * (4 * 2 * kTile * 128 + 4 * 128 * 4) + kWarps * 128 + 1024;
+  return static_cast<size_t>(kWarpsFp8) * (kFp8Stages * 2 * kTile * 128 + kFp8Stages * 128 * 4) + kWarpsFp8 * 128 + 1024;
 }
 
 template <int G>
@@ -379,7 +401,7 @@ int32_t launch_fp8(const DecodeParams& p, int n_ctas, const CUtensorMap& map_k, 
   constexpr size_t smem = fp8_smem_bytes();
   cudaError_t e = cudaFuncSetAttribute(mepic_decode_splitkv_fp8<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("decode_fp8: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
-  mepic_decode_splitkv_fp8<G><<<n_ctas, kWarps * 32, smem, stream>>>(p, map_k, map_v);
+  mepic_decode_splitkv_fp8<G><<<n_ctas, kWarpsFp8 * 32, smem, stream>>>(p, map_k, map_v);
   e = launch_dependent(mepic_decode_merge<128, G>, dim3(p.batch * p.n_kv_heads), dim3(G * 128), stream, p);
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("decode_fp8: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
@@ -429,7 +451,7 @@ extern "C" int32_t mepic_attn_decode_fp8(const mepic_config_t* cfg, const mepic_
   const int sms = sm_count_of_current_device();
   if (sms <= 0) { mepic_set_error("decode_fp8: no CUDA device"); return MEPIC_E_CUDA; }
   const int G = cfg->n_q_heads / cfg->n_kv_heads, D = cfg->head_dim;
-  const size_t slots = static_cast<size_t>(a->batch) * cfg->n_kv_heads + static_cast<size_t>(sms) * kWarps;
+  const size_t slots = static_cast<size_t>(a->batch) * cfg->n_kv_heads + static_cast<size_t>(sms) * kMaxWarps;
   const size_t need = slots * G * (D + 2) * sizeof(float);      // the same as mepic_attn_decode_workspace
   if (a->workspace_bytes < need) { mepic_set_error("decode_fp8: workspace %zu < %zu bytes", a->workspace_bytes, need); return MEPIC_E_INVAL; }
 
@@ -449,7 +471,7 @@ extern "C" int32_t mepic_attn_decode_fp8(const mepic_config_t* cfg, const mepic_
   int l2 = 0; while ((kTile << l2) < cfg->page_size) ++l2;
   p.log2_tpp = l2;
   p.num_pages = cfg->num_pages; p.max_position = cfg->max_position;
-  p.n_workers = sms * kWarps;
+  p.n_workers = sms * kWarpsFp8; p.n_workers_dram = p.n_workers;       // half the bytes per tile: never DRAM-bound
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
   p.spin_limit = mepic_test_spin_limit(kSpinLimit); p.skip_tile = mepic_test_skip_tile();
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);

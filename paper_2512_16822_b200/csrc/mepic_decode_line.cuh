@@ -12,7 +12,13 @@ constexpr int kTile = 16;      // tokens per staged tile
 #ifndef MEPIC_DECODE_WARPS
 #define MEPIC_DECODE_WARPS 8
 #endif
-constexpr int kWarps = MEPIC_DECODE_WARPS;      // workers per CTA
+constexpr int kWarps = MEPIC_DECODE_WARPS;      // warps per CTA of the bf16 kernel that take part when every byte may come from DRAM
+constexpr int kWarpsShared = 12;                // ... and when the requests are known to alias pages (see cut_of_line)
+#ifndef MEPIC_FP8_WARPS
+#define MEPIC_FP8_WARPS 12
+#endif
+constexpr int kWarpsFp8 = MEPIC_FP8_WARPS;      // ... of the 8-bit kernel (half the bytes per stage, fewer registers: room for more)
+constexpr int kMaxWarps = kWarpsFp8 > kWarpsShared ? kWarpsFp8 : kWarpsShared;   // the workspace holds a partial per worker of either kernel
 constexpr int kMinPiece = 4;   // never cut the line into pieces shorter than this many tiles
 
 struct DecodeParams {
@@ -31,6 +37,7 @@ struct DecodeParams {
   uint16_t* out;
   int32_t* status;
   int table_stride, batch, n_kv_heads, page_size, log2_tpp, num_pages, max_position, n_workers;
+  int n_workers_dram;   // workers used when the batch cannot be known to alias pages (see cut_of_line); <= n_workers
   int spin_limit;   // polls before a bounded wait gives up
   int skip_tile;    // test hook: worker 0 leaves out the staged copy of its tile with this index (-1: none)
   float scale_log2;   // sm_scale * log2(e)
@@ -44,16 +51,24 @@ __device__ __forceinline__ int warp_sum(int v) {
 __device__ __forceinline__ int tiles_of(int kv_len) { return kv_len > 0 ? (kv_len + kTile - 1) / kTile : 0; }
 
 // The cut of the tile line, recomputed by every warp from kv_len (no host mirror, no plan upload).
-struct Cut { long long total; long long piece; };
-__device__ __forceinline__ Cut cut_of_line(const int32_t* kv_len, int batch, int n_kv_heads, int n_workers, int lane) {
+//
+// How many workers take part is decided here as well, the same way by every warp of both kernels.  The decode has two
+// regimes: when every byte comes from DRAM it is bound by DRAM, and more tiles in flight than n_workers_dram workers
+// keep there only lower the DRAM rate; when requests alias pages most tile loads are L2 hits, the kernel is bound by
+// the latency of its own dependent instructions and all n_workers help.  If the batch has at least 1.5 table entries
+// per page of the pool its requests must alias pages, and all workers run; otherwise only the first n_workers_dram
+// (the warps beyond them in each CTA leave at once).
+struct Cut { long long total; long long piece; int workers; };
+__device__ __forceinline__ Cut cut_of_line(const DecodeParams& p, int lane) {
   long long tiles = 0;
-  for (int b0 = 0; b0 < batch; b0 += 32) {
-    const int n = (b0 + lane < batch) ? tiles_of(kv_len[b0 + lane]) : 0;
+  for (int b0 = 0; b0 < p.batch; b0 += 32) {
+    const int n = (b0 + lane < p.batch) ? tiles_of(p.kv_len[b0 + lane]) : 0;
     tiles += warp_sum(n);
   }
   Cut c;
-  c.total = tiles * n_kv_heads;
-  long long piece = (c.total + n_workers - 1) / n_workers;
+  c.total = tiles * p.n_kv_heads;
+  c.workers = 2 * (tiles >> p.log2_tpp) >= 3ll * p.num_pages ? p.n_workers : p.n_workers_dram;
+  long long piece = (c.total + c.workers - 1) / c.workers;
   c.piece = piece < kMinPiece ? kMinPiece : piece;
   return c;
 }
@@ -109,7 +124,7 @@ __global__ void mepic_decode_merge(const DecodeParams p) {
   const int lane = threadIdx.x & 31;
   __shared__ long long sh[3];
   if (threadIdx.x < 32) {
-    const Cut cut = cut_of_line(p.kv_len, p.batch, p.n_kv_heads, p.n_workers, lane);
+    const Cut cut = cut_of_line(p, lane);
     long long before = 0;
     for (int b0 = 0; b0 < b; b0 += 32) {
       const int n = (b0 + lane < b) ? tiles_of(p.kv_len[b0 + lane]) : 0;
