@@ -1008,8 +1008,11 @@ def run_ours(args):
                 "traffic": tr["dram_bytes_per_launch"] if tr else None, "traffic_source": tr,
                 "effective": {"achieved": effective, "frac": effective / peak, "frac_of_nominal_8TBs": effective / NOMINAL_HBM_GBS,
                               "what": "this line's value: logical bytes / time on the shared layout; includes L2 hits on shared pages"}}
+    roofline["effective"]["traffic"] = roofline["traffic"]
     if unshared is not None:
         # the DRAM-honest figure: the same kernel and the same logical bytes on the layout where no byte can come from L2
+        tru = ncu_traffic("mepic_decode_splitkv_unshared", f"config{args.config}")
+        roofline.update({"traffic": tru["dram_bytes_per_launch"] if tru else None, "traffic_source": tru})
         roofline.update({"achieved": unshared["value"], "frac": unshared["value"] / peak,
                          "frac_of_nominal_8TBs": unshared["value"] / NOMINAL_HBM_GBS,
                          "what": "unshared layout of the same batch (unshared_layout.ms_per_step): every byte comes from DRAM"})

@@ -77,7 +77,8 @@ def test_scaled_configs_all_elements(cfg_index, scale):
     _run_decode(make_workload(cfg_index, scale=scale))
 
 
-@pytest.mark.parametrize("cfg_index,sample", [(2, [0, 13, 31]), (4, [0, 7]), (5, [0, 1, 64, 127])])
+@pytest.mark.parametrize("cfg_index,sample", [(2, [0, 3, 7, 11, 13, 18, 22, 26, 29, 31]), (4, [0, 2, 5, 7]),
+                                               (5, [0, 1, 9, 23, 40, 64, 77, 90, 101, 113, 120, 127])])
 def test_full_size_configs_sampled_requests(cfg_index, sample):
     # The full configuration in the launch shape the benchmark times; the oracle checks whole sampled requests.
     _run_decode(make_workload(cfg_index), sample=sample)

@@ -157,11 +157,12 @@ def test_config3_scaled_all_rows():
 
 def test_config3_full_sampled_rows():
     # 8 requests x 768 rows over 16 640 cached tokens; the oracle checks sampled rows of every request
-    _config_run(3, 1.0, lambda R: [0, 1, 15, 16, 255, 256, R // 2, R - 257, R - 256, R - 2, R - 1])
+    # the corners (first rows, chunk-block boundaries, the question's first and last rows) plus every 13th row
+    _config_run(3, 1.0, lambda R: [0, 1, 15, 16, 255, 256, R // 2, R - 257, R - 256, R - 2, R - 1] + list(range(5, R, 13)))
 
 
 def test_config5_prefill_part_sampled_rows():
-    _config_run(5, 1.0, lambda R: [0, 15, 16, 100, R // 2, R - 1793, R - 1792, R - 1])
+    _config_run(5, 1.0, lambda R: [0, 15, 16, 100, R // 2, R - 1793, R - 1792, R - 1] + list(range(7, R, 41)))
 
 
 def test_bad_slot_and_bad_page_are_reported_not_faulted():
