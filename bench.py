@@ -620,6 +620,19 @@ def measure_variant(kind: str, args, wl, dev, tabs, q_bits, logical_bytes: int, 
                   "pages_per_GB_bf16": int(1e9 // (wl.page_size * kv_bytes_per_token(wl))),
                   "note": "e4m3 pages + fp32 scale per (page, kv head): half the K/V bytes of bf16 per context token; "
                           "value = 8-bit bytes / time; L2 flushed between steps"})
+        # the sharing-aware path over the same 8-bit pools
+        from paper_2512_16822_b200 import runtime as RT
+        gb = RT.Fp8GroupedDecodeBatch(batch.pools, page_ids, pos_base, kv_len, q_pos, q_bits)
+        for _ in range(3):
+            gb.run(wl.sm_scale, stream)
+        gms = summary(time_steps(lambda: gb.run(wl.sm_scale, stream), steps, flush, stream))
+        assert dev.read_status() == 0
+        staged = int(gb.plan_host[12]) * wl.page_size * bpt
+        gms.update({"value": tokens * bpt / (gms["ms_per_step"] * 1e-3) / 1e9, "unit": "GB/s",
+                    "staged_gbs": staged / (gms["ms_per_step"] * 1e-3) / 1e9,
+                    "note": "mepic_attn_decode_grouped_fp8: value = 8-bit bytes of the per-request decode / time"})
+        d["grouped"] = gms
+        del gb
     del batch
     return d
 

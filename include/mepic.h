@@ -482,6 +482,12 @@ typedef struct {
 size_t  mepic_attn_prefill_workspace(const mepic_config_t* cfg, int32_t batch, const int32_t* row_offsets_host);
 int32_t mepic_attn_prefill(const mepic_config_t* cfg, const mepic_prefill_args_t* args, void* cuda_stream);
 
+/* mepic_attn_decode_grouped_fp8: mepic_attn_decode_grouped over 8-bit pools (args->k_pool / v_pool are the e4m3 pools,
+ * k_scales / v_scales (DEVICE) their scales); plan, workspace and every other field as for mepic_attn_decode_grouped,
+ * what is computed and the tolerance as for mepic_attn_decode_fp8.  head_dim must be 128. */
+int32_t mepic_attn_decode_grouped_fp8(const mepic_config_t* cfg, const mepic_decode_grouped_args_t* args, const float* k_scales,
+                                      const float* v_scales, void* cuda_stream);
+
 /*
  * mepic_attn_prefill_fp8 - mepic_attn_prefill over 8-bit (e4m3) pools: Sections 3.3.1-3.3.3 with the KV-cache
  * quantisation the paper's related-work section calls combinable.  args->k_pool / v_pool are the 8-bit pools

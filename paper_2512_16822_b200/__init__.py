@@ -25,7 +25,7 @@ __all__ = [
     "mepic_request_release", "mepic_chunk_mark_uncomputed", "mepic_store_stats", "mepic_store_attach_remote", "mepic_store_test_hooks", "mepic_kernel_test_hooks", "mepic_rope_table_floats", "mepic_rope_table_fill",
     "mepic_attn_decode_workspace", "mepic_attn_decode", "mepic_attn_decode_static",
     "mepic_pages_quantize", "mepic_attn_decode_fp8", "mepic_decode_plan_max_ints", "mepic_decode_plan_build", "mepic_decode_plan_patch", "mepic_attn_decode_grouped_workspace",
-    "mepic_attn_decode_grouped",
+    "mepic_attn_decode_grouped", "mepic_attn_decode_grouped_fp8",
     "MEPIC_DECODE_STATIC_SCRATCH_BYTES", "mepic_attn_prefill_workspace",
     "mepic_attn_prefill", "mepic_attn_prefill_fp8", "mepic_last_error", "mepic_launch_count",
     "MEPIC_OK", "MEPIC_E_INVAL", "MEPIC_E_NOSPACE", "MEPIC_E_NOTFOUND", "MEPIC_E_CAPACITY",
@@ -153,6 +153,7 @@ _PROTOTYPES = {
                                             C.c_int32, C.c_void_p, C.POINTER(C.c_int32)]),
     "mepic_attn_decode_grouped_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_void_p]),
     "mepic_attn_decode_grouped": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeGroupedArgsC), C.c_void_p]),
+    "mepic_attn_decode_grouped_fp8": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_DecodeGroupedArgsC), C.c_void_p, C.c_void_p, C.c_void_p]),
     "mepic_attn_prefill_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32, C.c_void_p]),
     "mepic_attn_prefill": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_PrefillArgsC), C.c_void_p]),
     "mepic_attn_prefill_fp8": (C.c_int32, [C.POINTER(_ConfigC), C.POINTER(_PrefillArgsC), C.c_void_p, C.c_void_p, C.c_void_p]),
@@ -494,3 +495,14 @@ def mepic_attn_prefill_fp8(cfg: Config, *, q_new, k_new, v_new, row_offsets, q_s
                       sm_scale)
     c = cfg.c()
     _check(lib().mepic_attn_prefill_fp8(C.byref(c), C.byref(a), _ptr(k_scales), _ptr(v_scales), _stream_ptr(stream)))
+
+
+def mepic_attn_decode_grouped_fp8(cfg: Config, *, q, k_pool, v_pool, k_scales, v_scales, plan, plan_host: np.ndarray, kv_len, q_pos,
+                                  rope_table, out, workspace, workspace_bytes: int, status, batch: int, sm_scale: float,
+                                  stream=None) -> None:
+    """Sharing-aware decode over 8-bit pools: k_pool / v_pool are uint8 code pools, k_scales / v_scales their fp32 scales."""
+    a = _DecodeGroupedArgsC(_ptr(q), _ptr(k_pool), _ptr(v_pool), _ptr(plan), plan_host.ctypes.data, _ptr(kv_len),
+                            _ptr(q_pos), _ptr(rope_table), _ptr(out), _ptr(workspace), workspace_bytes, _ptr(status),
+                            batch, sm_scale)
+    c = cfg.c()
+    _check(lib().mepic_attn_decode_grouped_fp8(C.byref(c), C.byref(a), _ptr(k_scales), _ptr(v_scales), _stream_ptr(stream)))

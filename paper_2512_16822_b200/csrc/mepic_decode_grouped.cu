@@ -39,6 +39,8 @@ struct GroupedParams {
   const int32_t* q_pos;
   const float* rope;
   const int32_t* plan;
+  const float* k_scales;   // 8-bit pools only: [num_pages][n_kv_heads] scale of each (page, kv head) block of K
+  const float* v_scales;   // ... and of V
   float* part_o;    // [slots][G][D]
   float* part_ml;   // [slots][G][2] = (max in log2 units, sum)
   uint16_t* out;
@@ -51,7 +53,13 @@ struct GroupedParams {
   float scale_log2;   // sm_scale * log2(e)
 };
 
-template <int D, int G>
+// FP8: the pools hold e4m3 codes with one scale per (page, kv head) block (head_dim 128 only).  A staged tile is then
+// 16 rows x 128 bytes per pool; codes are widened exactly to fp16, both contractions run as fp16 MMAs, the K scale
+// goes on the fp32 scores and the V scale on P.  16-bit ldmatrix on 8-bit rows hands a lane four consecutive dims of a
+// key and the transposing 8-bit ldmatrix four consecutive keys of a dim, so the dim pairs of a lane are 16j + 4t + 2r
+// (bf16: 16j + 2t + 8r) and the key columns of the two score n-tiles are {0,1,4,5,..} / {2,3,6,7,..}: a lane's four
+// scores are keys 4t..4t+3, the keys its V fragments carry.
+template <int D, int G, bool FP8>
 __global__ void __launch_bounds__(kWarps * 32, 1)
 mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
   constexpr int R = plan_group_requests(G);
@@ -61,8 +69,9 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
   constexpr int KS = D / 16;                 // k-steps of the QK^T contraction
   constexpr int KH = KS / 2;                 // k-steps per half: step j pairs with step j + KH
   constexpr int ND = D / 8;                  // n-tiles of the PV product
-  constexpr int kBlockBytes = kTile * 128;   // one [16 rows x 64 dims] block
-  constexpr int kStageBytes = 2 * NB * kBlockBytes;   // K blocks then V blocks
+  constexpr int kBlockBytes = kTile * 128;   // one [16 rows x 128 bytes] block: 64 bf16 dims, or all 128 dims of 8-bit pages
+  constexpr int KB = FP8 ? 1 : NB;           // such blocks per K or V tile
+  constexpr int kStageBytes = 2 * KB * kBlockBytes;   // K blocks then V blocks
   constexpr int kWarpBytes = kStages * kStageBytes;
 
   extern __shared__ unsigned char smem_dyn[];
@@ -76,14 +85,18 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
   float* step16 = reinterpret_cast<float*>(smem + static_cast<size_t>(kWarps) * kWarpBytes);
   unsigned char* misc = smem + static_cast<size_t>(kWarps) * kWarpBytes + D * 4 + wic * 128;
   uint64_t* bars = reinterpret_cast<uint64_t*>(misc);                       // kStages x 8 bytes
-  volatile int32_t* meta = reinterpret_cast<volatile int32_t*>(misc + 32);  // [kStages][8]
+  volatile int32_t* meta = reinterpret_cast<volatile int32_t*>(misc + 32);  // [kStages][8] (64-byte misc + 32 .. + 128)
+  volatile float* scl = reinterpret_cast<volatile float*>(smem + static_cast<size_t>(kWarps) * (kWarpBytes + 128) + D * 4 + wic * 32);   // 8-bit pools: [kStages][2] K / V scale of the staged tile
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the merge kernel may move in as CTAs of this one retire
   for (int i = threadIdx.x; i < D; i += kWarps * 32) step16[i] = __ldg(p.rope + static_cast<size_t>(kTile) * D + i);
   __syncthreads();
 
-  const int g = lane >> 2;       // fragment row group: rows g and g + 8 (A, C) / key g (B)
+  const int g = lane >> 2;       // fragment row group: rows g and g + 8 (A, C) / key column g of a score n-tile (B)
   const int t = lane & 3;        // fragment column group
+  // first dim of the pair this lane's fragment register r of k-step j covers; the keys behind column g of the two n-tiles
+  auto pair_of = [&](int j, int r) { return FP8 ? 16 * j + 4 * t + 2 * r : 16 * j + 2 * t + 8 * r; };
+  const int keyA = FP8 ? 4 * (g >> 1) + (g & 1) : g, keyB = FP8 ? keyA + 2 : g + 8;
   // the two rows this lane owns: row = j * G + h = (request of the group, query head of the kv head)
   const int jA = g / G, hA = g % G, jB = (g + 8) / G, hB = (g + 8) % G;
 
@@ -110,10 +123,10 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
     for (int j = 0; j < KH; ++j)
 #pragma unroll
       for (int r = 0; r < 2; ++r) {
-        const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(g + 8 * kq) * D + 2 * (16 * j + 2 * t + 8 * r)));
-        kc[kq][j][r] = pack_bf16x2(cs.x, cs.z);
-        ksn[kq][j][r] = pack_bf16x2(cs.y, cs.w);
-        kns[kq][j][r] = pack_bf16x2(-cs.y, -cs.w);
+        const float4 cs = __ldg(reinterpret_cast<const float4*>(p.rope + static_cast<size_t>(kq ? keyB : keyA) * D + 2 * pair_of(j, r)));
+        kc[kq][j][r] = FP8 ? pack_f16x2(cs.x, cs.z) : pack_bf16x2(cs.x, cs.z);
+        ksn[kq][j][r] = FP8 ? pack_f16x2(cs.y, cs.w) : pack_bf16x2(cs.y, cs.w);
+        kns[kq][j][r] = FP8 ? pack_f16x2(-cs.y, -cs.w) : pack_bf16x2(-cs.y, -cs.w);
       }
 
   const int32_t* items = p.plan + p.off_items;
@@ -159,10 +172,17 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
       const uint32_t bar = smem_u32(&bars[stage]);
       const uint32_t dst = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
       mbar_expect_tx(bar, kStageBytes);
+      if constexpr (FP8) {
+        scl[stage * 2] = __ldg(p.k_scales + static_cast<size_t>(page) * p.n_kv_heads + ph);      // (an out-of-range page was replaced by 0 above)
+        scl[stage * 2 + 1] = __ldg(p.v_scales + static_cast<size_t>(page) * p.n_kv_heads + ph);
+        tma_load_2d(dst, &map_k, 0, y, bar);
+        tma_load_2d(dst + kBlockBytes, &map_v, 0, y, bar);
+      } else {
 #pragma unroll
-      for (int nb = 0; nb < NB; ++nb) {
-        tma_load_2d(dst + nb * kBlockBytes, &map_k, nb * 64, y, bar);
-        tma_load_2d(dst + (NB + nb) * kBlockBytes, &map_v, nb * 64, y, bar);
+        for (int nb = 0; nb < NB; ++nb) {
+          tma_load_2d(dst + nb * kBlockBytes, &map_k, nb * 64, y, bar);
+          tma_load_2d(dst + (NB + nb) * kBlockBytes, &map_v, nb * 64, y, bar);
+        }
       }
     }
     if (++pt == p_nt) {
@@ -213,7 +233,7 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
       for (int j = 0; j < KH; ++j)
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
-          const float4 cs = *reinterpret_cast<const float4*>(step16 + 2 * (16 * j + 2 * t + 8 * r));
+          const float4 cs = *reinterpret_cast<const float4*>(step16 + 2 * pair_of(j, r));
           const float l0 = ql[j][r][0], h0 = qh[j][r][0], l1 = ql[j][r][1], h1 = qh[j][r][1];
           ql[j][r][0] = l0 * cs.x + h0 * cs.y; qh[j][r][0] = h0 * cs.x - l0 * cs.y;      // rotation by -16 positions
           ql[j][r][1] = l1 * cs.z + h1 * cs.w; qh[j][r][1] = h1 * cs.z - l1 * cs.w;
@@ -229,7 +249,7 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
       for (int j = 0; j < KH; ++j)
 #pragma unroll
         for (int r = 0; r < 2; ++r) {
-          const int pair = 16 * j + 2 * t + 8 * r;              // dims pair, pair+1 and their partners + D/2
+          const int pair = pair_of(j, r);                        // dims pair, pair+1 and their partners + D/2
           const float2 lo = bf16x2_to_float2(__ldg(src + pair / 2));
           const float2 hi = bf16x2_to_float2(__ldg(src + (pair + D / 2) / 2));
           const float4 cs = __ldg(reinterpret_cast<const float4*>(row + 2 * pair));
@@ -276,7 +296,7 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
     }
 
     const uint32_t ks_addr = smem_u32(stage0 + static_cast<size_t>(stage) * kStageBytes);
-    const uint32_t vs_addr = ks_addr + NB * kBlockBytes;
+    const uint32_t vs_addr = ks_addr + KB * kBlockBytes;
     // only the partly filled last page of a request (always in its single-request item) has invalid slots
     int n_valid = kTile;
     if (u_tail >= 0 && (ct >> p.log2_tpp) == (c_nt >> p.log2_tpp) - 1)
@@ -298,8 +318,8 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
       // slots at or past kv_len may hold anything (NaN bit patterns included): their P is 0, but 0 x NaN is NaN,
       // so V must be finite there.
       if (n_valid < kTile) {
-        for (int idx = n_valid * 8 * NB + lane; idx < kTile * 8 * NB; idx += 32) {
-          const int key = idx / (8 * NB), chk = idx % (8 * NB);
+        for (int idx = n_valid * 8 * KB + lane; idx < kTile * 8 * KB; idx += 32) {
+          const int key = idx / (8 * KB), chk = idx % (8 * KB);
           const uint32_t a = vs_addr + (chk / 8) * kBlockBytes + key * 128 + (((chk % 8) ^ (key & 7)) << 4);
           asm volatile("st.shared.v4.b32 [%0], {%1,%1,%1,%1};" ::"r"(a), "r"(0) : "memory");
         }
@@ -308,12 +328,25 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
         __syncwarp();
       }
 
-      // ---- S^T = Q K'^T : B fragments by ldmatrix, rotated in registers, two key n-tiles (keys 0-7, 8-15)
+      // ---- S^T = Q K'^T : B fragments by ldmatrix, rotated in registers, two key n-tiles
       float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int j = 0; j < KH; ++j) {
         uint32_t lo[4], hi[4];      // lo: k-step j, hi: k-step j + KH; [b0 nt0, b1 nt0, b0 nt1, b1 nt1]
-        {
+        if constexpr (FP8) {
+          uint32_t raw[4];          // [n-tile 0 lower, n-tile 1 lower, n-tile 0 upper, n-tile 1 upper], 4 dims each
+          {
+            // lane -> (matrix mi = lane / 8, row = lane % 8): key of that row in n-tile (mi & 1), 16-byte chunk j (+ KH)
+            const int mi = lane >> 3, rr = lane & 7;
+            const int key = 4 * (rr >> 1) + (rr & 1) + 2 * (mi & 1);
+            const int chk = j + KH * (mi >> 1);
+            ldmatrix_x4(raw, ks_addr + key * 128 + ((chk ^ (key & 7)) << 4));
+          }
+          e4m3x4_to_f16x2x2(raw[0], lo[0], lo[1]);
+          e4m3x4_to_f16x2x2(raw[1], lo[2], lo[3]);
+          e4m3x4_to_f16x2x2(raw[2], hi[0], hi[1]);
+          e4m3x4_to_f16x2x2(raw[3], hi[2], hi[3]);
+        } else {
           // lane -> (matrix mi = lane / 8, row = lane % 8): key = 8 (mi / 2) + row, 16-byte chunk 2 j + (mi & 1)
           const int mi = lane >> 3, key = ((mi >> 1) << 3) + (lane & 7);
           const int cl = 2 * j + (mi & 1), chh = 2 * (j + KH) + (mi & 1);
@@ -322,30 +355,45 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
         }
 #pragma unroll
         for (int f = 0; f < 4; ++f) {
-          const int kq = f >> 1, r = f & 1;       // key g + 8 kq, fragment register r
+          const int kq = f >> 1, r = f & 1;       // key column of n-tile kq, fragment register r
           const uint32_t a = lo[f], b = hi[f];
-          lo[f] = bf16x2_fma(a, kc[kq][j][r], bf16x2_mul(b, kns[kq][j][r]));     // lo cos - hi sin
-          hi[f] = bf16x2_fma(a, ksn[kq][j][r], bf16x2_mul(b, kc[kq][j][r]));     // lo sin + hi cos
+          if constexpr (FP8) {
+            lo[f] = f16x2_fma(a, kc[kq][j][r], f16x2_mul(b, kns[kq][j][r]));     // lo cos - hi sin
+            hi[f] = f16x2_fma(a, ksn[kq][j][r], f16x2_mul(b, kc[kq][j][r]));     // lo sin + hi cos
+          } else {
+            lo[f] = bf16x2_fma(a, kc[kq][j][r], bf16x2_mul(b, kns[kq][j][r]));
+            hi[f] = bf16x2_fma(a, ksn[kq][j][r], bf16x2_mul(b, kc[kq][j][r]));
+          }
         }
-        // A fragments: a0 / a2 = row g dims 16j+2t.. / 16j+8+2t.., a1 / a3 = row g + 8
-        const uint32_t a0 = pack_bf16x2(qlA[j][0][0], qlA[j][0][1]), a2 = pack_bf16x2(qlA[j][1][0], qlA[j][1][1]);
-        const uint32_t a1 = pack_bf16x2(qlB[j][0][0], qlB[j][0][1]), a3 = pack_bf16x2(qlB[j][1][0], qlB[j][1][1]);
-        mma_bf16(s0, a0, a1, a2, a3, lo[0], lo[1]);
-        mma_bf16(s1, a0, a1, a2, a3, lo[2], lo[3]);
-        const uint32_t b0 = pack_bf16x2(qhA[j][0][0], qhA[j][0][1]), b2 = pack_bf16x2(qhA[j][1][0], qhA[j][1][1]);
-        const uint32_t b1 = pack_bf16x2(qhB[j][0][0], qhB[j][0][1]), b3 = pack_bf16x2(qhB[j][1][0], qhB[j][1][1]);
-        mma_bf16(s0, b0, b1, b2, b3, hi[0], hi[1]);
-        mma_bf16(s1, b0, b1, b2, b3, hi[2], hi[3]);
+        // A fragments: a0 / a2 = row g, the pairs of fragment registers 0 / 1 of this k-step; a1 / a3 = row g + 8
+        auto pk = [](float x, float y) { return FP8 ? pack_f16x2(x, y) : pack_bf16x2(x, y); };
+        const uint32_t a0 = pk(qlA[j][0][0], qlA[j][0][1]), a2 = pk(qlA[j][1][0], qlA[j][1][1]);
+        const uint32_t a1 = pk(qlB[j][0][0], qlB[j][0][1]), a3 = pk(qlB[j][1][0], qlB[j][1][1]);
+        const uint32_t b0 = pk(qhA[j][0][0], qhA[j][0][1]), b2 = pk(qhA[j][1][0], qhA[j][1][1]);
+        const uint32_t b1 = pk(qhB[j][0][0], qhB[j][0][1]), b3 = pk(qhB[j][1][0], qhB[j][1][1]);
+        if constexpr (FP8) {
+          mma_f16(s0, a0, a1, a2, a3, lo[0], lo[1]);
+          mma_f16(s1, a0, a1, a2, a3, lo[2], lo[3]);
+          mma_f16(s0, b0, b1, b2, b3, hi[0], hi[1]);
+          mma_f16(s1, b0, b1, b2, b3, hi[2], hi[3]);
+        } else {
+          mma_bf16(s0, a0, a1, a2, a3, lo[0], lo[1]);
+          mma_bf16(s1, a0, a1, a2, a3, lo[2], lo[3]);
+          mma_bf16(s0, b0, b1, b2, b3, hi[0], hi[1]);
+          mma_bf16(s1, b0, b1, b2, b3, hi[2], hi[3]);
+        }
       }
 
-      // ---- online softmax of the two rows (log2 domain); this lane holds keys 2t, 2t+1, 8+2t, 9+2t of each
-      float sa[4] = {s0[0], s0[1], s1[0], s1[1]}, sb[4] = {s0[2], s0[3], s1[2], s1[3]};
+      // ---- online softmax of the two rows (log2 domain); this lane holds, of each row, the keys kk[0..3]:
+      // 2t, 2t+1, 8+2t, 9+2t (bf16 pages) or 4t .. 4t+3 (8-bit pages)
+      const float k_scale = FP8 ? scl[stage * 2] : 1.f, v_scale = FP8 ? scl[stage * 2 + 1] : 1.f;
+      float sa[4] = {s0[0] * k_scale, s0[1] * k_scale, s1[0] * k_scale, s1[1] * k_scale};
+      float sb[4] = {s0[2] * k_scale, s0[3] * k_scale, s1[2] * k_scale, s1[3] * k_scale};
       if (n_valid < kTile) {
-        const int k0 = 2 * t;
-        if (k0 >= n_valid) { sa[0] = -INFINITY; sb[0] = -INFINITY; }
-        if (k0 + 1 >= n_valid) { sa[1] = -INFINITY; sb[1] = -INFINITY; }
-        if (k0 + 8 >= n_valid) { sa[2] = -INFINITY; sb[2] = -INFINITY; }
-        if (k0 + 9 >= n_valid) { sa[3] = -INFINITY; sb[3] = -INFINITY; }
+        const int kk[4] = {FP8 ? 4 * t : 2 * t, FP8 ? 4 * t + 1 : 2 * t + 1, FP8 ? 4 * t + 2 : 2 * t + 8, FP8 ? 4 * t + 3 : 2 * t + 9};
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (kk[i] >= n_valid) { sa[i] = -INFINITY; sb[i] = -INFINITY; }
       }
       float mxa = fmaxf(fmaxf(sa[0], sa[1]), fmaxf(sa[2], sa[3])), mxb = fmaxf(fmaxf(sb[0], sb[1]), fmaxf(sb[2], sb[3]));
       mxa = fmaxf(mxa, __shfl_xor_sync(kFull, mxa, 1)); mxb = fmaxf(mxb, __shfl_xor_sync(kFull, mxb, 1));
@@ -361,21 +409,46 @@ mepic_decode_grouped(const GroupedParams p, const __grid_constant__ CUtensorMap 
       const float pb0 = ex2(sb[0] - mB), pb1 = ex2(sb[1] - mB), pb2 = ex2(sb[2] - mB), pb3 = ex2(sb[3] - mB);
       lA += (pa0 + pa1) + (pa2 + pa3);
       lB += (pb0 + pb1) + (pb2 + pb3);
-      // A fragment of P: a0 row g keys 2t.., a1 row g+8 keys 2t.., a2 row g keys 8+2t.., a3 row g+8 keys 8+2t..
-      const uint32_t f0 = pack_bf16x2(pa0, pa1), f1 = pack_bf16x2(pb0, pb1), f2 = pack_bf16x2(pa2, pa3), f3 = pack_bf16x2(pb2, pb3);
+      // A fragment of P (carrying the V scale of the tile on 8-bit pages): a0 row g keys kk[0], kk[1]; a1 row g+8 the
+      // same keys; a2 row g keys kk[2], kk[3]; a3 row g+8 the same
+      uint32_t f0, f1, f2, f3;
+      if constexpr (FP8) {
+        f0 = pack_f16x2(pa0 * v_scale, pa1 * v_scale); f1 = pack_f16x2(pb0 * v_scale, pb1 * v_scale);
+        f2 = pack_f16x2(pa2 * v_scale, pa3 * v_scale); f3 = pack_f16x2(pb2 * v_scale, pb3 * v_scale);
+      } else {
+        f0 = pack_bf16x2(pa0, pa1); f1 = pack_bf16x2(pb0, pb1); f2 = pack_bf16x2(pa2, pa3); f3 = pack_bf16x2(pb2, pb3);
+      }
 
-      // ---- O += P V : B fragments of V by transposing ldmatrix, two dim n-tiles per load
+      // ---- O += P V : B fragments of V by transposing ldmatrix
+      if constexpr (FP8) {
+        // the transposing 8-bit ldmatrix hands this lane keys 4t..4t+3 of dims g and g + 8 of a 16-dim block
 #pragma unroll
-      for (int nd = 0; nd < ND; nd += 2) {
-        uint32_t vb[4];             // [b0, b1] of n-tile nd, [b0, b1] of n-tile nd+1
-        {
-          // lane -> (matrix mi, row): key = 8 (mi & 1) + row, 16-byte chunk nd + (mi >> 1)
-          const int mi = lane >> 3, key = ((mi & 1) << 3) + (lane & 7);
-          const int chk = nd + (mi >> 1);
-          ldmatrix_x4_trans(vb, vs_addr + (chk / 8) * kBlockBytes + key * 128 + (((chk % 8) ^ (key & 7)) << 4));
+        for (int c = 0; c < D / 16; c += 2) {
+          uint32_t raw[4];          // [block c: dim g, dim g + 8 | block c + 1: dim g, dim g + 8]
+          {
+            const int key = lane & 15, chk = c + (lane >> 4);
+            ldmatrix_b8_trans_x2(raw, vs_addr + key * 128 + ((chk ^ (key & 7)) << 4));
+          }
+#pragma unroll
+          for (int m = 0; m < 4; ++m) {
+            uint32_t v0, v1;
+            e4m3x4_to_f16x2x2(raw[m], v0, v1);
+            mma_f16(acc[2 * c + m], f0, f1, f2, f3, v0, v1);
+          }
         }
-        mma_bf16(acc[nd], f0, f1, f2, f3, vb[0], vb[1]);
-        mma_bf16(acc[nd + 1], f0, f1, f2, f3, vb[2], vb[3]);
+      } else {
+#pragma unroll
+        for (int nd = 0; nd < ND; nd += 2) {
+          uint32_t vb[4];             // [b0, b1] of n-tile nd, [b0, b1] of n-tile nd+1
+          {
+            // lane -> (matrix mi, row): key = 8 (mi & 1) + row, 16-byte chunk nd + (mi >> 1)
+            const int mi = lane >> 3, key = ((mi & 1) << 3) + (lane & 7);
+            const int chk = nd + (mi >> 1);
+            ldmatrix_x4_trans(vb, vs_addr + (chk / 8) * kBlockBytes + key * 128 + (((chk % 8) ^ (key & 7)) << 4));
+          }
+          mma_bf16(acc[nd], f0, f1, f2, f3, vb[0], vb[1]);
+          mma_bf16(acc[nd + 1], f0, f1, f2, f3, vb[2], vb[3]);
+        }
       }
     }
     __syncwarp();   // every lane is done with this stage
@@ -445,18 +518,19 @@ __global__ void __launch_bounds__(128) mepic_decode_grouped_merge(const GroupedP
   }
 }
 
-template <int D, int G>
+template <int D, int G, bool FP8>
 constexpr size_t grouped_smem_bytes() {
-  // per warp: 3 stages of (K blocks + V blocks) and 128 bytes of barriers and tile bases; one table row; 1 KB alignment slack
-  return static_cast<size_t>(kWarps) * (3 * 2 * (D / 64) * kTile * 128 + 128) + D * 4 + 1024;
+  // per warp: 3 stages of (K blocks + V blocks), 128 bytes of barriers and tile bases, 32 bytes of tile scales; one table
+  // row; 1 KB alignment slack
+  return static_cast<size_t>(kWarps) * (3 * 2 * (FP8 ? 1 : D / 64) * kTile * 128 + 128 + 32) + D * 4 + 1024;
 }
 
-template <int D, int G>
+template <int D, int G, bool FP8>
 int32_t launch_grouped(const GroupedParams& p, int n_ctas, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
-  constexpr size_t smem = grouped_smem_bytes<D, G>();
-  cudaError_t e = cudaFuncSetAttribute(mepic_decode_grouped<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  constexpr size_t smem = grouped_smem_bytes<D, G, FP8>();
+  cudaError_t e = cudaFuncSetAttribute(mepic_decode_grouped<D, G, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("decode_grouped: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
-  mepic_decode_grouped<D, G><<<n_ctas, kWarps * 32, smem, stream>>>(p, map_k, map_v);
+  mepic_decode_grouped<D, G, FP8><<<n_ctas, kWarps * 32, smem, stream>>>(p, map_k, map_v);
   e = launch_dependent(mepic_decode_grouped_merge<D, G>, dim3(p.batch * p.n_kv_heads * G), dim3(128), stream, p);
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("decode_grouped: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
@@ -486,8 +560,11 @@ extern "C" size_t mepic_attn_decode_grouped_workspace(const mepic_config_t* cfg,
   return grouped_slots(cfg, plan_host) * G * (cfg->head_dim + 2) * sizeof(float);
 }
 
-extern "C" int32_t mepic_attn_decode_grouped(const mepic_config_t* cfg, const mepic_decode_grouped_args_t* a, void* cuda_stream) {
+static int32_t grouped_call(const mepic_config_t* cfg, const mepic_decode_grouped_args_t* a, const float* k_scales, const float* v_scales,
+                            bool fp8, void* cuda_stream) {
   if (!mepic_config_ok(cfg)) return MEPIC_E_INVAL;
+  if (fp8 && cfg->head_dim != 128) { mepic_set_error("decode_grouped_fp8: head_dim %d: 8-bit pages are built for head_dim 128", cfg->head_dim); return MEPIC_E_INVAL; }
+  if (fp8 && (!k_scales || !v_scales)) { mepic_set_error("decode_grouped_fp8: NULL scale pointer"); return MEPIC_E_INVAL; }
   if (!a || !a->q || !a->k_pool || !a->v_pool || !a->plan || !a->plan_host || !a->kv_len || !a->q_pos ||
       !a->rope_table || !a->out || !a->workspace || !a->status) { mepic_set_error("decode_grouped: NULL pointer argument"); return MEPIC_E_INVAL; }
   if (a->batch < 1) { mepic_set_error("decode_grouped: batch must be positive"); return MEPIC_E_INVAL; }
@@ -504,6 +581,7 @@ extern "C" int32_t mepic_attn_decode_grouped(const mepic_config_t* cfg, const me
   GroupedParams p;
   p.q = static_cast<const uint16_t*>(a->q);
   p.kv_len = a->kv_len; p.q_pos = a->q_pos; p.rope = a->rope_table; p.plan = a->plan;
+  p.k_scales = k_scales; p.v_scales = v_scales;
   p.part_o = static_cast<float*>(a->workspace);
   p.part_ml = p.part_o + slots * G * D;
   p.out = static_cast<uint16_t*>(a->out);
@@ -519,16 +597,33 @@ extern "C" int32_t mepic_attn_decode_grouped(const mepic_config_t* cfg, const me
   p.spin_limit = mepic_test_spin_limit(kSpinLimit); p.skip_tile = mepic_test_skip_tile();
   cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
   alignas(64) CUtensorMap map_k, map_v;
-  int32_t rc = mepic_make_pool_map(cfg, a->k_pool, &map_k);
+  int32_t rc = fp8 ? mepic_make_pool_map_u8(cfg, a->k_pool, &map_k) : mepic_make_pool_map(cfg, a->k_pool, &map_k);
   if (rc != MEPIC_OK) return rc;
-  rc = mepic_make_pool_map(cfg, a->v_pool, &map_v);
+  rc = fp8 ? mepic_make_pool_map_u8(cfg, a->v_pool, &map_v) : mepic_make_pool_map(cfg, a->v_pool, &map_v);
   if (rc != MEPIC_OK) return rc;
   const int n_ctas = h[kPhWorkers] / kWarps;
+  if (fp8) {
+    switch (G) {
+#define MEPIC_GROUPED_FP8_CASE(GG) case GG: return launch_grouped<128, GG, true>(p, n_ctas, map_k, map_v, st);
+      MEPIC_GROUPED_FP8_CASE(1) MEPIC_GROUPED_FP8_CASE(2) MEPIC_GROUPED_FP8_CASE(3) MEPIC_GROUPED_FP8_CASE(4)
+      MEPIC_GROUPED_FP8_CASE(5) MEPIC_GROUPED_FP8_CASE(6) MEPIC_GROUPED_FP8_CASE(7) MEPIC_GROUPED_FP8_CASE(8)
+#undef MEPIC_GROUPED_FP8_CASE
+    }
+  }
 
-#define MEPIC_GROUPED_CASE(DD, GG) if (D == DD && G == GG) return launch_grouped<DD, GG>(p, n_ctas, map_k, map_v, st);
+#define MEPIC_GROUPED_CASE(DD, GG) if (D == DD && G == GG) return launch_grouped<DD, GG, false>(p, n_ctas, map_k, map_v, st);
   MEPIC_GROUPED_CASE(128, 1) MEPIC_GROUPED_CASE(128, 2) MEPIC_GROUPED_CASE(128, 3) MEPIC_GROUPED_CASE(128, 4) MEPIC_GROUPED_CASE(128, 5) MEPIC_GROUPED_CASE(128, 6) MEPIC_GROUPED_CASE(128, 7) MEPIC_GROUPED_CASE(128, 8)
   MEPIC_GROUPED_CASE(64, 1) MEPIC_GROUPED_CASE(64, 2) MEPIC_GROUPED_CASE(64, 3) MEPIC_GROUPED_CASE(64, 4) MEPIC_GROUPED_CASE(64, 5) MEPIC_GROUPED_CASE(64, 6) MEPIC_GROUPED_CASE(64, 7) MEPIC_GROUPED_CASE(64, 8)
 #undef MEPIC_GROUPED_CASE
   mepic_set_error("decode_grouped: unsupported head_dim %d / group size %d", D, G);
   return MEPIC_E_INVAL;
+}
+
+extern "C" int32_t mepic_attn_decode_grouped(const mepic_config_t* cfg, const mepic_decode_grouped_args_t* a, void* cuda_stream) {
+  return grouped_call(cfg, a, nullptr, nullptr, false, cuda_stream);
+}
+
+extern "C" int32_t mepic_attn_decode_grouped_fp8(const mepic_config_t* cfg, const mepic_decode_grouped_args_t* a, const float* k_scales,
+                                                 const float* v_scales, void* cuda_stream) {
+  return grouped_call(cfg, a, k_scales, v_scales, true, cuda_stream);
 }

@@ -12,7 +12,7 @@ import numpy as np
 import torch
 
 from . import (Config, Segment, Store, MEPIC_SEG_CHUNK, MEPIC_SEG_PROMPT, mepic_attn_decode,
-               mepic_decode_plan_build, mepic_decode_plan_patch, mepic_attn_decode_grouped, mepic_attn_decode_grouped_workspace,
+               mepic_decode_plan_build, mepic_decode_plan_patch, mepic_attn_decode_grouped, mepic_attn_decode_grouped_fp8, mepic_attn_decode_grouped_workspace,
                mepic_pages_quantize, mepic_attn_decode_fp8,
                mepic_attn_decode_workspace, mepic_attn_prefill, mepic_attn_prefill_fp8, mepic_attn_prefill_workspace,
                mepic_rope_table_fill)
@@ -301,4 +301,22 @@ class Fp8PrefillBatch(PrefillBatch):
                                workspace_bytes=self.ws_bytes, status=self.dev.status,
                                row_offsets_host=self.row_offsets_host, table_stride=self.stride, batch=self.batch,
                                sm_scale=sm_scale, stream=s)
+        return self.out
+
+
+class Fp8GroupedDecodeBatch(GroupedDecodeBatch):
+    """The sharing-aware decode path over the 8-bit pools."""
+
+    def __init__(self, pools: Fp8Pools, page_ids, pos_base, kv_len, q_pos, q_bits=None, n_sms: int = 0):
+        super().__init__(pools.dev, page_ids, pos_base, kv_len, q_pos, q_bits, n_sms)
+        self.pools = pools
+
+    def run(self, sm_scale: float, stream=None) -> torch.Tensor:
+        s = stream if stream is not None else torch.cuda.current_stream(self.dev.device)
+        mepic_attn_decode_grouped_fp8(self.dev.cfg, q=self.q, k_pool=self.pools.k_codes, v_pool=self.pools.v_codes,
+                                      k_scales=self.pools.k_scales, v_scales=self.pools.v_scales, plan=self.plan,
+                                      plan_host=self.plan_host, kv_len=self.kv_len, q_pos=self.q_pos,
+                                      rope_table=self.dev.rope, out=self.out, workspace=self.workspace,
+                                      workspace_bytes=self.ws_bytes, status=self.dev.status, batch=self.batch,
+                                      sm_scale=sm_scale, stream=s)
         return self.out

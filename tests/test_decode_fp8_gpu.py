@@ -77,7 +77,12 @@ def _run(cfg, kp, vp, page_ids, pos_base, kv_len, q_pos, q, sm_scale, theta, sam
     out = batch.run(sm_scale)
     torch.cuda.synchronize()
     assert dev.read_status() == 0
-    got = RT.bf16_bits(out)
+    got = RT.bf16_bits(out).copy()
+    # the sharing-aware path over the same 8-bit pools (mepic_attn_decode_grouped_fp8): same definition, same tolerance
+    gout = RT.Fp8GroupedDecodeBatch(fp, page_ids, pos_base, kv_len, q_pos, q).run(sm_scale)
+    torch.cuda.synchronize()
+    assert dev.read_status() == 0
+    ggot = RT.bf16_bits(gout)
     # the oracle works on the oracle's own codes and scales (identical to the device's, see the quantiser test)
     kc, ks = O.quantize_pages(kp); vc, vs = O.quantize_pages(vp)
     kf, vf = O.dequantize_pages(kc, ks), O.dequantize_pages(vc, vs)
@@ -87,6 +92,7 @@ def _run(cfg, kp, vp, page_ids, pos_base, kv_len, q_pos, q, sm_scale, theta, sam
         want = O.decode_attention_one(q[b], kf, vf, list(page_ids[b, :n]), list(pos_base[b, :n]), int(kv_len[b]),
                                       int(q_pos[b]), sm_scale, theta)
         _check(got[b], want, f"request {b}")
+        _check(ggot[b], want, f"request {b}, grouped")
     return got, (kf, vf)
 
 

@@ -89,11 +89,15 @@ class _Side:
         q_pos = np.array([t[1][(t[2] - 1) // P] + (t[2] - 1) % P for t in tables], dtype=np.int32)
         out = RT.Fp8DecodeBatch(self.pools, ids, base, kvl, q_pos, q).run(sm); torch.cuda.synchronize()
         assert self.dev.read_status() == 0, what
-        got = RT.bf16_bits(out)
+        got = RT.bf16_bits(out).copy()
         kf, vf = O.dequantize_pages(self.okc, self.oks), O.dequantize_pages(self.ovc, self.ovs)
+        gout = RT.Fp8GroupedDecodeBatch(self.pools, ids, base, kvl, q_pos, q).run(sm); torch.cuda.synchronize()
+        assert self.dev.read_status() == 0, what
+        ggot = RT.bf16_bits(gout)
         for b, t in enumerate(tables):
             want = O.decode_attention_one(q[b], kf, vf, list(t[0]), list(t[1]), int(t[2]), int(q_pos[b]), sm, self.theta)
             _check(got[b], want, 1e-2, f"{what} decode request {b}")
+            _check(ggot[b], want, 1e-2, f"{what} grouped decode request {b}")
 
 
 @pytest.mark.parametrize("Hq,Hkv,P,n_chunks,chunk_pages,question", [(8, 2, 16, 3, 9, 40), (10, 2, 16, 2, 5, 21), (4, 4, 64, 2, 3, 70),
