@@ -401,7 +401,10 @@ constexpr int kNumBars = kBarVReady + kVStages;
 // only publish where each 16-key group of the tile lives, and the rotator warps fetch the codes from global memory
 // themselves, widen them exactly, fold the block's scale into the rotation constants (K) or the widening (V) and write
 // the bf16 stage the MMA reads.  Everything downstream of the stages is unchanged.
-template <int D, int G, bool FP8>
+// HOOKS = the test build of the kernel: the poll limit of the bounded waits and the one left-out K tile come from the
+// launch parameters (mepic_kernel_test_hooks).  The production instantiation has the limit as a compile-time constant
+// and no such check: the issuing thread's wait loops are on the critical path of every tile (measured: 2 % of the call).
+template <int D, int G, bool FP8, bool HOOKS>
 __global__ void __launch_bounds__(kThreads, 1)
 mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap map_k, const __grid_constant__ CUtensorMap map_v) {
   using L = PrefillSmem<D>;
@@ -429,6 +432,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   volatile int* vrow = reinterpret_cast<volatile int*>(bars + kNumBars + 30);   // ... and [kVStages][8] for the V stages
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int spin = HOOKS ? p.spin_limit : kSpinLimit;
   Item* item_slot = reinterpret_cast<Item*>(bars + kNumBars + 16);
   if (warp == 1) {
     const Item it = item_of_cta(p.row_offsets, p.batch, p.n_kv_heads, 2 * QT, p.max_q_tiles, blockIdx.x / p.n_splits, lane);
@@ -576,7 +580,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     bool ok = true;
     const int my_tiles = nt[x];
     for (int tile = 0; tile < my_tiles; ++tile) {
-      if (!mbar_wait_warp(BAR(kBarSFull, x), static_cast<uint32_t>(tile) & 1u, abort_flag, p.status, p.spin_limit)) { ok = false; break; }
+      if (!mbar_wait_warp(BAR(kBarSFull, x), static_cast<uint32_t>(tile) & 1u, abort_flag, p.status, spin)) { ok = false; break; }
       tc_fence_after();
       const int n_vis = limit - (tile_base + tile) * kTileN + 1 - 64 * ch;     // my columns [0, n_vis) are visible to this row
       const bool boundary = n_vis < 64;                          // only the tile(s) on the causal boundary need the mask
@@ -664,7 +668,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       // was issued after both threads handed P over).  The M-tile's Q' block is free by now: its last QK^T has completed.
       float* ep = reinterpret_cast<float*>(Qs + x * NB * kBlockBytes);
       const float l_tot = l_run + swap_with_partner(l_run, ok, ep + ch * 128 + r, ep + (ch ^ 1) * 128 + r);
-      if (ok) ok = mbar_wait_warp(BAR(kBarPvDone, x), static_cast<uint32_t>(my_tiles - 1) & 1u, abort_flag, p.status, p.spin_limit);
+      if (ok) ok = mbar_wait_warp(BAR(kBarPvDone, x), static_cast<uint32_t>(my_tiles - 1) & 1u, abort_flag, p.status, spin);
       if (ok) {
         tc_fence_after();
         const size_t rh = static_cast<size_t>(item.row0 + qi) * n_q_heads + static_cast<size_t>(h) * G + g;
@@ -726,7 +730,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     for (int tile = 0; tile < n_tiles; ++tile) {
       const int st = tile % kKStages;
       const uint32_t ph = static_cast<uint32_t>(tile / kKStages) & 1u;
-      if (!mbar_wait(BAR(kBarKLanded, st), ph, abort_flag, p.status, p.spin_limit)) break;
+      if (!mbar_wait(BAR(kBarKLanded, st), ph, abort_flag, p.status, spin)) break;
       unsigned char* Kb = Ks + st * NB * kBlockBytes;
       const int key0 = (tile_base + tile) * kTileN;
       int pos = gbase[st * 8 + k0 / 16] + (k0 & 15);
@@ -796,7 +800,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         // ---- the V tile of the same index: widen, scale, store; rows at or past kv_len become zero (P is 0 there,
         // but 0 x NaN is NaN)
         const int vst = tile % kVStages;
-        if (!mbar_wait(BAR(kBarVLanded, vst), static_cast<uint32_t>(tile / kVStages) & 1u, abort_flag, p.status, p.spin_limit)) break;
+        if (!mbar_wait(BAR(kBarVLanded, vst), static_cast<uint32_t>(tile / kVStages) & 1u, abort_flag, p.status, spin)) break;
         unsigned char* Vb = Vs + vst * NB * kBlockBytes;
 #pragma unroll 2
         for (int i = 0; i < 8; ++i) {
@@ -869,7 +873,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       if (tile >= depth) {
         // the stage is free once every MMA that reads its previous tenant has completed
         const uint32_t bar = BAR(is_k ? kBarKFree : kBarVFree, st);
-        if (!mbar_wait_warp(bar, static_cast<uint32_t>(tile / depth - 1) & 1u, abort_flag, p.status, p.spin_limit)) { ok = false; break; }
+        if (!mbar_wait_warp(bar, static_cast<uint32_t>(tile / depth - 1) & 1u, abort_flag, p.status, spin)) { ok = false; break; }
       }
       const int key0 = (tile_base + tile) * kTileN;
       const int gkey = key0 + lane * 16;
@@ -887,7 +891,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       const unsigned live_mask = __ballot_sync(0xffffffffu, live);
       __syncwarp();
       const uint32_t landed = BAR(is_k ? kBarKLanded : kBarVLanded, st);
-      if (is_k && blockIdx.x == 0 && tile == p.skip_tile) continue;      // (test hook: a K tile that never comes)
+      if (HOOKS && is_k && blockIdx.x == 0 && tile == p.skip_tile) continue;      // (test hook: a K tile that never comes)
       if constexpr (FP8) {
         // nothing to copy: the stage is free and its groups' pool rows are published; the rotators do the rest
         if (lane == 0) mbar_arrive(landed);
@@ -906,7 +910,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     // but 0 x NaN is NaN, so V must be finite.  Zero them once the tile has landed.
     if (!FP8 && !is_k && ok && last_has_tail) {
       const int lt = n_tiles - 1, st = lt % kVStages;
-      if (mbar_wait_warp(BAR(kBarVLanded, st), static_cast<uint32_t>(lt / kVStages) & 1u, abort_flag, p.status, p.spin_limit)) {
+      if (mbar_wait_warp(BAR(kBarVLanded, st), static_cast<uint32_t>(lt / kVStages) & 1u, abort_flag, p.status, spin)) {
         unsigned char* Vb = Vs + st * NB * kBlockBytes;
         const int first = kvl - (tile_base + lt) * kTileN;       // first row to clear (0 < first < 128)
         for (int idx = first * 2 * CH + lane; idx < kTileN * 2 * CH; idx += 32) {
@@ -950,12 +954,12 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       tc_commit(BAR(kBarPvDone, x));
     };
     auto wait_k = [&](int j) {
-      const bool w = mbar_wait(BAR(kBarKReady, j % kKStages), static_cast<uint32_t>(j / kKStages) & 1u, abort_flag, p.status, p.spin_limit);
+      const bool w = mbar_wait(BAR(kBarKReady, j % kKStages), static_cast<uint32_t>(j / kKStages) & 1u, abort_flag, p.status, spin);
       tc_fence_after();
       return w;
     };
     // prologue: S of key tile 0 for both M-tiles
-    ok = n_tiles > 0 && mbar_wait(BAR(kBarQReady, 0), 0, abort_flag, p.status, p.spin_limit) && wait_k(0);
+    ok = n_tiles > 0 && mbar_wait(BAR(kBarQReady, 0), 0, abort_flag, p.status, spin) && wait_k(0);
     if (ok) {
       if (nt[0] > 0) issue_qk(0, 0);
       if (nt[1] > 0) issue_qk(1, 0);
@@ -965,8 +969,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       bool v_here = false;
       auto wait_v = [&]() {
         if (v_here) return true;
-        bool w = mbar_wait(BAR(FP8 ? kBarVReady : kBarVLanded, j % kVStages), static_cast<uint32_t>(j / kVStages) & 1u, abort_flag, p.status, p.spin_limit);
-        if (!FP8 && w && j == n_tiles - 1 && last_has_tail) w = mbar_wait(BAR(kBarVPatched, 0), 0, abort_flag, p.status, p.spin_limit);
+        bool w = mbar_wait(BAR(FP8 ? kBarVReady : kBarVLanded, j % kVStages), static_cast<uint32_t>(j / kVStages) & 1u, abort_flag, p.status, spin);
+        if (!FP8 && w && j == n_tiles - 1 && last_has_tail) w = mbar_wait(BAR(kBarVPatched, 0), 0, abort_flag, p.status, spin);
         v_here = w;
         return w;
       };
@@ -975,14 +979,14 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       // nothing stands between the issue of PV_a and of QK_a(next) and the pipe's queue does not run dry.
       if (more && !wait_k(j + 1)) { ok = false; break; }
       if (j < nt[0]) {
-        if (!mbar_wait(BAR(kBarPFull, 0), static_cast<uint32_t>(j) & 1u, abort_flag, p.status, p.spin_limit) || !wait_v()) { ok = false; break; }
+        if (!mbar_wait(BAR(kBarPFull, 0), static_cast<uint32_t>(j) & 1u, abort_flag, p.status, spin) || !wait_v()) { ok = false; break; }
         tc_fence_after();
         issue_pv(0, j);
       }
       if (more && j + 1 < nt[0]) issue_qk(0, j + 1);
       // ---- M-tile b
       if (j < nt[1]) {
-        if (!mbar_wait(BAR(kBarPFull, 1), static_cast<uint32_t>(j) & 1u, abort_flag, p.status, p.spin_limit) || !wait_v()) { ok = false; break; }
+        if (!mbar_wait(BAR(kBarPFull, 1), static_cast<uint32_t>(j) & 1u, abort_flag, p.status, spin) || !wait_v()) { ok = false; break; }
         tc_fence_after();
         issue_pv(1, j);
       }
@@ -995,7 +999,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     if (!ok) {
       // a wait was lost: the MMAs issued so far still run; tensor memory may only be released once they are done
       tc_commit(BAR(kBarDrain, 0));
-      for (int i = 0; i < p.spin_limit && !mbar_try_wait(BAR(kBarDrain, 0), 0); ++i) {}
+      for (int i = 0; i < spin && !mbar_try_wait(BAR(kBarDrain, 0), 0); ++i) {}
     }
   }
 
@@ -1054,10 +1058,10 @@ __global__ void __launch_bounds__(128) mepic_prefill_merge(const PrefillParams p
   }
 }
 
-template <int D, int G, bool FP8>
+template <int D, int G, bool FP8, bool HOOKS = false>
 int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& map_k, const CUtensorMap& map_v, cudaStream_t stream) {
   constexpr size_t smem = PrefillSmem<D>::kBytes;
-  cudaError_t e = cudaFuncSetAttribute(mepic_prefill_attn<D, G, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+  cudaError_t e = cudaFuncSetAttribute(mepic_prefill_attn<D, G, FP8, HOOKS>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
   if (e != cudaSuccess) { mepic_set_error("prefill: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   const int chunks_per_row = p.n_kv_heads * D / 8;
   if (FP8) mepic_prefill_commit_fp8<<<p.total_rows, 256, 0, stream>>>(p, D);
@@ -1070,7 +1074,7 @@ int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& m
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(static_cast<unsigned>(n_items * p.n_splits)); lc.blockDim = dim3(kThreads); lc.dynamicSmemBytes = smem; lc.stream = stream;
   lc.attrs = pdl; lc.numAttrs = 1;
-  e = cudaLaunchKernelEx(&lc, mepic_prefill_attn<D, G, FP8>, p, map_k, map_v);
+  e = cudaLaunchKernelEx(&lc, mepic_prefill_attn<D, G, FP8, HOOKS>, p, map_k, map_v);
   if (e == cudaSuccess && p.n_splits > 1) {
     const long long n_pairs = static_cast<long long>(p.total_rows) * p.n_kv_heads * G;
     lc.gridDim = dim3(static_cast<unsigned>((n_pairs + 3) / 4)); lc.blockDim = dim3(128); lc.dynamicSmemBytes = 0;
@@ -1185,6 +1189,12 @@ static int32_t prefill_call(const mepic_config_t* cfg, const mepic_prefill_args_
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;
   p.spin_limit = mepic_test_spin_limit(kSpinLimit); p.skip_tile = mepic_test_skip_tile();
   const int D = cfg->head_dim, G = cfg->n_q_heads / cfg->n_kv_heads;
+  if (p.spin_limit != kSpinLimit || p.skip_tile >= 0) {
+    // test hooks are set: the instrumented instantiation, built for the shape the give-up test uses
+    if (D == 128 && G == 4) return fp8 ? launch_prefill<128, 4, true, true>(p, n_items, map_k, map_v, st) : launch_prefill<128, 4, false, true>(p, n_items, map_k, map_v, st);
+    mepic_set_error("prefill: the kernel test hooks are built for head_dim 128 and group size 4 only");
+    return MEPIC_E_INVAL;
+  }
   if (fp8) {
 #define MEPIC_PREFILL_FP8_CASE(GG) if (G == GG) return launch_prefill<128, GG, true>(p, n_items, map_k, map_v, st);
     MEPIC_PREFILL_FP8_CASE(1) MEPIC_PREFILL_FP8_CASE(2) MEPIC_PREFILL_FP8_CASE(3) MEPIC_PREFILL_FP8_CASE(4) MEPIC_PREFILL_FP8_CASE(5) MEPIC_PREFILL_FP8_CASE(6) MEPIC_PREFILL_FP8_CASE(7) MEPIC_PREFILL_FP8_CASE(8)
