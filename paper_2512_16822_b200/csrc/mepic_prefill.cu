@@ -802,27 +802,38 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         const int vst = tile % kVStages;
         if (!mbar_wait(BAR(kBarVLanded, vst), static_cast<uint32_t>(tile / kVStages) & 1u, abort_flag, p.status, spin)) break;
         unsigned char* Vb = Vs + vst * NB * kBlockBytes;
-#pragma unroll 2
-        for (int i = 0; i < 8; ++i) {
-          const int idx = rt + 128 * i;              // 16-byte chunk of codes: key idx / 8, dims [16 (idx % 8), +16)
-          const int kk = idx >> 3, c16 = idx & 7;
-          const int vr = vrow[vst * 8 + (kk >> 4)];
-          uint32_t w[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-          if (vr >= 0 && key0 + kk < kvl) {
-            const uint4 cd = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(p.v_pool) + static_cast<size_t>(vr + (kk & 15)) * D + 16 * c16));
-            const float sc = __ldg(p.v_scales + vr / p.page_size);
-            const uint32_t cw[4] = {cd.x, cd.y, cd.z, cd.w};
+        {
+          // all of the thread's eight 16-byte chunks of codes are requested before the first is used: one load latency
+          // per tile instead of four.  Chunk idx = rt + 128 i: key idx / 8, dims [16 (idx % 8), +16)
+          uint4 cd[8];
+          float sc[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int idx = rt + 128 * i, kk = idx >> 3, c16 = idx & 7;
+            const int vr = vrow[vst * 8 + (kk >> 4)];
+            const bool live = vr >= 0 && key0 + kk < kvl;
+            cd[i] = make_uint4(0, 0, 0, 0); sc[i] = 0.f;
+            if (live) {
+              cd[i] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(p.v_pool) + static_cast<size_t>(vr + (kk & 15)) * D + 16 * c16));
+              sc[i] = __ldg(p.v_scales + vr / p.page_size);
+            }
+          }
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int idx = rt + 128 * i, kk = idx >> 3, c16 = idx & 7;
+            const uint32_t cw[4] = {cd[i].x, cd[i].y, cd[i].z, cd[i].w};
+            uint32_t w[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
               uint32_t hh;
               asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(hh) : "h"(static_cast<uint16_t>(cw[j >> 1] >> (16 * (j & 1)))));
               const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hh));
-              w[j] = pack_bf16x2(f.x * sc, f.y * sc);
+              w[j] = pack_bf16x2(f.x * sc[i], f.y * sc[i]);       // a dead row: codes 0 and scale 0 give zeros
             }
+            const int ch0 = 2 * c16;                   // bf16 chunk (8 dims) index within the row
+            *reinterpret_cast<uint4*>(Vb + (ch0 / 8) * kBlockBytes + sw128(kk, ch0 % 8)) = make_uint4(w[0], w[1], w[2], w[3]);
+            *reinterpret_cast<uint4*>(Vb + (ch0 / 8) * kBlockBytes + sw128(kk, ch0 % 8 + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
           }
-          const int ch0 = 2 * c16;                   // bf16 chunk (8 dims) index within the row
-          *reinterpret_cast<uint4*>(Vb + (ch0 / 8) * kBlockBytes + sw128(kk, ch0 % 8)) = make_uint4(w[0], w[1], w[2], w[3]);
-          *reinterpret_cast<uint4*>(Vb + (ch0 / 8) * kBlockBytes + sw128(kk, ch0 % 8 + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
         }
         fence_async_smem();
         mbar_arrive(BAR(kBarVReady, vst));
