@@ -134,7 +134,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   atomicOr(status, MEPIC_DEV_WAIT_EXPIRED);
   return false;
 }
-// Same, with one verdict for the whole warp (the callers run warp-collective instructions afterwards).
+// Same, with one answer for the whole warp (the callers run warp-collective instructions afterwards).
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* status, int limit) {
   const bool w = mbar_wait(bar, parity, abort_flag, status, limit);
   return __all_sync(0xffffffffu, w) != 0;
