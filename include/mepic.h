@@ -454,6 +454,13 @@ int32_t mepic_attn_decode_fp8(const mepic_config_t* cfg, const mepic_decode_args
  * key range is cut into up to eight shares, one CTA each, whose per-row partials (reference, sum, unnormalised
  * output: 4 (head_dim + 2) bytes per row, q head and share) go to the workspace and are merged by a third kernel;
  * given a smaller workspace the call runs one CTA per item instead.  Errors as for decode.
+ * The attention kernel is enqueued twice.  The first launch expresses a tile's softmax weights against the reference
+ * its rows agreed on earlier (one pass over the scores); that is exact as long as no score lies more than 2^64 above
+ * the running reference, which a CTA notices from its row sums and records in the first word of the workspace (also
+ * its only use of the first 16 bytes; the commit kernel clears it).  The second launch returns at once unless that
+ * word is set, and otherwise does every item again with the reference found from the tile's own scores first (two
+ * passes), overwriting the first launch's results; either way `out` holds the exact-softmax result when the call's
+ * kernels have run.
  * A request may have no rows (row_offsets[b] == row_offsets[b+1]).  A call with no rows at all returns MEPIC_OK
  * without launching anything or reading any pointer but row_offsets_host.
  */

@@ -58,6 +58,7 @@ constexpr int kRotatorWarps = 4;
 constexpr int kKLoaderWarp = 20, kVLoaderWarp = 21, kMmaWarp = 22;   // warp 23 idles
 constexpr int kThreads = 768;
 constexpr float kRescaleThreshold = 8.f;   // move the reference maximum only when it lags by 2^8
+constexpr float kSaturation = 64.f;        // fast launch: a score more than this above the reference it was scaled by means "repeat"
 
 struct Item { int32_t b, h, row0, nq; };   // rows row0 .. row0+nq-1 (global row indices) of request b
 
@@ -83,6 +84,8 @@ struct PrefillParams {
   float scale_log2;
   float* k_scales;      // 8-bit pools only: [num_pages][n_kv_heads] scale of each (page, kv head) block of K (the commit writes them)
   float* v_scales;      // ... and of V
+  int32_t* redo_flag;   // first word of the workspace: set by a CTA of the fast launch one of whose rows outran its reference
+  int exact;            // 0: the fast launch; 1: the repeat launch (two passes on every tile; returns at once unless *redo_flag)
   int spin_limit;       // polls before a bounded wait gives up
   int skip_tile;        // test hook: CTA 0's K loader leaves out the copies of its key tile with this index (-1: none)
 };
@@ -211,6 +214,7 @@ __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.
 __global__ void mepic_prefill_commit(const PrefillParams p, int chunks_per_row) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the attention kernel may stage its queries meanwhile
   const int row = blockIdx.x;
+  if (row == 0 && threadIdx.x == 0) *p.redo_flag = 0;              // (an attention CTA that could set it waits for this grid first)
   __shared__ int sh_b;
   if (threadIdx.x == 0) {
     int b = 0;
@@ -247,6 +251,7 @@ __device__ __forceinline__ uint32_t e4m3x4_of(float a, float b, float c, float d
 __global__ void __launch_bounds__(256) mepic_prefill_commit_fp8(const PrefillParams p, int head_dim) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int row = blockIdx.x;
+  if (row == 0 && threadIdx.x == 0) *p.redo_flag = 0;
   __shared__ int sh_b;
   __shared__ unsigned sh_amax[2][8];         // [K | V][kv head], bit patterns of non-negative floats order like integers
   __shared__ float sh_scale[2][8];
@@ -433,6 +438,12 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int spin = HOOKS ? p.spin_limit : kSpinLimit;
+  if (p.exact == 1) {
+    // the repeat launch: nothing to do unless a CTA of the fast launch asked for it (then every item is done again)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (*reinterpret_cast<volatile int32_t*>(p.redo_flag) == 0) return;
+  }
+  volatile int* sat_flag = reinterpret_cast<volatile int*>(bars + kNumBars + 14);   // fast launch: a row outran its reference
   Item* item_slot = reinterpret_cast<Item*>(bars + kNumBars + 16);
   if (warp == 1) {
     const Item it = item_of_cta(p.row_offsets, p.batch, p.n_kv_heads, 2 * QT, p.max_q_tiles, blockIdx.x / p.n_splits, lane);
@@ -472,6 +483,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     mbar_init(BAR(kBarDrain, 0), 1);                         // tcgen05.commit
     for (int s = 0; s < kVStages; ++s) mbar_init(BAR(kBarVReady, s), kRotatorWarps * 32);
     *abort_flag = 0;
+    *sat_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_smem();
   }
@@ -563,8 +575,13 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       limit = p.q_slot[item.row0 + qi];
       if (limit < 0 || limit >= kvl) { atomicOr(p.status, MEPIC_DEV_BAD_SLOT); limit = limit < 0 ? 0 : kvl - 1; }
     }
-    float* mine = xchg + (x * 2 + ch) * 128 + r;
-    const float* theirs = xchg + (x * 2 + (ch ^ 1)) * 128 + r;
+    // exchange slots of the row's two threads, 2 KB in all.  First 1 KB: maxima of the two-pass tiles as bf16 (both
+    // threads take the rounded values, so they decide alike).  Second 1 KB: one byte per (tile parity, thread), the
+    // exponent of the thread's sum of P over the tile, which the partner reads one tile later without a meeting.
+    volatile uint16_t* mine = reinterpret_cast<volatile uint16_t*>(xchg) + (x * 2 + ch) * 128 + r;
+    const volatile uint16_t* theirs = reinterpret_cast<const volatile uint16_t*>(xchg) + (x * 2 + (ch ^ 1)) * 128 + r;
+    volatile unsigned char* lz_mine = reinterpret_cast<volatile unsigned char*>(xchg) + 1024 + (x * 2 + ch) * 128 + r;
+    const volatile unsigned char* lz_theirs = reinterpret_cast<const volatile unsigned char*>(xchg) + 1024 + (x * 2 + (ch ^ 1)) * 128 + r;
     const int pair_id = 1 + x * 4 + q4;         // hardware barrier of the two warps that share these 32 rows (0 is the CTA's)
     // publish `v`, meet the partner warp, return the partner's value of the same row.  The meeting point is a
     // hardware barrier (a waiting warp takes no issue slots and wakes at once); it has no time limit of its own, so
@@ -576,7 +593,25 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       if (*abort_flag) ok_io = false;
       return *src;
     };
-    float m_ref = -INFINITY, l_run = 0.f;
+    // the row's maximum over both halves, as both threads see it (bf16, round to nearest)
+    auto row_max_of = [&](float v, bool& ok_io) {
+      const uint32_t mine_r = pack_bf16x2(v, v);
+      *mine = static_cast<uint16_t>(mine_r);
+      asm volatile("bar.sync %0, 64;" ::"r"(pair_id) : "memory");
+      if (*abort_flag) ok_io = false;
+      return fmaxf(__uint_as_float(mine_r << 16), __uint_as_float(static_cast<uint32_t>(*theirs) << 16));
+    };
+    // The reference 2^m_ref that P is expressed in only has to be the same for both threads of the row, not far above
+    // the row's maximum so far (else every P of a row could vanish) and close enough below the scores for P to stay in
+    // range.  The first tile finds it in a pass of its own over the scores and a meeting of the two threads (two
+    // passes).  In the fast launch later tiles make one pass with the reference they have; what tells them to raise it
+    // is the sum of P of the tile before: each thread leaves the exponent of its sum in shared memory before it
+    // hands P over, and reads its partner's at the next tile (the hand-over, the MMA and the next S order the two).
+    // floor(log2(sum)) + 1 added to the reference puts it above every score of that tile by at most 8.  A thread whose
+    // sum reaches 2^kSaturation (or overflows) raises sat_flag: the call then repeats every item with two passes on every
+    // tile (the repeat launch).
+    float m_ref = -INFINITY, m_next = -INFINITY, l_run = 0.f;
+    int e_prev = 0;                               // exponent field of my sum of P over the tile before
     bool ok = true;
     const int my_tiles = nt[x];
     for (int tile = 0; tile < my_tiles; ++tile) {
@@ -584,9 +619,17 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       tc_fence_after();
       const int n_vis = limit - (tile_base + tile) * kTileN + 1 - 64 * ch;     // my columns [0, n_vis) are visible to this row
       const bool boundary = n_vis < 64;                          // only the tile(s) on the causal boundary need the mask
-      // ---- pass 1: maximum of my 64 scores
+      // two passes: the repeat launch, the first tile, and any tile at which a row of this warp has no reference yet
+      // (both warps of the pair hold the same rows and the same references: they decide alike)
+      if (!p.exact && tile > 0) {
+        const int e = max(e_prev, static_cast<int>(lz_theirs[((tile - 1) & 1) * 512]));
+        if (e > 127 + static_cast<int>(kRescaleThreshold) && m_ref != -INFINITY) m_next = m_ref + static_cast<float>(e - 126);
+      }
+      const bool two_pass = p.exact || tile == 0 || __any_sync(0xffffffffu, m_next == -INFINITY);
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
-      {
+      float alpha = 1.f;
+      if (two_pass) {
+        // ---- pass 1: maximum of my 64 scores
         uint32_t sv[64];                  // both loads in flight at once: one wait
         TMEM_LD32(t_H, sv, 0);
         TMEM_LD32(t_H + 32, sv, 32);
@@ -600,16 +643,19 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
 #pragma unroll
           for (int k = 0; k < 4; ++k) mx4[k] = fmaxf(mx4[k], __uint_as_float(sv[c + k]));
         }
-      }
-      float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-      mx = fmaxf(mx, swap_with_partner(mx, ok, mine, theirs));
-      if (!ok) break;
-      // move the reference only when it lags by more than the threshold (both threads of the row decide alike);
-      // always true on the first tile: m_ref = -inf and key 0 is visible to every row
-      float alpha = 1.f;
-      if (mx > m_ref + kRescaleThreshold) {
-        alpha = ex2(m_ref - mx);
-        m_ref = mx;
+        const float mx = row_max_of(fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])), ok);
+        if (!ok) break;
+        // move the reference only when it lags by more than the threshold (both threads of the row decide alike);
+        // always true on the first tile that shows the row a key
+        const float m_new = mx > m_next + kRescaleThreshold ? mx : m_next;      // m_next >= m_ref: a raise still pending
+        if (m_new != m_ref) {
+          alpha = ex2(m_ref - m_new);
+          m_ref = m_new;
+        }
+        m_next = m_ref;
+      } else if (m_next != m_ref) {
+        alpha = ex2(m_ref - m_next);
+        m_ref = m_next;
       }
       // O holds every earlier tile's PV, all complete: this tile's S was issued after them.  Each thread of the
       // row rescales its own half of the O columns.
@@ -651,7 +697,11 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         }
         TMEM_ST16(t_H + 16 * q, pw);      // chunk q's P over columns that hold only consumed scores
       }
-      l_run = l_run * alpha + (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
+      const float l_tile = (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
+      l_run = l_run * alpha + l_tile;
+      e_prev = static_cast<int>((__float_as_uint(l_tile) >> 23) & 0xffu);
+      lz_mine[(tile & 1) * 512] = static_cast<unsigned char>(e_prev);
+      if (!(l_tile < 1.8446744e19f)) *sat_flag = 1;             // 2^64 and beyond, inf or NaN: repeat (the repeat launch never gets here with such a sum)
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(BAR(kBarPFull, x));
@@ -1025,6 +1075,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
+  if (tid == 0 && *sat_flag) *p.redo_flag = 1;
 }
 
 constexpr int kMaxSplits = 8;           // most shares a work item's key range is cut into
@@ -1085,7 +1136,14 @@ int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& m
   cudaLaunchConfig_t lc = {};
   lc.gridDim = dim3(static_cast<unsigned>(n_items * p.n_splits)); lc.blockDim = dim3(kThreads); lc.dynamicSmemBytes = smem; lc.stream = stream;
   lc.attrs = pdl; lc.numAttrs = 1;
-  e = cudaLaunchKernelEx(&lc, mepic_prefill_attn<D, G, FP8, HOOKS>, p, map_k, map_v);
+  // the fast launch, then the repeat launch, which does nothing unless a row outran its reference in the first
+  PrefillParams pf = p;
+  pf.exact = 0;
+  e = cudaLaunchKernelEx(&lc, mepic_prefill_attn<D, G, FP8, HOOKS>, pf, map_k, map_v);
+  if (e == cudaSuccess) {
+    pf.exact = 1;
+    e = cudaLaunchKernelEx(&lc, mepic_prefill_attn<D, G, FP8, HOOKS>, pf, map_k, map_v);
+  }
   if (e == cudaSuccess && p.n_splits > 1) {
     const long long n_pairs = static_cast<long long>(p.total_rows) * p.n_kv_heads * G;
     lc.gridDim = dim3(static_cast<unsigned>((n_pairs + 3) / 4)); lc.blockDim = dim3(128); lc.dynamicSmemBytes = 0;
@@ -1093,7 +1151,7 @@ int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& m
   }
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("prefill: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
-  mepic_count_launches(p.n_splits > 1 ? 3 : 2);
+  mepic_count_launches(p.n_splits > 1 ? 4 : 3);
   return MEPIC_OK;
 }
 
@@ -1195,6 +1253,8 @@ static int32_t prefill_call(const mepic_config_t* cfg, const mepic_prefill_args_
   p.max_q_tiles = max_q_tiles;
   p.n_splits = splits_for(n_items);
   if (a->workspace_bytes < split_workspace_bytes(cfg, total_rows, p.n_splits)) p.n_splits = 1;     // no room for partials: one CTA per item
+  p.redo_flag = static_cast<int32_t*>(a->workspace);
+  p.exact = 0;
   p.part_o = reinterpret_cast<float*>(static_cast<unsigned char*>(a->workspace) + 16);
   p.part_ml = p.part_o + static_cast<size_t>(p.n_splits) * total_rows * cfg->n_q_heads * cfg->head_dim;
   p.scale_log2 = a->sm_scale * 1.4426950408889634f;

@@ -283,6 +283,10 @@ class PrefillBatch:
                            sm_scale=sm_scale, stream=s)
         return self.out
 
+    def repeated(self) -> bool:
+        """Whether the last call ran its repeat launch (first workspace word; synchronises the device)."""
+        return int(self.workspace[:4].view(torch.int32).item()) != 0
+
 
 class Fp8PrefillBatch(PrefillBatch):
     """A prefill batch that commits into, and attends over, the 8-bit pools."""

@@ -34,7 +34,7 @@ def _check(got_bits, want, what=""):
     assert rel <= REL_L2, (what, rel)
 
 
-def _run_prefill(cfg, kp, vp, page_ids, pos_base, kv_len, q_slots, rows, sm_scale, theta, sample_rows=None):
+def _run_prefill(cfg, kp, vp, page_ids, pos_base, kv_len, q_slots, rows, sm_scale, theta, sample_rows=None, expect_repeat=False):
     """q_slots: list (per request) of int arrays; rows: list of PrefillRows-like (q_new, k_new, v_new)."""
     B = len(q_slots)
     row_offsets = np.zeros(B + 1, dtype=np.int32)
@@ -48,6 +48,7 @@ def _run_prefill(cfg, kp, vp, page_ids, pos_base, kv_len, q_slots, rows, sm_scal
     out = batch.run(sm_scale)
     torch.cuda.synchronize()
     assert dev.read_status() == 0
+    assert batch.repeated() == expect_repeat, "the fast launch must do (only) for ordinary scores"
     got = RT.bf16_bits(out)
     got_k, got_v = RT.bf16_bits(dev.k_pool), RT.bf16_bits(dev.v_pool)
     # oracle: commits into its own copy of the pools, request by request
@@ -195,7 +196,7 @@ def test_small_grids_split_the_key_range_and_agree_with_the_unsplit_run():
     batch.ws_bytes = 16                                     # no room for partials: the library must fall back to one CTA per item
     out = batch.run(0.1)
     torch.cuda.synchronize()
-    assert dev.read_status() == 0 and M.mepic_launch_count() - launches == 2
+    assert dev.read_status() == 0 and M.mepic_launch_count() - launches == 3
     ok, ov = kp.copy(), vp.copy()
     want = O.prefill_attention_one(rows[0].q_new, rows[0].k_new, rows[0].v_new, list(slots[0]), ok, ov, list(ids[0, :-(-L // 16)]),
                                    list(base[0, :-(-L // 16)]), L, 0.1, 5e5)
@@ -233,18 +234,42 @@ def test_request_without_new_rows_and_call_without_any():
     assert np.array_equal(RT.bf16_bits(dev.k_pool), kp) and np.array_equal(RT.bf16_bits(dev.v_pool), vp)
 
 
-def test_one_dominant_key_in_a_late_tile_rescales_everything_accumulated_before():
-    # A key ~80 nats above all others in the fourth 128-key tile: the rows' reference jumps there, O and the row sums
+@pytest.mark.parametrize("big_value,repeat", [(15.0, False), (30.0, True)])
+def test_one_dominant_key_in_a_late_tile_rescales_everything_accumulated_before(big_value, repeat):
+    # A key far above all others in the fourth 128-key tile: the rows' reference jumps there, O and the row sums
     # of the first three tiles are multiplied down to nothing, later tiles leave the reference alone.  The big
     # components sit in the slowest-rotating pair (63, 127), so the score barely depends on the positions.
-    specs = [(1000, list(range(0, 16)) + list(range(900, 1000)))]
+    # 15 x 15: the score is ~29 (log2 units) above the rest: the fast launch carries P up to 2^29 through that tile and
+    # raises its reference one tile later.  30 x 30: ~115 above, beyond what the fast launch may carry (2^64): it must
+    # ask for the repeat launch, whose two-pass softmax gives the result.
+    # (One request: its four work items are cut into eight key-range shares of four tiles each; the key sits in the
+    # third tile of the third share, so that share meets it in a one-pass tile.)
+    specs = [(4000, list(range(0, 16)) + list(range(3900, 4000)))]
     cfg, kp, vp, ids, base, kvl, slots, rows = _manual(41, Hq=8, Hkv=2, D=128, P=16, specs=specs)
-    big = f32_to_bf16_bits(np.array([30.0], dtype=np.float32))[0]
+    big = f32_to_bf16_bits(np.array([big_value], dtype=np.float32))[0]
     rows[0].q_new[:, :, 63] = big
-    t = 450
+    t = 10 * 128 + 5
     kp[ids[0, t // 16], :, t % 16, 63] = big
-    dev, batch = _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 1.0 / np.sqrt(128), 1e4)
+    dev, batch = _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 1.0 / np.sqrt(128), 1e4, expect_repeat=repeat)
     got = bf16_bits_to_f64(RT.bf16_bits(batch.out))                                  # [116, 8, 128]
     v_star = np.repeat(bf16_bits_to_f64(vp[ids[0, t // 16], :, t % 16, :]), 4, axis=0)
-    late = got[16:]                                                                  # rows at slots 900..999 see the key
+    late = got[16:]                                                                  # rows at slots 3900..3999 see the key
     assert np.abs(late - v_star[None]).max() <= 2e-2
+    # the same batch again with ordinary queries: the flag of the call before must not linger
+    if repeat:
+        rows[0].q_new[:, :, 63] = f32_to_bf16_bits(np.array([0.5], dtype=np.float32))[0]
+        _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 1.0 / np.sqrt(128), 1e4, expect_repeat=False)
+
+
+def test_dominant_key_with_many_work_items_takes_the_repeat_launch_unsplit():
+    # as above on a batch that fills more than one wave of CTAs (no key-range shares): 40 requests, one of which
+    # holds the dominant key; every item is done again by the repeat launch and all of them must still match the oracle
+    specs = [(700, list(range(0, 16)) + list(range(500, 700))) for _ in range(40)]
+    cfg, kp, vp, ids, base, kvl, slots, rows = _manual(43, Hq=8, Hkv=2, D=128, P=16, specs=specs)
+    big = f32_to_bf16_bits(np.array([30.0], dtype=np.float32))[0]
+    rows[7].q_new[:, :, 63] = big
+    t = 300
+    kp[ids[7, t // 16], :, t % 16, 63] = big
+    dev, batch = _run_prefill(cfg, kp, vp, ids, base, kvl, slots, rows, 1.0 / np.sqrt(128), 1e4,
+                              sample_rows=lambda R: [0, 15, 16, R // 2, R - 1], expect_repeat=True)
+    assert batch.ws_bytes == 16, "this grid is expected to run one CTA per item"
