@@ -381,8 +381,8 @@ struct PrefillSmem {
   static constexpr int kQ = 0;                                     // two M-tiles of Q'
   static constexpr int kK = kQ + 2 * NB * kBlockBytes;
   static constexpr int kV = kK + kKStages * NB * kBlockBytes;
-  static constexpr int kXchg = kV + kVStages * NB * kBlockBytes;   // float [2 M-tiles][2 halves][128 rows]: row-half exchange
-  static constexpr int kBars = kXchg + 2 * 2 * 128 * 4;            // mbarriers and small state
+  static constexpr int kXchg = kV + kVStages * NB * kBlockBytes;   // float [2 M-tiles][2 halves][128 rows], then a byte each: the exchange of a row's two threads
+  static constexpr int kBars = kXchg + 2 * 2 * 128 * 4 + 2 * 2 * 128;   // mbarriers and small state
   static constexpr int kBytes = kBars + 512;
 };
 
@@ -575,13 +575,15 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       limit = p.q_slot[item.row0 + qi];
       if (limit < 0 || limit >= kvl) { atomicOr(p.status, MEPIC_DEV_BAD_SLOT); limit = limit < 0 ? 0 : kvl - 1; }
     }
-    // exchange slots of the row's two threads, 2 KB in all.  First 1 KB: maxima of the two-pass tiles as bf16 (both
-    // threads take the rounded values, so they decide alike).  Second 1 KB: one byte per (tile parity, thread), the
-    // exponent of the thread's sum of P over the tile, which the partner reads one tile later without a meeting.
-    volatile uint16_t* mine = reinterpret_cast<volatile uint16_t*>(xchg) + (x * 2 + ch) * 128 + r;
-    const volatile uint16_t* theirs = reinterpret_cast<const volatile uint16_t*>(xchg) + (x * 2 + (ch ^ 1)) * 128 + r;
-    volatile unsigned char* lz_mine = reinterpret_cast<volatile unsigned char*>(xchg) + 1024 + (x * 2 + ch) * 128 + r;
-    const volatile unsigned char* lz_theirs = reinterpret_cast<const volatile unsigned char*>(xchg) + 1024 + (x * 2 + (ch ^ 1)) * 128 + r;
+    // exchange slots of the row's two threads.  2 KB: the fp32 maximum of a two-pass tile, one word per thread.  512
+    // bytes after them: one byte per thread that tells the partner, one tile later and without a meeting, how far the
+    // thread's sum of P over a tile ran ahead of the reference: two 4-bit codes, low nibble for even tiles, high nibble
+    // for odd ones (the owner keeps the byte in a register and stores all of it, so a tile's code stays readable until
+    // the tile after next overwrites it).
+    volatile float* mine = xchg + (x * 2 + ch) * 128 + r;
+    const volatile float* theirs = xchg + (x * 2 + (ch ^ 1)) * 128 + r;
+    volatile unsigned char* lz_mine = reinterpret_cast<volatile unsigned char*>(xchg + 512) + (x * 2 + ch) * 128 + r;
+    const volatile unsigned char* lz_theirs = reinterpret_cast<const volatile unsigned char*>(xchg + 512) + (x * 2 + (ch ^ 1)) * 128 + r;
     const int pair_id = 1 + x * 4 + q4;         // hardware barrier of the two warps that share these 32 rows (0 is the CTA's)
     // publish `v`, meet the partner warp, return the partner's value of the same row.  The meeting point is a
     // hardware barrier (a waiting warp takes no issue slots and wakes at once); it has no time limit of its own, so
@@ -593,25 +595,26 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       if (*abort_flag) ok_io = false;
       return *src;
     };
-    // the row's maximum over both halves, as both threads see it (bf16, round to nearest)
+    // the row's maximum over both halves.  (The partner reads this thread's word right after the meeting; the word
+    // is next written in a later two-pass tile, after an S that was issued once both threads had handed P over.)
     auto row_max_of = [&](float v, bool& ok_io) {
-      const uint32_t mine_r = pack_bf16x2(v, v);
-      *mine = static_cast<uint16_t>(mine_r);
+      *mine = v;
       asm volatile("bar.sync %0, 64;" ::"r"(pair_id) : "memory");
       if (*abort_flag) ok_io = false;
-      return fmaxf(__uint_as_float(mine_r << 16), __uint_as_float(static_cast<uint32_t>(*theirs) << 16));
+      return fmaxf(v, *theirs);
     };
     // The reference 2^m_ref that P is expressed in only has to be the same for both threads of the row, not far above
     // the row's maximum so far (else every P of a row could vanish) and close enough below the scores for P to stay in
     // range.  The first tile finds it in a pass of its own over the scores and a meeting of the two threads (two
     // passes).  In the fast launch later tiles make one pass with the reference they have; what tells them to raise it
-    // is the sum of P of the tile before: each thread leaves the exponent of its sum in shared memory before it
-    // hands P over, and reads its partner's at the next tile (the hand-over, the MMA and the next S order the two).
-    // floor(log2(sum)) + 1 added to the reference puts it above every score of that tile by at most 8.  A thread whose
-    // sum reaches 2^kSaturation (or overflows) raises sat_flag: the call then repeats every item with two passes on every
-    // tile (the repeat launch).
+    // is the sum of P of the tile before: a thread whose sum exceeds 2^8 leaves the code c = ceil((floor(log2(sum)) + 1)
+    // / 8) in shared memory before it hands P over, and reads its partner's at the next tile (the hand-over, the MMA
+    // and the next S order the two); 8 max(c, c') added to the reference puts it above every score of that tile by
+    // less than 16.  A thread whose sum reaches 2^kSaturation (or overflows) raises sat_flag: the call then repeats
+    // every item with two passes on every tile (the repeat launch).
     float m_ref = -INFINITY, m_next = -INFINITY, l_run = 0.f;
-    int e_prev = 0;                               // exponent field of my sum of P over the tile before
+    int c_prev = 0;                               // my code for the tile before
+    uint32_t lz_byte = 0;                         // my byte of codes as it stands in shared memory
     bool ok = true;
     const int my_tiles = nt[x];
     for (int tile = 0; tile < my_tiles; ++tile) {
@@ -622,8 +625,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       // two passes: the repeat launch, the first tile, and any tile at which a row of this warp has no reference yet
       // (both warps of the pair hold the same rows and the same references: they decide alike)
       if (!p.exact && tile > 0) {
-        const int e = max(e_prev, static_cast<int>(lz_theirs[((tile - 1) & 1) * 512]));
-        if (e > 127 + static_cast<int>(kRescaleThreshold) && m_ref != -INFINITY) m_next = m_ref + static_cast<float>(e - 126);
+        const int c = max(c_prev, (static_cast<int>(*lz_theirs) >> (4 * ((tile - 1) & 1))) & 15);
+        if (c > 0 && m_ref != -INFINITY) m_next = m_ref + static_cast<float>(8 * c);
       }
       const bool two_pass = p.exact || tile == 0 || __any_sync(0xffffffffu, m_next == -INFINITY);
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
@@ -699,8 +702,12 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       }
       const float l_tile = (sum2[0].x + sum2[0].y) + (sum2[1].x + sum2[1].y);
       l_run = l_run * alpha + l_tile;
-      e_prev = static_cast<int>((__float_as_uint(l_tile) >> 23) & 0xffu);
-      lz_mine[(tile & 1) * 512] = static_cast<unsigned char>(e_prev);
+      {
+        const int e = static_cast<int>((__float_as_uint(l_tile) >> 23) & 0xffu);       // floor(log2(sum)) + 127
+        c_prev = e > 127 + static_cast<int>(kRescaleThreshold) ? min(15, (e - 126 + 7) >> 3) : 0;
+        lz_byte = (tile & 1) ? (lz_byte & 0x0fu) | (static_cast<uint32_t>(c_prev) << 4) : (lz_byte & 0xf0u) | static_cast<uint32_t>(c_prev);
+        *lz_mine = static_cast<unsigned char>(lz_byte);
+      }
       if (!(l_tile < 1.8446744e19f)) *sat_flag = 1;             // 2^64 and beyond, inf or NaN: repeat (the repeat launch never gets here with such a sum)
       tmem_wait_st();
       tc_fence_before();
