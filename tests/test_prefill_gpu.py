@@ -67,6 +67,10 @@ def _run_prefill(cfg, kp, vp, page_ids, pos_base, kv_len, q_slots, rows, sm_scal
                                        rows=sel)
         g = got[row_offsets[b]:row_offsets[b + 1]]
         _check(g if sel is None else g[sel], want, f"request {b}")
+        if q_slots[b][0] == 0:
+            # a row at slot 0 sees one key, its own: softmax weight exactly 1, the output is that row's V bit for bit
+            G = cfg.n_q_heads // cfg.n_kv_heads
+            assert np.array_equal(g[0], np.repeat(rows[b].v_new[0], G, axis=0)), f"request {b}: row at slot 0 is not its V"
     assert np.array_equal(got_k, ok) and np.array_equal(got_v, ov), "pool after commit differs from the oracle's"
     return dev, batch
 
