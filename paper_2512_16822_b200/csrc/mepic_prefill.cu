@@ -55,7 +55,7 @@ constexpr int kBlockBytes = 128 * 128; // one [128 rows x 64 bf16] swizzled bloc
 constexpr int kTmemCols = 512;         // S of M-tile a: 0..127, of b: 128..255; O of a: 256.., of b: 384..
 constexpr int kSoftmaxWarps = 16;       // 2 M-tiles x 2 column halves x 4 lane quadrants: two threads share a row
 constexpr int kRotatorWarps = 4;
-constexpr int kKLoaderWarp = 20, kVLoaderWarp = 21, kMmaWarp = 22;   // warp 23 idles
+constexpr int kKLoaderWarp = 20, kVLoaderWarp = 21, kMmaWarp = 22, kSpareWarp = 23;   // the spare warp idles unless the pages are 8-bit
 constexpr int kThreads = 768;
 constexpr float kRescaleThreshold = 8.f;   // move the reference maximum only when it lags by 2^8
 constexpr float kSaturation = 64.f;        // fast launch: a score more than this above the reference it was scaled by means "repeat"
@@ -481,7 +481,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     mbar_init(BAR(kBarVPatched, 0), 1);
     mbar_init(BAR(kBarQReady, 0), kSoftmaxWarps * 32);      // the softmax warps stage Q'
     mbar_init(BAR(kBarDrain, 0), 1);                         // tcgen05.commit
-    for (int s = 0; s < kVStages; ++s) mbar_init(BAR(kBarVReady, s), kRotatorWarps * 32);
+    for (int s = 0; s < kVStages; ++s) mbar_init(BAR(kBarVReady, s), 2 * 32);            // the two V converter warps
     *abort_flag = 0;
     *sat_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -854,47 +854,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         }
         fence_async_smem();
         mbar_arrive(BAR(kBarKReady, st));
-        // ---- the V tile of the same index: widen, scale, store; rows at or past kv_len become zero (P is 0 there,
-        // but 0 x NaN is NaN)
-        const int vst = tile % kVStages;
-        if (!mbar_wait(BAR(kBarVLanded, vst), static_cast<uint32_t>(tile / kVStages) & 1u, abort_flag, p.status, spin)) break;
-        unsigned char* Vb = Vs + vst * NB * kBlockBytes;
-        {
-          // all of the thread's eight 16-byte chunks of codes are requested before the first is used: one load latency
-          // per tile instead of four.  Chunk idx = rt + 128 i: key idx / 8, dims [16 (idx % 8), +16)
-          uint4 cd[8];
-          float sc[8];
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int idx = rt + 128 * i, kk = idx >> 3, c16 = idx & 7;
-            const int vr = vrow[vst * 8 + (kk >> 4)];
-            const bool live = vr >= 0 && key0 + kk < kvl;
-            cd[i] = make_uint4(0, 0, 0, 0); sc[i] = 0.f;
-            if (live) {
-              cd[i] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(p.v_pool) + static_cast<size_t>(vr + (kk & 15)) * D + 16 * c16));
-              sc[i] = __ldg(p.v_scales + vr / p.page_size);
-            }
-          }
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int idx = rt + 128 * i, kk = idx >> 3, c16 = idx & 7;
-            const uint32_t cw[4] = {cd[i].x, cd[i].y, cd[i].z, cd[i].w};
-            uint32_t w[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-              uint32_t hh;
-              asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(hh) : "h"(static_cast<uint16_t>(cw[j >> 1] >> (16 * (j & 1)))));
-              const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hh));
-              w[j] = pack_bf16x2(f.x * sc[i], f.y * sc[i]);       // a dead row: codes 0 and scale 0 give zeros
-            }
-            const int ch0 = 2 * c16;                   // bf16 chunk (8 dims) index within the row
-            *reinterpret_cast<uint4*>(Vb + (ch0 / 8) * kBlockBytes + sw128(kk, ch0 % 8)) = make_uint4(w[0], w[1], w[2], w[3]);
-            *reinterpret_cast<uint4*>(Vb + (ch0 / 8) * kBlockBytes + sw128(kk, ch0 % 8 + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
-          }
-        }
-        fence_async_smem();
-        mbar_arrive(BAR(kBarVReady, vst));
-        continue;
+        continue;                    // (the V tile is the V converters' work)
       }
 #pragma unroll 2
       for (int i = 0; i < CH; ++i) {
@@ -925,6 +885,67 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       }
       fence_async_smem();
       mbar_arrive(BAR(kBarKReady, st));
+    }
+  } else if (FP8 && (warp == kVLoaderWarp || warp == kSpareWarp)) {
+    // =============================================================== 8-bit pages: the V converters
+    // The V loader (which has nothing to copy) and the spare warp widen the V tile, 64 keys each: codes from global
+    // memory, times the block's scale, rounded to bf16 into the stage the PV MMA reads; rows at or past kv_len become
+    // zero (P is 0 there, but 0 x NaN is NaN).  Every decision that precedes a shuffle is the whole warp's.
+    const int half = warp == kVLoaderWarp ? 0 : 1;
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // this role reads the pools itself: after the commit kernel
+    for (int tile = 0; tile < n_tiles; ++tile) {
+      const int vst = tile % kVStages;
+      if (tile >= kVStages &&
+          !mbar_wait_warp(BAR(kBarVFree, vst), static_cast<uint32_t>(tile / kVStages - 1) & 1u, abort_flag, p.status, spin)) break;
+      const int key0 = (tile_base + tile) * kTileN;
+      // lane g (mod 4) looks up 16-key group 4 half + g: pool row of its first key (-1: none below kv_len), its block's scale
+      const int gkey = key0 + (half * 4 + (lane & 3)) * 16;
+      int row = -1;
+      float scl = 0.f;
+      if (gkey < kvl) {
+        const int e = gkey / p.page_size;
+        int page = __ldg(ids + e);
+        if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
+        row = (page * p.n_kv_heads + h) * p.page_size + gkey % p.page_size;
+        scl = __ldg(p.v_scales + page * p.n_kv_heads + h);
+      }
+      unsigned char* Vb = Vs + vst * NB * kBlockBytes;
+#pragma unroll 1
+      for (int i0 = 0; i0 < 16; i0 += 8) {
+        // a lane's 16 chunks of 16 codes in two batches of eight requests: chunk idx = lane + 32 i of the warp's 64 keys
+        // is key idx / 8, dims [16 (idx % 8), +16); the eight chunks of a batch lie in groups (i0 + u) / 4
+        uint4 cd[8];
+        float sc[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int idx = lane + 32 * (i0 + u), kl = idx >> 3, c16 = idx & 7;
+          const int vr = __shfl_sync(0xffffffffu, row, (i0 + u) >> 2);
+          const float gs = __shfl_sync(0xffffffffu, scl, (i0 + u) >> 2);
+          cd[u] = make_uint4(0, 0, 0, 0); sc[u] = 0.f;
+          if (vr >= 0 && key0 + half * 64 + kl < kvl) {
+            cd[u] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(p.v_pool) + static_cast<size_t>(vr + (kl & 15)) * D + 16 * c16));
+            sc[u] = gs;
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          const int idx = lane + 32 * (i0 + u), kk = half * 64 + (idx >> 3), c16 = idx & 7;
+          const uint32_t cw[4] = {cd[u].x, cd[u].y, cd[u].z, cd[u].w};
+          uint32_t w[8];
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            uint32_t hh;
+            asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(hh) : "h"(static_cast<uint16_t>(cw[j >> 1] >> (16 * (j & 1)))));
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&hh));
+            w[j] = pack_bf16x2(f.x * sc[u], f.y * sc[u]);       // a dead row: codes 0 and scale 0 give zeros
+          }
+          const int ch0 = 2 * c16;                   // bf16 chunk (8 dims) index within the row
+          *reinterpret_cast<uint4*>(Vb + (ch0 / 8) * kBlockBytes + sw128(kk, ch0 % 8)) = make_uint4(w[0], w[1], w[2], w[3]);
+          *reinterpret_cast<uint4*>(Vb + (ch0 / 8) * kBlockBytes + sw128(kk, ch0 % 8 + 1)) = make_uint4(w[4], w[5], w[6], w[7]);
+        }
+      }
+      fence_async_smem();
+      mbar_arrive(BAR(kBarVReady, vst));
     }
   } else if (warp == kKLoaderWarp || warp == kVLoaderWarp) {
     // =============================================================== loader warps: lane g loads 16-key group g
