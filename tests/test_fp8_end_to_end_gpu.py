@@ -165,3 +165,48 @@ def test_store_prefill_decode_on_8bit_pools_only(Hq, Hkv, P, n_chunks, chunk_pag
             side.prefill(new_tabs, new_rows, sm, what=f"append step {step}")
             tabs = new_tabs
         side.decode(tabs, bits((2, Hq, D)), sm, what="after the appends")
+
+
+def test_config3_full_size_prefill_on_8bit_pools_sampled_rows():
+    # The launch bench.py times (8 requests x 768 rows over 16 640 cached tokens, 8-bit pools, no bf16 copy while the
+    # call runs).  The oracle quantises the pages request 0 reads (the library's codes and scales for them must agree
+    # bit for bit), commits request 0's rows by its own rule and evaluates sampled rows on those codes and scales.
+    from mepic_inputs import make_workload
+    wl = make_workload(3)
+    cfg = M.Config(wl.page_size, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.num_pages, wl.max_position,
+                   wl.rope_theta, wl.pad_token_id)
+    kp, vp = wl.kv_pool()
+    with M.Store(cfg) as st:
+        tables = RT.build_tables(st, wl.chunks, wl.prefill_requests)
+    page_ids, pos_base, kv_len, _ = RT.pack_tables(tables, wl.page_size)
+    q_slots = [np.asarray(t.recompute_slots, dtype=np.int32) for t in tables]
+    rows = [wl.prefill_rows(i, len(s)) for i, s in enumerate(q_slots)]
+    ro = np.concatenate([[0], np.cumsum([len(s) for s in q_slots])]).astype(np.int32)
+    dev = RT.Device(cfg, kp, vp)
+    pools = RT.Fp8Pools(dev)                              # the library's quantiser over the whole pool
+    torch.cuda.synchronize()
+    dev.k_pool = dev.v_pool = None                        # from here on the 8-bit pools are the only pools
+    torch.cuda.empty_cache()
+    n0 = -(-int(kv_len[0]) // wl.page_size)
+    mine = np.unique(page_ids[0, :n0])
+    okc, oks = O.quantize_pages(kp[mine]); ovc, ovs = O.quantize_pages(vp[mine])
+    sel = torch.from_numpy(mine.astype(np.int64)).to(dev.device)
+    assert np.array_equal(pools.k_codes[sel].cpu().numpy(), okc) and np.array_equal(pools.k_scales[sel].cpu().numpy(), oks)
+    assert np.array_equal(pools.v_codes[sel].cpu().numpy(), ovc) and np.array_equal(pools.v_scales[sel].cpu().numpy(), ovs)
+    pb = RT.Fp8PrefillBatch(pools, page_ids, pos_base, kv_len, ro, np.concatenate(q_slots),
+                            np.concatenate([r.q_new for r in rows]), np.concatenate([r.k_new for r in rows]),
+                            np.concatenate([r.v_new for r in rows]))
+    out = pb.run(wl.sm_scale); torch.cuda.synchronize()
+    assert dev.read_status() == 0 and not pb.repeated()
+    # the oracle's copy of request 0's pages, renumbered 0 .. len(mine) - 1
+    local = {int(pg): i for i, pg in enumerate(mine)}
+    ids0 = [local[int(pg)] for pg in page_ids[0, :n0]]
+    O.commit_rows_fp8(okc, oks, ovc, ovs, ids0, list(q_slots[0]), rows[0].k_new, rows[0].v_new)
+    assert np.array_equal(pools.k_codes[sel].cpu().numpy(), okc) and np.array_equal(pools.k_scales[sel].cpu().numpy(), oks)
+    assert np.array_equal(pools.v_codes[sel].cpu().numpy(), ovc) and np.array_equal(pools.v_scales[sel].cpu().numpy(), ovs)
+    R = len(q_slots[0])
+    pick = sorted(set([0, 1, 15, 16, 255, 256, R // 2, R - 257, R - 256, R - 2, R - 1] + list(range(5, R, 61))))
+    want = O.prefill_attention_one(rows[0].q_new, rows[0].k_new, rows[0].v_new, list(q_slots[0]),
+                                   O.dequantize_pages(okc, oks), O.dequantize_pages(ovc, ovs), ids0, list(pos_base[0, :n0]),
+                                   int(kv_len[0]), wl.sm_scale, wl.rope_theta, rows=pick)
+    _check(RT.bf16_bits(out)[:R][pick], want, 2e-2, "config 3, request 0, 8-bit pools")
