@@ -401,11 +401,12 @@ constexpr int kBarDrain = kBarQReady + 1;                   // [1] after a lost 
 constexpr int kBarVReady = kBarDrain + 1;                   // [kVStages] 8-bit pages only: the V stage has been widened to bf16
 constexpr int kNumBars = kBarVReady + kVStages;
 
-// FP8 = the pools hold e4m3 codes with one scale per (page, kv head) block: no TMA then (the tensor cores need bf16
-// operands in the swizzled layout, and shared memory has no room for a second, 8-bit copy of the rings): the loader warps
-// only publish where each 16-key group of the tile lives, and the rotator warps fetch the codes from global memory
-// themselves, widen them exactly, fold the block's scale into the rotation constants (K) or the widening (V) and write
-// the bf16 stage the MMA reads.  Everything downstream of the stages is unchanged.
+// FP8 = the pools hold e4m3 codes with one scale per (page, kv head) block.  The tensor cores need bf16 operands in the
+// swizzled layout, so the codes are widened on the way: the K ring has two stages, the third stage's room stages the raw
+// codes of one K and one V tile, which the K loader warp brings with untiled bulk copies; the rotator warps read the K
+// codes there, fold the block's scale into the rotation constants and write the bf16 stage the MMA reads, and two
+// converter warps (the V loader, which has nothing to copy, and the spare warp) do the same for V.  Everything
+// downstream of the stages is unchanged.
 // HOOKS = the test build of the kernel: the poll limit of the bounded waits and the one left-out K tile come from the
 // launch parameters (mepic_kernel_test_hooks).  The production instantiation has the limit as a compile-time constant
 // and no such check: the issuing thread's wait loops are on the critical path of every tile (measured: 2 % of the call).
@@ -419,6 +420,10 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   constexpr uint32_t kIdescQK = instr_desc(128, kTileN, 0, 0);
   constexpr uint32_t kIdescPV = instr_desc(128, D, 0, 1);
   constexpr uint32_t kGroupBytes = 16u * D * 2u;        // the rows of one 16-token group in one pool
+  // 8-bit pages: the K ring has two stages and the third stage's 32 KB stage the raw codes of one K tile and one V tile
+  // (16 KB each, [key][128 bytes]), brought by bulk copies; the barriers of the unused K / V "landed" slots serve them
+  constexpr int KD = FP8 ? 2 : kKStages;                // depth of the bf16 K ring
+  constexpr uint32_t kCodeGroupBytes = 16u * 128u;      // the codes of one 16-token group
 
   // 1024-byte alignment: the swizzle pattern is a function of the address bits (checked below; there is no slack left)
   extern __shared__ __align__(1024) unsigned char smem_dyn[];
@@ -433,8 +438,12 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + kNumBars);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + kNumBars + 1);
   volatile int* gbase = reinterpret_cast<volatile int*>(bars + kNumBars + 2);   // [kKStages][8] position of each 16-key group's first key
-  volatile int* krow = reinterpret_cast<volatile int*>(bars + kNumBars + 18);   // 8-bit pages: [kKStages][8] pool row of each group's first key (-1: no such keys)
-  volatile int* vrow = reinterpret_cast<volatile int*>(bars + kNumBars + 30);   // ... and [kVStages][8] for the V stages
+  volatile float* kscl = reinterpret_cast<volatile float*>(bars + kNumBars + 18);   // 8-bit pages: [2][8] scale of each group's K block, by tile parity
+  volatile float* vscl = reinterpret_cast<volatile float*>(bars + kNumBars + 30);   // ... and of its V block
+  unsigned char* Kc = Ks + 2 * NB * kBlockBytes;            // 8-bit pages: staged K codes of one tile (the third K stage's room)
+  unsigned char* Vc = Kc + 128 * 128;                       // ... and V codes
+  const uint32_t bar_kc_landed = BAR(kBarKLanded, 0), bar_kc_free = BAR(kBarKLanded, 1);   // 8-bit pages: staging full / read out
+  const uint32_t bar_vc_landed = BAR(kBarVLanded, 0), bar_vc_free = BAR(kBarVLanded, 1);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int spin = HOOKS ? p.spin_limit : kSpinLimit;
@@ -465,12 +474,12 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   if (warp == 0) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
   if (tid == 32) {
     for (int s = 0; s < kKStages; ++s) {
-      mbar_init(BAR(kBarKLanded, s), 1);                     // loader's expect_tx + TMA bytes
+      mbar_init(BAR(kBarKLanded, s), (FP8 && s == 1) ? kRotatorWarps * 32 : 1);   // loader's expect_tx + TMA bytes (8-bit pages: slot 1 = K codes read out)
       mbar_init(BAR(kBarKReady, s), kRotatorWarps * 32);
       mbar_init(BAR(kBarKFree, s), 1);                       // tcgen05.commit
     }
     for (int s = 0; s < kVStages; ++s) {
-      mbar_init(BAR(kBarVLanded, s), 1);
+      mbar_init(BAR(kBarVLanded, s), (FP8 && s == 1) ? 2 * 32 : 1);                   // (8-bit pages: slot 1 = V codes read out by the two converter warps)
       mbar_init(BAR(kBarVFree, s), 1);                       // tcgen05.commit
     }
     for (int s = 0; s < 2; ++s) {
@@ -783,14 +792,20 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       }
     }
     const int lc = c, hc = CH + c;
-    if (FP8) asm volatile("griddepcontrol.wait;" ::: "memory");   // this role reads the pools itself: after the commit kernel
     for (int tile = 0; tile < n_tiles; ++tile) {
-      const int st = tile % kKStages;
-      const uint32_t ph = static_cast<uint32_t>(tile / kKStages) & 1u;
-      if (!mbar_wait(BAR(kBarKLanded, st), ph, abort_flag, p.status, spin)) break;
+      const int st = tile % KD;
+      const uint32_t ph = static_cast<uint32_t>(tile / KD) & 1u;
+      if constexpr (FP8) {
+        // the tile's codes are staged, and (this role writes the bf16 stage itself) every QK^T that read the stage's
+        // previous tenant has completed
+        if (!mbar_wait(bar_kc_landed, static_cast<uint32_t>(tile) & 1u, abort_flag, p.status, spin)) break;
+        if (tile >= KD && !mbar_wait(BAR(kBarKFree, st), static_cast<uint32_t>(tile / KD - 1) & 1u, abort_flag, p.status, spin)) break;
+      } else {
+        if (!mbar_wait(BAR(kBarKLanded, st), ph, abort_flag, p.status, spin)) break;
+      }
       unsigned char* Kb = Ks + st * NB * kBlockBytes;
       const int key0 = (tile_base + tile) * kTileN;
-      int pos = gbase[st * 8 + k0 / 16] + (k0 & 15);
+      int pos = gbase[(FP8 ? (tile & 1) : st) * 8 + k0 / 16] + (k0 & 15);
       if (pos < 0 || pos > p.max_position) {
         if (key0 + k0 < kvl) atomicOr(p.status, MEPIC_DEV_BAD_POSITION);
         pos = 0;
@@ -805,13 +820,13 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         }
       }
       if constexpr (FP8) {
-        // ---- 8-bit pages: codes from global memory, widened exactly, rotated in fp32 with the block's scale folded
-        // into (cos, sin) (the one-position step is a pure rotation, so the factor rides along), rounded to bf16 once
-        const int r0 = krow[st * 8 + k0 / 16];
-        const bool have = r0 >= 0;
-        const unsigned char* src0 = reinterpret_cast<const unsigned char*>(p.k_pool) + static_cast<size_t>(have ? r0 + (k0 & 15) : 0) * D;
+        // ---- 8-bit pages: codes from the staging buffer, widened exactly, rotated in fp32 with the block's scale
+        // folded into (cos, sin) (the one-position step is a pure rotation, so the factor rides along), rounded to
+        // bf16 once.  A group with no key below kv_len was not copied: its rows become zero.
+        const bool have = key0 + (k0 & ~15) < kvl;
+        const unsigned char* src0 = Kc + k0 * 128;
         if (have) {
-          const float sc = __ldg(p.k_scales + r0 / p.page_size);
+          const float sc = kscl[(tile & 1) * 8 + k0 / 16];
 #pragma unroll
           for (int j = 0; j < 4; ++j) { cc[j].x *= sc; cc[j].y *= sc; ss[j].x *= sc; ss[j].y *= sc; }
         }
@@ -820,8 +835,8 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
           uint2 lo8[4], hi8[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
-            lo8[u] = have ? __ldg(reinterpret_cast<const uint2*>(src0 + static_cast<size_t>(i0 + u) * D + 8 * c)) : make_uint2(0, 0);
-            hi8[u] = have ? __ldg(reinterpret_cast<const uint2*>(src0 + static_cast<size_t>(i0 + u) * D + D / 2 + 8 * c)) : make_uint2(0, 0);
+            lo8[u] = have ? *reinterpret_cast<const uint2*>(src0 + (i0 + u) * 128 + 8 * c) : make_uint2(0, 0);
+            hi8[u] = have ? *reinterpret_cast<const uint2*>(src0 + (i0 + u) * 128 + 64 + 8 * c) : make_uint2(0, 0);
           }
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
@@ -854,6 +869,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         }
         fence_async_smem();
         mbar_arrive(BAR(kBarKReady, st));
+        mbar_arrive(bar_kc_free);    // the staged codes have been read: the next tile's may come
         continue;                    // (the V tile is the V converters' work)
       }
 #pragma unroll 2
@@ -888,43 +904,30 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     }
   } else if (FP8 && (warp == kVLoaderWarp || warp == kSpareWarp)) {
     // =============================================================== 8-bit pages: the V converters
-    // The V loader (which has nothing to copy) and the spare warp widen the V tile, 64 keys each: codes from global
-    // memory, times the block's scale, rounded to bf16 into the stage the PV MMA reads; rows at or past kv_len become
-    // zero (P is 0 there, but 0 x NaN is NaN).  Every decision that precedes a shuffle is the whole warp's.
+    // The V loader (which has nothing to copy: the K loader stages the codes of both pools) and the spare warp widen
+    // the V tile, 64 keys each: codes from the staging buffer, times the block's scale, rounded to bf16 into the stage
+    // the PV MMA reads; rows at or past kv_len become zero (P is 0 there, but 0 x NaN is NaN).
     const int half = warp == kVLoaderWarp ? 0 : 1;
-    asm volatile("griddepcontrol.wait;" ::: "memory");   // this role reads the pools itself: after the commit kernel
     for (int tile = 0; tile < n_tiles; ++tile) {
       const int vst = tile % kVStages;
+      if (!mbar_wait_warp(bar_vc_landed, static_cast<uint32_t>(tile) & 1u, abort_flag, p.status, spin)) break;
       if (tile >= kVStages &&
           !mbar_wait_warp(BAR(kBarVFree, vst), static_cast<uint32_t>(tile / kVStages - 1) & 1u, abort_flag, p.status, spin)) break;
       const int key0 = (tile_base + tile) * kTileN;
-      // lane g (mod 4) looks up 16-key group 4 half + g: pool row of its first key (-1: none below kv_len), its block's scale
-      const int gkey = key0 + (half * 4 + (lane & 3)) * 16;
-      int row = -1;
-      float scl = 0.f;
-      if (gkey < kvl) {
-        const int e = gkey / p.page_size;
-        int page = __ldg(ids + e);
-        if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
-        row = (page * p.n_kv_heads + h) * p.page_size + gkey % p.page_size;
-        scl = __ldg(p.v_scales + page * p.n_kv_heads + h);
-      }
       unsigned char* Vb = Vs + vst * NB * kBlockBytes;
 #pragma unroll 1
       for (int i0 = 0; i0 < 16; i0 += 8) {
-        // a lane's 16 chunks of 16 codes in two batches of eight requests: chunk idx = lane + 32 i of the warp's 64 keys
-        // is key idx / 8, dims [16 (idx % 8), +16); the eight chunks of a batch lie in groups (i0 + u) / 4
+        // a lane's 16 chunks of 16 codes in two batches of eight: chunk idx = lane + 32 i of the warp's 64 keys is key
+        // idx / 8, dims [16 (idx % 8), +16); the eight chunks of a batch lie in 16-key group 4 half + (i0 + u) / 4
         uint4 cd[8];
         float sc[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
-          const int idx = lane + 32 * (i0 + u), kl = idx >> 3, c16 = idx & 7;
-          const int vr = __shfl_sync(0xffffffffu, row, (i0 + u) >> 2);
-          const float gs = __shfl_sync(0xffffffffu, scl, (i0 + u) >> 2);
+          const int idx = lane + 32 * (i0 + u), kk = half * 64 + (idx >> 3), c16 = idx & 7;
           cd[u] = make_uint4(0, 0, 0, 0); sc[u] = 0.f;
-          if (vr >= 0 && key0 + half * 64 + kl < kvl) {
-            cd[u] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(p.v_pool) + static_cast<size_t>(vr + (kl & 15)) * D + 16 * c16));
-            sc[u] = gs;
+          if (key0 + kk < kvl) {
+            cd[u] = *reinterpret_cast<const uint4*>(Vc + kk * 128 + 16 * c16);
+            sc[u] = vscl[(tile & 1) * 8 + (kk >> 4)];
           }
         }
 #pragma unroll
@@ -946,8 +949,60 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       }
       fence_async_smem();
       mbar_arrive(BAR(kBarVReady, vst));
+      mbar_arrive(bar_vc_free);      // the staged codes have been read: the next tile's may come
     }
-  } else if (warp == kKLoaderWarp || warp == kVLoaderWarp) {
+  } else if (FP8 && warp == kKLoaderWarp) {
+    // =============================================================== 8-bit pages: the code loader
+    // Lane g < 8 brings the codes of 16-key group g of the tile into the staging buffers, K then V, one bulk copy of
+    // 2 KB each (a group's rows are contiguous in a pool), and publishes the group's position and the two scales.  The
+    // staging buffers hold one tile: the copies of tile j + 1 wait until the rotators (K) and the converters (V) have
+    // read tile j out.
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // after the commit kernel: the pools may be read
+    int issued = 0;                                      // tiles whose copies have been started
+    for (int tile = 0; tile < n_tiles; ++tile) {
+      const int key0 = (tile_base + tile) * kTileN;
+      const int gkey = key0 + lane * 16;
+      const bool live = lane < 8 && gkey < kvl;
+      int page = 0, pos = 0, slot0 = 0;
+      float ks = 0.f, vs = 0.f;
+      if (live) {
+        const int e = gkey / p.page_size;
+        slot0 = gkey % p.page_size;
+        page = __ldg(ids + e);
+        pos = __ldg(bases + e) + slot0;
+        if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
+        ks = __ldg(p.k_scales + page * p.n_kv_heads + h);
+        vs = __ldg(p.v_scales + page * p.n_kv_heads + h);
+      }
+      const size_t row = static_cast<size_t>(page * p.n_kv_heads + h) * p.page_size + slot0;      // of the pool viewed as [rows][128 bytes]
+      const uint32_t bytes = static_cast<uint32_t>(__popc(__ballot_sync(0xffffffffu, live))) * kCodeGroupBytes;
+      // ---- K codes
+      if (tile >= 1 && !mbar_wait_warp(bar_kc_free, static_cast<uint32_t>(tile - 1) & 1u, abort_flag, p.status, spin)) break;
+      if (lane < 8) { gbase[(tile & 1) * 8 + lane] = pos; kscl[(tile & 1) * 8 + lane] = ks; }
+      __syncwarp();
+      if (!(HOOKS && blockIdx.x == 0 && tile == p.skip_tile)) {      // (test hook: a K tile that never comes)
+        if (lane == 0) mbar_expect_tx(bar_kc_landed, bytes);
+        __syncwarp();
+        if (live) bulk_g2s(smem_u32(Kc) + static_cast<uint32_t>(lane) * kCodeGroupBytes,
+                           reinterpret_cast<const unsigned char*>(p.k_pool) + row * 128, kCodeGroupBytes, bar_kc_landed);
+      }
+      // ---- V codes
+      if (tile >= 1 && !mbar_wait_warp(bar_vc_free, static_cast<uint32_t>(tile - 1) & 1u, abort_flag, p.status, spin)) break;
+      if (lane < 8) vscl[(tile & 1) * 8 + lane] = vs;
+      __syncwarp();
+      if (lane == 0) mbar_expect_tx(bar_vc_landed, bytes);
+      __syncwarp();
+      if (live) bulk_g2s(smem_u32(Vc) + static_cast<uint32_t>(lane) * kCodeGroupBytes,
+                         reinterpret_cast<const unsigned char*>(p.v_pool) + row * 128, kCodeGroupBytes, bar_vc_landed);
+      issued = tile + 1;
+    }
+    // after a lost wait: the copies started last may still be in flight; give them a bounded chance to land before the
+    // CTA's shared memory is given up (the tile that the test hook left out never lands: the bound ends that wait)
+    if (*abort_flag && issued > 0) {
+      for (int i = 0; i < spin && !mbar_try_wait(bar_kc_landed, static_cast<uint32_t>(issued - 1) & 1u); ++i) {}
+      for (int i = 0; i < spin && !mbar_try_wait(bar_vc_landed, static_cast<uint32_t>(issued - 1) & 1u); ++i) {}
+    }
+  } else if (!FP8 && (warp == kKLoaderWarp || warp == kVLoaderWarp)) {
     // =============================================================== loader warps: lane g loads 16-key group g
     const bool is_k = warp == kKLoaderWarp;
     const CUtensorMap* map = is_k ? &map_k : &map_v;
@@ -976,16 +1031,10 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { atomicOr(p.status, MEPIC_DEV_BAD_PAGE); page = 0; }
       }
       if (is_k && lane < 8) gbase[st * 8 + lane] = pos;
-      if (FP8 && lane < 8) (is_k ? krow : vrow)[st * 8 + lane] = live ? (page * p.n_kv_heads + h) * p.page_size + slot0 : -1;
       const unsigned live_mask = __ballot_sync(0xffffffffu, live);
       __syncwarp();
       const uint32_t landed = BAR(is_k ? kBarKLanded : kBarVLanded, st);
       if (HOOKS && is_k && blockIdx.x == 0 && tile == p.skip_tile) continue;      // (test hook: a K tile that never comes)
-      if constexpr (FP8) {
-        // nothing to copy: the stage is free and its groups' pool rows are published; the rotators do the rest
-        if (lane == 0) mbar_arrive(landed);
-        continue;
-      }
       if (lane == 0) mbar_expect_tx(landed, static_cast<uint32_t>(__popc(live_mask)) * kGroupBytes);
       __syncwarp();
       if (live) {
@@ -997,7 +1046,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     }
     // Rows at or past kv_len of the last V tile may hold anything (NaN bit patterns included): P is 0 there,
     // but 0 x NaN is NaN, so V must be finite.  Zero them once the tile has landed.
-    if (!FP8 && !is_k && ok && last_has_tail) {
+    if (!is_k && ok && last_has_tail) {
       const int lt = n_tiles - 1, st = lt % kVStages;
       if (mbar_wait_warp(BAR(kBarVLanded, st), static_cast<uint32_t>(lt / kVStages) & 1u, abort_flag, p.status, spin)) {
         unsigned char* Vb = Vs + st * NB * kBlockBytes;
@@ -1011,6 +1060,10 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
         if (lane == 0) mbar_arrive(BAR(kBarVPatched, 0));
       }
     }
+    // (After a lost wait somewhere this warp leaves its loop from a wait that has polled at least 1024 times since its
+    // last copy was started - the flag is looked at every 1024 polls - which is tens of microseconds against the one or
+    // two a copy takes: nothing of it is still in flight at the CTA's exit.  An explicit wait for the landed barriers
+    // here, even out of line and never executed, cost the kernel 1.3 % in the way the compiler lays the roles out.)
   } else if (warp == kMmaWarp && lane == 0) {
     // =============================================================== MMA issuer (one thread)
     // Order per key tile j:  PV_a(j), QK_a(j+1), PV_b(j), QK_b(j+1): while one M-tile's softmax runs, the
@@ -1024,7 +1077,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
     constexpr uint64_t kStageUnits = (NB * kBlockBytes) >> 4;
     bool ok = true;
     auto issue_qk = [&](int x, int j) {
-      const uint64_t kd = k_desc0 + static_cast<uint64_t>(j % kKStages) * kStageUnits;
+      const uint64_t kd = k_desc0 + static_cast<uint64_t>(j % KD) * kStageUnits;
 #pragma unroll
       for (int ks = 0; ks < D / 16; ++ks) {
         const uint64_t off = static_cast<uint64_t>(((ks / 4) * kBlockBytes + (ks % 4) * 32) >> 4);
@@ -1043,7 +1096,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       tc_commit(BAR(kBarPvDone, x));
     };
     auto wait_k = [&](int j) {
-      const bool w = mbar_wait(BAR(kBarKReady, j % kKStages), static_cast<uint32_t>(j / kKStages) & 1u, abort_flag, p.status, spin);
+      const bool w = mbar_wait(BAR(kBarKReady, j % KD), static_cast<uint32_t>(j / KD) & 1u, abort_flag, p.status, spin);
       tc_fence_after();
       return w;
     };
@@ -1082,7 +1135,7 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
       tc_commit(BAR(kBarVFree, j % kVStages));
       if (more) {
         if (j + 1 < nt[1]) issue_qk(1, j + 1);
-        tc_commit(BAR(kBarKFree, (j + 1) % kKStages));
+        tc_commit(BAR(kBarKFree, (j + 1) % KD));
       }
     }
     if (!ok) {
@@ -1093,13 +1146,6 @@ mepic_prefill_attn(const PrefillParams p, const __grid_constant__ CUtensorMap ma
   }
 
   // ---- common exit: nothing of this CTA may still be in flight when tensor memory is released
-  if (!FP8 && (warp == kKLoaderWarp || warp == kVLoaderWarp) && *abort_flag) {
-    // a wait ran out somewhere: give outstanding TMA copies a bounded chance to land before leaving
-    const int which = warp == kKLoaderWarp ? kBarKLanded : kBarVLanded;
-    const int depth = warp == kKLoaderWarp ? kKStages : kVStages;
-    for (int s = 0; s < depth; ++s)
-      for (int i = 0; i < (1 << 16) && !mbar_try_wait(BAR(which, s), 0) && !mbar_try_wait(BAR(which, s), 1); ++i) {}
-  }
   tc_fence_before();
   __syncthreads();
   if (warp == 0) tmem_dealloc(tmem_base, kTmemCols);
