@@ -244,6 +244,16 @@ int32_t mepic_store_test_hooks(mepic_store_t* store, uint64_t hash_mask, int32_t
  */
 int32_t mepic_kernel_test_hooks(int32_t spin_limit, int32_t skip_tile);
 
+/*
+ * mepic_prefill_test_two_pass - lets a test compare the two softmax schedules of mepic_attn_prefill (the paper has no
+ * counterpart).  on != 0: calls made from now on enqueue the attention kernel once, with the reference found from each
+ * tile's own scores (the repeat launch's schedule) for every item; the first word of the workspace stays clear;
+ * 0 restores the fast launch followed by the conditional repeat launch.  Both schedules compute the same softmax;
+ * their outputs differ by the rounding of P to bf16 under different references only.  Process-wide; not for
+ * production use.  Always returns MEPIC_OK.
+ */
+int32_t mepic_prefill_test_two_pass(int32_t on);
+
 /* ---------------------------------------------------------------- rope table (host, set-up)
  *
  * Section 3.3.3 has the kernel apply each block's rotary offset but gives no formula; the table

@@ -22,7 +22,7 @@ from .build import LIB_PATH, build_library
 __all__ = [
     "MepicError", "Config", "Segment", "Store", "lib",
     "mepic_store_create", "mepic_store_destroy", "mepic_chunk_register", "mepic_build_block_table",
-    "mepic_request_release", "mepic_chunk_mark_uncomputed", "mepic_store_stats", "mepic_store_attach_remote", "mepic_store_test_hooks", "mepic_kernel_test_hooks", "mepic_rope_table_floats", "mepic_rope_table_fill",
+    "mepic_request_release", "mepic_chunk_mark_uncomputed", "mepic_store_stats", "mepic_store_attach_remote", "mepic_store_test_hooks", "mepic_kernel_test_hooks", "mepic_prefill_test_two_pass", "mepic_rope_table_floats", "mepic_rope_table_fill",
     "mepic_attn_decode_workspace", "mepic_attn_decode", "mepic_attn_decode_static",
     "mepic_pages_quantize", "mepic_attn_decode_fp8", "mepic_decode_plan_max_ints", "mepic_decode_plan_build", "mepic_decode_plan_patch", "mepic_attn_decode_grouped_workspace",
     "mepic_attn_decode_grouped", "mepic_attn_decode_grouped_fp8",
@@ -138,6 +138,7 @@ _PROTOTYPES = {
     "mepic_store_attach_remote": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int64, C.c_void_p]),
     "mepic_store_test_hooks": (C.c_int32, [C.c_void_p, C.c_uint64, C.c_int32]),
     "mepic_kernel_test_hooks": (C.c_int32, [C.c_int32, C.c_int32]),
+    "mepic_prefill_test_two_pass": (C.c_int32, [C.c_int32]),
     "mepic_rope_table_floats": (C.c_size_t, [C.POINTER(_ConfigC)]),
     "mepic_rope_table_fill": (C.c_int32, [C.POINTER(_ConfigC), C.c_void_p]),
     "mepic_attn_decode_workspace": (C.c_size_t, [C.POINTER(_ConfigC), C.c_int32]),
@@ -289,6 +290,10 @@ def mepic_store_test_hooks(store: int, hash_mask: int = 0xFFFFFFFFFFFFFFFF, fail
 
 def mepic_kernel_test_hooks(spin_limit: int = 0, skip_tile: int = -1) -> None:
     _check(lib().mepic_kernel_test_hooks(spin_limit, skip_tile))
+
+
+def mepic_prefill_test_two_pass(on: bool) -> None:
+    _check(lib().mepic_prefill_test_two_pass(1 if on else 0))
 
 
 class Store:

@@ -15,5 +15,6 @@ int32_t mepic_make_pool_map_u8(const mepic_config_t* cfg, const void* pool, void
 // wait (the built-in limit when no test changed it) and the index of the one staged copy that is left out (-1: none).
 int mepic_test_spin_limit(int built_in);
 int mepic_test_skip_tile();
+int mepic_test_prefill_two_pass();       // mepic_prefill_test_two_pass: the prefill enqueues its two-pass schedule only
 
 #endif

@@ -85,7 +85,7 @@ struct PrefillParams {
   float* k_scales;      // 8-bit pools only: [num_pages][n_kv_heads] scale of each (page, kv head) block of K (the commit writes them)
   float* v_scales;      // ... and of V
   int32_t* redo_flag;   // first word of the workspace: set by a CTA of the fast launch one of whose rows outran its reference
-  int exact;            // 0: the fast launch; 1: the repeat launch (two passes on every tile; returns at once unless *redo_flag)
+  int exact;            // 0: the fast launch; 1: the repeat launch (two passes on every tile; returns at once unless *redo_flag); 2: two passes, unconditionally (test hook)
   int spin_limit;       // polls before a bounded wait gives up
   int skip_tile;        // test hook: CTA 0's K loader leaves out the copies of its key tile with this index (-1: none)
 };
@@ -1212,9 +1212,10 @@ int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& m
   lc.attrs = pdl; lc.numAttrs = 1;
   // the fast launch, then the repeat launch, which does nothing unless a row outran its reference in the first
   PrefillParams pf = p;
-  pf.exact = 0;
+  const bool two_pass_only = mepic_test_prefill_two_pass() != 0;       // (test hook: the repeat launch's schedule, unconditionally)
+  pf.exact = two_pass_only ? 2 : 0;
   e = cudaLaunchKernelEx(&lc, mepic_prefill_attn<D, G, FP8, HOOKS>, pf, map_k, map_v);
-  if (e == cudaSuccess) {
+  if (e == cudaSuccess && !two_pass_only) {
     pf.exact = 1;
     e = cudaLaunchKernelEx(&lc, mepic_prefill_attn<D, G, FP8, HOOKS>, pf, map_k, map_v);
   }
@@ -1225,7 +1226,7 @@ int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& m
   }
   if (e == cudaSuccess) e = cudaGetLastError();
   if (e != cudaSuccess) { mepic_set_error("prefill: launch: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
-  mepic_count_launches(p.n_splits > 1 ? 4 : 3);
+  mepic_count_launches((p.n_splits > 1 ? 4 : 3) - (two_pass_only ? 1 : 0));
   return MEPIC_OK;
 }
 

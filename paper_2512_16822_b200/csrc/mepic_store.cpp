@@ -549,6 +549,13 @@ extern "C" int32_t mepic_kernel_test_hooks(int32_t spin_limit, int32_t skip_tile
   return MEPIC_OK;
 }
 
+static std::atomic<int> g_prefill_two_pass{0};
+int mepic_test_prefill_two_pass() { return g_prefill_two_pass.load(std::memory_order_relaxed); }
+extern "C" int32_t mepic_prefill_test_two_pass(int32_t on) {
+  g_prefill_two_pass.store(on != 0, std::memory_order_relaxed);
+  return MEPIC_OK;
+}
+
 // ---------------------------------------------------------------- launch counter
 static std::atomic<int64_t> g_launches{0};
 void mepic_count_launches(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
