@@ -23,9 +23,12 @@
 //                   two M-tiles: PV_a(j), QK_a(j+1), PV_b(j), QK_b(j+1).
 //   softmax warps : two warpgroups per M-tile; row r is shared by two threads, one per half of
 //                   the tile's 128 score columns: tcgen05.ld the scores, causal mask by logical
-//                   slot, online softmax in the log2 domain with a lazily moved reference
-//                   maximum that the two threads agree on once per tile (values through shared
-//                   memory, the meeting on a hardware barrier of their two warps),
+//                   slot, online softmax in the log2 domain against a reference that both threads
+//                   of the row share.  The first tile finds it from its own scores (the two
+//                   threads meet on a hardware barrier of their two warps, values through shared
+//                   memory); later tiles of the fast launch keep the reference they have and raise
+//                   it one tile late, from the sums of P, without a meeting; a row that outruns it
+//                   asks for the repeat launch, which finds it from every tile's own scores,
 //                   P -> bf16 -> tensor memory (over the first columns of each half of the S
 //                   buffer, from where the PV MMA takes it as its A operand); each rescales its
 //                   half of the O columns in tensor memory when the reference moved; the
