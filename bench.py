@@ -420,6 +420,34 @@ def decode_error(wl, lay, out_bits, sample) -> dict:
     return e
 
 
+def fp8_decode_error(wl, lay, pools, tabs, out, grouped_out, b: int = 0) -> dict:
+    """8-bit pages: the oracle quantises the pages request ``b`` reads from the bf16 pool (the library's codes and scales
+    for them must agree bit for bit) and evaluates the request on those codes and scales; error figures of the
+    per-request and of the sharing-aware 8-bit decode against it."""
+    import torch
+    from mepic_inputs import bf16_bits_to_f64
+    from oracle import mepic_oracle as O
+    from paper_2512_16822_b200 import runtime as RT
+    page_ids, pos_base, kv_len, q_pos = tabs
+    n = -(-int(kv_len[b]) // wl.page_size)
+    mine = np.unique(page_ids[b, :n])
+    okc, oks = O.quantize_pages(lay["kp"][mine]); ovc, ovs = O.quantize_pages(lay["vp"][mine])
+    sel = torch.from_numpy(mine.astype(np.int64)).to(pools.k_codes.device)
+    same = bool(np.array_equal(pools.k_codes[sel].cpu().numpy(), okc) and np.array_equal(pools.k_scales[sel].cpu().numpy(), oks) and
+                np.array_equal(pools.v_codes[sel].cpu().numpy(), ovc) and np.array_equal(pools.v_scales[sel].cpu().numpy(), ovs))
+    local = {int(pg): i for i, pg in enumerate(mine)}
+    ids = [local[int(pg)] for pg in page_ids[b, :n]]
+    want = O.decode_attention_one(wl.decode_q()[b], O.dequantize_pages(okc, oks), O.dequantize_pages(ovc, ovs), ids, list(pos_base[b, :n]),
+                                  int(kv_len[b]), int(q_pos[b]), wl.sm_scale, wl.rope_theta)
+    e = error_figures(bf16_bits_to_f64(RT.bf16_bits(out))[b], want)
+    g = error_figures(bf16_bits_to_f64(RT.bf16_bits(grouped_out))[b], want)
+    e.update({"sample": f"request {b} against the fp64 oracle evaluated on the oracle's own codes and scales of the {len(mine)} pages it reads",
+              "codes_and_scales_bit_exact": same,
+              "within_tolerance": bool(same and e["max_abs"] <= MAX_ABS and e["mean_abs"] <= MEAN_ABS),
+              "grouped": {**g, "within_tolerance": bool(g["max_abs"] <= MAX_ABS and g["mean_abs"] <= MEAN_ABS)}})
+    return e
+
+
 def decode_legs(index: int, args, device: str, peak: float, *, scale=1.0, kinds=("plain", "unshared", "e2e", "error")):
     """Decode of one configuration through mepic_attn_decode: shared layout (flushed / not), unshared layout, end to
     end, error figures.  Returns the per-config object."""
@@ -523,6 +551,36 @@ def prefill_error(wl, lay, pb, q_slots, rows, tabs, n_rows=12) -> dict:
     return e
 
 
+def prefill_error_fp8(wl, lay, pools, pb, q_slots, rows, tabs, n_rows=12) -> dict:
+    """8-bit pages: the oracle quantises the pages request 0 reads from the bf16 pool, commits request 0's rows into
+    them by its own rule (codes and scales of those pages must then equal the library's bit for bit) and evaluates
+    sampled rows on those codes and scales."""
+    import torch
+    from mepic_inputs import bf16_bits_to_f64
+    from oracle import mepic_oracle as O
+    from paper_2512_16822_b200 import runtime as RT
+    page_ids, pos_base, kv_len, row_offsets = tabs
+    ne = -(-int(kv_len[0]) // wl.page_size)
+    mine = np.unique(page_ids[0][:ne])
+    okc, oks = O.quantize_pages(lay["kp"][mine]); ovc, ovs = O.quantize_pages(lay["vp"][mine])
+    local = {int(pg): i for i, pg in enumerate(mine)}
+    ids0 = [local[int(pg)] for pg in page_ids[0][:ne]]
+    O.commit_rows_fp8(okc, oks, ovc, ovs, ids0, list(q_slots[0]), rows[0].k_new, rows[0].v_new)
+    sel = torch.from_numpy(mine.astype(np.int64)).to(pools.k_codes.device)
+    same = bool(np.array_equal(pools.k_codes[sel].cpu().numpy(), okc) and np.array_equal(pools.k_scales[sel].cpu().numpy(), oks) and
+                np.array_equal(pools.v_codes[sel].cpu().numpy(), ovc) and np.array_equal(pools.v_scales[sel].cpu().numpy(), ovs))
+    R = len(q_slots[0])
+    pick = sorted(set(np.linspace(0, R - 1, n_rows).astype(int).tolist()))
+    want = O.prefill_attention_one(rows[0].q_new, rows[0].k_new, rows[0].v_new, list(q_slots[0]), O.dequantize_pages(okc, oks),
+                                   O.dequantize_pages(ovc, ovs), ids0, list(pos_base[0][:ne]), int(kv_len[0]), wl.sm_scale, wl.rope_theta, rows=pick)
+    e = error_figures(bf16_bits_to_f64(RT.bf16_bits(pb.out[:R]))[pick], want)
+    e.update({"sample": f"{len(pick)} of the {R} rows of request 0 (first to last), all heads and dims, against the fp64 oracle "
+                        f"evaluated on the oracle's own codes and scales of the {len(mine)} pages the request reads",
+              "committed_codes_and_scales_bit_exact": same,
+              "within_tolerance": bool(same and e["max_abs"] <= MAX_ABS and e["mean_abs"] <= MEAN_ABS)})
+    return e
+
+
 def prefill_leg(index: int, args, device: str, *, scale=1.0, error=True, lay=None, fp8=False):
     """One step = one mepic_attn_prefill call (commit + attention) over the configuration's prefill requests.
     fp8: the same requests over 8-bit (e4m3) pools made from the workload's pool by the library's quantiser, the
@@ -543,7 +601,7 @@ def prefill_leg(index: int, args, device: str, *, scale=1.0, error=True, lay=Non
                                  np.concatenate([r.v_new for r in rows]))
         del pb
         pb = pb8
-        error = False
+        error8, error = error, False
     stream = torch.cuda.current_stream()
     for _ in range(3):
         pb.run(wl.sm_scale, stream)
@@ -573,16 +631,18 @@ def prefill_leg(index: int, args, device: str, *, scale=1.0, error=True, lay=Non
                   "pages_per_GB": int(1e9 // (wl.page_size * bpt + 2 * wl.n_kv_heads * 4)),
                   "pages_per_GB_bf16": int(1e9 // (wl.page_size * kv_bytes_per_token(wl))),
                   "note": "e4m3 pages + one fp32 scale per (page, kv head); no bf16 copy of the pool on the device; "
-                          "parity of this path is the GPU test suite's (tests/test_fp8_end_to_end_gpu.py)"})
+                          "more shapes, appends and a NaN element in tests/test_fp8_end_to_end_gpu.py"})
         d["roofline"]["kernel"] = "mepic_prefill_attn, 8-bit pages (+ commit kernel: the C-ABI call is timed as a whole)"
         d["roofline"]["traffic"] = None; d["roofline"]["traffic_source"] = None
+        if error8:
+            d["error"] = prefill_error_fp8(wl, lay, pools, pb, q_slots, rows, tabs)
     if error:
         d["error"] = prefill_error(wl, lay, pb, q_slots, rows, tabs)
     return d, lay, pb
 
 
 # ---------------------------------------------------------------- the other decode paths on the headline batch
-def measure_variant(kind: str, args, wl, dev, tabs, q_bits, logical_bytes: int, peak: float):
+def measure_variant(kind: str, args, wl, dev, tabs, q_bits, logical_bytes: int, peak: float, lay=None):
     """The headline batch through mepic_attn_decode_grouped ("grouped") or mepic_attn_decode_fp8 ("fp8")."""
     import torch
     import paper_2512_16822_b200 as M
@@ -632,6 +692,8 @@ def measure_variant(kind: str, args, wl, dev, tabs, q_bits, logical_bytes: int, 
                     "staged_gbs": staged / (gms["ms_per_step"] * 1e-3) / 1e9,
                     "note": "mepic_attn_decode_grouped_fp8: value = 8-bit bytes of the per-request decode / time"})
         d["grouped"] = gms
+        if lay is not None:
+            d["error"] = fp8_decode_error(wl, lay, batch.pools, tabs, batch.out, gb.out)
         del gb
     del batch
     return d
@@ -968,7 +1030,7 @@ def run_ours(args):
         error = decode_error(wl, lay, RT.bf16_bits(batch.out), sorted({0, B // 2, B - 1}))
         if wl.head_dim == 128:
             with sampler.window("fp8"):
-                fp8 = measure_variant("fp8", args, wl, dev, tabs, q_bits, logical_bytes, peak)
+                fp8 = measure_variant("fp8", args, wl, dev, tabs, q_bits, logical_bytes, peak, lay=lay)
         with sampler.window("grouped"):
             grouped = measure_variant("grouped", args, wl, dev, tabs, q_bits, logical_bytes, peak)
     del batch
