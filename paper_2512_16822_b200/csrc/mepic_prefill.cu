@@ -217,25 +217,24 @@ __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // ---------------------------------------------------------------- commit (Section 3.3.2)
-// One CTA per new row: its K and V bits go, un-rotated, to (page, slot) of the pools.
-__global__ void mepic_prefill_commit(const PrefillParams p, int chunks_per_row) {
+// One warp per new row (eight rows to a CTA): its K and V bits go, un-rotated, to (page, slot) of the pools.
+constexpr int kCommitRows = 8;          // rows per CTA of the commit kernel, one warp each
+__global__ void __launch_bounds__(kCommitRows * 32) mepic_prefill_commit(const PrefillParams p, int chunks_per_row) {
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the attention kernel may stage its queries meanwhile
-  const int row = blockIdx.x;
-  if (row == 0 && threadIdx.x == 0) *p.redo_flag = 0;              // (an attention CTA that could set it waits for this grid first)
-  __shared__ int sh_b;
-  if (threadIdx.x == 0) {
-    int b = 0;
-    while (b + 1 < p.batch && row >= p.row_offsets[b + 1]) ++b;
-    sh_b = b;
-  }
-  __syncthreads();
-  const int b = sh_b;
+  if (blockIdx.x == 0 && threadIdx.x == 0) *p.redo_flag = 0;       // (an attention CTA that could set it waits for this grid first)
+  // a warp per row: the row's look-ups (request, slot, page) are a chain of dependent loads, and a CTA's eight chains
+  // run side by side
+  const int lane = threadIdx.x & 31;
+  const int row = blockIdx.x * kCommitRows + (threadIdx.x >> 5);
+  if (row >= p.total_rows) return;
+  int b = 0;
+  while (b + 1 < p.batch && row >= p.row_offsets[b + 1]) ++b;
   const int slot = p.q_slot[row];
-  if (slot < 0 || slot >= p.kv_len[b]) { if (threadIdx.x == 0) atomicOr(p.status, MEPIC_DEV_BAD_SLOT); return; }
+  if (slot < 0 || slot >= p.kv_len[b]) { if (lane == 0) atomicOr(p.status, MEPIC_DEV_BAD_SLOT); return; }
   const int page = p.page_ids[static_cast<size_t>(b) * p.table_stride + slot / p.page_size];
-  if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { if (threadIdx.x == 0) atomicOr(p.status, MEPIC_DEV_BAD_PAGE); return; }
+  if (static_cast<unsigned>(page) >= static_cast<unsigned>(p.num_pages)) { if (lane == 0) atomicOr(p.status, MEPIC_DEV_BAD_PAGE); return; }
   const int D8 = chunks_per_row / p.n_kv_heads;        // 16-byte chunks per head row
-  for (int c = threadIdx.x; c < chunks_per_row; c += blockDim.x) {
+  for (int c = lane; c < chunks_per_row; c += 32) {
     const int h = c / D8, cc = c % D8;
     const size_t dst = (((static_cast<size_t>(page) * p.n_kv_heads + h) * p.page_size + slot % p.page_size) * D8 + cc);
     const size_t src = static_cast<size_t>(row) * chunks_per_row + c;
@@ -1208,7 +1207,7 @@ int32_t launch_prefill(const PrefillParams& p, int n_items, const CUtensorMap& m
   if (e != cudaSuccess) { mepic_set_error("prefill: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MEPIC_E_CUDA; }
   const int chunks_per_row = p.n_kv_heads * D / 8;
   if (FP8) mepic_prefill_commit_fp8<<<p.total_rows, 256, 0, stream>>>(p, D);
-  else mepic_prefill_commit<<<p.total_rows, 128, 0, stream>>>(p, chunks_per_row);
+  else mepic_prefill_commit<<<(p.total_rows + kCommitRows - 1) / kCommitRows, kCommitRows * 32, 0, stream>>>(p, chunks_per_row);
   // each kernel may become resident while its predecessor drains (programmatic dependent launch); it waits with
   // griddepcontrol.wait before it touches what the predecessor writes
   cudaLaunchAttribute pdl[1];
