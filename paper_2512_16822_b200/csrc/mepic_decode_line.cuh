@@ -144,14 +144,34 @@ __global__ void mepic_decode_merge(const DecodeParams p) {
   const long long u0 = sh[1] * p.n_kv_heads + static_cast<long long>(h) * nt;
   const long long w_first = u0 / piece, w_last = (u0 + nt - 1) / piece;
   const long long unit = static_cast<long long>(b) * p.n_kv_heads + h;
+  // the partials of a line are read four pieces at a time (the loads of a batch are independent: one round trip to L2
+  // instead of four) and combined in piece order
   float m_star = -INFINITY;
-  for (long long wk = w_first; wk <= w_last; ++wk) m_star = fmaxf(m_star, p.part_ml[((unit + wk) * G + g) * 2]);
+  for (long long wk = w_first; wk <= w_last; wk += 4) {
+    float m4[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) m4[k] = wk + k <= w_last ? p.part_ml[((unit + wk + k) * G + g) * 2] : -INFINITY;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) m_star = fmaxf(m_star, m4[k]);
+  }
   float l_star = 0.f, o_star = 0.f;
-  for (long long wk = w_first; wk <= w_last; ++wk) {
-    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + ((unit + wk) * G + g) * 2);
-    const float wgt = ex2(ml.x - m_star);
-    l_star += ml.y * wgt;
-    o_star += p.part_o[((unit + wk) * G + g) * D + d] * wgt;
+  for (long long wk = w_first; wk <= w_last; wk += 4) {
+    float2 ml4[4];
+    float o4[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const bool in = wk + k <= w_last;
+      ml4[k] = in ? *reinterpret_cast<const float2*>(p.part_ml + ((unit + wk + k) * G + g) * 2) : make_float2(-INFINITY, 0.f);
+      o4[k] = in ? p.part_o[((unit + wk + k) * G + g) * D + d] : 0.f;
+    }
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (wk + k <= w_last) {
+        const float wgt = ex2(ml4[k].x - m_star);
+        l_star += ml4[k].y * wgt;
+        o_star += o4[k] * wgt;
+      }
+    }
   }
   const float r = o_star / l_star;
   // fp32 -> bf16, round to nearest even
